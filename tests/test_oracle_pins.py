@@ -1,0 +1,368 @@
+"""Pins for the CPU oracle: each test checks it against something the paper or
+the mathematics fixes, never against itself."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import faar_oracle as fo
+from paper_2603_22370_b200 import inputs
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_pairs(name):
+    out = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                out.append(line.split())
+    return out
+
+
+def small_layer(seed=0, O=8, K=64, T=48):
+    W, X = inputs.config1(seed, O, K, T)
+    return W, X
+
+
+# ---- I1: node table ("NVFP4 Overview") -----------------------------------
+
+def test_nodes_match_paper():
+    gold = np.array([float(r[0]) for r in _read_pairs("e2m1_nodes.txt")])
+    assert np.array_equal(fo.NODES, gold)
+
+
+def test_nodes_are_e2m1_bit_patterns():
+    # E2M1: 2 exponent bits (bias 1), 1 mantissa bit, subnormal at e = 0.
+    for c in range(8):
+        e, m = c >> 1, c & 1
+        val = m * 0.5 if e == 0 else (1 + m / 2) * 2.0 ** (e - 1)
+        assert fo.NODES[c] == val
+
+
+# ---- I2: E4M3 -------------------------------------------------------------
+
+def test_e4m3_decode_golden():
+    for hx, val in _read_pairs("e4m3_values.txt"):
+        got = fo.e4m3_decode(int(hx, 16))
+        assert got == float(val) and np.signbit(got) == (int(hx, 16) >= 0x80)
+    assert np.isnan(fo.e4m3_decode(0x7F)) and np.isnan(fo.e4m3_decode(0xFF))
+
+
+def test_e4m3_decode_matches_torch_float8():
+    b = torch.arange(256, dtype=torch.int32).to(torch.uint8)
+    ref = b.view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    got = fo.e4m3_decode(np.arange(256))
+    assert np.array_equal(np.isnan(ref), np.isnan(got))
+    ok = ~np.isnan(ref)
+    assert np.array_equal(ref[ok].astype(np.float64), got[ok])
+
+
+def test_e4m3_encode_roundtrip_monotone_midpoints():
+    vals = fo.e4m3_decode(np.arange(0x7F))
+    assert np.all(np.diff(vals) > 0)
+    assert np.array_equal(fo.e4m3_encode(vals), np.arange(0x7F, dtype=np.uint8))
+    mid = (vals[:-1] + vals[1:]) / 2
+    enc = fo.e4m3_encode(mid)
+    assert np.all(enc % 2 == 0)                              # ties to even mantissa
+    assert np.all((enc == np.arange(0x7E)) | (enc == np.arange(1, 0x7F)))
+    eps = np.minimum(1e-7, np.diff(vals) / 8)
+    assert np.array_equal(fo.e4m3_encode(mid - eps), np.arange(0x7E, dtype=np.uint8))
+    assert np.array_equal(fo.e4m3_encode(mid + eps), np.arange(1, 0x7F, dtype=np.uint8))
+    # saturating, never NaN
+    assert fo.e4m3_encode(np.array([448.0, 449.0, 464.0, 1e9, np.inf])).tolist() == [0x7E] * 5
+
+
+def test_e4m3_encode_matches_torch_cast_in_range():
+    rng = np.random.default_rng(1)
+    q = np.concatenate([rng.uniform(0, 448, 20000), rng.uniform(0, 0.05, 20000),
+                        np.exp(rng.uniform(np.log(1e-4), np.log(448), 20000))]).astype(np.float32)
+    ref = torch.from_numpy(q).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(fo.e4m3_encode(q), ref)
+
+
+def test_bf16_round_matches_torch_and_is_single_rounding():
+    rng = np.random.default_rng(2)
+    x = (rng.standard_normal(50000) * np.exp(rng.uniform(-20, 20, 50000))).astype(np.float32)
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    assert np.array_equal(fo.bf16_round(x.astype(np.float64)).astype(np.float32), ref)
+    # 1 + 2^-8 + 2^-30 lies above the midpoint of [1, 1+2^-7]: one rounding goes up,
+    # rounding through binary32 first would land on the tie and go down to even.
+    assert fo.bf16_round(1 + 2.0 ** -8 + 2.0 ** -30) == 1 + 2.0 ** -7
+    assert fo.bf16_round(1 + 2.0 ** -8) == 1.0 and fo.bf16_round(1 + 3 * 2.0 ** -8) == 1 + 2.0 ** -6
+    assert fo.bf16_round(0.0) == 0.0 and fo.bf16_round(-2.0 ** -133) == -2.0 ** -133
+
+
+# ---- I3 / I4: scales and bracket -----------------------------------------
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_scale_bound_and_bracket_invariants(seed):
+    W, _ = inputs.config1(seed, 64, 256, 8)
+    scales, sg = fo.compute_scales(W)
+    assert sg == np.float32(np.abs(W).max()) / np.float32(2688.0)
+    s = fo.effective_scale(scales, sg).astype(np.float64)
+    amax_g = np.abs(W).reshape(64, 16, 16).max(axis=2).astype(np.float64)
+    normal = scales >= 0x08
+    # E4M3 RNE has relative error <= 2^-4 on normal numbers
+    assert np.all(6 * s[normal] >= amax_g[normal] * (1 - 2.0 ** -4) * (1 - 1e-6))
+    assert np.all(6 * s[normal] <= amax_g[normal] * (1 + 2.0 ** -4) * (1 + 1e-6))
+    assert scales.max() <= 0x7E
+    # the tensor-wide maximum maps to the top of the E4M3 range
+    assert scales.max() == 0x7E
+    k, neg, v = fo.bracket(W, scales, sg)
+    sfull = np.repeat(s, 16, axis=1)
+    wt = np.abs(W.astype(np.float64)) / sfull
+    assert wt.max() <= 6 * (1 + 2.0 ** -4) * (1 + 1e-6)
+    wtc = np.minimum(wt, 6.0)
+    lo, hi = fo.NODES[k], fo.NODES[k + 1]
+    assert np.all(lo <= wtc * (1 + 1e-6)) and np.all(wtc <= hi * (1 + 1e-6))
+    assert set(np.unique(hi - lo)) <= {0.5, 1.0, 2.0}
+    assert v.dtype == np.float32 and v.min() >= 0 and v.max() <= 1
+    # Eq. 4 inverted: sign * (lo + v (hi - lo)) * s reproduces w unless clamped
+    rec = np.where(neg, -1.0, 1.0) * (lo + v.astype(np.float64) * (hi - lo)) * sfull
+    un = wt <= 6.0
+    assert np.allclose(rec[un], W[un], rtol=3e-7, atol=1e-12)
+    assert np.array_equal(neg, W < 0)
+
+
+def test_bracket_exact_nodes_ties_clamp_zero_block_and_sign_of_zero():
+    # one row, four blocks; s_global chosen so that every block scale is exactly 1.0 * s_global
+    sgl = np.float32(2.0 ** -10)
+    blk = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5, -6], dtype=np.float32)
+    W = np.zeros((1, 64), dtype=np.float32)
+    W[0, 0:16] = blk * sgl
+    W[0, 16:32] = -blk * sgl
+    W[0, 32:48] = 0.0                                   # all-zero block
+    W[0, 48:64] = np.float32(6.0) * sgl
+    W[0, 48] = -0.0
+    scales, sg = fo.compute_scales(W, s_global_in=float(sgl))
+    assert scales.tolist() == [[0x38, 0x38, 0x00, 0x38]]
+    k, neg, v = fo.bracket(W, scales, sg)
+    # a value on a node takes it as `lo` (v = 0); 6 is the closed end (k = 6, v = 1)
+    assert k[0, :16].tolist() == [0, 1, 2, 3, 4, 5, 6, 6, 0, 1, 2, 3, 4, 5, 6, 6]
+    assert v[0, :16].tolist() == [0, 0, 0, 0, 0, 0, 0, 1, .5, .5, .5, .5, .5, .5, .5, 1]
+    assert neg[0, :16].tolist() == [False] * 15 + [True]
+    assert neg[0, 16:32].tolist() == [False] + [True] * 14 + [False]      # -0.0 counts as +
+    assert np.all(k[0, 32:48] == 0) and np.all(v[0, 32:48] == 0) and not neg[0, 32:48].any()
+    assert not neg[0, 48]
+    # ties harden upward (Eq. 7 uses >=)
+    packed, vh, Wf = fo.harden_pack(v, fo.pack_code(k, neg), scales, sg)
+    assert vh[0, 8:15].all()
+    # w~ slightly above 6 after the block scale rounds down: clamp to the top node
+    W2 = np.full((1, 16), 1.0, dtype=np.float32)
+    W2[0, 0] = 1.06                                     # amax/6/s_global = 1.06 -> E4M3 1.0
+    sc2, sg2 = fo.compute_scales(W2, s_global_in=1.0 / 6.0)
+    k2, _, v2 = fo.bracket(W2, sc2, sg2)
+    assert sc2[0, 0] == 0x38 and k2[0, 0] == 6 and v2[0, 0] == 1.0
+    # all-zero tensor
+    sc0, sg0 = fo.compute_scales(np.zeros((2, 16), np.float32))
+    assert sg0 == 1.0 and not sc0.any()
+
+
+# ---- I5: limits of Eq. 3 ---------------------------------------------------
+
+def test_h_limits_and_floor_ceil():
+    for beta in (0.5, 4.0, 32.0, 1e4):
+        assert fo.h_beta(0.5, beta) == 0.5
+    W, _ = small_layer()
+    scales, sg, code, V = fo.softquant_init(W)
+    k, neg = fo.unpack_code(code)
+    s = np.repeat(fo.effective_scale(scales, sg), 16, axis=1).astype(np.float64)
+    sgn = np.where(neg, -1.0, 1.0)
+    Wlo, _ = fo.soft_weights(np.zeros_like(V), code, scales, sg, 80.0)
+    Whi, _ = fo.soft_weights(np.ones_like(V), code, scales, sg, 80.0)
+    assert np.allclose(Wlo, sgn * fo.NODES[k] * s, rtol=0, atol=1e-17)
+    assert np.allclose(Whi, sgn * fo.NODES[k + 1] * s, rtol=1e-15, atol=1e-17)
+    # beta -> infinity is a step function; no NaN on overflow
+    h = fo.h_beta(np.array([0.0, 0.49, 0.51, 1.0]), 1e6)
+    assert h.tolist() == [0.0, 0.0, 1.0, 1.0]
+    # monotone in v, symmetric about 0.5
+    v = np.linspace(0, 1, 101)
+    hh = fo.h_beta(v, 7.0)
+    assert np.all(np.diff(hh) > 0) and np.allclose(hh + hh[::-1], 1.0)
+
+
+# ---- I6 / I7: hardening, packing -------------------------------------------
+
+@pytest.mark.parametrize("seed", [0, 3])
+def test_harden_vinit_is_rtn_and_pack_roundtrip(seed):
+    W, _ = inputs.config1(seed, 32, 128, 8)
+    scales, sg, code, V = fo.softquant_init(W)
+    k, neg = fo.unpack_code(code)
+    packed, vh, Wf = fo.harden_pack(V, code, scales, sg)
+    mag_rtn = fo.rtn_nearest(W, scales, sg)
+    nib = np.empty(W.shape, np.uint8)
+    nib[:, 0::2], nib[:, 1::2] = packed & 0xF, packed >> 4
+    assert np.array_equal(nib & 7, mag_rtn)
+    assert np.array_equal(nib >> 3, (W < 0).astype(np.uint8))
+    assert np.array_equal(fo.dequant_packed(packed, scales, sg).view(np.uint32), Wf.view(np.uint32))
+    # RTN error is within half the local interval
+    s = np.repeat(fo.effective_scale(scales, sg), 16, axis=1).astype(np.float64)
+    wt = np.minimum(np.abs(W) / s, 6.0)
+    assert np.all(np.abs(np.abs(Wf) / s - wt) <= (fo.NODES[k + 1] - fo.NODES[k]) / 2 + 1e-6)
+    p0, _, _ = fo.harden_pack(np.zeros_like(V), code, scales, sg)
+    p1, _, _ = fo.harden_pack(np.ones_like(V), code, scales, sg)
+    assert np.array_equal(p0, code)
+    assert np.array_equal(p1, code + 0x11)
+    d = fo.pack_decisions(vh)
+    assert d.shape == (32, 16) and ((d[0, 0] >> 3) & 1) == int(vh[0, 3])
+
+
+# ---- I8: finite differences of Eq. 5 ---------------------------------------
+
+@pytest.mark.parametrize("opt_beta,lam,c", [(4.0, 1.0, 1.0), (11.0, 0.3, 0.01), (32.0, 5.0, 1.0)])
+def test_dv_matches_finite_differences(opt_beta, lam, c):
+    W, X = small_layer(5, 6, 32, 40)
+    scales, sg, code, V0 = fo.softquant_init(W)
+    Yref = fo.layer_ref(X, W)
+    rng = np.random.default_rng(0)
+    V = rng.uniform(0.05, 0.95, V0.shape)
+
+    def loss(Vx):
+        l, _, _ = fo.layer_fwd(X, Yref, Vx, code, scales, sg, opt_beta, c, mode="smooth")
+        return l + lam * fo.round_loss(Vx)
+
+    _, dY, _ = fo.layer_fwd(X, Yref, V, code, scales, sg, opt_beta, c, mode="smooth")
+    dV, _ = fo.layer_grad(dY, X, V, code, scales, sg, opt_beta, lam)
+    idx = rng.choice(V.size, 64, replace=False)
+    eps = 1e-6
+    for i in idx:
+        o, kk = divmod(int(i), V.shape[1])
+        Vp, Vm = V.copy(), V.copy()
+        Vp[o, kk] += eps
+        Vm[o, kk] -= eps
+        fd = (loss(Vp) - loss(Vm)) / (2 * eps)
+        assert abs(fd - dV[o, kk]) <= 1e-6 * max(abs(dV[o, kk]), np.abs(dV).max() * 1e-3), (o, kk, fd, dV[o, kk])
+
+
+# ---- I9: Round Loss closed forms -------------------------------------------
+
+def test_round_loss_closed_forms():
+    rng = np.random.default_rng(0)
+    assert fo.round_loss(rng.integers(0, 2, (7, 32)).astype(float)) == 0.0
+    assert fo.round_loss(np.full((3, 16), 0.5)) == 1.0
+    n = 100001
+    grid = np.linspace(0, 1, n).reshape(1, n)
+    # (1/N) sum 4v(1-v) on a fine uniform grid tends to the integral of 4v(1-v) over [0,1] = 2/3
+    assert abs(fo.round_loss(grid) - 2 / 3) < 1e-4
+    assert abs(fo.round_loss(np.array([[0.25, 0.75]])) - 0.75) < 1e-15
+    # its gradient is (4 - 8v)/N: isolate it with a zero data term
+    V = rng.uniform(0, 1, (4, 16))
+    code = np.zeros((4, 8), np.uint8)
+    scales = np.zeros((4, 1), np.uint8)                   # s = 0 -> no data gradient
+    dV, _ = fo.layer_grad(np.zeros((5, 4)), np.zeros((5, 16)), V, code, scales, 1.0, 4.0, 2.5)
+    assert np.allclose(dV, 2.5 / 64 * (4 - 8 * V), rtol=1e-15)
+
+
+# ---- I10: optimiser closed forms -------------------------------------------
+
+def test_adam_first_step_and_clip():
+    g = np.array([3.0, -0.2, 1e-3, -7.0, 0.0])
+    V = np.array([0.5, 0.5, 0.5, 0.995, 0.3])
+    Vn, m, u = fo.adam_update(V, g, np.zeros(5), np.zeros(5), 1e-2, 0.9, 0.999, 1e-8, 1)
+    expect = np.clip(V - 1e-2 * g / (np.abs(g) + 1e-8), 0, 1)
+    assert np.allclose(Vn, expect, rtol=1e-12)
+    assert Vn[3] == 1.0 and Vn[4] == 0.3
+    assert np.allclose(m, 0.1 * g) and np.allclose(u, 0.001 * g * g)
+    # constant gradient: every bias-corrected step moves by lr
+    Vc, m, u = np.array([0.9]), np.zeros(1), np.zeros(1)
+    for t in range(1, 6):
+        Vc, m, u = fo.adam_update(Vc, np.array([2.0]), m, u, 1e-2, 0.9, 0.999, 0.0, t)
+    assert np.allclose(Vc, 0.85)
+    assert fo.sgd_update(np.array([0.1, 0.9]), np.array([50.0, -50.0]), 0.01).tolist() == [0.0, 1.0]
+
+
+# ---- I11: exhaustive search on a tiny layer (Eq. 1) -------------------------
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_brute_force_4x16(seed):
+    W, X = inputs.config1(seed, 4, 16, 64)
+    scales, sg, code, V0 = fo.softquant_init(W)
+    Yref = fo.layer_ref(X, W)
+    k, neg = fo.unpack_code(code)
+    s = np.repeat(fo.effective_scale(scales, sg), 16, axis=1).astype(np.float64)
+    sgn = np.where(neg, -1.0, 1.0)
+    bits = ((np.arange(1 << 16)[:, None] >> np.arange(16)[None, :]) & 1).astype(np.float64)   # [65536,16]
+    Xd = X.astype(np.float64)
+
+    def hard_loss(vh):
+        Wq = sgn * (fo.NODES[k] + vh * (fo.NODES[k + 1] - fo.NODES[k])) * s
+        return np.sum((Xd @ Wq.T - Yref) ** 2, axis=0)                                       # per output row
+
+    # the loss separates over output rows, so 4 * 2^16 evaluations cover all 2^64 assignments
+    l_opt = np.empty(4)
+    for o in range(4):
+        cand = sgn[o] * (fo.NODES[k[o]] + bits * (fo.NODES[k[o] + 1] - fo.NODES[k[o]])) * s[o]   # [65536,16]
+        l_opt[o] = np.min(np.sum((Xd @ cand.T - Yref[:, o:o + 1]) ** 2, axis=0))
+    l_rtn = hard_loss(fo.harden(V0).astype(np.float64))
+    res = fo.run_layer(X, Yref, W, steps=150, lr=1e-2, mode="smooth")
+    l_faar = hard_loss(fo.harden(res["V"]).astype(np.float64))
+    assert np.all(l_opt <= l_rtn * (1 + 1e-12))
+    assert np.all(l_faar >= l_opt * (1 - 1e-12))
+    # hardening the soft solution matches evaluating Eq. 2 with a step function
+    _, _, Wf = fo.harden_pack(res["V"], code, scales, sg)
+    assert np.allclose(np.sum((Xd @ Wf.astype(np.float64).T - Yref) ** 2, axis=0), l_faar, rtol=1e-5)
+    # the optimiser does reduce the soft objective it is given
+    first, last = sum(res["hist"][0][:1]) + res["hist"][0][1], res["hist"][-1][0] + res["hist"][-1][1]
+    assert last < first
+
+
+# ---- I12: textbook GEMM special case ---------------------------------------
+
+def test_forward_reduces_to_naive_matmul_on_hard_weights():
+    W, X = small_layer(7, 5, 32, 9)
+    scales, sg, code, V0 = fo.softquant_init(W)
+    rng = np.random.default_rng(0)
+    Vh = rng.integers(0, 2, V0.shape).astype(np.float64)
+    _, _, Wf = fo.harden_pack(Vh, code, scales, sg)
+    Yq_naive = np.zeros((9, 5))
+    for t, o, kk in itertools.product(range(9), range(5), range(32)):
+        Yq_naive[t, o] += float(X[t, kk]) * float(Wf[o, kk])
+    loss, dY, Yq = fo.layer_fwd(X, np.zeros((9, 5)), Vh, code, scales, sg, 200.0, 1.0, mode="smooth")
+    assert np.allclose(Yq, Yq_naive, rtol=1e-6, atol=1e-9)
+    assert np.isclose(loss, np.sum(Yq_naive ** 2), rtol=1e-6)
+    assert np.allclose(dY, 2 * Yq_naive, rtol=1e-6, atol=1e-9)
+    # gradient GEMM against a naive loop
+    _, G = fo.layer_grad(dY, X, Vh, code, scales, sg, 4.0, 0.0)
+    Gn = np.zeros((5, 32))
+    for t, o, kk in itertools.product(range(9), range(5), range(32)):
+        Gn[o, kk] += dY[t, o] * float(X[t, kk])
+    assert np.allclose(G, Gn, rtol=1e-12, atol=1e-12)
+
+
+# ---- I13: zero-residual fixed point ----------------------------------------
+
+def test_zero_residual_leaves_only_round_term():
+    W, X = small_layer(9, 6, 32, 20)
+    scales, sg, code, V0 = fo.softquant_init(W)
+    rng = np.random.default_rng(0)
+    V = rng.uniform(0.02, 0.98, V0.shape)
+    Wsoft, _ = fo.soft_weights(V, code, scales, sg, 6.0)
+    Yref = X.astype(np.float64) @ Wsoft.T
+    hp = fo.HParams(beta=6.0, lambda_round=2.0, opt=0, lr=0.5)
+    Vn, _, _, l_mse, l_round, dV = fo.layer_step(X, Yref, V, code, scales, sg, None, None, hp, mode="smooth")
+    assert l_mse < 1e-20
+    assert np.allclose(dV, 2.0 / V.size * (4 - 8 * V), rtol=1e-9, atol=1e-15)
+    # the round term pushes each v toward the nearer of {0, 1}
+    away = V != 0.5
+    assert np.all(np.abs(Vn[away] - 0.5) > np.abs(V[away] - 0.5))
+
+
+# ---- rounding points of mode "bf16" ----------------------------------------
+
+def test_bf16_mode_rounds_only_at_the_stated_points():
+    W, X = inputs.config2(0, 16, 64, 32)
+    scales, sg, code, V = fo.softquant_init(W)
+    Yref = inputs.to_bf16_f32(fo.layer_ref(X, W))
+    l_b, dY_b, Yq_b = fo.layer_fwd(X, Yref, V, code, scales, sg, 4.0, 1.0, mode="bf16")
+    Ws, _ = fo.soft_weights(V, code, scales, sg, 4.0)
+    Wb = torch.from_numpy(Ws.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    # (binary32 then BF16 may differ from one rounding only on exact ties; none occur here)
+    assert np.array_equal(Wb, fo.bf16_round(Ws))
+    assert np.array_equal(Yq_b, X.astype(np.float64) @ Wb.T)
+    assert np.array_equal(dY_b, fo.bf16_round(2 * (Yq_b - Yref)))
+    Vn, m, u, *_ = fo.layer_step(X, Yref, V, code, scales, sg, np.zeros_like(V), np.zeros_like(V), fo.HParams(), "bf16")
+    assert Vn.dtype == np.float32 and m.dtype == np.float32 and u.dtype == np.float32
