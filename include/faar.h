@@ -1,0 +1,205 @@
+/*
+ * faar.h -- C ABI of libfaar.so: one FAAR layer-wise rounding-optimisation step
+ * for a linear layer, on one NVIDIA B200 (sm_100a).
+ *
+ * The operations are the ones the paper's Procedure table lists for Stage 1
+ * (steps 2-13) and for hardening (steps 25-26); each entry point below cites
+ * the step / equation it implements.
+ *
+ * Conventions
+ *   - nn.Linear orientation: W[O,K] row-major (K contiguous), X[T,K], Y[T,O] = X W^T.
+ *     N = O*K is the number of quantised weights of the layer.  NVFP4 scale
+ *     blocks are 16 consecutive elements along K; K % 16 == 0 is required.
+ *   - Every tensor argument is a caller-owned DEVICE pointer unless it says
+ *     "host".  The library never allocates device memory: scratch comes from
+ *     the caller's `workspace` (size from faar_workspace_size).  Hyper-
+ *     parameters are passed by value in host structs.  Scalar results (losses,
+ *     s_global) are written to device memory; no call synchronises the stream.
+ *   - All work is enqueued on the context's stream.  A context is not
+ *     thread-safe.  V, adam_m, adam_u are updated in place.
+ *   - Every function returns an int status (FAAR_OK == 0).  Nothing throws or
+ *     aborts.  On a device that is not sm_100 every compute call returns
+ *     FAAR_ERR_ARCH; there is no CPU fallback.
+ *   - The tensor-core kernels bound every wait on a barrier.  If a wait gives
+ *     up, the kernel records a code in the workspace status word, releases its
+ *     tensor memory and returns; faar_check_status reports it as
+ *     FAAR_ERR_TIMEOUT after the caller has synchronised the stream.
+ *
+ * Packed formats
+ *   code   [O, K/2] u8: element 2j in bits 3:0, element 2j+1 in bits 7:4 of byte j;
+ *          nibble = sign<<3 | k, k in 0..6 the index of the LOWER bracketing node
+ *          in (0, 0.5, 1, 1.5, 2, 3, 4, 6) -- i.e. the E2M1 code of that node.
+ *   scales [O, K/16] u8: FP8 E4M3 block scales, linear row-major.
+ *   packed [O, K/2] u8: same nibble order, nibble = sign<<3 | (k + v_hat): the
+ *          deployable E2M1 weight code.
+ */
+#ifndef FAAR_H_
+#define FAAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define FAAR_API __attribute__((visibility("default")))
+#else
+#define FAAR_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  FAAR_OK = 0,
+  FAAR_ERR_INVALID_ARG = 1, /* null pointer, bad enum, bad hyper-parameter      */
+  FAAR_ERR_SHAPE = 2,       /* O/K/T <= 0, K % 16 != 0, leading dim too small   */
+  FAAR_ERR_ALIGN = 3,       /* pointer not 16-byte aligned / ld not multiple of 8 */
+  FAAR_ERR_DTYPE = 4,
+  FAAR_ERR_WORKSPACE = 5,   /* workspace null, misaligned or too small          */
+  FAAR_ERR_ARCH = 6,        /* device is not compute capability 10.x            */
+  FAAR_ERR_CUDA = 7,        /* a CUDA call failed; see faar_last_cuda_error     */
+  FAAR_ERR_TIMEOUT = 8      /* a bounded device-side wait gave up               */
+};
+
+typedef struct faar_ctx faar_ctx;
+
+typedef enum { FAAR_BF16 = 0, FAAR_F32 = 1 } faar_dtype;
+
+/* Hyper-parameters of one step (host struct, by pointer, read at call time).
+ * beta: temperature of Eq. 3.  lambda_round: weight of the Round Loss in Eq. 5.
+ * mse_scale: factor c on the squared Frobenius norm (the paper's Eq. 5 has c = 1).
+ * opt: 0 = gradient descent, 1 = Adam (bias-corrected, no weight decay).
+ * step: 1-based step index (Adam bias correction). */
+typedef struct {
+  float beta, lambda_round, mse_scale;
+  int opt;
+  float lr, beta1, beta2, eps;
+  int step;
+} faar_hparams;
+
+/* Layer geometry.  Leading dimensions are in ELEMENTS.
+ * ldw : row stride of W[O,K]          (>= K)
+ * ldx : row stride of X[T,K]          (>= K, multiple of 8)
+ * ldxt: row stride of Xt[K,T] = X^T   (>= T, multiple of 8)
+ * ldy : row stride of Y_ref[T,O] and of the optional Y_q output (>= O)
+ * V, code, scales, adam_m, adam_u, dV are dense (row strides K, K/2, K/16, K). */
+typedef struct {
+  int O, K, T;
+  int64_t ldw, ldx, ldxt, ldy;
+  int w_dtype;    /* faar_dtype of W      */
+  int yref_dtype; /* faar_dtype of Y_ref  */
+} faar_shape;
+
+/* ---- context -------------------------------------------------------------- */
+
+/* Creates a context bound to `device` and to `stream` (a cudaStream_t, may be 0).
+ * Returns FAAR_ERR_ARCH if the device is not sm_100.  Host memory only. */
+FAAR_API int faar_create(faar_ctx** out, int device, void* stream);
+FAAR_API int faar_destroy(faar_ctx* ctx);
+FAAR_API int faar_set_stream(faar_ctx* ctx, void* stream);
+FAAR_API const char* faar_status_string(int status);
+/* Last cudaError_t seen by this context (0 if none). */
+FAAR_API int faar_last_cuda_error(const faar_ctx* ctx);
+
+/* Bytes of workspace that any call on this shape needs (host out-pointer).
+ * The workspace must be 256-byte aligned.  Its first 256 bytes hold the status
+ * word; the caller zeroes them once (faar_workspace_init) before first use. */
+FAAR_API int faar_workspace_size(const faar_shape* shape, size_t* bytes);
+/* Enqueues the zeroing of the workspace header (status word, counters). */
+FAAR_API int faar_workspace_init(faar_ctx* ctx, void* workspace, size_t workspace_bytes);
+/* Synchronises the context's stream and returns FAAR_ERR_TIMEOUT if a kernel
+ * recorded a wait that gave up (detail_out, host, nullable: the raw code),
+ * FAAR_ERR_CUDA if the stream is in error, else FAAR_OK. */
+FAAR_API int faar_check_status(faar_ctx* ctx, const void* workspace, uint32_t* detail_out);
+
+/* ---- part 1: soft-quantisation set-up, once per layer ----------------------
+ * Procedure steps 2-5, "NVFP4 Overview", Eq. 4.
+ * Computes the FP32 tensor scale (s_global = amax|W| / (6*448) unless
+ * s_global_in > 0 is given), the E4M3 block scales s_g = E4M3(amax_block /
+ * (6*s_global)) (round to nearest even, saturating at 448), and per weight the
+ * normalised magnitude w~ = |w| / (s_g*s_global) clamped to 6, the index k of
+ * the lower bracketing node (intervals half-open, the last closed), the sign
+ * bit, and V_init = (w~ - lo) / (hi - lo).  All arithmetic IEEE binary32, one
+ * correctly rounded operation at a time, so the byte outputs are reproducible.
+ *   W           in : [O,K] (w_dtype, ldw)
+ *   scales      out: [O,K/16] u8      s_global_out out: 1 float (device)
+ *   code        out: [O,K/2] u8       V_init       out: [O,K] float */
+FAAR_API int faar_softquant_init(faar_ctx* ctx, const faar_shape* shape, const void* W, float s_global_in,
+                        uint8_t* scales, float* s_global_out, uint8_t* code, float* V_init,
+                        void* workspace, size_t workspace_bytes);
+
+/* ---- part 2: soft weights, FP32 view ---------------------------------------
+ * Procedure steps 6-7, Eq. 2 and Eq. 3:  h = sigmoid(beta*(v-0.5)),
+ * W_soft = sign*(lo + h*(hi-lo))*s_g*s_global.  This is the FP32 view of what
+ * the forward GEMM's operand is built from; either output may be null.
+ *   W_soft out: [O,K] float (nullable)    h out: [O,K] float (nullable) */
+FAAR_API int faar_softquant_eval(faar_ctx* ctx, const faar_shape* shape, const float* V, const uint8_t* code,
+                        const uint8_t* scales, const float* s_global, float beta,
+                        float* W_soft, float* h);
+
+/* ---- layout helper ----------------------------------------------------------
+ * out[c, r] = in[r, c] for a BF16 matrix in[rows, cols] (ld_in) -> out[cols, rows]
+ * (ld_out).  Used once per layer to build Xt = X^T, the K-major operand of the
+ * dW GEMM (no counterpart in the paper: a storage choice of this library). */
+FAAR_API int faar_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in, int64_t ld_in,
+                        void* out, int64_t ld_out);
+
+/* ---- frozen target ----------------------------------------------------------
+ * Procedure step 8: Y_fp = X W^T with the original BF16 weights (w_dtype must
+ * be FAAR_BF16, ldw multiple of 8), FP32 accumulation on the tensor cores,
+ * written as yref_dtype to Y_ref[T,O] (ldy). */
+FAAR_API int faar_layer_ref(faar_ctx* ctx, const faar_shape* shape, const void* X, const void* W, void* Y_ref,
+                   void* workspace, size_t workspace_bytes);
+
+/* ---- part 3: forward GEMM + MSE ---------------------------------------------
+ * Procedure steps 6-10, first term of Eq. 5.  Builds W_soft (Eq. 2, rounded to
+ * BF16), computes Y_q = X W_soft^T on the tensor cores with FP32 accumulation,
+ * r = Y_q - Y_ref, L_MSE = mse_scale * sum r^2 and dY = 2*mse_scale*r.
+ *   X        in : [T,K] bf16 (ldx)           Y_ref in: [T,O] (yref_dtype, ldy)
+ *   dYt      out: [O, ceil8(T)] bf16, dY transposed (row stride = T rounded up to 8)
+ *   loss_mse out: 1 float (device)           Y_q out: [T,O] bf16 (ldy), nullable */
+FAAR_API int faar_layer_fwd(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp, const void* X,
+                   const void* Y_ref, const float* V, const uint8_t* code, const uint8_t* scales,
+                   const float* s_global, void* dYt, float* loss_mse, void* Y_q,
+                   void* workspace, size_t workspace_bytes);
+
+/* ---- part 4: Round Loss, backward, update -----------------------------------
+ * Eq. 5, second term without lambda: L_round = (1/N) sum (1 - (2v-1)^2).
+ *   V in: N floats     loss_round out: 1 float (device) */
+FAAR_API int faar_round_loss(faar_ctx* ctx, const float* V, int64_t N, float* loss_round,
+                    void* workspace, size_t workspace_bytes);
+
+/* Procedure step 13 with the clip that Stage 1 prescribes.  G = dY^T X on the
+ * tensor cores (contraction over T), then per weight
+ *   dV = G*sign*s*(hi-lo)*beta*h*(1-h) + (lambda_round/N)*(4-8v)
+ * (the derivative of Eq. 5 through Eq. 2 and Eq. 3), the optimiser update and
+ * v <- clamp(v, 0, 1).  All of it at the pre-update V.
+ *   dYt in: [O, ceil8(T)] bf16 (from faar_layer_fwd)   Xt in: [K,T] bf16 (ldxt)
+ *   V in/out: [O,K] float    adam_m, adam_u in/out: [O,K] float (null for opt 0)
+ *   dV out: [O,K] float, nullable */
+FAAR_API int faar_layer_bwd(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp, const void* dYt,
+                   const void* Xt, float* V, const uint8_t* code, const uint8_t* scales,
+                   const float* s_global, float* adam_m, float* adam_u, float* dV,
+                   void* workspace, size_t workspace_bytes);
+
+/* Forward, Round Loss and backward + update back to back: one pass of Procedure
+ * steps 6-13.  loss_out2 (device) receives {L_MSE, L_round}, both at the
+ * pre-update V.  dYt lives in the workspace. */
+FAAR_API int faar_layer_step(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp, const void* X,
+                    const void* Xt, const void* Y_ref, float* V, const uint8_t* code,
+                    const uint8_t* scales, const float* s_global, float* adam_m, float* adam_u,
+                    float* loss_out2, void* workspace, size_t workspace_bytes);
+
+/* ---- part 5: harden + pack ---------------------------------------------------
+ * Procedure steps 25-26, Eq. 7: v_hat = (v >= 0.5); weight code = k + v_hat.
+ *   packed     out: [O,K/2] u8           scales_out out: [O,K/16] u8 (copy; nullable)
+ *   decisions  out: [O,K/8] u8 bitmask, element 8j+i in bit i of byte j (nullable)
+ *   W_final    out: [O,K] of wfinal_dtype = sign*node*s_g*s_global (nullable) */
+FAAR_API int faar_harden_pack(faar_ctx* ctx, const faar_shape* shape, const float* V, const uint8_t* code,
+                     const uint8_t* scales, const float* s_global, uint8_t* packed,
+                     uint8_t* scales_out, uint8_t* decisions, void* W_final, int wfinal_dtype);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FAAR_H_ */

@@ -1,0 +1,349 @@
+// extern "C" entry points of libfaar.so: argument validation, workspace carving,
+// kernel sequencing.  No device memory is allocated here.
+#include <math.h>
+#include <new>
+
+#include "faar_internal.cuh"
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(faar_ctx* ctx, int e) {
+  if (e == 0) return FAAR_OK;
+  ctx->last_cuda_error = e;
+  return FAAR_ERR_CUDA;
+}
+
+int check_shape(const faar_shape* s) {
+  if (!s) return FAAR_ERR_INVALID_ARG;
+  if (s->O <= 0 || s->K <= 0 || s->T <= 0) return FAAR_ERR_SHAPE;
+  if (s->K % 16 != 0) return FAAR_ERR_SHAPE;
+  return FAAR_OK;
+}
+
+int check_ws(const faar_shape* s, const void* ws, size_t ws_bytes) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return FAAR_ERR_WORKSPACE;
+  if (ws_bytes < faar_ws_plan(s).total) return FAAR_ERR_WORKSPACE;
+  return FAAR_OK;
+}
+
+int check_hp(const faar_hparams* hp, bool need_opt) {
+  if (!hp) return FAAR_ERR_INVALID_ARG;
+  if (!(hp->beta > 0.f) || !isfinite(hp->beta) || !isfinite(hp->mse_scale) || !isfinite(hp->lambda_round))
+    return FAAR_ERR_INVALID_ARG;
+  if (need_opt) {
+    if (hp->opt != 0 && hp->opt != 1) return FAAR_ERR_INVALID_ARG;
+    if (!isfinite(hp->lr)) return FAAR_ERR_INVALID_ARG;
+    if (hp->opt == 1 && (hp->step < 1 || !(hp->beta1 >= 0.f && hp->beta1 < 1.f) ||
+                         !(hp->beta2 >= 0.f && hp->beta2 < 1.f) || !(hp->eps >= 0.f)))
+      return FAAR_ERR_INVALID_ARG;
+  }
+  return FAAR_OK;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  explicit DeviceGuard(int dev) { cudaGetDevice(&prev); if (prev != dev) cudaSetDevice(dev); else prev = -1; }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Y_ref,
+             const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
+             void* Y_q, uint8_t* ws, const faar_ws_layout& l, int* n_partials) {
+  __nv_bfloat16* wsoft = reinterpret_cast<__nv_bfloat16*>(ws + l.off_wsoft);
+  int e = faar_launch_softquant_bf16(ctx, s, V, code, scales, s_global, hp->beta, wsoft);
+  if (e) return e;
+  faar_gemm_args a = {};
+  a.mode = FAAR_GEMM_FWD;
+  a.M = s->O; a.N = s->T; a.Kc = s->K;
+  a.A = wsoft; a.lda = s->K;
+  a.B = X; a.ldb = s->ldx;
+  a.status = reinterpret_cast<uint32_t*>(ws);
+  a.Yout = Y_q; a.yout_dtype = FAAR_BF16; a.ldy = s->ldy;
+  a.Yref = Y_ref; a.yref_dtype = s->yref_dtype;
+  a.dYt = reinterpret_cast<__nv_bfloat16*>(dYt); a.ld_dyt = l.ld_dyt;
+  a.mse2c = 2.0f * hp->mse_scale;
+  a.partials = reinterpret_cast<float*>(ws + l.off_mse_partials);
+  return faar_launch_gemm(ctx, &a, n_partials);
+}
+
+int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* dYt, const void* Xt,
+             float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
+             float* adam_u, float* dV, uint8_t* ws, const faar_ws_layout& l, int* n_partials) {
+  faar_gemm_args a = {};
+  a.mode = FAAR_GEMM_BWD;
+  a.M = s->O; a.N = s->K; a.Kc = s->T;
+  a.A = dYt; a.lda = l.ld_dyt;
+  a.B = Xt; a.ldb = s->ldxt;
+  a.status = reinterpret_cast<uint32_t*>(ws);
+  a.partials = reinterpret_cast<float*>(ws + l.off_round_partials);
+  a.V = V; a.code = code; a.scales = scales; a.s_global = s_global;
+  a.adam_m = adam_m; a.adam_u = adam_u; a.dV = dV;
+  a.beta = hp->beta;
+  a.lam_over_n = (float)((double)hp->lambda_round / ((double)s->O * (double)s->K));
+  a.lr = hp->lr; a.b1 = hp->beta1; a.b2 = hp->beta2; a.eps = hp->eps; a.opt = hp->opt;
+  if (hp->opt == 1) {
+    a.inv_bc1 = (float)(1.0 / (1.0 - pow((double)hp->beta1, (double)hp->step)));
+    a.inv_bc2 = (float)(1.0 / (1.0 - pow((double)hp->beta2, (double)hp->step)));
+  }
+  return faar_launch_gemm(ctx, &a, n_partials);
+}
+
+int check_gemm_operands(const faar_shape* s, bool need_x, bool need_xt) {
+  if (need_x && (s->ldx < s->K || s->ldx % 8)) return s->ldx < s->K ? FAAR_ERR_SHAPE : FAAR_ERR_ALIGN;
+  if (need_xt && (s->ldxt < s->T || s->ldxt % 8)) return s->ldxt < s->T ? FAAR_ERR_SHAPE : FAAR_ERR_ALIGN;
+  return FAAR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* faar_status_string(int status) {
+  switch (status) {
+    case FAAR_OK: return "ok";
+    case FAAR_ERR_INVALID_ARG: return "invalid argument";
+    case FAAR_ERR_SHAPE: return "unsupported shape";
+    case FAAR_ERR_ALIGN: return "misaligned pointer or leading dimension";
+    case FAAR_ERR_DTYPE: return "unsupported dtype";
+    case FAAR_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case FAAR_ERR_ARCH: return "device is not sm_100";
+    case FAAR_ERR_CUDA: return "CUDA error";
+    case FAAR_ERR_TIMEOUT: return "device-side wait gave up";
+  }
+  return "unknown status";
+}
+
+int faar_create(faar_ctx** out, int device, void* stream) {
+  if (!out) return FAAR_ERR_INVALID_ARG;
+  *out = nullptr;
+  cudaDeviceProp prop;
+  cudaError_t e = cudaGetDeviceProperties(&prop, device);
+  if (e != cudaSuccess) return FAAR_ERR_CUDA;
+  if (prop.major != 10) return FAAR_ERR_ARCH;
+  faar_ctx* c = new (std::nothrow) faar_ctx();
+  if (!c) return FAAR_ERR_INVALID_ARG;
+  c->device = device;
+  c->num_sms = prop.multiProcessorCount;
+  c->stream = reinterpret_cast<cudaStream_t>(stream);
+  c->last_cuda_error = 0;
+  c->encode_tiled = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q);
+  if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !c->encode_tiled) {
+    delete c;
+    return FAAR_ERR_CUDA;
+  }
+  *out = c;
+  return FAAR_OK;
+}
+
+int faar_destroy(faar_ctx* ctx) {
+  delete ctx;
+  return FAAR_OK;
+}
+
+int faar_set_stream(faar_ctx* ctx, void* stream) {
+  if (!ctx) return FAAR_ERR_INVALID_ARG;
+  ctx->stream = reinterpret_cast<cudaStream_t>(stream);
+  return FAAR_OK;
+}
+
+int faar_last_cuda_error(const faar_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int faar_workspace_size(const faar_shape* shape, size_t* bytes) {
+  if (!bytes) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(shape);
+  if (st) return st;
+  *bytes = faar_ws_plan(shape).total;
+  return FAAR_OK;
+}
+
+int faar_workspace_init(faar_ctx* ctx, void* workspace, size_t workspace_bytes) {
+  if (!ctx) return FAAR_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
+    return FAAR_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  return cuda_fail(ctx, (int)cudaMemsetAsync(workspace, 0, FAAR_WS_HEADER, ctx->stream));
+}
+
+int faar_check_status(faar_ctx* ctx, const void* workspace, uint32_t* detail_out) {
+  if (!ctx || !workspace) return FAAR_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  uint32_t word = 0;
+  cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e == cudaSuccess) e = cudaMemcpy(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+  if (detail_out) *detail_out = word;
+  return word ? FAAR_ERR_TIMEOUT : FAAR_OK;
+}
+
+int faar_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float s_global_in, uint8_t* scales,
+                        float* s_global_out, uint8_t* code, float* V_init, void* workspace,
+                        size_t workspace_bytes) {
+  if (!ctx || !W || !scales || !s_global_out || !code || !V_init) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if (s->w_dtype != FAAR_BF16 && s->w_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
+  if (s->ldw < s->K) return FAAR_ERR_SHAPE;
+  if (s->ldw % 8 || !aligned16(W) || !aligned16(V_init) || !aligned16(code)) return FAAR_ERR_ALIGN;
+  if (!isfinite(s_global_in) || s_global_in < 0.f) return FAAR_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
+    return FAAR_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  uint32_t* amax_word = reinterpret_cast<uint32_t*>(workspace) + 1;
+  return cuda_fail(ctx, faar_launch_softquant_init(ctx, s, W, s_global_in, scales, s_global_out, code, V_init,
+                                                   amax_word));
+}
+
+int faar_softquant_eval(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
+                        const uint8_t* scales, const float* s_global, float beta, float* W_soft, float* h) {
+  if (!ctx || !V || !code || !scales || !s_global) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if (!(beta > 0.f) || !isfinite(beta)) return FAAR_ERR_INVALID_ARG;
+  if (!aligned16(V) || !aligned16(code) || (W_soft && !aligned16(W_soft)) || (h && !aligned16(h)))
+    return FAAR_ERR_ALIGN;
+  if (!W_soft && !h) return FAAR_OK;
+  DeviceGuard g(ctx->device);
+  return cuda_fail(ctx, faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, beta, W_soft, h));
+}
+
+int faar_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in, int64_t ld_in, void* out,
+                        int64_t ld_out) {
+  if (!ctx || !in || !out) return FAAR_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || ld_in < cols || ld_out < rows) return FAAR_ERR_SHAPE;
+  DeviceGuard g(ctx->device);
+  return cuda_fail(ctx, faar_launch_transpose_bf16(ctx, rows, cols, in, ld_in, out, ld_out));
+}
+
+int faar_layer_ref(faar_ctx* ctx, const faar_shape* s, const void* X, const void* W, void* Y_ref,
+                   void* workspace, size_t workspace_bytes) {
+  if (!ctx || !X || !W || !Y_ref) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if (s->w_dtype != FAAR_BF16) return FAAR_ERR_DTYPE;
+  if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
+  if (s->ldw < s->K || s->ldy < s->O) return FAAR_ERR_SHAPE;
+  if ((st = check_gemm_operands(s, true, false))) return st;
+  if (s->ldw % 8 || !aligned16(X) || !aligned16(W)) return FAAR_ERR_ALIGN;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
+    return FAAR_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  faar_gemm_args a = {};
+  a.mode = FAAR_GEMM_REF;
+  a.M = s->O; a.N = s->T; a.Kc = s->K;
+  a.A = W; a.lda = s->ldw;
+  a.B = X; a.ldb = s->ldx;
+  a.status = reinterpret_cast<uint32_t*>(workspace);
+  a.Yout = Y_ref; a.yout_dtype = s->yref_dtype; a.ldy = s->ldy;
+  return cuda_fail(ctx, faar_launch_gemm(ctx, &a, nullptr));
+}
+
+int faar_layer_fwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Y_ref,
+                   const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
+                   float* loss_mse, void* Y_q, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !X || !Y_ref || !V || !code || !scales || !s_global || !dYt || !loss_mse) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if ((st = check_hp(hp, false))) return st;
+  if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
+  if (s->ldy < s->O) return FAAR_ERR_SHAPE;
+  if ((st = check_gemm_operands(s, true, false))) return st;
+  if (!aligned16(X) || !aligned16(V) || !aligned16(code) || !aligned16(dYt)) return FAAR_ERR_ALIGN;
+  if ((st = check_ws(s, workspace, workspace_bytes))) return st;
+  DeviceGuard g(ctx->device);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const faar_ws_layout l = faar_ws_plan(s);
+  int np = 0;
+  int e = fwd_impl(ctx, s, hp, X, Y_ref, V, code, scales, s_global, dYt, Y_q, ws, l, &np);
+  if (e) return cuda_fail(ctx, e);
+  e = faar_launch_finalize(ctx, reinterpret_cast<float*>(ws + l.off_mse_partials), np, hp->mse_scale, loss_mse,
+                           nullptr, 0, 0.f, nullptr);
+  return cuda_fail(ctx, e);
+}
+
+int faar_round_loss(faar_ctx* ctx, const float* V, int64_t N, float* loss_round, void* workspace,
+                    size_t workspace_bytes) {
+  if (!ctx || !V || !loss_round) return FAAR_ERR_INVALID_ARG;
+  if (N <= 0) return FAAR_ERR_SHAPE;
+  if (!aligned16(V)) return FAAR_ERR_ALIGN;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+      workspace_bytes < FAAR_WS_HEADER + 2 * sizeof(float) * FAAR_MAX_PARTIALS)
+    return FAAR_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  float* partials = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + FAAR_WS_HEADER +
+                                             sizeof(float) * FAAR_MAX_PARTIALS);
+  int np = 0;
+  int e = faar_launch_round_partials(ctx, V, N, partials, &np);
+  if (e) return cuda_fail(ctx, e);
+  e = faar_launch_finalize(ctx, partials, np, (float)(1.0 / (double)N), loss_round, nullptr, 0, 0.f, nullptr);
+  return cuda_fail(ctx, e);
+}
+
+int faar_layer_bwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* dYt, const void* Xt,
+                   float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
+                   float* adam_u, float* dV, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !dYt || !Xt || !V || !code || !scales || !s_global) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if ((st = check_hp(hp, true))) return st;
+  if (hp->opt == 1 && (!adam_m || !adam_u)) return FAAR_ERR_INVALID_ARG;
+  if ((st = check_gemm_operands(s, false, true))) return st;
+  if (!aligned16(dYt) || !aligned16(Xt) || !aligned16(V) || !aligned16(code) || (adam_m && !aligned16(adam_m)) ||
+      (adam_u && !aligned16(adam_u)) || (dV && !aligned16(dV)))
+    return FAAR_ERR_ALIGN;
+  if ((st = check_ws(s, workspace, workspace_bytes))) return st;
+  DeviceGuard g(ctx->device);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const faar_ws_layout l = faar_ws_plan(s);
+  return cuda_fail(ctx, bwd_impl(ctx, s, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, dV, ws, l, nullptr));
+}
+
+int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Xt,
+                    const void* Y_ref, float* V, const uint8_t* code, const uint8_t* scales, const float* s_global,
+                    float* adam_m, float* adam_u, float* loss_out2, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !X || !Xt || !Y_ref || !V || !code || !scales || !s_global || !loss_out2) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if ((st = check_hp(hp, true))) return st;
+  if (hp->opt == 1 && (!adam_m || !adam_u)) return FAAR_ERR_INVALID_ARG;
+  if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
+  if (s->ldy < s->O) return FAAR_ERR_SHAPE;
+  if ((st = check_gemm_operands(s, true, true))) return st;
+  if (!aligned16(X) || !aligned16(Xt) || !aligned16(V) || !aligned16(code) || (adam_m && !aligned16(adam_m)) ||
+      (adam_u && !aligned16(adam_u)))
+    return FAAR_ERR_ALIGN;
+  if ((st = check_ws(s, workspace, workspace_bytes))) return st;
+  DeviceGuard g(ctx->device);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const faar_ws_layout l = faar_ws_plan(s);
+  void* dYt = ws + l.off_dyt;
+  int np_mse = 0, np_round = 0;
+  int e = fwd_impl(ctx, s, hp, X, Y_ref, V, code, scales, s_global, dYt, nullptr, ws, l, &np_mse);
+  if (e) return cuda_fail(ctx, e);
+  e = bwd_impl(ctx, s, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, nullptr, ws, l, &np_round);
+  if (e) return cuda_fail(ctx, e);
+  e = faar_launch_finalize(ctx, reinterpret_cast<float*>(ws + l.off_mse_partials), np_mse, hp->mse_scale, loss_out2,
+                           reinterpret_cast<float*>(ws + l.off_round_partials), np_round,
+                           (float)(1.0 / ((double)s->O * (double)s->K)), loss_out2 + 1);
+  return cuda_fail(ctx, e);
+}
+
+int faar_harden_pack(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code, const uint8_t* scales,
+                     const float* s_global, uint8_t* packed, uint8_t* scales_out, uint8_t* decisions, void* W_final,
+                     int wfinal_dtype) {
+  if (!ctx || !V || !code || !scales || !packed) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if (W_final && !s_global) return FAAR_ERR_INVALID_ARG;
+  if (W_final && wfinal_dtype != FAAR_BF16 && wfinal_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
+  if (!aligned16(V) || !aligned16(code) || !aligned16(packed) || (W_final && !aligned16(W_final)))
+    return FAAR_ERR_ALIGN;
+  DeviceGuard g(ctx->device);
+  return cuda_fail(ctx, faar_launch_harden_pack(ctx, s, V, code, scales, s_global, packed, scales_out, decisions,
+                                                W_final, wfinal_dtype));
+}
+
+}  // extern "C"

@@ -1,0 +1,395 @@
+// HBM-bound kernels of the FAAR layer step: soft-quantisation set-up (scales,
+// bracket, V_init), the FP32 soft-weight view, the BF16 soft-weight operand,
+// Round Loss reduction, hardening + packing, and a BF16 transpose.
+//
+// Work decomposition used by all per-weight kernels: one thread owns 8
+// consecutive weights of a row (half a scale block), so V moves as two float4,
+// the code as one 32-bit word and BF16 data as one 16-byte vector; the two
+// threads of a block exchange their maxima with one shuffle.
+#include "faar_internal.cuh"
+
+namespace {
+
+constexpr int EW_THREADS = 256;
+
+__device__ __forceinline__ void load8(const void* W, int w_dtype, int64_t idx, float (&w)[8]) {
+  if (w_dtype == FAAR_BF16) {
+    uint4 raw = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W) + idx);
+    const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      w[2 * i] = __uint_as_float(r[i] << 16);
+      w[2 * i + 1] = __uint_as_float(r[i] & 0xFFFF0000u);
+    }
+  } else {
+    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(W) + idx);
+    float4 a = p[0], b = p[1];
+    w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
+    w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
+  }
+}
+
+// ---- pass 1: max |W| over the tensor -----------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, uint32_t* amax_word) {
+  const int64_t groups_per_row = K / 8;
+  const int64_t total = (int64_t)O * groups_per_row;
+  float amax = 0.f;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total;
+       g += (int64_t)gridDim.x * blockDim.x) {
+    int64_t row = g / groups_per_row, col = (g - row * groups_per_row) * 8;
+    float w[8];
+    load8(W, w_dtype, row * ldw + col, w);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[i]));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  __shared__ float s_max[EW_THREADS / 32];
+  if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m = 0.f;
+    for (int i = 0; i < EW_THREADS / 32; ++i) m = fmaxf(m, s_max[i]);
+    atomicMax(amax_word, __float_as_uint(m));   // non-negative floats order like their bit patterns
+  }
+}
+
+// ---- pass 2: block scales, bracket, V_init -------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw,
+                      float s_global_in, const uint32_t* __restrict__ amax_word,
+                      uint8_t* __restrict__ scales, float* __restrict__ s_global_out,
+                      uint8_t* __restrict__ code, float* __restrict__ V) {
+  float s_global;
+  if (s_global_in > 0.f) {
+    s_global = s_global_in;
+  } else {
+    float amax_t = __uint_as_float(*amax_word);
+    s_global = amax_t == 0.f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) *s_global_out = s_global;
+  const float d = __fmul_rn(s_global, 6.0f);
+
+  const int64_t groups_per_row = K / 8;
+  const int64_t total = (int64_t)O * groups_per_row;
+  // the grid is sized so that every warp is either fully inside or the tail is padded with idle lanes
+  for (int64_t g0 = (int64_t)blockIdx.x * blockDim.x; g0 < total; g0 += (int64_t)gridDim.x * blockDim.x) {
+    int64_t g = g0 + threadIdx.x;
+    bool valid = g < total;
+    int64_t gc = valid ? g : total - 1;
+    int64_t row = gc / groups_per_row, col = (gc - row * groups_per_row) * 8;
+    float w[8];
+    load8(W, w_dtype, row * ldw + col, w);
+    float amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[i]));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));   // partner holds the other half-block
+    const uint32_t sb = faar_float_to_e4m3(__fdiv_rn(amax, d));
+    const float s = __fmul_rn(faar_e4m3_to_float(sb), s_global);
+    uint32_t cw = 0;
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float wt = s > 0.f ? __fdiv_rn(fabsf(w[i]), s) : 0.f;
+      wt = fminf(wt, 6.0f);
+      int k = (wt >= 0.5f) + (wt >= 1.0f) + (wt >= 1.5f) + (wt >= 2.0f) + (wt >= 3.0f) + (wt >= 4.0f);
+      float lo = faar_node(k);
+      float inv_w = k < 4 ? 2.0f : (k < 6 ? 1.0f : 0.5f);
+      v[i] = __fmul_rn(__fsub_rn(wt, lo), inv_w);
+      uint32_t neg = (w[i] < 0.f) ? 8u : 0u;
+      cw |= ((uint32_t)k | neg) << (4 * i);
+    }
+    if (valid) {
+      int64_t e = row * (int64_t)K + col;
+      float4* vp = reinterpret_cast<float4*>(V + e);
+      vp[0] = make_float4(v[0], v[1], v[2], v[3]);
+      vp[1] = make_float4(v[4], v[5], v[6], v[7]);
+      *reinterpret_cast<uint32_t*>(code + e / 2) = cw;
+      if ((col & 8) == 0) scales[e / 16] = (uint8_t)sb;
+    }
+  }
+}
+
+// ---- Eq. 2 / Eq. 3 in FP32 (parity view) -----------------------------------------
+// The argument beta*(v-0.5) is formed as an unevaluated sum hi + lo so that the
+// relative error of h stays near one ulp even where h is tiny.
+__device__ __forceinline__ float sigmoid_precise(float beta, float v) {
+  float p = __fmul_rn(beta, v);
+  float pe = __fmaf_rn(beta, v, -p);          // exact error of the product
+  float c = 0.5f * beta;                      // exact
+  float hi = __fsub_rn(p, c);
+  float bb = __fsub_rn(hi, p);                // two-sum of p + (-c)
+  float lo = __fadd_rn(__fsub_rn(p, __fsub_rn(hi, bb)), __fsub_rn(-c, bb));
+  lo = __fadd_rn(lo, pe);
+  // h = 1 / (1 + exp(-(hi+lo)));  exp(-(hi+lo)) = exp(-hi) * (1 - lo + ...)
+  float e = expf(-fabsf(hi));
+  float adj = hi >= 0.f ? -lo : lo;           // exp(-|hi| - sign*lo)
+  e = __fmaf_rn(e, adj, e);
+  float hs = __fdiv_rn(1.0f, 1.0f + e);       // sigmoid(|z|)
+  return hi >= 0.f ? hs : __fmul_rn(e, hs);   // sigmoid(-|z|) = e / (1 + e)
+}
+
+__global__ void __launch_bounds__(EW_THREADS)
+softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code,
+                      const uint8_t* __restrict__ scales, const float* __restrict__ s_global_p,
+                      float beta, int64_t n_groups, float* __restrict__ W_soft, float* __restrict__ H) {
+  const float s_global = *s_global_p;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups;
+       g += (int64_t)gridDim.x * blockDim.x) {
+    int64_t e = g * 8;
+    const float4* vp = reinterpret_cast<const float4*>(V + e);
+    float4 a = vp[0], b = vp[1];
+    float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t cw = *reinterpret_cast<const uint32_t*>(code + e / 2);
+    float s = __fmul_rn(faar_e4m3_to_float(scales[e / 16]), s_global);
+    float ws[8], h[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t nib = (cw >> (4 * i)) & 0xF;
+      int k = nib & 7;
+      h[i] = sigmoid_precise(beta, v[i]);
+      float mag = __fmul_rn(__fmaf_rn(h[i], faar_width(k), faar_node(k)), s);
+      ws[i] = (nib & 8) ? -mag : mag;
+    }
+    if (W_soft) {
+      float4* p = reinterpret_cast<float4*>(W_soft + e);
+      p[0] = make_float4(ws[0], ws[1], ws[2], ws[3]);
+      p[1] = make_float4(ws[4], ws[5], ws[6], ws[7]);
+    }
+    if (H) {
+      float4* p = reinterpret_cast<float4*>(H + e);
+      p[0] = make_float4(h[0], h[1], h[2], h[3]);
+      p[1] = make_float4(h[4], h[5], h[6], h[7]);
+    }
+  }
+}
+
+// ---- Eq. 2 / Eq. 3 -> BF16 GEMM operand ---------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+softquant_bf16_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code,
+                      const uint8_t* __restrict__ scales, const float* __restrict__ s_global_p,
+                      float beta, int64_t n_groups, __nv_bfloat16* __restrict__ W_soft) {
+  const float s_global = *s_global_p;
+  const float nhb = -0.5f * beta;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups;
+       g += (int64_t)gridDim.x * blockDim.x) {
+    int64_t e = g * 8;
+    const float4* vp = reinterpret_cast<const float4*>(V + e);
+    float4 a = vp[0], b = vp[1];
+    float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t cw = *reinterpret_cast<const uint32_t*>(code + e / 2);
+    float s = __fmul_rn(faar_e4m3_to_float(scales[e / 16]), s_global);
+    uint32_t out[4];
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+      float r[2];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        uint32_t nib = (cw >> (4 * (i + j))) & 0xF;
+        int k = nib & 7;
+        float z = fmaf(beta, v[i + j], nhb);
+        float ex = __expf(-fabsf(z));
+        float hs = __fdividef(1.0f, 1.0f + ex);
+        float h = z >= 0.f ? hs : ex * hs;
+        float mag = fmaf(h, faar_width(k), faar_node(k)) * s;
+        r[j] = (nib & 8) ? -mag : mag;
+      }
+      __nv_bfloat162 p = __floats2bfloat162_rn(r[0], r[1]);
+      out[i / 2] = *reinterpret_cast<uint32_t*>(&p);
+    }
+    *reinterpret_cast<uint4*>(W_soft + e) = make_uint4(out[0], out[1], out[2], out[3]);
+  }
+}
+
+// ---- Round Loss partial sums ------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+round_partials_kernel(const float* __restrict__ V, int64_t N, float* __restrict__ partials) {
+  float acc = 0.f;
+  const int64_t n4 = N / 4;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    float4 a = reinterpret_cast<const float4*>(V)[i];
+    float t0 = 2.f * a.x - 1.f, t1 = 2.f * a.y - 1.f, t2 = 2.f * a.z - 1.f, t3 = 2.f * a.w - 1.f;
+    acc += (1.f - t0 * t0) + (1.f - t1 * t1) + (1.f - t2 * t2) + (1.f - t3 * t3);
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (int)(N - n4 * 4)) {
+    float t = 2.f * V[n4 * 4 + threadIdx.x] - 1.f;
+    acc += 1.f - t * t;
+  }
+  acc = faar_warp_sum(acc);
+  __shared__ float s_sum[EW_THREADS / 32];
+  if ((threadIdx.x & 31) == 0) s_sum[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < EW_THREADS / 32; ++i) t += s_sum[i];
+    partials[blockIdx.x] = t;
+  }
+}
+
+// Fixed-order final sums (one block; double accumulation).
+__global__ void __launch_bounds__(256)
+finalize_kernel(const float* __restrict__ p0, int n0, float scale0, float* out0,
+                const float* __restrict__ p1, int n1, float scale1, float* out1) {
+  __shared__ double sh[256];
+  for (int which = 0; which < 2; ++which) {
+    const float* p = which ? p1 : p0;
+    int n = which ? n1 : n0;
+    float* out = which ? out1 : out0;
+    if (n <= 0 || out == nullptr) continue;
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n; i += 256) acc += (double)p[i];
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) {
+      if (threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = (float)(sh[0] * (double)(which ? scale1 : scale0));
+    __syncthreads();
+  }
+}
+
+// ---- Eq. 7: harden + pack ---------------------------------------------------------------
+__global__ void __launch_bounds__(EW_THREADS)
+harden_pack_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code,
+                   const uint8_t* __restrict__ scales, const float* __restrict__ s_global_p,
+                   int64_t n_groups, uint8_t* __restrict__ packed, uint8_t* __restrict__ scales_out,
+                   uint8_t* __restrict__ decisions, void* __restrict__ W_final, int wfinal_dtype) {
+  const float s_global = W_final ? *s_global_p : 0.f;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups;
+       g += (int64_t)gridDim.x * blockDim.x) {
+    int64_t e = g * 8;
+    const float4* vp = reinterpret_cast<const float4*>(V + e);
+    float4 a = vp[0], b = vp[1];
+    float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t cw = *reinterpret_cast<const uint32_t*>(code + e / 2);
+    uint32_t dec = 0, add = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t up = v[i] >= 0.5f ? 1u : 0u;
+      dec |= up << i;
+      add |= up << (4 * i);
+    }
+    uint32_t pw = cw + add;      // k <= 6, so k + 1 never carries into the sign bit
+    *reinterpret_cast<uint32_t*>(packed + e / 2) = pw;
+    if (decisions) decisions[g] = (uint8_t)dec;
+    if (scales_out && (g & 1) == 0) scales_out[e / 16] = scales[e / 16];
+    if (W_final) {
+      float s = __fmul_rn(faar_e4m3_to_float(scales[e / 16]), s_global);
+      float wf[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        uint32_t nib = (pw >> (4 * i)) & 0xF;
+        float mag = __fmul_rn(faar_node(nib & 7), s);
+        wf[i] = (nib & 8) ? -mag : mag;
+      }
+      if (wfinal_dtype == FAAR_F32) {
+        float4* p = reinterpret_cast<float4*>(reinterpret_cast<float*>(W_final) + e);
+        p[0] = make_float4(wf[0], wf[1], wf[2], wf[3]);
+        p[1] = make_float4(wf[4], wf[5], wf[6], wf[7]);
+      } else {
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          __nv_bfloat162 p2 = __floats2bfloat162_rn(wf[2 * i], wf[2 * i + 1]);
+          o[i] = *reinterpret_cast<uint32_t*>(&p2);
+        }
+        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(W_final) + e) = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+    }
+  }
+}
+
+// ---- BF16 transpose through shared memory -----------------------------------------------
+__global__ void __launch_bounds__(256)
+transpose_bf16_kernel(const uint16_t* __restrict__ in, int rows, int cols, int64_t ld_in,
+                      uint16_t* __restrict__ out, int64_t ld_out) {
+  __shared__ uint16_t tile[64][66];
+  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;   // 64 x 4
+  for (int i = ty; i < 64; i += 4) {
+    int r = r0 + i, c = c0 + tx;
+    tile[i][tx] = (r < rows && c < cols) ? in[(int64_t)r * ld_in + c] : (uint16_t)0;
+  }
+  __syncthreads();
+  for (int i = ty; i < 64; i += 4) {
+    int c = c0 + i, r = r0 + tx;
+    if (c < cols && r < rows) out[(int64_t)c * ld_out + r] = tile[tx][i];
+  }
+}
+
+int grid_for(const faar_ctx* ctx, int64_t work_items, int per_sm) {
+  int64_t blocks = (work_items + EW_THREADS - 1) / EW_THREADS;
+  int64_t cap = (int64_t)ctx->num_sms * per_sm;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+}  // namespace
+
+int faar_launch_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float s_global_in,
+                               uint8_t* scales, float* s_global_out, uint8_t* code, float* V,
+                               uint32_t* amax_word) {
+  const int64_t groups = (int64_t)s->O * (s->K / 8);
+  const int grid = grid_for(ctx, groups, 8);
+  if (!(s_global_in > 0.f)) {
+    cudaError_t e = cudaMemsetAsync(amax_word, 0, sizeof(uint32_t), ctx->stream);
+    if (e != cudaSuccess) return (int)e;
+    amax_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, amax_word);
+  }
+  softquant_init_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, s_global_in,
+                                                               amax_word, scales, s_global_out, code, V);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_softquant_eval(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
+                               const uint8_t* scales, const float* s_global, float beta, float* W_soft,
+                               float* h) {
+  const int64_t groups = (int64_t)s->O * (s->K / 8);
+  softquant_eval_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(V, code, scales, s_global, beta,
+                                                                                  groups, W_soft, h);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_softquant_bf16(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
+                               const uint8_t* scales, const float* s_global, float beta,
+                               __nv_bfloat16* W_soft) {
+  const int64_t groups = (int64_t)s->O * (s->K / 8);
+  softquant_bf16_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(V, code, scales, s_global, beta,
+                                                                                  groups, W_soft);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in, int64_t ld_in, void* out,
+                               int64_t ld_out) {
+  dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+  transpose_bf16_kernel<<<grid, 256, 0, ctx->stream>>>(reinterpret_cast<const uint16_t*>(in), rows, cols, ld_in,
+                                                       reinterpret_cast<uint16_t*>(out), ld_out);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_round_partials(faar_ctx* ctx, const float* V, int64_t N, float* partials, int* n_partials) {
+  int grid = grid_for(ctx, (N + 3) / 4, 4);
+  if (grid > FAAR_MAX_PARTIALS) grid = FAAR_MAX_PARTIALS;
+  round_partials_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(V, N, partials);
+  *n_partials = grid;
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_finalize(faar_ctx* ctx, const float* p0, int n0, float scale0, float* out0, const float* p1,
+                         int n1, float scale1, float* out1) {
+  finalize_kernel<<<1, 256, 0, ctx->stream>>>(p0, n0, scale0, out0, p1, n1, scale1, out1);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_harden_pack(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
+                            const uint8_t* scales, const float* s_global, uint8_t* packed,
+                            uint8_t* scales_out, uint8_t* decisions, void* W_final, int wfinal_dtype) {
+  const int64_t groups = (int64_t)s->O * (s->K / 8);
+  harden_pack_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(
+      V, code, scales, s_global, groups, packed, scales_out, decisions, W_final, wfinal_dtype);
+  return (int)cudaGetLastError();
+}

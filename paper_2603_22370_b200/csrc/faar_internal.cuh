@@ -1,0 +1,138 @@
+// Internal declarations shared by the translation units of libfaar.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "faar.h"
+
+struct faar_ctx {
+  int device;
+  int num_sms;
+  cudaStream_t stream;
+  int last_cuda_error;
+  void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+// ---- workspace layout -------------------------------------------------------
+// [0, 256)            header: word 0 = status (0 = ok), word 1 = |W| max bits
+// [256, 256+P)        loss partials (float): MSE region then Round region
+// [..]                W_soft bf16 [O,K]
+// [..]                dYt bf16 [O, ceil8(T)]
+constexpr size_t FAAR_WS_HEADER = 256;
+constexpr int FAAR_MAX_PARTIALS = 16384;  // per loss term
+
+struct faar_ws_layout {
+  size_t off_mse_partials, off_round_partials, off_wsoft, off_dyt, total;
+  int64_t ld_dyt;
+};
+
+static inline size_t faar_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static inline faar_ws_layout faar_ws_plan(const faar_shape* s) {
+  faar_ws_layout l;
+  l.ld_dyt = ((int64_t)s->T + 7) / 8 * 8;
+  size_t off = FAAR_WS_HEADER;
+  l.off_mse_partials = off;
+  off += sizeof(float) * FAAR_MAX_PARTIALS;
+  l.off_round_partials = off;
+  off += sizeof(float) * FAAR_MAX_PARTIALS;
+  off = faar_align_up(off, 1024);
+  l.off_wsoft = off;
+  off += (size_t)s->O * (size_t)s->K * 2;
+  off = faar_align_up(off, 1024);
+  l.off_dyt = off;
+  off += (size_t)s->O * (size_t)l.ld_dyt * 2;
+  l.total = faar_align_up(off, 1024);
+  return l;
+}
+
+// ---- launchers (each returns a cudaError_t as int) ---------------------------
+int faar_launch_softquant_init(faar_ctx*, const faar_shape*, const void* W, float s_global_in,
+                               uint8_t* scales, float* s_global_out, uint8_t* code, float* V,
+                               uint32_t* amax_word);
+int faar_launch_softquant_eval(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
+                               const uint8_t* scales, const float* s_global, float beta,
+                               float* W_soft, float* h);
+int faar_launch_softquant_bf16(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
+                               const uint8_t* scales, const float* s_global, float beta,
+                               __nv_bfloat16* W_soft);
+int faar_launch_transpose_bf16(faar_ctx*, int rows, int cols, const void* in, int64_t ld_in, void* out,
+                               int64_t ld_out);
+int faar_launch_round_partials(faar_ctx*, const float* V, int64_t N, float* partials, int* n_partials);
+// out[0] = scale0 * sum(p0[0..n0)), out[1] = scale1 * sum(p1[0..n1)) (either may have n = 0 -> skipped)
+int faar_launch_finalize(faar_ctx*, const float* p0, int n0, float scale0, float* out0, const float* p1,
+                         int n1, float scale1, float* out1);
+int faar_launch_harden_pack(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
+                            const uint8_t* scales, const float* s_global, uint8_t* packed,
+                            uint8_t* scales_out, uint8_t* decisions, void* W_final, int wfinal_dtype);
+
+enum { FAAR_GEMM_REF = 0, FAAR_GEMM_FWD = 1, FAAR_GEMM_BWD = 2 };
+
+struct faar_gemm_args {
+  int mode;
+  int M, N, Kc;           // C[M,N] = A[M,Kc] * B[N,Kc]^T, both operands bf16 with Kc contiguous
+  const void* A; int64_t lda;
+  const void* B; int64_t ldb;
+  uint32_t* status;       // workspace status word
+  // REF / FWD
+  void* Yout; int yout_dtype; int64_t ldy;     // [N(T), M(O)] written transposed; nullable in FWD
+  const void* Yref; int yref_dtype;            // FWD
+  __nv_bfloat16* dYt; int64_t ld_dyt;          // FWD: [M(O), ld_dyt]
+  float mse2c;                                 // FWD: 2 * mse_scale
+  float* partials;                             // FWD: sum r^2 partials; BWD: Round Loss partials
+  // BWD: M = O, N = K
+  float* V; const uint8_t* code; const uint8_t* scales; const float* s_global;
+  float* adam_m; float* adam_u; float* dV;
+  float beta, lam_over_n, lr, b1, b2, eps, inv_bc1, inv_bc2; int opt;
+};
+// n_partials_out: number of floats written to args.partials
+int faar_launch_gemm(faar_ctx*, const faar_gemm_args*, int* n_partials_out);
+int faar_gemm_max_partials(const faar_ctx*, int M, int N);
+
+// ---- device helpers -----------------------------------------------------------
+#ifdef __CUDACC__
+
+// E2M1 magnitude of code c (0..7): 0, .5, 1, 1.5, 2, 3, 4, 6.
+__device__ __forceinline__ float faar_node(int c) {
+  int e = c >> 1, m = c & 1;
+  // e == 0: m * 0.5 ; else (1 + m/2) * 2^(e-1)
+  float normal = __uint_as_float(((uint32_t)(e + 126) << 23) | ((uint32_t)m << 22));
+  return e == 0 ? 0.5f * (float)m : normal;
+}
+
+// width of interval k (0..6): .5 .5 .5 .5 1 1 2
+__device__ __forceinline__ float faar_width(int k) { return k < 4 ? 0.5f : (k < 6 ? 1.0f : 2.0f); }
+
+// FP8 E4M3 byte -> float (finite codes only).
+__device__ __forceinline__ float faar_e4m3_to_float(uint32_t b) {
+  uint32_t e = (b >> 3) & 0xF, m = b & 7;
+  float sub = (float)m * 0.001953125f;  // m * 2^-9
+  float nor = __uint_as_float(((e + 120u) << 23) | (m << 20));
+  return e == 0 ? sub : nor;
+}
+
+// Non-negative finite float -> nearest finite E4M3 byte, ties to even, saturating at 448.
+__device__ __forceinline__ uint32_t faar_float_to_e4m3(float q) {
+  if (!(q < 448.0f)) return 0x7Eu;
+  if (q < 0.015625f) {                       // below 2^-6: fixed quantum 2^-9
+    return (uint32_t)__float2int_rn(q * 512.0f);   // 0..8; 8 is the smallest normal
+  }
+  uint32_t bits = __float_as_uint(q);
+  uint32_t lsb = (bits >> 20) & 1u;
+  bits += 0x7FFFFu + lsb;                    // round to nearest even at bit 20
+  bits &= 0xFFF00000u;
+  if (bits > 0x43E00000u) return 0x7Eu;      // above 448
+  uint32_t e = (bits >> 23) - 120u;
+  uint32_t m = (bits >> 20) & 7u;
+  return (e << 3) | m;
+}
+
+__device__ __forceinline__ float faar_warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+#endif  // __CUDACC__

@@ -1,0 +1,189 @@
+"""ctypes binding of libfaar.so.  Argument marshalling only: every function
+below has the name and the arguments of the C entry point it calls; tensors
+are torch CUDA tensors whose `data_ptr()` is handed through.  There is no
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfaar.so")
+
+OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(9)
+BF16, F32 = 0, 1
+
+EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string", "faar_last_cuda_error",
+           "faar_workspace_size", "faar_workspace_init", "faar_check_status", "faar_softquant_init",
+           "faar_softquant_eval", "faar_transpose_bf16", "faar_layer_ref", "faar_layer_fwd", "faar_round_loss",
+           "faar_layer_bwd", "faar_layer_step", "faar_harden_pack"]
+
+
+class HParams(C.Structure):
+    _fields_ = [("beta", C.c_float), ("lambda_round", C.c_float), ("mse_scale", C.c_float), ("opt", C.c_int),
+                ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("step", C.c_int)]
+
+
+class Shape(C.Structure):
+    _fields_ = [("O", C.c_int), ("K", C.c_int), ("T", C.c_int), ("ldw", C.c_int64), ("ldx", C.c_int64),
+                ("ldxt", C.c_int64), ("ldy", C.c_int64), ("w_dtype", C.c_int), ("yref_dtype", C.c_int)]
+
+
+class FaarError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libfaar.so (built in-tree by `paper_2603_22370_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} is missing; run `python -m paper_2603_22370_b200.build`")
+        l = C.CDLL(LIB_PATH)
+        for name in EXPORTS:
+            getattr(l, name).restype = C.c_int
+        l.faar_status_string.restype = C.c_char_p
+        l.faar_status_string.argtypes = [C.c_int]
+        _lib = l
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().faar_status_string(int(status)).decode()
+
+
+def _p(t):
+    if t is None:
+        return C.c_void_p(0)
+    if isinstance(t, int):
+        return C.c_void_p(t)
+    assert t.is_cuda, "device tensors only"
+    return C.c_void_p(t.data_ptr())
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise FaarError(status, where)
+
+
+def make_shape(O, K, T, ldw=None, ldx=None, ldxt=None, ldy=None, w_dtype=BF16, yref_dtype=BF16) -> Shape:
+    return Shape(O, K, T, ldw if ldw is not None else K, ldx if ldx is not None else K,
+                 ldxt if ldxt is not None else (T + 7) // 8 * 8, ldy if ldy is not None else O, w_dtype, yref_dtype)
+
+
+def make_hparams(beta=4.0, lambda_round=1.0, mse_scale=1.0, opt=1, lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8,
+                 step=1) -> HParams:
+    return HParams(beta, lambda_round, mse_scale, opt, lr, beta1, beta2, eps, step)
+
+
+class Context:
+    """Owns a faar_ctx bound to a device and a stream, plus (optionally) a workspace tensor."""
+
+    def __init__(self, device: int = 0, stream: torch.cuda.Stream | None = None):
+        self._h = C.c_void_p(0)
+        self.device = device
+        s = stream.cuda_stream if stream is not None else torch.cuda.current_stream(device).cuda_stream
+        _check(lib().faar_create(C.byref(self._h), device, C.c_void_p(s)), "faar_create")
+        self.ws = None
+
+    def close(self):
+        if self._h:
+            lib().faar_destroy(self._h)
+            self._h = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_stream(self, stream: torch.cuda.Stream):
+        _check(lib().faar_set_stream(self._h, C.c_void_p(stream.cuda_stream)), "faar_set_stream")
+
+    def last_cuda_error(self) -> int:
+        return lib().faar_last_cuda_error(self._h)
+
+    def workspace(self, shape: Shape) -> torch.Tensor:
+        """Allocates (with torch) and initialises a workspace large enough for `shape`."""
+        n = workspace_size(shape)
+        if self.ws is None or self.ws.numel() < n:
+            self.ws = torch.empty(n, dtype=torch.uint8, device=f"cuda:{self.device}")
+            workspace_init(self, self.ws)
+        return self.ws
+
+
+def workspace_size(shape: Shape) -> int:
+    n = C.c_size_t(0)
+    _check(lib().faar_workspace_size(C.byref(shape), C.byref(n)), "faar_workspace_size")
+    return n.value
+
+
+def workspace_init(ctx: Context, ws: torch.Tensor):
+    _check(lib().faar_workspace_init(ctx._h, _p(ws), C.c_size_t(ws.numel())), "faar_workspace_init")
+
+
+def check_status(ctx: Context, ws: torch.Tensor) -> int:
+    d = C.c_uint32(0)
+    st = lib().faar_check_status(ctx._h, _p(ws), C.byref(d))
+    if st != OK:
+        raise FaarError(st, f"faar_check_status (detail 0x{d.value:x})")
+    return st
+
+
+def softquant_init(ctx, shape, W, s_global_in, scales, s_global_out, code, V_init, ws):
+    _check(lib().faar_softquant_init(ctx._h, C.byref(shape), _p(W), C.c_float(s_global_in), _p(scales),
+                                     _p(s_global_out), _p(code), _p(V_init), _p(ws), C.c_size_t(ws.numel())),
+           "faar_softquant_init")
+
+
+def softquant_eval(ctx, shape, V, code, scales, s_global, beta, W_soft, h):
+    _check(lib().faar_softquant_eval(ctx._h, C.byref(shape), _p(V), _p(code), _p(scales), _p(s_global),
+                                     C.c_float(beta), _p(W_soft), _p(h)), "faar_softquant_eval")
+
+
+def transpose_bf16(ctx, rows, cols, inp, ld_in, out, ld_out):
+    _check(lib().faar_transpose_bf16(ctx._h, rows, cols, _p(inp), C.c_int64(ld_in), _p(out), C.c_int64(ld_out)),
+           "faar_transpose_bf16")
+
+
+def layer_ref(ctx, shape, X, W, Y_ref, ws):
+    _check(lib().faar_layer_ref(ctx._h, C.byref(shape), _p(X), _p(W), _p(Y_ref), _p(ws), C.c_size_t(ws.numel())),
+           "faar_layer_ref")
+
+
+def layer_fwd(ctx, shape, hp, X, Y_ref, V, code, scales, s_global, dYt, loss_mse, Y_q, ws):
+    _check(lib().faar_layer_fwd(ctx._h, C.byref(shape), C.byref(hp), _p(X), _p(Y_ref), _p(V), _p(code), _p(scales),
+                                _p(s_global), _p(dYt), _p(loss_mse), _p(Y_q), _p(ws), C.c_size_t(ws.numel())),
+           "faar_layer_fwd")
+
+
+def round_loss(ctx, V, N, loss_round, ws):
+    _check(lib().faar_round_loss(ctx._h, _p(V), C.c_int64(N), _p(loss_round), _p(ws), C.c_size_t(ws.numel())),
+           "faar_round_loss")
+
+
+def layer_bwd(ctx, shape, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, dV, ws):
+    _check(lib().faar_layer_bwd(ctx._h, C.byref(shape), C.byref(hp), _p(dYt), _p(Xt), _p(V), _p(code), _p(scales),
+                                _p(s_global), _p(adam_m), _p(adam_u), _p(dV), _p(ws), C.c_size_t(ws.numel())),
+           "faar_layer_bwd")
+
+
+def layer_step(ctx, shape, hp, X, Xt, Y_ref, V, code, scales, s_global, adam_m, adam_u, loss_out2, ws):
+    _check(lib().faar_layer_step(ctx._h, C.byref(shape), C.byref(hp), _p(X), _p(Xt), _p(Y_ref), _p(V), _p(code),
+                                 _p(scales), _p(s_global), _p(adam_m), _p(adam_u), _p(loss_out2), _p(ws),
+                                 C.c_size_t(ws.numel())), "faar_layer_step")
+
+
+def harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, decisions, W_final, wfinal_dtype=F32):
+    _check(lib().faar_harden_pack(ctx._h, C.byref(shape), _p(V), _p(code), _p(scales), _p(s_global), _p(packed),
+                                  _p(scales_out), _p(decisions), _p(W_final), C.c_int(wfinal_dtype)),
+           "faar_harden_pack")

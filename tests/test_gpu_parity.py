@@ -1,0 +1,401 @@
+"""GPU parity: every entry point of libfaar.so, called through the C ABI, against
+the CPU oracle on the same seeded inputs.
+
+Tolerances (from the build's target statement):
+  * bytes (E4M3 scales, lower-node codes, hardened nibbles, decisions): bit-exact;
+  * V_init: bit-exact (binary32 contract);
+  * W_soft, h in FP32: |gpu - oracle| <= 1e-6 * |oracle|;
+  * loss: relative 2e-3; dV, updated V: ||gpu - oracle||_2 <= 2e-3 ||oracle||_2 and
+    max|gpu - oracle| <= 2e-3 max|oracle| (element-wise relative error is not defined
+    where the dW dot product cancels to ~0);
+  * the optimiser arithmetic alone (oracle update applied to the GPU's own dV): 3e-7
+    absolute on V, 2e-6 relative on the Adam moments.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import faar_oracle as fo
+from paper_2603_22370_b200 import faar, inputs
+from tests.gpu_helpers import DEV, GpuLayer, dev_bf16, dev_f32, dev_u8, host, max_rel_to_peak, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2603_22370_b200 import build
+    build.build()
+    c = faar.Context(0)
+    yield c
+    torch.cuda.synchronize()
+    c.close()
+
+
+def f32hp(**kw):
+    """Hyper-parameters as the binary32 values the library receives, for both sides."""
+    d = dict(beta=4.0, lambda_round=1.0, mse_scale=1.0, opt=1, lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, step=1)
+    d.update(kw)
+    for k in ("beta", "lambda_round", "mse_scale", "lr", "beta1", "beta2", "eps"):
+        d[k] = float(np.float32(d[k]))
+    return faar.make_hparams(**d), fo.HParams(**d)
+
+
+def adversarial_weights():
+    """Rows exercising exact nodes, exact ties, an all-zero block, -0, clamping above 6,
+    the largest / smallest BF16 normals next to ordinary values, and subnormal block scales."""
+    rng = np.random.default_rng(0)
+    W = (0.02 * rng.standard_normal((16, 128))).astype(np.float32)
+    blk = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5, -6], dtype=np.float32)
+    W[0, 0:16] = blk * np.float32(2.0 ** -8)
+    W[0, 16:32] = -blk * np.float32(2.0 ** -8)
+    W[1, 0:16] = 0.0
+    W[1, 16] = -0.0
+    W[2, 0:16] = 1.0
+    W[2, 0] = 1.06
+    W[3, 0:16] = np.float32(2.0 ** -20)          # far below the tensor maximum: subnormal / zero block scale
+    W[3, 16:32] = np.float32(3e-6)
+    W[4, 0] = 8.0                                  # the tensor maximum
+    W[5, :] = np.float32(2.0 ** -126)
+    return inputs.to_bf16_f32(W)
+
+
+# ---------------------------------------------------------------------------------------------
+# part 1: soft-quantisation set-up
+# ---------------------------------------------------------------------------------------------
+
+def _check_init(ctx, W, w_dtype, s_global_in=0.0, ldw=None):
+    O, K = W.shape
+    lay = GpuLayer(ctx, W, np.zeros((8, K), np.float32), w_dtype=w_dtype)
+    if ldw is not None:
+        buf = torch.full((O, ldw), 7.0, dtype=lay.W.dtype, device=DEV)
+        buf[:, :K] = lay.W
+        lay.W = buf
+        lay.shape.ldw = ldw
+    lay.init(s_global_in)
+    lay.check()
+    scales, sg, code, V = fo.softquant_init(W, s_global_in)
+    assert host(lay.s_global)[0] == sg
+    assert np.array_equal(host(lay.scales), scales)
+    assert np.array_equal(host(lay.code), code)
+    assert np.array_equal(host(lay.V).view(np.uint32), V.view(np.uint32))
+    return lay
+
+
+def test_softquant_init_config1_fp32(ctx):
+    W, _ = inputs.config1(0)
+    _check_init(ctx, W, faar.F32)
+
+
+@pytest.mark.parametrize("O,K", [(96, 512), (1, 16), (300, 1040), (257, 48)])
+def test_softquant_init_bf16_shapes(ctx, O, K):
+    W, _ = inputs.config2(1, O, K, 8)
+    _check_init(ctx, W, faar.BF16)
+
+
+def test_softquant_init_adversarial_values_strided_and_given_scale(ctx):
+    W = adversarial_weights()
+    _check_init(ctx, W, faar.BF16)
+    _check_init(ctx, W, faar.F32, ldw=136)
+    _check_init(ctx, W, faar.BF16, s_global_in=float(np.float32(2.0 ** -8)))
+    _check_init(ctx, np.zeros((4, 32), np.float32), faar.BF16)
+
+
+# ---------------------------------------------------------------------------------------------
+# part 2: soft weights in FP32
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("beta", [0.5, 4.0, 11.3, 32.0])
+def test_softquant_eval_matches_eq2_eq3(ctx, beta):
+    W, _ = inputs.config1(2, 64, 256, 8)
+    lay = _check_init(ctx, W, faar.F32)
+    rng = np.random.default_rng(0)
+    V = rng.uniform(0, 1, W.shape).astype(np.float32)
+    V[0, :8] = [0, 1, 0.5, 0.25, 0.75, 1e-3, 0.999, 0.5000001]
+    lay.set_state(V=V)
+    Ws = torch.empty_like(lay.V)
+    H = torch.empty_like(lay.V)
+    b = float(np.float32(beta))
+    faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, b, Ws, H)
+    lay.check()
+    Wo, Ho = fo.soft_weights(V, host(lay.code), host(lay.scales), host(lay.s_global)[0], b)
+    assert np.all(np.abs(host(H) - Ho) <= 1e-6 * np.abs(Ho))
+    assert np.all(np.abs(host(Ws) - Wo) <= 1e-6 * np.abs(Wo) + 1e-38)
+    # each output alone
+    H2 = torch.empty_like(lay.V)
+    faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, b, None, H2)
+    assert torch.equal(H, H2)
+
+
+def test_softquant_eval_saturates_to_floor_and_ceil(ctx):
+    W, _ = inputs.config1(3, 32, 64, 8)
+    lay = _check_init(ctx, W, faar.F32)
+    k, neg = fo.unpack_code(host(lay.code))
+    s = np.repeat(fo.effective_scale(host(lay.scales), host(lay.s_global)[0]), 16, axis=1)
+    sgn = np.where(neg, -1.0, 1.0).astype(np.float32)
+    Ws = torch.empty_like(lay.V)
+    H = torch.empty_like(lay.V)
+    for fill, node in ((0.0, fo.NODES[k]), (1.0, fo.NODES[k + 1])):
+        lay.V.fill_(fill)
+        faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, 1e4, Ws, H)
+        assert np.array_equal(host(H), np.full(W.shape, fill, np.float32))
+        assert np.array_equal(host(Ws), sgn * (node.astype(np.float32) * s))
+    lay.check()
+
+
+# ---------------------------------------------------------------------------------------------
+# Round Loss, harden + pack, transpose
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n", [16, 1000003, 4 * 1024 * 1024])
+def test_round_loss(ctx, n):
+    rng = np.random.default_rng(n)
+    V = rng.uniform(0, 1, n).astype(np.float32)
+    lay_shape = faar.make_shape(16, 16, 8)
+    ws = ctx.workspace(lay_shape)
+    out = torch.zeros(1, device=DEV)
+    faar.round_loss(ctx, dev_f32(V), n, out, ws)
+    torch.cuda.synchronize()
+    ref = fo.round_loss(V)
+    assert abs(host(out)[0] - ref) <= 1e-5 * ref
+
+
+def test_harden_pack_bit_exact(ctx):
+    W = adversarial_weights()
+    lay = _check_init(ctx, W, faar.BF16)
+    rng = np.random.default_rng(1)
+    for V in (host(lay.V), rng.uniform(0, 1, W.shape).astype(np.float32), np.zeros(W.shape, np.float32),
+              np.ones(W.shape, np.float32), np.full(W.shape, 0.5, np.float32),
+              np.full(W.shape, np.nextafter(np.float32(0.5), np.float32(0)), np.float32)):
+        lay.set_state(V=V)
+        O, K = W.shape
+        packed = torch.zeros((O, K // 2), dtype=torch.uint8, device=DEV)
+        sc_out = torch.zeros((O, K // 16), dtype=torch.uint8, device=DEV)
+        dec = torch.zeros((O, K // 8), dtype=torch.uint8, device=DEV)
+        Wf = torch.zeros((O, K), dtype=torch.float32, device=DEV)
+        Wfb = torch.zeros((O, K), dtype=torch.bfloat16, device=DEV)
+        faar.harden_pack(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, packed, sc_out, dec, Wf, faar.F32)
+        faar.harden_pack(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, packed, None, None, Wfb, faar.BF16)
+        lay.check()
+        p_o, vh_o, Wf_o = fo.harden_pack(V, host(lay.code), host(lay.scales), host(lay.s_global)[0])
+        assert np.array_equal(host(packed), p_o)
+        assert np.array_equal(host(dec), fo.pack_decisions(vh_o))
+        assert np.array_equal(host(sc_out), host(lay.scales))
+        assert np.array_equal(host(Wf).view(np.uint32), Wf_o.view(np.uint32))
+        assert np.array_equal(host(Wfb), inputs.to_bf16_f32(Wf_o))
+        assert np.array_equal(fo.dequant_packed(host(packed), host(sc_out), host(lay.s_global)[0]).view(np.uint32),
+                              host(Wf).view(np.uint32))
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 1), (77, 130), (600, 1040)])
+def test_transpose(ctx, rows, cols):
+    rng = np.random.default_rng(0)
+    a = dev_bf16(rng.standard_normal((rows, cols)))
+    ld = (rows + 7) // 8 * 8
+    out = torch.zeros((cols, ld), dtype=torch.bfloat16, device=DEV)
+    faar.transpose_bf16(ctx, rows, cols, a, cols, out, ld)
+    torch.cuda.synchronize()
+    assert torch.equal(out[:, :rows], a.t())
+
+
+# ---------------------------------------------------------------------------------------------
+# parts 3-4: GEMM kernels
+# ---------------------------------------------------------------------------------------------
+
+# (O, K, T): one tile; ragged in every dimension over several 128-wide tiles; enough 256-wide
+# tiles to take the wide-tile path in the forward (O x T) and in the backward (O x K) GEMM.
+GEMM_SHAPES = [(128, 256, 1024), (100, 80, 77), (300, 1040, 600), (1500, 272, 3300), (1500, 3344, 200)]
+
+
+def _problem(O, K, T, seed=0):
+    W, X = inputs.config2(seed, O, K, T)
+    Yref = inputs.to_bf16_f32(fo.layer_ref(X, W))
+    return W, X, Yref
+
+
+@pytest.mark.parametrize("O,K,T", GEMM_SHAPES)
+@pytest.mark.parametrize("yref_dtype", [faar.BF16, faar.F32])
+def test_layer_ref(ctx, O, K, T, yref_dtype):
+    if yref_dtype == faar.F32 and (O, K, T) != GEMM_SHAPES[2]:
+        pytest.skip("FP32 output covered on one shape")
+    W, X = inputs.config2(0, O, K, T)
+    lay = GpuLayer(ctx, W, X, yref_dtype=yref_dtype)
+    Y = torch.zeros((T, O), dtype=torch.bfloat16 if yref_dtype == faar.BF16 else torch.float32, device=DEV)
+    faar.layer_ref(ctx, lay.shape, lay.X, lay.W, Y, lay.ws)
+    lay.check()
+    ref = fo.layer_ref(X, W)
+    tol = 2.0 ** -8 if yref_dtype == faar.BF16 else 1e-5
+    assert np.all(np.abs(host(Y) - ref) <= tol * np.abs(ref) + 1e-5 * np.abs(ref).max())
+
+
+@pytest.mark.parametrize("O,K,T", GEMM_SHAPES)
+def test_layer_fwd(ctx, O, K, T):
+    W, X, Yref = _problem(O, K, T)
+    lay = GpuLayer(ctx, W, X)
+    lay.init()
+    lay.set_yref(Yref)
+    rng = np.random.default_rng(1)
+    V = rng.uniform(0, 1, W.shape).astype(np.float32)
+    lay.set_state(V=V)
+    hp, hpo = f32hp(beta=7.0, mse_scale=0.5)
+    Yq = lay.fwd(hp, want_yq=True)
+    lay.check()
+    l_o, dY_o, Yq_o = fo.layer_fwd(X, Yref, V, host(lay.code), host(lay.scales), host(lay.s_global)[0],
+                                   hpo.beta, hpo.mse_scale, "bf16")
+    assert abs(host(lay.loss)[0] - l_o) <= 2e-3 * l_o
+    dY_g = host(lay.dYt)[:, :T].T
+    assert rel_l2(dY_g, dY_o) <= 2e-3 and max_rel_to_peak(dY_g, dY_o) <= 2e-3
+    assert rel_l2(host(Yq), Yq_o) <= 2e-3 and max_rel_to_peak(host(Yq), Yq_o) <= 4e-3   # BF16 output: 2^-8 rounding
+
+
+@pytest.mark.parametrize("O,K,T", GEMM_SHAPES)
+@pytest.mark.parametrize("opt", [1, 0])
+def test_layer_bwd(ctx, O, K, T, opt):
+    W, X, Yref = _problem(O, K, T)
+    lay = GpuLayer(ctx, W, X)
+    lay.init()
+    rng = np.random.default_rng(2)
+    V = rng.uniform(0, 1, W.shape).astype(np.float32)
+    m0 = (1e-2 * rng.standard_normal(W.shape)).astype(np.float32)
+    u0 = (1e-4 * rng.uniform(0, 1, W.shape)).astype(np.float32)
+    code, scales, sg = host(lay.code), host(lay.scales), host(lay.s_global)[0]
+    hp, hpo = f32hp(beta=9.0, lambda_round=3.0, opt=opt, lr=1e-2 if opt == 1 else 1e-4, step=3)
+    # the oracle's dY (already BF16) is the input of both sides
+    _, dY_o, _ = fo.layer_fwd(X, Yref, V, code, scales, sg, hpo.beta, 1.0, "bf16")
+    lay.dYt.zero_()
+    lay.dYt[:, :T] = dev_bf16(dY_o.T)
+    lay.set_state(V=V, m=m0, u=u0)
+    dV = lay.bwd(hp, want_dv=True)
+    lay.check()
+    dV_o, _ = fo.layer_grad(dY_o, X, V, code, scales, sg, hpo.beta, hpo.lambda_round)
+    dV_g = host(dV)
+    assert rel_l2(dV_g, dV_o) <= 2e-3 and max_rel_to_peak(dV_g, dV_o) <= 2e-3
+    # optimiser arithmetic, given the same gradient
+    if opt == 1:
+        Vn, mn, un = fo.adam_update(V.astype(np.float64), dV_g.astype(np.float64), m0.astype(np.float64),
+                                    u0.astype(np.float64), hpo.lr, hpo.beta1, hpo.beta2, hpo.eps, hpo.step)
+        assert np.all(np.abs(host(lay.m) - mn) <= 2e-6 * np.abs(mn) + 1e-30)
+        assert np.all(np.abs(host(lay.u) - un) <= 2e-6 * np.abs(un) + 1e-30)
+    else:
+        Vn = fo.sgd_update(V.astype(np.float64), dV_g.astype(np.float64), hpo.lr)
+        assert np.array_equal(host(lay.m), m0) and np.array_equal(host(lay.u), u0)
+    Vg = host(lay.V)
+    assert Vg.min() >= 0.0 and Vg.max() <= 1.0
+    assert np.all(np.abs(Vg - Vn) <= 3e-7)
+    # and against the oracle's own update
+    if opt == 1:
+        Vo, _, _ = fo.adam_update(V.astype(np.float64), dV_o, m0.astype(np.float64), u0.astype(np.float64),
+                                  hpo.lr, hpo.beta1, hpo.beta2, hpo.eps, hpo.step)
+    else:
+        Vo = fo.sgd_update(V.astype(np.float64), dV_o, hpo.lr)
+    assert rel_l2(Vg, Vo) <= 2e-3 and max_rel_to_peak(Vg, Vo) <= 2e-3
+    # without the optional dV output the state update is identical
+    lay.set_state(V=V, m=m0, u=u0)
+    lay.bwd(hp, want_dv=False)
+    assert np.array_equal(host(lay.V), Vg)
+
+
+@pytest.mark.parametrize("O,K,T", [(128, 256, 1024), (300, 1040, 600)])
+def test_layer_step_is_fwd_then_bwd_and_matches_oracle(ctx, O, K, T):
+    W, X, Yref = _problem(O, K, T, seed=3)
+    lay = GpuLayer(ctx, W, X)
+    lay.init()
+    lay.set_yref(Yref)
+    V0 = host(lay.V).copy()
+    hp, hpo = f32hp(beta=5.0, lambda_round=2.0, step=1)
+    lay.step(hp)
+    lay.check()
+    V_step, loss_step = host(lay.V).copy(), host(lay.loss).copy()
+    # the same through the separate calls
+    lay.set_state(V=V0, m=np.zeros_like(V0), u=np.zeros_like(V0))
+    lay.fwd(hp)
+    l_mse = host(lay.loss)[0]
+    lr_out = torch.zeros(1, device=DEV)
+    faar.round_loss(ctx, lay.V, O * K, lr_out, lay.ws)
+    lay.bwd(hp, want_dv=False)
+    lay.check()
+    assert np.array_equal(host(lay.V), V_step)
+    assert loss_step[0] == l_mse and abs(loss_step[1] - host(lr_out)[0]) <= 1e-6 * loss_step[1]
+    # oracle
+    Vo, mo, uo, l_mse_o, l_round_o, _ = fo.layer_step(X, Yref, V0, host(lay.code), host(lay.scales),
+                                                      host(lay.s_global)[0], np.zeros_like(V0), np.zeros_like(V0),
+                                                      hpo, "bf16")
+    assert abs(loss_step[0] - l_mse_o) <= 2e-3 * l_mse_o
+    assert abs(loss_step[1] - l_round_o) <= 2e-3 * l_round_o
+    # Adam's first step is -lr * sign(g): entries whose gradient is ~0 may take the other sign, so the
+    # bound on the maximum is the step size; the norm-wise bound stays 2e-3.
+    assert rel_l2(V_step, Vo) <= 2e-3 and np.max(np.abs(V_step - Vo)) <= 2.0 * hpo.lr + 1e-6
+
+
+def test_config1_trajectory_100_steps(ctx):
+    """BASELINE config 1 end to end: FP32 weights and target, BF16 GEMM operands, 100 Adam steps
+    with the geometric beta schedule, harden + pack."""
+    W, X = inputs.config1(0)
+    Xb = inputs.to_bf16_f32(X)
+    Yref = fo.layer_ref(X, W).astype(np.float32)
+    steps = 100
+    lay = GpuLayer(ctx, W, Xb, w_dtype=faar.F32, yref_dtype=faar.F32)
+    lay.init()
+    lay.set_yref(Yref)
+    scales, sg, code, V = fo.softquant_init(W)
+    assert np.array_equal(host(lay.V), V)
+    m, u = np.zeros_like(V), np.zeros_like(V)
+    hist_g, hist_o = [], []
+    for t in range(steps):
+        hp, hpo = f32hp(beta=fo.beta_schedule(t, steps), step=t + 1)
+        lay.step(hp)
+        hist_g.append(host(lay.loss).copy())
+        V, m, u, l_mse, l_round, _ = fo.layer_step(Xb, Yref, V, code, scales, sg, m, u, hpo, "bf16")
+        hist_o.append((l_mse, l_round))
+    lay.check()
+    hist_g, hist_o = np.array(hist_g, np.float64), np.array(hist_o)
+    assert np.all(np.abs(hist_g - hist_o) <= 2e-3 * hist_o)
+    Vg = host(lay.V)
+    assert rel_l2(Vg, V) <= 2e-3
+    # decisions: any disagreement must sit on the threshold in the oracle's trajectory
+    flips = fo.harden(Vg) != fo.harden(V)
+    assert flips.sum() <= 1e-4 * V.size + 1
+    assert np.all(np.abs(V[flips] - 0.5) < 5e-3)
+    # harden + pack is bit-exact on the same V
+    packed = torch.zeros((128, 128), dtype=torch.uint8, device=DEV)
+    faar.harden_pack(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, packed, None, None, None)
+    p_o, _, _ = fo.harden_pack(Vg, code, scales, sg)
+    assert np.array_equal(host(packed), p_o)
+    # the optimisation did what it is for: the soft objective fell
+    assert hist_g[-1].sum() < hist_g[0].sum()
+
+
+# ---------------------------------------------------------------------------------------------
+# argument validation on a live context
+# ---------------------------------------------------------------------------------------------
+
+def test_error_statuses(ctx):
+    import ctypes as C
+    lib = faar.lib()
+    W, X, Yref = _problem(32, 64, 16)
+    lay = GpuLayer(ctx, W, X)
+    lay.init()
+    lay.set_yref(Yref)
+    hp, _ = f32hp()
+
+    def step_status(shape=None, hp_=None, ws_bytes=None, X_=None):
+        s = shape or lay.shape
+        return lib.faar_layer_step(ctx._h, C.byref(s), C.byref(hp_ or hp), C.c_void_p((lay.X if X_ is None else X_).data_ptr()),
+                                   C.c_void_p(lay.Xt.data_ptr()), C.c_void_p(lay.Yref.data_ptr()),
+                                   C.c_void_p(lay.V.data_ptr()), C.c_void_p(lay.code.data_ptr()),
+                                   C.c_void_p(lay.scales.data_ptr()), C.c_void_p(lay.s_global.data_ptr()),
+                                   C.c_void_p(lay.m.data_ptr()), C.c_void_p(lay.u.data_ptr()),
+                                   C.c_void_p(lay.loss.data_ptr()), C.c_void_p(lay.ws.data_ptr()),
+                                   C.c_size_t(lay.ws.numel() if ws_bytes is None else ws_bytes))
+
+    assert step_status() == faar.OK
+    assert step_status(shape=faar.make_shape(32, 72, 16)) == faar.ERR_SHAPE            # K % 16
+    assert step_status(shape=faar.make_shape(32, 64, 16, ldx=60)) == faar.ERR_SHAPE    # ld < K
+    assert step_status(shape=faar.make_shape(32, 64, 16, ldx=68)) == faar.ERR_ALIGN    # ld % 8
+    assert step_status(shape=faar.make_shape(32, 64, 16, yref_dtype=5)) == faar.ERR_DTYPE
+    assert step_status(ws_bytes=1024) == faar.ERR_WORKSPACE
+    bad_hp = faar.make_hparams(beta=-1.0)
+    assert step_status(hp_=bad_hp) == faar.ERR_INVALID_ARG
+    assert step_status(hp_=faar.make_hparams(step=0)) == faar.ERR_INVALID_ARG
+    assert step_status(X_=lay.X.view(-1)[1:]) == faar.ERR_ALIGN
+    lay.check()
