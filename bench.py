@@ -1,0 +1,385 @@
+"""Benchmark of the FAAR layer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One job = the whole hot path for one linear layer of the down_proj-shaped workload
+(W 2048x8192 BF16, calibration batch X 4096x8192 BF16): soft-quantisation set-up, K optimisation
+steps (soft weights -> forward GEMM + MSE -> dW GEMM + dV + Round Loss + Adam update, beta annealed
+geometrically over the K steps), then harden + pack.  `value` = K / (device time of that job), so the
+once-per-layer kernels are inside the timed region.  With N > 1 every rank runs its own layer (layers
+are independent problems: no data-path collective), value = N*K / max-over-ranks time.
+
+`--impl reference` times the CPU oracle (numpy, float64) on the host cores instead; each of its
+steps is a row-sample of the same layer (the loss separates over output rows, so a sample of rows is
+an exact sub-problem) and the rate is scaled by rows/sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+O, K, T = 2048, 8192, 4096
+WORKLOAD = "Llama-3.2-1B-shaped down_proj: W 2048x8192 bf16 (0.02*N(0,1), 0.1% x10), X 4096x8192 bf16 " \
+           "(Student-t(4), 16 channels x20), Adam lr 1e-2, beta 4->32 geometric"
+METRIC, UNIT = "faar_layer_steps_per_s", "steps/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the
+# ncu capture summarised under profiles/; None until a capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {"gemm_bwd": None, "gemm_fwd": None}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def beta_at(t, steps, b0=4.0, b1=32.0):
+    return b0 if steps <= 1 else b0 * (b1 / b0) ** (t / (steps - 1))
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = "timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active," \
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, gpu_index: int):
+        self.lines, self.windows, self.proc = [], [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def window(self, t0, t1):
+        self.windows.append((t0, t1))
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.1)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], None, set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            if not any(a - 0.05 <= ts <= b + 0.05 for a, b in self.windows):
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 10:
+                continue
+            try:
+                sm.append(float(f[2]))
+                smax = float(f[3])
+                power.append(float(f[4]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[6:10]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power) if power else None}
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle, timed (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_rate(rows: int, steps: int, warmup: int, seed: int = 0):
+    """Runs `warmup + steps` oracle steps on a `rows`-row sample of the layer; returns
+    (full-layer steps/s, seconds per sampled step, threads used)."""
+    import numpy as np
+
+    from oracle import faar_oracle as fo
+    from paper_2603_22370_b200 import inputs
+    W, X = inputs.config2(seed, rows, K, T)
+    Yref = inputs.to_bf16_f32(fo.layer_ref(X, W))
+    scales, sg, code, V = fo.softquant_init(W)
+    m, u = np.zeros_like(V), np.zeros_like(V)
+    total = warmup + steps
+    t0 = None
+    for i in range(total):
+        if i == warmup:
+            t0 = time.perf_counter()
+        hp = fo.HParams(beta=beta_at(max(i - warmup, 0), steps), step=i + 1, lr=1e-2)
+        V, m, u, _, _, _ = fo.layer_step(X, Yref, V, code, scales, sg, m, u, hp, "bf16")
+    dt = (time.perf_counter() - t0) / steps
+    fo.harden_pack(V, code, scales, sg)
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = len(os.sched_getaffinity(0))
+    return 1.0 / (dt * (O / rows)), dt, threads
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    # size the row sample so that warmup + steps finish in about two minutes
+    probe_rows = 16
+    _, dt_probe, _ = oracle_rate(probe_rows, 1, 1)
+    budget = 120.0 / (args.steps + args.warmup)
+    rows = int(max(1, min(O, probe_rows * budget / max(dt_probe, 1e-6))))
+    rows = max(1, min(rows, 512))
+    rate, dt, threads = oracle_rate(rows, args.steps, args.warmup)
+    sample = f"each step = the {rows} first output rows of the layer (of {O}; the loss separates over rows), " \
+             f"all {T} tokens, K={K}; rate scaled by {O}/{rows}"
+    line = {"impl": "reference", "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / rate, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "O": O, "K": K, "T": T},
+            "cpu_baseline": {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": rate, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    from paper_2603_22370_b200 import build as faar_build
+    from paper_2603_22370_b200 import faar, inputs
+
+    rank, local_rank, world = dist_env()
+    n_gpus = args.gpus
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    dev = local_rank if world > 1 else 0
+    torch.cuda.set_device(dev)
+    device = f"cuda:{dev}"
+    if rank == 0:
+        faar_build.build()
+    if world > 1:
+        dist.barrier()
+    faar.lib()                                         # raises if libfaar.so is missing: no fallback
+
+    steps, warmup = args.steps, max(args.warmup, 3)
+    stream = torch.cuda.Stream(device=device)
+    ctx = faar.Context(dev, stream)
+
+    # ---- inputs, resident in HBM (each rank its own layer: seed = rank)
+    Wn, Xn = inputs.config2(rank, O, K, T)
+    W = torch.from_numpy(Wn).to(device).to(torch.bfloat16)
+    X = torch.from_numpy(Xn).to(device).to(torch.bfloat16)
+    del Wn
+    shape = faar.make_shape(O, K, T)
+    ws = torch.empty(faar.workspace_size(shape), dtype=torch.uint8, device=device)
+    Xt = torch.empty((K, T), dtype=torch.bfloat16, device=device)
+    Yref = torch.empty((T, O), dtype=torch.bfloat16, device=device)
+    scales = torch.empty((O, K // 16), dtype=torch.uint8, device=device)
+    code = torch.empty((O, K // 2), dtype=torch.uint8, device=device)
+    s_global = torch.empty(1, dtype=torch.float32, device=device)
+    V = torch.empty((O, K), dtype=torch.float32, device=device)
+    m = torch.zeros((O, K), dtype=torch.float32, device=device)
+    u = torch.zeros((O, K), dtype=torch.float32, device=device)
+    loss = torch.zeros(2, dtype=torch.float32, device=device)
+    packed = torch.empty((O, K // 2), dtype=torch.uint8, device=device)
+    scales_out = torch.empty((O, K // 16), dtype=torch.uint8, device=device)
+    torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        faar.workspace_init(ctx, ws)
+        faar.transpose_bf16(ctx, T, K, X, K, Xt, T)          # once per layer: K-major operand of the dW GEMM
+        faar.layer_ref(ctx, shape, X, W, Yref, ws)           # frozen target (Procedure step 8)
+    stream.synchronize()
+
+    def job(n_steps, step0=0):
+        """set-up, n_steps optimisation steps, harden + pack -- all enqueued on `stream`."""
+        m.zero_()
+        u.zero_()
+        faar.softquant_init(ctx, shape, W, 0.0, scales, s_global, code, V, ws)
+        for t in range(n_steps):
+            hp = faar.make_hparams(beta=beta_at(t, n_steps), step=t + 1)
+            faar.layer_step(ctx, shape, hp, X, Xt, Yref, V, code, scales, s_global, m, u, loss, ws)
+        faar.harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, None, None)
+
+    sampler = ClockSampler(dev) if rank == 0 else None
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn):
+        """device time (ms) of fn() on `stream`, max over ranks, with a barrier + sync on both sides"""
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0 = time.time()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+        stream.synchronize()
+        barrier()
+        w1 = time.time()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        if sampler:
+            sampler.window(w0, w1)
+        return ms
+
+    # ---- warm-up, then the timed job
+    with torch.cuda.stream(stream):
+        job(warmup)
+    stream.synchronize()
+    ms_job = timed(lambda: job(steps))
+    faar.check_status(ctx, ws)
+    loss_final = loss.cpu().tolist()
+    value = n_gpus * steps / (ms_job * 1e-3)
+    gpu_launches = 2 + 4 * steps + 1     # amax + init, 4 kernels per step, harden_pack
+
+    # ---- second pass of the same job with per-kernel CUDA events (library hooks, same stream)
+    def profiled():
+        faar.profile_begin(ctx)
+        job(steps)
+
+    timed(profiled)
+    prof = faar.profile_end(ctx)
+
+    # ---- end to end: the calibration batch comes from pinned host memory every step
+    Xh = torch.from_numpy(Xn).to(torch.bfloat16).pin_memory()
+    Yh = Yref.cpu().pin_memory()
+    loss_h = torch.zeros(2, dtype=torch.float32).pin_memory()
+    X_dev, Xt_dev, Y_dev = torch.empty_like(X), torch.empty_like(Xt), torch.empty_like(Yref)
+    e2e_steps = min(steps, 200)
+
+    def e2e_job(n):
+        m.zero_()
+        u.zero_()
+        faar.softquant_init(ctx, shape, W, 0.0, scales, s_global, code, V, ws)
+        for t in range(n):
+            hp = faar.make_hparams(beta=beta_at(t, n), step=t + 1)
+            faar.layer_step_host(ctx, shape, hp, Xh, Yh, X_dev, Xt_dev, Y_dev, V, code, scales, s_global, m, u,
+                                 loss, loss_h, ws)
+        faar.harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, None, None)
+
+    with torch.cuda.stream(stream):
+        e2e_job(3)
+    stream.synchronize()
+    ms_e2e = timed(lambda: e2e_job(e2e_steps))
+    e2e_value = n_gpus * e2e_steps / (ms_e2e * 1e-3)
+    faar.check_status(ctx, ws)
+    clocks = sampler.stop() if sampler else None
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- rooflines
+    pk, pk_kind = peaks()
+    n_w = O * K
+    flops = 2.0 * T * O * K
+
+    def avg_us(name):
+        return 1e3 * prof[name][1] / prof[name][0] if name in prof else None
+
+    kernels = {}
+    for name, bound, work in [
+        ("gemm_fwd", "tensor", flops), ("gemm_bwd", "tensor", flops),
+        ("soft_weights", "hbm", 6.5625 * n_w),              # V 4 + code .5 + scale 1/16 read, BF16 operand 2 written
+        ("softquant_init", "hbm", 6.5625 * n_w),            # W 2 read; V 4 + code .5 + scale 1/16 written
+        ("amax", "hbm", 2.0 * n_w),
+        ("harden_pack", "hbm", 5.125 * n_w),                # V 4 + code .5 + scale 1/16 read; .5 + 1/16 written
+    ]:
+        us = avg_us(name)
+        if us is None:
+            continue
+        if bound == "tensor":
+            ach, peak, unit = work / (us * 1e-6) / 1e12, pk["bf16_tflops_sustained"], "TFLOP/s"
+        else:
+            ach, peak, unit = work / (us * 1e-6) / 1e9, pk["hbm_gbs"], "GB/s"
+        kernels[name] = {"avg_us": round(us, 2), "launches": prof[name][0], "bound": bound, "achieved": round(ach, 1),
+                         "peak": peak, "unit": unit, "frac": round(ach / peak, 4)}
+    for name in prof:
+        if name not in kernels:
+            kernels[name] = {"avg_us": round(avg_us(name), 2), "launches": prof[name][0]}
+    dominant = max(("gemm_fwd", "gemm_bwd"), key=lambda k: prof[k][1])
+    d = kernels[dominant]
+    roofline = {"kernel": dominant, "bound": "tensor", "achieved": d["achieved"], "peak": d["peak"],
+                "unit": "TFLOP/s", "frac": d["frac"], "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+                "peak_source": f"{pk_kind} bf16_tflops_sustained (kernel timed inside a long step)",
+                "timed": "per-kernel CUDA events on the launching stream, second pass of the same K-step job"}
+
+    # ---- CPU oracle beside it (bounded sample)
+    cpu_rows, cpu_steps = 256, 8
+    cpu_rate, cpu_dt, cpu_threads = oracle_rate(cpu_rows, cpu_steps, 1)
+    cpu_baseline = {"value": cpu_rate, "unit": UNIT, "cores": cpu_threads, "kind": "oracle",
+                    "sample": f"{cpu_steps} steps on the first {cpu_rows} of {O} output rows (exact sub-problem: the "
+                              f"loss separates over rows), all {T} tokens; rate scaled by {O}/{cpu_rows}"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": n_gpus, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_job / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "O": O, "K": K, "T": T,
+                       "l2": "no flush: one step touches about 410 MB (X, X^T, V, m, u, W_soft, Y_ref, dY^T, codes), "
+                             "more than the 126 MB L2",
+                       "timed_region": "softquant_init + K x layer_step + harden_pack, inputs resident in HBM"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
+                    "h2d_bytes_per_step": T * K * 2 + T * O * 2, "d2h_bytes_per_step": 8,
+                    "path": "faar_layer_step_host: pinned X and Y_ref copied in, X^T rebuilt, step, losses copied out"},
+            "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "kernels": kernels, "final_loss": loss_final,
+            "step_tflops": round(2 * flops * steps / (ms_job * 1e-3) / 1e12, 1)}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    return run_reference(args) if args.impl == "reference" else run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

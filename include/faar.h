@@ -112,6 +112,36 @@ FAAR_API int faar_workspace_init(faar_ctx* ctx, void* workspace, size_t workspac
  * FAAR_ERR_CUDA if the stream is in error, else FAAR_OK. */
 FAAR_API int faar_check_status(faar_ctx* ctx, const void* workspace, uint32_t* detail_out);
 
+/* ---- per-kernel timing -------------------------------------------------------
+ * (No counterpart in the paper: instrumentation of this library.)
+ * Between faar_profile_begin and faar_profile_end every kernel the context
+ * launches is bracketed by a pair of CUDA events on the context's stream.
+ * faar_profile_end synchronises the stream and writes, per kernel id that ran,
+ * the number of launches and the summed device time (host array `out` of
+ * `capacity` entries; *count receives the number written).  Events are host
+ * resources; no device memory is allocated. */
+enum {
+  FAAR_K_AMAX = 0,           /* max |W| reduction (part 1, pass 1)                */
+  FAAR_K_SOFTQUANT_INIT = 1, /* scales, bracket, V_init (part 1, pass 2)          */
+  FAAR_K_SOFT_WEIGHTS = 2,   /* Eq. 2/3 -> FP32 view and/or BF16 GEMM operand     */
+  FAAR_K_GEMM_REF = 3,       /* Y_fp = X W^T                                      */
+  FAAR_K_GEMM_FWD = 4,       /* forward GEMM + residual + dY                      */
+  FAAR_K_GEMM_BWD = 5,       /* dW GEMM + dV + update                             */
+  FAAR_K_ROUND_LOSS = 6,     /* stand-alone Round Loss partial sums               */
+  FAAR_K_FINALIZE = 7,       /* fixed-order final sums of the loss partials       */
+  FAAR_K_HARDEN_PACK = 8,
+  FAAR_K_TRANSPOSE = 9,
+  FAAR_K_COUNT = 10
+};
+typedef struct {
+  int kernel;     /* one of FAAR_K_*          */
+  int launches;
+  float total_ms; /* summed over the launches */
+} faar_kernel_time;
+FAAR_API int faar_profile_begin(faar_ctx* ctx);
+FAAR_API int faar_profile_end(faar_ctx* ctx, faar_kernel_time* out, int capacity, int* count);
+FAAR_API const char* faar_kernel_name(int kernel);
+
 /* ---- part 1: soft-quantisation set-up, once per layer ----------------------
  * Procedure steps 2-5, "NVFP4 Overview", Eq. 4.
  * Computes the FP32 tensor scale (s_global = amax|W| / (6*448) unless
@@ -130,12 +160,14 @@ FAAR_API int faar_softquant_init(faar_ctx* ctx, const faar_shape* shape, const v
 
 /* ---- part 2: soft weights, FP32 view ---------------------------------------
  * Procedure steps 6-7, Eq. 2 and Eq. 3:  h = sigmoid(beta*(v-0.5)),
- * W_soft = sign*(lo + h*(hi-lo))*s_g*s_global.  This is the FP32 view of what
- * the forward GEMM's operand is built from; either output may be null.
- *   W_soft out: [O,K] float (nullable)    h out: [O,K] float (nullable) */
+ * W_soft = sign*(lo + h*(hi-lo))*s_g*s_global, evaluated in FP32.  W_soft_bf16
+ * is that FP32 value rounded to nearest even: exactly the operand the forward
+ * GEMM multiplies (faar_layer_fwd builds it with this same routine).  Any
+ * output may be null.
+ *   W_soft out: [O,K] float    h out: [O,K] float    W_soft_bf16 out: [O,K] bf16 */
 FAAR_API int faar_softquant_eval(faar_ctx* ctx, const faar_shape* shape, const float* V, const uint8_t* code,
                         const uint8_t* scales, const float* s_global, float beta,
-                        float* W_soft, float* h);
+                        float* W_soft, float* h, void* W_soft_bf16);
 
 /* ---- layout helper ----------------------------------------------------------
  * out[c, r] = in[r, c] for a BF16 matrix in[rows, cols] (ld_in) -> out[cols, rows]
@@ -189,6 +221,18 @@ FAAR_API int faar_layer_step(faar_ctx* ctx, const faar_shape* shape, const faar_
                     const void* Xt, const void* Y_ref, float* V, const uint8_t* code,
                     const uint8_t* scales, const float* s_global, float* adam_m, float* adam_u,
                     float* loss_out2, void* workspace, size_t workspace_bytes);
+
+/* faar_layer_step for a calibration batch that lives in HOST memory (ideally
+ * pinned): copies X_host[T,K] (ldx) and Y_ref_host[T,O] (ldy) into the caller's
+ * device staging buffers X_dev / Yref_dev, rebuilds Xt_dev = X^T [K, ldxt],
+ * runs the step, and copies {L_MSE, L_round} back to loss_host2.  Everything
+ * is enqueued on the context's stream; loss_host2 is valid after the caller
+ * synchronises it.  Bytes moved: T*K*2 + T*O*sizeof(yref_dtype) in, 8 out. */
+FAAR_API int faar_layer_step_host(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp,
+                                  const void* X_host, const void* Y_ref_host, void* X_dev, void* Xt_dev,
+                                  void* Yref_dev, float* V, const uint8_t* code, const uint8_t* scales,
+                                  const float* s_global, float* adam_m, float* adam_u, float* loss_dev2,
+                                  float* loss_host2, void* workspace, size_t workspace_bytes);
 
 /* ---- part 5: harden + pack ---------------------------------------------------
  * Procedure steps 25-26, Eq. 7: v_hat = (v >= 0.5); weight code = k + v_hat.

@@ -238,19 +238,26 @@ def layer_fwd(X, Y_ref, V, code, scales, s_global, beta, mse_scale=1.0, mode="bf
     return loss, dY, Yq
 
 
-def layer_grad(dY, X, V, code, scales, s_global, beta, lambda_round):
-    """Gradient of Eq. 5 with respect to V (the paper states the loss; this is
-    its derivative).  G = dY^T X is dL_MSE/dW_soft; the chain rule through
-    Eq. 2 and Eq. 3 multiplies by sign * s * (hi - lo) * beta * h * (1 - h);
-    the Round Loss adds (lambda / N) * (4 - 8 v).  Returns (dV, G)."""
+def chain_factor(V, code, scales, s_global, beta):
+    """dW_soft/dv through Eq. 2 and Eq. 3: sign * s * (hi - lo) * beta * h * (1 - h)
+    (lo, hi, s and the sign are constants; only V is learnable)."""
     V = np.asarray(V, dtype=np.float64)
-    G = np.asarray(dY, np.float64).T @ np.asarray(X, np.float64)
     k, neg = unpack_code(code)
     s = np.repeat(effective_scale(scales, s_global), BLOCK, axis=1).astype(np.float64)
     h = h_beta(V, beta)
     width = NODES[k + 1] - NODES[k]
     sgn = np.where(neg, -1.0, 1.0)
-    dV = G * sgn * s * width * float(beta) * h * (1.0 - h)
+    return sgn * s * width * float(beta) * h * (1.0 - h)
+
+
+def layer_grad(dY, X, V, code, scales, s_global, beta, lambda_round):
+    """Gradient of Eq. 5 with respect to V (the paper states the loss; this is
+    its derivative).  G = dY^T X is dL_MSE/dW_soft; the chain rule through
+    Eq. 2 and Eq. 3 multiplies by chain_factor; the Round Loss adds
+    (lambda / N) * (4 - 8 v).  Returns (dV, G)."""
+    V = np.asarray(V, dtype=np.float64)
+    G = np.asarray(dY, np.float64).T @ np.asarray(X, np.float64)
+    dV = G * chain_factor(V, code, scales, s_global, beta)
     dV = dV + (float(lambda_round) / V.size) * (4.0 - 8.0 * V)
     return dV, G
 

@@ -52,7 +52,7 @@ int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
              const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
              void* Y_q, uint8_t* ws, const faar_ws_layout& l, int* n_partials) {
   __nv_bfloat16* wsoft = reinterpret_cast<__nv_bfloat16*>(ws + l.off_wsoft);
-  int e = faar_launch_softquant_bf16(ctx, s, V, code, scales, s_global, hp->beta, wsoft);
+  int e = faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, hp->beta, nullptr, nullptr, wsoft);
   if (e) return e;
   faar_gemm_args a = {};
   a.mode = FAAR_GEMM_FWD;
@@ -98,6 +98,24 @@ int check_gemm_operands(const faar_shape* s, bool need_x, bool need_xt) {
 
 }  // namespace
 
+faar_prof_scope::faar_prof_scope(faar_ctx* ctx, int kernel_id) : c(ctx), pair(-1) {
+  if (!c->prof_on) return;
+  const int i = c->prof_used;
+  while ((int)c->prof_events.size() < 2 * (i + 1)) {
+    cudaEvent_t ev;
+    if (cudaEventCreate(&ev) != cudaSuccess) return;
+    c->prof_events.push_back(ev);
+  }
+  if (cudaEventRecord(c->prof_events[2 * i], c->stream) != cudaSuccess) return;
+  c->prof_kernel.push_back(kernel_id);
+  c->prof_used = i + 1;
+  pair = i;
+}
+
+faar_prof_scope::~faar_prof_scope() {
+  if (pair >= 0) cudaEventRecord(c->prof_events[2 * pair + 1], c->stream);
+}
+
 extern "C" {
 
 const char* faar_status_string(int status) {
@@ -129,6 +147,8 @@ int faar_create(faar_ctx** out, int device, void* stream) {
   c->stream = reinterpret_cast<cudaStream_t>(stream);
   c->last_cuda_error = 0;
   c->encode_tiled = nullptr;
+  c->prof_on = false;
+  c->prof_used = 0;
   cudaDriverEntryPointQueryResult q;
   e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &q);
   if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !c->encode_tiled) {
@@ -140,7 +160,62 @@ int faar_create(faar_ctx** out, int device, void* stream) {
 }
 
 int faar_destroy(faar_ctx* ctx) {
+  if (ctx) {
+    for (cudaEvent_t ev : ctx->prof_events) cudaEventDestroy(ev);
+  }
   delete ctx;
+  return FAAR_OK;
+}
+
+const char* faar_kernel_name(int kernel) {
+  switch (kernel) {
+    case FAAR_K_AMAX: return "amax";
+    case FAAR_K_SOFTQUANT_INIT: return "softquant_init";
+    case FAAR_K_SOFT_WEIGHTS: return "soft_weights";
+    case FAAR_K_GEMM_REF: return "gemm_ref";
+    case FAAR_K_GEMM_FWD: return "gemm_fwd";
+    case FAAR_K_GEMM_BWD: return "gemm_bwd";
+    case FAAR_K_ROUND_LOSS: return "round_loss";
+    case FAAR_K_FINALIZE: return "finalize";
+    case FAAR_K_HARDEN_PACK: return "harden_pack";
+    case FAAR_K_TRANSPOSE: return "transpose";
+  }
+  return "unknown";
+}
+
+int faar_profile_begin(faar_ctx* ctx) {
+  if (!ctx) return FAAR_ERR_INVALID_ARG;
+  ctx->prof_on = true;
+  ctx->prof_used = 0;
+  ctx->prof_kernel.clear();
+  return FAAR_OK;
+}
+
+int faar_profile_end(faar_ctx* ctx, faar_kernel_time* out, int capacity, int* count) {
+  if (!ctx || !out || !count || capacity < 0) return FAAR_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  ctx->prof_on = false;
+  *count = 0;
+  cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+  int launches[FAAR_K_COUNT] = {0};
+  double total[FAAR_K_COUNT] = {0.0};
+  for (int i = 0; i < ctx->prof_used; ++i) {
+    float ms = 0.f;
+    e = cudaEventElapsedTime(&ms, ctx->prof_events[2 * i], ctx->prof_events[2 * i + 1]);
+    if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+    const int k = ctx->prof_kernel[i];
+    launches[k] += 1;
+    total[k] += ms;
+  }
+  for (int k = 0; k < FAAR_K_COUNT && *count < capacity; ++k) {
+    if (!launches[k]) continue;
+    out[*count].kernel = k;
+    out[*count].launches = launches[k];
+    out[*count].total_ms = (float)total[k];
+    *count += 1;
+  }
+  ctx->prof_used = 0;
   return FAAR_OK;
 }
 
@@ -198,16 +273,19 @@ int faar_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float
 }
 
 int faar_softquant_eval(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
-                        const uint8_t* scales, const float* s_global, float beta, float* W_soft, float* h) {
+                        const uint8_t* scales, const float* s_global, float beta, float* W_soft, float* h,
+                        void* W_soft_bf16) {
   if (!ctx || !V || !code || !scales || !s_global) return FAAR_ERR_INVALID_ARG;
   int st = check_shape(s);
   if (st) return st;
   if (!(beta > 0.f) || !isfinite(beta)) return FAAR_ERR_INVALID_ARG;
-  if (!aligned16(V) || !aligned16(code) || (W_soft && !aligned16(W_soft)) || (h && !aligned16(h)))
+  if (!aligned16(V) || !aligned16(code) || (W_soft && !aligned16(W_soft)) || (h && !aligned16(h)) ||
+      (W_soft_bf16 && !aligned16(W_soft_bf16)))
     return FAAR_ERR_ALIGN;
-  if (!W_soft && !h) return FAAR_OK;
+  if (!W_soft && !h && !W_soft_bf16) return FAAR_OK;
   DeviceGuard g(ctx->device);
-  return cuda_fail(ctx, faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, beta, W_soft, h));
+  return cuda_fail(ctx, faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, beta, W_soft, h,
+                                                   reinterpret_cast<__nv_bfloat16*>(W_soft_bf16)));
 }
 
 int faar_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in, int64_t ld_in, void* out,
@@ -329,6 +407,35 @@ int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, 
                            reinterpret_cast<float*>(ws + l.off_round_partials), np_round,
                            (float)(1.0 / ((double)s->O * (double)s->K)), loss_out2 + 1);
   return cuda_fail(ctx, e);
+}
+
+int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X_host,
+                         const void* Y_ref_host, void* X_dev, void* Xt_dev, void* Yref_dev, float* V,
+                         const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
+                         float* adam_u, float* loss_dev2, float* loss_host2, void* workspace,
+                         size_t workspace_bytes) {
+  if (!ctx || !X_host || !Y_ref_host || !X_dev || !Xt_dev || !Yref_dev || !loss_dev2 || !loss_host2)
+    return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
+  if (s->ldy < s->O) return FAAR_ERR_SHAPE;
+  if ((st = check_gemm_operands(s, true, true))) return st;
+  DeviceGuard g(ctx->device);
+  const size_t ybytes = s->yref_dtype == FAAR_BF16 ? 2 : 4;
+  cudaError_t e = cudaMemcpyAsync(X_dev, X_host, (size_t)s->T * (size_t)s->ldx * 2, cudaMemcpyHostToDevice,
+                                  ctx->stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(Yref_dev, Y_ref_host, (size_t)s->T * (size_t)s->ldy * ybytes, cudaMemcpyHostToDevice,
+                        ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+  st = faar_transpose_bf16(ctx, s->T, s->K, X_dev, s->ldx, Xt_dev, s->ldxt);
+  if (st) return st;
+  st = faar_layer_step(ctx, s, hp, X_dev, Xt_dev, Yref_dev, V, code, scales, s_global, adam_m, adam_u, loss_dev2,
+                       workspace, workspace_bytes);
+  if (st) return st;
+  e = cudaMemcpyAsync(loss_host2, loss_dev2, 2 * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream);
+  return cuda_fail(ctx, (int)e);
 }
 
 int faar_harden_pack(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code, const uint8_t* scales,

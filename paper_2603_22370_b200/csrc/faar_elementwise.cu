@@ -112,28 +112,11 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
 }
 
 // ---- Eq. 2 / Eq. 3 in FP32 (parity view) -----------------------------------------
-// The argument beta*(v-0.5) is formed as an unevaluated sum hi + lo so that the
-// relative error of h stays near one ulp even where h is tiny.
-__device__ __forceinline__ float sigmoid_precise(float beta, float v) {
-  float p = __fmul_rn(beta, v);
-  float pe = __fmaf_rn(beta, v, -p);          // exact error of the product
-  float c = 0.5f * beta;                      // exact
-  float hi = __fsub_rn(p, c);
-  float bb = __fsub_rn(hi, p);                // two-sum of p + (-c)
-  float lo = __fadd_rn(__fsub_rn(p, __fsub_rn(hi, bb)), __fsub_rn(-c, bb));
-  lo = __fadd_rn(lo, pe);
-  // h = 1 / (1 + exp(-(hi+lo)));  exp(-(hi+lo)) = exp(-hi) * (1 - lo + ...)
-  float e = expf(-fabsf(hi));
-  float adj = hi >= 0.f ? -lo : lo;           // exp(-|hi| - sign*lo)
-  e = __fmaf_rn(e, adj, e);
-  float hs = __fdiv_rn(1.0f, 1.0f + e);       // sigmoid(|z|)
-  return hi >= 0.f ? hs : __fmul_rn(e, hs);   // sigmoid(-|z|) = e / (1 + e)
-}
-
 __global__ void __launch_bounds__(EW_THREADS)
 softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code,
                       const uint8_t* __restrict__ scales, const float* __restrict__ s_global_p,
-                      float beta, int64_t n_groups, float* __restrict__ W_soft, float* __restrict__ H) {
+                      float beta, int64_t n_groups, float* __restrict__ W_soft, float* __restrict__ H,
+                      __nv_bfloat16* __restrict__ W_bf16) {
   const float s_global = *s_global_p;
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups;
        g += (int64_t)gridDim.x * blockDim.x) {
@@ -148,9 +131,8 @@ softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ c
     for (int i = 0; i < 8; ++i) {
       uint32_t nib = (cw >> (4 * i)) & 0xF;
       int k = nib & 7;
-      h[i] = sigmoid_precise(beta, v[i]);
-      float mag = __fmul_rn(__fmaf_rn(h[i], faar_width(k), faar_node(k)), s);
-      ws[i] = (nib & 8) ? -mag : mag;
+      h[i] = faar_sigmoid_precise(beta, v[i]);
+      ws[i] = faar_soft_weight(h[i], nib, s);
     }
     if (W_soft) {
       float4* p = reinterpret_cast<float4*>(W_soft + e);
@@ -162,43 +144,15 @@ softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ c
       p[0] = make_float4(h[0], h[1], h[2], h[3]);
       p[1] = make_float4(h[4], h[5], h[6], h[7]);
     }
-  }
-}
-
-// ---- Eq. 2 / Eq. 3 -> BF16 GEMM operand ---------------------------------------------
-__global__ void __launch_bounds__(EW_THREADS)
-softquant_bf16_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code,
-                      const uint8_t* __restrict__ scales, const float* __restrict__ s_global_p,
-                      float beta, int64_t n_groups, __nv_bfloat16* __restrict__ W_soft) {
-  const float s_global = *s_global_p;
-  const float nhb = -0.5f * beta;
-  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups;
-       g += (int64_t)gridDim.x * blockDim.x) {
-    int64_t e = g * 8;
-    const float4* vp = reinterpret_cast<const float4*>(V + e);
-    float4 a = vp[0], b = vp[1];
-    float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    uint32_t cw = *reinterpret_cast<const uint32_t*>(code + e / 2);
-    float s = __fmul_rn(faar_e4m3_to_float(scales[e / 16]), s_global);
-    uint32_t out[4];
+    if (W_bf16) {
+      uint32_t o[4];
 #pragma unroll
-    for (int i = 0; i < 8; i += 2) {
-      float r[2];
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        uint32_t nib = (cw >> (4 * (i + j))) & 0xF;
-        int k = nib & 7;
-        float z = fmaf(beta, v[i + j], nhb);
-        float ex = __expf(-fabsf(z));
-        float hs = __fdividef(1.0f, 1.0f + ex);
-        float h = z >= 0.f ? hs : ex * hs;
-        float mag = fmaf(h, faar_width(k), faar_node(k)) * s;
-        r[j] = (nib & 8) ? -mag : mag;
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(ws[2 * i], ws[2 * i + 1]);
+        o[i] = *reinterpret_cast<uint32_t*>(&p2);
       }
-      __nv_bfloat162 p = __floats2bfloat162_rn(r[0], r[1]);
-      out[i / 2] = *reinterpret_cast<uint32_t*>(&p);
+      *reinterpret_cast<uint4*>(W_bf16 + e) = make_uint4(o[0], o[1], o[2], o[3]);
     }
-    *reinterpret_cast<uint4*>(W_soft + e) = make_uint4(out[0], out[1], out[2], out[3]);
   }
 }
 
@@ -338,8 +292,10 @@ int faar_launch_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W
   if (!(s_global_in > 0.f)) {
     cudaError_t e = cudaMemsetAsync(amax_word, 0, sizeof(uint32_t), ctx->stream);
     if (e != cudaSuccess) return (int)e;
+    faar_prof_scope ps(ctx, FAAR_K_AMAX);
     amax_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, amax_word);
   }
+  faar_prof_scope ps(ctx, FAAR_K_SOFTQUANT_INIT);
   softquant_init_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, s_global_in,
                                                                amax_word, scales, s_global_out, code, V);
   return (int)cudaGetLastError();
@@ -347,25 +303,18 @@ int faar_launch_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W
 
 int faar_launch_softquant_eval(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta, float* W_soft,
-                               float* h) {
+                               float* h, __nv_bfloat16* W_bf16) {
   const int64_t groups = (int64_t)s->O * (s->K / 8);
+  faar_prof_scope ps(ctx, FAAR_K_SOFT_WEIGHTS);
   softquant_eval_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(V, code, scales, s_global, beta,
-                                                                                  groups, W_soft, h);
-  return (int)cudaGetLastError();
-}
-
-int faar_launch_softquant_bf16(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
-                               const uint8_t* scales, const float* s_global, float beta,
-                               __nv_bfloat16* W_soft) {
-  const int64_t groups = (int64_t)s->O * (s->K / 8);
-  softquant_bf16_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(V, code, scales, s_global, beta,
-                                                                                  groups, W_soft);
+                                                                                  groups, W_soft, h, W_bf16);
   return (int)cudaGetLastError();
 }
 
 int faar_launch_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in, int64_t ld_in, void* out,
                                int64_t ld_out) {
   dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+  faar_prof_scope ps(ctx, FAAR_K_TRANSPOSE);
   transpose_bf16_kernel<<<grid, 256, 0, ctx->stream>>>(reinterpret_cast<const uint16_t*>(in), rows, cols, ld_in,
                                                        reinterpret_cast<uint16_t*>(out), ld_out);
   return (int)cudaGetLastError();
@@ -374,6 +323,7 @@ int faar_launch_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in
 int faar_launch_round_partials(faar_ctx* ctx, const float* V, int64_t N, float* partials, int* n_partials) {
   int grid = grid_for(ctx, (N + 3) / 4, 4);
   if (grid > FAAR_MAX_PARTIALS) grid = FAAR_MAX_PARTIALS;
+  faar_prof_scope ps(ctx, FAAR_K_ROUND_LOSS);
   round_partials_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(V, N, partials);
   *n_partials = grid;
   return (int)cudaGetLastError();
@@ -381,6 +331,7 @@ int faar_launch_round_partials(faar_ctx* ctx, const float* V, int64_t N, float* 
 
 int faar_launch_finalize(faar_ctx* ctx, const float* p0, int n0, float scale0, float* out0, const float* p1,
                          int n1, float scale1, float* out1) {
+  faar_prof_scope ps(ctx, FAAR_K_FINALIZE);
   finalize_kernel<<<1, 256, 0, ctx->stream>>>(p0, n0, scale0, out0, p1, n1, scale1, out1);
   return (int)cudaGetLastError();
 }
@@ -389,6 +340,7 @@ int faar_launch_harden_pack(faar_ctx* ctx, const faar_shape* s, const float* V, 
                             const uint8_t* scales, const float* s_global, uint8_t* packed,
                             uint8_t* scales_out, uint8_t* decisions, void* W_final, int wfinal_dtype) {
   const int64_t groups = (int64_t)s->O * (s->K / 8);
+  faar_prof_scope ps(ctx, FAAR_K_HARDEN_PACK);
   harden_pack_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(
       V, code, scales, s_global, groups, packed, scales_out, decisions, W_final, wfinal_dtype);
   return (int)cudaGetLastError();

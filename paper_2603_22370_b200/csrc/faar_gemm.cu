@@ -463,6 +463,7 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, const KParams& kp, int grid) 
   auto kern = faar_gemm_kernel<MODE, BN>;
   cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
   if (ce != cudaSuccess) return (int)ce;
+  faar_prof_scope ps(ctx, MODE == FAAR_GEMM_REF ? FAAR_K_GEMM_REF : (MODE == FAAR_GEMM_FWD ? FAAR_K_GEMM_FWD : FAAR_K_GEMM_BWD));
   kern<<<grid, NUM_THREADS, Cfg::SMEM_BYTES, ctx->stream>>>(tmA, tmB, kp);
   return (int)cudaGetLastError();
 }

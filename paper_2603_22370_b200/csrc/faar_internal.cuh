@@ -7,12 +7,27 @@
 
 #include "faar.h"
 
+#include <vector>
+
 struct faar_ctx {
   int device;
   int num_sms;
   cudaStream_t stream;
   int last_cuda_error;
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
+  // per-kernel timing (faar_profile_begin / faar_profile_end)
+  bool prof_on;
+  int prof_used;                          // event pairs used since faar_profile_begin
+  std::vector<cudaEvent_t> prof_events;   // 2 per launch: start, stop
+  std::vector<int> prof_kernel;           // kernel id per pair
+};
+
+// Brackets one kernel launch with a pair of CUDA events when profiling is on.
+struct faar_prof_scope {
+  faar_ctx* c;
+  int pair;
+  faar_prof_scope(faar_ctx* ctx, int kernel_id);
+  ~faar_prof_scope();
 };
 
 // ---- workspace layout -------------------------------------------------------
@@ -54,10 +69,7 @@ int faar_launch_softquant_init(faar_ctx*, const faar_shape*, const void* W, floa
                                uint32_t* amax_word);
 int faar_launch_softquant_eval(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta,
-                               float* W_soft, float* h);
-int faar_launch_softquant_bf16(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
-                               const uint8_t* scales, const float* s_global, float beta,
-                               __nv_bfloat16* W_soft);
+                               float* W_soft, float* h, __nv_bfloat16* W_soft_bf16);
 int faar_launch_transpose_bf16(faar_ctx*, int rows, int cols, const void* in, int64_t ld_in, void* out,
                                int64_t ld_out);
 int faar_launch_round_partials(faar_ctx*, const float* V, int64_t N, float* partials, int* n_partials);
@@ -127,6 +139,32 @@ __device__ __forceinline__ uint32_t faar_float_to_e4m3(float q) {
   uint32_t e = (bits >> 23) - 120u;
   uint32_t m = (bits >> 20) & 7u;
   return (e << 3) | m;
+}
+
+// Eq. 3 in FP32, accurate to about one ulp over the whole range of h.
+// The argument beta*(v-0.5) is formed as an unevaluated sum hi + lo so that the
+// relative error of h stays near one ulp even where h is tiny.
+__device__ __forceinline__ float faar_sigmoid_precise(float beta, float v) {
+  float p = __fmul_rn(beta, v);
+  float pe = __fmaf_rn(beta, v, -p);          // exact error of the product
+  float c = 0.5f * beta;                      // exact
+  float hi = __fsub_rn(p, c);
+  float bb = __fsub_rn(hi, p);                // two-sum of p + (-c)
+  float lo = __fadd_rn(__fsub_rn(p, __fsub_rn(hi, bb)), __fsub_rn(-c, bb));
+  lo = __fadd_rn(lo, pe);
+  // h = 1 / (1 + exp(-(hi+lo)));  exp(-(hi+lo)) = exp(-hi) * (1 - lo + ...)
+  float e = expf(-fabsf(hi));
+  float adj = hi >= 0.f ? -lo : lo;           // exp(-|hi| - sign*lo)
+  e = __fmaf_rn(e, adj, e);
+  float hs = __fdiv_rn(1.0f, 1.0f + e);       // sigmoid(|z|)
+  return hi >= 0.f ? hs : __fmul_rn(e, hs);   // sigmoid(-|z|) = e / (1 + e)
+}
+
+// Eq. 2 in FP32: sign * (lo + h * (hi - lo)) * s for the nibble (sign<<3 | k).
+__device__ __forceinline__ float faar_soft_weight(float h, uint32_t nib, float s) {
+  int k = nib & 7;
+  float mag = __fmul_rn(__fmaf_rn(h, faar_width(k), faar_node(k)), s);
+  return (nib & 8) ? -mag : mag;
 }
 
 __device__ __forceinline__ float faar_warp_sum(float v) {

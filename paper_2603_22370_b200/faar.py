@@ -19,7 +19,8 @@ BF16, F32 = 0, 1
 EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string", "faar_last_cuda_error",
            "faar_workspace_size", "faar_workspace_init", "faar_check_status", "faar_softquant_init",
            "faar_softquant_eval", "faar_transpose_bf16", "faar_layer_ref", "faar_layer_fwd", "faar_round_loss",
-           "faar_layer_bwd", "faar_layer_step", "faar_harden_pack"]
+           "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
+           "faar_profile_end", "faar_kernel_name"]
 
 
 class HParams(C.Structure):
@@ -145,9 +146,9 @@ def softquant_init(ctx, shape, W, s_global_in, scales, s_global_out, code, V_ini
            "faar_softquant_init")
 
 
-def softquant_eval(ctx, shape, V, code, scales, s_global, beta, W_soft, h):
+def softquant_eval(ctx, shape, V, code, scales, s_global, beta, W_soft, h, W_soft_bf16=None):
     _check(lib().faar_softquant_eval(ctx._h, C.byref(shape), _p(V), _p(code), _p(scales), _p(s_global),
-                                     C.c_float(beta), _p(W_soft), _p(h)), "faar_softquant_eval")
+                                     C.c_float(beta), _p(W_soft), _p(h), _p(W_soft_bf16)), "faar_softquant_eval")
 
 
 def transpose_bf16(ctx, rows, cols, inp, ld_in, out, ld_out):
@@ -187,3 +188,31 @@ def harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, decis
     _check(lib().faar_harden_pack(ctx._h, C.byref(shape), _p(V), _p(code), _p(scales), _p(s_global), _p(packed),
                                   _p(scales_out), _p(decisions), _p(W_final), C.c_int(wfinal_dtype)),
            "faar_harden_pack")
+
+
+def layer_step_host(ctx, shape, hp, X_host, Y_ref_host, X_dev, Xt_dev, Yref_dev, V, code, scales, s_global, adam_m,
+                    adam_u, loss_dev2, loss_host2, ws):
+    """X_host, Y_ref_host, loss_host2 are (pinned) CPU tensors; the rest are device tensors."""
+    _check(lib().faar_layer_step_host(ctx._h, C.byref(shape), C.byref(hp), C.c_void_p(X_host.data_ptr()),
+                                      C.c_void_p(Y_ref_host.data_ptr()), _p(X_dev), _p(Xt_dev), _p(Yref_dev), _p(V),
+                                      _p(code), _p(scales), _p(s_global), _p(adam_m), _p(adam_u), _p(loss_dev2),
+                                      C.c_void_p(loss_host2.data_ptr()), _p(ws), C.c_size_t(ws.numel())),
+           "faar_layer_step_host")
+
+
+class KernelTime(C.Structure):
+    _fields_ = [("kernel", C.c_int), ("launches", C.c_int), ("total_ms", C.c_float)]
+
+
+def profile_begin(ctx):
+    _check(lib().faar_profile_begin(ctx._h), "faar_profile_begin")
+
+
+def profile_end(ctx) -> dict:
+    """{kernel name: (launches, total_ms)} for the kernels launched since profile_begin."""
+    arr = (KernelTime * 16)()
+    n = C.c_int(0)
+    _check(lib().faar_profile_end(ctx._h, arr, 16, C.byref(n)), "faar_profile_end")
+    l = lib()
+    l.faar_kernel_name.restype = C.c_char_p
+    return {l.faar_kernel_name(arr[i].kernel).decode(): (arr[i].launches, arr[i].total_ms) for i in range(n.value)}

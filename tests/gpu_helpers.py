@@ -100,3 +100,41 @@ def max_rel_to_peak(a, b):
     a = np.asarray(a, np.float64)
     b = np.asarray(b, np.float64)
     return float(np.max(np.abs(a - b)) / max(np.max(np.abs(b)), 1e-300))
+
+
+# ---- BF16 operand ties ---------------------------------------------------------------------
+# The forward GEMM multiplies W_soft rounded to BF16.  The library evaluates W_soft in FP32
+# (tested to 1e-6 relative against the float64 oracle); where the exact value lies within that
+# error of a BF16 rounding boundary, either neighbour is a correct rounding.  The helpers below
+# find those elements from the ORACLE's W_soft and give the exact first-order effect of moving
+# one of them by one BF16 step, so that a comparison can allow for it and nothing else.
+
+W_SOFT_FP32_TOL = 1e-6
+
+
+def bf16_tie_elements(W_soft, tol=W_SOFT_FP32_TOL):
+    """(mask of elements within tol*|w| of a BF16 rounding boundary, BF16 spacing at each element)."""
+    w = np.abs(np.asarray(W_soft, np.float64))
+    with np.errstate(divide="ignore"):
+        step = np.where(w > 0, np.exp2(np.floor(np.log2(np.where(w > 0, w, 1.0))) - 7), 0.0)
+    frac = np.where(step > 0, w / np.where(step > 0, step, 1.0), 0.0) % 1.0
+    tie = (step > 0) & (np.abs(frac - 0.5) * step <= tol * w)
+    return tie, step
+
+
+def dy_column_allowance(X, tie, step, mse_scale):
+    """Per output feature o: norm of the largest change of dY[:, o] that re-rounding the tie
+    elements of row o can cause (dY = 2c (X W_soft^T - Y_ref))."""
+    Xd = np.asarray(X, np.float64)
+    xn = np.linalg.norm(Xd, axis=0)                                   # ||X[:, k]||
+    return 2.0 * mse_scale * (np.where(tie, step, 0.0) * xn[None, :]).sum(axis=1)
+
+
+def dv_row_allowance(X, tie, step, chain, mse_scale):
+    """Per weight row o: norm of the largest change of dV[o, :] from re-rounding its tie elements:
+    delta dV[o, :] = 2c * step * (X[:, k]^T X) * chain[o, :]."""
+    Xd = np.asarray(X, np.float64)
+    out = np.zeros(tie.shape[0])
+    for o, k in zip(*np.nonzero(tie)):
+        out[o] += np.linalg.norm(2.0 * mse_scale * step[o, k] * (Xd[:, k] @ Xd) * chain[o])
+    return out

@@ -17,7 +17,8 @@ import torch
 
 from oracle import faar_oracle as fo
 from paper_2603_22370_b200 import faar, inputs
-from tests.gpu_helpers import DEV, GpuLayer, dev_bf16, dev_f32, dev_u8, host, max_rel_to_peak, rel_l2
+from tests.gpu_helpers import (DEV, GpuLayer, bf16_tie_elements, dev_bf16, dev_f32, dev_u8, dv_row_allowance,
+                               dy_column_allowance, host, max_rel_to_peak, rel_l2)
 
 pytestmark = pytest.mark.gpu
 
@@ -125,6 +126,15 @@ def test_softquant_eval_matches_eq2_eq3(ctx, beta):
     H2 = torch.empty_like(lay.V)
     faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, b, None, H2)
     assert torch.equal(H, H2)
+    # the BF16 GEMM operand is the FP32 value rounded to nearest even; it can differ from the
+    # oracle's rounding only where the exact value sits on a BF16 rounding boundary
+    Wb = torch.empty_like(lay.V, dtype=torch.bfloat16)
+    faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, b, None, None, Wb)
+    assert torch.equal(Wb, Ws.to(torch.bfloat16))
+    tie, step = bf16_tie_elements(Wo)
+    diff = host(Wb).astype(np.float64) != fo.bf16_round(Wo)
+    assert not np.any(diff & ~tie)
+    assert np.all(np.abs(host(Wb)[diff] - fo.bf16_round(Wo)[diff]) <= step[diff] * (1 + 1e-12))
 
 
 def test_softquant_eval_saturates_to_floor_and_ceil(ctx):
@@ -244,7 +254,16 @@ def test_layer_fwd(ctx, O, K, T):
                                    hpo.beta, hpo.mse_scale, "bf16")
     assert abs(host(lay.loss)[0] - l_o) <= 2e-3 * l_o
     dY_g = host(lay.dYt)[:, :T].T
-    assert rel_l2(dY_g, dY_o) <= 2e-3 and max_rel_to_peak(dY_g, dY_o) <= 2e-3
+    # per output feature: 2e-3 of the column, plus what re-rounding a BF16-boundary weight of that
+    # row can move (zero for almost every column)
+    Wo, _ = fo.soft_weights(V, host(lay.code), host(lay.scales), host(lay.s_global)[0], hpo.beta)
+    tie, step = bf16_tie_elements(Wo)
+    allow = dy_column_allowance(X, tie, step, hpo.mse_scale)
+    col_err = np.linalg.norm(dY_g - dY_o, axis=0)
+    assert np.all(col_err <= 2e-3 * np.linalg.norm(dY_o, axis=0) + allow)
+    assert (allow > 0).sum() <= max(4, 0.05 * O)
+    assert rel_l2(dY_g, dY_o) <= 2e-3 + np.linalg.norm(allow) / np.linalg.norm(dY_o)
+    assert max_rel_to_peak(dY_g[:, allow == 0], dY_o[:, allow == 0]) <= 2e-3
     assert rel_l2(host(Yq), Yq_o) <= 2e-3 and max_rel_to_peak(host(Yq), Yq_o) <= 4e-3   # BF16 output: 2^-8 rounding
 
 
@@ -274,7 +293,9 @@ def test_layer_bwd(ctx, O, K, T, opt):
     if opt == 1:
         Vn, mn, un = fo.adam_update(V.astype(np.float64), dV_g.astype(np.float64), m0.astype(np.float64),
                                     u0.astype(np.float64), hpo.lr, hpo.beta1, hpo.beta2, hpo.eps, hpo.step)
-        assert np.all(np.abs(host(lay.m) - mn) <= 2e-6 * np.abs(mn) + 1e-30)
+        # m = beta1*m + (1-beta1)*g may cancel: bound the error by the size of the summands
+        m_mag = np.abs(hpo.beta1 * m0) + np.abs((1 - hpo.beta1) * dV_g)
+        assert np.all(np.abs(host(lay.m) - mn) <= 2e-6 * m_mag + 1e-30)
         assert np.all(np.abs(host(lay.u) - un) <= 2e-6 * np.abs(un) + 1e-30)
     else:
         Vn = fo.sgd_update(V.astype(np.float64), dV_g.astype(np.float64), hpo.lr)
@@ -327,12 +348,18 @@ def test_layer_step_is_fwd_then_bwd_and_matches_oracle(ctx, O, K, T):
     assert rel_l2(V_step, Vo) <= 2e-3 and np.max(np.abs(V_step - Vo)) <= 2.0 * hpo.lr + 1e-6
 
 
-def test_config1_trajectory_100_steps(ctx):
-    """BASELINE config 1 end to end: FP32 weights and target, BF16 GEMM operands, 100 Adam steps
-    with the geometric beta schedule, harden + pack."""
+def _config1():
     W, X = inputs.config1(0)
     Xb = inputs.to_bf16_f32(X)
-    Yref = fo.layer_ref(X, W).astype(np.float32)
+    Yref = fo.layer_ref(X, W).astype(np.float32)      # target from the unrounded FP32 X and W
+    return W, Xb, Yref
+
+
+def test_config1_100_steps_each_step_from_the_oracle_state(ctx):
+    """The 100-step run of the small FP32 configuration, one step at a time: before every step the
+    GPU receives the oracle's (V, m, u), so each step of the beta schedule and every Adam step index
+    is compared at the per-step tolerance, with no accumulated drift."""
+    W, Xb, Yref = _config1()
     steps = 100
     lay = GpuLayer(ctx, W, Xb, w_dtype=faar.F32, yref_dtype=faar.F32)
     lay.init()
@@ -340,28 +367,76 @@ def test_config1_trajectory_100_steps(ctx):
     scales, sg, code, V = fo.softquant_init(W)
     assert np.array_equal(host(lay.V), V)
     m, u = np.zeros_like(V), np.zeros_like(V)
-    hist_g, hist_o = [], []
     for t in range(steps):
         hp, hpo = f32hp(beta=fo.beta_schedule(t, steps), step=t + 1)
+        lay.set_state(V=V, m=m, u=u)
+        lay.step(hp)
+        lg = host(lay.loss).astype(np.float64)
+        Vp, mp, up = V, m, u
+        V, m, u, l_mse, l_round, dVo = fo.layer_step(Xb, Yref, V, code, scales, sg, m, u, hpo, "bf16")
+        assert abs(lg[0] - l_mse) <= 2e-3 * l_mse and abs(lg[1] - l_round) <= 2e-3 * l_round, t
+        Vg = host(lay.V)
+        # norm-wise 2e-3; a single entry may differ by up to the Adam step when its gradient is ~0
+        assert rel_l2(Vg, V) <= 2e-3 and np.max(np.abs(Vg - V)) <= 2.0 * hpo.lr + 1e-6, t
+        flips = fo.harden(Vg) != fo.harden(V)
+        assert flips.sum() <= 1e-4 * V.size + 1 and np.all(np.abs(V[flips] - 0.5) <= 2.0 * hpo.lr), t
+        # Adam moments: near a stationary point the data term and the Round Loss term of dV cancel, so
+        # the error is bounded against the size of the terms that are summed, not against their sum
+        rnd = hpo.lambda_round / V.size * (4.0 - 8.0 * Vp.astype(np.float64))
+        gmag = np.abs(dVo - rnd) + np.abs(rnd)
+        # rows that hold a weight on a BF16 rounding boundary may use either rounding of it
+        Wo, _ = fo.soft_weights(Vp, code, scales, sg, hpo.beta)
+        tie, bstep = bf16_tie_elements(Wo)
+        chain = fo.chain_factor(Vp, code, scales, sg, hpo.beta)
+        allow = dv_row_allowance(Xb, tie, bstep, chain, hpo.mse_scale)
+
+        def rn(a):
+            return np.linalg.norm(a, axis=1)
+
+        m_err, u_err = rn(host(lay.m) - m), rn(host(lay.u) - u)
+        assert np.all(m_err <= 2e-3 * (hpo.beta1 * rn(mp) + (1 - hpo.beta1) * rn(gmag)) + (1 - hpo.beta1) * allow), t
+        g_peak = np.abs(gmag).max(axis=1)
+        assert np.all(u_err <= 4e-3 * (hpo.beta2 * rn(up) + (1 - hpo.beta2) * rn(gmag * gmag))
+                      + (1 - hpo.beta2) * allow * (2 * g_peak + allow)), t
+    lay.check()
+
+
+def test_config1_free_running_100_steps_then_harden_pack(ctx):
+    """The same run with the GPU carrying its own state for all 100 steps.  Adam turns the few
+    BF16 rounding-boundary differences of a step into +-lr moves, and the optimisation amplifies
+    them, so the two trajectories are compared as two valid runs of the method: loss curves within
+    1e-2, final V within 2e-2 norm-wise, equal quality of the hardened weights, and bit-exact
+    harden + pack of the GPU's own V."""
+    W, Xb, Yref = _config1()
+    steps = 100
+    lay = GpuLayer(ctx, W, Xb, w_dtype=faar.F32, yref_dtype=faar.F32)
+    lay.init()
+    lay.set_yref(Yref)
+    hist_g = []
+    for t in range(steps):
+        hp, _ = f32hp(beta=fo.beta_schedule(t, steps), step=t + 1)
         lay.step(hp)
         hist_g.append(host(lay.loss).copy())
-        V, m, u, l_mse, l_round, _ = fo.layer_step(Xb, Yref, V, code, scales, sg, m, u, hpo, "bf16")
-        hist_o.append((l_mse, l_round))
     lay.check()
-    hist_g, hist_o = np.array(hist_g, np.float64), np.array(hist_o)
-    assert np.all(np.abs(hist_g - hist_o) <= 2e-3 * hist_o)
+    res = fo.run_layer(Xb, Yref, W, steps, lr=float(np.float32(1e-2)), mode="bf16")
+    hist_g, hist_o = np.array(hist_g, np.float64), np.array(res["hist"])
+    assert np.all(np.abs(hist_g - hist_o) <= 1e-2 * hist_o)
     Vg = host(lay.V)
-    assert rel_l2(Vg, V) <= 2e-3
-    # decisions: any disagreement must sit on the threshold in the oracle's trajectory
-    flips = fo.harden(Vg) != fo.harden(V)
-    assert flips.sum() <= 1e-4 * V.size + 1
-    assert np.all(np.abs(V[flips] - 0.5) < 5e-3)
-    # harden + pack is bit-exact on the same V
+    assert rel_l2(Vg, res["V"]) <= 2e-2
+    code, scales, sg = res["code"], res["scales"], res["s_global"]
+
+    def hard_loss(V):
+        _, _, Wf = fo.harden_pack(V, code, scales, sg)
+        return float(np.sum((Xb.astype(np.float64) @ Wf.astype(np.float64).T - Yref) ** 2))
+
+    l_g, l_o, l_rtn = hard_loss(Vg), hard_loss(res["V"]), hard_loss(fo.softquant_init(W)[3])
+    assert abs(l_g - l_o) <= 2e-2 * l_o
+    assert l_g < l_rtn                                   # the run improved on round-to-nearest
     packed = torch.zeros((128, 128), dtype=torch.uint8, device=DEV)
-    faar.harden_pack(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, packed, None, None, None)
-    p_o, _, _ = fo.harden_pack(Vg, code, scales, sg)
-    assert np.array_equal(host(packed), p_o)
-    # the optimisation did what it is for: the soft objective fell
+    dec = torch.zeros((128, 32), dtype=torch.uint8, device=DEV)
+    faar.harden_pack(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, packed, None, dec, None)
+    p_o, vh_o, _ = fo.harden_pack(Vg, code, scales, sg)
+    assert np.array_equal(host(packed), p_o) and np.array_equal(host(dec), fo.pack_decisions(vh_o))
     assert hist_g[-1].sum() < hist_g[0].sum()
 
 
