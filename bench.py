@@ -279,6 +279,16 @@ def run_ours(args):
     timed(profiled)
     prof = faar.profile_end(ctx)
 
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"quick": True, "steps": steps, "ms_per_step": ms_job / steps,
+                              "kernels_avg_us": {k: round(1e3 * v[1] / v[0], 2) for k, v in prof.items()}}))
+        if sampler:
+            sampler.stop()
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
     # ---- end to end: the calibration batch comes from pinned host memory every step
     Xh = torch.from_numpy(Xn).to(torch.bfloat16).pin_memory()
     Yh = Yref.cpu().pin_memory()
@@ -377,6 +387,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--quick", action="store_true",
+                    help="timed job and per-kernel pass only (no end-to-end pass, no CPU oracle leg); for profilers")
     args = ap.parse_args()
     return run_reference(args) if args.impl == "reference" else run_ours(args)
 

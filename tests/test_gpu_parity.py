@@ -261,7 +261,8 @@ def test_layer_fwd(ctx, O, K, T):
     allow = dy_column_allowance(X, tie, step, hpo.mse_scale)
     col_err = np.linalg.norm(dY_g - dY_o, axis=0)
     assert np.all(col_err <= 2e-3 * np.linalg.norm(dY_o, axis=0) + allow)
-    assert (allow > 0).sum() <= max(4, 0.05 * O)
+    # a weight is a tie with probability ~ 2 * 1e-6 / 2^-8, so only a few columns get an allowance
+    assert (allow > 0).sum() <= 4 + 3 * O * K * 2 * 1e-6 * 256
     assert rel_l2(dY_g, dY_o) <= 2e-3 + np.linalg.norm(allow) / np.linalg.norm(dY_o)
     assert max_rel_to_peak(dY_g[:, allow == 0], dY_o[:, allow == 0]) <= 2e-3
     assert rel_l2(host(Yq), Yq_o) <= 2e-3 and max_rel_to_peak(host(Yq), Yq_o) <= 4e-3   # BF16 output: 2^-8 rounding
