@@ -201,6 +201,27 @@ FAAR_API int faar_layer_fwd(faar_ctx* ctx, const faar_shape* shape, const faar_h
 FAAR_API int faar_round_loss(faar_ctx* ctx, const float* V, int64_t N, float* loss_round,
                     void* workspace, size_t workspace_bytes);
 
+/* The same Round Loss for callers that cannot allocate device memory (no
+ * counterpart in the paper: a deployment variant of faar_round_loss).  Meant for
+ * code that is handed raw device pointers and nothing else -- a plugin inside
+ * another runtime's memory pool, a serving loop in which cudaMalloc is forbidden
+ * or would stall the device -- and so has no workspace to give.  The partial
+ * sums live in a fixed 256 KB array inside the library's device image instead
+ * (one copy per GPU that loads the library, held until the process exits); the
+ * call allocates nothing, on the device or through any library.
+ *   V in: N floats, 16-byte aligned     loss_round out: 1 float (device)
+ * Limit: N <= faar_round_loss_static_max_n() (268 435 456 = 65536 partials x 4096
+ * elements); a larger N returns FAAR_ERR_SHAPE and launches nothing.
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call before
+ * any stream capture begins.  Every call on a device uses the same array and
+ * overwrites the slots it later reads, so nothing needs clearing between calls,
+ * but two calls that overlap on the GPU (different streams, no ordering between
+ * them) race on it: order them.  One partial per 4096 consecutive elements, so
+ * the result does not depend on the device's SM count. */
+FAAR_API int faar_round_loss_static(faar_ctx* ctx, const float* V, int64_t N, float* loss_round);
+FAAR_API int64_t faar_round_loss_static_max_n(void);
+
 /* Procedure step 13 with the clip that Stage 1 prescribes.  G = dY^T X on the
  * tensor cores (contraction over T), then per weight
  *   dV = G*sign*s*(hi-lo)*beta*h*(1-h) + (lambda_round/N)*(4-8v)

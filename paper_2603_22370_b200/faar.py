@@ -20,7 +20,7 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
            "faar_workspace_size", "faar_workspace_init", "faar_check_status", "faar_softquant_init",
            "faar_softquant_eval", "faar_transpose_bf16", "faar_layer_ref", "faar_layer_fwd", "faar_round_loss",
            "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
-           "faar_profile_end", "faar_kernel_name"]
+           "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n"]
 
 
 class HParams(C.Structure):
@@ -170,6 +170,18 @@ def layer_fwd(ctx, shape, hp, X, Y_ref, V, code, scales, s_global, dYt, loss_mse
 def round_loss(ctx, V, N, loss_round, ws):
     _check(lib().faar_round_loss(ctx._h, _p(V), C.c_int64(N), _p(loss_round), _p(ws), C.c_size_t(ws.numel())),
            "faar_round_loss")
+
+
+def round_loss_static(ctx, V, N, loss_round):
+    """Round Loss without a workspace: for callers that may not allocate device memory.  The scratch
+    is a fixed array inside libfaar.so; N is limited to round_loss_static_max_n()."""
+    _check(lib().faar_round_loss_static(ctx._h, _p(V), C.c_int64(N), _p(loss_round)), "faar_round_loss_static")
+
+
+def round_loss_static_max_n() -> int:
+    f = lib().faar_round_loss_static_max_n
+    f.restype = C.c_int64
+    return int(f())
 
 
 def layer_bwd(ctx, shape, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, dV, ws):
