@@ -27,6 +27,7 @@ constexpr int UMMA_K = 16;
 constexpr int NUM_EPI_WARPS = 8;
 constexpr int NUM_THREADS = 32 * (2 + NUM_EPI_WARPS);
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+constexpr int EPI_WARP_BYTES = 32 * 32 * 4;   // one 32 x 32 FP32 accumulator block per epilogue warp
 
 template <int BN> struct TileCfg {
   static constexpr int STAGES = BN == 256 ? 4 : 6;
@@ -34,7 +35,8 @@ template <int BN> struct TileCfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int EPI_BYTES = NUM_EPI_WARPS * EPI_WARP_BYTES;   // BWD: per-warp transposition buffers
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
@@ -122,6 +124,24 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -219,73 +239,94 @@ __device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const 
   return ss;
 }
 
-// BWD: acc = G[o, k0..k0+15] (one scale block).  Returns the Round Loss contribution of the
-// pre-update v's.
-__device__ __forceinline__ float epi_bwd(const KParams& p, int o, int k0, const uint32_t (&acc)[16], float s_global) {
-  if (o >= p.M || k0 >= p.N) return 0.f;
-  const long long e = (long long)o * p.N + k0;
-  float v[16];
-  {
-    const float4* vp = reinterpret_cast<const float4*>(p.V + e);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) { float4 t = vp[q]; v[4*q] = t.x; v[4*q+1] = t.y; v[4*q+2] = t.z; v[4*q+3] = t.w; }
-  }
-  const uint2 cw2 = *reinterpret_cast<const uint2*>(p.code + e / 2);
-  const float s = __fmul_rn(faar_e4m3_to_float(p.scales[e / 16]), s_global);
-  const float sb = s * p.beta;
-  float g[16];
+// BWD.  A warp's 32 x 32 block of G (row = output feature o, column = input feature k) has been
+// staged in shared memory, row r at stg + 128 r, its eight 16-byte units XOR-swizzled by (r & 7).
+// Here lane (a, b) = (lane / 8, lane % 8) handles, in pass q, row 4q + a and columns 4b..4b+3, so
+// that eight lanes cover 128 contiguous bytes of a row of V / m / u and every global access is a
+// full line.  Returns the Round Loss contribution of the pre-update v's.
+__device__ __forceinline__ float sqrt_approx(float x) {       // sqrt(0) = 0, about 1 ulp
+  float y;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float width_of(uint32_t k) {       // interval widths .5 .5 .5 .5 1 1 2
+  return __uint_as_float((126u + ((0x2500u >> (2u * k)) & 3u)) << 23);
+}
+
+template <int OPT>
+__device__ __forceinline__ float epi_bwd_block(const KParams& p, uint32_t stg, int lane, int o_first, int k_first,
+                                               float s_global) {
+  const int a = lane >> 3, b = lane & 7;
+  const int kcol = k_first + 4 * b;
+  const bool col_ok = kcol < p.N;
+  const float hb = -0.5f * p.beta;
+  const float c1 = 1.f - p.b1, c2 = 1.f - p.b2;
   float rl = 0.f;
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    uint32_t nib = ((j < 8 ? cw2.x : cw2.y) >> (4 * (j & 7))) & 0xF;
-    int k = nib & 7;
-    float z = fmaf(p.beta, v[j], -0.5f * p.beta);
-    float ex = __expf(-fabsf(z));
-    float hs = __fdividef(1.0f, 1.0f + ex);
-    float dh = ex * hs * hs;                        // h (1 - h)
-    float chain = sb * faar_width(k) * dh;
-    chain = (nib & 8) ? -chain : chain;
-    g[j] = fmaf(__uint_as_float(acc[j]), chain, p.lam_over_n * fmaf(-8.f, v[j], 4.f));
-    float t = fmaf(2.f, v[j], -1.f);
-    rl += fmaf(-t, t, 1.f);
-  }
-  if (p.dV) {
-    float4* dp = reinterpret_cast<float4*>(p.dV + e);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) dp[q] = make_float4(g[4*q], g[4*q+1], g[4*q+2], g[4*q+3]);
-  }
-  float vn[16];
-  if (p.opt == 1) {
-    float4* mp = reinterpret_cast<float4*>(p.adam_m + e);
-    float4* up = reinterpret_cast<float4*>(p.adam_u + e);
-    float m[16], u[16];
+  for (int half = 0; half < 2; ++half) {
+    float4 v[4], m[4], u[4];
+    uint32_t cw[4], sb[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      float4 t = mp[q]; m[4*q] = t.x; m[4*q+1] = t.y; m[4*q+2] = t.z; m[4*q+3] = t.w;
-      float4 w = up[q]; u[4*q] = w.x; u[4*q+1] = w.y; u[4*q+2] = w.z; u[4*q+3] = w.w;
-    }
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      m[j] = fmaf(p.b1, m[j], (1.f - p.b1) * g[j]);
-      u[j] = fmaf(p.b2, u[j], (1.f - p.b2) * g[j] * g[j]);
-      float mh = m[j] * p.inv_bc1;
-      float uh = u[j] * p.inv_bc2;
-      vn[j] = v[j] - p.lr * mh / (sqrtf(uh) + p.eps);
+      const int o = o_first + 16 * half + 4 * q + a;
+      if (col_ok && o < p.M) {
+        const long long e = (long long)o * p.N + kcol;
+        v[q] = *reinterpret_cast<const float4*>(p.V + e);
+        cw[q] = *reinterpret_cast<const uint16_t*>(p.code + (e >> 1));
+        sb[q] = p.scales[e >> 4];
+        if (OPT == 1) {
+          m[q] = *reinterpret_cast<const float4*>(p.adam_m + e);
+          u[q] = *reinterpret_cast<const float4*>(p.adam_u + e);
+        }
+      }
     }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      mp[q] = make_float4(m[4*q], m[4*q+1], m[4*q+2], m[4*q+3]);
-      up[q] = make_float4(u[4*q], u[4*q+1], u[4*q+2], u[4*q+3]);
+      const int row = 16 * half + 4 * q + a;
+      const int o = o_first + row;
+      if (col_ok && o < p.M) {
+        const long long e = (long long)o * p.N + kcol;
+        const float4 g4 = lds128(stg + (uint32_t)row * 128u + (uint32_t)((b ^ (row & 7)) << 4));
+        const float G[4] = {g4.x, g4.y, g4.z, g4.w};
+        const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+        const float sbeta = __fmul_rn(faar_e4m3_to_float(sb[q]), s_global) * p.beta;
+        float g[4], vn[4], mn[4], un[4];
+        float mm[4], uu[4];
+        if (OPT == 1) {
+          mm[0] = m[q].x; mm[1] = m[q].y; mm[2] = m[q].z; mm[3] = m[q].w;
+          uu[0] = u[q].x; uu[1] = u[q].y; uu[2] = u[q].z; uu[3] = u[q].w;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t nib = (cw[q] >> (4 * i)) & 0xFu;
+          const float z = fmaf(p.beta, vv[i], hb);
+          const float ex = __expf(-fabsf(z));
+          const float hs = __fdividef(1.0f, 1.0f + ex);
+          const float dh = ex * hs * hs;                                     // h (1 - h)
+          float chain = sbeta * width_of(nib & 7u) * dh;
+          chain = __uint_as_float(__float_as_uint(chain) ^ ((nib & 8u) << 28));   // sign of w
+          g[i] = fmaf(G[i], chain, p.lam_over_n * fmaf(-8.f, vv[i], 4.f));
+          const float t = fmaf(2.f, vv[i], -1.f);
+          rl += fmaf(-t, t, 1.f);
+          if (OPT == 1) {
+            mn[i] = fmaf(p.b1, mm[i], c1 * g[i]);
+            un[i] = fmaf(p.b2, uu[i], c2 * g[i] * g[i]);
+            const float den = sqrt_approx(un[i] * p.inv_bc2) + p.eps;
+            vn[i] = fmaf(-p.lr * p.inv_bc1, __fdividef(mn[i], den), vv[i]);
+          } else {
+            vn[i] = fmaf(-p.lr, g[i], vv[i]);
+          }
+          vn[i] = fminf(fmaxf(vn[i], 0.f), 1.f);
+        }
+        if (p.dV) *reinterpret_cast<float4*>(p.dV + e) = make_float4(g[0], g[1], g[2], g[3]);
+        if (OPT == 1) {
+          *reinterpret_cast<float4*>(p.adam_m + e) = make_float4(mn[0], mn[1], mn[2], mn[3]);
+          *reinterpret_cast<float4*>(p.adam_u + e) = make_float4(un[0], un[1], un[2], un[3]);
+        }
+        *reinterpret_cast<float4*>(p.V + e) = make_float4(vn[0], vn[1], vn[2], vn[3]);
+      }
     }
-  } else {
-#pragma unroll
-    for (int j = 0; j < 16; ++j) vn[j] = fmaf(-p.lr, g[j], v[j]);
   }
-  float4* vp = reinterpret_cast<float4*>(p.V + e);
-#pragma unroll
-  for (int q = 0; q < 4; ++q)
-    vp[q] = make_float4(fminf(fmaxf(vn[4*q], 0.f), 1.f), fminf(fmaxf(vn[4*q+1], 0.f), 1.f),
-                        fminf(fmaxf(vn[4*q+2], 0.f), 1.f), fminf(fmaxf(vn[4*q+3], 0.f), 1.f));
   return rl;
 }
 
@@ -298,8 +339,9 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - raw);
-  uint8_t* ctl = smem + Cfg::STAGES * Cfg::STAGE_BYTES;
-  const uint32_t ctl_u32 = base + Cfg::STAGES * Cfg::STAGE_BYTES;
+  const uint32_t epi_u32 = base + Cfg::STAGES * Cfg::STAGE_BYTES;
+  uint8_t* ctl = smem + Cfg::STAGES * Cfg::STAGE_BYTES + Cfg::EPI_BYTES;
+  const uint32_t ctl_u32 = epi_u32 + Cfg::EPI_BYTES;
   // control block: full[S], empty[S], tmem_full[2], tmem_empty[2], tmem base, abort flag
   auto full_bar = [&](int s) { return ctl_u32 + 8u * s; };
   auto empty_bar = [&](int s) { return ctl_u32 + 8u * (Cfg::STAGES + s); };
@@ -406,15 +448,33 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
       const int o = m0 + quarter * 32 + lane;
       const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+      if constexpr (MODE == FAAR_GEMM_BWD) {
+        const uint32_t stg = epi_u32 + (uint32_t)ew * EPI_WARP_BYTES;
 #pragma unroll 1
-      for (int c = col_begin; c < col_begin + BN / 2; c += 16) {
-        if (n0 + c >= p.N) break;                    // warp-uniform
-        uint32_t r[16];
-        tmem_ld16(trow + (uint32_t)c, r);
-        tmem_ld_wait();
-        if (MODE == FAAR_GEMM_REF) epi_ref(p, o, n0 + c, r);
-        else if (MODE == FAAR_GEMM_FWD) warp_acc += epi_fwd(p, o, n0 + c, r);
-        else warp_acc += epi_bwd(p, o, n0 + c, r, s_global);
+        for (int c = col_begin; c < col_begin + BN / 2; c += 32) {
+          if (n0 + c >= p.N) break;                    // warp-uniform
+          uint32_t r[32];
+          tmem_ld32(trow + (uint32_t)c, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            sts128(stg + (uint32_t)lane * 128u + (uint32_t)((u ^ (lane & 7)) << 4), r[4 * u], r[4 * u + 1], r[4 * u + 2],
+                   r[4 * u + 3]);
+          __syncwarp();
+          warp_acc += p.opt == 1 ? epi_bwd_block<1>(p, stg, lane, m0 + quarter * 32, n0 + c, s_global)
+                                 : epi_bwd_block<0>(p, stg, lane, m0 + quarter * 32, n0 + c, s_global);
+          __syncwarp();                                // the block is consumed before the next one lands
+        }
+      } else {
+#pragma unroll 1
+        for (int c = col_begin; c < col_begin + BN / 2; c += 16) {
+          if (n0 + c >= p.N) break;                    // warp-uniform
+          uint32_t r[16];
+          tmem_ld16(trow + (uint32_t)c, r);
+          tmem_ld_wait();
+          if (MODE == FAAR_GEMM_REF) epi_ref(p, o, n0 + c, r);
+          else warp_acc += epi_fwd(p, o, n0 + c, r);
+        }
       }
       tc_fence_before();
       __syncwarp();
