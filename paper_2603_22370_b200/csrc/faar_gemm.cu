@@ -1,55 +1,84 @@
 // Tensor-core kernels of the FAAR layer step for sm_100a.
 //
-// One persistent, warp-specialised kernel computes C[M,N] = A[M,Kc] * B[N,Kc]^T
-// for BF16 operands that both have the contraction dimension contiguous:
-//   warp 0      : TMA producer  (cp.async.bulk.tensor, 128-byte swizzle, 4-6 stage ring)
-//   warp 1      : MMA issuer    (tcgen05.mma kind::f16, 128 x BN x 16, FP32 accumulators in TMEM)
-//   warps 2..9  : epilogue      (tcgen05.ld, two accumulator buffers so the epilogue of one
-//                                tile overlaps the main loop of the next)
+// One persistent, warp-specialised kernel computes C[M,N] = A[M,Kc] * B[N,Kc]^T for BF16 operands that
+// both have the contraction dimension contiguous.  It runs as clusters of two CTAs that share one
+// 256 x BN output tile (tcgen05 cta_group::2): CTA r of the pair loads rows [128 r, 128 r + 128) of the
+// A tile and rows [BN/2 r, BN/2 (r+1)) of the B tile into its own shared memory, the leader CTA (r = 0)
+// issues the 256 x BN x 16 MMAs for both, and each CTA ends up with its 128 accumulator rows x BN
+// columns (FP32) in its own tensor memory.  Halving the B tile per CTA halves the shared-memory
+// traffic per flop, which is what bounds a single-CTA 128 x 256 tile.
+//   warp 0      : TMA producer  (cp.async.bulk.tensor, 128-byte swizzle, multi-stage ring; both CTAs,
+//                                both crediting the leader's "full" barrier)
+//   warp 1      : MMA issuer    (leader CTA only; tcgen05.mma kind::f16, tcgen05.commit to the
+//                                "empty" / "accumulator full" barriers of both CTAs)
+//   warps 2..   : epilogue      (tcgen05.ld; two accumulator buffers, so the epilogue of one tile
+//                                overlaps the main loop of the next)
 // The three epilogues are the operations of the layer step:
 //   REF : Y_fp = X W^T                                   (Procedure step 8)
 //   FWD : r = Y_q - Y_ref, sum r^2, dY = 2c r -> dY^T     (steps 9-10, Eq. 5 first term)
 //   BWD : G = dY^T X -> dV -> optimiser update + clip     (step 13, Eq. 5, with Eq. 2/3 chain rule)
 // In all of them the accumulator row (TMEM lane) is the output feature o.
 //
-// Every wait on an mbarrier is bounded: after about two seconds the waiting
-// thread records a code in the status word, raises a CTA-wide abort flag and
-// every role leaves its loop; the CTA then frees its tensor memory and exits.
+// Every wait on an mbarrier is bounded: after about two seconds the waiting thread records a code in
+// the status word, raises a CTA-wide abort flag and every role leaves its loop; both CTAs then meet at
+// the closing cluster barrier, free their tensor memory and exit.
 #include <cuda.h>
 
 #include "faar_internal.cuh"
 
 namespace {
 
-constexpr int BM = 128;
+constexpr int BM = 128;                // accumulator rows per CTA; the CTA pair covers 256
 constexpr int BK = 64;                 // 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
-constexpr int NUM_EPI_WARPS = 8;
-constexpr int NUM_THREADS = 32 * (2 + NUM_EPI_WARPS);
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 constexpr int EPI_WARP_BYTES = 32 * 32 * 4;   // one 32 x 32 FP32 accumulator block per epilogue warp
+constexpr int SMEM_LIMIT = 227 * 1024;
+constexpr int CTL_BYTES = 512;
+constexpr int MAX_EPI_WARPS = 16;
 
-template <int BN> struct TileCfg {
-  static constexpr int STAGES = BN == 256 ? 4 : 6;
+template <int MODE, int BN> struct Cfg {
+  static constexpr int EPI_WARPS = MODE == FAAR_GEMM_BWD ? 16 : 8;
+  static constexpr int THREADS = 32 * (2 + EPI_WARPS);
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = (BN / 2) * BK * 2;            // this CTA's half of the B tile
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int EPI_BYTES = MODE == FAAR_GEMM_BWD ? EPI_WARPS * EPI_WARP_BYTES : 0;
+  static constexpr int FIT = (SMEM_LIMIT - 1024 - CTL_BYTES - EPI_BYTES) / STAGE_BYTES;
+  static constexpr int STAGES = FIT > 8 ? 8 : FIT;
   static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
-  static constexpr int EPI_BYTES = NUM_EPI_WARPS * EPI_WARP_BYTES;   // BWD: per-warp transposition buffers
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int COL_GROUPS = EPI_WARPS / 4;             // warps sharing one TMEM lane quarter
+  static constexpr int COLS_PER_WARP = BN / COL_GROUPS;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + CTL_BYTES;
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address, in CTA `rank` of the cluster, of the object that sits at shared::cta address `addr` here
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+// arrive on a barrier given by its shared::cluster address (this CTA's or the peer's)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t done;
@@ -62,7 +91,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
 
@@ -91,31 +120,36 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
   return mbar_wait_slow(bar, parity, ac, code);
 }
 
+// 2-D tiled TMA load into this CTA's shared memory; the byte count is credited to `bar`, which may be
+// a barrier of either CTA of the pair (shared::cluster address).  No multicast.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// When all MMAs issued so far have completed, arrive on the barrier at offset `bar` in both CTAs.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
 }
 __device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
                                             uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -135,6 +169,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -143,7 +178,6 @@ __device__ __forceinline__ float4 lds128(uint32_t addr) {
   asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
   return v;
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: rows of 64 bf16 (128 B) with 128-byte swizzle, contraction
 // dimension contiguous; groups of 8 rows are 1024 B apart.
@@ -156,9 +190,9 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                          // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: D = F32, A = B = BF16, both K-major, M = 128, N = BN.
+// Instruction descriptor: D = F32, A = B = BF16, both K-major, M = 256 (the CTA pair), N = BN.
 template <int BN> __device__ __forceinline__ constexpr uint32_t make_idesc() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 }
 
 struct KParams {
@@ -170,7 +204,7 @@ struct KParams {
   __nv_bfloat16* dYt; long long ld_dyt;
   float mse2c;
   float* partials;
-  // BWD
+  // BWD: M = O, N = K
   float* V; const uint8_t* code; const uint8_t* scales; const float* s_global;
   float* adam_m; float* adam_u; float* dV;
   float beta, lam_over_n, lr, b1, b2, eps, inv_bc1, inv_bc2; int opt;
@@ -239,11 +273,7 @@ __device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const 
   return ss;
 }
 
-// BWD.  A warp's 32 x 32 block of G (row = output feature o, column = input feature k) has been
-// staged in shared memory, row r at stg + 128 r, its eight 16-byte units XOR-swizzled by (r & 7).
-// Here lane (a, b) = (lane / 8, lane % 8) handles, in pass q, row 4q + a and columns 4b..4b+3, so
-// that eight lanes cover 128 contiguous bytes of a row of V / m / u and every global access is a
-// full line.  Returns the Round Loss contribution of the pre-update v's.
+// ---- BWD epilogue ----------------------------------------------------------------------------
 __device__ __forceinline__ float sqrt_approx(float x) {       // sqrt(0) = 0, about 1 ulp
   float y;
   asm("sqrt.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -253,39 +283,54 @@ __device__ __forceinline__ float width_of(uint32_t k) {       // interval widths
   return __uint_as_float((126u + ((0x2500u >> (2u * k)) & 3u)) << 23);
 }
 
-template <int OPT>
+// A warp's 32 x 32 block of G (row = output feature o, column = input feature k) has been staged in
+// shared memory, row r at stg + 128 r, its eight 16-byte units XOR-swizzled by (r & 7).  Lane
+// (a, b) = (lane / 8, lane % 8) handles, in pass q = 0..7, row 4q + a and columns 4b..4b+3, so that
+// eight lanes cover 128 contiguous bytes of a row of V / m / u and every global access is a full
+// line moved as 16-byte vectors.  The per-weight state of two passes is requested together before
+// either is computed.  FULL: the block lies wholly inside the matrix (no bounds tests).
+// Returns the Round Loss contribution of the pre-update v's.
+template <int OPT, bool FULL>
 __device__ __forceinline__ float epi_bwd_block(const KParams& p, uint32_t stg, int lane, int o_first, int k_first,
                                                float s_global) {
   const int a = lane >> 3, b = lane & 7;
   const int kcol = k_first + 4 * b;
-  const bool col_ok = kcol < p.N;
+  const bool col_ok = FULL || kcol < p.N;
+  const long long e0 = (long long)(o_first + a) * p.N + kcol;     // pass 0 element of this lane
+  float* const Vp = p.V + e0;
+  float* const Mp = p.adam_m + e0;
+  float* const Up = p.adam_u + e0;
+  const uint8_t* const Cp = p.code + (e0 >> 1);
+  const uint8_t* const Sp = p.scales + (e0 >> 4);
   const float hb = -0.5f * p.beta;
   const float c1 = 1.f - p.b1, c2 = 1.f - p.b2;
+  const float step_size = p.lr * p.inv_bc1;
   float rl = 0.f;
 #pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    float4 v[4], m[4], u[4];
-    uint32_t cw[4], sb[4];
+  for (int grp = 0; grp < 4; ++grp) {
+    float4 v[2], m[2], u[2];
+    uint32_t cw[2], sb[2];
+    bool ok[2];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int o = o_first + 16 * half + 4 * q + a;
-      if (col_ok && o < p.M) {
-        const long long e = (long long)o * p.N + kcol;
-        v[q] = *reinterpret_cast<const float4*>(p.V + e);
-        cw[q] = *reinterpret_cast<const uint16_t*>(p.code + (e >> 1));
-        sb[q] = p.scales[e >> 4];
+    for (int q = 0; q < 2; ++q) {
+      const int row = 8 * grp + 4 * q + a;
+      ok[q] = FULL || (col_ok && o_first + row < p.M);
+      if (ok[q]) {
+        const int off = (8 * grp + 4 * q) * p.N;                    // rows below pass 0, in elements
+        v[q] = *reinterpret_cast<const float4*>(Vp + off);
+        cw[q] = *reinterpret_cast<const uint16_t*>(Cp + (off >> 1));
+        sb[q] = Sp[off >> 4];
         if (OPT == 1) {
-          m[q] = *reinterpret_cast<const float4*>(p.adam_m + e);
-          u[q] = *reinterpret_cast<const float4*>(p.adam_u + e);
+          m[q] = *reinterpret_cast<const float4*>(Mp + off);
+          u[q] = *reinterpret_cast<const float4*>(Up + off);
         }
       }
     }
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int row = 16 * half + 4 * q + a;
-      const int o = o_first + row;
-      if (col_ok && o < p.M) {
-        const long long e = (long long)o * p.N + kcol;
+    for (int q = 0; q < 2; ++q) {
+      if (ok[q]) {
+        const int row = 8 * grp + 4 * q + a;
+        const int off = (8 * grp + 4 * q) * p.N;
         const float4 g4 = lds128(stg + (uint32_t)row * 128u + (uint32_t)((b ^ (row & 7)) << 4));
         const float G[4] = {g4.x, g4.y, g4.z, g4.w};
         const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
@@ -312,18 +357,18 @@ __device__ __forceinline__ float epi_bwd_block(const KParams& p, uint32_t stg, i
             mn[i] = fmaf(p.b1, mm[i], c1 * g[i]);
             un[i] = fmaf(p.b2, uu[i], c2 * g[i] * g[i]);
             const float den = sqrt_approx(un[i] * p.inv_bc2) + p.eps;
-            vn[i] = fmaf(-p.lr * p.inv_bc1, __fdividef(mn[i], den), vv[i]);
+            vn[i] = fmaf(-step_size, __fdividef(mn[i], den), vv[i]);
           } else {
             vn[i] = fmaf(-p.lr, g[i], vv[i]);
           }
           vn[i] = fminf(fmaxf(vn[i], 0.f), 1.f);
         }
-        if (p.dV) *reinterpret_cast<float4*>(p.dV + e) = make_float4(g[0], g[1], g[2], g[3]);
+        if (p.dV) *reinterpret_cast<float4*>(p.dV + e0 + off) = make_float4(g[0], g[1], g[2], g[3]);
         if (OPT == 1) {
-          *reinterpret_cast<float4*>(p.adam_m + e) = make_float4(mn[0], mn[1], mn[2], mn[3]);
-          *reinterpret_cast<float4*>(p.adam_u + e) = make_float4(un[0], un[1], un[2], un[3]);
+          *reinterpret_cast<float4*>(Mp + off) = make_float4(mn[0], mn[1], mn[2], mn[3]);
+          *reinterpret_cast<float4*>(Up + off) = make_float4(un[0], un[1], un[2], un[3]);
         }
-        *reinterpret_cast<float4*>(p.V + e) = make_float4(vn[0], vn[1], vn[2], vn[3]);
+        *reinterpret_cast<float4*>(Vp + off) = make_float4(vn[0], vn[1], vn[2], vn[3]);
       }
     }
   }
@@ -331,81 +376,85 @@ __device__ __forceinline__ float epi_bwd_block(const KParams& p, uint32_t stg, i
 }
 
 // ---- the kernel ------------------------------------------------------------------------------
-template <int MODE, int BN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+// Launched as clusters of two CTAs along x: CTAs 2c and 2c+1 form pair c.
+template <int MODE, int BN, int OPT>
+__global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1)
 faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const KParams p) {
-  using Cfg = TileCfg<BN>;
+  using C = Cfg<MODE, BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t base = (raw + 1023u) & ~1023u;       // the same offset in both CTAs of the pair
   uint8_t* smem = smem_raw + (base - raw);
-  const uint32_t epi_u32 = base + Cfg::STAGES * Cfg::STAGE_BYTES;
-  uint8_t* ctl = smem + Cfg::STAGES * Cfg::STAGE_BYTES + Cfg::EPI_BYTES;
-  const uint32_t ctl_u32 = epi_u32 + Cfg::EPI_BYTES;
+  const uint32_t epi_u32 = base + C::STAGES * C::STAGE_BYTES;
+  uint8_t* ctl = smem + C::STAGES * C::STAGE_BYTES + C::EPI_BYTES;
+  const uint32_t ctl_u32 = epi_u32 + C::EPI_BYTES;
   // control block: full[S], empty[S], tmem_full[2], tmem_empty[2], tmem base, abort flag
   auto full_bar = [&](int s) { return ctl_u32 + 8u * s; };
-  auto empty_bar = [&](int s) { return ctl_u32 + 8u * (Cfg::STAGES + s); };
-  auto tfull_bar = [&](int a) { return ctl_u32 + 8u * (2 * Cfg::STAGES + a); };
-  auto tempty_bar = [&](int a) { return ctl_u32 + 8u * (2 * Cfg::STAGES + 2 + a); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctl + 8 * (2 * Cfg::STAGES + 4));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + 8 * (2 * Cfg::STAGES + 4) + 4);
+  auto empty_bar = [&](int s) { return ctl_u32 + 8u * (C::STAGES + s); };
+  auto tfull_bar = [&](int a) { return ctl_u32 + 8u * (2 * C::STAGES + a); };
+  auto tempty_bar = [&](int a) { return ctl_u32 + 8u * (2 * C::STAGES + 2 + a); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctl + 8 * (2 * C::STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + 8 * (2 * C::STAGES + 4) + 4);
   const AbortCtl ac{abort_flag, p.status};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tiles = (p.M + BM - 1) / BM, n_tiles = (p.N + BN - 1) / BN;
+  const uint32_t rank = cluster_ctarank();             // 0 = leader of the pair
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM), n_tiles = (p.N + BN - 1) / BN;
   const int total_tiles = m_tiles * n_tiles;
   const int k_blocks = (p.Kc + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < Cfg::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), NUM_EPI_WARPS); }
+    for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    // accumulator-empty barriers are used in the leader only: every epilogue warp of both CTAs arrives there
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * C::EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
-  __syncthreads();
+  cluster_sync_all();                                  // barriers of both CTAs are initialised
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ---------------- TMA producer ----------------
+    // ---------------- TMA producer (both CTAs) ----------------
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+        const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;
+        const int n0 = (tile / m_tiles) * BN + (int)rank * (BN / 2);
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(empty_bar(stage), phase ^ 1u, ac, 0x100u | stage);
           if (!ok) break;
-          const uint32_t sa = base + stage * Cfg::STAGE_BYTES, sb = sa + Cfg::A_BYTES;
-          mbar_expect_tx(full_bar(stage), Cfg::STAGE_BYTES);
-          tma_load_2d(sa, &tmA, kb * BK, m0, full_bar(stage));
-          tma_load_2d(sb, &tmB, kb * BK, n0, full_bar(stage));
-          if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+          const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+          // the leader's barrier collects the bytes of both CTAs' copies
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * C::STAGE_BYTES);
+          const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
+          tma_load_2d(sa, &tmA, kb * BK, m0, leader_full);
+          tma_load_2d(sb, &tmB, kb * BK, n0, leader_full);
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
         // give copies already in flight a bounded chance to land before the CTA exits
-        for (int s = 0; s < Cfg::STAGES; ++s) {
-          unsigned long long t0 = global_ns();
-          const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
-          while (!mbar_try_wait(full_bar(s), par) && global_ns() - t0 < 50000000ull) {}
-        }
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 2000000ull) {}
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = make_idesc<BN>();
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1;
         ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, ac, 0x200u | acc);
@@ -416,43 +465,44 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           ok = mbar_wait(full_bar(stage), phase, ac, 0x300u | stage);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t sa = base + stage * Cfg::STAGE_BYTES, sb = sa + Cfg::A_BYTES;
+          const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
           const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sb);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 bf16 = 32 bytes inside the swizzled row: +2 in the 16-byte address field
             tc_mma_bf16(tmem_d, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          tc_commit(empty_bar(stage));
-          if (++stage == Cfg::STAGES) { stage = 0; phase ^= 1u; }
+          tc_commit_pair(empty_bar(stage));            // frees this stage in both CTAs
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (ok) tc_commit(tfull_bar(acc));
+        if (ok) tc_commit_pair(tfull_bar(acc));        // accumulator ready in both CTAs
       }
     }
   } else {
-    // ---------------- epilogue ----------------
+    // ---------------- epilogue (both CTAs) ----------------
     const int ew = warp - 2;
-    const int quarter = warp & 3;                    // TMEM lanes this warp may read
-    const int col_begin = (ew >> 2) * (BN / 2);
+    const int quarter = warp & 3;                      // TMEM lanes this warp may read
+    const int col_begin = (ew >> 2) * C::COLS_PER_WARP;
     float warp_acc = 0.f;
     float s_global = 0.f;
     if (MODE == FAAR_GEMM_BWD) s_global = *p.s_global;
     int it = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+    for (int tile = pair; tile < total_tiles; tile += n_pairs, ++it) {
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, ac, 0x400u | acc);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+      const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM, n0 = (tile / m_tiles) * BN;
       const int o = m0 + quarter * 32 + lane;
       const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
       if constexpr (MODE == FAAR_GEMM_BWD) {
         const uint32_t stg = epi_u32 + (uint32_t)ew * EPI_WARP_BYTES;
+        const int o_first = m0 + quarter * 32;
 #pragma unroll 1
-        for (int c = col_begin; c < col_begin + BN / 2; c += 32) {
-          if (n0 + c >= p.N) break;                    // warp-uniform
+        for (int c = col_begin; c < col_begin + C::COLS_PER_WARP; c += 32) {
+          if (n0 + c >= p.N || o_first >= p.M) break;  // warp-uniform
           uint32_t r[32];
           tmem_ld32(trow + (uint32_t)c, r);
           tmem_ld_wait();
@@ -461,13 +511,15 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             sts128(stg + (uint32_t)lane * 128u + (uint32_t)((u ^ (lane & 7)) << 4), r[4 * u], r[4 * u + 1], r[4 * u + 2],
                    r[4 * u + 3]);
           __syncwarp();
-          warp_acc += p.opt == 1 ? epi_bwd_block<1>(p, stg, lane, m0 + quarter * 32, n0 + c, s_global)
-                                 : epi_bwd_block<0>(p, stg, lane, m0 + quarter * 32, n0 + c, s_global);
+          if (o_first + 32 <= p.M && n0 + c + 32 <= p.N)
+            warp_acc += epi_bwd_block<OPT, true>(p, stg, lane, o_first, n0 + c, s_global);
+          else
+            warp_acc += epi_bwd_block<OPT, false>(p, stg, lane, o_first, n0 + c, s_global);
           __syncwarp();                                // the block is consumed before the next one lands
         }
       } else {
 #pragma unroll 1
-        for (int c = col_begin; c < col_begin + BN / 2; c += 16) {
+        for (int c = col_begin; c < col_begin + C::COLS_PER_WARP; c += 16) {
           if (n0 + c >= p.N) break;                    // warp-uniform
           uint32_t r[16];
           tmem_ld16(trow + (uint32_t)c, r);
@@ -478,19 +530,22 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
     }
     if (MODE != FAAR_GEMM_REF) {
       warp_acc = faar_warp_sum(warp_acc);
-      if (lane == 0) p.partials[blockIdx.x * NUM_EPI_WARPS + ew] = warp_acc;
+      if (lane == 0) p.partials[blockIdx.x * C::EPI_WARPS + ew] = warp_acc;
     }
   }
 
+  __syncwarp();
+  // Neither CTA may leave while the other can still read its shared memory, write its tensor memory
+  // or arrive on its barriers.
   tc_fence_before();
-  __syncthreads();
+  cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
 
@@ -512,31 +567,61 @@ int make_map(faar_ctx* ctx, CUtensorMap* map, const void* ptr, int rows, int col
   return r == CUDA_SUCCESS ? 0 : (int)cudaErrorInvalidValue;
 }
 
-template <int MODE, int BN>
-int launch(faar_ctx* ctx, const faar_gemm_args* a, const KParams& kp, int grid) {
-  using Cfg = TileCfg<BN>;
+template <int MODE, int BN, int OPT = 0>
+int launch(faar_ctx* ctx, const faar_gemm_args* a, const KParams& kp, int* n_partials_out) {
+  using C = Cfg<MODE, BN>;
+  static_assert(C::STAGES >= 3, "ring too short");
+  static_assert(C::SMEM_BYTES <= SMEM_LIMIT, "shared memory budget");
+  static_assert(C::EPI_WARPS <= MAX_EPI_WARPS, "partials budget");
   CUtensorMap tmA, tmB;
   int e = make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
   if (e) return e;
-  e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, BN);
+  e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, BN / 2);
   if (e) return e;
-  auto kern = faar_gemm_kernel<MODE, BN>;
-  cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+  auto kern = faar_gemm_kernel<MODE, BN, OPT>;
+  cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (ce != cudaSuccess) return (int)ce;
+
+  const long long tiles = (long long)((a->M + 2 * BM - 1) / (2 * BM)) * ((a->N + BN - 1) / BN);
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(C::THREADS, 1, 1);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = ctx->stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  // how many CTA pairs the device can hold at once (a GPC with an odd SM count strands one SM)
+  static int max_pairs = 0;                      // per kernel instantiation
+  if (max_pairs == 0) {
+    cfg.gridDim = dim3(2 * (ctx->num_sms / 2), 1, 1);
+    int n = 0;
+    ce = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+    if (ce != cudaSuccess || n <= 0) { (void)cudaGetLastError(); n = ctx->num_sms / 2; }
+    if (n > ctx->num_sms / 2) n = ctx->num_sms / 2;
+    max_pairs = n;
+  }
+  const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  if (n_partials_out) *n_partials_out = 2 * pairs * C::EPI_WARPS;
   faar_prof_scope ps(ctx, MODE == FAAR_GEMM_REF ? FAAR_K_GEMM_REF : (MODE == FAAR_GEMM_FWD ? FAAR_K_GEMM_FWD : FAAR_K_GEMM_BWD));
-  kern<<<grid, NUM_THREADS, Cfg::SMEM_BYTES, ctx->stream>>>(tmA, tmB, kp);
+  ce = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, kp);
+  if (ce != cudaSuccess) return (int)ce;
   return (int)cudaGetLastError();
 }
 
 int pick_bn(const faar_ctx* ctx, int M, int N) {
   // the wide tile unless it leaves most SMs idle
-  long long tiles256 = (long long)((M + BM - 1) / BM) * ((N + 255) / 256);
-  return tiles256 >= ctx->num_sms ? 256 : 128;
+  long long tiles256 = (long long)((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
+  return tiles256 >= ctx->num_sms / 2 ? 256 : 128;
 }
 
 }  // namespace
 
-int faar_gemm_max_partials(const faar_ctx* ctx, int, int) { return ctx->num_sms * NUM_EPI_WARPS; }
+int faar_gemm_max_partials(const faar_ctx* ctx, int, int) { return ctx->num_sms * MAX_EPI_WARPS; }
 
 int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out) {
   KParams kp;
@@ -548,18 +633,21 @@ int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out
   kp.adam_m = a->adam_m; kp.adam_u = a->adam_u; kp.dV = a->dV;
   kp.beta = a->beta; kp.lam_over_n = a->lam_over_n; kp.lr = a->lr; kp.b1 = a->b1; kp.b2 = a->b2; kp.eps = a->eps;
   kp.inv_bc1 = a->inv_bc1; kp.inv_bc2 = a->inv_bc2; kp.opt = a->opt;
+  // the BWD epilogue forms row offsets of up to 28 rows in 32-bit element counts
+  if (a->mode == FAAR_GEMM_BWD && (long long)a->N * 32 > 0x7FFFFFFFll) return (int)cudaErrorInvalidValue;
 
   const int bn = pick_bn(ctx, a->M, a->N);
-  const long long tiles = (long long)((a->M + BM - 1) / BM) * ((a->N + bn - 1) / bn);
-  const int grid = (int)(tiles < ctx->num_sms ? tiles : ctx->num_sms);
-  if (n_partials_out) *n_partials_out = grid * NUM_EPI_WARPS;
   switch (a->mode * 2 + (bn == 256 ? 1 : 0)) {
-    case FAAR_GEMM_REF * 2 + 0: return launch<FAAR_GEMM_REF, 128>(ctx, a, kp, grid);
-    case FAAR_GEMM_REF * 2 + 1: return launch<FAAR_GEMM_REF, 256>(ctx, a, kp, grid);
-    case FAAR_GEMM_FWD * 2 + 0: return launch<FAAR_GEMM_FWD, 128>(ctx, a, kp, grid);
-    case FAAR_GEMM_FWD * 2 + 1: return launch<FAAR_GEMM_FWD, 256>(ctx, a, kp, grid);
-    case FAAR_GEMM_BWD * 2 + 0: return launch<FAAR_GEMM_BWD, 128>(ctx, a, kp, grid);
-    case FAAR_GEMM_BWD * 2 + 1: return launch<FAAR_GEMM_BWD, 256>(ctx, a, kp, grid);
+    case FAAR_GEMM_REF * 2 + 0: return launch<FAAR_GEMM_REF, 128>(ctx, a, kp, n_partials_out);
+    case FAAR_GEMM_REF * 2 + 1: return launch<FAAR_GEMM_REF, 256>(ctx, a, kp, n_partials_out);
+    case FAAR_GEMM_FWD * 2 + 0: return launch<FAAR_GEMM_FWD, 128>(ctx, a, kp, n_partials_out);
+    case FAAR_GEMM_FWD * 2 + 1: return launch<FAAR_GEMM_FWD, 256>(ctx, a, kp, n_partials_out);
+    case FAAR_GEMM_BWD * 2 + 0:
+      return a->opt == 1 ? launch<FAAR_GEMM_BWD, 128, 1>(ctx, a, kp, n_partials_out)
+                         : launch<FAAR_GEMM_BWD, 128, 0>(ctx, a, kp, n_partials_out);
+    case FAAR_GEMM_BWD * 2 + 1:
+      return a->opt == 1 ? launch<FAAR_GEMM_BWD, 256, 1>(ctx, a, kp, n_partials_out)
+                         : launch<FAAR_GEMM_BWD, 256, 0>(ctx, a, kp, n_partials_out);
   }
   return (int)cudaErrorInvalidValue;
 }
