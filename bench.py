@@ -175,7 +175,7 @@ def run_ours(args):
     import torch
 
     from paper_2603_22370_b200 import build as faar_build
-    from paper_2603_22370_b200 import faar, inputs
+    from paper_2603_22370_b200 import faar, inputs, shard
 
     rank, local_rank, world = dist_env()
     n_gpus = args.gpus
@@ -252,11 +252,7 @@ def run_ours(args):
         stream.synchronize()
         barrier()
         w1 = time.time()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        _, ms = shard.job_rate(1.0, e0.elapsed_time(e1), device)     # max over ranks
         if sampler:
             sampler.window(w0, w1)
         return ms
