@@ -141,23 +141,27 @@ __device__ __forceinline__ uint32_t faar_float_to_e4m3(float q) {
   return (e << 3) | m;
 }
 
-// Eq. 3 in FP32, accurate to about one ulp over the whole range of h.
-// The argument beta*(v-0.5) is formed as an unevaluated sum hi + lo so that the
-// relative error of h stays near one ulp even where h is tiny.
+// Eq. 3 in FP32 with a relative error of a few 1e-7 over the whole range of h, also where h is tiny.
+// z = beta*(v-0.5) is kept as an unevaluated sum (v-0.5 is exact or off by < 2^-26; the product's
+// rounding error is recovered with one FMA), -|z|*log2(e) likewise, so the argument of the hardware
+// 2^x carries no error that grows with |z|; the low parts enter as a first-order correction.
 __device__ __forceinline__ float faar_sigmoid_precise(float beta, float v) {
-  float p = __fmul_rn(beta, v);
-  float pe = __fmaf_rn(beta, v, -p);          // exact error of the product
-  float c = 0.5f * beta;                      // exact
-  float hi = __fsub_rn(p, c);
-  float bb = __fsub_rn(hi, p);                // two-sum of p + (-c)
-  float lo = __fadd_rn(__fsub_rn(p, __fsub_rn(hi, bb)), __fsub_rn(-c, bb));
-  lo = __fadd_rn(lo, pe);
-  // h = 1 / (1 + exp(-(hi+lo)));  exp(-(hi+lo)) = exp(-hi) * (1 - lo + ...)
-  float e = expf(-fabsf(hi));
-  float adj = hi >= 0.f ? -lo : lo;           // exp(-|hi| - sign*lo)
-  e = __fmaf_rn(e, adj, e);
-  float hs = __fdiv_rn(1.0f, 1.0f + e);       // sigmoid(|z|)
-  return hi >= 0.f ? hs : __fmul_rn(e, hs);   // sigmoid(-|z|) = e / (1 + e)
+  const float d = __fsub_rn(v, 0.5f);
+  const float zh = __fmul_rn(beta, d);
+  const float zl = __fmaf_rn(beta, d, -zh);              // exact error of the product
+  const float az = -fabsf(zh);
+  const float sl = zh >= 0.f ? -zl : zl;                  // low part of -|z| (sign follows zh)
+  const float L1 = 1.4426950216293335f;                   // float(log2 e)
+  const float L2 = 1.9259629911266175e-8f;                // log2 e - L1
+  const float th = __fmul_rn(az, L1);
+  float tl = __fmaf_rn(az, L1, -th);
+  tl = __fmaf_rn(az, L2, tl);
+  tl = __fmaf_rn(sl, L1, tl);
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(th));
+  e = __fmaf_rn(e, tl * 0.6931471805599453f, e);          // 2^(th+tl) = 2^th (1 + tl ln 2)
+  const float hs = __fdividef(1.0f, 1.0f + e);            // sigmoid(|z|)
+  return zh >= 0.f ? hs : __fmul_rn(e, hs);               // sigmoid(-|z|) = e / (1 + e)
 }
 
 // Eq. 2 in FP32: sign * (lo + h * (hi - lo)) * s for the nibble (sign<<3 | k).
