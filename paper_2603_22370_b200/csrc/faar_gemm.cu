@@ -32,7 +32,7 @@ constexpr int BM = 128;                // accumulator rows per CTA; the CTA pair
 constexpr int BK = 64;                 // 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
-constexpr int EPI_WARP_BYTES = 32 * 32 * 4;   // one 32 x 32 FP32 accumulator block per epilogue warp
+constexpr int PANEL_BYTES = 32 * 128 * 4;      // BWD epilogue: one 32-row x 128-column FP32 panel per TMEM lane quarter
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int CTL_BYTES = 512;
 constexpr int MAX_EPI_WARPS = 16;
@@ -43,7 +43,7 @@ template <int MODE, int BN> struct Cfg {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = (BN / 2) * BK * 2;            // this CTA's half of the B tile
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int EPI_BYTES = MODE == FAAR_GEMM_BWD ? EPI_WARPS * EPI_WARP_BYTES : 0;
+  static constexpr int EPI_BYTES = MODE == FAAR_GEMM_BWD ? 4 * PANEL_BYTES : 0;
   static constexpr int FIT = (SMEM_LIMIT - 1024 - CTL_BYTES - EPI_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = FIT > 8 ? 8 : FIT;
   static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
@@ -72,6 +72,9 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -122,10 +125,34 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
 
 // 2-D tiled TMA load into this CTA's shared memory; the byte count is credited to `bar`, which may be
 // a barrier of either CTA of the pair (shared::cluster address).  No multicast.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
+                                            uint64_t l2_policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(l2_policy) : "memory");
+}
+// L2 eviction policies: GEMM operands are re-read by many CTAs and should stay; the per-weight
+// optimiser state streams through once per step and should be the first to go.
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_stream() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ float4 ldg128_stream(const float* ptr, uint64_t pol) {
+  float4 v;
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr), "l"(pol));
+  return v;
+}
+__device__ __forceinline__ void stg128_stream(float* ptr, float a, float b, float c, float d, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(ptr), "f"(a), "f"(b), "f"(c), "f"(d), "l"(pol)
+               : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -283,20 +310,21 @@ __device__ __forceinline__ float width_of(uint32_t k) {       // interval widths
   return __uint_as_float((126u + ((0x2500u >> (2u * k)) & 3u)) << 23);
 }
 
-// A warp's 32 x 32 block of G (row = output feature o, column = input feature k) has been staged in
-// shared memory, row r at stg + 128 r, its eight 16-byte units XOR-swizzled by (r & 7).  Lane
-// (a, b) = (lane / 8, lane % 8) handles, in pass q = 0..7, row 4q + a and columns 4b..4b+3, so that
-// eight lanes cover 128 contiguous bytes of a row of V / m / u and every global access is a full
-// line moved as 16-byte vectors.  The per-weight state of two passes is requested together before
-// either is computed.  FULL: the block lies wholly inside the matrix (no bounds tests).
+// The four epilogue warps that share a TMEM lane quarter stage a 32-row x 128-column panel of G in
+// shared memory (row r at panel + 512 r, its 16-byte units XOR-swizzled by (r & 7)); then warp `sub`
+// of the quarter takes rows 8 sub .. 8 sub + 7 and lane l the columns 4l..4l+3, so that one warp
+// instruction moves 512 contiguous bytes of one row of V / m / u: long bursts for the HBM, full lines
+// as 16-byte vectors.  The per-weight state of two rows is requested together before either is
+// computed.  FULL: the panel lies wholly inside the matrix (no bounds tests).
+// o_first: output feature of panel row 0; k_first: input feature of panel column 0.
 // Returns the Round Loss contribution of the pre-update v's.
 template <int OPT, bool FULL>
-__device__ __forceinline__ float epi_bwd_block(const KParams& p, uint32_t stg, int lane, int o_first, int k_first,
-                                               float s_global) {
-  const int a = lane >> 3, b = lane & 7;
-  const int kcol = k_first + 4 * b;
+__device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, int lane, int sub, int o_first,
+                                              int k_first, float s_global) {
+  const int kcol = k_first + 4 * lane;
   const bool col_ok = FULL || kcol < p.N;
-  const long long e0 = (long long)(o_first + a) * p.N + kcol;     // pass 0 element of this lane
+  const int r0 = 8 * sub;
+  const long long e0 = (long long)(o_first + r0) * p.N + kcol;     // row r0 element of this lane
   float* const Vp = p.V + e0;
   float* const Mp = p.adam_m + e0;
   float* const Up = p.adam_u + e0;
@@ -305,6 +333,7 @@ __device__ __forceinline__ float epi_bwd_block(const KParams& p, uint32_t stg, i
   const float hb = -0.5f * p.beta;
   const float c1 = 1.f - p.b1, c2 = 1.f - p.b2;
   const float step_size = p.lr * p.inv_bc1;
+  const uint64_t stream = l2_policy_stream();
   float rl = 0.f;
 #pragma unroll
   for (int grp = 0; grp < 4; ++grp) {
@@ -313,25 +342,26 @@ __device__ __forceinline__ float epi_bwd_block(const KParams& p, uint32_t stg, i
     bool ok[2];
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
-      const int row = 8 * grp + 4 * q + a;
-      ok[q] = FULL || (col_ok && o_first + row < p.M);
+      const int i = 2 * grp + q;                                      // row r0 + i
+      ok[q] = FULL || (col_ok && o_first + r0 + i < p.M);
       if (ok[q]) {
-        const int off = (8 * grp + 4 * q) * p.N;                    // rows below pass 0, in elements
-        v[q] = *reinterpret_cast<const float4*>(Vp + off);
+        const int off = i * p.N;
+        v[q] = ldg128_stream(Vp + off, stream);
         cw[q] = *reinterpret_cast<const uint16_t*>(Cp + (off >> 1));
         sb[q] = Sp[off >> 4];
         if (OPT == 1) {
-          m[q] = *reinterpret_cast<const float4*>(Mp + off);
-          u[q] = *reinterpret_cast<const float4*>(Up + off);
+          m[q] = ldg128_stream(Mp + off, stream);
+          u[q] = ldg128_stream(Up + off, stream);
         }
       }
     }
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
       if (ok[q]) {
-        const int row = 8 * grp + 4 * q + a;
-        const int off = (8 * grp + 4 * q) * p.N;
-        const float4 g4 = lds128(stg + (uint32_t)row * 128u + (uint32_t)((b ^ (row & 7)) << 4));
+        const int i = 2 * grp + q;
+        const int row = r0 + i;
+        const int off = i * p.N;
+        const float4 g4 = lds128(panel + (uint32_t)row * 512u + (uint32_t)((lane ^ (row & 7)) << 4));
         const float G[4] = {g4.x, g4.y, g4.z, g4.w};
         const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
         const float sbeta = __fmul_rn(faar_e4m3_to_float(sb[q]), s_global) * p.beta;
@@ -342,33 +372,33 @@ __device__ __forceinline__ float epi_bwd_block(const KParams& p, uint32_t stg, i
           uu[0] = u[q].x; uu[1] = u[q].y; uu[2] = u[q].z; uu[3] = u[q].w;
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint32_t nib = (cw[q] >> (4 * i)) & 0xFu;
-          const float z = fmaf(p.beta, vv[i], hb);
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t nib = (cw[q] >> (4 * j)) & 0xFu;
+          const float z = fmaf(p.beta, vv[j], hb);
           const float ex = __expf(-fabsf(z));
           const float hs = __fdividef(1.0f, 1.0f + ex);
           const float dh = ex * hs * hs;                                     // h (1 - h)
           float chain = sbeta * width_of(nib & 7u) * dh;
           chain = __uint_as_float(__float_as_uint(chain) ^ ((nib & 8u) << 28));   // sign of w
-          g[i] = fmaf(G[i], chain, p.lam_over_n * fmaf(-8.f, vv[i], 4.f));
-          const float t = fmaf(2.f, vv[i], -1.f);
+          g[j] = fmaf(G[j], chain, p.lam_over_n * fmaf(-8.f, vv[j], 4.f));
+          const float t = fmaf(2.f, vv[j], -1.f);
           rl += fmaf(-t, t, 1.f);
           if (OPT == 1) {
-            mn[i] = fmaf(p.b1, mm[i], c1 * g[i]);
-            un[i] = fmaf(p.b2, uu[i], c2 * g[i] * g[i]);
-            const float den = sqrt_approx(un[i] * p.inv_bc2) + p.eps;
-            vn[i] = fmaf(-step_size, __fdividef(mn[i], den), vv[i]);
+            mn[j] = fmaf(p.b1, mm[j], c1 * g[j]);
+            un[j] = fmaf(p.b2, uu[j], c2 * g[j] * g[j]);
+            const float den = sqrt_approx(un[j] * p.inv_bc2) + p.eps;
+            vn[j] = fmaf(-step_size, __fdividef(mn[j], den), vv[j]);
           } else {
-            vn[i] = fmaf(-p.lr, g[i], vv[i]);
+            vn[j] = fmaf(-p.lr, g[j], vv[j]);
           }
-          vn[i] = fminf(fmaxf(vn[i], 0.f), 1.f);
+          vn[j] = fminf(fmaxf(vn[j], 0.f), 1.f);
         }
-        if (p.dV) *reinterpret_cast<float4*>(p.dV + e0 + off) = make_float4(g[0], g[1], g[2], g[3]);
+        if (p.dV) stg128_stream(p.dV + e0 + off, g[0], g[1], g[2], g[3], stream);
         if (OPT == 1) {
-          *reinterpret_cast<float4*>(Mp + off) = make_float4(mn[0], mn[1], mn[2], mn[3]);
-          *reinterpret_cast<float4*>(Up + off) = make_float4(un[0], un[1], un[2], un[3]);
+          stg128_stream(Mp + off, mn[0], mn[1], mn[2], mn[3], stream);
+          stg128_stream(Up + off, un[0], un[1], un[2], un[3], stream);
         }
-        *reinterpret_cast<float4*>(Vp + off) = make_float4(vn[0], vn[1], vn[2], vn[3]);
+        stg128_stream(Vp + off, vn[0], vn[1], vn[2], vn[3], stream);
       }
     }
   }
@@ -408,6 +438,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     // accumulator-empty barriers are used in the leader only: every epilogue warp of both CTAs arrives there
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * C::EPI_WARPS); }
+    for (int q = 0; q < 8; ++q) mbar_init(ctl_u32 + 256u + 8u * q, 4);   // panel staged / panel consumed, per lane quarter
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -424,6 +455,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   if (warp == 0) {
     // ---------------- TMA producer (both CTAs) ----------------
     if (lane == 0) {
+      const uint64_t keep = l2_policy_keep();
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
@@ -436,8 +468,8 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           // the leader's barrier collects the bytes of both CTAs' copies
           if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * C::STAGE_BYTES);
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-          tma_load_2d(sa, &tmA, kb * BK, m0, leader_full);
-          tma_load_2d(sb, &tmB, kb * BK, n0, leader_full);
+          tma_load_2d(sa, &tmA, kb * BK, m0, leader_full, keep);
+          tma_load_2d(sb, &tmB, kb * BK, n0, leader_full, keep);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -486,6 +518,8 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     float warp_acc = 0.f;
     float s_global = 0.f;
     if (MODE == FAAR_GEMM_BWD) s_global = *p.s_global;
+    uint32_t pn = 0;                                   // panels this quarter has staged so far
+    bool dead = false;
     int it = 0;
     for (int tile = pair; tile < total_tiles; tile += n_pairs, ++it) {
       const int acc = it & 1;
@@ -498,25 +532,53 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int o = m0 + quarter * 32 + lane;
       const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
       if constexpr (MODE == FAAR_GEMM_BWD) {
-        const uint32_t stg = epi_u32 + (uint32_t)ew * EPI_WARP_BYTES;
+        // 128-column panels, staged by the four warps of this lane quarter together (see epi_bwd_rows)
+        const int sub = ew >> 2;
+        const uint32_t panel = epi_u32 + (uint32_t)quarter * PANEL_BYTES;
+        const uint32_t pfull = ctl_u32 + 256u + 16u * quarter, pdone = pfull + 8u;
         const int o_first = m0 + quarter * 32;
+        bool released = false;
 #pragma unroll 1
-        for (int c = col_begin; c < col_begin + C::COLS_PER_WARP; c += 32) {
-          if (n0 + c >= p.N || o_first >= p.M) break;  // warp-uniform
-          uint32_t r[32];
-          tmem_ld32(trow + (uint32_t)c, r);
-          tmem_ld_wait();
+        for (int pc = 0; pc < BN; pc += 128) {
+          if (n0 + pc >= p.N || o_first >= p.M) break;   // the same decision in all four warps
+          // the quarter's previous panel has been consumed by all four warps
+          bool okp = mbar_wait(pdone, (pn & 1u) ^ 1u, ac, 0x500u | quarter);
+          if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
+          const int c = pc + 32 * sub;
+          if (n0 + c < p.N) {
+            uint32_t r[32];
+            tmem_ld32(trow + (uint32_t)c, r);
+            tmem_ld_wait();
 #pragma unroll
-          for (int u = 0; u < 8; ++u)
-            sts128(stg + (uint32_t)lane * 128u + (uint32_t)((u ^ (lane & 7)) << 4), r[4 * u], r[4 * u + 1], r[4 * u + 2],
-                   r[4 * u + 3]);
+            for (int u = 0; u < 8; ++u)
+              sts128(panel + (uint32_t)lane * 512u + (uint32_t)(((8 * sub + u) ^ (lane & 7)) << 4), r[4 * u], r[4 * u + 1],
+                     r[4 * u + 2], r[4 * u + 3]);
+          }
+          if (pc + 128 >= BN || n0 + pc + 128 >= p.N) {  // this warp's last read of the accumulator
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+            released = true;
+          }
           __syncwarp();
-          if (o_first + 32 <= p.M && n0 + c + 32 <= p.N)
-            warp_acc += epi_bwd_block<OPT, true>(p, stg, lane, o_first, n0 + c, s_global);
+          if (lane == 0) mbar_arrive(pfull);
+          okp = mbar_wait(pfull, pn & 1u, ac, 0x600u | quarter);
+          if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
+          if (o_first + 32 <= p.M && n0 + pc + 128 <= p.N)
+            warp_acc += epi_bwd_rows<OPT, true>(p, panel, lane, sub, o_first, n0 + pc, s_global);
           else
-            warp_acc += epi_bwd_block<OPT, false>(p, stg, lane, o_first, n0 + c, s_global);
-          __syncwarp();                                // the block is consumed before the next one lands
+            warp_acc += epi_bwd_rows<OPT, false>(p, panel, lane, sub, o_first, n0 + pc, s_global);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(pdone);
+          ++pn;
         }
+        if (dead) break;
+        if (!released) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+        }
+        continue;
       } else {
 #pragma unroll 1
         for (int c = col_begin; c < col_begin + C::COLS_PER_WARP; c += 16) {
