@@ -275,10 +275,40 @@ def run_ours(args):
     timed(profiled)
     prof = faar.profile_end(ctx)
 
+    # ---- the once-per-layer / HBM-bound kernels alone: back-to-back launches over rotated buffer sets
+    # (3 sets x 150 MB > L2), one event pair around all of them, so launch overhead is amortised
+    def elementwise_rates(rounds=10, sets=3):
+        bufs = []
+        for r in range(sets):
+            bufs.append(dict(W=W.clone(), V=torch.rand((O, K), dtype=torch.float32, device=device), code=code.clone(),
+                             scales=scales.clone(), packed=torch.empty_like(packed), so=torch.empty_like(scales_out),
+                             wsoft=torch.empty((O, K), dtype=torch.bfloat16, device=device)))
+        calls = {
+            "softquant_init": lambda b: faar.softquant_init(ctx, shape, b["W"], 0.0, b["scales"], s_global, b["code"],
+                                                            b["V"], ws),
+            "soft_weights": lambda b: faar.softquant_eval(ctx, shape, b["V"], b["code"], b["scales"], s_global, 8.0,
+                                                          None, None, b["wsoft"]),
+            "harden_pack": lambda b: faar.harden_pack(ctx, shape, b["V"], b["code"], b["scales"], s_global, b["packed"],
+                                                      b["so"], None, None),
+        }
+        out = {}
+        for name in ("soft_weights", "harden_pack", "softquant_init"):      # init last: it overwrites V
+            fn = calls[name]
+            with torch.cuda.stream(stream):
+                for b in bufs:
+                    fn(b)
+            stream.synchronize()
+            ms = timed(lambda: [fn(b) for _ in range(rounds) for b in bufs])
+            out[name] = 1e3 * ms / (rounds * sets)
+        return out
+
+    ew_us = elementwise_rates()
+
     if args.quick:
         if rank == 0:
             print(json.dumps({"quick": True, "steps": steps, "ms_per_step": ms_job / steps,
-                              "kernels_avg_us": {k: round(1e3 * v[1] / v[0], 2) for k, v in prof.items()}}))
+                              "kernels_avg_us": {k: round(1e3 * v[1] / v[0], 2) for k, v in prof.items()},
+                              "elementwise_alone_us": {k: round(v, 2) for k, v in ew_us.items()}}))
         if sampler:
             sampler.stop()
         if world > 1:
