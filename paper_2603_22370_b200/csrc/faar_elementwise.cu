@@ -111,13 +111,36 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
   }
 }
 
-// ---- Eq. 2 / Eq. 3 in FP32 (parity view) -----------------------------------------
+// ---- Eq. 2 / Eq. 3 -----------------------------------------------------------------------------
+// FP32 outputs (W_soft, H): the parity view, relative error below 1e-6.
+// BF16 output: the operand of the forward GEMM.  It is rounded from a cheaper FP32 evaluation whose
+// relative error is below 3e-6 (z = beta*v - beta/2 and z*log2(e) each rounded once, hardware 2^x and
+// reciprocal), far inside the BF16 spacing of 2^-8; it can differ from the rounding of the exact
+// value only where that value lies within 3e-6 of a BF16 rounding boundary.
+// Per nibble (sign<<3 | k) the signed lower node and the signed interval width come from a
+// 16-entry table in shared memory: mag = lo + h*width needs one 8-byte load.
+__device__ __forceinline__ float sigmoid_fast(float beta, float neg_half_beta, float v) {
+  const float z = fmaf(beta, v, neg_half_beta);
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-fabsf(z) * 1.4426950408889634f));
+  const float hs = __fdividef(1.0f, 1.0f + e);
+  return z >= 0.f ? hs : e * hs;
+}
+
 __global__ void __launch_bounds__(EW_THREADS)
 softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code,
                       const uint8_t* __restrict__ scales, const float* __restrict__ s_global_p,
                       float beta, int64_t n_groups, float* __restrict__ W_soft, float* __restrict__ H,
                       __nv_bfloat16* __restrict__ W_bf16) {
+  __shared__ float2 lut[16];
+  if (threadIdx.x < 16) {
+    const int k = threadIdx.x & 7;
+    const float sgn = (threadIdx.x & 8) ? -1.f : 1.f;
+    lut[threadIdx.x] = make_float2(sgn * faar_node(k), sgn * faar_width(k));
+  }
+  __syncthreads();
   const float s_global = *s_global_p;
+  const float nhb = -0.5f * beta;
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups;
        g += (int64_t)gridDim.x * blockDim.x) {
     int64_t e = g * 8;
@@ -126,29 +149,36 @@ softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ c
     float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
     uint32_t cw = *reinterpret_cast<const uint32_t*>(code + e / 2);
     float s = __fmul_rn(faar_e4m3_to_float(scales[e / 16]), s_global);
-    float ws[8], h[8];
+    if (W_soft || H) {
+      float ws[8], h[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      uint32_t nib = (cw >> (4 * i)) & 0xF;
-      int k = nib & 7;
-      h[i] = faar_sigmoid_precise(beta, v[i]);
-      ws[i] = faar_soft_weight(h[i], nib, s);
-    }
-    if (W_soft) {
-      float4* p = reinterpret_cast<float4*>(W_soft + e);
-      p[0] = make_float4(ws[0], ws[1], ws[2], ws[3]);
-      p[1] = make_float4(ws[4], ws[5], ws[6], ws[7]);
-    }
-    if (H) {
-      float4* p = reinterpret_cast<float4*>(H + e);
-      p[0] = make_float4(h[0], h[1], h[2], h[3]);
-      p[1] = make_float4(h[4], h[5], h[6], h[7]);
+      for (int i = 0; i < 8; ++i) {
+        uint32_t nib = (cw >> (4 * i)) & 0xF;
+        h[i] = faar_sigmoid_precise(beta, v[i]);
+        ws[i] = faar_soft_weight(h[i], nib, s);
+      }
+      if (W_soft) {
+        float4* p = reinterpret_cast<float4*>(W_soft + e);
+        p[0] = make_float4(ws[0], ws[1], ws[2], ws[3]);
+        p[1] = make_float4(ws[4], ws[5], ws[6], ws[7]);
+      }
+      if (H) {
+        float4* p = reinterpret_cast<float4*>(H + e);
+        p[0] = make_float4(h[0], h[1], h[2], h[3]);
+        p[1] = make_float4(h[4], h[5], h[6], h[7]);
+      }
     }
     if (W_bf16) {
+      float wf[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float2 nw = lut[(cw >> (4 * i)) & 0xF];
+        wf[i] = fmaf(sigmoid_fast(beta, nhb, v[i]), nw.y, nw.x) * s;
+      }
       uint32_t o[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 p2 = __floats2bfloat162_rn(ws[2 * i], ws[2 * i + 1]);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(wf[2 * i], wf[2 * i + 1]);
         o[i] = *reinterpret_cast<uint32_t*>(&p2);
       }
       *reinterpret_cast<uint4*>(W_bf16 + e) = make_uint4(o[0], o[1], o[2], o[3]);

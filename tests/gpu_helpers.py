@@ -103,13 +103,14 @@ def max_rel_to_peak(a, b):
 
 
 # ---- BF16 operand ties ---------------------------------------------------------------------
-# The forward GEMM multiplies W_soft rounded to BF16.  The library evaluates W_soft in FP32
-# (tested to 1e-6 relative against the float64 oracle); where the exact value lies within that
-# error of a BF16 rounding boundary, either neighbour is a correct rounding.  The helpers below
+# The forward GEMM multiplies W_soft rounded to BF16.  The library rounds the operand from an FP32
+# evaluation whose relative error is below 3e-6 (the separate FP32 parity view is tested to 1e-6);
+# where the exact value lies within that error of a BF16 rounding boundary, either neighbour is a
+# correct rounding.  The helpers below
 # find those elements from the ORACLE's W_soft and give the exact first-order effect of moving
 # one of them by one BF16 step, so that a comparison can allow for it and nothing else.
 
-W_SOFT_FP32_TOL = 1e-6
+W_SOFT_FP32_TOL = 3e-6
 
 
 def bf16_tie_elements(W_soft, tol=W_SOFT_FP32_TOL):

@@ -126,11 +126,13 @@ def test_softquant_eval_matches_eq2_eq3(ctx, beta):
     H2 = torch.empty_like(lay.V)
     faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, b, None, H2)
     assert torch.equal(H, H2)
-    # the BF16 GEMM operand is the FP32 value rounded to nearest even; it can differ from the
-    # oracle's rounding only where the exact value sits on a BF16 rounding boundary
+    # the BF16 GEMM operand is a 3e-6-accurate FP32 value rounded to nearest even; it can differ from
+    # the oracle's rounding only where the exact value sits that close to a BF16 rounding boundary
     Wb = torch.empty_like(lay.V, dtype=torch.bfloat16)
     faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, b, None, None, Wb)
-    assert torch.equal(Wb, Ws.to(torch.bfloat16))
+    Wb2 = torch.empty_like(Wb)
+    faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, b, Ws, None, Wb2)
+    assert torch.equal(Wb, Wb2)                       # the same operand whatever else is requested
     tie, step = bf16_tie_elements(Wo)
     diff = host(Wb).astype(np.float64) != fo.bf16_round(Wo)
     assert not np.any(diff & ~tie)
@@ -261,8 +263,8 @@ def test_layer_fwd(ctx, O, K, T):
     allow = dy_column_allowance(X, tie, step, hpo.mse_scale)
     col_err = np.linalg.norm(dY_g - dY_o, axis=0)
     assert np.all(col_err <= 2e-3 * np.linalg.norm(dY_o, axis=0) + allow)
-    # a weight is a tie with probability ~ 2 * 1e-6 / 2^-8, so only a few columns get an allowance
-    assert (allow > 0).sum() <= 4 + 3 * O * K * 2 * 1e-6 * 256
+    # a weight is a tie with probability ~ 2 * 3e-6 / 2^-8, so only a few columns get an allowance
+    assert (allow > 0).sum() <= 4 + 3 * O * K * 2 * 3e-6 * 256
     assert rel_l2(dY_g, dY_o) <= 2e-3 + np.linalg.norm(allow) / np.linalg.norm(dY_o)
     assert max_rel_to_peak(dY_g[:, allow == 0], dY_o[:, allow == 0]) <= 2e-3
     assert rel_l2(host(Yq), Yq_o) <= 2e-3 and max_rel_to_peak(host(Yq), Yq_o) <= 4e-3   # BF16 output: 2^-8 rounding
