@@ -101,6 +101,15 @@ FAAR_API const char* faar_status_string(int status);
 /* Last cudaError_t seen by this context (0 if none). */
 FAAR_API int faar_last_cuda_error(const faar_ctx* ctx);
 
+/* ---- GEMM tiling (no counterpart in the paper: tuning and introspection of this library) -------
+ * The tensor-core kernels cover the output with 256-row tiles whose width is chosen per launch (a
+ * multiple of 16 in [128, 256]): the widest unless the problem is too small to give every CTA pair a
+ * tile.  faar_tune_tile_n forces a width for the following launches on this context
+ * (0 = automatic again).  faar_last_gemm_config reports the width and the number of CTA pairs of the
+ * most recent GEMM launch (host out-pointers). */
+FAAR_API int faar_tune_tile_n(faar_ctx* ctx, int bn);
+FAAR_API int faar_last_gemm_config(const faar_ctx* ctx, int* bn, int* cta_pairs);
+
 /* Bytes of workspace that any call on this shape needs (host out-pointer).
  * The workspace must be 256-byte aligned.  Its first 256 bytes hold the status
  * word; the caller zeroes them once (faar_workspace_init) before first use. */

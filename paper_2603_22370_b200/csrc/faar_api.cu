@@ -147,6 +147,9 @@ int faar_create(faar_ctx** out, int device, void* stream) {
   c->stream = reinterpret_cast<cudaStream_t>(stream);
   c->last_cuda_error = 0;
   c->encode_tiled = nullptr;
+  c->tune_bn = 0;
+  c->last_gemm_bn = 0;
+  c->last_gemm_pairs = 0;
   c->prof_on = false;
   c->prof_used = 0;
   cudaDriverEntryPointQueryResult q;
@@ -226,6 +229,20 @@ int faar_set_stream(faar_ctx* ctx, void* stream) {
 }
 
 int faar_last_cuda_error(const faar_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int faar_tune_tile_n(faar_ctx* ctx, int bn) {
+  if (!ctx) return FAAR_ERR_INVALID_ARG;
+  if (bn != 0 && (bn < 128 || bn > 256 || bn % 16 != 0)) return FAAR_ERR_INVALID_ARG;
+  ctx->tune_bn = bn;
+  return FAAR_OK;
+}
+
+int faar_last_gemm_config(const faar_ctx* ctx, int* bn, int* cta_pairs) {
+  if (!ctx || !bn || !cta_pairs) return FAAR_ERR_INVALID_ARG;
+  *bn = ctx->last_gemm_bn;
+  *cta_pairs = ctx->last_gemm_pairs;
+  return FAAR_OK;
+}
 
 int faar_workspace_size(const faar_shape* shape, size_t* bytes) {
   if (!bytes) return FAAR_ERR_INVALID_ARG;

@@ -2,9 +2,9 @@
 //
 // One persistent, warp-specialised kernel computes C[M,N] = A[M,Kc] * B[N,Kc]^T for BF16 operands that
 // both have the contraction dimension contiguous.  It runs as clusters of two CTAs that share one
-// 256 x BN output tile (tcgen05 cta_group::2): CTA r of the pair loads rows [128 r, 128 r + 128) of the
-// A tile and rows [BN/2 r, BN/2 (r+1)) of the B tile into its own shared memory, the leader CTA (r = 0)
-// issues the 256 x BN x 16 MMAs for both, and each CTA ends up with its 128 accumulator rows x BN
+// 256 x bn output tile (tcgen05 cta_group::2): CTA r of the pair loads rows [128 r, 128 r + 128) of the
+// A tile and rows [bn/2 r, bn/2 (r+1)) of the B tile into its own shared memory, the leader CTA (r = 0)
+// issues the 256 x bn x 16 MMAs for both, and each CTA ends up with its 128 accumulator rows x bn
 // columns (FP32) in its own tensor memory.  Halving the B tile per CTA halves the shared-memory
 // traffic per flop, which is what bounds a single-CTA 128 x 256 tile.
 //   warp 0      : TMA producer  (cp.async.bulk.tensor, 128-byte swizzle, multi-stage ring; both CTAs,
@@ -37,18 +37,20 @@ constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int CTL_BYTES = 512;
 constexpr int MAX_EPI_WARPS = 16;
 
-template <int MODE, int BN> struct Cfg {
+// The tile width bn (accumulator columns, a multiple of 16 up to 256) is a launch parameter chosen by
+// the host (pick_bn).  Shared memory and tensor memory are laid out for the widest tile.
+constexpr int BN_MAX = 256;
+template <int MODE> struct Cfg {
   static constexpr int EPI_WARPS = MODE == FAAR_GEMM_BWD ? 16 : 8;
   static constexpr int THREADS = 32 * (2 + EPI_WARPS);
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = (BN / 2) * BK * 2;            // this CTA's half of the B tile
+  static constexpr int B_BYTES = (BN_MAX / 2) * BK * 2;        // this CTA's half of the B tile (slot size)
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int EPI_BYTES = MODE == FAAR_GEMM_BWD ? 4 * PANEL_BYTES : 0;
   static constexpr int FIT = (SMEM_LIMIT - 1024 - CTL_BYTES - EPI_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = FIT > 8 ? 8 : FIT;
-  static constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
+  static constexpr int TMEM_COLS = 2 * BN_MAX;                 // two accumulator buffers
   static constexpr int COL_GROUPS = EPI_WARPS / 4;             // warps sharing one TMEM lane quarter
-  static constexpr int COLS_PER_WARP = BN / COL_GROUPS;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + CTL_BYTES;
 };
 
@@ -217,13 +219,14 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                          // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: D = F32, A = B = BF16, both K-major, M = 256 (the CTA pair), N = BN.
-template <int BN> __device__ __forceinline__ constexpr uint32_t make_idesc() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+// Instruction descriptor: D = F32, A = B = BF16, both K-major, M = 256 (the CTA pair), N = bn.
+__device__ __forceinline__ uint32_t make_idesc(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 }
 
 struct KParams {
   int M, N, Kc;
+  int bn;                 // tile width
   uint32_t* status;
   // REF / FWD
   void* Yout; int yout_dtype; long long ldy;
@@ -316,13 +319,14 @@ __device__ __forceinline__ float width_of(uint32_t k) {       // interval widths
 // instruction moves 512 contiguous bytes of one row of V / m / u: long bursts for the HBM, full lines
 // as 16-byte vectors.  The per-weight state of two rows is requested together before either is
 // computed.  FULL: the panel lies wholly inside the matrix (no bounds tests).
-// o_first: output feature of panel row 0; k_first: input feature of panel column 0.
+// o_first: output feature of panel row 0; k_first: input feature of panel column 0; k_end: first
+// input feature beyond the tile (or the matrix).
 // Returns the Round Loss contribution of the pre-update v's.
 template <int OPT, bool FULL>
 __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, int lane, int sub, int o_first,
-                                              int k_first, float s_global) {
+                                              int k_first, int k_end, float s_global) {
   const int kcol = k_first + 4 * lane;
-  const bool col_ok = FULL || kcol < p.N;
+  const bool col_ok = FULL || kcol < k_end;
   const int r0 = 8 * sub;
   const long long e0 = (long long)(o_first + r0) * p.N + kcol;     // row r0 element of this lane
   float* const Vp = p.V + e0;
@@ -407,10 +411,11 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
 
 // ---- the kernel ------------------------------------------------------------------------------
 // Launched as clusters of two CTAs along x: CTAs 2c and 2c+1 form pair c.
-template <int MODE, int BN, int OPT>
-__global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1)
+template <int MODE, int OPT>
+__global__ void __launch_bounds__(Cfg<MODE>::THREADS, 1)
 faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const KParams p) {
-  using C = Cfg<MODE, BN>;
+  using C = Cfg<MODE>;
+  const int BN = p.bn;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;       // the same offset in both CTAs of the pair
@@ -466,7 +471,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (!ok) break;
           const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
           // the leader's barrier collects the bytes of both CTAs' copies
-          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * C::STAGE_BYTES);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * (uint32_t)(C::A_BYTES + (BN / 2) * BK * 2));
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
           tma_load_2d(sa, &tmA, kb * BK, m0, leader_full, keep);
           tma_load_2d(sb, &tmB, kb * BK, n0, leader_full, keep);
@@ -482,7 +487,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   } else if (warp == 1) {
     // ---------------- MMA issuer (leader CTA only) ----------------
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = make_idesc<BN>();
+      const uint32_t idesc = make_idesc(BN);
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
@@ -492,7 +497,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, ac, 0x200u | acc);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tmem_d = tmem_base + acc * BN;
+        const uint32_t tmem_d = tmem_base + acc * BN_MAX;
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(full_bar(stage), phase, ac, 0x300u | stage);
           if (!ok) break;
@@ -514,7 +519,10 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ---------------- epilogue (both CTAs) ----------------
     const int ew = warp - 2;
     const int quarter = warp & 3;                      // TMEM lanes this warp may read
-    const int col_begin = (ew >> 2) * C::COLS_PER_WARP;
+    // REF / FWD: the warps that share a lane quarter split the tile's columns in 16-column chunks
+    const int cols_per_warp = ((BN / C::COL_GROUPS + 15) / 16) * 16;
+    const int col_begin = (ew >> 2) * cols_per_warp;
+    const int col_end = min(col_begin + cols_per_warp, BN);
     float warp_acc = 0.f;
     float s_global = 0.f;
     if (MODE == FAAR_GEMM_BWD) s_global = *p.s_global;
@@ -530,7 +538,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       tc_fence_after();
       const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM, n0 = (tile / m_tiles) * BN;
       const int o = m0 + quarter * 32 + lane;
-      const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+      const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN_MAX);
       if constexpr (MODE == FAAR_GEMM_BWD) {
         // 128-column panels, staged by the four warps of this lane quarter together (see epi_bwd_rows)
         const int sub = ew >> 2;
@@ -545,7 +553,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           bool okp = mbar_wait(pdone, (pn & 1u) ^ 1u, ac, 0x500u | quarter);
           if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
           const int c = pc + 32 * sub;
-          if (n0 + c < p.N) {
+          if (c < BN && n0 + c < p.N) {
             uint32_t r[32];
             tmem_ld32(trow + (uint32_t)c, r);
             tmem_ld_wait();
@@ -564,10 +572,11 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (lane == 0) mbar_arrive(pfull);
           okp = mbar_wait(pfull, pn & 1u, ac, 0x600u | quarter);
           if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
-          if (o_first + 32 <= p.M && n0 + pc + 128 <= p.N)
-            warp_acc += epi_bwd_rows<OPT, true>(p, panel, lane, sub, o_first, n0 + pc, s_global);
+          const int k_end = min(p.N, n0 + BN);           // columns of this tile that exist
+          if (o_first + 32 <= p.M && n0 + pc + 128 <= k_end)
+            warp_acc += epi_bwd_rows<OPT, true>(p, panel, lane, sub, o_first, n0 + pc, k_end, s_global);
           else
-            warp_acc += epi_bwd_rows<OPT, false>(p, panel, lane, sub, o_first, n0 + pc, s_global);
+            warp_acc += epi_bwd_rows<OPT, false>(p, panel, lane, sub, o_first, n0 + pc, k_end, s_global);
           __syncwarp();
           if (lane == 0) mbar_arrive(pdone);
           ++pn;
@@ -581,7 +590,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         continue;
       } else {
 #pragma unroll 1
-        for (int c = col_begin; c < col_begin + C::COLS_PER_WARP; c += 16) {
+        for (int c = col_begin; c < col_end; c += 16) {
           if (n0 + c >= p.N) break;                    // warp-uniform
           uint32_t r[16];
           tmem_ld16(trow + (uint32_t)c, r);
@@ -629,22 +638,28 @@ int make_map(faar_ctx* ctx, CUtensorMap* map, const void* ptr, int rows, int col
   return r == CUDA_SUCCESS ? 0 : (int)cudaErrorInvalidValue;
 }
 
-template <int MODE, int BN, int OPT = 0>
-int launch(faar_ctx* ctx, const faar_gemm_args* a, const KParams& kp, int* n_partials_out) {
-  using C = Cfg<MODE, BN>;
+// Tile width for an M x N output.  Measured on the down_proj-shaped layer, a tile's time is set by the
+// operand bytes it pulls through the SM (A rows are not shared between tiles), not by its columns, so
+// narrower tiles never pay while the widest ones already fill the device; they are used only to get at
+// least one tile per CTA pair on small problems.
+int pick_bn(const faar_ctx* ctx, int M, int N, int pairs) {
+  if (ctx->tune_bn >= 128 && ctx->tune_bn <= BN_MAX && ctx->tune_bn % 16 == 0) return ctx->tune_bn;
+  const long long m_tiles = (M + 2 * BM - 1) / (2 * BM);
+  for (int bn = BN_MAX; bn > 128; bn -= 32)
+    if (m_tiles * ((N + bn - 1) / bn) >= pairs) return bn;
+  return 128;
+}
+
+template <int MODE, int OPT = 0>
+int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_out) {
+  using C = Cfg<MODE>;
   static_assert(C::STAGES >= 3, "ring too short");
   static_assert(C::SMEM_BYTES <= SMEM_LIMIT, "shared memory budget");
   static_assert(C::EPI_WARPS <= MAX_EPI_WARPS, "partials budget");
-  CUtensorMap tmA, tmB;
-  int e = make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
-  if (e) return e;
-  e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, BN / 2);
-  if (e) return e;
-  auto kern = faar_gemm_kernel<MODE, BN, OPT>;
+  auto kern = faar_gemm_kernel<MODE, OPT>;
   cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (ce != cudaSuccess) return (int)ce;
 
-  const long long tiles = (long long)((a->M + 2 * BM - 1) / (2 * BM)) * ((a->N + BN - 1) / BN);
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -666,19 +681,23 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, const KParams& kp, int* n_par
     if (n > ctx->num_sms / 2) n = ctx->num_sms / 2;
     max_pairs = n;
   }
+  const int bn = pick_bn(ctx, a->M, a->N, max_pairs);
+  kp.bn = bn;
+  CUtensorMap tmA, tmB;
+  int e = make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
+  if (e) return e;
+  e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, bn / 2);
+  if (e) return e;
+  const long long tiles = (long long)((a->M + 2 * BM - 1) / (2 * BM)) * ((a->N + bn - 1) / bn);
   const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   if (n_partials_out) *n_partials_out = 2 * pairs * C::EPI_WARPS;
+  ctx->last_gemm_bn = bn;
+  ctx->last_gemm_pairs = pairs;
   faar_prof_scope ps(ctx, MODE == FAAR_GEMM_REF ? FAAR_K_GEMM_REF : (MODE == FAAR_GEMM_FWD ? FAAR_K_GEMM_FWD : FAAR_K_GEMM_BWD));
   ce = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, kp);
   if (ce != cudaSuccess) return (int)ce;
   return (int)cudaGetLastError();
-}
-
-int pick_bn(const faar_ctx* ctx, int M, int N) {
-  // the wide tile unless it leaves most SMs idle
-  long long tiles256 = (long long)((M + 2 * BM - 1) / (2 * BM)) * ((N + 255) / 256);
-  return tiles256 >= ctx->num_sms / 2 ? 256 : 128;
 }
 
 }  // namespace
@@ -687,7 +706,7 @@ int faar_gemm_max_partials(const faar_ctx* ctx, int, int) { return ctx->num_sms 
 
 int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out) {
   KParams kp;
-  kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.status = a->status;
+  kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.bn = BN_MAX; kp.status = a->status;
   kp.Yout = a->Yout; kp.yout_dtype = a->yout_dtype; kp.ldy = a->ldy;
   kp.Yref = a->Yref; kp.yref_dtype = a->yref_dtype;
   kp.dYt = a->dYt; kp.ld_dyt = a->ld_dyt; kp.mse2c = a->mse2c; kp.partials = a->partials;
@@ -695,21 +714,15 @@ int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out
   kp.adam_m = a->adam_m; kp.adam_u = a->adam_u; kp.dV = a->dV;
   kp.beta = a->beta; kp.lam_over_n = a->lam_over_n; kp.lr = a->lr; kp.b1 = a->b1; kp.b2 = a->b2; kp.eps = a->eps;
   kp.inv_bc1 = a->inv_bc1; kp.inv_bc2 = a->inv_bc2; kp.opt = a->opt;
-  // the BWD epilogue forms row offsets of up to 28 rows in 32-bit element counts
-  if (a->mode == FAAR_GEMM_BWD && (long long)a->N * 32 > 0x7FFFFFFFll) return (int)cudaErrorInvalidValue;
+  // the BWD epilogue forms row offsets of up to 7 rows in 32-bit element counts
+  if (a->mode == FAAR_GEMM_BWD && (long long)a->N * 8 > 0x7FFFFFFFll) return (int)cudaErrorInvalidValue;
 
-  const int bn = pick_bn(ctx, a->M, a->N);
-  switch (a->mode * 2 + (bn == 256 ? 1 : 0)) {
-    case FAAR_GEMM_REF * 2 + 0: return launch<FAAR_GEMM_REF, 128>(ctx, a, kp, n_partials_out);
-    case FAAR_GEMM_REF * 2 + 1: return launch<FAAR_GEMM_REF, 256>(ctx, a, kp, n_partials_out);
-    case FAAR_GEMM_FWD * 2 + 0: return launch<FAAR_GEMM_FWD, 128>(ctx, a, kp, n_partials_out);
-    case FAAR_GEMM_FWD * 2 + 1: return launch<FAAR_GEMM_FWD, 256>(ctx, a, kp, n_partials_out);
-    case FAAR_GEMM_BWD * 2 + 0:
-      return a->opt == 1 ? launch<FAAR_GEMM_BWD, 128, 1>(ctx, a, kp, n_partials_out)
-                         : launch<FAAR_GEMM_BWD, 128, 0>(ctx, a, kp, n_partials_out);
-    case FAAR_GEMM_BWD * 2 + 1:
-      return a->opt == 1 ? launch<FAAR_GEMM_BWD, 256, 1>(ctx, a, kp, n_partials_out)
-                         : launch<FAAR_GEMM_BWD, 256, 0>(ctx, a, kp, n_partials_out);
+  switch (a->mode) {
+    case FAAR_GEMM_REF: return launch<FAAR_GEMM_REF>(ctx, a, kp, n_partials_out);
+    case FAAR_GEMM_FWD: return launch<FAAR_GEMM_FWD>(ctx, a, kp, n_partials_out);
+    case FAAR_GEMM_BWD:
+      return a->opt == 1 ? launch<FAAR_GEMM_BWD, 1>(ctx, a, kp, n_partials_out)
+                         : launch<FAAR_GEMM_BWD, 0>(ctx, a, kp, n_partials_out);
   }
   return (int)cudaErrorInvalidValue;
 }

@@ -15,6 +15,8 @@ struct faar_ctx {
   cudaStream_t stream;
   int last_cuda_error;
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
+  int tune_bn;                            // 0 = choose the GEMM tile width automatically
+  int last_gemm_bn, last_gemm_pairs;      // what the last GEMM launch used
   // per-kernel timing (faar_profile_begin / faar_profile_end)
   bool prof_on;
   int prof_used;                          // event pairs used since faar_profile_begin

@@ -20,7 +20,8 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
            "faar_workspace_size", "faar_workspace_init", "faar_check_status", "faar_softquant_init",
            "faar_softquant_eval", "faar_transpose_bf16", "faar_layer_ref", "faar_layer_fwd", "faar_round_loss",
            "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
-           "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n"]
+           "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n", "faar_tune_tile_n",
+           "faar_last_gemm_config"]
 
 
 class HParams(C.Structure):
@@ -120,6 +121,18 @@ class Context:
             self.ws = torch.empty(n, dtype=torch.uint8, device=f"cuda:{self.device}")
             workspace_init(self, self.ws)
         return self.ws
+
+
+def tune_tile_n(ctx: Context, bn: int):
+    """Forces the GEMM tile width (multiple of 16 in [128, 256]); 0 restores the automatic choice."""
+    _check(lib().faar_tune_tile_n(ctx._h, C.c_int(bn)), "faar_tune_tile_n")
+
+
+def last_gemm_config(ctx: Context) -> tuple[int, int]:
+    """(tile width, CTA pairs) of the most recent GEMM launch on this context."""
+    bn, pairs = C.c_int(0), C.c_int(0)
+    _check(lib().faar_last_gemm_config(ctx._h, C.byref(bn), C.byref(pairs)), "faar_last_gemm_config")
+    return bn.value, pairs.value
 
 
 def workspace_size(shape: Shape) -> int:

@@ -477,3 +477,37 @@ def test_error_statuses(ctx):
     assert step_status(hp_=faar.make_hparams(step=0)) == faar.ERR_INVALID_ARG
     assert step_status(X_=lay.X.view(-1)[1:]) == faar.ERR_ALIGN
     lay.check()
+
+
+@pytest.mark.parametrize("bn", [128, 144, 176, 224, 240])
+@pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (520, 272, 1300)])
+def test_forced_tile_widths_give_the_same_step(ctx, O, K, T, bn):
+    """The tile width only changes how the output is cut up: every forced width must reproduce the
+    automatic choice bit for bit (each output element is the same sum in the same order); the loss is a
+    sum of differently grouped partials."""
+    W, X, Yref = _problem(O, K, T, seed=5)
+    hp, _ = f32hp(beta=6.0, step=2)
+    rng = np.random.default_rng(3)
+    V0 = rng.uniform(0, 1, W.shape).astype(np.float32)
+    m0 = (1e-3 * rng.standard_normal(W.shape)).astype(np.float32)
+    u0 = (1e-6 * rng.uniform(0, 1, W.shape)).astype(np.float32)
+    out = []
+    try:
+        for width in (0, bn):
+            faar.tune_tile_n(ctx, width)
+            lay = GpuLayer(ctx, W, X)
+            lay.init()
+            lay.set_yref(Yref)
+            lay.set_state(V=V0, m=m0, u=u0)
+            lay.fwd(hp)
+            dYt = host(lay.dYt).copy()
+            if width:
+                assert faar.last_gemm_config(ctx)[0] == bn
+            dV = host(lay.bwd(hp, want_dv=True)).copy()
+            lay.check()
+            out.append((dYt, dV, host(lay.V).copy(), host(lay.m).copy(), host(lay.u).copy(), host(lay.loss)[0]))
+    finally:
+        faar.tune_tile_n(ctx, 0)
+    for a, b in zip(out[0][:5], out[1][:5]):
+        assert np.array_equal(a, b)
+    assert abs(out[0][5] - out[1][5]) <= 1e-5 * abs(out[0][5])
