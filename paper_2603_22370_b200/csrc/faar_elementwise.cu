@@ -35,8 +35,23 @@ amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, 
   const int64_t groups_per_row = K / 8;
   const int64_t total = (int64_t)O * groups_per_row;
   float amax = 0.f;
-  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total;
-       g += (int64_t)gridDim.x * blockDim.x) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // four independent 16-byte (32-byte for FP32) loads in flight per thread
+  for (; g + 3 * stride < total; g += 4 * stride) {
+    float w[4][8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t gj = g + j * stride;
+      const int64_t row = gj / groups_per_row, col = (gj - row * groups_per_row) * 8;
+      load8(W, w_dtype, row * ldw + col, w[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[j][i]));
+  }
+  for (; g < total; g += stride) {
     int64_t row = g / groups_per_row, col = (g - row * groups_per_row) * 8;
     float w[8];
     load8(W, w_dtype, row * ldw + col, w);
@@ -93,9 +108,13 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
     for (int i = 0; i < 8; ++i) {
       float wt = s > 0.f ? __fdiv_rn(fabsf(w[i]), s) : 0.f;
       wt = fminf(wt, 6.0f);
-      int k = (wt >= 0.5f) + (wt >= 1.0f) + (wt >= 1.5f) + (wt >= 2.0f) + (wt >= 3.0f) + (wt >= 4.0f);
+      // interval index from the bits of w~ (exponent and top mantissa bit order like the nodes):
+      // [.5,.75) -> 0, [.75,1) -> 1, [1,1.5) -> 2, [1.5,2) -> 3, [2,3) -> 4, [3,4) -> 5, [4,6) -> 6, 6 -> 7
+      const int t = (int)(__float_as_uint(wt) >> 22) - 252;
+      int k = wt < 0.5f ? 0 : max(t, 1);
+      k = min(k, 6);
       float lo = faar_node(k);
-      float inv_w = k < 4 ? 2.0f : (k < 6 ? 1.0f : 0.5f);
+      float inv_w = __uint_as_float((uint32_t)(128 - (k >= 4) - (k >= 6)) << 23);   // 2, 1, 0.5
       v[i] = __fmul_rn(__fsub_rn(wt, lo), inv_w);
       uint32_t neg = (w[i] < 0.f) ? 8u : 0u;
       cw |= ((uint32_t)k | neg) << (4 * i);
