@@ -279,6 +279,7 @@ int faar_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float
   if (st) return st;
   if (s->w_dtype != FAAR_BF16 && s->w_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
   if (s->ldw < s->K) return FAAR_ERR_SHAPE;
+  if ((int64_t)s->O * (s->K / 8) > 0xFFFFFFFFll) return FAAR_ERR_SHAPE;   // 8-element groups are counted in 32 bits
   if (s->ldw % 8 || !aligned16(W) || !aligned16(V_init) || !aligned16(code)) return FAAR_ERR_ALIGN;
   if (!isfinite(s_global_in) || s_global_in < 0.f) return FAAR_ERR_INVALID_ARG;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)

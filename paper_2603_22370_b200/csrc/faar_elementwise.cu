@@ -29,11 +29,20 @@ __device__ __forceinline__ void load8(const void* W, int w_dtype, int64_t idx, f
   }
 }
 
+// Element offset in W of 8-element group g.  Dense rows (ldw == K) need no division; otherwise the
+// row comes from a 32-bit division (the host checks that the group count fits).
+__device__ __forceinline__ int64_t w_offset(int64_t g, uint32_t groups_per_row, int64_t ldw, bool dense) {
+  if (dense) return g * 8;
+  const uint32_t row = (uint32_t)g / groups_per_row;
+  return (int64_t)row * ldw + (int64_t)((uint32_t)g - row * groups_per_row) * 8;
+}
+
 // ---- pass 1: max |W| over the tensor -----------------------------------------
 __global__ void __launch_bounds__(EW_THREADS)
 amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, uint32_t* amax_word) {
-  const int64_t groups_per_row = K / 8;
+  const uint32_t groups_per_row = K / 8;
   const int64_t total = (int64_t)O * groups_per_row;
+  const bool dense = ldw == K;
   float amax = 0.f;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -42,9 +51,7 @@ amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, 
     float w[4][8];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int64_t gj = g + j * stride;
-      const int64_t row = gj / groups_per_row, col = (gj - row * groups_per_row) * 8;
-      load8(W, w_dtype, row * ldw + col, w[j]);
+      load8(W, w_dtype, w_offset(g + j * stride, groups_per_row, ldw, dense), w[j]);
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j)
@@ -52,9 +59,8 @@ amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, 
       for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[j][i]));
   }
   for (; g < total; g += stride) {
-    int64_t row = g / groups_per_row, col = (g - row * groups_per_row) * 8;
     float w[8];
-    load8(W, w_dtype, row * ldw + col, w);
+    load8(W, w_dtype, w_offset(g, groups_per_row, ldw, dense), w);
 #pragma unroll
     for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[i]));
   }
@@ -86,16 +92,16 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
   if (blockIdx.x == 0 && threadIdx.x == 0) *s_global_out = s_global;
   const float d = __fmul_rn(s_global, 6.0f);
 
-  const int64_t groups_per_row = K / 8;
+  const uint32_t groups_per_row = K / 8;
   const int64_t total = (int64_t)O * groups_per_row;
+  const bool dense = ldw == K;
   // the grid is sized so that every warp is either fully inside or the tail is padded with idle lanes
   for (int64_t g0 = (int64_t)blockIdx.x * blockDim.x; g0 < total; g0 += (int64_t)gridDim.x * blockDim.x) {
     int64_t g = g0 + threadIdx.x;
     bool valid = g < total;
     int64_t gc = valid ? g : total - 1;
-    int64_t row = gc / groups_per_row, col = (gc - row * groups_per_row) * 8;
     float w[8];
-    load8(W, w_dtype, row * ldw + col, w);
+    load8(W, w_dtype, w_offset(gc, groups_per_row, ldw, dense), w);
     float amax = 0.f;
 #pragma unroll
     for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[i]));
@@ -120,12 +126,13 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
       cw |= ((uint32_t)k | neg) << (4 * i);
     }
     if (valid) {
-      int64_t e = row * (int64_t)K + col;
+      const int64_t e = g * 8;                 // V, code, scales are dense
+      const bool first_half = (g & 1) == 0;    // K % 16 == 0: even groups start a scale block
       float4* vp = reinterpret_cast<float4*>(V + e);
       vp[0] = make_float4(v[0], v[1], v[2], v[3]);
       vp[1] = make_float4(v[4], v[5], v[6], v[7]);
       *reinterpret_cast<uint32_t*>(code + e / 2) = cw;
-      if ((col & 8) == 0) scales[e / 16] = (uint8_t)sb;
+      if (first_half) scales[e / 16] = (uint8_t)sb;
     }
   }
 }
