@@ -265,7 +265,7 @@ def run_ours(args):
     faar.check_status(ctx, ws)
     loss_final = loss.cpu().tolist()
     value = n_gpus * steps / (ms_job * 1e-3)
-    gpu_launches = 2 + 4 * steps + 1     # amax + init, 4 kernels per step, harden_pack
+    gpu_launches = 2 + 3 * steps + 1     # amax + init, 3 kernels per step (soft weights, forward, backward), harden_pack
 
     # ---- second pass of the same job with per-kernel CUDA events (library hooks, same stream)
     def profiled():

@@ -70,8 +70,18 @@ int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
 
 int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* dYt, const void* Xt,
              float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
-             float* adam_u, float* dV, uint8_t* ws, const faar_ws_layout& l, int* n_partials) {
+             float* adam_u, float* dV, uint8_t* ws, const faar_ws_layout& l, int* n_partials,
+             float* loss_out2 = nullptr, int n_mse_partials = 0) {
   faar_gemm_args a = {};
+  if (loss_out2) {
+    // the kernel's last CTA sums the forward's MSE partials and its own Round Loss partials
+    a.fin_counter = reinterpret_cast<uint32_t*>(ws) + 2;
+    a.fin_mse_partials = reinterpret_cast<const float*>(ws + l.off_mse_partials);
+    a.fin_n_mse = n_mse_partials;
+    a.fin_scale_mse = hp->mse_scale;
+    a.fin_scale_round = (float)(1.0 / ((double)s->O * (double)s->K));
+    a.fin_out2 = loss_out2;
+  }
   a.mode = FAAR_GEMM_BWD;
   a.M = s->O; a.N = s->K; a.Kc = s->T;
   a.A = dYt; a.lda = l.ld_dyt;
@@ -419,11 +429,8 @@ int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, 
   int np_mse = 0, np_round = 0;
   int e = fwd_impl(ctx, s, hp, X, Y_ref, V, code, scales, s_global, dYt, nullptr, ws, l, &np_mse);
   if (e) return cuda_fail(ctx, e);
-  e = bwd_impl(ctx, s, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, nullptr, ws, l, &np_round);
-  if (e) return cuda_fail(ctx, e);
-  e = faar_launch_finalize(ctx, reinterpret_cast<float*>(ws + l.off_mse_partials), np_mse, hp->mse_scale, loss_out2,
-                           reinterpret_cast<float*>(ws + l.off_round_partials), np_round,
-                           (float)(1.0 / ((double)s->O * (double)s->K)), loss_out2 + 1);
+  e = bwd_impl(ctx, s, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, nullptr, ws, l, &np_round, loss_out2,
+               np_mse);
   return cuda_fail(ctx, e);
 }
 

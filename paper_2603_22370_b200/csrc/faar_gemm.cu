@@ -238,6 +238,10 @@ struct KParams {
   float* V; const uint8_t* code; const uint8_t* scales; const float* s_global;
   float* adam_m; float* adam_u; float* dV;
   float beta, lam_over_n, lr, b1, b2, eps, inv_bc1, inv_bc2; int opt;
+  // BWD, optional: the CTA that finishes last also forms the step's two loss values
+  uint32_t* fin_counter;            // workspace word, zero between launches
+  const float* fin_mse_partials; int fin_n_mse; float fin_scale_mse;
+  float fin_scale_round; float* fin_out2;   // {L_MSE, L_round}; null = no final sums here
 };
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
@@ -618,6 +622,42 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_after();
     tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
+
+  if constexpr (MODE == FAAR_GEMM_BWD) {
+    // Final loss sums by whichever CTA finishes last: always the same partials in the same order
+    // (strided double accumulation, then a tree), so the result does not depend on which CTA it is.
+    if (p.fin_out2 != nullptr) {
+      double* sh = reinterpret_cast<double*>(smem);          // the operand ring is idle by now
+      volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 256 * sizeof(double));
+      if (threadIdx.x == 0) {
+        __threadfence();                                     // this CTA's partials, ordered by the barrier above
+        const uint32_t prev = atomicAdd(p.fin_counter, 1u);
+        const int last = prev == gridDim.x - 1;
+        if (last) *p.fin_counter = 0u;                       // ready for the next launch
+        __threadfence();
+        *last_flag = last;
+      }
+      __syncthreads();
+      if (*last_flag) {
+        const int n_round = (int)gridDim.x * C::EPI_WARPS;
+        for (int which = 0; which < 2; ++which) {
+          const float* src = which ? p.partials : p.fin_mse_partials;
+          const int n = which ? n_round : p.fin_n_mse;
+          double acc = 0.0;
+          if (threadIdx.x < 256)
+            for (int i = threadIdx.x; i < n; i += 256) acc += (double)__ldcg(src + i);
+          __syncthreads();
+          if (threadIdx.x < 256) sh[threadIdx.x] = acc;
+          __syncthreads();
+          for (int st = 128; st > 0; st >>= 1) {
+            if (threadIdx.x < st) sh[threadIdx.x] += sh[threadIdx.x + st];
+            __syncthreads();
+          }
+          if (threadIdx.x == 0) p.fin_out2[which] = (float)(sh[0] * (double)(which ? p.fin_scale_round : p.fin_scale_mse));
+        }
+      }
+    }
+  }
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -714,6 +754,8 @@ int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out
   kp.adam_m = a->adam_m; kp.adam_u = a->adam_u; kp.dV = a->dV;
   kp.beta = a->beta; kp.lam_over_n = a->lam_over_n; kp.lr = a->lr; kp.b1 = a->b1; kp.b2 = a->b2; kp.eps = a->eps;
   kp.inv_bc1 = a->inv_bc1; kp.inv_bc2 = a->inv_bc2; kp.opt = a->opt;
+  kp.fin_counter = a->fin_counter; kp.fin_mse_partials = a->fin_mse_partials; kp.fin_n_mse = a->fin_n_mse;
+  kp.fin_scale_mse = a->fin_scale_mse; kp.fin_scale_round = a->fin_scale_round; kp.fin_out2 = a->fin_out2;
   // the BWD epilogue forms row offsets of up to 7 rows in 32-bit element counts
   if (a->mode == FAAR_GEMM_BWD && (long long)a->N * 8 > 0x7FFFFFFFll) return (int)cudaErrorInvalidValue;
 

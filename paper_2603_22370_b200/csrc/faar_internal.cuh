@@ -33,7 +33,8 @@ struct faar_prof_scope {
 };
 
 // ---- workspace layout -------------------------------------------------------
-// [0, 256)            header: word 0 = status (0 = ok), word 1 = |W| max bits
+// [0, 256)            header: word 0 = status (0 = ok), word 1 = |W| max bits, word 2 = count of dW-GEMM
+//                     CTAs that have finished (zero between launches)
 // [256, 256+P)        loss partials (float): MSE region then Round region
 // [..]                W_soft bf16 [O,K]
 // [..]                dYt bf16 [O, ceil8(T)]
@@ -100,6 +101,9 @@ struct faar_gemm_args {
   float* V; const uint8_t* code; const uint8_t* scales; const float* s_global;
   float* adam_m; float* adam_u; float* dV;
   float beta, lam_over_n, lr, b1, b2, eps, inv_bc1, inv_bc2; int opt;
+  // BWD, optional: final loss sums by the last CTA (fin_out2 null = not wanted)
+  uint32_t* fin_counter; const float* fin_mse_partials; int fin_n_mse; float fin_scale_mse, fin_scale_round;
+  float* fin_out2;
 };
 // n_partials_out: number of floats written to args.partials
 int faar_launch_gemm(faar_ctx*, const faar_gemm_args*, int* n_partials_out);
