@@ -375,6 +375,21 @@ def dequant_packed(packed, scales, s_global):
     return np.where((nib >> 3).astype(bool), -val, val)
 
 
+def act_fake_quant(X, s_global_in=0.0):
+    """Quantised activations X_q of the Stage-1 objective (Eq. 5 uses X_q W_q).  The paper gives no
+    rule for them; reading used: the same NVFP4 format as the weights (blocks of 16 along the
+    contraction dimension, E4M3 block scales under an FP32 tensor scale, amax rule) with
+    round-to-nearest, a tie going to the larger magnitude -- i.e. Eq. 7 applied to the initial
+    position v_init.  Returns (Xq_units float64 [T,K] = sign * node * s_g, exactly representable in
+    BF16; s_global float32; packed u8 [T,K/2]; scales u8 [T,K/16]); X_q = Xq_units * s_global."""
+    scales, s_global, code, v = softquant_init(X, s_global_in)
+    packed, _, _ = harden_pack(v, code, scales, s_global)
+    k_mag, neg = unpack_code(packed)
+    sg = np.repeat(e4m3_decode(scales), BLOCK, axis=1)
+    units = np.where(neg, -1.0, 1.0) * NODES[k_mag] * sg
+    return units, s_global, packed, scales
+
+
 def rtn_nearest(W, scales, s_global):
     """Round-to-nearest onto the node set, written independently of the
     bracket: argmin over all 8 nodes of |w~ - node|, a tie going to the larger

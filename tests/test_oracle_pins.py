@@ -366,3 +366,39 @@ def test_bf16_mode_rounds_only_at_the_stated_points():
     assert np.array_equal(dY_b, fo.bf16_round(2 * (Yq_b - Yref)))
     Vn, m, u, *_ = fo.layer_step(X, Yref, V, code, scales, sg, np.zeros_like(V), np.zeros_like(V), fo.HParams(), "bf16")
     assert Vn.dtype == np.float32 and m.dtype == np.float32 and u.dtype == np.float32
+
+
+# ---------------------------------------------------------------------------------------------
+# activation fake-quantisation (the X_q of Eq. 5)
+# ---------------------------------------------------------------------------------------------
+
+def test_act_fake_quant_is_nearest_node_and_fits_bf16():
+    import torch
+    rng = np.random.default_rng(5)
+    X = (rng.standard_t(4, size=(24, 64)) * np.where(rng.random(64) < 0.1, 20.0, 1.0)).astype(np.float32)
+    X[0, :16] = 0.0                                   # an all-zero block
+    X[1, 0] = -0.0
+    units, sg, packed, scales = fo.act_fake_quant(X)
+    # every value is sign * node * block scale, and those products need at most 7 significant bits
+    assert np.array_equal(torch.from_numpy(units.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy(), units)
+    # independent nearest-node search (ties to the larger node) gives the same magnitude codes
+    codes = fo.rtn_nearest(X, scales, sg)
+    k_mag, neg = fo.unpack_code(packed)
+    assert np.array_equal(k_mag, codes)
+    assert np.array_equal(neg, np.signbit(X) & (X != 0))
+    # dequantised NVFP4 == units * s_global (up to the one binary32 rounding of the product)
+    deq = fo.dequant_packed(packed, scales, sg).astype(np.float64)
+    assert np.all(np.abs(deq - units * float(sg)) <= 2.0 ** -23 * np.abs(deq))
+    # quantisation error of an in-range value is at most half the local node spacing (times the scale)
+    s = np.repeat(fo.effective_scale(scales, sg), 16, axis=1).astype(np.float64)
+    ok = s > 0
+    err = np.abs(np.abs(X.astype(np.float64)) - np.abs(units) * float(sg))[ok] / s[ok]
+    assert err.max() <= 1.0 + 1e-6                   # widest interval [4, 6]: half of 2
+
+
+def test_act_fake_quant_exact_on_representable_inputs():
+    # inputs that are already node * 2^e with block maximum 6 * 2^e survive unchanged
+    nodes = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6, -0.5, -1, -1.5, -2, -3, -4, -6, 6], dtype=np.float32)
+    X = np.stack([nodes * 2.0 ** e for e in (-3, 0, 2)]).astype(np.float32)
+    units, sg, _, scales = fo.act_fake_quant(X, s_global_in=2.0 ** -3)
+    assert np.array_equal((units * float(sg)).astype(np.float32), X)
