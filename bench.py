@@ -282,7 +282,8 @@ def run_ours(args):
         for r in range(sets):
             bufs.append(dict(W=W.clone(), V=torch.rand((O, K), dtype=torch.float32, device=device), code=code.clone(),
                              scales=scales.clone(), packed=torch.empty_like(packed), so=torch.empty_like(scales_out),
-                             wsoft=torch.empty((O, K), dtype=torch.bfloat16, device=device)))
+                             wsoft=torch.empty((O, K), dtype=torch.bfloat16, device=device),
+                             X=X.clone(), Xq=torch.empty_like(X), sx=torch.empty(1, dtype=torch.float32, device=device)))
         calls = {
             "softquant_init": lambda b: faar.softquant_init(ctx, shape, b["W"], 0.0, b["scales"], s_global, b["code"],
                                                             b["V"], ws),
@@ -291,8 +292,9 @@ def run_ours(args):
             "harden_pack": lambda b: faar.harden_pack(ctx, shape, b["V"], b["code"], b["scales"], s_global, b["packed"],
                                                       b["so"], None, None),
         }
+        calls["act_fakequant"] = lambda b: faar.act_fakequant(ctx, T, K, b["X"], K, 0.0, b["Xq"], K, b["sx"], None, None, ws)
         out = {}
-        for name in ("soft_weights", "harden_pack", "softquant_init"):      # init last: it overwrites V
+        for name in ("soft_weights", "harden_pack", "act_fakequant", "softquant_init"):   # init last: it overwrites V
             fn = calls[name]
             with torch.cuda.stream(stream):
                 for b in bufs:
@@ -359,6 +361,7 @@ def run_ours(args):
         ("soft_weights", "hbm", 6.5625 * n_w),              # V 4 + code .5 + scale 1/16 read, BF16 operand 2 written
         ("softquant_init", "hbm", 6.5625 * n_w),            # W 2 read; V 4 + code .5 + scale 1/16 written
         ("harden_pack", "hbm", 5.125 * n_w),                # V 4 + code .5 + scale 1/16 read; .5 + 1/16 written
+        ("act_fakequant", "hbm", 4.0 * T * K),              # X 2 read, X_q units 2 written (+2 for the amax pass)
     ]:
         if bound == "tensor":
             us = avg_us(name)

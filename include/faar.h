@@ -75,6 +75,10 @@ typedef struct {
   int opt;
   float lr, beta1, beta2, eps;
   int step;
+  /* FP32 tensor scale of quantised activations (faar_act_fakequant): the activation matrix passed to
+   * the forward / backward calls then holds X_q / act_scale, and Y_q and the weight gradient are
+   * multiplied by act_scale in the GEMM epilogues.  0 (or 1) = activations as given. */
+  float act_scale;
 } faar_hparams;
 
 /* Layer geometry.  Leading dimensions are in ELEMENTS.
@@ -140,7 +144,8 @@ enum {
   FAAR_K_FINALIZE = 7,       /* fixed-order final sums of the loss partials       */
   FAAR_K_HARDEN_PACK = 8,
   FAAR_K_TRANSPOSE = 9,
-  FAAR_K_COUNT = 10
+  FAAR_K_ACT_FAKEQUANT = 10, /* activations to NVFP4 values (the X_q of Eq. 5)          */
+  FAAR_K_COUNT = 11
 };
 typedef struct {
   int kernel;     /* one of FAAR_K_*          */
@@ -184,6 +189,21 @@ FAAR_API int faar_softquant_eval(faar_ctx* ctx, const faar_shape* shape, const f
  * dW GEMM (no counterpart in the paper: a storage choice of this library). */
 FAAR_API int faar_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in, int64_t ld_in,
                         void* out, int64_t ld_out);
+
+/* ---- quantised activations -------------------------------------------------
+ * The X_q of Eq. 5 ("Stage 1": the quantised output is X_q W_q).  The paper gives
+ * no rule for X_q; reading taken: the weights' NVFP4 format and scale rule
+ * (blocks of 16 along K, E4M3 block scales, FP32 tensor scale = amax / (6*448)
+ * unless s_global_in > 0), every value to its nearest node, a tie to the larger
+ * magnitude.  Xq_units receives sign * node * block scale (exact in BF16); the
+ * quantised activations are Xq_units * *s_global_out.  Pass Xq_units (and its
+ * transpose) as X / Xt and the tensor scale as faar_hparams.act_scale.
+ *   X in: [T,K] bf16 (ldx, multiple of 8)      Xq_units out: [T,K] bf16 (ldq, multiple of 8)
+ *   s_global_out out: 1 float (device)
+ *   packed out: [T,K/2] u8 E2M1 codes, nullable   scales out: [T,K/16] u8 E4M3, nullable */
+FAAR_API int faar_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_t ldx, float s_global_in,
+                                void* Xq_units, int64_t ldq, float* s_global_out, uint8_t* packed,
+                                uint8_t* scales, void* workspace, size_t workspace_bytes);
 
 /* ---- frozen target ----------------------------------------------------------
  * Procedure step 8: Y_fp = X W^T with the original BF16 weights (w_dtype must

@@ -32,6 +32,7 @@ int check_hp(const faar_hparams* hp, bool need_opt) {
   if (!hp) return FAAR_ERR_INVALID_ARG;
   if (!(hp->beta > 0.f) || !isfinite(hp->beta) || !isfinite(hp->mse_scale) || !isfinite(hp->lambda_round))
     return FAAR_ERR_INVALID_ARG;
+  if (!(hp->act_scale >= 0.f) || !isfinite(hp->act_scale)) return FAAR_ERR_INVALID_ARG;
   if (need_opt) {
     if (hp->opt != 0 && hp->opt != 1) return FAAR_ERR_INVALID_ARG;
     if (!isfinite(hp->lr)) return FAAR_ERR_INVALID_ARG;
@@ -64,6 +65,7 @@ int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
   a.Yref = Y_ref; a.yref_dtype = s->yref_dtype;
   a.dYt = reinterpret_cast<__nv_bfloat16*>(dYt); a.ld_dyt = l.ld_dyt;
   a.mse2c = 2.0f * hp->mse_scale;
+  a.act_scale = hp->act_scale > 0.f ? hp->act_scale : 1.0f;
   a.partials = reinterpret_cast<float*>(ws + l.off_mse_partials);
   return faar_launch_gemm(ctx, &a, n_partials);
 }
@@ -91,6 +93,7 @@ int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
   a.V = V; a.code = code; a.scales = scales; a.s_global = s_global;
   a.adam_m = adam_m; a.adam_u = adam_u; a.dV = dV;
   a.beta = hp->beta;
+  a.act_scale = hp->act_scale > 0.f ? hp->act_scale : 1.0f;
   a.lam_over_n = (float)((double)hp->lambda_round / ((double)s->O * (double)s->K));
   a.lr = hp->lr; a.b1 = hp->beta1; a.b2 = hp->beta2; a.eps = hp->eps; a.opt = hp->opt;
   if (hp->opt == 1) {
@@ -192,6 +195,7 @@ const char* faar_kernel_name(int kernel) {
     case FAAR_K_FINALIZE: return "finalize";
     case FAAR_K_HARDEN_PACK: return "harden_pack";
     case FAAR_K_TRANSPOSE: return "transpose";
+    case FAAR_K_ACT_FAKEQUANT: return "act_fakequant";
   }
   return "unknown";
 }
@@ -322,6 +326,22 @@ int faar_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in, int64
   if (rows <= 0 || cols <= 0 || ld_in < cols || ld_out < rows) return FAAR_ERR_SHAPE;
   DeviceGuard g(ctx->device);
   return cuda_fail(ctx, faar_launch_transpose_bf16(ctx, rows, cols, in, ld_in, out, ld_out));
+}
+
+int faar_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_t ldx, float s_global_in, void* Xq_units,
+                       int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales, void* workspace,
+                       size_t workspace_bytes) {
+  if (!ctx || !X || !Xq_units || !s_global_out) return FAAR_ERR_INVALID_ARG;
+  if (T <= 0 || K <= 0 || K % 16 != 0 || ldx < K || ldq < K) return FAAR_ERR_SHAPE;
+  if ((int64_t)T * (K / 8) > 0xFFFFFFFFll) return FAAR_ERR_SHAPE;
+  if (ldx % 8 || ldq % 8 || !aligned16(X) || !aligned16(Xq_units) || (packed && !aligned16(packed))) return FAAR_ERR_ALIGN;
+  if (!isfinite(s_global_in) || s_global_in < 0.f) return FAAR_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
+    return FAAR_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  uint32_t* amax_word = reinterpret_cast<uint32_t*>(workspace) + 1;
+  return cuda_fail(ctx, faar_launch_act_fakequant(ctx, T, K, X, ldx, s_global_in, Xq_units, ldq, s_global_out, packed,
+                                                  scales, amax_word));
 }
 
 int faar_layer_ref(faar_ctx* ctx, const faar_shape* s, const void* X, const void* W, void* Y_ref,

@@ -137,6 +137,73 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
   }
 }
 
+// ---- activation fake-quantisation: the X_q of Eq. 5 --------------------------------------------
+// Same format and scale rule as the weights; each value goes to the nearest node, a tie to the larger
+// magnitude (Eq. 7 applied to the initial position).  The output holds sign * node * block scale, which
+// needs at most 7 significant bits and is therefore exact in BF16; the FP32 tensor scale stays outside
+// (X_q = Xq_units * s_global) and is applied by the GEMM epilogues.
+__global__ void __launch_bounds__(EW_THREADS)
+act_fakequant_kernel(const __nv_bfloat16* __restrict__ X, int T, int K, int64_t ldx, float s_global_in,
+                     const uint32_t* __restrict__ amax_word, __nv_bfloat16* __restrict__ Xq, int64_t ldq,
+                     float* __restrict__ s_global_out, uint8_t* __restrict__ packed, uint8_t* __restrict__ scales) {
+  float s_global;
+  if (s_global_in > 0.f) {
+    s_global = s_global_in;
+  } else {
+    float amax_t = __uint_as_float(*amax_word);
+    s_global = amax_t == 0.f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) *s_global_out = s_global;
+  const float d = __fmul_rn(s_global, 6.0f);
+  const uint32_t groups_per_row = K / 8;
+  const int64_t total = (int64_t)T * groups_per_row;
+  for (int64_t g0 = (int64_t)blockIdx.x * blockDim.x; g0 < total; g0 += (int64_t)gridDim.x * blockDim.x) {
+    int64_t g = g0 + threadIdx.x;
+    bool valid = g < total;
+    int64_t gc = valid ? g : total - 1;
+    const uint32_t row = (uint32_t)gc / groups_per_row, col = ((uint32_t)gc - row * groups_per_row) * 8;
+    float w[8];
+    load8(X, FAAR_BF16, (int64_t)row * ldx + col, w);
+    float amax = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[i]));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));   // partner holds the other half-block
+    const uint32_t sb = faar_float_to_e4m3(__fdiv_rn(amax, d));
+    const float sg = faar_e4m3_to_float(sb);
+    const float s = __fmul_rn(sg, s_global);
+    uint32_t cw = 0;
+    float q[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float wt = s > 0.f ? __fdiv_rn(fabsf(w[i]), s) : 0.f;
+      wt = fminf(wt, 6.0f);
+      const int t = (int)(__float_as_uint(wt) >> 22) - 252;
+      int k = wt < 0.5f ? 0 : max(t, 1);
+      k = min(k, 6);
+      const float lo = faar_node(k);
+      const float inv_w = __uint_as_float((uint32_t)(128 - (k >= 4) - (k >= 6)) << 23);   // 2, 1, 0.5
+      const float v = __fmul_rn(__fsub_rn(wt, lo), inv_w);
+      const int c = k + (v >= 0.5f ? 1 : 0);
+      const float mag = __fmul_rn(faar_node(c), sg);              // exact: 3 x 4 significant bits
+      const bool neg = w[i] < 0.f;
+      q[i] = neg ? -mag : mag;
+      cw |= ((uint32_t)c | (neg ? 8u : 0u)) << (4 * i);
+    }
+    if (valid) {
+      uint32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(q[2 * i], q[2 * i + 1]);
+        o[i] = *reinterpret_cast<uint32_t*>(&p2);
+      }
+      *reinterpret_cast<uint4*>(Xq + (int64_t)row * ldq + col) = make_uint4(o[0], o[1], o[2], o[3]);
+      const int64_t e = g * 8;                 // packed and scales are dense
+      if (packed) *reinterpret_cast<uint32_t*>(packed + e / 2) = cw;
+      if (scales && (g & 1) == 0) scales[e / 16] = (uint8_t)sb;
+    }
+  }
+}
+
 // ---- Eq. 2 / Eq. 3 -----------------------------------------------------------------------------
 // FP32 outputs (W_soft, H): the parity view, relative error below 1e-6.
 // BF16 output: the operand of the forward GEMM.  It is rounded from a cheaper FP32 evaluation whose
@@ -354,6 +421,23 @@ int faar_launch_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W
   faar_prof_scope ps(ctx, FAAR_K_SOFTQUANT_INIT);
   softquant_init_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, s_global_in,
                                                                amax_word, scales, s_global_out, code, V);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_t ldx, float s_global_in, void* Xq,
+                              int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales, uint32_t* amax_word) {
+  const int64_t groups = (int64_t)T * (K / 8);
+  const int grid = grid_for(ctx, groups, 8);
+  if (!(s_global_in > 0.f)) {
+    cudaError_t e = cudaMemsetAsync(amax_word, 0, sizeof(uint32_t), ctx->stream);
+    if (e != cudaSuccess) return (int)e;
+    faar_prof_scope ps(ctx, FAAR_K_AMAX);
+    amax_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(X, FAAR_BF16, T, K, ldx, amax_word);
+  }
+  faar_prof_scope ps(ctx, FAAR_K_ACT_FAKEQUANT);
+  act_fakequant_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(reinterpret_cast<const __nv_bfloat16*>(X), T, K, ldx,
+                                                            s_global_in, amax_word, reinterpret_cast<__nv_bfloat16*>(Xq),
+                                                            ldq, s_global_out, packed, scales);
   return (int)cudaGetLastError();
 }
 

@@ -233,6 +233,7 @@ struct KParams {
   const void* Yref; int yref_dtype;
   __nv_bfloat16* dYt; long long ld_dyt;
   float mse2c;
+  float act_scale;        // FWD: Y_q = act_scale * acc; BWD: G = act_scale * acc
   float* partials;
   // BWD: M = O, N = K
   float* V; const uint8_t* code; const uint8_t* scales; const float* s_global;
@@ -283,7 +284,7 @@ __device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const 
   float dy[16];
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
-    float a = __uint_as_float(acc[j]);
+    float a = __uint_as_float(acc[j]) * p.act_scale;
     float r = (t0 + j < p.N) ? a - yr[j] : 0.f;
     ss = fmaf(r, r, ss);
     dy[j] = p.mse2c * r;
@@ -302,7 +303,7 @@ __device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const 
     __nv_bfloat16* yq = reinterpret_cast<__nv_bfloat16*>(p.Yout);
 #pragma unroll
     for (int j = 0; j < 16; ++j)
-      if (t0 + j < p.N) yq[(long long)(t0 + j) * p.ldy + o] = __float2bfloat16_rn(__uint_as_float(acc[j]));
+      if (t0 + j < p.N) yq[(long long)(t0 + j) * p.ldy + o] = __float2bfloat16_rn(__uint_as_float(acc[j]) * p.act_scale);
   }
   return ss;
 }
@@ -372,7 +373,7 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
         const float4 g4 = lds128(panel + (uint32_t)row * 512u + (uint32_t)((lane ^ (row & 7)) << 4));
         const float G[4] = {g4.x, g4.y, g4.z, g4.w};
         const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
-        const float sbeta = __fmul_rn(faar_e4m3_to_float(sb[q]), s_global) * p.beta;
+        const float sbeta = __fmul_rn(faar_e4m3_to_float(sb[q]), s_global) * p.beta * p.act_scale;   // act_scale: G = act_scale * acc
         float g[4], vn[4], mn[4], un[4];
         float mm[4], uu[4];
         if (OPT == 1) {
@@ -749,7 +750,7 @@ int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out
   kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.bn = BN_MAX; kp.status = a->status;
   kp.Yout = a->Yout; kp.yout_dtype = a->yout_dtype; kp.ldy = a->ldy;
   kp.Yref = a->Yref; kp.yref_dtype = a->yref_dtype;
-  kp.dYt = a->dYt; kp.ld_dyt = a->ld_dyt; kp.mse2c = a->mse2c; kp.partials = a->partials;
+  kp.dYt = a->dYt; kp.ld_dyt = a->ld_dyt; kp.mse2c = a->mse2c; kp.act_scale = a->act_scale; kp.partials = a->partials;
   kp.V = a->V; kp.code = a->code; kp.scales = a->scales; kp.s_global = a->s_global;
   kp.adam_m = a->adam_m; kp.adam_u = a->adam_u; kp.dV = a->dV;
   kp.beta = a->beta; kp.lam_over_n = a->lam_over_n; kp.lr = a->lr; kp.b1 = a->b1; kp.b2 = a->b2; kp.eps = a->eps;

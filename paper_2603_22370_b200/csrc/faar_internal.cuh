@@ -73,6 +73,8 @@ int faar_launch_softquant_init(faar_ctx*, const faar_shape*, const void* W, floa
 int faar_launch_softquant_eval(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta,
                                float* W_soft, float* h, __nv_bfloat16* W_soft_bf16);
+int faar_launch_act_fakequant(faar_ctx*, int T, int K, const void* X, int64_t ldx, float s_global_in, void* Xq,
+                              int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales, uint32_t* amax_word);
 int faar_launch_transpose_bf16(faar_ctx*, int rows, int cols, const void* in, int64_t ld_in, void* out,
                                int64_t ld_out);
 int faar_launch_round_partials(faar_ctx*, const float* V, int64_t N, float* partials, int* n_partials);
@@ -96,6 +98,7 @@ struct faar_gemm_args {
   const void* Yref; int yref_dtype;            // FWD
   __nv_bfloat16* dYt; int64_t ld_dyt;          // FWD: [M(O), ld_dyt]
   float mse2c;                                 // FWD: 2 * mse_scale
+  float act_scale;                             // FWD, BWD: tensor scale of quantised activations (1 = none)
   float* partials;                             // FWD: sum r^2 partials; BWD: Round Loss partials
   // BWD: M = O, N = K
   float* V; const uint8_t* code; const uint8_t* scales; const float* s_global;

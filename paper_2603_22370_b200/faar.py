@@ -21,13 +21,13 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
            "faar_softquant_eval", "faar_transpose_bf16", "faar_layer_ref", "faar_layer_fwd", "faar_round_loss",
            "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
            "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n", "faar_tune_tile_n",
-           "faar_last_gemm_config"]
+           "faar_last_gemm_config", "faar_act_fakequant"]
 
 
 class HParams(C.Structure):
     _fields_ = [("beta", C.c_float), ("lambda_round", C.c_float), ("mse_scale", C.c_float), ("opt", C.c_int),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("step", C.c_int)]
+                ("step", C.c_int), ("act_scale", C.c_float)]
 
 
 class Shape(C.Structure):
@@ -83,8 +83,8 @@ def make_shape(O, K, T, ldw=None, ldx=None, ldxt=None, ldy=None, w_dtype=BF16, y
 
 
 def make_hparams(beta=4.0, lambda_round=1.0, mse_scale=1.0, opt=1, lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8,
-                 step=1) -> HParams:
-    return HParams(beta, lambda_round, mse_scale, opt, lr, beta1, beta2, eps, step)
+                 step=1, act_scale=0.0) -> HParams:
+    return HParams(beta, lambda_round, mse_scale, opt, lr, beta1, beta2, eps, step, act_scale)
 
 
 class Context:
@@ -162,6 +162,12 @@ def softquant_init(ctx, shape, W, s_global_in, scales, s_global_out, code, V_ini
 def softquant_eval(ctx, shape, V, code, scales, s_global, beta, W_soft, h, W_soft_bf16=None):
     _check(lib().faar_softquant_eval(ctx._h, C.byref(shape), _p(V), _p(code), _p(scales), _p(s_global),
                                      C.c_float(beta), _p(W_soft), _p(h), _p(W_soft_bf16)), "faar_softquant_eval")
+
+
+def act_fakequant(ctx, T, K, X, ldx, s_global_in, Xq_units, ldq, s_global_out, packed, scales, ws):
+    _check(lib().faar_act_fakequant(ctx._h, T, K, _p(X), C.c_int64(ldx), C.c_float(s_global_in), _p(Xq_units),
+                                    C.c_int64(ldq), _p(s_global_out), _p(packed), _p(scales), _p(ws),
+                                    C.c_size_t(ws.numel())), "faar_act_fakequant")
 
 
 def transpose_bf16(ctx, rows, cols, inp, ld_in, out, ld_out):
