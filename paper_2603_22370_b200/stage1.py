@@ -1,0 +1,81 @@
+"""Stage-1 driver: layer-wise rounding optimisation of one linear, or of the linears of a block, with
+libfaar.  Host loop and buffer management only -- every arithmetic step (set-up, soft weights, both
+GEMMs, update, hardening, packing) is a call into the CUDA library through `faar`.
+
+    res = optimise_layer(ctx, W, X, steps=200)          # W [O,K], X [T,K]: torch tensors on the GPU
+    res["packed"], res["scales"], res["s_global"]        # deployable NVFP4 weights
+"""
+from __future__ import annotations
+
+import torch
+
+from . import faar, shard
+
+
+def beta_schedule(t: int, steps: int, beta0: float = 4.0, beta1: float = 32.0) -> float:
+    """Temperature of the rounding function at step t: geometric from beta0 to beta1 (the method asks
+    for a small value that grows; the values are this harness's)."""
+    return beta0 if steps <= 1 else beta0 * (beta1 / beta0) ** (t / (steps - 1))
+
+
+def optimise_layer(ctx: faar.Context, W: torch.Tensor, X: torch.Tensor, steps: int = 200, lr: float = 1e-2,
+                   lambda_round: float = 1.0, mse_scale: float = 1.0, opt: int = 1, beta0: float = 4.0,
+                   beta1: float = 32.0, quantise_activations: bool = False, loss_every: int = 0) -> dict:
+    """Runs the whole path for one linear layer: soft-quantisation set-up, the frozen target, `steps`
+    optimisation steps, hardening and packing.  W [O,K] and X [T,K] are BF16 CUDA tensors (row-major).
+    With quantise_activations the GEMMs consume NVFP4-quantised activations (the target still comes from
+    the unquantised X).  Returns the packed weights, their scales, the final V and the losses read back
+    every `loss_every` steps (0 = only at the end)."""
+    assert W.is_cuda and X.is_cuda and W.dtype == torch.bfloat16 and X.dtype == torch.bfloat16
+    dev = W.device
+    O, K = W.shape
+    T = X.shape[0]
+    ldt = (T + 7) // 8 * 8
+    shape = faar.make_shape(O, K, T, ldxt=ldt)
+    ws = torch.empty(faar.workspace_size(shape), dtype=torch.uint8, device=dev)
+    faar.workspace_init(ctx, ws)
+    scales = torch.empty((O, K // 16), dtype=torch.uint8, device=dev)
+    code = torch.empty((O, K // 2), dtype=torch.uint8, device=dev)
+    s_global = torch.empty(1, dtype=torch.float32, device=dev)
+    V = torch.empty((O, K), dtype=torch.float32, device=dev)
+    m = torch.zeros((O, K), dtype=torch.float32, device=dev) if opt == 1 else None
+    u = torch.zeros((O, K), dtype=torch.float32, device=dev) if opt == 1 else None
+    Yref = torch.empty((T, O), dtype=torch.bfloat16, device=dev)
+    loss = torch.zeros(2, dtype=torch.float32, device=dev)
+
+    faar.softquant_init(ctx, shape, W, 0.0, scales, s_global, code, V, ws)
+    faar.layer_ref(ctx, shape, X, W, Yref, ws)
+    act_scale = 0.0
+    Xg = X
+    if quantise_activations:
+        Xg = torch.empty_like(X)
+        sx = torch.empty(1, dtype=torch.float32, device=dev)
+        faar.act_fakequant(ctx, T, K, X, K, 0.0, Xg, K, sx, None, None, ws)
+        act_scale = float(sx.item())                     # one read-back at set-up
+    Xt = torch.zeros((K, ldt), dtype=torch.bfloat16, device=dev)
+    faar.transpose_bf16(ctx, T, K, Xg, K, Xt, ldt)
+
+    history = []
+    for t in range(steps):
+        hp = faar.make_hparams(beta=beta_schedule(t, steps, beta0, beta1), lambda_round=lambda_round,
+                               mse_scale=mse_scale, opt=opt, lr=lr, step=t + 1, act_scale=act_scale)
+        faar.layer_step(ctx, shape, hp, Xg, Xt, Yref, V, code, scales, s_global, m, u, loss, ws)
+        if loss_every and (t + 1) % loss_every == 0:
+            history.append((t + 1, *loss.tolist()))
+    packed = torch.empty((O, K // 2), dtype=torch.uint8, device=dev)
+    faar.harden_pack(ctx, shape, V, code, scales, s_global, packed, None, None, None)
+    faar.check_status(ctx, ws)
+    history.append((steps, *loss.tolist()))
+    return {"packed": packed, "scales": scales, "s_global": s_global, "code": code, "V": V, "history": history,
+            "act_scale": act_scale}
+
+
+def optimise_block(ctx: faar.Context, linears: list, steps: int, rank: int = 0, world: int = 1, **kw) -> dict:
+    """Optimises the linears of a decoder block, `linears` = [(name, W, X), ...].  Layer problems are
+    independent, so with several processes each rank takes its share (round-robin) and no data moves
+    between ranks; the caller gathers the returned dicts if it needs them in one place."""
+    out = {}
+    for i in shard.layers_for_rank(len(linears), rank, world):
+        name, W, X = linears[i]
+        out[name] = optimise_layer(ctx, W, X, steps=steps, **kw)
+    return out
