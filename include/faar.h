@@ -276,8 +276,14 @@ FAAR_API int faar_layer_step(faar_ctx* ctx, const faar_shape* shape, const faar_
  * pinned): copies X_host[T,K] (ldx) and Y_ref_host[T,O] (ldy) into the caller's
  * device staging buffers X_dev / Yref_dev, rebuilds Xt_dev = X^T [K, ldxt],
  * runs the step, and copies {L_MSE, L_round} back to loss_host2.  Everything
- * is enqueued on the context's stream; loss_host2 is valid after the caller
- * synchronises it.  Bytes moved: T*K*2 + T*O*sizeof(yref_dtype) in, 8 out. */
+ * is ordered with the context's stream; loss_host2 is valid after the caller
+ * synchronises it.  Bytes moved: T*K*2 + T*O*sizeof(yref_dtype) in, 8 out.
+ * The host-to-device copies run on a copy stream that the context creates on
+ * the first call (with three events: host resources, no device memory).  A
+ * caller that alternates between two sets of staging buffers (X_dev, Xt_dev,
+ * Yref_dev) on consecutive calls gets the copy of batch n+1 overlapped with step
+ * n; with a single set the copy waits for the previous step.  After a change of
+ * the context's stream (faar_set_stream) synchronise before the next call. */
 FAAR_API int faar_layer_step_host(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp,
                                   const void* X_host, const void* Y_ref_host, void* X_dev, void* Xt_dev,
                                   void* Yref_dev, float* V, const uint8_t* code, const uint8_t* scales,

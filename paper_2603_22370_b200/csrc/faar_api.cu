@@ -161,6 +161,11 @@ int faar_create(faar_ctx** out, int device, void* stream) {
   c->last_cuda_error = 0;
   c->encode_tiled = nullptr;
   c->tune_bn = 0;
+  c->copy_stream = nullptr;
+  c->ev_copied = nullptr;
+  c->ev_done[0] = c->ev_done[1] = nullptr;
+  c->host_calls = 0;
+  c->last_staging = nullptr;
   c->last_gemm_bn = 0;
   c->last_gemm_pairs = 0;
   c->prof_on = false;
@@ -178,6 +183,10 @@ int faar_create(faar_ctx** out, int device, void* stream) {
 int faar_destroy(faar_ctx* ctx) {
   if (ctx) {
     for (cudaEvent_t ev : ctx->prof_events) cudaEventDestroy(ev);
+    if (ctx->ev_copied) cudaEventDestroy(ctx->ev_copied);
+    for (int i = 0; i < 2; ++i)
+      if (ctx->ev_done[i]) cudaEventDestroy(ctx->ev_done[i]);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   }
   delete ctx;
   return FAAR_OK;
@@ -467,12 +476,34 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
   if (s->ldy < s->O) return FAAR_ERR_SHAPE;
   if ((st = check_gemm_operands(s, true, true))) return st;
   DeviceGuard g(ctx->device);
+  cudaError_t e = cudaSuccess;
+  if (!ctx->copy_stream) {                       // host resources of this path, created on first use
+    e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_copied, cudaEventDisableTiming);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+  }
+  // The staging buffers of this call were last read by the step of two calls ago when the caller
+  // alternates between two sets (then this copy overlaps the previous step), by the previous step
+  // when it reuses one set (then the copy waits for it).
+  const unsigned long long n = ctx->host_calls++;
+  const int slot = (int)(n & 1);
+  if (n >= 2) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot], 0);
+  if (e == cudaSuccess && n >= 1 && ctx->last_staging == X_dev)
+    e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot ^ 1], 0);
+  if (e == cudaSuccess && n == 0) {              // order after whatever the caller enqueued before (set-up)
+    e = cudaEventRecord(ctx->ev_done[slot], ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot], 0);
+  }
+  ctx->last_staging = X_dev;
   const size_t ybytes = s->yref_dtype == FAAR_BF16 ? 2 : 4;
-  cudaError_t e = cudaMemcpyAsync(X_dev, X_host, (size_t)s->T * (size_t)s->ldx * 2, cudaMemcpyHostToDevice,
-                                  ctx->stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(X_dev, X_host, (size_t)s->T * (size_t)s->ldx * 2, cudaMemcpyHostToDevice, ctx->copy_stream);
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(Yref_dev, Y_ref_host, (size_t)s->T * (size_t)s->ldy * ybytes, cudaMemcpyHostToDevice,
-                        ctx->stream);
+                        ctx->copy_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_copied, ctx->copy_stream);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->stream, ctx->ev_copied, 0);
   if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
   st = faar_transpose_bf16(ctx, s->T, s->K, X_dev, s->ldx, Xt_dev, s->ldxt);
   if (st) return st;
@@ -480,6 +511,7 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
                        workspace, workspace_bytes);
   if (st) return st;
   e = cudaMemcpyAsync(loss_host2, loss_dev2, 2 * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_done[slot], ctx->stream);
   return cuda_fail(ctx, (int)e);
 }
 

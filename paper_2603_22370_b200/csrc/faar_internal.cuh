@@ -17,6 +17,11 @@ struct faar_ctx {
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
   int tune_bn;                            // 0 = choose the GEMM tile width automatically
   int last_gemm_bn, last_gemm_pairs;      // what the last GEMM launch used
+  // host-batch path (faar_layer_step_host): copies run on their own stream, ordered by events
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_copied, ev_done[2];
+  unsigned long long host_calls;
+  const void* last_staging;
   // per-kernel timing (faar_profile_begin / faar_profile_end)
   bool prof_on;
   int prof_used;                          // event pairs used since faar_profile_begin

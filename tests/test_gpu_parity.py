@@ -511,3 +511,43 @@ def test_forced_tile_widths_give_the_same_step(ctx, O, K, T, bn):
     for a, b in zip(out[0][:5], out[1][:5]):
         assert np.array_equal(a, b)
     assert abs(out[0][5] - out[1][5]) <= 1e-5 * abs(out[0][5])
+
+
+@pytest.mark.parametrize("two_sets", [True, False])
+def test_layer_step_host_matches_device_steps(ctx, two_sets):
+    """Batches that arrive from pinned host memory (copied on the library's copy stream, with one or
+    two staging sets) must give the same trajectory as the same batches already on the device."""
+    O, K, T = 128, 256, 512
+    W, _ = inputs.config2(2, O, K, T)
+    batches = [inputs.config2(20 + i, 8, K, T)[1] for i in range(5)]
+    yrefs = [inputs.to_bf16_f32(fo.layer_ref(Xb, W)) for Xb in batches]
+    out = []
+    for mode in ("device", "host"):
+        lay = GpuLayer(ctx, W, batches[0])
+        lay.init()
+        losses = []
+        sets = [(torch.empty_like(lay.X), torch.empty_like(lay.Xt), torch.empty((T, O), dtype=torch.bfloat16, device=DEV))
+                for _ in range(2 if two_sets else 1)]
+        pinned = [(torch.from_numpy(Xb).to(torch.bfloat16).pin_memory(), torch.from_numpy(Yb).to(torch.bfloat16).pin_memory())
+                  for Xb, Yb in zip(batches, yrefs)]
+        loss_h = torch.zeros(2).pin_memory()
+        for t, (Xb, Yb) in enumerate(zip(batches, yrefs)):
+            hp = faar.make_hparams(beta=4.0 + t, step=t + 1)
+            if mode == "device":
+                lay.X.copy_(dev_bf16(Xb))
+                faar.transpose_bf16(ctx, T, K, lay.X, K, lay.Xt, lay.ldt)
+                lay.set_yref(Yb)
+                lay.step(hp)
+                torch.cuda.synchronize()
+                losses.append(host(lay.loss).copy())
+            else:
+                Xd, Xtd, Yd = sets[t % len(sets)]
+                faar.layer_step_host(ctx, lay.shape, hp, pinned[t][0], pinned[t][1], Xd, Xtd, Yd, lay.V, lay.code,
+                                     lay.scales, lay.s_global, lay.m, lay.u, lay.loss, loss_h, lay.ws)
+                if t == len(batches) - 1 or not two_sets:
+                    torch.cuda.synchronize()
+                    losses.append(loss_h.numpy().copy())
+        lay.check()
+        out.append((host(lay.V).copy(), host(lay.m).copy(), losses[-1]))
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
+    assert np.array_equal(out[0][2], out[1][2])
