@@ -307,7 +307,7 @@ def layer_step(X, Y_ref, V, code, scales, s_global, m, u, hp, mode="bf16"):
 
 def beta_schedule(t, steps, beta0=4.0, beta1=32.0):
     """Geometric annealing from beta0 to beta1 (the paper says beta starts
-    small and is increased; it gives no values -- these are this build's)."""
+    small and is increased; it gives no values -- these are this harness's)."""
     if steps <= 1:
         return float(beta0)
     return float(beta0 * (beta1 / beta0) ** (t / (steps - 1)))

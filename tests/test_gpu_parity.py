@@ -1,7 +1,7 @@
 """GPU parity: every entry point of libfaar.so, called through the C ABI, against
 the CPU oracle on the same seeded inputs.
 
-Tolerances (from the build's target statement):
+Tolerances:
   * bytes (E4M3 scales, lower-node codes, hardened nibbles, decisions): bit-exact;
   * V_init: bit-exact (binary32 contract);
   * W_soft, h in FP32: |gpu - oracle| <= 1e-6 * |oracle|;
@@ -216,7 +216,8 @@ def test_transpose(ctx, rows, cols):
 
 # (O, K, T): one tile; ragged in every dimension over several 128-wide tiles; enough 256-wide
 # tiles to take the wide-tile path in the forward (O x T) and in the backward (O x K) GEMM.
-GEMM_SHAPES = [(128, 256, 1024), (100, 80, 77), (300, 1040, 600), (1500, 272, 3300), (1500, 3344, 200)]
+GEMM_SHAPES = [(128, 256, 1024), (100, 80, 77), (300, 1040, 600), (1500, 272, 3300), (1500, 3344, 200),
+               (1, 16, 1), (129, 48, 9)]
 
 
 def _problem(O, K, T, seed=0):
