@@ -390,6 +390,23 @@ def act_fake_quant(X, s_global_in=0.0):
     return units, s_global, packed, scales
 
 
+def swizzle_scales(scales):
+    """Block scales [rows, cols] (cols = K/16) in the tiled order that block-scaled tensor-core GEMMs
+    read: the matrix is padded with zeros to multiples of 128 rows and 4 columns and cut into
+    128 x 4 tiles stored one after another (tiles of a row band first); inside a tile the byte of
+    (r, c) sits at (r % 32) * 16 + (r // 32) * 4 + c.  ("Directly deployable" output; the paper gives no
+    layout -- this is the hardware's.)  Written as the definition: one element at a time."""
+    rows, cols = scales.shape
+    rt, ct = (rows + 127) // 128, (cols + 3) // 4
+    out = np.zeros(rt * ct * 512, dtype=np.uint8)
+    for r in range(rows):
+        for c in range(cols):
+            tile = (r // 128) * ct + (c // 4)
+            rr, cc = r % 128, c % 4
+            out[tile * 512 + (rr % 32) * 16 + (rr // 32) * 4 + cc] = scales[r, c]
+    return out
+
+
 def rtn_nearest(W, scales, s_global):
     """Round-to-nearest onto the node set, written independently of the
     bracket: argmin over all 8 nodes of |w~ - node|, a tie going to the larger

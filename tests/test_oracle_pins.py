@@ -402,3 +402,23 @@ def test_act_fake_quant_exact_on_representable_inputs():
     X = np.stack([nodes * 2.0 ** e for e in (-3, 0, 2)]).astype(np.float32)
     units, sg, _, scales = fo.act_fake_quant(X, s_global_in=2.0 ** -3)
     assert np.array_equal((units * float(sg)).astype(np.float32), X)
+
+
+def test_swizzled_scale_layout_is_a_padded_permutation():
+    rng = np.random.default_rng(0)
+    for rows, cols in [(128, 4), (130, 5), (300, 65), (1, 1)]:
+        sc = rng.integers(1, 0x7F, size=(rows, cols)).astype(np.uint8)
+        sw = fo.swizzle_scales(sc)
+        rt, ct = -(-rows // 128), -(-cols // 4)
+        assert sw.size == rt * ct * 512
+        # the same bytes, every one exactly once, the rest padding
+        assert np.array_equal(np.sort(sw[sw != 0]), np.sort(sc.ravel()))
+        # reshape route: [row tile][col tile][r % 32][r // 32][c] is the padded matrix re-indexed
+        padded = np.zeros((rt * 128, ct * 4), np.uint8)
+        padded[:rows, :cols] = sc
+        view = sw.reshape(rt, ct, 32, 4, 4)                     # tile, r % 32, r // 32, c
+        back = view.transpose(0, 3, 2, 1, 4).reshape(rt * 128, ct * 4)   # rows = (rt, r // 32, r % 32)
+        assert np.array_equal(back, padded)
+    # the first 16 bytes of a tile: rows 0, 32, 64, 96 of its four columns
+    sc = np.arange(128 * 4, dtype=np.uint8).reshape(128, 4)
+    assert list(fo.swizzle_scales(sc)[:16]) == [sc[r, c] for r in (0, 32, 64, 96) for c in range(4)]
