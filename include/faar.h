@@ -299,6 +299,19 @@ FAAR_API int faar_harden_pack(faar_ctx* ctx, const faar_shape* shape, const floa
                      const uint8_t* scales, const float* s_global, uint8_t* packed,
                      uint8_t* scales_out, uint8_t* decisions, void* W_final, int wfinal_dtype);
 
+/* ---- deployable scale-factor layout ---------------------------------------
+ * "Hardening and Inference": the final weights are "directly deployable on NVFP4
+ * hardware".  Block-scaled tensor-core GEMMs read the E4M3 block scales not
+ * row-major but in 128-row x 4-column tiles of 512 bytes (tiles of a row band
+ * one after another; byte (r, c) of a tile at (r%32)*16 + (r/32)*4 + c; the
+ * matrix zero-padded to multiples of 128 rows and 4 columns).  This call
+ * rewrites linear scales [rows, cols] (from faar_harden_pack or
+ * faar_act_fakequant; cols = K/16) into that order.
+ *   scales in: [rows, cols] u8      scales_tiled out: ceil(rows/128)*ceil(cols/4)*512 bytes
+ *   (tiled_bytes: size of the output buffer; too small is FAAR_ERR_SHAPE) */
+FAAR_API int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales, uint8_t* scales_tiled,
+                                 size_t tiled_bytes);
+
 #ifdef __cplusplus
 }
 #endif

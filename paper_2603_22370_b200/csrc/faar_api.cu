@@ -515,6 +515,16 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
   return cuda_fail(ctx, (int)e);
 }
 
+int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales, uint8_t* scales_tiled,
+                        size_t tiled_bytes) {
+  if (!ctx || !scales || !scales_tiled) return FAAR_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0) return FAAR_ERR_SHAPE;
+  if (tiled_bytes < (size_t)((rows + 127) / 128) * (size_t)((cols + 3) / 4) * 512) return FAAR_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(scales_tiled) & 3u) return FAAR_ERR_ALIGN;
+  DeviceGuard g(ctx->device);
+  return cuda_fail(ctx, faar_launch_swizzle_scales(ctx, rows, cols, scales, scales_tiled));
+}
+
 int faar_harden_pack(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code, const uint8_t* scales,
                      const float* s_global, uint8_t* packed, uint8_t* scales_out, uint8_t* decisions, void* W_final,
                      int wfinal_dtype) {

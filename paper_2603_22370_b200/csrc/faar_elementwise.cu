@@ -379,6 +379,28 @@ harden_pack_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code
   }
 }
 
+// ---- block scales into the tiled order of block-scaled tensor-core GEMMs ----------------------------
+// Output: 128 x 4 tiles of 512 bytes, tiles of a row band first; byte (r, c) of a tile at
+// (r % 32) * 16 + (r / 32) * 4 + c; rows and columns beyond the matrix are zero.  One thread per output
+// 4-byte word (the four columns of one row of one tile).
+__global__ void __launch_bounds__(EW_THREADS)
+swizzle_scales_kernel(const uint8_t* __restrict__ in, int rows, int cols, uint32_t* __restrict__ out, int64_t n_words) {
+  const int col_tiles = (cols + 3) / 4;
+  for (int64_t w = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; w < n_words; w += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t tile = w >> 7;
+    const int in_tile = (int)(w & 127);                 // (r % 32) * 4 + r / 32
+    const int r = (int)(tile / col_tiles) * 128 + (in_tile & 3) * 32 + (in_tile >> 2);
+    const int c0 = (int)(tile % col_tiles) * 4;
+    uint32_t v = 0;
+    if (r < rows) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (c0 + j < cols) v |= (uint32_t)in[(int64_t)r * cols + c0 + j] << (8 * j);
+    }
+    out[w] = v;
+  }
+}
+
 // ---- BF16 transpose through shared memory -----------------------------------------------
 __global__ void __launch_bounds__(256)
 transpose_bf16_kernel(const uint16_t* __restrict__ in, int rows, int cols, int64_t ld_in,
@@ -457,6 +479,14 @@ int faar_launch_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in
   faar_prof_scope ps(ctx, FAAR_K_TRANSPOSE);
   transpose_bf16_kernel<<<grid, 256, 0, ctx->stream>>>(reinterpret_cast<const uint16_t*>(in), rows, cols, ld_in,
                                                        reinterpret_cast<uint16_t*>(out), ld_out);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* in, uint8_t* out) {
+  const int64_t n_words = (int64_t)((rows + 127) / 128) * ((cols + 3) / 4) * 128;
+  faar_prof_scope ps(ctx, FAAR_K_HARDEN_PACK);
+  swizzle_scales_kernel<<<grid_for(ctx, n_words, 8), EW_THREADS, 0, ctx->stream>>>(in, rows, cols,
+                                                                                  reinterpret_cast<uint32_t*>(out), n_words);
   return (int)cudaGetLastError();
 }
 

@@ -82,6 +82,7 @@ int faar_launch_act_fakequant(faar_ctx*, int T, int K, const void* X, int64_t ld
                               int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales, uint32_t* amax_word);
 int faar_launch_transpose_bf16(faar_ctx*, int rows, int cols, const void* in, int64_t ld_in, void* out,
                                int64_t ld_out);
+int faar_launch_swizzle_scales(faar_ctx*, int rows, int cols, const uint8_t* in, uint8_t* out);
 int faar_launch_round_partials(faar_ctx*, const float* V, int64_t N, float* partials, int* n_partials);
 // out[0] = scale0 * sum(p0[0..n0)), out[1] = scale1 * sum(p1[0..n1)) (either may have n = 0 -> skipped)
 int faar_launch_finalize(faar_ctx*, const float* p0, int n0, float scale0, float* out0, const float* p1,

@@ -21,7 +21,7 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
            "faar_softquant_eval", "faar_transpose_bf16", "faar_layer_ref", "faar_layer_fwd", "faar_round_loss",
            "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
            "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n", "faar_tune_tile_n",
-           "faar_last_gemm_config", "faar_act_fakequant"]
+           "faar_last_gemm_config", "faar_act_fakequant", "faar_swizzle_scales"]
 
 
 class HParams(C.Structure):
@@ -168,6 +168,11 @@ def act_fakequant(ctx, T, K, X, ldx, s_global_in, Xq_units, ldq, s_global_out, p
     _check(lib().faar_act_fakequant(ctx._h, T, K, _p(X), C.c_int64(ldx), C.c_float(s_global_in), _p(Xq_units),
                                     C.c_int64(ldq), _p(s_global_out), _p(packed), _p(scales), _p(ws),
                                     C.c_size_t(ws.numel())), "faar_act_fakequant")
+
+
+def swizzle_scales(ctx, rows, cols, scales, scales_tiled):
+    _check(lib().faar_swizzle_scales(ctx._h, rows, cols, _p(scales), _p(scales_tiled), C.c_size_t(scales_tiled.numel())),
+           "faar_swizzle_scales")
 
 
 def transpose_bf16(ctx, rows, cols, inp, ld_in, out, ld_out):
