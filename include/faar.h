@@ -112,6 +112,12 @@ FAAR_API int faar_last_cuda_error(const faar_ctx* ctx);
  * (0 = automatic again).  faar_last_gemm_config reports the width and the number of CTA pairs of the
  * most recent GEMM launch (host out-pointers). */
 FAAR_API int faar_tune_tile_n(faar_ctx* ctx, int bn);
+/* The last, partly empty wave of tiles: the trailing tile columns can be cut into half-width tiles so
+ * that more CTA pairs share it and the final, un-overlapped epilogue is half as long.  The number of
+ * columns cut is chosen per launch from a cost model; faar_tune_tail_split forces it (-1 = automatic,
+ * 0 = none).  faar_last_tail_split reports what the most recent GEMM launch used. */
+FAAR_API int faar_tune_tail_split(faar_ctx* ctx, int columns);
+FAAR_API int faar_last_tail_split(const faar_ctx* ctx, int* columns);
 FAAR_API int faar_last_gemm_config(const faar_ctx* ctx, int* bn, int* cta_pairs);
 
 /* Bytes of workspace that any call on this shape needs (host out-pointer).

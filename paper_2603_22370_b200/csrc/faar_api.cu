@@ -161,6 +161,8 @@ int faar_create(faar_ctx** out, int device, void* stream) {
   c->last_cuda_error = 0;
   c->encode_tiled = nullptr;
   c->tune_bn = 0;
+  c->tune_tail = -1;
+  c->last_gemm_split = 0;
   c->copy_stream = nullptr;
   c->ev_copied = nullptr;
   c->ev_done[0] = c->ev_done[1] = nullptr;
@@ -257,6 +259,18 @@ int faar_tune_tile_n(faar_ctx* ctx, int bn) {
   if (!ctx) return FAAR_ERR_INVALID_ARG;
   if (bn != 0 && (bn < 128 || bn > 256 || bn % 16 != 0)) return FAAR_ERR_INVALID_ARG;
   ctx->tune_bn = bn;
+  return FAAR_OK;
+}
+
+int faar_tune_tail_split(faar_ctx* ctx, int columns) {
+  if (!ctx || columns < -1) return FAAR_ERR_INVALID_ARG;
+  ctx->tune_tail = columns;
+  return FAAR_OK;
+}
+
+int faar_last_tail_split(const faar_ctx* ctx, int* columns) {
+  if (!ctx || !columns) return FAAR_ERR_INVALID_ARG;
+  *columns = ctx->last_gemm_split;
   return FAAR_OK;
 }
 

@@ -227,6 +227,7 @@ __device__ __forceinline__ uint32_t make_idesc(int bn) {
 struct KParams {
   int M, N, Kc;
   int bn;                 // tile width
+  int n_full_cols;        // tile columns of full width; the columns after them are bn/2 wide (tail split)
   uint32_t* status;
   // REF / FWD
   void* Yout; int yout_dtype; long long ldy;
@@ -244,6 +245,31 @@ struct KParams {
   const float* fin_mse_partials; int fin_n_mse; float fin_scale_mse;
   float fin_scale_round; float* fin_out2;   // {L_MSE, L_round}; null = no final sums here
 };
+
+// Tile t of the launch: the first n_full_cols tile columns are bn wide, the remaining columns bn/2
+// (half-width tiles fill the last, partly empty wave of the CTA pairs and halve the epilogue that
+// nothing overlaps).  Tiles are numbered row block fastest, all full-width tiles first.
+struct TileCoord { int m0, n0, w; };
+__device__ __forceinline__ TileCoord tile_coord(const KParams& p, int t, int m_tiles) {
+  const int full_tiles = m_tiles * p.n_full_cols;
+  TileCoord c;
+  if (t < full_tiles) {
+    c.m0 = (t % m_tiles) * (2 * BM);
+    c.n0 = (t / m_tiles) * p.bn;
+    c.w = p.bn;
+  } else {
+    const int u = t - full_tiles;
+    c.m0 = (u % m_tiles) * (2 * BM);
+    c.n0 = p.n_full_cols * p.bn + (u / m_tiles) * (p.bn / 2);
+    c.w = p.bn / 2;
+  }
+  return c;
+}
+__device__ __forceinline__ int tile_count(const KParams& p, int m_tiles) {
+  const int rest = p.N - p.n_full_cols * p.bn;                    // columns covered by half-width tiles
+  const int half_cols = rest > 0 ? (rest + p.bn / 2 - 1) / (p.bn / 2) : 0;
+  return m_tiles * (p.n_full_cols + half_cols);
+}
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
@@ -418,7 +444,8 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
 // Launched as clusters of two CTAs along x: CTAs 2c and 2c+1 form pair c.
 template <int MODE, int OPT>
 __global__ void __launch_bounds__(Cfg<MODE>::THREADS, 1)
-faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const KParams p) {
+faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmBh, const KParams p) {
   using C = Cfg<MODE>;
   const int BN = p.bn;
   extern __shared__ uint8_t smem_raw[];
@@ -440,8 +467,8 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();             // 0 = leader of the pair
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM), n_tiles = (p.N + BN - 1) / BN;
-  const int total_tiles = m_tiles * n_tiles;
+  const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM);
+  const int total_tiles = tile_count(p, m_tiles);
   const int k_blocks = (p.Kc + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -469,17 +496,19 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
-        const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;
-        const int n0 = (tile / m_tiles) * BN + (int)rank * (BN / 2);
+        const TileCoord tc = tile_coord(p, tile, m_tiles);
+        const int m0 = tc.m0 + (int)rank * BM;
+        const int n0 = tc.n0 + (int)rank * (tc.w / 2);
+        const CUtensorMap* mapB = tc.w == BN ? &tmB : &tmBh;      // box of w/2 rows
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(empty_bar(stage), phase ^ 1u, ac, 0x100u | stage);
           if (!ok) break;
           const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
           // the leader's barrier collects the bytes of both CTAs' copies
-          if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * (uint32_t)(C::A_BYTES + (BN / 2) * BK * 2));
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * (uint32_t)(C::A_BYTES + (tc.w / 2) * BK * 2));
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
           tma_load_2d(sa, &tmA, kb * BK, m0, leader_full, keep);
-          tma_load_2d(sb, &tmB, kb * BK, n0, leader_full, keep);
+          tma_load_2d(sb, mapB, kb * BK, n0, leader_full, keep);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -492,7 +521,6 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   } else if (warp == 1) {
     // ---------------- MMA issuer (leader CTA only) ----------------
     if (lane == 0 && rank == 0) {
-      const uint32_t idesc = make_idesc(BN);
       int stage = 0; uint32_t phase = 0;
       int it = 0;
       bool ok = true;
@@ -503,6 +531,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN_MAX;
+        const uint32_t idesc = make_idesc(tile_coord(p, tile, m_tiles).w);
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(full_bar(stage), phase, ac, 0x300u | stage);
           if (!ok) break;
@@ -525,9 +554,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int ew = warp - 2;
     const int quarter = warp & 3;                      // TMEM lanes this warp may read
     // REF / FWD: the warps that share a lane quarter split the tile's columns in 16-column chunks
-    const int cols_per_warp = ((BN / C::COL_GROUPS + 15) / 16) * 16;
-    const int col_begin = (ew >> 2) * cols_per_warp;
-    const int col_end = min(col_begin + cols_per_warp, BN);
+    const int cg = ew >> 2;                            // which of the warps sharing this lane quarter
     float warp_acc = 0.f;
     float s_global = 0.f;
     if (MODE == FAAR_GEMM_BWD) s_global = *p.s_global;
@@ -541,7 +568,11 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM, n0 = (tile / m_tiles) * BN;
+      const TileCoord tc = tile_coord(p, tile, m_tiles);
+      const int m0 = tc.m0 + (int)rank * BM, n0 = tc.n0, TW = tc.w;
+      const int cols_per_warp = ((TW / C::COL_GROUPS + 15) / 16) * 16;
+      const int col_begin = cg * cols_per_warp;
+      const int col_end = min(col_begin + cols_per_warp, TW);
       const int o = m0 + quarter * 32 + lane;
       const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN_MAX);
       if constexpr (MODE == FAAR_GEMM_BWD) {
@@ -552,13 +583,13 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int o_first = m0 + quarter * 32;
         bool released = false;
 #pragma unroll 1
-        for (int pc = 0; pc < BN; pc += 128) {
+        for (int pc = 0; pc < TW; pc += 128) {
           if (n0 + pc >= p.N || o_first >= p.M) break;   // the same decision in all four warps
           // the quarter's previous panel has been consumed by all four warps
           bool okp = mbar_wait(pdone, (pn & 1u) ^ 1u, ac, 0x500u | quarter);
           if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
           const int c = pc + 32 * sub;
-          if (c < BN && n0 + c < p.N) {
+          if (c < TW && n0 + c < p.N) {
             uint32_t r[32];
             tmem_ld32(trow + (uint32_t)c, r);
             tmem_ld_wait();
@@ -567,7 +598,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
               sts128(panel + (uint32_t)lane * 512u + (uint32_t)(((8 * sub + u) ^ (lane & 7)) << 4), r[4 * u], r[4 * u + 1],
                      r[4 * u + 2], r[4 * u + 3]);
           }
-          if (pc + 128 >= BN || n0 + pc + 128 >= p.N) {  // this warp's last read of the accumulator
+          if (pc + 128 >= TW || n0 + pc + 128 >= p.N) {  // this warp's last read of the accumulator
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
@@ -577,7 +608,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (lane == 0) mbar_arrive(pfull);
           okp = mbar_wait(pfull, pn & 1u, ac, 0x600u | quarter);
           if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
-          const int k_end = min(p.N, n0 + BN);           // columns of this tile that exist
+          const int k_end = min(p.N, n0 + TW);           // columns of this tile that exist
           if (o_first + 32 <= p.M && n0 + pc + 128 <= k_end)
             warp_acc += epi_bwd_rows<OPT, true>(p, panel, lane, sub, o_first, n0 + pc, k_end, s_global);
           else
@@ -691,6 +722,35 @@ int pick_bn(const faar_ctx* ctx, int M, int N, int pairs) {
   return 128;
 }
 
+// How many trailing tile columns to cut into half-width tiles.  Tiles go to CTA pairs round-robin, all
+// full-width tiles first.  A half tile costs 0.75 of a full one (its A rows are loaded all the same), and
+// the epilogue of a pair's last tile is not overlapped by anything (0.4 of that tile's cost).  Returns the
+// number of full-width columns that minimises the busiest pair's time (ties: fewer half tiles).
+int pick_full_cols(const faar_ctx* ctx, int M, int N, int bn, int pairs) {
+  const int m_tiles = (M + 2 * BM - 1) / (2 * BM);
+  const int n_cols = (N + bn - 1) / bn;
+  if (bn % 32 != 0) return n_cols;
+  if (ctx->tune_tail >= 0) return ctx->tune_tail < n_cols ? n_cols - ctx->tune_tail : 0;
+  double best = -1.0;
+  int best_full = n_cols;
+  for (int split = 0; split <= n_cols && split <= 16; ++split) {
+    const int full_cols = n_cols - split;
+    const long long full_tiles = (long long)m_tiles * full_cols;
+    const int rest = N - full_cols * bn;
+    const long long half_tiles = rest > 0 ? (long long)m_tiles * ((rest + bn / 2 - 1) / (bn / 2)) : 0;
+    const long long total = full_tiles + half_tiles;
+    double worst = 0.0;
+    for (int p = 0; p < pairs && p < total; ++p) {
+      double load = 0.0, last = 0.0;
+      for (long long t = p; t < total; t += pairs) { last = t < full_tiles ? 1.0 : 0.75; load += last; }
+      load += 0.4 * last;
+      if (load > worst) worst = load;
+    }
+    if (best < 0.0 || worst < best - 1e-9) { best = worst; best_full = full_cols; }
+  }
+  return best_full;
+}
+
 template <int MODE, int OPT = 0>
 int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_out) {
   using C = Cfg<MODE>;
@@ -724,19 +784,25 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
   }
   const int bn = pick_bn(ctx, a->M, a->N, max_pairs);
   kp.bn = bn;
-  CUtensorMap tmA, tmB;
+  kp.n_full_cols = pick_full_cols(ctx, a->M, a->N, bn, max_pairs);
+  CUtensorMap tmA, tmB, tmBh;
   int e = make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
   if (e) return e;
   e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, bn / 2);
   if (e) return e;
-  const long long tiles = (long long)((a->M + 2 * BM - 1) / (2 * BM)) * ((a->N + bn - 1) / bn);
+  e = make_map(ctx, &tmBh, a->B, a->N, a->Kc, a->ldb, bn % 32 == 0 ? bn / 4 : bn / 2);   // half-width tiles
+  if (e) return e;
+  const int rest_cols = a->N - kp.n_full_cols * bn;
+  const long long tiles = (long long)((a->M + 2 * BM - 1) / (2 * BM)) *
+                          (kp.n_full_cols + (rest_cols > 0 ? (rest_cols + bn / 2 - 1) / (bn / 2) : 0));
   const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   if (n_partials_out) *n_partials_out = 2 * pairs * C::EPI_WARPS;
   ctx->last_gemm_bn = bn;
   ctx->last_gemm_pairs = pairs;
+  ctx->last_gemm_split = (a->N + bn - 1) / bn - kp.n_full_cols;
   faar_prof_scope ps(ctx, MODE == FAAR_GEMM_REF ? FAAR_K_GEMM_REF : (MODE == FAAR_GEMM_FWD ? FAAR_K_GEMM_FWD : FAAR_K_GEMM_BWD));
-  ce = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, kp);
+  ce = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmBh, kp);
   if (ce != cudaSuccess) return (int)ce;
   return (int)cudaGetLastError();
 }
@@ -747,7 +813,7 @@ int faar_gemm_max_partials(const faar_ctx* ctx, int, int) { return ctx->num_sms 
 
 int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out) {
   KParams kp;
-  kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.bn = BN_MAX; kp.status = a->status;
+  kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.bn = BN_MAX; kp.n_full_cols = 0; kp.status = a->status;
   kp.Yout = a->Yout; kp.yout_dtype = a->yout_dtype; kp.ldy = a->ldy;
   kp.Yref = a->Yref; kp.yref_dtype = a->yref_dtype;
   kp.dYt = a->dYt; kp.ld_dyt = a->ld_dyt; kp.mse2c = a->mse2c; kp.act_scale = a->act_scale; kp.partials = a->partials;

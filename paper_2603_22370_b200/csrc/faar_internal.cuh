@@ -16,7 +16,8 @@ struct faar_ctx {
   int last_cuda_error;
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
   int tune_bn;                            // 0 = choose the GEMM tile width automatically
-  int last_gemm_bn, last_gemm_pairs;      // what the last GEMM launch used
+  int tune_tail;                          // -1 = choose the tail split automatically, else columns to split
+  int last_gemm_bn, last_gemm_pairs, last_gemm_split;   // what the last GEMM launch used
   // host-batch path (faar_layer_step_host): copies run on their own stream, ordered by events
   cudaStream_t copy_stream;
   cudaEvent_t ev_copied, ev_done[2];

@@ -21,7 +21,8 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
            "faar_softquant_eval", "faar_transpose_bf16", "faar_layer_ref", "faar_layer_fwd", "faar_round_loss",
            "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
            "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n", "faar_tune_tile_n",
-           "faar_last_gemm_config", "faar_act_fakequant", "faar_swizzle_scales"]
+           "faar_last_gemm_config", "faar_act_fakequant", "faar_swizzle_scales", "faar_tune_tail_split",
+           "faar_last_tail_split"]
 
 
 class HParams(C.Structure):
@@ -126,6 +127,17 @@ class Context:
 def tune_tile_n(ctx: Context, bn: int):
     """Forces the GEMM tile width (multiple of 16 in [128, 256]); 0 restores the automatic choice."""
     _check(lib().faar_tune_tile_n(ctx._h, C.c_int(bn)), "faar_tune_tile_n")
+
+
+def tune_tail_split(ctx: Context, columns: int):
+    """Forces how many trailing tile columns are cut into half-width tiles (-1 = automatic, 0 = none)."""
+    _check(lib().faar_tune_tail_split(ctx._h, C.c_int(columns)), "faar_tune_tail_split")
+
+
+def last_tail_split(ctx: Context) -> int:
+    n = C.c_int(0)
+    _check(lib().faar_last_tail_split(ctx._h, C.byref(n)), "faar_last_tail_split")
+    return n.value
 
 
 def last_gemm_config(ctx: Context) -> tuple[int, int]:

@@ -552,3 +552,37 @@ def test_layer_step_host_matches_device_steps(ctx, two_sets):
         out.append((host(lay.V).copy(), host(lay.m).copy(), losses[-1]))
     assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
     assert np.array_equal(out[0][2], out[1][2])
+
+
+@pytest.mark.parametrize("split", [1, 3, 100])
+@pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (520, 784, 1300)])
+def test_half_width_tail_tiles_give_the_same_step(ctx, O, K, T, split):
+    """Cutting trailing tile columns into half-width tiles only re-partitions the output."""
+    W, X, Yref = _problem(O, K, T, seed=6)
+    hp, _ = f32hp(beta=6.0, step=2)
+    rng = np.random.default_rng(4)
+    V0 = rng.uniform(0, 1, W.shape).astype(np.float32)
+    m0 = (1e-3 * rng.standard_normal(W.shape)).astype(np.float32)
+    u0 = (1e-6 * rng.uniform(0, 1, W.shape)).astype(np.float32)
+    out = []
+    try:
+        faar.tune_tile_n(ctx, 256)
+        for cols in (0, split):
+            faar.tune_tail_split(ctx, cols)
+            lay = GpuLayer(ctx, W, X)
+            lay.init()
+            lay.set_yref(Yref)
+            lay.set_state(V=V0, m=m0, u=u0)
+            lay.fwd(hp)
+            dYt = host(lay.dYt).copy()
+            dV = host(lay.bwd(hp, want_dv=True)).copy()
+            if cols:
+                assert faar.last_tail_split(ctx) == min(cols, -(-K // 256))
+            lay.check()
+            out.append((dYt, dV, host(lay.V).copy(), host(lay.m).copy(), host(lay.u).copy(), host(lay.loss)[0]))
+    finally:
+        faar.tune_tail_split(ctx, -1)
+        faar.tune_tile_n(ctx, 0)
+    for a, b in zip(out[0][:5], out[1][:5]):
+        assert np.array_equal(a, b)
+    assert abs(out[0][5] - out[1][5]) <= 1e-5 * abs(out[0][5])
