@@ -131,6 +131,13 @@ FAAR_API int faar_workspace_init(faar_ctx* ctx, void* workspace, size_t workspac
  * FAAR_ERR_CUDA if the stream is in error, else FAAR_OK. */
 FAAR_API int faar_check_status(faar_ctx* ctx, const void* workspace, uint32_t* detail_out);
 
+/* Self-test of the bounded waits (no counterpart in the paper).  Launches one small kernel whose only
+ * wait can never be satisfied and whose limit is `limit_us` microseconds (1 .. 1 000 000): the wait gives
+ * up, records code 0x700 in the workspace status word and the kernel exits normally, so a following
+ * faar_check_status returns FAAR_ERR_TIMEOUT with that code and the context stays usable.  Re-arm with
+ * faar_workspace_init. */
+FAAR_API int faar_selftest_wait_timeout(faar_ctx* ctx, void* workspace, size_t workspace_bytes, unsigned int limit_us);
+
 /* ---- per-kernel timing -------------------------------------------------------
  * (No counterpart in the paper: instrumentation of this library.)
  * Between faar_profile_begin and faar_profile_end every kernel the context

@@ -308,6 +308,15 @@ int faar_check_status(faar_ctx* ctx, const void* workspace, uint32_t* detail_out
   return word ? FAAR_ERR_TIMEOUT : FAAR_OK;
 }
 
+int faar_selftest_wait_timeout(faar_ctx* ctx, void* workspace, size_t workspace_bytes, unsigned int limit_us) {
+  if (!ctx) return FAAR_ERR_INVALID_ARG;
+  if (limit_us == 0 || limit_us > 1000000u) return FAAR_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
+    return FAAR_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  return cuda_fail(ctx, faar_launch_wait_selftest(ctx, reinterpret_cast<uint32_t*>(workspace), 1000ull * limit_us));
+}
+
 int faar_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float s_global_in, uint8_t* scales,
                         float* s_global_out, uint8_t* code, float* V_init, void* workspace,
                         size_t workspace_bytes) {

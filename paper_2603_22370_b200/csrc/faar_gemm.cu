@@ -103,6 +103,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 struct AbortCtl {
   volatile int* flag;     // shared memory
   uint32_t* status;       // global status word
+  unsigned long long limit_ns = WAIT_LIMIT_NS;
 };
 
 // Returns false if the wait was abandoned (time limit, or another thread raised the flag).
@@ -112,7 +113,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 0xFF) == 0) {
       if (*ac.flag) return false;
-      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+      if (global_ns() - t0 > ac.limit_ns) {
         atomicCAS(ac.status, 0u, code);
         *ac.flag = 1;
         return false;
@@ -692,6 +693,24 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
 }
 
+// A wait that nothing will ever satisfy, with a short limit: exercises the give-up path of the bounded
+// waits (status word, flag, orderly exit) without any other kernel machinery.
+__global__ void __launch_bounds__(64, 1) wait_selftest_kernel(uint32_t* status, unsigned long long limit_ns) {
+  __shared__ alignas(8) unsigned long long bar;
+  __shared__ int flag;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  AbortCtl ac{&flag, status, limit_ns};
+  if (threadIdx.x == 0) (void)mbar_wait(b, 0u, ac, 0x700u);       // nobody arrives: gives up after limit_ns
+  __syncthreads();
+  if (threadIdx.x == 32) (void)mbar_wait(b, 0u, ac, 0x701u);      // sees the raised flag and leaves at once
+}
+
 // ---- host side ----------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -808,6 +827,11 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
 }
 
 }  // namespace
+
+int faar_launch_wait_selftest(faar_ctx* ctx, uint32_t* status, unsigned long long limit_ns) {
+  wait_selftest_kernel<<<1, 64, 0, ctx->stream>>>(status, limit_ns);
+  return (int)cudaGetLastError();
+}
 
 int faar_gemm_max_partials(const faar_ctx* ctx, int, int) { return ctx->num_sms * MAX_EPI_WARPS; }
 

@@ -118,6 +118,7 @@ struct faar_gemm_args {
 // n_partials_out: number of floats written to args.partials
 int faar_launch_gemm(faar_ctx*, const faar_gemm_args*, int* n_partials_out);
 int faar_gemm_max_partials(const faar_ctx*, int M, int N);
+int faar_launch_wait_selftest(faar_ctx*, uint32_t* status, unsigned long long limit_ns);
 
 // ---- device helpers -----------------------------------------------------------
 #ifdef __CUDACC__

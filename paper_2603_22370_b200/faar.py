@@ -22,7 +22,7 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
            "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
            "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n", "faar_tune_tile_n",
            "faar_last_gemm_config", "faar_act_fakequant", "faar_swizzle_scales", "faar_tune_tail_split",
-           "faar_last_tail_split"]
+           "faar_last_tail_split", "faar_selftest_wait_timeout"]
 
 
 class HParams(C.Structure):
@@ -155,6 +155,11 @@ def workspace_size(shape: Shape) -> int:
 
 def workspace_init(ctx: Context, ws: torch.Tensor):
     _check(lib().faar_workspace_init(ctx._h, _p(ws), C.c_size_t(ws.numel())), "faar_workspace_init")
+
+
+def selftest_wait_timeout(ctx: Context, ws: torch.Tensor, limit_us: int = 1000):
+    _check(lib().faar_selftest_wait_timeout(ctx._h, _p(ws), C.c_size_t(ws.numel()), C.c_uint(limit_us)),
+           "faar_selftest_wait_timeout")
 
 
 def check_status(ctx: Context, ws: torch.Tensor) -> int:

@@ -586,3 +586,23 @@ def test_half_width_tail_tiles_give_the_same_step(ctx, O, K, T, split):
     for a, b in zip(out[0][:5], out[1][:5]):
         assert np.array_equal(a, b)
     assert abs(out[0][5] - out[1][5]) <= 1e-5 * abs(out[0][5])
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives(ctx):
+    """The tensor-core kernels bound every barrier wait.  The self-test kernel waits (1 ms limit) on a
+    barrier that nothing arrives at: it must exit by itself, leave its code in the status word, and the
+    library must keep working afterwards."""
+    ws = torch.zeros(4096, dtype=torch.uint8, device=DEV)
+    faar.workspace_init(ctx, ws)
+    faar.selftest_wait_timeout(ctx, ws, 1000)
+    with pytest.raises(faar.FaarError) as err:
+        faar.check_status(ctx, ws)
+    assert err.value.status == faar.ERR_TIMEOUT and "0x700" in str(err.value)
+    faar.workspace_init(ctx, ws)
+    assert faar.check_status(ctx, ws) == faar.OK
+    W, X, Yref = _problem(128, 256, 256)
+    lay = GpuLayer(ctx, W, X)
+    lay.init()
+    lay.set_yref(Yref)
+    lay.step(f32hp()[0])
+    lay.check()
