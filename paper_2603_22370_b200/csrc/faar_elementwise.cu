@@ -232,6 +232,7 @@ softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ c
     lut[threadIdx.x] = make_float2(sgn * faar_node(k), sgn * faar_width(k));
   }
   __syncthreads();
+  faar_pdl_sync();                                   // V comes from the previous step's backward kernel
   const float s_global = *s_global_p;
   const float nhb = -0.5f * beta;
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups;
@@ -468,8 +469,18 @@ int faar_launch_softquant_eval(faar_ctx* ctx, const faar_shape* s, const float* 
                                float* h, __nv_bfloat16* W_bf16) {
   const int64_t groups = (int64_t)s->O * (s->K / 8);
   faar_prof_scope ps(ctx, FAAR_K_SOFT_WEIGHTS);
-  softquant_eval_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(V, code, scales, s_global, beta,
-                                                                                  groups, W_soft, h, W_bf16);
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = dim3(grid_for(ctx, groups, 8), 1, 1);
+  cfg.blockDim = dim3(EW_THREADS, 1, 1);
+  cfg.stream = ctx->stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, softquant_eval_kernel, V, code, scales, s_global, beta, (int64_t)groups, W_soft,
+                                     h, W_bf16);
+  if (e != cudaSuccess) return (int)e;
   return (int)cudaGetLastError();
 }
 

@@ -488,6 +488,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   tc_fence_before();
   cluster_sync_all();                                  // barriers of both CTAs are initialised
   tc_fence_after();
+  faar_pdl_sync();                                     // set-up done; now wait for the previous kernel's data
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
@@ -781,16 +782,18 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
   if (ce != cudaSuccess) return (int)ce;
 
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.blockDim = dim3(C::THREADS, 1, 1);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = ctx->stream;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   // how many CTA pairs the device can hold at once (a GPC with an odd SM count strands one SM)
   static int max_pairs = 0;                      // per kernel instantiation
   if (max_pairs == 0) {

@@ -188,6 +188,15 @@ __device__ __forceinline__ float faar_soft_weight(float h, uint32_t nib, float s
   return (nib & 8) ? -mag : mag;
 }
 
+// Programmatic dependent launch: the step's kernels are launched with stream serialisation relaxed, so
+// that a kernel's CTAs may start (and run their set-up) on SMs that the previous kernel has already
+// left.  faar_pdl_sync() lets the next kernel do the same and then waits until the previous kernel has
+// completed and its memory is visible; nothing before it may touch global data.
+__device__ __forceinline__ void faar_pdl_sync() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ float faar_warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
