@@ -262,6 +262,16 @@ def layer_grad(dY, X, V, code, scales, s_global, beta, lambda_round):
     return dV, G
 
 
+def layer_dx(dY, V, code, scales, s_global, beta, mode="bf16"):
+    """Gradient with respect to the layer's input: dX = dY W_soft (the derivative of Y_q = X W_soft^T;
+    what full-model alignment, Procedure steps 16-23, must pass on to the layer below).  In mode "bf16"
+    W_soft is the BF16 operand of the forward GEMM.  Returns dX [T,K], float64."""
+    W_soft, _ = soft_weights(V, code, scales, s_global, beta)
+    if mode == "bf16":
+        W_soft = bf16_round(W_soft)
+    return np.asarray(dY, np.float64) @ W_soft
+
+
 def adam_update(V, g, m, u, lr, beta1, beta2, eps, step):
     """Adam with bias correction (step is 1-based), then the clip to [0, 1]
     that Stage 1 prescribes after each gradient update.  float64 in/out."""

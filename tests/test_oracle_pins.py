@@ -422,3 +422,27 @@ def test_swizzled_scale_layout_is_a_padded_permutation():
     # the first 16 bytes of a tile: rows 0, 32, 64, 96 of its four columns
     sc = np.arange(128 * 4, dtype=np.uint8).reshape(128, 4)
     assert list(fo.swizzle_scales(sc)[:16]) == [sc[r, c] for r in (0, 32, 64, 96) for c in range(4)]
+
+
+def test_layer_dx_matches_finite_differences_of_the_mse_term():
+    rng = np.random.default_rng(11)
+    W = (0.02 * rng.standard_normal((6, 32))).astype(np.float32)
+    X = rng.standard_normal((5, 32))
+    scales, sg, code, V = fo.softquant_init(W)
+    V = rng.uniform(0, 1, V.shape)
+    Yref = fo.layer_ref(X, W)
+    beta, c = 6.0, 0.7
+    _, dY, _ = fo.layer_fwd(X, Yref, V, code, scales, sg, beta, c, "smooth")
+    dX = fo.layer_dx(dY, V, code, scales, sg, beta, "smooth")
+    eps = 1e-6
+    for (t, k) in [(0, 0), (4, 31), (2, 17), (3, 5)]:
+        Xp, Xm = X.copy(), X.copy()
+        Xp[t, k] += eps
+        Xm[t, k] -= eps
+        lp, _, _ = fo.layer_fwd(Xp, Yref, V, code, scales, sg, beta, c, "smooth")
+        lm, _, _ = fo.layer_fwd(Xm, Yref, V, code, scales, sg, beta, c, "smooth")
+        fd = (lp - lm) / (2 * eps)
+        assert abs(fd - dX[t, k]) <= 1e-6 * max(abs(dX[t, k]), 1e-6) + 1e-9
+    # transposed operand or a missing factor would show here: dX has X's shape and scales with dY
+    assert dX.shape == X.shape
+    assert np.allclose(fo.layer_dx(2 * dY, V, code, scales, sg, beta, "smooth"), 2 * dX)
