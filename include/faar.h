@@ -237,6 +237,17 @@ FAAR_API int faar_layer_fwd(faar_ctx* ctx, const faar_shape* shape, const faar_h
                    const float* s_global, void* dYt, float* loss_mse, void* Y_q,
                    void* workspace, size_t workspace_bytes);
 
+/* ---- input gradient (towards full-model alignment) ----------------------------
+ * Procedure steps 16-23 train the rounding variables of all layers through the
+ * whole model; a layer must then also pass the gradient on to its input:
+ * dX = dY W_soft (the derivative of Y_q = X W_soft^T, W_soft as in faar_layer_fwd).
+ * Soft weights, a transpose into the caller's scratch and one tensor-core GEMM.
+ *   dY     in : [T,O] bf16 (ldy, multiple of 8)      dX out: [T,K] bf16 (ldx, multiple of 8)
+ *   WsoftT scratch: [K, O rounded up to 8] bf16, overwritten */
+FAAR_API int faar_layer_dx(faar_ctx* ctx, const faar_shape* shape, float beta, const void* dY, const float* V,
+                           const uint8_t* code, const uint8_t* scales, const float* s_global, void* WsoftT,
+                           void* dX, void* workspace, size_t workspace_bytes);
+
 /* ---- part 4: Round Loss, backward, update -----------------------------------
  * Eq. 5, second term without lambda: L_round = (1/N) sum (1 - (2v-1)^2).
  *   V in: N floats     loss_round out: 1 float (device) */

@@ -399,6 +399,38 @@ int faar_layer_ref(faar_ctx* ctx, const faar_shape* s, const void* X, const void
   return cuda_fail(ctx, faar_launch_gemm(ctx, &a, nullptr));
 }
 
+int faar_layer_dx(faar_ctx* ctx, const faar_shape* s, float beta, const void* dY, const float* V, const uint8_t* code,
+                  const uint8_t* scales, const float* s_global, void* WsoftT, void* dX, void* workspace,
+                  size_t workspace_bytes) {
+  if (!ctx || !dY || !V || !code || !scales || !s_global || !WsoftT || !dX) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if (!(beta > 0.f) || !isfinite(beta)) return FAAR_ERR_INVALID_ARG;
+  if (s->ldy < s->O || s->ldx < s->K) return FAAR_ERR_SHAPE;
+  if (s->ldy % 8 || s->ldx % 8 || !aligned16(dY) || !aligned16(V) || !aligned16(code) || !aligned16(WsoftT) ||
+      !aligned16(dX))
+    return FAAR_ERR_ALIGN;
+  if ((st = check_ws(s, workspace, workspace_bytes))) return st;
+  DeviceGuard g(ctx->device);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const faar_ws_layout l = faar_ws_plan(s);
+  __nv_bfloat16* wsoft = reinterpret_cast<__nv_bfloat16*>(ws + l.off_wsoft);
+  const int64_t ldo = ((int64_t)s->O + 7) / 8 * 8;
+  int e = faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, beta, nullptr, nullptr, wsoft);
+  if (e) return cuda_fail(ctx, e);
+  e = faar_launch_transpose_bf16(ctx, s->O, s->K, wsoft, s->K, WsoftT, ldo);
+  if (e) return cuda_fail(ctx, e);
+  // dX^T[K,T] = WsoftT[K,O] * dY[T,O]^T, written transposed as dX[T,K]
+  faar_gemm_args a = {};
+  a.mode = FAAR_GEMM_REF;
+  a.M = s->K; a.N = s->T; a.Kc = s->O;
+  a.A = WsoftT; a.lda = ldo;
+  a.B = dY; a.ldb = s->ldy;
+  a.status = reinterpret_cast<uint32_t*>(ws);
+  a.Yout = dX; a.yout_dtype = FAAR_BF16; a.ldy = s->ldx;
+  return cuda_fail(ctx, faar_launch_gemm(ctx, &a, nullptr));
+}
+
 int faar_layer_fwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Y_ref,
                    const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
                    float* loss_mse, void* Y_q, void* workspace, size_t workspace_bytes) {

@@ -22,7 +22,7 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
            "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
            "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n", "faar_tune_tile_n",
            "faar_last_gemm_config", "faar_act_fakequant", "faar_swizzle_scales", "faar_tune_tail_split",
-           "faar_last_tail_split", "faar_selftest_wait_timeout"]
+           "faar_last_tail_split", "faar_selftest_wait_timeout", "faar_layer_dx"]
 
 
 class HParams(C.Structure):
@@ -206,6 +206,11 @@ def layer_fwd(ctx, shape, hp, X, Y_ref, V, code, scales, s_global, dYt, loss_mse
     _check(lib().faar_layer_fwd(ctx._h, C.byref(shape), C.byref(hp), _p(X), _p(Y_ref), _p(V), _p(code), _p(scales),
                                 _p(s_global), _p(dYt), _p(loss_mse), _p(Y_q), _p(ws), C.c_size_t(ws.numel())),
            "faar_layer_fwd")
+
+
+def layer_dx(ctx, shape, beta, dY, V, code, scales, s_global, WsoftT, dX, ws):
+    _check(lib().faar_layer_dx(ctx._h, C.byref(shape), C.c_float(beta), _p(dY), _p(V), _p(code), _p(scales),
+                               _p(s_global), _p(WsoftT), _p(dX), _p(ws), C.c_size_t(ws.numel())), "faar_layer_dx")
 
 
 def round_loss(ctx, V, N, loss_round, ws):

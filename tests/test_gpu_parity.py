@@ -606,3 +606,25 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(ctx):
     lay.set_yref(Yref)
     lay.step(f32hp()[0])
     lay.check()
+
+
+@pytest.mark.parametrize("O,K,T", [(128, 256, 1024), (304, 1040, 600), (96, 80, 77)])
+def test_layer_dx(ctx, O, K, T):
+    W, X, _ = _problem(O, K, T, seed=8)
+    lay = GpuLayer(ctx, W, X)
+    lay.init()
+    rng = np.random.default_rng(5)
+    V = rng.uniform(0, 1, W.shape).astype(np.float32)
+    lay.set_state(V=V)
+    dY = inputs.to_bf16_f32(rng.standard_normal((T, O)).astype(np.float32))
+    ldo = (O + 7) // 8 * 8
+    dYd = torch.zeros((T, ldo), dtype=torch.bfloat16, device=DEV)
+    dYd[:, :O] = dev_bf16(dY)
+    lay.shape.ldy = ldo
+    WsT = torch.empty((K, ldo), dtype=torch.bfloat16, device=DEV)
+    dX = torch.empty((T, K), dtype=torch.bfloat16, device=DEV)
+    beta = float(np.float32(7.0))
+    faar.layer_dx(ctx, lay.shape, beta, dYd, lay.V, lay.code, lay.scales, lay.s_global, WsT, dX, lay.ws)
+    lay.check()
+    dX_o = fo.layer_dx(dY, V, host(lay.code), host(lay.scales), host(lay.s_global)[0], beta, "bf16")
+    assert rel_l2(host(dX), dX_o) <= 3e-3 and max_rel_to_peak(host(dX), dX_o) <= 4e-3     # BF16 output: 2^-8 rounding
