@@ -85,13 +85,16 @@ typedef struct {
  * ldw : row stride of W[O,K]          (>= K)
  * ldx : row stride of X[T,K]          (>= K, multiple of 8)
  * ldxt: row stride of Xt[K,T] = X^T   (>= T, multiple of 8)
- * ldy : row stride of Y_ref[T,O] and of the optional Y_q output (>= O)
+ * ldy : row stride of Y_ref[T,O] and of the optional Y_q output (>= O); with yref_transposed != 0
+ *       both are stored as [O, ldy] (one row per output feature), ldy >= T rounded up to 16, so that
+ *       the forward epilogue reads its target values as 16-byte vectors
  * V, code, scales, adam_m, adam_u, dV are dense (row strides K, K/2, K/16, K). */
 typedef struct {
   int O, K, T;
   int64_t ldw, ldx, ldxt, ldy;
   int w_dtype;    /* faar_dtype of W      */
   int yref_dtype; /* faar_dtype of Y_ref  */
+  int yref_transposed; /* 0: Y_ref[T,O]; 1: Y_ref stored as [O, ldy] */
 } faar_shape;
 
 /* ---- context -------------------------------------------------------------- */

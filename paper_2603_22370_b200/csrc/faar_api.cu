@@ -22,6 +22,16 @@ int check_shape(const faar_shape* s) {
   return FAAR_OK;
 }
 
+// Leading dimension of Y_ref / Y_q for the layout the shape declares.
+int check_ldy(const faar_shape* s) {
+  if (s->yref_transposed) {
+    if (s->ldy < ((int64_t)s->T + 15) / 16 * 16) return FAAR_ERR_SHAPE;
+    if (s->ldy % 8) return FAAR_ERR_ALIGN;
+    return FAAR_OK;
+  }
+  return s->ldy < s->O ? FAAR_ERR_SHAPE : FAAR_OK;
+}
+
 int check_ws(const faar_shape* s, const void* ws, size_t ws_bytes) {
   if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return FAAR_ERR_WORKSPACE;
   if (ws_bytes < faar_ws_plan(s).total) return FAAR_ERR_WORKSPACE;
@@ -62,7 +72,7 @@ int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
   a.B = X; a.ldb = s->ldx;
   a.status = reinterpret_cast<uint32_t*>(ws);
   a.Yout = Y_q; a.yout_dtype = FAAR_BF16; a.ldy = s->ldy;
-  a.Yref = Y_ref; a.yref_dtype = s->yref_dtype;
+  a.Yref = Y_ref; a.yref_dtype = s->yref_dtype; a.yref_t = s->yref_transposed;
   a.dYt = reinterpret_cast<__nv_bfloat16*>(dYt); a.ld_dyt = l.ld_dyt;
   a.mse2c = 2.0f * hp->mse_scale;
   a.act_scale = hp->act_scale > 0.f ? hp->act_scale : 1.0f;
@@ -383,7 +393,8 @@ int faar_layer_ref(faar_ctx* ctx, const faar_shape* s, const void* X, const void
   if (st) return st;
   if (s->w_dtype != FAAR_BF16) return FAAR_ERR_DTYPE;
   if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
-  if (s->ldw < s->K || s->ldy < s->O) return FAAR_ERR_SHAPE;
+  if (s->ldw < s->K) return FAAR_ERR_SHAPE;
+  if ((st = check_ldy(s))) return st;
   if ((st = check_gemm_operands(s, true, false))) return st;
   if (s->ldw % 8 || !aligned16(X) || !aligned16(W)) return FAAR_ERR_ALIGN;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
@@ -395,7 +406,7 @@ int faar_layer_ref(faar_ctx* ctx, const faar_shape* s, const void* X, const void
   a.A = W; a.lda = s->ldw;
   a.B = X; a.ldb = s->ldx;
   a.status = reinterpret_cast<uint32_t*>(workspace);
-  a.Yout = Y_ref; a.yout_dtype = s->yref_dtype; a.ldy = s->ldy;
+  a.Yout = Y_ref; a.yout_dtype = s->yref_dtype; a.ldy = s->ldy; a.yref_t = s->yref_transposed;
   return cuda_fail(ctx, faar_launch_gemm(ctx, &a, nullptr));
 }
 
@@ -439,7 +450,7 @@ int faar_layer_fwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, c
   if (st) return st;
   if ((st = check_hp(hp, false))) return st;
   if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
-  if (s->ldy < s->O) return FAAR_ERR_SHAPE;
+  if ((st = check_ldy(s))) return st;
   if ((st = check_gemm_operands(s, true, false))) return st;
   if (!aligned16(X) || !aligned16(V) || !aligned16(code) || !aligned16(dYt)) return FAAR_ERR_ALIGN;
   if ((st = check_ws(s, workspace, workspace_bytes))) return st;
@@ -500,7 +511,7 @@ int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, 
   if ((st = check_hp(hp, true))) return st;
   if (hp->opt == 1 && (!adam_m || !adam_u)) return FAAR_ERR_INVALID_ARG;
   if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
-  if (s->ldy < s->O) return FAAR_ERR_SHAPE;
+  if ((st = check_ldy(s))) return st;
   if ((st = check_gemm_operands(s, true, true))) return st;
   if (!aligned16(X) || !aligned16(Xt) || !aligned16(V) || !aligned16(code) || (adam_m && !aligned16(adam_m)) ||
       (adam_u && !aligned16(adam_u)))
@@ -528,7 +539,7 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
   int st = check_shape(s);
   if (st) return st;
   if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
-  if (s->ldy < s->O) return FAAR_ERR_SHAPE;
+  if ((st = check_ldy(s))) return st;
   if ((st = check_gemm_operands(s, true, true))) return st;
   DeviceGuard g(ctx->device);
   cudaError_t e = cudaSuccess;
@@ -555,7 +566,8 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(X_dev, X_host, (size_t)s->T * (size_t)s->ldx * 2, cudaMemcpyHostToDevice, ctx->copy_stream);
   if (e == cudaSuccess)
-    e = cudaMemcpyAsync(Yref_dev, Y_ref_host, (size_t)s->T * (size_t)s->ldy * ybytes, cudaMemcpyHostToDevice,
+    e = cudaMemcpyAsync(Yref_dev, Y_ref_host, (size_t)(s->yref_transposed ? s->O : s->T) * (size_t)s->ldy * ybytes,
+                        cudaMemcpyHostToDevice,
                         ctx->copy_stream);
   if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_copied, ctx->copy_stream);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->stream, ctx->ev_copied, 0);

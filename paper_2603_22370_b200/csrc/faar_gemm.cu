@@ -233,6 +233,7 @@ struct KParams {
   // REF / FWD
   void* Yout; int yout_dtype; long long ldy;
   const void* Yref; int yref_dtype;
+  int yref_t;             // Y_ref / Y_out stored transposed: [O, ldy] with ldy >= T rounded up to 16
   __nv_bfloat16* dYt; long long ld_dyt;
   float mse2c;
   float act_scale;        // FWD: Y_q = act_scale * acc; BWD: G = act_scale * acc
@@ -281,6 +282,26 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
 // REF: write acc to Y[t, o].
 __device__ __forceinline__ void epi_ref(const KParams& p, int o, int t0, const uint32_t (&acc)[16]) {
   if (o >= p.M) return;
+  if (p.yref_t) {                                    // row o of the transposed target: 16 contiguous values
+    // (the row is padded to a multiple of 16, so a full vector store stays inside it)
+    if (p.yout_dtype == FAAR_BF16) {
+      uint4* d4 = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.Yout) + (long long)o * p.ldy + t0);
+      float a[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) a[j] = (t0 + j < p.N) ? __uint_as_float(acc[j]) : 0.f;
+      d4[0] = make_uint4(pack_bf16x2(a[0], a[1]), pack_bf16x2(a[2], a[3]), pack_bf16x2(a[4], a[5]), pack_bf16x2(a[6], a[7]));
+      d4[1] = make_uint4(pack_bf16x2(a[8], a[9]), pack_bf16x2(a[10], a[11]), pack_bf16x2(a[12], a[13]), pack_bf16x2(a[14], a[15]));
+    } else {
+      float4* d4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.Yout) + (long long)o * p.ldy + t0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        d4[q] = make_float4((t0 + 4 * q < p.N) ? __uint_as_float(acc[4 * q]) : 0.f,
+                            (t0 + 4 * q + 1 < p.N) ? __uint_as_float(acc[4 * q + 1]) : 0.f,
+                            (t0 + 4 * q + 2 < p.N) ? __uint_as_float(acc[4 * q + 2]) : 0.f,
+                            (t0 + 4 * q + 3 < p.N) ? __uint_as_float(acc[4 * q + 3]) : 0.f);
+    }
+    return;
+  }
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     int t = t0 + j;
@@ -295,9 +316,26 @@ __device__ __forceinline__ void epi_ref(const KParams& p, int o, int t0, const u
 }
 
 // FWD: residual, sum of squares, dY^T.
-__device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const uint32_t (&acc)[16]) {
-  if (o >= p.M) return 0.f;
-  float yr[16];
+// Y_ref[t0..t0+15, o] for this lane's output feature o.
+__device__ __forceinline__ void load_yref(const KParams& p, int o, int t0, float (&yr)[16]) {
+  if (o >= p.M) return;
+  if (p.yref_t) {
+    if (p.yref_dtype == FAAR_BF16) {
+      const uint4* y4 = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.Yref) + (long long)o * p.ldy + t0);
+      const uint4 a = y4[0], b = y4[1];
+      const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        yr[2 * i] = __uint_as_float(w[i] << 16);
+        yr[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+      }
+    } else {
+      const float4* y4 = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.Yref) + (long long)o * p.ldy + t0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) { const float4 v = y4[q]; yr[4 * q] = v.x; yr[4 * q + 1] = v.y; yr[4 * q + 2] = v.z; yr[4 * q + 3] = v.w; }
+    }
+    return;
+  }
   if (p.yref_dtype == FAAR_BF16) {
     const __nv_bfloat16* y = reinterpret_cast<const __nv_bfloat16*>(p.Yref);
 #pragma unroll
@@ -307,6 +345,10 @@ __device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const 
 #pragma unroll
     for (int j = 0; j < 16; ++j) yr[j] = (t0 + j < p.N) ? y[(long long)(t0 + j) * p.ldy + o] : 0.f;
   }
+}
+
+__device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const uint32_t (&acc)[16], const float (&yr)[16]) {
+  if (o >= p.M) return 0.f;
   float ss = 0.f;
   float dy[16];
 #pragma unroll
@@ -330,7 +372,9 @@ __device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const 
     __nv_bfloat16* yq = reinterpret_cast<__nv_bfloat16*>(p.Yout);
 #pragma unroll
     for (int j = 0; j < 16; ++j)
-      if (t0 + j < p.N) yq[(long long)(t0 + j) * p.ldy + o] = __float2bfloat16_rn(__uint_as_float(acc[j]) * p.act_scale);
+      if (t0 + j < p.N)
+        yq[p.yref_t ? (long long)o * p.ldy + t0 + j : (long long)(t0 + j) * p.ldy + o] =
+            __float2bfloat16_rn(__uint_as_float(acc[j]) * p.act_scale);
   }
   return ss;
 }
@@ -627,14 +671,54 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         continue;
       } else {
+        if (MODE == FAAR_GEMM_FWD && p.yref_t && p.yref_dtype == FAAR_BF16) {
+          // transposed BF16 target: this lane's 64 values of four chunks are requested together
+          // (eight 16-byte loads in flight), so a tile costs two load latencies instead of one per chunk
 #pragma unroll 1
-        for (int c = col_begin; c < col_end; c += 16) {
-          if (n0 + c >= p.N) break;                    // warp-uniform
-          uint32_t r[16];
-          tmem_ld16(trow + (uint32_t)c, r);
-          tmem_ld_wait();
-          if (MODE == FAAR_GEMM_REF) epi_ref(p, o, n0 + c, r);
-          else warp_acc += epi_fwd(p, o, n0 + c, r);
+          for (int cb = col_begin; cb < col_end; cb += 64) {
+            if (n0 + cb >= p.N) break;                   // warp-uniform
+            uint4 yraw[8];
+            if (o < p.M) {
+              const uint4* y4 = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.Yref) +
+                                                               (long long)o * p.ldy + n0 + cb);
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                if (cb + 16 * q < col_end && n0 + cb + 16 * q < p.N) { yraw[2 * q] = y4[2 * q]; yraw[2 * q + 1] = y4[2 * q + 1]; }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const int c = cb + 16 * q;
+              if (c < col_end && n0 + c < p.N) {         // warp-uniform
+                uint32_t r[16];
+                tmem_ld16(trow + (uint32_t)c, r);
+                tmem_ld_wait();
+                const uint32_t w[8] = {yraw[2 * q].x, yraw[2 * q].y, yraw[2 * q].z, yraw[2 * q].w,
+                                       yraw[2 * q + 1].x, yraw[2 * q + 1].y, yraw[2 * q + 1].z, yraw[2 * q + 1].w};
+                float yr[16];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  yr[2 * i] = __uint_as_float(w[i] << 16);
+                  yr[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+                }
+                warp_acc += epi_fwd(p, o, n0 + c, r, yr);
+              }
+            }
+          }
+        } else {
+#pragma unroll 1
+          for (int c = col_begin; c < col_end; c += 16) {
+            if (n0 + c >= p.N) break;                    // warp-uniform
+            uint32_t r[16];
+            tmem_ld16(trow + (uint32_t)c, r);
+            tmem_ld_wait();
+            if (MODE == FAAR_GEMM_REF) {
+              epi_ref(p, o, n0 + c, r);
+            } else {
+              float yr[16];
+              load_yref(p, o, n0 + c, yr);
+              warp_acc += epi_fwd(p, o, n0 + c, r, yr);
+            }
+          }
         }
       }
       tc_fence_before();
@@ -842,7 +926,7 @@ int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out
   KParams kp;
   kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.bn = BN_MAX; kp.n_full_cols = 0; kp.status = a->status;
   kp.Yout = a->Yout; kp.yout_dtype = a->yout_dtype; kp.ldy = a->ldy;
-  kp.Yref = a->Yref; kp.yref_dtype = a->yref_dtype;
+  kp.Yref = a->Yref; kp.yref_dtype = a->yref_dtype; kp.yref_t = a->yref_t;
   kp.dYt = a->dYt; kp.ld_dyt = a->ld_dyt; kp.mse2c = a->mse2c; kp.act_scale = a->act_scale; kp.partials = a->partials;
   kp.V = a->V; kp.code = a->code; kp.scales = a->scales; kp.s_global = a->s_global;
   kp.adam_m = a->adam_m; kp.adam_u = a->adam_u; kp.dV = a->dV;

@@ -103,6 +103,7 @@ struct faar_gemm_args {
   // REF / FWD
   void* Yout; int yout_dtype; int64_t ldy;     // [N(T), M(O)] written transposed; nullable in FWD
   const void* Yref; int yref_dtype;            // FWD
+  int yref_t;                                  // REF, FWD: Y stored transposed [O, ldy]
   __nv_bfloat16* dYt; int64_t ld_dyt;          // FWD: [M(O), ld_dyt]
   float mse2c;                                 // FWD: 2 * mse_scale
   float act_scale;                             // FWD, BWD: tensor scale of quantised activations (1 = none)

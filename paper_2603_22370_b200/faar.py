@@ -33,7 +33,8 @@ class HParams(C.Structure):
 
 class Shape(C.Structure):
     _fields_ = [("O", C.c_int), ("K", C.c_int), ("T", C.c_int), ("ldw", C.c_int64), ("ldx", C.c_int64),
-                ("ldxt", C.c_int64), ("ldy", C.c_int64), ("w_dtype", C.c_int), ("yref_dtype", C.c_int)]
+                ("ldxt", C.c_int64), ("ldy", C.c_int64), ("w_dtype", C.c_int), ("yref_dtype", C.c_int),
+                ("yref_transposed", C.c_int)]
 
 
 class FaarError(RuntimeError):
@@ -78,9 +79,13 @@ def _check(status: int, where: str):
         raise FaarError(status, where)
 
 
-def make_shape(O, K, T, ldw=None, ldx=None, ldxt=None, ldy=None, w_dtype=BF16, yref_dtype=BF16) -> Shape:
+def make_shape(O, K, T, ldw=None, ldx=None, ldxt=None, ldy=None, w_dtype=BF16, yref_dtype=BF16,
+               yref_transposed=0) -> Shape:
+    """yref_transposed: Y_ref (and the optional Y_q) are stored [O, ldy], ldy >= T rounded up to 16."""
+    if ldy is None:
+        ldy = (T + 15) // 16 * 16 if yref_transposed else O
     return Shape(O, K, T, ldw if ldw is not None else K, ldx if ldx is not None else K,
-                 ldxt if ldxt is not None else (T + 7) // 8 * 8, ldy if ldy is not None else O, w_dtype, yref_dtype)
+                 ldxt if ldxt is not None else (T + 7) // 8 * 8, ldy, w_dtype, yref_dtype, yref_transposed)
 
 
 def make_hparams(beta=4.0, lambda_round=1.0, mse_scale=1.0, opt=1, lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8,

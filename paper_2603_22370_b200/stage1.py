@@ -31,7 +31,7 @@ def optimise_layer(ctx: faar.Context, W: torch.Tensor, X: torch.Tensor, steps: i
     O, K = W.shape
     T = X.shape[0]
     ldt = (T + 7) // 8 * 8
-    shape = faar.make_shape(O, K, T, ldxt=ldt)
+    shape = faar.make_shape(O, K, T, ldxt=ldt, yref_transposed=1)   # the target lives one row per output feature
     ws = torch.empty(faar.workspace_size(shape), dtype=torch.uint8, device=dev)
     faar.workspace_init(ctx, ws)
     scales = torch.empty((O, K // 16), dtype=torch.uint8, device=dev)
@@ -40,7 +40,7 @@ def optimise_layer(ctx: faar.Context, W: torch.Tensor, X: torch.Tensor, steps: i
     V = torch.empty((O, K), dtype=torch.float32, device=dev)
     m = torch.zeros((O, K), dtype=torch.float32, device=dev) if opt == 1 else None
     u = torch.zeros((O, K), dtype=torch.float32, device=dev) if opt == 1 else None
-    Yref = torch.empty((T, O), dtype=torch.bfloat16, device=dev)
+    Yref = torch.zeros((O, shape.ldy), dtype=torch.bfloat16, device=dev)
     loss = torch.zeros(2, dtype=torch.float32, device=dev)
 
     faar.softquant_init(ctx, shape, W, 0.0, scales, s_global, code, V, ws)

@@ -30,13 +30,15 @@ class GpuLayer:
     """Device state of one layer problem: buffers allocated with torch, every
     operation performed by libfaar."""
 
-    def __init__(self, ctx, W, X, w_dtype=faar.BF16, yref_dtype=faar.BF16):
+    def __init__(self, ctx, W, X, w_dtype=faar.BF16, yref_dtype=faar.BF16, yref_transposed=0):
         self.ctx = ctx
         O, K = W.shape
         T = X.shape[0]
         self.O, self.K, self.T = O, K, T
         self.ldt = (T + 7) // 8 * 8
-        self.shape = faar.make_shape(O, K, T, ldxt=self.ldt, w_dtype=w_dtype, yref_dtype=yref_dtype)
+        self.yt = yref_transposed
+        self.shape = faar.make_shape(O, K, T, ldxt=self.ldt, w_dtype=w_dtype, yref_dtype=yref_dtype,
+                                     yref_transposed=yref_transposed)
         self.ws = ctx.workspace(self.shape)
         self.W = dev_bf16(W) if w_dtype == faar.BF16 else dev_f32(W)
         self.X = dev_bf16(X)
@@ -57,7 +59,12 @@ class GpuLayer:
                             self.V, self.ws)
 
     def set_yref(self, Yref):
-        self.Yref = dev_bf16(Yref) if self.shape.yref_dtype == faar.BF16 else dev_f32(Yref)
+        y = dev_bf16(Yref) if self.shape.yref_dtype == faar.BF16 else dev_f32(Yref)
+        if self.yt:                                   # stored [O, ldy], rows padded to a multiple of 16
+            buf = torch.zeros((self.O, self.shape.ldy), dtype=y.dtype, device=DEV)
+            buf[:, :self.T] = y.t()
+            y = buf
+        self.Yref = y
 
     def set_state(self, V=None, m=None, u=None):
         if V is not None:
@@ -68,10 +75,12 @@ class GpuLayer:
             self.u.copy_(dev_f32(u))
 
     def fwd(self, hp, want_yq=False):
-        Yq = torch.empty((self.T, self.O), dtype=torch.bfloat16, device=DEV) if want_yq else None
+        Yq = None
+        if want_yq:
+            Yq = torch.zeros((self.O, self.shape.ldy) if self.yt else (self.T, self.O), dtype=torch.bfloat16, device=DEV)
         faar.layer_fwd(self.ctx, self.shape, hp, self.X, self.Yref, self.V, self.code, self.scales, self.s_global,
                        self.dYt, self.loss[0:1], Yq, self.ws)
-        return Yq
+        return Yq[:, :self.T].t() if (want_yq and self.yt) else Yq
 
     def bwd(self, hp, want_dv=True):
         dV = torch.empty((self.O, self.K), dtype=torch.float32, device=DEV) if want_dv else None

@@ -628,3 +628,37 @@ def test_layer_dx(ctx, O, K, T):
     lay.check()
     dX_o = fo.layer_dx(dY, V, host(lay.code), host(lay.scales), host(lay.s_global)[0], beta, "bf16")
     assert rel_l2(host(dX), dX_o) <= 3e-3 and max_rel_to_peak(host(dX), dX_o) <= 4e-3     # BF16 output: 2^-8 rounding
+
+
+@pytest.mark.parametrize("yref_dtype", [faar.BF16, faar.F32])
+@pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (129, 48, 9), (128, 256, 1024)])
+def test_transposed_target_layout_gives_the_same_results(ctx, O, K, T, yref_dtype):
+    """Y_ref (and Y_q) stored one row per output feature: the frozen target, the forward pass and a whole
+    step must equal, bit for bit, what the [T, O] layout gives (the loss up to the grouping of its sum)."""
+    W, X, Yref = _problem(O, K, T, seed=9)
+    hp, _ = f32hp(beta=6.0, step=1)
+    res = []
+    for yt in (0, 1):
+        lay = GpuLayer(ctx, W, X, yref_dtype=yref_dtype, yref_transposed=yt)
+        lay.init()
+        ldy = lay.shape.ldy
+        Y = torch.zeros((O, ldy) if yt else (T, O), dtype=torch.bfloat16 if yref_dtype == faar.BF16 else torch.float32,
+                        device=DEV)
+        faar.layer_ref(ctx, lay.shape, lay.X, lay.W, Y, lay.ws)
+        Yg = host(Y)[:, :T].T if yt else host(Y)
+        lay.set_yref(Yref)
+        Yq = lay.fwd(hp, want_yq=True)
+        dYt = host(lay.dYt).copy()
+        l_fwd = host(lay.loss)[0]
+        lay.step(hp)
+        lay.check()
+        res.append((Yg.copy(), host(Yq).copy(), dYt, host(lay.V).copy(), l_fwd))
+    for a, b in zip(res[0][:4], res[1][:4]):
+        assert np.array_equal(a, b)
+    assert abs(res[0][4] - res[1][4]) <= 1e-5 * abs(res[0][4])
+    # a row stride below T rounded up to 16 is refused
+    bad = faar.make_shape(O, K, T, yref_transposed=1, ldy=T if T % 16 else T - 16)
+    lay = GpuLayer(ctx, W, X)
+    with pytest.raises(faar.FaarError) as e:
+        faar.layer_ref(ctx, bad, lay.X, lay.W, torch.zeros(O * (T + 16), dtype=torch.bfloat16, device=DEV), lay.ws)
+    assert e.value.status in (faar.ERR_SHAPE, faar.ERR_ALIGN)
