@@ -385,6 +385,16 @@ __device__ __forceinline__ float sqrt_approx(float x) {       // sqrt(0) = 0, ab
   asm("sqrt.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ float width_of(uint32_t k) {       // interval widths .5 .5 .5 .5 1 1 2
   return __uint_as_float((126u + ((0x2500u >> (2u * k)) & 3u)) << 23);
 }
@@ -393,11 +403,13 @@ __device__ __forceinline__ float width_of(uint32_t k) {       // interval widths
 // shared memory (row r at panel + 512 r, its 16-byte units XOR-swizzled by (r & 7)); then warp `sub`
 // of the quarter takes rows 8 sub .. 8 sub + 7 and lane l the columns 4l..4l+3, so that one warp
 // instruction moves 512 contiguous bytes of one row of V / m / u: long bursts for the HBM, full lines
-// as 16-byte vectors.  The per-weight state of two rows is requested together before either is
-// computed.  FULL: the panel lies wholly inside the matrix (no bounds tests).
+// as 16-byte vectors.  The per-weight state of RPG rows is requested together before any of them is
+// computed (one row measured fastest: the sixteen warps of a CTA already keep 24 KB of state loads in
+// flight between them).  FULL: the panel lies wholly inside the matrix (no bounds tests).
 // o_first: output feature of panel row 0; k_first: input feature of panel column 0; k_end: first
 // input feature beyond the tile (or the matrix).
 // Returns the Round Loss contribution of the pre-update v's.
+constexpr int RPG = 1;
 template <int OPT, bool FULL>
 __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, int lane, int sub, int o_first,
                                               int k_first, int k_end, float s_global) {
@@ -410,19 +422,22 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
   float* const Up = p.adam_u + e0;
   const uint8_t* const Cp = p.code + (e0 >> 1);
   const uint8_t* const Sp = p.scales + (e0 >> 4);
-  const float hb = -0.5f * p.beta;
+  const float bl = p.beta * 1.44269504088896341f;                 // beta log2(e): e^x as 2^(x log2 e)
+  const float hbl = -0.5f * bl;
   const float c1 = 1.f - p.b1, c2 = 1.f - p.b2;
   const float step_size = p.lr * p.inv_bc1;
+  const float rbc2 = sqrtf(p.inv_bc2);                            // sqrt(u / bc2) = sqrt(u) sqrt(1 / bc2)
+  const float lam4 = -4.f * p.lam_over_n;                         // (lambda / N) (4 - 8 v) = lam4 (2 v - 1)
   const uint64_t stream = l2_policy_stream();
-  float rl = 0.f;
+  float tt = 0.f, n_el = 0.f;                                     // sum of (2 v - 1)^2, elements seen
 #pragma unroll
-  for (int grp = 0; grp < 4; ++grp) {
-    float4 v[2], m[2], u[2];
-    uint32_t cw[2], sb[2];
-    bool ok[2];
+  for (int grp = 0; grp < 8 / RPG; ++grp) {
+    float4 v[RPG], m[RPG], u[RPG];
+    uint32_t cw[RPG], sb[RPG];
+    bool ok[RPG];
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      const int i = 2 * grp + q;                                      // row r0 + i
+    for (int q = 0; q < RPG; ++q) {
+      const int i = RPG * grp + q;                                      // row r0 + i
       ok[q] = FULL || (col_ok && o_first + r0 + i < p.M);
       if (ok[q]) {
         const int off = i * p.N;
@@ -436,9 +451,9 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
       }
     }
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
+    for (int q = 0; q < RPG; ++q) {
       if (ok[q]) {
-        const int i = 2 * grp + q;
+        const int i = RPG * grp + q;
         const int row = r0 + i;
         const int off = i * p.N;
         const float4 g4 = lds128(panel + (uint32_t)row * 512u + (uint32_t)((lane ^ (row & 7)) << 4));
@@ -454,24 +469,22 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const uint32_t nib = (cw[q] >> (4 * j)) & 0xFu;
-          const float z = fmaf(p.beta, vv[j], hb);
-          const float ex = __expf(-fabsf(z));
-          const float hs = __fdividef(1.0f, 1.0f + ex);
+          const float ex = ex2_approx(-fabsf(fmaf(bl, vv[j], hbl)));         // e^-|beta (v - 0.5)|
+          const float hs = rcp_approx(1.0f + ex);
           const float dh = ex * hs * hs;                                     // h (1 - h)
           float chain = sbeta * width_of(nib & 7u) * dh;
           chain = __uint_as_float(__float_as_uint(chain) ^ ((nib & 8u) << 28));   // sign of w
-          g[j] = fmaf(G[j], chain, p.lam_over_n * fmaf(-8.f, vv[j], 4.f));
           const float t = fmaf(2.f, vv[j], -1.f);
-          rl += fmaf(-t, t, 1.f);
+          g[j] = fmaf(G[j], chain, lam4 * t);
+          tt = fmaf(t, t, tt);
           if (OPT == 1) {
             mn[j] = fmaf(p.b1, mm[j], c1 * g[j]);
             un[j] = fmaf(p.b2, uu[j], c2 * g[j] * g[j]);
-            const float den = sqrt_approx(un[j] * p.inv_bc2) + p.eps;
-            vn[j] = fmaf(-step_size, __fdividef(mn[j], den), vv[j]);
+            const float den = fmaf(sqrt_approx(un[j]), rbc2, p.eps);
+            vn[j] = __saturatef(fmaf(-step_size, mn[j] * rcp_approx(den), vv[j]));   // clip to [0, 1]
           } else {
-            vn[j] = fmaf(-p.lr, g[j], vv[j]);
+            vn[j] = __saturatef(fmaf(-p.lr, g[j], vv[j]));
           }
-          vn[j] = fminf(fmaxf(vn[j], 0.f), 1.f);
         }
         if (p.dV) stg128_stream(p.dV + e0 + off, g[0], g[1], g[2], g[3], stream);
         if (OPT == 1) {
@@ -479,10 +492,11 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
           stg128_stream(Up + off, un[0], un[1], un[2], un[3], stream);
         }
         stg128_stream(Vp + off, vn[0], vn[1], vn[2], vn[3], stream);
+        n_el += 4.f;
       }
     }
   }
-  return rl;
+  return n_el - tt;                                               // sum of 1 - (2 v - 1)^2
 }
 
 // ---- the kernel ------------------------------------------------------------------------------
