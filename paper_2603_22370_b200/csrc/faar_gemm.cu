@@ -395,9 +395,6 @@ __device__ __forceinline__ float rcp_approx(float x) {
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ float width_of(uint32_t k) {       // interval widths .5 .5 .5 .5 1 1 2
-  return __uint_as_float((126u + ((0x2500u >> (2u * k)) & 3u)) << 23);
-}
 
 // The four epilogue warps that share a TMEM lane quarter stage a 32-row x 128-column panel of G in
 // shared memory (row r at panel + 512 r, its 16-byte units XOR-swizzled by (r & 7)); then warp `sub`
@@ -459,7 +456,10 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
         const float4 g4 = lds128(panel + (uint32_t)row * 512u + (uint32_t)((lane ^ (row & 7)) << 4));
         const float G[4] = {g4.x, g4.y, g4.z, g4.w};
         const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
-        const float sbeta = __fmul_rn(faar_e4m3_to_float(sb[q]), s_global) * p.beta * p.act_scale;   // act_scale: G = act_scale * acc
+        // s beta / 2 (the narrowest interval is 0.5 wide); act_scale: G = act_scale * acc
+        const float sbh = __fmul_rn(faar_e4m3_to_float(sb[q]), s_global) * (0.5f * p.beta * p.act_scale);
+        // byte j: log2 of (interval width / 0.5) of element j, looked up by its interval index k (0 0 0 0 1 1 2)
+        const uint32_t wlog = __byte_perm(0u, 0x00020101u, cw[q] & 0x7777u);
         float g[4], vn[4], mn[4], un[4];
         float mm[4], uu[4];
         if (OPT == 1) {
@@ -468,12 +468,14 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const uint32_t nib = (cw[q] >> (4 * j)) & 0xFu;
           const float ex = ex2_approx(-fabsf(fmaf(bl, vv[j], hbl)));         // e^-|beta (v - 0.5)|
           const float hs = rcp_approx(1.0f + ex);
           const float dh = ex * hs * hs;                                     // h (1 - h)
-          float chain = sbeta * width_of(nib & 7u) * dh;
-          chain = __uint_as_float(__float_as_uint(chain) ^ ((nib & 8u) << 28));   // sign of w
+          // dh times the width factor by an add to its exponent field (a dh flushed to 0 becomes ~1e-38), then
+          // the sign of w from bit 3 of the nibble
+          const uint32_t wexp = (j < 3 ? wlog << (23 - 8 * j) : wlog >> 1) & 0x01800000u;
+          float chain = sbh * __uint_as_float(__float_as_uint(dh) + wexp);
+          chain = __uint_as_float(__float_as_uint(chain) ^ ((cw[q] << (28 - 4 * j)) & 0x80000000u));
           const float t = fmaf(2.f, vv[j], -1.f);
           g[j] = fmaf(G[j], chain, lam4 * t);
           tt = fmaf(t, t, tt);
