@@ -32,7 +32,8 @@ constexpr int BM = 128;                // accumulator rows per CTA; the CTA pair
 constexpr int BK = 64;                 // 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
-constexpr int PANEL_BYTES = 32 * 128 * 4;      // BWD epilogue: one 32-row x 128-column FP32 panel per TMEM lane quarter
+constexpr int PW = 64;                         // BWD epilogue: columns of a staged panel of G
+constexpr int PANEL_BYTES = 32 * PW * 4;       // one 32-row x PW-column FP32 panel per TMEM lane quarter
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int CTL_BYTES = 512;
 constexpr int MAX_EPI_WARPS = 16;
@@ -187,16 +188,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -396,23 +387,29 @@ __device__ __forceinline__ float rcp_approx(float x) {
   return y;
 }
 
-// The four epilogue warps that share a TMEM lane quarter stage a 32-row x 128-column panel of G in
-// shared memory (row r at panel + 512 r, its 16-byte units XOR-swizzled by (r & 7)); then warp `sub`
-// of the quarter takes rows 8 sub .. 8 sub + 7 and lane l the columns 4l..4l+3, so that one warp
-// instruction moves 512 contiguous bytes of one row of V / m / u: long bursts for the HBM, full lines
-// as 16-byte vectors.  The per-weight state of RPG rows is requested together before any of them is
-// computed (one row measured fastest: the sixteen warps of a CTA already keep 24 KB of state loads in
-// flight between them).  FULL: the panel lies wholly inside the matrix (no bounds tests).
+// The four epilogue warps that share a TMEM lane quarter stage a 32-row x PW-column panel of G in
+// shared memory (row r at panel + 4 PW r, its 16-byte units XOR-swizzled by (r & 7)); then warp `sub`
+// of the quarter takes rows 8 sub .. 8 sub + 7, LPR = PW / 4 lanes per row and lane l the columns
+// 4 (l % LPR)..+3, so that one warp instruction moves 512 bytes of V / m / u as 32 / LPR row pieces of
+// 4 PW contiguous bytes each: whole lines as 16-byte vectors.  (A panel of 128 columns gives one 512-byte
+// piece per instruction but leaves room for five TMA stages only; the sixth stage is worth more.)
+// The per-weight state of RPG such instructions is requested together before any of it is computed
+// (one measured fastest: the sixteen warps of a CTA already keep 24 KB of state loads in flight).
+// FULL: the panel lies wholly inside the matrix (no bounds tests).
 // o_first: output feature of panel row 0; k_first: input feature of panel column 0; k_end: first
 // input feature beyond the tile (or the matrix).
 // Returns the Round Loss contribution of the pre-update v's.
 constexpr int RPG = 1;
+constexpr int LPR = PW / 4;                     // lanes per panel row
+constexpr int RPI = 32 / LPR;                   // rows per warp instruction
+constexpr int ITS = 8 / RPI;                    // instructions per warp and panel
 template <int OPT, bool FULL>
 __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, int lane, int sub, int o_first,
                                               int k_first, int k_end, float s_global) {
-  const int kcol = k_first + 4 * lane;
+  const int cu = lane % LPR;                                       // 16-byte unit of the row
+  const int kcol = k_first + 4 * cu;
   const bool col_ok = FULL || kcol < k_end;
-  const int r0 = 8 * sub;
+  const int r0 = 8 * sub + lane / LPR;                             // this lane's row in the first instruction
   const long long e0 = (long long)(o_first + r0) * p.N + kcol;     // row r0 element of this lane
   float* const Vp = p.V + e0;
   float* const Mp = p.adam_m + e0;
@@ -428,13 +425,13 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
   const uint64_t stream = l2_policy_stream();
   float tt = 0.f, n_el = 0.f;                                     // sum of (2 v - 1)^2, elements seen
 #pragma unroll
-  for (int grp = 0; grp < 8 / RPG; ++grp) {
+  for (int grp = 0; grp < ITS / RPG; ++grp) {
     float4 v[RPG], m[RPG], u[RPG];
     uint32_t cw[RPG], sb[RPG];
     bool ok[RPG];
 #pragma unroll
     for (int q = 0; q < RPG; ++q) {
-      const int i = RPG * grp + q;                                      // row r0 + i
+      const int i = RPI * (RPG * grp + q);                              // row r0 + i
       ok[q] = FULL || (col_ok && o_first + r0 + i < p.M);
       if (ok[q]) {
         const int off = i * p.N;
@@ -450,10 +447,10 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
 #pragma unroll
     for (int q = 0; q < RPG; ++q) {
       if (ok[q]) {
-        const int i = RPG * grp + q;
+        const int i = RPI * (RPG * grp + q);
         const int row = r0 + i;
         const int off = i * p.N;
-        const float4 g4 = lds128(panel + (uint32_t)row * 512u + (uint32_t)((lane ^ (row & 7)) << 4));
+        const float4 g4 = lds128(panel + (uint32_t)row * (4u * PW) + (uint32_t)((cu ^ (row & 7)) << 4));
         const float G[4] = {g4.x, g4.y, g4.z, g4.w};
         const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
         // s beta / 2 (the narrowest interval is 0.5 wide); act_scale: G = act_scale * acc
@@ -638,29 +635,30 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const int o = m0 + quarter * 32 + lane;
       const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN_MAX);
       if constexpr (MODE == FAAR_GEMM_BWD) {
-        // 128-column panels, staged by the four warps of this lane quarter together (see epi_bwd_rows)
+        // PW-column panels, staged by the four warps of this lane quarter together (see epi_bwd_rows)
         const int sub = ew >> 2;
         const uint32_t panel = epi_u32 + (uint32_t)quarter * PANEL_BYTES;
         const uint32_t pfull = ctl_u32 + 256u + 16u * quarter, pdone = pfull + 8u;
         const int o_first = m0 + quarter * 32;
         bool released = false;
 #pragma unroll 1
-        for (int pc = 0; pc < TW; pc += 128) {
+        for (int pc = 0; pc < TW; pc += PW) {
           if (n0 + pc >= p.N || o_first >= p.M) break;   // the same decision in all four warps
           // the quarter's previous panel has been consumed by all four warps
           bool okp = mbar_wait(pdone, (pn & 1u) ^ 1u, ac, 0x500u | quarter);
           if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
-          const int c = pc + 32 * sub;
+          static_assert(PW == 64, "each of the four warps stages PW / 4 = 16 accumulator columns");
+          const int c = pc + 16 * sub;
           if (c < TW && n0 + c < p.N) {
-            uint32_t r[32];
-            tmem_ld32(trow + (uint32_t)c, r);
+            uint32_t r[16];
+            tmem_ld16(trow + (uint32_t)c, r);
             tmem_ld_wait();
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
-              sts128(panel + (uint32_t)lane * 512u + (uint32_t)(((8 * sub + u) ^ (lane & 7)) << 4), r[4 * u], r[4 * u + 1],
-                     r[4 * u + 2], r[4 * u + 3]);
+            for (int u = 0; u < 4; ++u)
+              sts128(panel + (uint32_t)lane * (4u * PW) + (uint32_t)(((4 * sub + u) ^ (lane & 7)) << 4), r[4 * u],
+                     r[4 * u + 1], r[4 * u + 2], r[4 * u + 3]);
           }
-          if (pc + 128 >= TW || n0 + pc + 128 >= p.N) {  // this warp's last read of the accumulator
+          if (pc + PW >= TW || n0 + pc + PW >= p.N) {    // this warp's last read of the accumulator
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
@@ -671,7 +669,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           okp = mbar_wait(pfull, pn & 1u, ac, 0x600u | quarter);
           if (!__all_sync(0xffffffffu, okp)) { dead = true; break; }
           const int k_end = min(p.N, n0 + TW);           // columns of this tile that exist
-          if (o_first + 32 <= p.M && n0 + pc + 128 <= k_end)
+          if (o_first + 32 <= p.M && n0 + pc + PW <= k_end)
             warp_acc += epi_bwd_rows<OPT, true>(p, panel, lane, sub, o_first, n0 + pc, k_end, s_global);
           else
             warp_acc += epi_bwd_rows<OPT, false>(p, panel, lane, sub, o_first, n0 + pc, k_end, s_global);
