@@ -177,14 +177,14 @@ act_fakequant_kernel(const __nv_bfloat16* __restrict__ X, int T, int K, int64_t 
     for (int i = 0; i < 8; ++i) {
       float wt = s > 0.f ? __fdiv_rn(fabsf(w[i]), s) : 0.f;
       wt = fminf(wt, 6.0f);
-      const int t = (int)(__float_as_uint(wt) >> 22) - 252;
-      int k = wt < 0.5f ? 0 : max(t, 1);
-      k = min(k, 6);
-      const float lo = faar_node(k);
-      const float inv_w = __uint_as_float((uint32_t)(128 - (k >= 4) - (k >= 6)) << 23);   // 2, 1, 0.5
-      const float v = __fmul_rn(__fsub_rn(wt, lo), inv_w);
-      const int c = k + (v >= 0.5f ? 1 : 0);
-      const float mag = __fmul_rn(faar_node(c), sg);              // exact: 3 x 4 significant bits
+      // Nearest node, a tie to the larger one.  From 1 upwards the nodes are the floats with a one-bit
+      // mantissa: add a quarter of the binade and cut the mantissa to its top bit (5 -> 6, 3.5 -> 4,
+      // 1.25 -> 1.5; 6 stays 6).  Below 1 the nodes 0, 0.5, 1 are 0.5 apart.
+      const uint32_t rb = (__float_as_uint(wt) + 0x00200000u) & 0xFFC00000u;
+      const float node = wt >= 1.0f ? __uint_as_float(rb) : (wt >= 0.75f ? 1.0f : (wt >= 0.25f ? 0.5f : 0.0f));
+      // E2M1 magnitude code of the node: 0, 0.5 -> 0, 1; from 1 upwards exponent and mantissa bit count on
+      const int c = node >= 1.0f ? (int)(__float_as_uint(node) >> 22) - 252 : (node > 0.0f ? 1 : 0);
+      const float mag = __fmul_rn(node, sg);                      // exact: 2 x 4 significant bits
       const bool neg = w[i] < 0.f;
       q[i] = neg ? -mag : mag;
       cw |= ((uint32_t)c | (neg ? 8u : 0u)) << (4 * i);

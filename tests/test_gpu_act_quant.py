@@ -44,12 +44,17 @@ def test_act_fakequant_bit_exact(ctx, T, K, ldx, sg_in):
     _, X = inputs.config2(3, 8, K, T)
     X[0, :16] = 0.0
     X[1, 16] = -0.0
+    # a block whose scale is a power of two when the tensor scale is 2^-7 (block amax 6 * 8 * 2^-7), holding
+    # every midpoint between two nodes: exact ties, which go to the larger node
+    X[2, :16] = np.array([6, 5, 3.5, 2.5, 1.75, 1.25, 0.75, 0.25, -5, -3.5, -2.5, -1.75, -1.25, -0.75, -0.25, 0.125]) * 0.0625
     Xq, sx, packed, scales = _quantise(ctx, X, sg_in, ldx)
     units, sg, packed_o, scales_o = fo.act_fake_quant(X, sg_in)
     assert host(sx)[0] == sg
     assert np.array_equal(host(scales), scales_o)
     assert np.array_equal(host(packed), packed_o)
     assert np.array_equal(host(Xq).astype(np.float64), units)
+    if sg_in > 0:       # the ties went up: 5 -> 6, 3.5 -> 4, ..., 0.25 -> 0.5 in units of the block scale 8
+        assert np.array_equal(units[2, :16], 8.0 * np.array([6, 6, 4, 3, 2, 1.5, 1, 0.5, -6, -4, -3, -2, -1.5, -1, -0.5, 0]))
     # outputs are optional
     ws = ctx.workspace(faar.make_shape(16, 16, 8))
     Xq2 = torch.zeros_like(Xq)

@@ -102,6 +102,22 @@ def test_softquant_init_adversarial_values_strided_and_given_scale(ctx):
     _check_init(ctx, np.zeros((4, 32), np.float32), faar.BF16)
 
 
+def test_softquant_init_extreme_scales_and_exact_quotients(ctx):
+    """Bit for bit against the oracle where the quotient |w| / s is delicate: a scale whose significand is
+    all ones (tensor scale (2 - 2^-23) * 2^-9 times a power-of-two block scale), scales near the ends of
+    the exponent range, values that are powers of two, node midpoints, or 2^-60 of the block's largest."""
+    rng = np.random.default_rng(17)
+    mids = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0, 1.0, 2.0, 4.0, 0.5, 3.0, 1.5, 0.125, 0.0])
+    for sg, mag in ((float(np.float32(2.0 - 2.0 ** -23) * np.float32(2.0 ** -9)), 2.0 ** -6),
+                    (float(np.float32(2.0 ** -70)), 2.0 ** -66), (float(np.float32(2.0 ** 62)), 2.0 ** 66)):
+        W = (rng.standard_normal((24, 64)) * mag).astype(np.float32)
+        W[0, :16] = mids * mag * 4
+        W[1, 16:32] = -mids * mag
+        W[2, :] = 2.0 ** np.floor(np.log2(mag)) * 2.0 ** -rng.integers(0, 4, 64)
+        W[3, :8] = mag * 2.0 ** -60
+        _check_init(ctx, W, faar.F32, s_global_in=sg)
+
+
 # ---------------------------------------------------------------------------------------------
 # part 2: soft weights in FP32
 # ---------------------------------------------------------------------------------------------
