@@ -232,13 +232,20 @@ def run_ours(args):
         faar.layer_ref(ctx, shape, X, W, Yref, ws)           # frozen target (Procedure step 8)
     stream.synchronize()
 
+    def chain_kw(t, n):
+        """--chain: the backward pass of step t also builds step t+1's soft weights and step t+1 skips the
+        soft-weights kernel (the same values bit for bit; two kernels per step instead of three)."""
+        if not args.chain:
+            return {}
+        return dict(wsoft_ready=int(t > 0), beta_next=beta_at(t + 1, n) if t + 1 < n else 0.0)
+
     def job(n_steps, step0=0):
         """set-up, n_steps optimisation steps, harden + pack -- all enqueued on `stream`."""
         m.zero_()
         u.zero_()
         faar.softquant_init(ctx, shape, W, 0.0, scales, s_global, code, V, ws)
         for t in range(n_steps):
-            hp = faar.make_hparams(beta=beta_at(t, n_steps), step=t + 1)
+            hp = faar.make_hparams(beta=beta_at(t, n_steps), step=t + 1, **chain_kw(t, n_steps))
             faar.layer_step(ctx, shape, hp, X, Xt, Yref, V, code, scales, s_global, m, u, loss, ws)
         faar.harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, None, None)
 
@@ -275,7 +282,8 @@ def run_ours(args):
     faar.check_status(ctx, ws)
     loss_final = loss.cpu().tolist()
     value = n_gpus * steps / (ms_job * 1e-3)
-    gpu_launches = 2 + 3 * steps + 1     # amax + init, 3 kernels per step (soft weights, forward, backward), harden_pack
+    # amax + init; soft weights + forward + backward per step (chained: one soft-weights launch in all); harden_pack
+    gpu_launches = 2 + (1 + 2 * steps if args.chain else 3 * steps) + 1
 
     # ---- second pass of the same job with per-kernel CUDA events (library hooks, same stream)
     def profiled():
@@ -340,7 +348,7 @@ def run_ours(args):
         u.zero_()
         faar.softquant_init(ctx, shape, W, 0.0, scales, s_global, code, V, ws)
         for t in range(n):
-            hp = faar.make_hparams(beta=beta_at(t, n), step=t + 1)
+            hp = faar.make_hparams(beta=beta_at(t, n), step=t + 1, **chain_kw(t, n))
             X_dev, Xt_dev, Y_dev = stage_sets[t & 1]
             faar.layer_step_host(ctx, shape, hp, Xh, Yh, X_dev, Xt_dev, Y_dev, V, code, scales, s_global, m, u,
                                  loss, loss_h, ws)
@@ -411,7 +419,8 @@ def run_ours(args):
             "config": {"workload": WORKLOAD, "O": O, "K": K, "T": T,
                        "l2": "no flush: one step touches about 410 MB (X, X^T, V, m, u, W_soft, Y_ref, dY^T, codes), "
                              "more than the 126 MB L2",
-                       "timed_region": "softquant_init + K x layer_step + harden_pack, inputs resident in HBM"},
+                       "timed_region": "softquant_init + K x layer_step + harden_pack, inputs resident in HBM",
+                       "chained_soft_weights": bool(args.chain)},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
                     "h2d_bytes_per_step": T * K * 2 + T * O * 2, "d2h_bytes_per_step": 8,
@@ -432,6 +441,9 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--chain", action="store_true",
+                    help="build each step's soft weights inside the previous step's backward kernel (same values; the "
+                         "job is faster, the backward kernel slower, so its roofline line is not comparable)")
     ap.add_argument("--quick", action="store_true",
                     help="timed job and per-kernel pass only (no end-to-end pass, no CPU oracle leg); for profilers")
     args = ap.parse_args()

@@ -79,6 +79,17 @@ typedef struct {
    * the forward / backward calls then holds X_q / act_scale, and Y_q and the weight gradient are
    * multiplied by act_scale in the GEMM epilogues.  0 (or 1) = activations as given. */
   float act_scale;
+  /* Chaining of consecutive steps on one workspace (both 0 = every step stands alone).  Eq. 2 is a
+   * function of each weight's own v, so the backward pass, which holds the updated v' in registers,
+   * can build the next step's forward operand on the way out.
+   * beta_next > 0: the backward pass also writes, into the workspace, the BF16 forward operand
+   *   W_soft(V', beta_next) of the NEXT step.
+   * wsoft_ready != 0: the caller states that the previous backward (or step) call on this workspace
+   *   was given beta_next == this step's beta and that V has not been touched since; the forward pass
+   *   then reads that operand instead of rebuilding it from V (the soft-weights kernel is skipped).
+   * The values, and so every result, are the same bit for bit either way. */
+  float beta_next;
+  int wsoft_ready;
 } faar_hparams;
 
 /* Layer geometry.  Leading dimensions are in ELEMENTS.
@@ -293,7 +304,9 @@ FAAR_API int faar_layer_bwd(faar_ctx* ctx, const faar_shape* shape, const faar_h
 
 /* Forward, Round Loss and backward + update back to back: one pass of Procedure
  * steps 6-13.  loss_out2 (device) receives {L_MSE, L_round}, both at the
- * pre-update V.  dYt lives in the workspace. */
+ * pre-update V.  dYt lives in the workspace.  With hp->beta_next / hp->wsoft_ready
+ * (see faar_hparams) a loop of steps builds each step's soft weights inside the
+ * previous step's backward pass: two kernels per step instead of three. */
 FAAR_API int faar_layer_step(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp, const void* X,
                     const void* Xt, const void* Y_ref, float* V, const uint8_t* code,
                     const uint8_t* scales, const float* s_global, float* adam_m, float* adam_u,

@@ -43,6 +43,7 @@ int check_hp(const faar_hparams* hp, bool need_opt) {
   if (!(hp->beta > 0.f) || !isfinite(hp->beta) || !isfinite(hp->mse_scale) || !isfinite(hp->lambda_round))
     return FAAR_ERR_INVALID_ARG;
   if (!(hp->act_scale >= 0.f) || !isfinite(hp->act_scale)) return FAAR_ERR_INVALID_ARG;
+  if (!(hp->beta_next >= 0.f) || !isfinite(hp->beta_next)) return FAAR_ERR_INVALID_ARG;
   if (need_opt) {
     if (hp->opt != 0 && hp->opt != 1) return FAAR_ERR_INVALID_ARG;
     if (!isfinite(hp->lr)) return FAAR_ERR_INVALID_ARG;
@@ -63,8 +64,11 @@ int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
              const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
              void* Y_q, uint8_t* ws, const faar_ws_layout& l, int* n_partials) {
   __nv_bfloat16* wsoft = reinterpret_cast<__nv_bfloat16*>(ws + l.off_wsoft);
-  int e = faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, hp->beta, nullptr, nullptr, wsoft);
-  if (e) return e;
+  int e = 0;
+  if (!hp->wsoft_ready) {   // else: the previous backward pass left this step's operand in the workspace
+    e = faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, hp->beta, nullptr, nullptr, wsoft);
+    if (e) return e;
+  }
   faar_gemm_args a = {};
   a.mode = FAAR_GEMM_FWD;
   a.M = s->O; a.N = s->T; a.Kc = s->K;
@@ -103,6 +107,10 @@ int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
   a.V = V; a.code = code; a.scales = scales; a.s_global = s_global;
   a.adam_m = adam_m; a.adam_u = adam_u; a.dV = dV;
   a.beta = hp->beta;
+  if (hp->beta_next > 0.f) {
+    a.wsoft_next = reinterpret_cast<__nv_bfloat16*>(ws + l.off_wsoft);
+    a.beta_next = hp->beta_next;
+  }
   a.act_scale = hp->act_scale > 0.f ? hp->act_scale : 1.0f;
   a.lam_over_n = (float)((double)hp->lambda_round / ((double)s->O * (double)s->K));
   a.lr = hp->lr; a.b1 = hp->beta1; a.b2 = hp->beta2; a.eps = hp->eps; a.opt = hp->opt;

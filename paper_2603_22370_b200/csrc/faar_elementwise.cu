@@ -207,19 +207,11 @@ act_fakequant_kernel(const __nv_bfloat16* __restrict__ X, int T, int K, int64_t 
 // ---- Eq. 2 / Eq. 3 -----------------------------------------------------------------------------
 // FP32 outputs (W_soft, H): the parity view, relative error below 1e-6.
 // BF16 output: the operand of the forward GEMM.  It is rounded from a cheaper FP32 evaluation whose
-// relative error is below 3e-6 (z = beta*v - beta/2 and z*log2(e) each rounded once, hardware 2^x and
-// reciprocal), far inside the BF16 spacing of 2^-8; it can differ from the rounding of the exact
+// relative error is below 3e-6 for beta <= 32 (beta*log2(e) rounded once, the exponent formed in one
+// FMA, hardware 2^x and reciprocal), far inside the BF16 spacing of 2^-8; it can differ from the rounding of the exact
 // value only where that value lies within 3e-6 of a BF16 rounding boundary.
 // Per nibble (sign<<3 | k) the signed lower node and the signed interval width come from a
 // 16-entry table in shared memory: mag = lo + h*width needs one 8-byte load.
-__device__ __forceinline__ float sigmoid_fast(float beta, float neg_half_beta, float v) {
-  const float z = fmaf(beta, v, neg_half_beta);
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-fabsf(z) * 1.4426950408889634f));
-  const float hs = __fdividef(1.0f, 1.0f + e);
-  return z >= 0.f ? hs : e * hs;
-}
-
 __global__ void __launch_bounds__(EW_THREADS)
 softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code,
                       const uint8_t* __restrict__ scales, const float* __restrict__ s_global_p,
@@ -234,7 +226,8 @@ softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ c
   __syncthreads();
   faar_pdl_sync();                                   // V comes from the previous step's backward kernel
   const float s_global = *s_global_p;
-  const float nhb = -0.5f * beta;
+  float nbl, hbl;
+  faar_operand_consts(beta, &nbl, &hbl);
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups;
        g += (int64_t)gridDim.x * blockDim.x) {
     int64_t e = g * 8;
@@ -267,7 +260,7 @@ softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ c
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const float2 nw = lut[(cw >> (4 * i)) & 0xF];
-        wf[i] = fmaf(sigmoid_fast(beta, nhb, v[i]), nw.y, nw.x) * s;
+        wf[i] = faar_operand_weight(faar_sigmoid_operand(nbl, hbl, v[i]), nw.x, nw.y, s);
       }
       uint32_t o[4];
 #pragma unroll

@@ -233,6 +233,8 @@ struct KParams {
   float* V; const uint8_t* code; const uint8_t* scales; const float* s_global;
   float* adam_m; float* adam_u; float* dV;
   float beta, lam_over_n, lr, b1, b2, eps, inv_bc1, inv_bc2; int opt;
+  // BWD, optional: the next step's BF16 forward operand, from the updated v (null = not wanted)
+  __nv_bfloat16* wsoft_next; float beta_next;
   // BWD, optional: the CTA that finishes last also forms the step's two loss values
   uint32_t* fin_counter;            // workspace word, zero between launches
   const float* fin_mse_partials; int fin_n_mse; float fin_scale_mse;
@@ -422,6 +424,8 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
   const float step_size = p.lr * p.inv_bc1;
   const float rbc2 = sqrtf(p.inv_bc2);                            // sqrt(u / bc2) = sqrt(u) sqrt(1 / bc2)
   const float lam4 = -4.f * p.lam_over_n;                         // (lambda / N) (4 - 8 v) = lam4 (2 v - 1)
+  float nbl_next, hbl_next;                                       // OPT & 2: constants of the next step's Eq. 3
+  faar_operand_consts(p.beta_next, &nbl_next, &hbl_next);
   const uint64_t stream = l2_policy_stream();
   float tt = 0.f, n_el = 0.f;                                     // sum of (2 v - 1)^2, elements seen
 #pragma unroll
@@ -438,7 +442,7 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
         v[q] = ldg128_stream(Vp + off, stream);
         cw[q] = *reinterpret_cast<const uint16_t*>(Cp + (off >> 1));
         sb[q] = Sp[off >> 4];
-        if (OPT == 1) {
+        if (OPT & 1) {
           m[q] = ldg128_stream(Mp + off, stream);
           u[q] = ldg128_stream(Up + off, stream);
         }
@@ -454,12 +458,21 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
         const float G[4] = {g4.x, g4.y, g4.z, g4.w};
         const float vv[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
         // s beta / 2 (the narrowest interval is 0.5 wide); act_scale: G = act_scale * acc
-        const float sbh = __fmul_rn(faar_e4m3_to_float(sb[q]), s_global) * (0.5f * p.beta * p.act_scale);
+        const float sc = __fmul_rn(faar_e4m3_to_float(sb[q]), s_global);
+        const float sbh = sc * (0.5f * p.beta * p.act_scale);
         // byte j: log2 of (interval width / 0.5) of element j, looked up by its interval index k (0 0 0 0 1 1 2)
-        const uint32_t wlog = __byte_perm(0u, 0x00020101u, cw[q] & 0x7777u);
+        const uint32_t ksel = cw[q] & 0x7777u;
+        const uint32_t wlog = __byte_perm(0u, 0x00020101u, ksel);
+        // OPT & 2: bytes 3 and 2 of the lower node's float (0 .5 1 1.5 2 3 4) by the same look-up
+        uint32_t lo_hi = 0u, lo_lo = 0u;
+        if (OPT & 2) {
+          lo_hi = __byte_perm(0x3F3F3F00u, 0x00404040u, ksel);
+          lo_lo = __byte_perm(0xC0800000u, 0x00804000u, ksel);
+        }
+        float wn[4];
         float g[4], vn[4], mn[4], un[4];
         float mm[4], uu[4];
-        if (OPT == 1) {
+        if (OPT & 1) {
           mm[0] = m[q].x; mm[1] = m[q].y; mm[2] = m[q].z; mm[3] = m[q].w;
           uu[0] = u[q].x; uu[1] = u[q].y; uu[2] = u[q].z; uu[3] = u[q].w;
         }
@@ -471,12 +484,13 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
           // dh times the width factor by an add to its exponent field (a dh flushed to 0 becomes ~1e-38), then
           // the sign of w from bit 3 of the nibble
           const uint32_t wexp = (j < 3 ? wlog << (23 - 8 * j) : wlog >> 1) & 0x01800000u;
+          const uint32_t sgn = (cw[q] << (28 - 4 * j)) & 0x80000000u;
           float chain = sbh * __uint_as_float(__float_as_uint(dh) + wexp);
-          chain = __uint_as_float(__float_as_uint(chain) ^ ((cw[q] << (28 - 4 * j)) & 0x80000000u));
+          chain = __uint_as_float(__float_as_uint(chain) ^ sgn);
           const float t = fmaf(2.f, vv[j], -1.f);
           g[j] = fmaf(G[j], chain, lam4 * t);
           tt = fmaf(t, t, tt);
-          if (OPT == 1) {
+          if (OPT & 1) {
             mn[j] = fmaf(p.b1, mm[j], c1 * g[j]);
             un[j] = fmaf(p.b2, uu[j], c2 * g[j] * g[j]);
             const float den = fmaf(sqrt_approx(un[j]), rbc2, p.eps);
@@ -484,9 +498,19 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
           } else {
             vn[j] = __saturatef(fmaf(-p.lr, g[j], vv[j]));
           }
+          if (OPT & 2) {
+            // Eq. 2 / Eq. 3 at the updated v with the next step's beta: (lo + h width) s with the sign of w, in
+            // the soft-weights kernel's operations, so that the BF16 operand is the same bit for bit
+            const float lo = __uint_as_float(__byte_perm(lo_hi, lo_lo, (uint32_t)((j << 12) | ((4 + j) << 8))) & 0xFFFF0000u);
+            const float wd = __uint_as_float(0x3F000000u + wexp);
+            const float mag = faar_operand_weight(faar_sigmoid_operand(nbl_next, hbl_next, vn[j]), lo, wd, sc);
+            wn[j] = __uint_as_float(__float_as_uint(mag) ^ sgn);
+          }
         }
+        if (OPT & 2)
+          *reinterpret_cast<uint2*>(p.wsoft_next + e0 + off) = make_uint2(pack_bf16x2(wn[0], wn[1]), pack_bf16x2(wn[2], wn[3]));
         if (p.dV) stg128_stream(p.dV + e0 + off, g[0], g[1], g[2], g[3], stream);
-        if (OPT == 1) {
+        if (OPT & 1) {
           stg128_stream(Mp + off, mn[0], mn[1], mn[2], mn[3], stream);
           stg128_stream(Up + off, un[0], un[1], un[2], un[3], stream);
         }
@@ -946,6 +970,7 @@ int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out
   kp.adam_m = a->adam_m; kp.adam_u = a->adam_u; kp.dV = a->dV;
   kp.beta = a->beta; kp.lam_over_n = a->lam_over_n; kp.lr = a->lr; kp.b1 = a->b1; kp.b2 = a->b2; kp.eps = a->eps;
   kp.inv_bc1 = a->inv_bc1; kp.inv_bc2 = a->inv_bc2; kp.opt = a->opt;
+  kp.wsoft_next = a->wsoft_next; kp.beta_next = a->beta_next;
   kp.fin_counter = a->fin_counter; kp.fin_mse_partials = a->fin_mse_partials; kp.fin_n_mse = a->fin_n_mse;
   kp.fin_scale_mse = a->fin_scale_mse; kp.fin_scale_round = a->fin_scale_round; kp.fin_out2 = a->fin_out2;
   // the BWD epilogue forms row offsets of up to 7 rows in 32-bit element counts
@@ -955,6 +980,10 @@ int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out
     case FAAR_GEMM_REF: return launch<FAAR_GEMM_REF>(ctx, a, kp, n_partials_out);
     case FAAR_GEMM_FWD: return launch<FAAR_GEMM_FWD>(ctx, a, kp, n_partials_out);
     case FAAR_GEMM_BWD:
+      // OPT bit 0: Adam; bit 1: also write the next step's forward operand
+      if (a->wsoft_next)
+        return a->opt == 1 ? launch<FAAR_GEMM_BWD, 3>(ctx, a, kp, n_partials_out)
+                           : launch<FAAR_GEMM_BWD, 2>(ctx, a, kp, n_partials_out);
       return a->opt == 1 ? launch<FAAR_GEMM_BWD, 1>(ctx, a, kp, n_partials_out)
                          : launch<FAAR_GEMM_BWD, 0>(ctx, a, kp, n_partials_out);
   }

@@ -112,6 +112,8 @@ struct faar_gemm_args {
   float* V; const uint8_t* code; const uint8_t* scales; const float* s_global;
   float* adam_m; float* adam_u; float* dV;
   float beta, lam_over_n, lr, b1, b2, eps, inv_bc1, inv_bc2; int opt;
+  // BWD, optional: also write the next step's BF16 operand W_soft(V', beta_next) (null = not wanted)
+  __nv_bfloat16* wsoft_next; float beta_next;
   // BWD, optional: final loss sums by the last CTA (fin_out2 null = not wanted)
   uint32_t* fin_counter; const float* fin_mse_partials; int fin_n_mse; float fin_scale_mse, fin_scale_round;
   float* fin_out2;
@@ -180,6 +182,27 @@ __device__ __forceinline__ float faar_sigmoid_precise(float beta, float v) {
   e = __fmaf_rn(e, tl * 0.6931471805599453f, e);          // 2^(th+tl) = 2^th (1 + tl ln 2)
   const float hs = __fdividef(1.0f, 1.0f + e);            // sigmoid(|z|)
   return zh >= 0.f ? hs : __fmul_rn(e, hs);               // sigmoid(-|z|) = e / (1 + e)
+}
+
+// Eq. 3 as the forward GEMM's BF16 operand is built (relative error below 3e-6):
+// h = 1 / (1 + 2^(-z log2 e)), z = beta (v - 0.5), with beta log2(e) rounded once, the exponent formed
+// in one FMA, hardware 2^x and reciprocal.  A 2^x that overflows (z < -88) gives h = 0, the value's
+// rounding.  nbl = -(beta * log2 e), hbl = -nbl / 2 (faar_operand_consts).
+__device__ __forceinline__ void faar_operand_consts(float beta, float* nbl, float* hbl) {
+  *nbl = -__fmul_rn(beta, 1.4426950408889634f);
+  *hbl = -0.5f * *nbl;
+}
+__device__ __forceinline__ float faar_sigmoid_operand(float nbl, float hbl, float v) {
+  float e, h;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(nbl, v, hbl)));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(h) : "f"(1.0f + e));
+  return h;
+}
+// The operand value before its rounding to BF16: (lo + h * width) * s with the sign of w, in exactly
+// these operations wherever it is produced (soft-weights kernel, dW epilogue), so that both give the
+// same bits.  lo and width may carry the sign already (rounding is symmetric).
+__device__ __forceinline__ float faar_operand_weight(float h, float lo, float width, float s) {
+  return fmaf(h, width, lo) * s;
 }
 
 // Eq. 2 in FP32: sign * (lo + h * (hi - lo)) * s for the nibble (sign<<3 | k).

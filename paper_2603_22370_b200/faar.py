@@ -28,7 +28,7 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
 class HParams(C.Structure):
     _fields_ = [("beta", C.c_float), ("lambda_round", C.c_float), ("mse_scale", C.c_float), ("opt", C.c_int),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("step", C.c_int), ("act_scale", C.c_float)]
+                ("step", C.c_int), ("act_scale", C.c_float), ("beta_next", C.c_float), ("wsoft_ready", C.c_int)]
 
 
 class Shape(C.Structure):
@@ -89,8 +89,8 @@ def make_shape(O, K, T, ldw=None, ldx=None, ldxt=None, ldy=None, w_dtype=BF16, y
 
 
 def make_hparams(beta=4.0, lambda_round=1.0, mse_scale=1.0, opt=1, lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8,
-                 step=1, act_scale=0.0) -> HParams:
-    return HParams(beta, lambda_round, mse_scale, opt, lr, beta1, beta2, eps, step, act_scale)
+                 step=1, act_scale=0.0, beta_next=0.0, wsoft_ready=0) -> HParams:
+    return HParams(beta, lambda_round, mse_scale, opt, lr, beta1, beta2, eps, step, act_scale, beta_next, wsoft_ready)
 
 
 class Context:

@@ -57,8 +57,11 @@ def optimise_layer(ctx: faar.Context, W: torch.Tensor, X: torch.Tensor, steps: i
 
     history = []
     for t in range(steps):
+        # the backward pass of step t builds step t+1's soft weights (same values, one kernel fewer per step)
         hp = faar.make_hparams(beta=beta_schedule(t, steps, beta0, beta1), lambda_round=lambda_round,
-                               mse_scale=mse_scale, opt=opt, lr=lr, step=t + 1, act_scale=act_scale)
+                               mse_scale=mse_scale, opt=opt, lr=lr, step=t + 1, act_scale=act_scale,
+                               wsoft_ready=int(t > 0),
+                               beta_next=beta_schedule(t + 1, steps, beta0, beta1) if t + 1 < steps else 0.0)
         faar.layer_step(ctx, shape, hp, Xg, Xt, Yref, V, code, scales, s_global, m, u, loss, ws)
         if loss_every and (t + 1) % loss_every == 0:
             history.append((t + 1, *loss.tolist()))

@@ -678,3 +678,50 @@ def test_transposed_target_layout_gives_the_same_results(ctx, O, K, T, yref_dtyp
     with pytest.raises(faar.FaarError) as e:
         faar.layer_ref(ctx, bad, lay.X, lay.W, torch.zeros(O * (T + 16), dtype=torch.bfloat16, device=DEV), lay.ws)
     assert e.value.status in (faar.ERR_SHAPE, faar.ERR_ALIGN)
+
+
+@pytest.mark.parametrize("opt", [1, 0])
+@pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (512, 256, 512)])
+def test_chained_steps_equal_standalone_steps(ctx, opt, O, K, T):
+    """With beta_next / wsoft_ready the backward pass writes the next step's BF16 operand and the forward
+    pass reads it.  Eq. 2 / Eq. 3 are evaluated in the same operations in both places, so a loop run that
+    way must reproduce, bit for bit, the loop in which every step rebuilds its operand from V (ragged and
+    tile-aligned shapes; separate forward / backward calls and the fused step call)."""
+    W, X, Yref = _problem(O, K, T, seed=7)
+    betas = [float(np.float32(fo.beta_schedule(t, 6))) for t in range(6)]
+    runs = []
+    for mode in ("alone", "chained step", "chained fwd+bwd"):
+        lay = GpuLayer(ctx, W, X)
+        lay.init()
+        lay.set_yref(Yref)
+        losses = []
+        for t, b in enumerate(betas):
+            kw = dict(beta=b, step=t + 1, opt=opt, lr=1e-2 if opt == 1 else 1e-4)
+            if mode != "alone":
+                kw.update(wsoft_ready=int(t > 0), beta_next=betas[t + 1] if t + 1 < len(betas) else 0.0)
+            hp = faar.make_hparams(**kw)
+            if mode == "chained fwd+bwd":
+                lay.fwd(hp)
+                lay.bwd(hp, want_dv=(t % 2 == 0))
+                losses.append(host(lay.loss)[0:1].copy())
+            else:
+                lay.step(hp)
+                losses.append(host(lay.loss).copy())
+        lay.check()
+        runs.append((host(lay.V).copy(), host(lay.m).copy(), host(lay.u).copy(), np.array(losses)))
+    for a, b in zip(runs[0], runs[1]):
+        assert np.array_equal(a, b)
+    for a, b in zip(runs[0][:3], runs[2][:3]):
+        assert np.array_equal(a, b)
+    assert np.array_equal(runs[0][3][:, 0], runs[2][3][:, 0])
+
+
+def test_chaining_arguments_are_checked(ctx):
+    W, X, Yref = _problem(64, 64, 64)
+    lay = GpuLayer(ctx, W, X)
+    lay.init()
+    lay.set_yref(Yref)
+    for bad in (float("nan"), -1.0, float("inf")):
+        with pytest.raises(faar.FaarError):
+            lay.step(faar.make_hparams(beta_next=bad))
+    lay.check()
