@@ -98,3 +98,13 @@ def test_layer_step_on_quantised_activations(ctx, O, K, T):
     lay.check()
     assert abs(host(lay.loss)[0] - l_mse) <= 2e-3 * l_mse
     assert rel_l2(host(lay.V), Vo) <= 2e-3
+    # two more steps, alone and chained (the backward pass writes the next operand): the same bits
+    ends = []
+    for chained in (False, True):
+        lay.set_state(V=V0, m=zeros, u=zeros)
+        for t in range(3):
+            extra = dict(wsoft_ready=int(t > 0), beta_next=5.0 + t + 1 if t < 2 else 0.0) if chained else {}
+            lay.step(faar.make_hparams(act_scale=float(sg), **{**kw, "beta": 5.0 + t, "step": t + 1}, **extra))
+        lay.check()
+        ends.append((host(lay.V).copy(), host(lay.loss).copy()))
+    assert np.array_equal(ends[0][0], ends[1][0]) and np.array_equal(ends[0][1], ends[1][1])

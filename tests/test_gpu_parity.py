@@ -539,7 +539,7 @@ def test_layer_step_host_matches_device_steps(ctx, two_sets):
     batches = [inputs.config2(20 + i, 8, K, T)[1] for i in range(5)]
     yrefs = [inputs.to_bf16_f32(fo.layer_ref(Xb, W)) for Xb in batches]
     out = []
-    for mode in ("device", "host"):
+    for mode in ("device", "host", "host chained"):
         lay = GpuLayer(ctx, W, batches[0])
         lay.init()
         losses = []
@@ -549,7 +549,8 @@ def test_layer_step_host_matches_device_steps(ctx, two_sets):
                   for Xb, Yb in zip(batches, yrefs)]
         loss_h = torch.zeros(2).pin_memory()
         for t, (Xb, Yb) in enumerate(zip(batches, yrefs)):
-            hp = faar.make_hparams(beta=4.0 + t, step=t + 1)
+            chain = dict(wsoft_ready=int(t > 0), beta_next=4.0 + t + 1 if t + 1 < len(batches) else 0.0)
+            hp = faar.make_hparams(beta=4.0 + t, step=t + 1, **(chain if mode == "host chained" else {}))
             if mode == "device":
                 lay.X.copy_(dev_bf16(Xb))
                 faar.transpose_bf16(ctx, T, K, lay.X, K, lay.Xt, lay.ldt)
@@ -566,8 +567,9 @@ def test_layer_step_host_matches_device_steps(ctx, two_sets):
                     losses.append(loss_h.numpy().copy())
         lay.check()
         out.append((host(lay.V).copy(), host(lay.m).copy(), losses[-1]))
-    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
-    assert np.array_equal(out[0][2], out[1][2])
+    for other in out[1:]:
+        assert np.array_equal(out[0][0], other[0]) and np.array_equal(out[0][1], other[1])
+        assert np.array_equal(out[0][2], other[2])
 
 
 @pytest.mark.parametrize("split", [1, 3, 100])
