@@ -20,14 +20,21 @@ def beta_schedule(t: int, steps: int, beta0: float = 4.0, beta1: float = 32.0) -
 
 def optimise_layer(ctx: faar.Context, W: torch.Tensor, X: torch.Tensor, steps: int = 200, lr: float = 1e-2,
                    lambda_round: float = 1.0, mse_scale: float = 1.0, opt: int = 1, beta0: float = 4.0,
-                   beta1: float = 32.0, quantise_activations: bool = False, loss_every: int = 0) -> dict:
+                   beta1: float = 32.0, quantise_activations: bool = False, loss_every: int = 0,
+                   rows: tuple[int, int] | None = None, s_global_in: float = 0.0) -> dict:
     """Runs the whole path for one linear layer: soft-quantisation set-up, the frozen target, `steps`
     optimisation steps, hardening and packing.  W [O,K] and X [T,K] are BF16 CUDA tensors (row-major).
     With quantise_activations the GEMMs consume NVFP4-quantised activations (the target still comes from
     the unquantised X).  Returns the packed weights, their scales, the final V and the losses read back
-    every `loss_every` steps (0 = only at the end)."""
+    every `loss_every` steps (0 = only at the end).
+    rows = (b, e) restricts the problem to output rows [b, e) of W (a row shard: Eq. 5 separates over
+    output features); the Round Loss weight lambda / N keeps the whole layer's N, and s_global_in must
+    then be the whole tensor's scale (optimise_layer_row_sharded finds it)."""
     assert W.is_cuda and X.is_cuda and W.dtype == torch.bfloat16 and X.dtype == torch.bfloat16
     dev = W.device
+    if rows is not None:
+        lambda_round = lambda_round * (rows[1] - rows[0]) / W.shape[0]
+        W = W[rows[0]:rows[1]].contiguous()
     O, K = W.shape
     T = X.shape[0]
     ldt = (T + 7) // 8 * 8
@@ -43,7 +50,7 @@ def optimise_layer(ctx: faar.Context, W: torch.Tensor, X: torch.Tensor, steps: i
     Yref = torch.zeros((O, shape.ldy), dtype=torch.bfloat16, device=dev)
     loss = torch.zeros(2, dtype=torch.float32, device=dev)
 
-    faar.softquant_init(ctx, shape, W, 0.0, scales, s_global, code, V, ws)
+    faar.softquant_init(ctx, shape, W, s_global_in, scales, s_global, code, V, ws)
     faar.layer_ref(ctx, shape, X, W, Yref, ws)
     act_scale = 0.0
     Xg = X
@@ -82,3 +89,31 @@ def optimise_block(ctx: faar.Context, linears: list, steps: int, rank: int = 0, 
         name, W, X = linears[i]
         out[name] = optimise_layer(ctx, W, X, steps=steps, **kw)
     return out
+
+
+def optimise_layer_row_sharded(ctx: faar.Context, W: torch.Tensor, X: torch.Tensor, rank: int, world: int,
+                               **kw) -> dict:
+    """One layer split by output rows over `world` processes (X replicated, W whole or at least this
+    rank's rows valid).  Set-up: each rank derives the tensor scale of its rows, the ranks take the largest
+    (one scalar MAX all-reduce); then every step is local.  Returns this rank's rows of the result, the row
+    range, and the whole layer's final losses."""
+    b, e = shard.rows_for_rank(W.shape[0], rank, world)
+    O, K = e - b, W.shape[1]
+    dev = W.device
+    if O == 0:                     # more ranks than rows: this rank only takes part in the two collectives
+        shard.global_tensor_scale(torch.zeros(1, dtype=torch.float32, device=dev))
+        return {"rows": (b, e), "layer_losses": shard.combine_losses(torch.zeros(2, device=dev), 0, W.shape[0]).tolist()}
+    Wl = W[b:e].contiguous()
+    shape = faar.make_shape(O, K, 8)
+    ws = torch.empty(faar.workspace_size(shape), dtype=torch.uint8, device=dev)
+    faar.workspace_init(ctx, ws)
+    s_local = torch.empty(1, dtype=torch.float32, device=dev)
+    faar.softquant_init(ctx, shape, Wl, 0.0, torch.empty((O, K // 16), dtype=torch.uint8, device=dev), s_local,
+                        torch.empty((O, K // 2), dtype=torch.uint8, device=dev),
+                        torch.empty((O, K), dtype=torch.float32, device=dev), ws)
+    s_all = float(shard.global_tensor_scale(s_local).item())
+    res = optimise_layer(ctx, W, X, rows=(b, e), s_global_in=s_all, **kw)
+    res["rows"] = (b, e)
+    last = torch.tensor(res["history"][-1][1:], dtype=torch.float32, device=dev)
+    res["layer_losses"] = shard.combine_losses(last, e - b, W.shape[0]).tolist()
+    return res

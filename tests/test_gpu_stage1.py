@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from oracle import faar_oracle as fo
-from paper_2603_22370_b200 import faar, inputs, stage1
+from paper_2603_22370_b200 import faar, inputs, shard, stage1
 from tests.gpu_helpers import dev_bf16, host
 
 pytestmark = pytest.mark.gpu
@@ -59,3 +59,39 @@ def test_optimise_block_covers_every_linear(ctx):
     assert out["q_proj"]["packed"].shape == (64, 64)
     part = stage1.optimise_block(ctx, lin, steps=2, rank=1, world=2)
     assert sorted(part) == ["k_proj"]
+
+
+@pytest.mark.parametrize("O,world", [(128, 2), (96, 3)])
+def test_row_shards_reproduce_the_whole_layer(ctx, O, world):
+    """Eq. 5 separates over output features: the ranks of a row-sharded layer, given the whole tensor's
+    scale, must arrive at the rows the unsharded run produces.  The ranks are run one after the other on
+    this GPU.  Two equal shards: bit for bit (lambda / N is formed from lambda / 2 exactly); three: the
+    Round Loss weight is rounded once more, so V may move in its last bits."""
+    K, T = 256, 512
+    W, X = inputs.config2(4, O, K, T)
+    Wd, Xd = dev_bf16(W), dev_bf16(X)
+    kw = dict(steps=12, lr=1e-2, loss_every=0)
+    whole = stage1.optimise_layer(ctx, Wd, Xd, **kw)
+    sg = float(host(whole["s_global"])[0])
+    mse_sum, round_sum = 0.0, 0.0
+    for r in range(world):
+        b, e = shard.rows_for_rank(O, r, world)
+        part = stage1.optimise_layer(ctx, Wd, Xd, rows=(b, e), s_global_in=sg, **kw)
+        assert np.array_equal(host(part["scales"]), host(whole["scales"])[b:e])
+        assert np.array_equal(host(part["code"]), host(whole["code"])[b:e])
+        Vp, Vw = host(part["V"]), host(whole["V"])[b:e]
+        if world == 2:
+            assert np.array_equal(Vp, Vw)
+            assert np.array_equal(host(part["packed"]), host(whole["packed"])[b:e])
+        else:
+            assert np.max(np.abs(Vp - Vw)) <= 1e-5
+            flips = (Vp >= 0.5) != (Vw >= 0.5)
+            assert np.all(np.abs(Vw[flips] - 0.5) < 1e-4)
+        mse_sum += part["history"][-1][1]
+        round_sum += part["history"][-1][2] * (e - b) / O
+    assert abs(mse_sum - whole["history"][-1][1]) <= 1e-4 * whole["history"][-1][1]
+    assert abs(round_sum - whole["history"][-1][2]) <= 1e-5
+    # the one-process form of the sharded driver is the whole layer
+    one = stage1.optimise_layer_row_sharded(ctx, Wd, Xd, 0, 1, **kw)
+    assert one["rows"] == (0, O) and np.array_equal(host(one["V"]), host(whole["V"]))
+    assert abs(one["layer_losses"][0] - whole["history"][-1][1]) <= 1e-6 * whole["history"][-1][1]
