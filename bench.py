@@ -324,11 +324,27 @@ def run_ours(args):
 
     ew_us = elementwise_rates()
 
+    # ---- the layer's input gradient dX = dY W_soft (soft weights + transpose + GEMM in one call), alone
+    def layer_dx_us(rounds=20):
+        dY = torch.randn((T, O), dtype=torch.float32, device=device).to(torch.bfloat16)
+        WsT = torch.empty((K, (O + 7) // 8 * 8), dtype=torch.bfloat16, device=device)
+        dX = torch.empty((T, K), dtype=torch.bfloat16, device=device)
+        plain = faar.make_shape(O, K, T)                       # dY is [T, O] here
+        fn = lambda: faar.layer_dx(ctx, plain, 8.0, dY, V, code, scales, s_global, WsT, dX, ws)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                fn()
+        stream.synchronize()
+        return 1e3 * timed(lambda: [fn() for _ in range(rounds)]) / rounds
+
+    dx_us = layer_dx_us()
+
     if args.quick:
         if rank == 0:
             print(json.dumps({"quick": True, "steps": steps, "ms_per_step": ms_job / steps,
                               "kernels_avg_us": {k: round(1e3 * v[1] / v[0], 2) for k, v in prof.items()},
-                              "elementwise_alone_us": {k: round(v, 2) for k, v in ew_us.items()}}))
+                              "elementwise_alone_us": {k: round(v, 2) for k, v in ew_us.items()},
+                              "layer_dx_us": round(dx_us, 2)}))
         if sampler:
             sampler.stop()
         if world > 1:
@@ -394,6 +410,11 @@ def run_ours(args):
             how = "30 back-to-back launches over 3 rotated buffer sets, one event pair"
         kernels[name] = {"avg_us": round(us, 2), "bound": bound, "achieved": round(ach, 1), "peak": peak, "unit": unit,
                          "frac": round(ach / peak, 4), "timed": how}
+    kernels["layer_dx"] = {"avg_us": round(dx_us, 2), "bound": "tensor", "achieved": round(flops / (dx_us * 1e-6) / 1e12, 1),
+                           "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                           "frac": round(flops / (dx_us * 1e-6) / 1e12 / pk["bf16_tflops_sustained"], 4),
+                           "timed": "20 back-to-back calls (soft weights, transpose and GEMM each), one event pair",
+                           "note": "input gradient dX = dY W_soft, not part of a Stage-1 step"}
     kernels["softquant_init"]["note"] = "amax pass + bracket pass together; the amax pass re-reads W (+2 B/weight, not " \
                                         "counted); the bracket pass is bound by its IEEE divisions, not by HBM"
     for name in prof:
