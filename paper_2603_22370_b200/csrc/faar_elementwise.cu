@@ -413,6 +413,43 @@ transpose_bf16_kernel(const uint16_t* __restrict__ in, int rows, int cols, int64
   }
 }
 
+// The same transpose with 16-byte global accesses, for the aligned case (cols, ld_in, ld_out multiples
+// of 8, 16-byte aligned bases, ld_out >= rows rounded up to 8).  A thread reads 8 columns of two
+// consecutive rows, pairs the values column by column (element r in the low half, r + 1 in the high half)
+// and stores the eight 32-bit pairs into tile[column][row pair]; a row of the tile is then a run of the
+// output row and leaves as 16-byte vectors.  Rows beyond the matrix enter as zeros and may be written
+// into the padding of the output rows.
+__global__ void __launch_bounds__(256)
+transpose_bf16_vec_kernel(const uint16_t* __restrict__ in, int rows, int cols, int64_t ld_in,
+                          uint16_t* __restrict__ out, int64_t ld_out) {
+  __shared__ __align__(16) uint32_t tile[64][36];
+  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+  {
+    const int rp = threadIdx.x & 31, cc = threadIdx.x >> 5;          // row pair, 8-column chunk
+    const int r = r0 + 2 * rp, c = c0 + 8 * cc;
+    uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+    if (c < cols) {
+      if (r < rows) a = *reinterpret_cast<const uint4*>(in + (int64_t)r * ld_in + c);
+      if (r + 1 < rows) b = *reinterpret_cast<const uint4*>(in + (int64_t)(r + 1) * ld_in + c);
+    }
+    const uint32_t x[4] = {a.x, a.y, a.z, a.w}, y[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      tile[8 * cc + 2 * j][rp] = __byte_perm(x[j], y[j], 0x5410);     // column 2j: low halves
+      tile[8 * cc + 2 * j + 1][rp] = __byte_perm(x[j], y[j], 0x7632); // column 2j + 1: high halves
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int idx = threadIdx.x + 256 * i;
+    const int cl = idx >> 3, q = idx & 7;                             // output row of the tile, 8-element chunk
+    const int c = c0 + cl, r = r0 + 8 * q;
+    if (c < cols && r < rows)
+      *reinterpret_cast<uint4*>(out + (int64_t)c * ld_out + r) = *reinterpret_cast<const uint4*>(&tile[cl][4 * q]);
+  }
+}
+
 int grid_for(const faar_ctx* ctx, int64_t work_items, int per_sm) {
   int64_t blocks = (work_items + EW_THREADS - 1) / EW_THREADS;
   int64_t cap = (int64_t)ctx->num_sms * per_sm;
@@ -481,6 +518,13 @@ int faar_launch_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in
                                int64_t ld_out) {
   dim3 grid((cols + 63) / 64, (rows + 63) / 64);
   faar_prof_scope ps(ctx, FAAR_K_TRANSPOSE);
+  const bool vec = cols % 8 == 0 && ld_in % 8 == 0 && ld_out % 8 == 0 && ld_out >= (int64_t)(rows + 7) / 8 * 8 &&
+                   ((uintptr_t)in & 15) == 0 && ((uintptr_t)out & 15) == 0;
+  if (vec) {
+    transpose_bf16_vec_kernel<<<grid, 256, 0, ctx->stream>>>(reinterpret_cast<const uint16_t*>(in), rows, cols, ld_in,
+                                                             reinterpret_cast<uint16_t*>(out), ld_out);
+    return (int)cudaGetLastError();
+  }
   transpose_bf16_kernel<<<grid, 256, 0, ctx->stream>>>(reinterpret_cast<const uint16_t*>(in), rows, cols, ld_in,
                                                        reinterpret_cast<uint16_t*>(out), ld_out);
   return (int)cudaGetLastError();

@@ -215,15 +215,21 @@ def test_harden_pack_bit_exact(ctx):
                               host(Wf).view(np.uint32))
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 1), (77, 130), (600, 1040)])
-def test_transpose(ctx, rows, cols):
+@pytest.mark.parametrize("rows,cols,ld_in", [(1, 1, 1), (77, 130, 130), (600, 1040, 1040), (77, 136, 144), (1, 8, 8),
+                                              (513, 64, 64), (64, 520, 520), (130, 72, 75)])
+def test_transpose(ctx, rows, cols, ld_in):
+    """Aligned shapes (columns and strides multiples of 8) take the 16-byte path, the others the element
+    path; ragged row counts, odd ones included, on both."""
     rng = np.random.default_rng(0)
-    a = dev_bf16(rng.standard_normal((rows, cols)))
-    ld = (rows + 7) // 8 * 8
-    out = torch.zeros((cols, ld), dtype=torch.bfloat16, device=DEV)
-    faar.transpose_bf16(ctx, rows, cols, a, cols, out, ld)
+    a = torch.full((rows, ld_in), 9.0, dtype=torch.bfloat16, device=DEV)
+    a[:, :cols] = dev_bf16(rng.standard_normal((rows, cols)))
+    ld = (rows + 7) // 8 * 8 + 8
+    out = torch.full((cols + 1, ld), 5.0, dtype=torch.bfloat16, device=DEV)
+    faar.transpose_bf16(ctx, rows, cols, a, ld_in, out, ld)
     torch.cuda.synchronize()
-    assert torch.equal(out[:, :rows], a.t())
+    assert torch.equal(out[:cols, :rows], a[:, :cols].t())
+    assert torch.all(out[cols] == 5.0)                              # the row after the last is untouched
+    assert torch.all(out[:cols, (rows + 7) // 8 * 8:] == 5.0)       # at most the padding up to 8 is written
 
 
 # ---------------------------------------------------------------------------------------------
