@@ -23,11 +23,15 @@ Parity pins (tests/test_oracle_pins.py): node table, E4M3 format, bracket
 invariants, beta-limits of Eq. 3, RTN == harden(V_init), pack/dequant
 round trip, finite differences of Eq. 5, Round Loss closed forms, Adam
 first-step closed form, exhaustive row-separable search on a 4x16 layer,
-textbook GEMM special case, zero-residual fixed point.
+textbook GEMM special case, zero-residual fixed point; for the alignment loss
+(Eq. 6): identical models, shift and temperature invariances, the two-class
+closed form, the uniform-model closed form, finite differences of both
+gradients.
 
 Parity unpinned (free parameters the paper names but gives no value for; both
 sides simply receive them as arguments): the beta schedule, lambda_round, the
-optimiser and its hyper-parameters, the calibration batch.
+optimiser and its hyper-parameters, the calibration batch, tau and lambda_KL
+of Eq. 6 and its reduction over tokens (a mean here).
 """
 from __future__ import annotations
 
@@ -430,3 +434,32 @@ def rtn_nearest(W, scales, s_global):
     best = dist.min(axis=2, keepdims=True)
     cand = np.where(dist == best, np.arange(8)[None, None, :], -1)
     return cand.max(axis=2)
+
+
+# --------------------------------------------------------------------------
+# Full-model alignment loss (Eq. 6, Procedure steps 18-20)
+# --------------------------------------------------------------------------
+
+def align_loss(Z_fp, Z_q, H_fp, H_q, tau=1.0, lambda_kl=1.0):
+    """The two data terms of Eq. 6 and their gradients towards the quantised model's outputs.
+
+    P_fp = softmax(Z_fp / tau), P_q = softmax(Z_q / tau) over the vocabulary (Procedure step 18);
+    L_KL = KL(P_fp || P_q) (step 19), summed over the vocabulary and averaged over the T tokens (the
+    paper gives no reduction over tokens; a mean keeps lambda_KL independent of the batch size);
+    L_MSE = ||H_fp - H_q||_F^2 (step 20), a sum.
+    Returns (L_KL, L_MSE, dZ_q, dH_q) with dZ_q = d(lambda_kl L_KL)/dZ_q = lambda_kl (P_q - P_fp) / (tau T)
+    and dH_q = dL_MSE/dH_q = 2 (H_q - H_fp).  float64 throughout; log-softmax by the max-shifted form."""
+    Zf = np.asarray(Z_fp, dtype=np.float64) / tau
+    Zq = np.asarray(Z_q, dtype=np.float64) / tau
+    T = Zf.shape[0]
+
+    def log_softmax(Z):
+        Zs = Z - Z.max(axis=1, keepdims=True)
+        return Zs - np.log(np.exp(Zs).sum(axis=1, keepdims=True))
+
+    lf, lq = log_softmax(Zf), log_softmax(Zq)
+    pf, pq = np.exp(lf), np.exp(lq)
+    l_kl = float((pf * (lf - lq)).sum() / T)
+    dZ = lambda_kl * (pq - pf) / (tau * T)
+    D = np.asarray(H_q, dtype=np.float64) - np.asarray(H_fp, dtype=np.float64)
+    return l_kl, float((D * D).sum()), dZ, 2.0 * D

@@ -446,3 +446,62 @@ def test_layer_dx_matches_finite_differences_of_the_mse_term():
     # transposed operand or a missing factor would show here: dX has X's shape and scales with dY
     assert dX.shape == X.shape
     assert np.allclose(fo.layer_dx(2 * dY, V, code, scales, sg, beta, "smooth"), 2 * dX)
+
+
+# ---- full-model alignment loss (Eq. 6, Procedure steps 18-20) ---------------------------------
+
+def test_align_loss_closed_forms():
+    rng = np.random.default_rng(0)
+    T, V, D = 5, 37, 8
+    Zf, Zq = rng.standard_normal((T, V)) * 3, rng.standard_normal((T, V)) * 3
+    Hf, Hq = rng.standard_normal((T, D)), rng.standard_normal((T, D))
+    # identical models: no divergence, no gradient
+    kl, mse, dZ, dH = fo.align_loss(Zf, Zf, Hf, Hf)
+    assert kl == 0.0 and mse == 0.0 and not dZ.any() and not dH.any()
+    # Gibbs: KL > 0 for different distributions; each token's gradient sums to zero over the vocabulary
+    kl, mse, dZ, dH = fo.align_loss(Zf, Zq, Hf, Hq, tau=1.7, lambda_kl=0.3)
+    assert kl > 0 and np.all(np.abs(dZ.sum(axis=1)) < 1e-15)
+    assert abs(mse - np.sum((Hf - Hq) ** 2)) < 1e-12 and np.allclose(dH, 2 * (Hq - Hf), rtol=0, atol=1e-15)
+    # softmax ignores a per-token shift of the logits
+    kl2, _, dZ2, _ = fo.align_loss(Zf + rng.standard_normal((T, 1)) * 50, Zq - 7.0, Hf, Hq, tau=1.7, lambda_kl=0.3)
+    assert abs(kl2 - kl) < 1e-12 and np.max(np.abs(dZ2 - dZ)) < 1e-15
+    # the temperature divides the logits: (tau Z, tau) is (Z, 1) up to the 1/tau of the gradient
+    kl3, _, dZ3, _ = fo.align_loss(1.7 * Zf, 1.7 * Zq, Hf, Hq, tau=1.7, lambda_kl=0.3)
+    kl4, _, dZ4, _ = fo.align_loss(Zf, Zq, Hf, Hq, tau=1.0, lambda_kl=0.3)
+    assert abs(kl3 - kl4) < 1e-12 and np.max(np.abs(dZ3 * 1.7 - dZ4)) < 1e-15
+    # two classes: KL of two Bernoulli distributions with p = sigmoid(a / tau), q = sigmoid(b / tau)
+    a, b, tau = 1.3, -0.4, 0.8
+    p, q = 1 / (1 + np.exp(-a / tau)), 1 / (1 + np.exp(-b / tau))
+    kl5, _, dZ5, _ = fo.align_loss(np.array([[a, 0.0]]), np.array([[b, 0.0]]), Hf[:1], Hf[:1], tau=tau)
+    assert abs(kl5 - (p * np.log(p / q) + (1 - p) * np.log((1 - p) / (1 - q)))) < 1e-14
+    assert abs(dZ5[0, 0] - (q - p) / tau) < 1e-15
+    # uniform quantised model: KL = log V - entropy(P_fp), averaged over the tokens
+    pf = np.exp(Zf - Zf.max(1, keepdims=True)); pf /= pf.sum(1, keepdims=True)
+    ent = -(pf * np.log(pf)).sum(1)
+    kl6, *_ = fo.align_loss(Zf, np.zeros_like(Zf), Hf, Hf)
+    assert abs(kl6 - np.mean(np.log(V) - ent)) < 1e-12
+    # logits far apart do not overflow
+    kl7, _, dZ7, _ = fo.align_loss(np.array([[800.0, 0.0, -800.0]]), np.array([[0.0, 0.0, 0.0]]), Hf[:1], Hf[:1])
+    assert np.isfinite(kl7) and abs(kl7 - np.log(3)) < 1e-12 and np.all(np.isfinite(dZ7))
+
+
+def test_align_loss_gradients_match_finite_differences():
+    rng = np.random.default_rng(1)
+    T, V, D = 4, 23, 6
+    Zf, Zq = rng.standard_normal((T, V)) * 2, rng.standard_normal((T, V)) * 2
+    Hf, Hq = rng.standard_normal((T, D)), rng.standard_normal((T, D))
+    tau, lam = 1.3, 0.7
+    _, _, dZ, dH = fo.align_loss(Zf, Zq, Hf, Hq, tau, lam)
+    eps = 1e-6
+    for _ in range(40):
+        t, v = rng.integers(T), rng.integers(V)
+        Zp, Zm = Zq.copy(), Zq.copy()
+        Zp[t, v] += eps; Zm[t, v] -= eps
+        fd = lam * (fo.align_loss(Zf, Zp, Hf, Hq, tau, lam)[0] - fo.align_loss(Zf, Zm, Hf, Hq, tau, lam)[0]) / (2 * eps)
+        assert abs(fd - dZ[t, v]) <= 1e-8 + 1e-6 * abs(dZ[t, v])
+    for _ in range(10):
+        t, d = rng.integers(T), rng.integers(D)
+        Hp, Hm = Hq.copy(), Hq.copy()
+        Hp[t, d] += eps; Hm[t, d] -= eps
+        fd = (fo.align_loss(Zf, Zq, Hf, Hp, tau, lam)[1] - fo.align_loss(Zf, Zq, Hf, Hm, tau, lam)[1]) / (2 * eps)
+        assert abs(fd - dH[t, d]) <= 1e-7
