@@ -172,7 +172,8 @@ enum {
   FAAR_K_HARDEN_PACK = 8,
   FAAR_K_TRANSPOSE = 9,
   FAAR_K_ACT_FAKEQUANT = 10, /* activations to NVFP4 values (the X_q of Eq. 5)          */
-  FAAR_K_COUNT = 11
+  FAAR_K_ALIGN_LOSS = 11,    /* Eq. 6: KL of the softmaxes + last-hidden error, gradients */
+  FAAR_K_COUNT = 12
 };
 typedef struct {
   int kernel;     /* one of FAAR_K_*          */
@@ -338,6 +339,28 @@ FAAR_API int faar_layer_step_host(faar_ctx* ctx, const faar_shape* shape, const 
 FAAR_API int faar_harden_pack(faar_ctx* ctx, const faar_shape* shape, const float* V, const uint8_t* code,
                      const uint8_t* scales, const float* s_global, uint8_t* packed,
                      uint8_t* scales_out, uint8_t* decisions, void* W_final, int wfinal_dtype);
+
+/* ---- full-model alignment loss (towards Stage 2) --------------------------------
+ * Eq. 6 / Procedure steps 18-20: P_fp = softmax(Z_fp / tau), P_q = softmax(Z_q / tau)
+ * over the vocabulary; L_KL = KL(P_fp || P_q) summed over the vocabulary and averaged
+ * over the T tokens (the paper gives no reduction over tokens); L_MSE = the squared
+ * Frobenius norm of H_fp - H_q.  Also the gradients towards the quantised model's
+ * outputs, which its backward pass starts from:
+ *   dZ_q = lambda_kl (P_q - P_fp) / (tau T)      dH_q = 2 (H_q - H_fp)
+ * (the Round Loss term of Eq. 6 is per layer: faar_round_loss / the backward epilogue).
+ *   Z_fp, Z_q in : [T, vocab] bf16, row stride ldz      dZ_q out: same layout, nullable
+ *   H_fp, H_q in : [T, hidden] bf16, row stride ldh     dH_q out: same layout, nullable
+ *   loss_out2 out: {L_KL, L_MSE} (device)
+ * ldz, ldh: multiples of 8 and at least the column count rounded up to 8 (the kernel
+ * reads whole 16-byte vectors; padding columns are read, never written); all bases
+ * 16-byte aligned.  vocab up to 409 600 (two rows of a token must fit the shared
+ * memory of a cluster of eight SMs); larger is FAAR_ERR_SHAPE.  The workspace
+ * (faar_align_loss_workspace_size, 256-byte aligned, header zeroed once by
+ * faar_workspace_init) holds the per-CTA partial sums. */
+FAAR_API int faar_align_loss_workspace_size(int T, int vocab, size_t* bytes);
+FAAR_API int faar_align_loss(faar_ctx* ctx, int T, int vocab, int hidden, const void* Z_fp, const void* Z_q,
+                             int64_t ldz, const void* H_fp, const void* H_q, int64_t ldh, float tau, float lambda_kl,
+                             void* dZ_q, void* dH_q, float* loss_out2, void* workspace, size_t workspace_bytes);
 
 /* ---- deployable scale-factor layout ---------------------------------------
  * "Hardening and Inference": the final weights are "directly deployable on NVFP4

@@ -225,6 +225,7 @@ const char* faar_kernel_name(int kernel) {
     case FAAR_K_HARDEN_PACK: return "harden_pack";
     case FAAR_K_TRANSPOSE: return "transpose";
     case FAAR_K_ACT_FAKEQUANT: return "act_fakequant";
+    case FAAR_K_ALIGN_LOSS: return "align_loss";
   }
   return "unknown";
 }
@@ -598,6 +599,44 @@ int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales
   if (reinterpret_cast<uintptr_t>(scales_tiled) & 3u) return FAAR_ERR_ALIGN;
   DeviceGuard g(ctx->device);
   return cuda_fail(ctx, faar_launch_swizzle_scales(ctx, rows, cols, scales, scales_tiled));
+}
+
+int faar_align_loss_workspace_size(int T, int vocab, size_t* bytes) {
+  if (!bytes) return FAAR_ERR_INVALID_ARG;
+  if (T <= 0 || vocab <= 0) return FAAR_ERR_SHAPE;
+  int chunk = 0;
+  const int cs = faar_align_cluster_size(vocab, &chunk);
+  if (cs == 0 || (long long)T * cs > 0x7FFFFFFFll) return FAAR_ERR_SHAPE;
+  *bytes = faar_align_up(FAAR_WS_HEADER + 2 * sizeof(float) * (size_t)T * (size_t)cs, 1024);
+  return FAAR_OK;
+}
+
+int faar_align_loss(faar_ctx* ctx, int T, int vocab, int hidden, const void* Z_fp, const void* Z_q, int64_t ldz,
+                    const void* H_fp, const void* H_q, int64_t ldh, float tau, float lambda_kl, void* dZ_q, void* dH_q,
+                    float* loss_out2, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !Z_fp || !Z_q || !H_fp || !H_q || !loss_out2) return FAAR_ERR_INVALID_ARG;
+  if (!(tau > 0.f) || !isfinite(tau) || !isfinite(lambda_kl)) return FAAR_ERR_INVALID_ARG;
+  if (T <= 0 || vocab <= 0 || hidden <= 0) return FAAR_ERR_SHAPE;
+  if (ldz < ((int64_t)vocab + 7) / 8 * 8 || ldh < ((int64_t)hidden + 7) / 8 * 8) return FAAR_ERR_SHAPE;
+  if (ldz % 8 || ldh % 8) return FAAR_ERR_ALIGN;
+  if (!aligned16(Z_fp) || !aligned16(Z_q) || !aligned16(H_fp) || !aligned16(H_q) || (dZ_q && !aligned16(dZ_q)) ||
+      (dH_q && !aligned16(dH_q)))
+    return FAAR_ERR_ALIGN;
+  size_t need = 0;
+  int st = faar_align_loss_workspace_size(T, vocab, &need);
+  if (st) return st;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need) return FAAR_ERR_WORKSPACE;
+  DeviceGuard g(ctx->device);
+  int chunk = 0;
+  const int cs = faar_align_cluster_size(vocab, &chunk);
+  float* kl_p = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + FAAR_WS_HEADER);
+  float* mse_p = kl_p + (size_t)T * cs;
+  int np = 0;
+  int e = faar_launch_align_loss(ctx, T, vocab, hidden, Z_fp, Z_q, ldz, H_fp, H_q, ldh, tau, lambda_kl, dZ_q, dH_q, kl_p,
+                                 mse_p, &np);
+  if (e) return cuda_fail(ctx, e);
+  e = faar_launch_finalize(ctx, kl_p, np, (float)(1.0 / (double)T), loss_out2, mse_p, np, 1.0f, loss_out2 + 1);
+  return cuda_fail(ctx, e);
 }
 
 int faar_harden_pack(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code, const uint8_t* scales,

@@ -22,7 +22,8 @@ EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string
            "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
            "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n", "faar_tune_tile_n",
            "faar_last_gemm_config", "faar_act_fakequant", "faar_swizzle_scales", "faar_tune_tail_split",
-           "faar_last_tail_split", "faar_selftest_wait_timeout", "faar_layer_dx"]
+           "faar_last_tail_split", "faar_selftest_wait_timeout", "faar_layer_dx", "faar_align_loss",
+           "faar_align_loss_workspace_size"]
 
 
 class HParams(C.Structure):
@@ -190,6 +191,18 @@ def act_fakequant(ctx, T, K, X, ldx, s_global_in, Xq_units, ldq, s_global_out, p
     _check(lib().faar_act_fakequant(ctx._h, T, K, _p(X), C.c_int64(ldx), C.c_float(s_global_in), _p(Xq_units),
                                     C.c_int64(ldq), _p(s_global_out), _p(packed), _p(scales), _p(ws),
                                     C.c_size_t(ws.numel())), "faar_act_fakequant")
+
+
+def align_loss_workspace_size(T, vocab) -> int:
+    n = C.c_size_t(0)
+    _check(lib().faar_align_loss_workspace_size(T, vocab, C.byref(n)), "faar_align_loss_workspace_size")
+    return n.value
+
+
+def align_loss(ctx, T, vocab, hidden, Z_fp, Z_q, ldz, H_fp, H_q, ldh, tau, lambda_kl, dZ_q, dH_q, loss_out2, ws):
+    _check(lib().faar_align_loss(ctx._h, T, vocab, hidden, _p(Z_fp), _p(Z_q), C.c_int64(ldz), _p(H_fp), _p(H_q),
+                                 C.c_int64(ldh), C.c_float(tau), C.c_float(lambda_kl), _p(dZ_q), _p(dH_q), _p(loss_out2),
+                                 _p(ws), C.c_size_t(ws.numel())), "faar_align_loss")
 
 
 def swizzle_scales(ctx, rows, cols, scales, scales_tiled):
