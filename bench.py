@@ -339,12 +339,36 @@ def run_ours(args):
 
     dx_us = layer_dx_us()
 
+    # ---- Eq. 6's alignment loss alone: 4096 tokens x 128 256 logits (3.2 GB moved per call, far above L2)
+    AL_T, AL_V, AL_D = 4096, 128256, 2048
+
+    def align_loss_us(rounds=5):
+        g = torch.Generator(device=device).manual_seed(1)
+        zf = (torch.randn((AL_T, AL_V), device=device, generator=g) * 3).to(torch.bfloat16)
+        zq = (zf.float() + 0.3 * torch.randn((AL_T, AL_V), device=device, generator=g)).to(torch.bfloat16)
+        hf = torch.randn((AL_T, AL_D), device=device, generator=g).to(torch.bfloat16)
+        hq = (hf.float() + 0.05 * torch.randn((AL_T, AL_D), device=device, generator=g)).to(torch.bfloat16)
+        dz, dh = torch.empty_like(zq), torch.empty_like(hq)
+        l2 = torch.zeros(2, dtype=torch.float32, device=device)
+        aws = torch.empty(faar.align_loss_workspace_size(AL_T, AL_V), dtype=torch.uint8, device=device)
+        faar.workspace_init(ctx, aws)
+        fn = lambda: faar.align_loss(ctx, AL_T, AL_V, AL_D, zf, zq, AL_V, hf, hq, AL_D, 1.0, 1.0, dz, dh, l2, aws)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                fn()
+        stream.synchronize()
+        us = 1e3 * timed(lambda: [fn() for _ in range(rounds)]) / rounds
+        faar.check_status(ctx, aws)
+        return us
+
+    al_us = align_loss_us()
+
     if args.quick:
         if rank == 0:
             print(json.dumps({"quick": True, "steps": steps, "ms_per_step": ms_job / steps,
                               "kernels_avg_us": {k: round(1e3 * v[1] / v[0], 2) for k, v in prof.items()},
                               "elementwise_alone_us": {k: round(v, 2) for k, v in ew_us.items()},
-                              "layer_dx_us": round(dx_us, 2)}))
+                              "layer_dx_us": round(dx_us, 2), "align_loss_us": round(al_us, 2)}))
         if sampler:
             sampler.stop()
         if world > 1:
@@ -415,6 +439,12 @@ def run_ours(args):
                            "frac": round(flops / (dx_us * 1e-6) / 1e12 / pk["bf16_tflops_sustained"], 4),
                            "timed": "20 back-to-back calls (soft weights, transpose and GEMM each), one event pair",
                            "note": "input gradient dX = dY W_soft, not part of a Stage-1 step"}
+    al_bytes = 3.0 * AL_T * AL_V * 2 + 3.0 * AL_T * AL_D * 2          # both logit / hidden tensors read, one gradient written
+    kernels["align_loss"] = {"avg_us": round(al_us, 2), "bound": "hbm", "achieved": round(al_bytes / (al_us * 1e-6) / 1e9, 1),
+                             "peak": pk["hbm_gbs"], "unit": "GB/s",
+                             "frac": round(al_bytes / (al_us * 1e-6) / 1e9 / pk["hbm_gbs"], 4),
+                             "timed": "5 back-to-back calls on 4096 tokens x 128256 logits (+ 2048 hidden), one event pair",
+                             "note": "Eq. 6's KL and last-hidden terms with gradients; not part of a Stage-1 step"}
     kernels["softquant_init"]["note"] = "amax pass + bracket pass together; the amax pass re-reads W (+2 B/weight, not " \
                                         "counted); the bracket pass is bound by its IEEE divisions, not by HBM"
     for name in prof:

@@ -353,10 +353,8 @@ FAAR_API int faar_harden_pack(faar_ctx* ctx, const faar_shape* shape, const floa
  *   loss_out2 out: {L_KL, L_MSE} (device)
  * ldz, ldh: multiples of 8 and at least the column count rounded up to 8 (the kernel
  * reads whole 16-byte vectors; padding columns are read, never written); all bases
- * 16-byte aligned.  vocab up to 409 600 (two rows of a token must fit the shared
- * memory of a cluster of eight SMs); larger is FAAR_ERR_SHAPE.  The workspace
- * (faar_align_loss_workspace_size, 256-byte aligned, header zeroed once by
- * faar_workspace_init) holds the per-CTA partial sums. */
+ * 16-byte aligned.  The workspace (faar_align_loss_workspace_size, 256-byte aligned,
+ * header zeroed once by faar_workspace_init) holds the per-CTA partial sums. */
 FAAR_API int faar_align_loss_workspace_size(int T, int vocab, size_t* bytes);
 FAAR_API int faar_align_loss(faar_ctx* ctx, int T, int vocab, int hidden, const void* Z_fp, const void* Z_q,
                              int64_t ldz, const void* H_fp, const void* H_q, int64_t ldh, float tau, float lambda_kl,

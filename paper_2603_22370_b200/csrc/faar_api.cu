@@ -604,10 +604,7 @@ int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales
 int faar_align_loss_workspace_size(int T, int vocab, size_t* bytes) {
   if (!bytes) return FAAR_ERR_INVALID_ARG;
   if (T <= 0 || vocab <= 0) return FAAR_ERR_SHAPE;
-  int chunk = 0;
-  const int cs = faar_align_cluster_size(vocab, &chunk);
-  if (cs == 0 || (long long)T * cs > 0x7FFFFFFFll) return FAAR_ERR_SHAPE;
-  *bytes = faar_align_up(FAAR_WS_HEADER + 2 * sizeof(float) * (size_t)T * (size_t)cs, 1024);
+  *bytes = faar_align_up(FAAR_WS_HEADER + 2 * sizeof(float) * (size_t)T, 1024);      // two partial sums per CTA
   return FAAR_OK;
 }
 
@@ -627,10 +624,8 @@ int faar_align_loss(faar_ctx* ctx, int T, int vocab, int hidden, const void* Z_f
   if (st) return st;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need) return FAAR_ERR_WORKSPACE;
   DeviceGuard g(ctx->device);
-  int chunk = 0;
-  const int cs = faar_align_cluster_size(vocab, &chunk);
   float* kl_p = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + FAAR_WS_HEADER);
-  float* mse_p = kl_p + (size_t)T * cs;
+  float* mse_p = kl_p + (size_t)T;
   int np = 0;
   int e = faar_launch_align_loss(ctx, T, vocab, hidden, Z_fp, Z_q, ldz, H_fp, H_q, ldh, tau, lambda_kl, dZ_q, dH_q, kl_p,
                                  mse_p, &np);

@@ -84,8 +84,7 @@ int faar_launch_act_fakequant(faar_ctx*, int T, int K, const void* X, int64_t ld
 int faar_launch_transpose_bf16(faar_ctx*, int rows, int cols, const void* in, int64_t ld_in, void* out,
                                int64_t ld_out);
 int faar_launch_swizzle_scales(faar_ctx*, int rows, int cols, const uint8_t* in, uint8_t* out);
-// Eq. 6's data terms: cluster size for a vocabulary (0 = too large) and the launch (one partial per CTA)
-int faar_align_cluster_size(int vocab, int* chunk_out);
+// Eq. 6's data terms: one partial per CTA, at most one CTA per token
 int faar_launch_align_loss(faar_ctx*, int T, int vocab, int hidden, const void* Z_fp, const void* Z_q, int64_t ldz,
                            const void* H_fp, const void* H_q, int64_t ldh, float tau, float lambda_kl, void* dZ_q,
                            void* dH_q, float* kl_partials, float* mse_partials, int* n_partials);

@@ -1,6 +1,6 @@
 """GPU parity of faar_align_loss (Eq. 6's data terms and their gradients) against the oracle: vocabularies
-that use clusters of 1, 2, 4 and 8 CTAs per token, ragged sizes, padded rows, several temperatures, and a
-full-size vocabulary checked on sampled tokens."""
+from one entry to 130 000 (fewer and more 16-byte groups than the CTA has threads), ragged sizes, padded
+rows, several temperatures, more tokens than SMs, and a full-size vocabulary checked on sampled tokens."""
 import numpy as np
 import pytest
 import torch
@@ -48,9 +48,8 @@ def _bf16(a):
     return inputs.to_bf16_f32(a.astype(np.float32))
 
 
-# vocabularies: one CTA per token; clusters of 2, 4, 8; ragged (not a multiple of 8, chunks that leave the
-# last CTA of the cluster almost or wholly empty)
 @pytest.mark.parametrize("T,V,D,tau,lam,pad", [(5, 37, 8, 1.0, 1.0, 0), (3, 18432, 64, 1.0, 1.0, 0), (4, 20003, 70, 1.7, 0.3, 8),
+                                               (333, 1000, 16, 1.0, 1.0, 0), (2, 8199, 8, 1.0, 1.0, 0),
                                                (3, 50257, 33, 0.7, 2.0, 0), (2, 130000, 100, 1.0, 1.0, 16),
                                                (2, 73729, 9, 2.5, 1.0, 0), (1, 1, 1, 1.0, 1.0, 0)])
 def test_align_loss_matches_oracle(ctx, T, V, D, tau, lam, pad):
@@ -90,7 +89,7 @@ def test_arguments_are_checked(ctx):
     loss = torch.zeros(2, device=DEV)
     ws = torch.empty(faar.align_loss_workspace_size(2, 64), dtype=torch.uint8, device=DEV)
     faar.workspace_init(ctx, ws)
-    bad = [dict(tau=0.0), dict(tau=float("nan")), dict(ldz=60), dict(ldz=68), dict(ldh=4), dict(V=500000)]
+    bad = [dict(tau=0.0), dict(tau=float("nan")), dict(ldz=60), dict(ldz=68), dict(ldh=4), dict(T=0)]
     for kw in bad:
         a = dict(T=2, V=64, D=8, ldz=64, ldh=8, tau=1.0)
         a.update(kw)
