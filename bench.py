@@ -340,7 +340,7 @@ def run_ours(args):
     dx_us = layer_dx_us()
 
     # ---- Eq. 6's alignment loss alone: 4096 tokens x 128 256 logits (3.2 GB moved per call, far above L2)
-    AL_T, AL_V, AL_D = 4096, 128256, 2048
+    AL_T, AL_V, AL_D = args.align_tokens, 128256, 2048
 
     def align_loss_us(rounds=5):
         g = torch.Generator(device=device).manual_seed(1)
@@ -443,7 +443,7 @@ def run_ours(args):
     kernels["align_loss"] = {"avg_us": round(al_us, 2), "bound": "hbm", "achieved": round(al_bytes / (al_us * 1e-6) / 1e9, 1),
                              "peak": pk["hbm_gbs"], "unit": "GB/s",
                              "frac": round(al_bytes / (al_us * 1e-6) / 1e9 / pk["hbm_gbs"], 4),
-                             "timed": "5 back-to-back calls on 4096 tokens x 128256 logits (+ 2048 hidden), one event pair",
+                             "timed": f"5 back-to-back calls on {AL_T} tokens x 128256 logits (+ 2048 hidden), one event pair",
                              "note": "Eq. 6's KL and last-hidden terms with gradients; not part of a Stage-1 step"}
     kernels["softquant_init"]["note"] = "amax pass + bracket pass together; the amax pass re-reads W (+2 B/weight, not " \
                                         "counted); the bracket pass is bound by its IEEE divisions, not by HBM"
@@ -492,6 +492,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--align-tokens", type=int, default=4096,
+                    help="tokens of the alignment-loss timing (128256 logits each); smaller for profiler captures")
     ap.add_argument("--chain", action="store_true",
                     help="build each step's soft weights inside the previous step's backward kernel (same values; the "
                          "job is faster, the backward kernel slower, so its roofline line is not comparable)")

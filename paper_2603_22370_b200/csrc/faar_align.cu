@@ -48,6 +48,16 @@ __device__ __forceinline__ uint64_t l2_stream_policy() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
+__device__ __forceinline__ uint64_t l2_keep_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint4 ldg128_policy(const uint4* ptr, uint64_t pol) {
+  uint4 v;
+  asm volatile("ld.global.L2::cache_hint.v4.b32 {%0,%1,%2,%3}, [%4], %5;" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr), "l"(pol));
+  return v;
+}
 // the gradient is written once and not read here: it should not push the rows out of L2
 __device__ __forceinline__ void stg128_policy(void* ptr, uint4 v, uint64_t pol) {
   asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w),
@@ -95,7 +105,7 @@ align_loss_kernel(const AlignParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int ngroups = (p.V + 7) / 8;                               // 16-byte groups of a row (rows are padded: ldz >= ceil8(V))
   const int tail = p.V & 7;                                        // valid columns of a partial last group, 0 = none
-  const uint64_t stream = l2_stream_policy();
+  const uint64_t stream = l2_stream_policy(), keep = l2_keep_policy();   // first pass: keep the rows in L2; second: done with them
   float kl = 0.f, mse = 0.f;                                       // this thread's share over all of the CTA's tokens
   for (int t = blockIdx.x; t < p.T; t += gridDim.x) {
     const uint4* gf = reinterpret_cast<const uint4*>(p.Zfp + (long long)t * p.ldz);
@@ -116,7 +126,8 @@ align_loss_kernel(const AlignParams p) {
     {
       int g = threadIdx.x;
       for (; g + AL_THREADS < ngroups; g += 2 * AL_THREADS) {      // two groups per tensor in flight; neither is the last
-        const uint4 a0 = gf[g], b0 = gq[g], a1 = gf[g + AL_THREADS], b1 = gq[g + AL_THREADS];
+        const uint4 a0 = ldg128_policy(gf + g, keep), b0 = ldg128_policy(gq + g, keep);
+        const uint4 a1 = ldg128_policy(gf + g + AL_THREADS, keep), b1 = ldg128_policy(gq + g + AL_THREADS, keep);
         online(a0, mf, sf);
         online(b0, mq, sq);
         if (tail && g + AL_THREADS == ngroups - 1) {
@@ -128,7 +139,7 @@ align_loss_kernel(const AlignParams p) {
         }
       }
       if (g < ngroups) {
-        uint4 a = gf[g], b = gq[g];
+        uint4 a = ldg128_policy(gf + g, keep), b = ldg128_policy(gq + g, keep);
         if (tail && g == ngroups - 1) { a = mask_tail(a, tail); b = mask_tail(b, tail); }
         online(a, mf, sf);
         online(b, mq, sq);
@@ -156,7 +167,7 @@ align_loss_kernel(const AlignParams p) {
     const float dlse = lse_f - lse_q;
     __nv_bfloat16* const gd = p.dZ ? p.dZ + (long long)t * p.ldz : nullptr;
     for (int g = threadIdx.x; g < ngroups; g += AL_THREADS) {
-      uint4 va = gf[g], vb = gq[g];
+      uint4 va = ldg128_policy(gf + g, stream), vb = ldg128_policy(gq + g, stream);
       const bool last_partial = tail && g == ngroups - 1;
       if (last_partial) { va = mask_tail(va, tail); vb = mask_tail(vb, tail); }
       float a[8], b[8], gr[8];
