@@ -114,16 +114,19 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
     for (int i = 0; i < 8; ++i) {
       float wt = s > 0.f ? __fdiv_rn(fabsf(w[i]), s) : 0.f;
       wt = fminf(wt, 6.0f);
-      // interval index from the bits of w~ (exponent and top mantissa bit order like the nodes):
-      // [.5,.75) -> 0, [.75,1) -> 1, [1,1.5) -> 2, [1.5,2) -> 3, [2,3) -> 4, [3,4) -> 5, [4,6) -> 6, 6 -> 7
-      const int t = (int)(__float_as_uint(wt) >> 22) - 252;
-      int k = wt < 0.5f ? 0 : max(t, 1);
-      k = min(k, 6);
-      float lo = faar_node(k);
-      float inv_w = __uint_as_float((uint32_t)(128 - (k >= 4) - (k >= 6)) << 23);   // 2, 1, 0.5
-      v[i] = __fmul_rn(__fsub_rn(wt, lo), inv_w);
-      uint32_t neg = (w[i] < 0.f) ? 8u : 0u;
-      cw |= ((uint32_t)k | neg) << (4 * i);
+      // From 1 upwards the nodes are the floats with a one-bit mantissa, so the bits of w~ give the bracket:
+      // lower node = w~ with the mantissa cut to its top bit, interval index = (bits >> 22) - 252
+      // ([1,1.5) -> 2, [1.5,2) -> 3, [2,3) -> 4, [3,4) -> 5, [4,6) -> 6), 1 / width = 2^(1 - exponent).
+      // Below 1 the nodes 0, 0.5, 1 are 0.5 apart.  w~ = 6 (the clamp) closes the last interval: k = 6, v = 1.
+      const uint32_t wb = __float_as_uint(wt);
+      const bool ge1 = wt >= 1.0f, geh = wt >= 0.5f;
+      const float lo = ge1 ? __uint_as_float(wb & 0xFFC00000u) : (geh ? 0.5f : 0.0f);
+      const float inv_w = ge1 ? __uint_as_float(0x7F800000u - (wb & 0x7F800000u)) : 2.0f;      // 2, 1, 0.5
+      uint32_t k = ge1 ? (wb >> 22) - 252u : (geh ? 1u : 0u);
+      float vi = __fmul_rn(__fsub_rn(wt, lo), inv_w);
+      if (wt >= 6.0f) { k = 6u; vi = 1.0f; }
+      v[i] = vi;
+      cw |= (k | (w[i] < 0.f ? 8u : 0u)) << (4 * i);                  // -0.0 counts as positive
     }
     if (valid) {
       const int64_t e = g * 8;                 // V, code, scales are dense
