@@ -427,6 +427,7 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
   float nbl_next, hbl_next;                                       // OPT & 2: constants of the next step's Eq. 3
   faar_operand_consts(p.beta_next, &nbl_next, &hbl_next);
   const uint64_t stream = l2_policy_stream();
+  const uint64_t vkeep = l2_policy_keep();       // the updated V is the next kernel's input (soft weights)
   float tt = 0.f, n_el = 0.f;                                     // sum of (2 v - 1)^2, elements seen
 #pragma unroll
   for (int grp = 0; grp < ITS / RPG; ++grp) {
@@ -514,7 +515,7 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
           stg128_stream(Mp + off, mn[0], mn[1], mn[2], mn[3], stream);
           stg128_stream(Up + off, un[0], un[1], un[2], un[3], stream);
         }
-        stg128_stream(Vp + off, vn[0], vn[1], vn[2], vn[3], stream);
+        stg128_stream(Vp + off, vn[0], vn[1], vn[2], vn[3], vkeep);
         n_el += 4.f;
       }
     }
