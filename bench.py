@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the
 # ncu capture summarised under profiles/; None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"gemm_bwd": 463.3e6, "gemm_fwd": 160.7e6}     # profiles/faar_gemm_kernel_down_proj.md
+NCU_TRAFFIC_BYTES = {"gemm_bwd": 463.0e6, "gemm_fwd": 159.5e6}     # profiles/faar_gemm_kernel_down_proj.md
 
 
 def peaks():
