@@ -125,7 +125,7 @@ align_loss_kernel(const AlignParams p) {
     };
     {
       int g = threadIdx.x;
-      for (; g + AL_THREADS < ngroups; g += 2 * AL_THREADS) {      // two groups per tensor in flight; neither is the last
+      for (; g + AL_THREADS < ngroups; g += 2 * AL_THREADS) {      // two groups per tensor in flight; only the second can be the row's last
         const uint4 a0 = ldg128_policy(gf + g, keep), b0 = ldg128_policy(gq + g, keep);
         const uint4 a1 = ldg128_policy(gf + g + AL_THREADS, keep), b1 = ldg128_policy(gq + g + AL_THREADS, keep);
         online(a0, mf, sf);
