@@ -853,16 +853,19 @@ int make_map(faar_ctx* ctx, CUtensorMap* map, const void* ptr, int rows, int col
   return r == CUDA_SUCCESS ? 0 : (int)cudaErrorInvalidValue;
 }
 
-// Tile width for an M x N output.  Measured on the down_proj-shaped layer, a tile's time is set by the
-// operand bytes it pulls through the SM (A rows are not shared between tiles), not by its columns, so
-// narrower tiles never pay while the widest ones already fill the device; they are used only to get at
-// least one tile per CTA pair on small problems.
-int pick_bn(const faar_ctx* ctx, int M, int N, int pairs) {
+// Tile width for an M x N output.  A tile's time is set by the operand bytes it pulls through the SM (A rows
+// are not shared between tiles), not by its columns, so 256-wide tiles win wherever they were measured
+// against narrower ones that fill more CTA pairs (down_proj-, gate-, q- and k_proj-shaped layers), with one
+// exception: the dW GEMM of a small layer, whose per-weight epilogue is heavy, gains from spreading 128-wide
+// tiles over twice as many pairs while fewer than half of the pairs would have a 256-wide tile.  A tile is
+// never wider than the output rounded up to 32 columns.
+int pick_bn(const faar_ctx* ctx, int mode, int M, int N, int pairs) {
   if (ctx->tune_bn >= 128 && ctx->tune_bn <= BN_MAX && ctx->tune_bn % 16 == 0) return ctx->tune_bn;
   const long long m_tiles = (M + 2 * BM - 1) / (2 * BM);
-  for (int bn = BN_MAX; bn > 128; bn -= 32)
-    if (m_tiles * ((N + bn - 1) / bn) >= pairs) return bn;
-  return 128;
+  int bn = BN_MAX;
+  if (N < BN_MAX) bn = N <= 128 ? 128 : (N + 31) / 32 * 32;
+  if (mode == FAAR_GEMM_BWD && 2 * m_tiles * ((N + BN_MAX - 1) / BN_MAX) < pairs) bn = 128;
+  return bn;
 }
 
 // How many trailing tile columns to cut into half-width tiles.  Tiles go to CTA pairs round-robin, all
@@ -927,7 +930,7 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
     if (n > ctx->num_sms / 2) n = ctx->num_sms / 2;
     max_pairs = n;
   }
-  const int bn = pick_bn(ctx, a->M, a->N, max_pairs);
+  const int bn = pick_bn(ctx, MODE, a->M, a->N, max_pairs);
   kp.bn = bn;
   kp.n_full_cols = pick_full_cols(ctx, a->M, a->N, bn, max_pairs);
   CUtensorMap tmA, tmB, tmBh;
