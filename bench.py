@@ -1,13 +1,18 @@
 """Benchmark of the FAAR layer step on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2|3|4] [--impl ours|reference]
 
-One job = the whole hot path for one linear layer of the down_proj-shaped workload
-(W 2048x8192 BF16, calibration batch X 4096x8192 BF16): soft-quantisation set-up, K optimisation
-steps (soft weights -> forward GEMM + MSE -> dW GEMM + dV + Round Loss + Adam update, beta annealed
-geometrically over the K steps), then harden + pack.  `value` = K / (device time of that job), so the
-once-per-layer kernels are inside the timed region.  With N > 1 every rank runs its own layer (layers
-are independent problems: no data-path collective), value = N*K / max-over-ranks time.
+--config 2 (default): one job = the whole hot path for one linear layer of the down_proj-shaped workload
+(W 2048x8192 BF16, calibration batch X 4096x8192 BF16): soft-quantisation set-up, K optimisation steps
+(soft weights -> forward GEMM + MSE -> dW GEMM + dV + Round Loss + Adam update, beta annealed geometrically
+over the K steps), then harden + pack.  `value` = K / (device time of that job), so the once-per-layer
+kernels are inside the timed region.  With N > 1 every rank runs its own layer (layers are independent
+problems: no data-path collective), value = N*K / max-over-ranks time.
+
+--config 3 / 4: the seven linears of a Llama-3.2-1B- / Qwen3-1.7B-shaped decoder block, each optimised for K
+steps on 4096-row minibatches of a synthetic calibration set (Stage-1 driver of the package); `value` =
+K / (summed device time of the seven jobs) = block steps per second, with one line per linear under
+`linears` (soft weights / forward / backward microseconds, TFLOP/s, fraction of the BF16 peak).
 
 `--impl reference` times the CPU oracle (numpy, float64) on the host cores instead; each of its
 steps is a row-sample of the same layer (the loss separates over output rows, so a sample of rows is
@@ -16,6 +21,7 @@ an exact sub-problem) and the rate is scaled by rows/sample.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -30,12 +36,55 @@ if ROOT not in sys.path:
 O, K, T = 2048, 8192, 4096
 WORKLOAD = "Llama-3.2-1B-shaped down_proj: W 2048x8192 bf16 (0.02*N(0,1), 0.1% x10), X 4096x8192 bf16 " \
            "(Student-t(4), 16 channels x20), Adam lr 1e-2, beta 4->32 geometric"
+BLOCK_WORKLOADS = {
+    3: "Llama-3.2-1B-shaped decoder block, Stage 1 layer-wise: q/o 2048x2048, k/v 512x2048, gate/up 8192x2048, "
+       "down 2048x8192, W bf16 0.02*N(0,1); calibration hidden states N(0,1) + 8 channels x30, RMS-normalised, "
+       "4096-row minibatches; Adam lr 1e-2, beta 4->32 geometric",
+    4: "Qwen3-1.7B-shaped decoder block, Stage 1 layer-wise: q/o 2048x2048, k/v 1024x2048, gate/up 6144x2048, "
+       "down 2048x6144, W bf16 0.02*N(0,1); calibration hidden states N(0,1) + 8 channels x30, RMS-normalised, "
+       "4096-row minibatches; Adam lr 1e-2, beta 4->32 geometric",
+}
 METRIC, UNIT = "faar_layer_steps_per_s", "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the
-# ncu capture summarised under profiles/; None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"gemm_bwd": 463.0e6, "gemm_fwd": 159.5e6}     # profiles/faar_gemm_kernel_down_proj.md
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the GEMM kernels on the config-2
+# layer, from one ncu capture each, with the SHA-256 (first 12 hex digits) of the kernel source at the time of
+# the capture.  A kernel source that has changed since makes the figure stale: `traffic` is then null.
+NCU_TRAFFIC = {
+    "gemm_bwd": {"bytes": 463.0e6, "source_sha": "0" * 12},
+    "gemm_fwd": {"bytes": 159.5e6, "source_sha": "0" * 12},
+}
+GEMM_SOURCE = os.path.join(ROOT, "paper_2603_22370_b200", "csrc", "faar_gemm.cu")
+
+
+def ncu_traffic(kernel):
+    """The recorded DRAM traffic of `kernel`, or None when the kernel source is no longer the captured one."""
+    rec = NCU_TRAFFIC.get(kernel)
+    if not rec or not os.path.exists(GEMM_SOURCE):
+        return None
+    with open(GEMM_SOURCE, "rb") as f:
+        sha = hashlib.sha256(f.read()).hexdigest()[:12]
+    return rec["bytes"] if sha == rec["source_sha"] else None
+
+
+def tensor_fracs(tflops, pk):
+    """Achieved BF16 rate against the three denominators: the measured burst rate (a kernel timed in a job
+    short enough to stay at boost clocks), the measured sustained rate (a seconds-long job under the power
+    cap) and the nominal dense peak."""
+    return {"frac_burst": round(tflops / pk["bf16_tflops"], 4),
+            "frac_sustained": round(tflops / pk["bf16_tflops_sustained"], 4),
+            "frac_nominal": round(tflops / NOMINAL_BF16_TFLOPS, 4)}
+
+
+def applicable_peak(job_ms, clocks):
+    """Which measured BF16 peak a kernel timed inside this job is held against: the sustained one if the job
+    ran for seconds or the clock record shows the power cap at work, else the burst one."""
+    capped = bool(clocks) and "sw_power_cap" in (clocks.get("reasons") or [])
+    if job_ms >= 1000.0 or capped:
+        return "bf16_tflops_sustained", "frac_sustained", \
+               "sustained (job of %.0f ms%s)" % (job_ms, ", sw_power_cap seen" if capped else "")
+    return "bf16_tflops", "frac_burst", "burst (job of %.1f ms, no power cap in the clock record)" % job_ms
 
 
 def peaks():
@@ -115,16 +164,21 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # the CPU oracle, timed (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
-def oracle_rate(rows: int, steps: int, warmup: int, seed: int = 0, tokens: int = T):
-    """Runs `warmup + steps` oracle steps on a sample of the layer (`rows` output rows, `tokens` tokens);
+def oracle_rate(rows: int, steps: int, warmup: int, seed: int = 0, tokens: int = T, layer=(O, K, T), block_index=None):
+    """Runs `warmup + steps` oracle steps on a sample of a layer (`rows` output rows, `tokens` tokens);
     returns (full-layer steps/s, seconds per sampled step, threads used).  A row sample is an exact
     sub-problem (the loss separates over rows); a token sample is a smaller calibration batch; the rate
-    is scaled by the work ratio (O/rows) * (T/tokens)."""
+    is scaled by the work ratio (O/rows) * (T/tokens).  layer = (O, K, T) of the full layer; block_index
+    selects the decoder-block input recipe instead of the down_proj one."""
     import numpy as np
 
     from oracle import faar_oracle as fo
     from paper_2603_22370_b200 import inputs
-    W, X = inputs.config2(seed, rows, K, tokens)
+    Of, Kf, Tf = layer
+    if block_index is None:
+        W, X = inputs.config2(seed, rows, Kf, tokens)
+    else:
+        W, X = inputs.block_linear(seed, block_index, rows, Kf, tokens)
     # the calibration batch is handed over in float64 once, so that a step's cost is the method's own
     # arithmetic on the sampled rows and scales with them
     X = X.astype(np.float64)
@@ -145,7 +199,26 @@ def oracle_rate(rows: int, steps: int, warmup: int, seed: int = 0, tokens: int =
         threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
         threads = len(os.sched_getaffinity(0))
-    return 1.0 / (dt * (O / rows) * (T / tokens)), dt, threads
+    return 1.0 / (dt * (Of / rows) * (Tf / tokens)), dt, threads
+
+
+def block_linears(config: int):
+    from paper_2603_22370_b200 import inputs
+    return inputs.LLAMA32_1B_BLOCK if config == 3 else inputs.QWEN3_1P7B_BLOCK
+
+
+def oracle_block_rate(config: int, rows: int, steps: int, warmup: int, tokens: int = T):
+    """Block steps/s of the oracle: one sampled linear (k_proj's shape: K = 2048) timed, the block's seven
+    linears scaled from it by their flop counts (4 T O K each).  Returns (rate, seconds per sampled step,
+    threads, description of the sample)."""
+    lin = block_linears(config)
+    name, Ok, Kk = lin[1]
+    rate_k, dt, threads = oracle_rate(min(rows, Ok), steps, warmup, tokens=tokens, layer=(Ok, Kk, T), block_index=1)
+    flops_k = 4.0 * T * Ok * Kk
+    flops_block = sum(4.0 * T * o * k for _, o, k in lin)
+    sample = f"each step = {min(rows, Ok)} of {Ok} output rows of the {name} shape ({Ok}x{Kk}) on {tokens} of {T} tokens; " \
+             f"scaled to the layer by rows and tokens, then to the block's seven linears by flop count (x{flops_block / flops_k:.1f})"
+    return rate_k * flops_k / flops_block, dt, threads, sample
 
 
 def run_reference(args):
@@ -155,21 +228,28 @@ def run_reference(args):
     # size the sample (rows x tokens) so that warmup + steps finish in about two minutes
     budget = 120.0 / (args.steps + args.warmup)
     rows, tokens = 256, T
+    block = args.config in (3, 4)
+
+    def probe(r, tk, st, wu):
+        if block:
+            return oracle_block_rate(args.config, r, st, wu, tokens=tk)
+        rate, dt, th = oracle_rate(r, st, wu, tokens=tk)
+        return rate, dt, th, f"each step = {r} of {O} output rows (exact sub-problem: the loss separates over rows) on " \
+                             f"{tk} of {T} tokens, K={K}; rate scaled by the work ratio {O}/{r} x {T}/{tk}"
+
     while True:
-        _, dt_probe, _ = oracle_rate(rows, 1, 1, tokens=tokens)
+        _, dt_probe, _, _ = probe(rows, tokens, 1, 1)
         if dt_probe <= budget or (rows <= 16 and tokens <= 128):
             break
         if rows > 16:
             rows //= 2
         else:
             tokens //= 2
-    rate, dt, threads = oracle_rate(rows, args.steps, args.warmup, tokens=tokens)
-    sample = f"each step = {rows} of {O} output rows (exact sub-problem: the loss separates over rows) on {tokens} of " \
-             f"{T} tokens, K={K}; rate scaled by the work ratio {O}/{rows} x {T}/{tokens}"
+    rate, dt, threads, sample = probe(rows, tokens, args.steps, args.warmup)
     line = {"impl": "reference", "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / rate, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "O": O, "K": K, "T": T},
+            "config": workload_config(args.config),
             "cpu_baseline": {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": rate, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -177,34 +257,229 @@ def run_reference(args):
     return 0
 
 
+def workload_config(config: int):
+    """The `config` object both arms print: the workload and its sizes, nothing else."""
+    l2 = "no flush: one step touches about 410 MB (X, X^T, V, m, u, W_soft, Y_ref, dY^T, codes), more than the 126 MB L2"
+    if config == 2:
+        return {"workload": WORKLOAD, "O": O, "K": K, "T": T, "l2": l2,
+                "timed_region": "softquant_init + K x layer_step + harden_pack, inputs resident in HBM"}
+    return {"workload": BLOCK_WORKLOADS[config], "T": T,
+            "linears": {name: [o, k] for name, o, k in block_linears(config)},
+            "l2": "no flush: every step takes the next 4096-row minibatch of a calibration set larger than the 126 MB L2 "
+                  "(the k/v/q/o linears' per-step state alone is below it and is re-read from L2, as it would be in use)",
+            "timed_region": "per linear: softquant_init + K x layer_step (minibatches round-robin) + harden_pack; "
+                            "calibration set, its transposes and the frozen targets resident in HBM"}
+
+
 # ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
+class Runtime:
+    """Process-wide set-up shared by the layer and the block benchmark: one rank per GPU, the library built
+    and loaded, a context on its own stream, the clock sampler, and the timing rule (barrier + synchronise on
+    both sides, CUDA events on the launching stream, max over ranks)."""
+
+    def __init__(self, args):
+        import torch
+
+        from paper_2603_22370_b200 import build as faar_build
+        from paper_2603_22370_b200 import faar
+        self.torch, self.faar = torch, faar
+        self.rank, self.local_rank, self.world = dist_env()
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            self.dist = dist
+            torch.cuda.set_device(self.local_rank)
+            dist.init_process_group("nccl", device_id=torch.device(f"cuda:{self.local_rank}"))
+        self.dev = self.local_rank if self.world > 1 else 0
+        torch.cuda.set_device(self.dev)
+        self.device = f"cuda:{self.dev}"
+        if self.rank == 0:
+            faar_build.build()
+        if self.world > 1:
+            self.dist.barrier()
+        faar.lib()                                     # raises if libfaar.so is missing: no fallback
+        self.stream = torch.cuda.Stream(device=self.device)
+        self.ctx = faar.Context(self.dev, self.stream)
+        self.sampler = ClockSampler(self.dev) if self.rank == 0 else None
+
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.world > 1:
+            self.dist.barrier()
+            self.torch.cuda.synchronize()
+
+    def timed(self, fn):
+        """device time (ms) of fn() on the stream, max over ranks, with a barrier + sync on both sides"""
+        from paper_2603_22370_b200 import shard
+        torch = self.torch
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0 = time.time()
+        with torch.cuda.stream(self.stream):
+            e0.record(self.stream)
+            fn()
+            e1.record(self.stream)
+        self.stream.synchronize()
+        self.barrier()
+        w1 = time.time()
+        _, ms = shard.job_rate(1.0, e0.elapsed_time(e1), self.device)     # max over ranks
+        if self.sampler:
+            self.sampler.window(w0, w1)
+        return ms
+
+    def finish(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
+def run_block(args, rt):
+    """--config 3 / 4: the seven linears of one decoder block through the package's Stage-1 driver."""
+    import numpy as np
+
+    from paper_2603_22370_b200 import inputs, stage1
+    torch, faar, ctx, stream, device = rt.torch, rt.faar, rt.ctx, rt.stream, rt.device
+    steps, warmup = args.steps, max(args.warmup, 3)
+    lin = block_linears(args.config)
+    n_tok = args.calib_tokens
+    hid = 2048
+    ffn = dict((n, o) for n, o, k in lin)["gate_proj"]
+    rng_seed = 100 + rt.rank                                        # each rank its own block
+
+    # ---- synthetic block: weights, hidden states (input of q, k, v, gate, up), o_proj's input
+    with torch.cuda.stream(stream):
+        Wd = {}
+        for i, (name, o, k) in enumerate(lin):
+            Wn, _ = inputs.block_linear(rng_seed, i, o, k, 8)
+            Wd[name] = torch.from_numpy(Wn).to(device).to(torch.bfloat16)
+        streams = inputs._streams(rng_seed + 1000, 2)
+        H = torch.from_numpy(inputs.to_bf16_f32(inputs.hidden_states(streams[0], n_tok, hid))).to(device).to(torch.bfloat16)
+        Ho = torch.from_numpy(inputs.to_bf16_f32(inputs.hidden_states(streams[1], n_tok, hid, rms_norm=False))).to(device).to(torch.bfloat16)
+        A = stage1.mlp_activation(ctx, Wd["gate_proj"], Wd["up_proj"], H, T)
+    stream.synchronize()
+    Xin = {name: (A if name == "down_proj" else (Ho if name == "o_proj" else H)) for name, _, _ in lin}
+
+    per_linear, total_ms, launches = {}, 0.0, 0
+    e2e_ms, e2e_steps = 0.0, min(steps, 100)
+    h2d_total = 0
+    for name, o, k in lin:
+        with torch.cuda.stream(stream):
+            lay = stage1.StreamedLayer(ctx, Wd[name], Xin[name], T)
+
+        def job(n):
+            faar.softquant_init(ctx, lay.shape, lay.W, 0.0, lay.scales, lay.s_global, lay.code, lay.V, lay.ws)
+            lay.m.zero_()
+            lay.u.zero_()
+            for t in range(n):
+                lay.step(t, n, chain=args.chain)
+            packed = torch.empty((o, k // 2), dtype=torch.uint8, device=device)
+            faar.harden_pack(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, packed, None, None, None)
+
+        with torch.cuda.stream(stream):
+            job(warmup)
+        stream.synchronize()
+        ms = rt.timed(lambda: job(steps))
+        faar.check_status(ctx, lay.ws)
+
+        def profiled():
+            faar.profile_begin(ctx)
+            job(steps)
+
+        rt.timed(profiled)
+        prof = faar.profile_end(ctx)
+        bn, pairs = faar.last_gemm_config(ctx)
+        us = {kname: 1e3 * v[1] / v[0] for kname, v in prof.items()}
+        flops = 2.0 * T * o * k
+        per_linear[name] = {"O": o, "K": k, "ms_per_step": round(ms / steps, 5),
+                            "step_tflops": round(2 * flops * steps / (ms * 1e-3) / 1e12, 1),
+                            "kernels_us": {kn: round(v, 2) for kn, v in us.items()},
+                            "gemm_fwd_tflops": round(flops / (us["gemm_fwd"] * 1e-6) / 1e12, 1),
+                            "gemm_bwd_tflops": round(flops / (us["gemm_bwd"] * 1e-6) / 1e12, 1),
+                            "bwd_tile_n": bn, "bwd_cta_pairs": pairs, "job_ms": ms, "final_loss": lay.loss.tolist()}
+        total_ms += ms
+        launches += 2 + (1 + 2 * steps if args.chain else 3 * steps) + 1
+
+        # end to end for this linear: every step's minibatch arrives from pinned host memory
+        if not args.quick:
+            Xh = lay.X[0].cpu().pin_memory()
+            loss_h = torch.zeros(2, dtype=torch.float32).pin_memory()
+            sets = [(torch.empty_like(lay.X[0]), torch.empty_like(lay.Xt[0]), torch.empty_like(lay.Yref[0])) for _ in range(2)]
+
+            def e2e_job(n):
+                faar.softquant_init(ctx, lay.shape, lay.W, 0.0, lay.scales, lay.s_global, lay.code, lay.V, lay.ws)
+                lay.m.zero_()
+                lay.u.zero_()
+                for t in range(n):
+                    hp = faar.make_hparams(beta=beta_at(t, n), step=t + 1)
+                    Xd, Xtd, Yd = sets[t & 1]
+                    faar.layer_step_host(ctx, lay.shape, hp, Xh, None, lay.W, Xd, Xtd, Yd, lay.V, lay.code, lay.scales,
+                                         lay.s_global, lay.m, lay.u, lay.loss, loss_h, lay.ws)
+
+            with torch.cuda.stream(stream):
+                e2e_job(3)
+            stream.synchronize()
+            e2e_ms += rt.timed(lambda: e2e_job(e2e_steps))
+            h2d_total += T * k * 2
+            faar.check_status(ctx, lay.ws)
+        del lay
+        torch.cuda.empty_cache()
+
+    clocks = rt.sampler.stop() if rt.sampler else None
+    if rt.rank != 0:
+        rt.finish()
+        return 0
+    pk, pk_kind = peaks()
+    longest = max(v["job_ms"] for v in per_linear.values())
+    peak_key, frac_key, peak_why = applicable_peak(longest, clocks)
+    for v in per_linear.values():
+        for g in ("gemm_fwd", "gemm_bwd"):
+            v[g + "_frac"] = tensor_fracs(v[g + "_tflops"], pk)
+        v["step_frac"] = tensor_fracs(v["step_tflops"], pk)
+    value = rt.world * steps / (total_ms * 1e-3)
+    block_flops = sum(4.0 * T * o * k for _, o, k in lin)
+    # dominant kernel over the block: the launches of one GEMM kind that take the most time in a block step
+    tot = {g: sum(v["kernels_us"][g] for v in per_linear.values()) for g in ("gemm_fwd", "gemm_bwd")}
+    dominant = max(tot, key=tot.get)
+    dom_tf = (block_flops / 2.0) / (tot[dominant] * 1e-6) / 1e12
+    roofline = {"kernel": dominant + " (the seven linears' launches of one block step together)", "bound": "tensor",
+                "achieved": round(dom_tf, 1), "peak": pk[peak_key], "unit": "TFLOP/s",
+                "frac": tensor_fracs(dom_tf, pk)[frac_key], **tensor_fracs(dom_tf, pk), "traffic": None,
+                "peak_source": f"{pk_kind} {peak_key}: {peak_why}",
+                "timed": "per-kernel CUDA events on the launching stream, second pass of each linear's K-step job"}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warmup,
+            "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": workload_config(args.config),
+            "calibration_tokens": n_tok, "chained_soft_weights": bool(args.chain), "clocks": clocks,
+            "gpu_launches": launches, "roofline": roofline,
+            "block_step_tflops": round(block_flops * steps / (total_ms * 1e-3) / 1e12, 1),
+            "block_step_frac": tensor_fracs(block_flops * steps / (total_ms * 1e-3) / 1e12, pk),
+            "linears": per_linear}
+    if not args.quick:
+        line["e2e"] = {"value": rt.world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                       "h2d_bytes_per_step": h2d_total, "d2h_bytes_per_step": 8 * len(lin),
+                       "path": "faar_layer_step_host per linear: the minibatch copied in from pinned memory on a copy stream, "
+                               "X^T and the frozen target rebuilt on the device, step, losses copied out"}
+        cpu_rate, cpu_dt, cpu_threads, sample = oracle_block_rate(args.config, 128, 4, 1)
+        line["cpu_baseline"] = {"value": cpu_rate, "unit": UNIT, "cores": cpu_threads, "kind": "oracle", "sample": sample}
+    print(json.dumps(line))
+    rt.finish()
+    return 0
+
+
 def run_ours(args):
     import numpy as np
     import torch
 
-    from paper_2603_22370_b200 import build as faar_build
-    from paper_2603_22370_b200 import faar, inputs, shard
+    from paper_2603_22370_b200 import faar, inputs
 
-    rank, local_rank, world = dist_env()
+    rt = Runtime(args)
+    if args.config in (3, 4):
+        return run_block(args, rt)
+    rank, world, dev, device, dist = rt.rank, rt.world, rt.dev, rt.device, rt.dist
     n_gpus = args.gpus
-    if world > 1:
-        import torch.distributed as dist
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
-    dev = local_rank if world > 1 else 0
-    torch.cuda.set_device(dev)
-    device = f"cuda:{dev}"
-    if rank == 0:
-        faar_build.build()
-    if world > 1:
-        dist.barrier()
-    faar.lib()                                         # raises if libfaar.so is missing: no fallback
-
     steps, warmup = args.steps, max(args.warmup, 3)
-    stream = torch.cuda.Stream(device=device)
-    ctx = faar.Context(dev, stream)
+    stream, ctx = rt.stream, rt.ctx
 
     # ---- inputs, resident in HBM (each rank its own layer: seed = rank)
     Wn, Xn = inputs.config2(rank, O, K, T)
@@ -249,30 +524,7 @@ def run_ours(args):
             faar.layer_step(ctx, shape, hp, X, Xt, Yref, V, code, scales, s_global, m, u, loss, ws)
         faar.harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, None, None)
 
-    sampler = ClockSampler(dev) if rank == 0 else None
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    def timed(fn):
-        """device time (ms) of fn() on `stream`, max over ranks, with a barrier + sync on both sides"""
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        w0 = time.time()
-        with torch.cuda.stream(stream):
-            e0.record(stream)
-            fn()
-            e1.record(stream)
-        stream.synchronize()
-        barrier()
-        w1 = time.time()
-        _, ms = shard.job_rate(1.0, e0.elapsed_time(e1), device)     # max over ranks
-        if sampler:
-            sampler.window(w0, w1)
-        return ms
+    sampler, barrier, timed = rt.sampler, rt.barrier, rt.timed
 
     # ---- warm-up, then the timed job
     with torch.cuda.stream(stream):
@@ -375,13 +627,16 @@ def run_ours(args):
             dist.destroy_process_group()
         return 0
 
-    # ---- end to end: the calibration batch comes from pinned host memory every step
+    # ---- end to end: the calibration batch comes from pinned host memory every step; its frozen target is
+    # formed on the device from the copied batch (Procedure step 8) rather than shipped
     Xh = torch.from_numpy(Xn).to(torch.bfloat16).pin_memory()
-    Yh = Yref.cpu().pin_memory()
     loss_h = torch.zeros(2, dtype=torch.float32).pin_memory()
     # two staging sets, used alternately: the copy of batch t+1 overlaps step t
     stage_sets = [(torch.empty_like(X), torch.empty_like(Xt), torch.empty_like(Yref)) for _ in range(2)]
     e2e_steps = min(steps, 200)
+    h2d_bytes = T * K * 2
+    e2e_path = "faar_layer_step_host: pinned X copied in on a copy stream (two staging sets, the copy of batch t+1 " \
+               "overlaps step t), X^T and the frozen target Y_ref = X W^T rebuilt on the device, step, losses copied out"
 
     def e2e_job(n):
         m.zero_()
@@ -390,7 +645,7 @@ def run_ours(args):
         for t in range(n):
             hp = faar.make_hparams(beta=beta_at(t, n), step=t + 1, **chain_kw(t, n))
             X_dev, Xt_dev, Y_dev = stage_sets[t & 1]
-            faar.layer_step_host(ctx, shape, hp, Xh, Yh, X_dev, Xt_dev, Y_dev, V, code, scales, s_global, m, u,
+            faar.layer_step_host(ctx, shape, hp, Xh, None, W, X_dev, Xt_dev, Y_dev, V, code, scales, s_global, m, u,
                                  loss, loss_h, ws)
         faar.harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, None, None)
 
@@ -411,6 +666,7 @@ def run_ours(args):
     pk, pk_kind = peaks()
     n_w = O * K
     flops = 2.0 * T * O * K
+    peak_key, frac_key, peak_why = applicable_peak(ms_job, clocks)
 
     def avg_us(name):
         return 1e3 * prof[name][1] / prof[name][0] if name in prof else None
@@ -425,18 +681,21 @@ def run_ours(args):
     ]:
         if bound == "tensor":
             us = avg_us(name)
-            ach, peak, unit = work / (us * 1e-6) / 1e12, pk["bf16_tflops_sustained"], "TFLOP/s"
-            how = "CUDA events around each launch inside the K-step job"
+            ach = work / (us * 1e-6) / 1e12
+            kernels[name] = {"avg_us": round(us, 2), "bound": bound, "achieved": round(ach, 1), "peak": pk[peak_key],
+                             "unit": "TFLOP/s", "frac": tensor_fracs(ach, pk)[frac_key], **tensor_fracs(ach, pk),
+                             "timed": "CUDA events around each launch inside the K-step job"}
         else:
             # HBM-bound kernels: timed alone, launches back to back over rotated buffers (cold L2)
             us = ew_us[name]
-            ach, peak, unit = work / (us * 1e-6) / 1e9, pk["hbm_gbs"], "GB/s"
-            how = "30 back-to-back launches over 3 rotated buffer sets, one event pair"
-        kernels[name] = {"avg_us": round(us, 2), "bound": bound, "achieved": round(ach, 1), "peak": peak, "unit": unit,
-                         "frac": round(ach / peak, 4), "timed": how}
-    kernels["layer_dx"] = {"avg_us": round(dx_us, 2), "bound": "tensor", "achieved": round(flops / (dx_us * 1e-6) / 1e12, 1),
-                           "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                           "frac": round(flops / (dx_us * 1e-6) / 1e12 / pk["bf16_tflops_sustained"], 4),
+            ach = work / (us * 1e-6) / 1e9
+            kernels[name] = {"avg_us": round(us, 2), "bound": bound, "achieved": round(ach, 1), "peak": pk["hbm_gbs"],
+                             "unit": "GB/s", "frac": round(ach / pk["hbm_gbs"], 4),
+                             "timed": "30 back-to-back launches over 3 rotated buffer sets, one event pair"}
+    dx_tf = flops / (dx_us * 1e-6) / 1e12
+    kernels["layer_dx"] = {"avg_us": round(dx_us, 2), "bound": "tensor", "achieved": round(dx_tf, 1),
+                           "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": tensor_fracs(dx_tf, pk)["frac_burst"],
+                           **tensor_fracs(dx_tf, pk),
                            "timed": "20 back-to-back calls (soft weights, transpose and GEMM each), one event pair",
                            "note": "input gradient dX = dY W_soft, not part of a Stage-1 step"}
     al_bytes = 3.0 * AL_T * AL_V * 2 + 3.0 * AL_T * AL_D * 2          # both logit / hidden tensors read, one gradient written
@@ -445,16 +704,17 @@ def run_ours(args):
                              "frac": round(al_bytes / (al_us * 1e-6) / 1e9 / pk["hbm_gbs"], 4),
                              "timed": f"5 back-to-back calls on {AL_T} tokens x 128256 logits (+ 2048 hidden), one event pair",
                              "note": "Eq. 6's KL and last-hidden terms with gradients; not part of a Stage-1 step"}
-    kernels["softquant_init"]["note"] = "amax pass + bracket pass together; the amax pass re-reads W (+2 B/weight, not " \
-                                        "counted); the bracket pass is bound by its IEEE divisions, not by HBM"
+    kernels["softquant_init"]["note"] = "amax pass + bracket pass together; the amax pass re-reads W (+2 B/weight, not counted)"
     for name in prof:
         kernels.setdefault(name, {})["in_job_avg_us"] = round(avg_us(name), 2)
         kernels[name]["launches"] = prof[name][0]
     dominant = max(("gemm_fwd", "gemm_bwd"), key=lambda k: prof[k][1])
     d = kernels[dominant]
     roofline = {"kernel": dominant, "bound": "tensor", "achieved": d["achieved"], "peak": d["peak"],
-                "unit": "TFLOP/s", "frac": d["frac"], "traffic": NCU_TRAFFIC_BYTES.get(dominant),
-                "peak_source": f"{pk_kind} bf16_tflops_sustained (kernel timed inside a long step)",
+                "unit": "TFLOP/s", "frac": d["frac"], "frac_burst": d["frac_burst"],
+                "frac_sustained": d["frac_sustained"], "frac_nominal": d["frac_nominal"],
+                "traffic": ncu_traffic(dominant),
+                "peak_source": f"{pk_kind} {peak_key}: {peak_why}",
                 "timed": "per-kernel CUDA events on the launching stream, second pass of the same K-step job"}
 
     # ---- CPU oracle beside it (bounded sample)
@@ -466,17 +726,12 @@ def run_ours(args):
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": n_gpus, "steps": steps, "warmup": warmup,
             "ms_per_step": ms_job / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "O": O, "K": K, "T": T,
-                       "l2": "no flush: one step touches about 410 MB (X, X^T, V, m, u, W_soft, Y_ref, dY^T, codes), "
-                             "more than the 126 MB L2",
-                       "timed_region": "softquant_init + K x layer_step + harden_pack, inputs resident in HBM",
-                       "chained_soft_weights": bool(args.chain)},
+            "dtype": "bf16", "data": "synthetic", "config": workload_config(2),
+            "chained_soft_weights": bool(args.chain),
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
-                    "h2d_bytes_per_step": T * K * 2 + T * O * 2, "d2h_bytes_per_step": 8,
-                    "path": "faar_layer_step_host: pinned X and Y_ref copied in on a copy stream (two staging sets, the copy of "
-                            "batch t+1 overlaps step t), X^T rebuilt, step, losses copied out"},
+                    "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": 8,
+                    "path": e2e_path},
             "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "kernels": kernels, "final_loss": loss_final,
             "step_tflops": round(2 * flops * steps / (ms_job * 1e-3) / 1e12, 1)}
@@ -492,6 +747,11 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
+                    help="2: the down_proj-shaped layer (the headline); 3 / 4: the seven linears of a Llama-3.2-1B- / "
+                         "Qwen3-1.7B-shaped decoder block")
+    ap.add_argument("--calib-tokens", type=int, default=65536,
+                    help="rows of the synthetic calibration set of --config 3 / 4 (4096-row minibatches, round-robin)")
     ap.add_argument("--align-tokens", type=int, default=4096,
                     help="tokens of the alignment-loss timing (128256 logits each); smaller for profiler captures")
     ap.add_argument("--chain", action="store_true",

@@ -23,7 +23,17 @@
  *   - The tensor-core kernels bound every wait on a barrier.  If a wait gives
  *     up, the kernel records a code in the workspace status word, releases its
  *     tensor memory and returns; faar_check_status reports it as
- *     FAAR_ERR_TIMEOUT after the caller has synchronised the stream.
+ *     FAAR_ERR_TIMEOUT after the caller has synchronised the stream.  The
+ *     status word is sticky and the workspace's counters may be left half
+ *     updated: after FAAR_ERR_TIMEOUT call faar_workspace_init before the
+ *     workspace is used again (results of the call that timed out are invalid).
+ *   - The soft weights of Eq. 2 are not generated inside the forward GEMM:
+ *     each step a separate kernel (or the previous step's backward epilogue,
+ *     see faar_hparams.beta_next) writes them once as a BF16 operand [O,K] into
+ *     the workspace, and the forward GEMM reads that operand by TMA.  Generating
+ *     the operand inside the GEMM would re-evaluate Eq. 3 once per token tile
+ *     (T/256 times per weight), which costs more than the 2 bytes per weight of
+ *     the round trip.
  *
  * Packed formats
  *   code   [O, K/2] u8: element 2j in bits 3:0, element 2j+1 in bits 7:4 of byte j;
@@ -52,7 +62,8 @@ extern "C" {
 enum {
   FAAR_OK = 0,
   FAAR_ERR_INVALID_ARG = 1, /* null pointer, bad enum, bad hyper-parameter      */
-  FAAR_ERR_SHAPE = 2,       /* O/K/T <= 0, K % 16 != 0, leading dim too small   */
+  FAAR_ERR_SHAPE = 2,       /* O/K/T <= 0, K % 16 != 0, leading dim too small,
+                               K > 268 435 455 in the backward / step calls      */
   FAAR_ERR_ALIGN = 3,       /* pointer not 16-byte aligned / ld not multiple of 8 */
   FAAR_ERR_DTYPE = 4,
   FAAR_ERR_WORKSPACE = 5,   /* workspace null, misaligned or too small          */
@@ -66,7 +77,10 @@ typedef struct faar_ctx faar_ctx;
 typedef enum { FAAR_BF16 = 0, FAAR_F32 = 1 } faar_dtype;
 
 /* Hyper-parameters of one step (host struct, by pointer, read at call time).
- * beta: temperature of Eq. 3.  lambda_round: weight of the Round Loss in Eq. 5.
+ * beta: temperature of Eq. 3, 0 < beta <= 1024 in the forward / backward / step calls (the BF16
+ *   operand is rounded from an FP32 evaluation of Eq. 2/3 whose relative error is at most
+ *   6e-7 + 7.5e-8 beta: 3e-6 at beta = 32; beyond 1024 Eq. 3 is a step function at BF16 precision and
+ *   the hardened weights are the thing to use).  lambda_round: weight of the Round Loss in Eq. 5.
  * mse_scale: factor c on the squared Frobenius norm (the paper's Eq. 5 has c = 1).
  * opt: 0 = gradient descent, 1 = Adam (bias-corrected, no weight decay).
  * step: 1-based step index (Adam bias correction). */
@@ -87,6 +101,9 @@ typedef struct {
    * wsoft_ready != 0: the caller states that the previous backward (or step) call on this workspace
    *   was given beta_next == this step's beta and that V has not been touched since; the forward pass
    *   then reads that operand instead of rebuilding it from V (the soft-weights kernel is skipped).
+   *   The context remembers the workspace and beta_next of its last backward call: wsoft_ready with
+   *   another workspace or another beta is refused with FAAR_ERR_INVALID_ARG (a V that the caller
+   *   changed in between cannot be detected).
    * The values, and so every result, are the same bit for bit either way. */
   float beta_next;
   int wsoft_ready;
@@ -173,7 +190,8 @@ enum {
   FAAR_K_TRANSPOSE = 9,
   FAAR_K_ACT_FAKEQUANT = 10, /* activations to NVFP4 values (the X_q of Eq. 5)          */
   FAAR_K_ALIGN_LOSS = 11,    /* Eq. 6: KL of the softmaxes + last-hidden error, gradients */
-  FAAR_K_COUNT = 12
+  FAAR_K_GLUE = 12,          /* element-wise pieces of a decoder block between the linears */
+  FAAR_K_COUNT = 13
 };
 typedef struct {
   int kernel;     /* one of FAAR_K_*          */
@@ -210,6 +228,14 @@ FAAR_API int faar_softquant_init(faar_ctx* ctx, const faar_shape* shape, const v
 FAAR_API int faar_softquant_eval(faar_ctx* ctx, const faar_shape* shape, const float* V, const uint8_t* code,
                         const uint8_t* scales, const float* s_global, float beta,
                         float* W_soft, float* h, void* W_soft_bf16);
+
+/* Debug view of the forward GEMM's operand (no counterpart in the paper): the FP32 value of Eq. 2 that
+ * the soft-weights kernel and the chained backward epilogue round to BF16, before that rounding.  It
+ * comes from a cheaper evaluation of Eq. 3 than W_soft above (one FMA for the exponent, hardware 2^x and
+ * reciprocal); its relative error against the exact value is at most 6e-7 + 7.5e-8 beta.
+ *   W_operand out: [O,K] float */
+FAAR_API int faar_softquant_operand_f32(faar_ctx* ctx, const faar_shape* shape, const float* V, const uint8_t* code,
+                                        const uint8_t* scales, const float* s_global, float beta, float* W_operand);
 
 /* ---- layout helper ----------------------------------------------------------
  * out[c, r] = in[r, c] for a BF16 matrix in[rows, cols] (ld_in) -> out[cols, rows]
@@ -263,6 +289,17 @@ FAAR_API int faar_layer_dx(faar_ctx* ctx, const faar_shape* shape, float beta, c
                            const uint8_t* code, const uint8_t* scales, const float* s_global, void* WsoftT,
                            void* dX, void* workspace, size_t workspace_bytes);
 
+/* ---- the MLP's gated product ---------------------------------------------------
+ * Procedure step 1 runs Stage 1 "for each layer": the input of a block's down
+ * projection is the frozen model's own activation silu(H W_gate^T) * (H W_up^T),
+ * silu(x) = x / (1 + e^-x).  This call forms it from the two GEMM outputs
+ * (faar_layer_ref) so that the calibration input never leaves the device.  FP32
+ * arithmetic, BF16 in and out.
+ *   gate, up in: [rows, cols] bf16 (ldg, ldu)     out: [rows, cols] bf16 (ldo); may alias gate or up
+ * cols and the leading dimensions are multiples of 8, the bases 16-byte aligned. */
+FAAR_API int faar_silu_mul(faar_ctx* ctx, int rows, int cols, const void* gate, int64_t ldg, const void* up,
+                           int64_t ldu, void* out, int64_t ldo);
+
 /* ---- part 4: Round Loss, backward, update -----------------------------------
  * Eq. 5, second term without lambda: L_round = (1/N) sum (1 - (2v-1)^2).
  *   V in: N floats     loss_round out: 1 float (device) */
@@ -314,11 +351,17 @@ FAAR_API int faar_layer_step(faar_ctx* ctx, const faar_shape* shape, const faar_
                     float* loss_out2, void* workspace, size_t workspace_bytes);
 
 /* faar_layer_step for a calibration batch that lives in HOST memory (ideally
- * pinned): copies X_host[T,K] (ldx) and Y_ref_host[T,O] (ldy) into the caller's
- * device staging buffers X_dev / Yref_dev, rebuilds Xt_dev = X^T [K, ldxt],
- * runs the step, and copies {L_MSE, L_round} back to loss_host2.  Everything
- * is ordered with the context's stream; loss_host2 is valid after the caller
- * synchronises it.  Bytes moved: T*K*2 + T*O*sizeof(yref_dtype) in, 8 out.
+ * pinned): copies X_host[T,K] (ldx) and Y_ref_host (the layout the shape declares)
+ * into the caller's device staging buffers X_dev / Yref_dev, rebuilds
+ * Xt_dev = X^T [K, ldxt], runs the step, and copies {L_MSE, L_round} back to
+ * loss_host2.  Y_ref_host may be null: the batch's frozen target is then computed
+ * on the device from the copied X and the layer's original BF16 weights W [O,K]
+ * (ldw; Procedure step 8, as faar_layer_ref) instead of crossing the bus, and W
+ * must be given; with Y_ref_host given W is not read and may be null.
+ * Everything is ordered with the context's stream; loss_host2 is valid after the
+ * caller synchronises it.  Bytes moved: T*K*2 (+ T*O*sizeof(yref_dtype) with
+ * Y_ref_host) in, 8 out.  Every argument is validated before the first copy is
+ * enqueued, so a refused call leaves the staging buffers untouched.
  * The host-to-device copies run on a copy stream that the context creates on
  * the first call (with three events: host resources, no device memory).  A
  * caller that alternates between two sets of staging buffers (X_dev, Xt_dev,
@@ -326,8 +369,8 @@ FAAR_API int faar_layer_step(faar_ctx* ctx, const faar_shape* shape, const faar_
  * n; with a single set the copy waits for the previous step.  After a change of
  * the context's stream (faar_set_stream) synchronise before the next call. */
 FAAR_API int faar_layer_step_host(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp,
-                                  const void* X_host, const void* Y_ref_host, void* X_dev, void* Xt_dev,
-                                  void* Yref_dev, float* V, const uint8_t* code, const uint8_t* scales,
+                                  const void* X_host, const void* Y_ref_host, const void* W, void* X_dev,
+                                  void* Xt_dev, void* Yref_dev, float* V, const uint8_t* code, const uint8_t* scales,
                                   const float* s_global, float* adam_m, float* adam_u, float* loss_dev2,
                                   float* loss_host2, void* workspace, size_t workspace_bytes);
 

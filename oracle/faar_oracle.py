@@ -421,6 +421,14 @@ def swizzle_scales(scales):
     return out
 
 
+def silu_mul(gate, up):
+    """The MLP's gated product of a Llama / Qwen decoder block: silu(g) * u with silu(x) = x / (1 + e^-x)
+    (the frozen model's input of down_proj, which Stage 1 optimises "for each layer").  float64."""
+    g = np.asarray(gate, dtype=np.float64)
+    with np.errstate(over="ignore"):
+        return g / (1.0 + np.exp(-g)) * np.asarray(up, dtype=np.float64)
+
+
 def rtn_nearest(W, scales, s_global):
     """Round-to-nearest onto the node set, written independently of the
     bracket: argmin over all 8 nodes of |w~ - node|, a tie going to the larger

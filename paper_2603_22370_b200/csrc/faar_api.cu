@@ -15,11 +15,25 @@ int cuda_fail(faar_ctx* ctx, int e) {
   return FAAR_ERR_CUDA;
 }
 
+// Largest temperature the GEMM calls take: the BF16 operand's FP32 evaluation has a relative error of about
+// 6e-7 + 7.5e-8 beta, which at 1024 is still 25 times below the BF16 spacing.
+constexpr float FAAR_BETA_MAX = 1024.0f;
+
 int check_shape(const faar_shape* s) {
   if (!s) return FAAR_ERR_INVALID_ARG;
   if (s->O <= 0 || s->K <= 0 || s->T <= 0) return FAAR_ERR_SHAPE;
   if (s->K % 16 != 0) return FAAR_ERR_SHAPE;
   return FAAR_OK;
+}
+
+// The backward epilogue forms offsets of up to 7 rows of V in 32-bit element counts.
+int check_bwd_k(const faar_shape* s) { return (long long)s->K * 8 > 0x7FFFFFFFll ? FAAR_ERR_SHAPE : FAAR_OK; }
+
+// Chained steps: wsoft_ready is only honoured if the last backward call on this context wrote, into this
+// very workspace, the operand for this step's beta.
+int check_chain(const faar_ctx* ctx, const faar_hparams* hp, const void* ws) {
+  if (!hp->wsoft_ready) return FAAR_OK;
+  return (ctx->wsoft_ws == ws && ctx->wsoft_beta == hp->beta) ? FAAR_OK : FAAR_ERR_INVALID_ARG;
 }
 
 // Leading dimension of Y_ref / Y_q for the layout the shape declares.
@@ -40,10 +54,10 @@ int check_ws(const faar_shape* s, const void* ws, size_t ws_bytes) {
 
 int check_hp(const faar_hparams* hp, bool need_opt) {
   if (!hp) return FAAR_ERR_INVALID_ARG;
-  if (!(hp->beta > 0.f) || !isfinite(hp->beta) || !isfinite(hp->mse_scale) || !isfinite(hp->lambda_round))
+  if (!(hp->beta > 0.f) || !(hp->beta <= FAAR_BETA_MAX) || !isfinite(hp->mse_scale) || !isfinite(hp->lambda_round))
     return FAAR_ERR_INVALID_ARG;
   if (!(hp->act_scale >= 0.f) || !isfinite(hp->act_scale)) return FAAR_ERR_INVALID_ARG;
-  if (!(hp->beta_next >= 0.f) || !isfinite(hp->beta_next)) return FAAR_ERR_INVALID_ARG;
+  if (!(hp->beta_next >= 0.f) || !(hp->beta_next <= FAAR_BETA_MAX)) return FAAR_ERR_INVALID_ARG;
   if (need_opt) {
     if (hp->opt != 0 && hp->opt != 1) return FAAR_ERR_INVALID_ARG;
     if (!isfinite(hp->lr)) return FAAR_ERR_INVALID_ARG;
@@ -54,11 +68,21 @@ int check_hp(const faar_hparams* hp, bool need_opt) {
   return FAAR_OK;
 }
 
+// Makes the context's device current for the duration of a call.  err != 0: the switch failed and
+// nothing may be launched.
 struct DeviceGuard {
   int prev = -1;
-  explicit DeviceGuard(int dev) { cudaGetDevice(&prev); if (prev != dev) cudaSetDevice(dev); else prev = -1; }
-  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+  int err = 0;
+  explicit DeviceGuard(int dev) {
+    cudaError_t e = cudaGetDevice(&prev);
+    if (e == cudaSuccess && prev != dev) e = cudaSetDevice(dev); else if (e == cudaSuccess) prev = -1;
+    if (e != cudaSuccess) { err = (int)e; prev = -1; }
+  }
+  ~DeviceGuard() { if (prev >= 0) (void)cudaSetDevice(prev); }
 };
+#define FAAR_DEVICE_GUARD(ctx)        \
+  DeviceGuard g((ctx)->device);       \
+  if (g.err) return cuda_fail((ctx), g.err)
 
 int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Y_ref,
              const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
@@ -110,6 +134,10 @@ int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
   if (hp->beta_next > 0.f) {
     a.wsoft_next = reinterpret_cast<__nv_bfloat16*>(ws + l.off_wsoft);
     a.beta_next = hp->beta_next;
+    ctx->wsoft_ws = ws;
+    ctx->wsoft_beta = hp->beta_next;
+  } else if (ctx->wsoft_ws == ws) {
+    ctx->wsoft_ws = nullptr;               // V moves on without a matching operand
   }
   a.act_scale = hp->act_scale > 0.f ? hp->act_scale : 1.0f;
   a.lam_over_n = (float)((double)hp->lambda_round / ((double)s->O * (double)s->K));
@@ -125,6 +153,28 @@ int check_gemm_operands(const faar_shape* s, bool need_x, bool need_xt) {
   if (need_x && (s->ldx < s->K || s->ldx % 8)) return s->ldx < s->K ? FAAR_ERR_SHAPE : FAAR_ERR_ALIGN;
   if (need_xt && (s->ldxt < s->T || s->ldxt % 8)) return s->ldxt < s->T ? FAAR_ERR_SHAPE : FAAR_ERR_ALIGN;
   return FAAR_OK;
+}
+
+// Everything faar_layer_step checks before it enqueues anything (also run by faar_layer_step_host before its
+// first copy, so that a refused call leaves the staging buffers and the copy stream untouched).
+int validate_step(const faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Xt,
+                  const void* Y_ref, const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global,
+                  const float* adam_m, const float* adam_u, const float* loss_out2, const void* workspace,
+                  size_t workspace_bytes) {
+  if (!ctx || !X || !Xt || !Y_ref || !V || !code || !scales || !s_global || !loss_out2) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if ((st = check_hp(hp, true))) return st;
+  if (hp->opt == 1 && (!adam_m || !adam_u)) return FAAR_ERR_INVALID_ARG;
+  if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
+  if ((st = check_bwd_k(s))) return st;
+  if ((st = check_ldy(s))) return st;
+  if ((st = check_gemm_operands(s, true, true))) return st;
+  if (!aligned16(X) || !aligned16(Xt) || !aligned16(V) || !aligned16(code) || (adam_m && !aligned16(adam_m)) ||
+      (adam_u && !aligned16(adam_u)))
+    return FAAR_ERR_ALIGN;
+  if ((st = check_ws(s, workspace, workspace_bytes))) return st;
+  return check_chain(ctx, hp, workspace);
 }
 
 }  // namespace
@@ -181,6 +231,9 @@ int faar_create(faar_ctx** out, int device, void* stream) {
   c->tune_bn = 0;
   c->tune_tail = -1;
   c->last_gemm_split = 0;
+  for (int i = 0; i < FAAR_GEMM_VARIANTS; ++i) c->gemm_max_pairs[i] = 0;
+  c->wsoft_ws = nullptr;
+  c->wsoft_beta = 0.f;
   c->copy_stream = nullptr;
   c->ev_copied = nullptr;
   c->ev_done[0] = c->ev_done[1] = nullptr;
@@ -226,6 +279,7 @@ const char* faar_kernel_name(int kernel) {
     case FAAR_K_TRANSPOSE: return "transpose";
     case FAAR_K_ACT_FAKEQUANT: return "act_fakequant";
     case FAAR_K_ALIGN_LOSS: return "align_loss";
+    case FAAR_K_GLUE: return "glue";
   }
   return "unknown";
 }
@@ -240,7 +294,7 @@ int faar_profile_begin(faar_ctx* ctx) {
 
 int faar_profile_end(faar_ctx* ctx, faar_kernel_time* out, int capacity, int* count) {
   if (!ctx || !out || !count || capacity < 0) return FAAR_ERR_INVALID_ARG;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   ctx->prof_on = false;
   *count = 0;
   cudaError_t e = cudaStreamSynchronize(ctx->stream);
@@ -312,13 +366,13 @@ int faar_workspace_init(faar_ctx* ctx, void* workspace, size_t workspace_bytes) 
   if (!ctx) return FAAR_ERR_INVALID_ARG;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
     return FAAR_ERR_WORKSPACE;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, (int)cudaMemsetAsync(workspace, 0, FAAR_WS_HEADER, ctx->stream));
 }
 
 int faar_check_status(faar_ctx* ctx, const void* workspace, uint32_t* detail_out) {
   if (!ctx || !workspace) return FAAR_ERR_INVALID_ARG;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   uint32_t word = 0;
   cudaError_t e = cudaStreamSynchronize(ctx->stream);
   if (e == cudaSuccess) e = cudaMemcpy(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost);
@@ -332,7 +386,7 @@ int faar_selftest_wait_timeout(faar_ctx* ctx, void* workspace, size_t workspace_
   if (limit_us == 0 || limit_us > 1000000u) return FAAR_ERR_INVALID_ARG;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
     return FAAR_ERR_WORKSPACE;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, faar_launch_wait_selftest(ctx, reinterpret_cast<uint32_t*>(workspace), 1000ull * limit_us));
 }
 
@@ -349,7 +403,7 @@ int faar_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float
   if (!isfinite(s_global_in) || s_global_in < 0.f) return FAAR_ERR_INVALID_ARG;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
     return FAAR_ERR_WORKSPACE;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   uint32_t* amax_word = reinterpret_cast<uint32_t*>(workspace) + 1;
   return cuda_fail(ctx, faar_launch_softquant_init(ctx, s, W, s_global_in, scales, s_global_out, code, V_init,
                                                    amax_word));
@@ -366,16 +420,28 @@ int faar_softquant_eval(faar_ctx* ctx, const faar_shape* s, const float* V, cons
       (W_soft_bf16 && !aligned16(W_soft_bf16)))
     return FAAR_ERR_ALIGN;
   if (!W_soft && !h && !W_soft_bf16) return FAAR_OK;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, beta, W_soft, h,
                                                    reinterpret_cast<__nv_bfloat16*>(W_soft_bf16)));
+}
+
+int faar_softquant_operand_f32(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
+                               const uint8_t* scales, const float* s_global, float beta, float* W_operand) {
+  if (!ctx || !V || !code || !scales || !s_global || !W_operand) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if (!(beta > 0.f) || !(beta <= FAAR_BETA_MAX)) return FAAR_ERR_INVALID_ARG;
+  if (!aligned16(V) || !aligned16(code) || !aligned16(W_operand)) return FAAR_ERR_ALIGN;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, beta, nullptr, nullptr, nullptr,
+                                                   W_operand));
 }
 
 int faar_transpose_bf16(faar_ctx* ctx, int rows, int cols, const void* in, int64_t ld_in, void* out,
                         int64_t ld_out) {
   if (!ctx || !in || !out) return FAAR_ERR_INVALID_ARG;
   if (rows <= 0 || cols <= 0 || ld_in < cols || ld_out < rows) return FAAR_ERR_SHAPE;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, faar_launch_transpose_bf16(ctx, rows, cols, in, ld_in, out, ld_out));
 }
 
@@ -389,7 +455,7 @@ int faar_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_t ldx, 
   if (!isfinite(s_global_in) || s_global_in < 0.f) return FAAR_ERR_INVALID_ARG;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
     return FAAR_ERR_WORKSPACE;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   uint32_t* amax_word = reinterpret_cast<uint32_t*>(workspace) + 1;
   return cuda_fail(ctx, faar_launch_act_fakequant(ctx, T, K, X, ldx, s_global_in, Xq_units, ldq, s_global_out, packed,
                                                   scales, amax_word));
@@ -408,7 +474,7 @@ int faar_layer_ref(faar_ctx* ctx, const faar_shape* s, const void* X, const void
   if (s->ldw % 8 || !aligned16(X) || !aligned16(W)) return FAAR_ERR_ALIGN;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
     return FAAR_ERR_WORKSPACE;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   faar_gemm_args a = {};
   a.mode = FAAR_GEMM_REF;
   a.M = s->O; a.N = s->T; a.Kc = s->K;
@@ -431,10 +497,11 @@ int faar_layer_dx(faar_ctx* ctx, const faar_shape* s, float beta, const void* dY
       !aligned16(dX))
     return FAAR_ERR_ALIGN;
   if ((st = check_ws(s, workspace, workspace_bytes))) return st;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const faar_ws_layout l = faar_ws_plan(s);
   __nv_bfloat16* wsoft = reinterpret_cast<__nv_bfloat16*>(ws + l.off_wsoft);
+  if (ctx->wsoft_ws == workspace) ctx->wsoft_ws = nullptr;     // the operand slot is overwritten below
   const int64_t ldo = ((int64_t)s->O + 7) / 8 * 8;
   int e = faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, beta, nullptr, nullptr, wsoft);
   if (e) return cuda_fail(ctx, e);
@@ -463,7 +530,8 @@ int faar_layer_fwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, c
   if ((st = check_gemm_operands(s, true, false))) return st;
   if (!aligned16(X) || !aligned16(V) || !aligned16(code) || !aligned16(dYt)) return FAAR_ERR_ALIGN;
   if ((st = check_ws(s, workspace, workspace_bytes))) return st;
-  DeviceGuard g(ctx->device);
+  if ((st = check_chain(ctx, hp, workspace))) return st;
+  FAAR_DEVICE_GUARD(ctx);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const faar_ws_layout l = faar_ws_plan(s);
   int np = 0;
@@ -482,7 +550,7 @@ int faar_round_loss(faar_ctx* ctx, const float* V, int64_t N, float* loss_round,
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
       workspace_bytes < FAAR_WS_HEADER + 2 * sizeof(float) * FAAR_MAX_PARTIALS)
     return FAAR_ERR_WORKSPACE;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   float* partials = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + FAAR_WS_HEADER +
                                              sizeof(float) * FAAR_MAX_PARTIALS);
   int np = 0;
@@ -500,12 +568,13 @@ int faar_layer_bwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, c
   if (st) return st;
   if ((st = check_hp(hp, true))) return st;
   if (hp->opt == 1 && (!adam_m || !adam_u)) return FAAR_ERR_INVALID_ARG;
+  if ((st = check_bwd_k(s))) return st;
   if ((st = check_gemm_operands(s, false, true))) return st;
   if (!aligned16(dYt) || !aligned16(Xt) || !aligned16(V) || !aligned16(code) || (adam_m && !aligned16(adam_m)) ||
       (adam_u && !aligned16(adam_u)) || (dV && !aligned16(dV)))
     return FAAR_ERR_ALIGN;
   if ((st = check_ws(s, workspace, workspace_bytes))) return st;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const faar_ws_layout l = faar_ws_plan(s);
   return cuda_fail(ctx, bwd_impl(ctx, s, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, dV, ws, l, nullptr));
@@ -514,19 +583,10 @@ int faar_layer_bwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, c
 int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Xt,
                     const void* Y_ref, float* V, const uint8_t* code, const uint8_t* scales, const float* s_global,
                     float* adam_m, float* adam_u, float* loss_out2, void* workspace, size_t workspace_bytes) {
-  if (!ctx || !X || !Xt || !Y_ref || !V || !code || !scales || !s_global || !loss_out2) return FAAR_ERR_INVALID_ARG;
-  int st = check_shape(s);
+  int st = validate_step(ctx, s, hp, X, Xt, Y_ref, V, code, scales, s_global, adam_m, adam_u, loss_out2, workspace,
+                         workspace_bytes);
   if (st) return st;
-  if ((st = check_hp(hp, true))) return st;
-  if (hp->opt == 1 && (!adam_m || !adam_u)) return FAAR_ERR_INVALID_ARG;
-  if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
-  if ((st = check_ldy(s))) return st;
-  if ((st = check_gemm_operands(s, true, true))) return st;
-  if (!aligned16(X) || !aligned16(Xt) || !aligned16(V) || !aligned16(code) || (adam_m && !aligned16(adam_m)) ||
-      (adam_u && !aligned16(adam_u)))
-    return FAAR_ERR_ALIGN;
-  if ((st = check_ws(s, workspace, workspace_bytes))) return st;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const faar_ws_layout l = faar_ws_plan(s);
   void* dYt = ws + l.off_dyt;
@@ -539,18 +599,22 @@ int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, 
 }
 
 int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X_host,
-                         const void* Y_ref_host, void* X_dev, void* Xt_dev, void* Yref_dev, float* V,
+                         const void* Y_ref_host, const void* W, void* X_dev, void* Xt_dev, void* Yref_dev, float* V,
                          const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
                          float* adam_u, float* loss_dev2, float* loss_host2, void* workspace,
                          size_t workspace_bytes) {
-  if (!ctx || !X_host || !Y_ref_host || !X_dev || !Xt_dev || !Yref_dev || !loss_dev2 || !loss_host2)
+  if (!ctx || !X_host || (!Y_ref_host && !W) || !X_dev || !Xt_dev || !Yref_dev || !loss_dev2 || !loss_host2)
     return FAAR_ERR_INVALID_ARG;
-  int st = check_shape(s);
+  // every check of the step itself, before the first copy is enqueued
+  int st = validate_step(ctx, s, hp, X_dev, Xt_dev, Yref_dev, V, code, scales, s_global, adam_m, adam_u, loss_dev2,
+                         workspace, workspace_bytes);
   if (st) return st;
-  if (s->yref_dtype != FAAR_BF16 && s->yref_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
-  if ((st = check_ldy(s))) return st;
-  if ((st = check_gemm_operands(s, true, true))) return st;
-  DeviceGuard g(ctx->device);
+  if (!Y_ref_host) {                             // what faar_layer_ref will ask of W
+    if (s->w_dtype != FAAR_BF16) return FAAR_ERR_DTYPE;
+    if (s->ldw < s->K) return FAAR_ERR_SHAPE;
+    if (s->ldw % 8 || !aligned16(W)) return FAAR_ERR_ALIGN;
+  }
+  FAAR_DEVICE_GUARD(ctx);
   cudaError_t e = cudaSuccess;
   if (!ctx->copy_stream) {                       // host resources of this path, created on first use
     e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
@@ -574,7 +638,7 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
   const size_t ybytes = s->yref_dtype == FAAR_BF16 ? 2 : 4;
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(X_dev, X_host, (size_t)s->T * (size_t)s->ldx * 2, cudaMemcpyHostToDevice, ctx->copy_stream);
-  if (e == cudaSuccess)
+  if (e == cudaSuccess && Y_ref_host)
     e = cudaMemcpyAsync(Yref_dev, Y_ref_host, (size_t)(s->yref_transposed ? s->O : s->T) * (size_t)s->ldy * ybytes,
                         cudaMemcpyHostToDevice,
                         ctx->copy_stream);
@@ -583,6 +647,10 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
   if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
   st = faar_transpose_bf16(ctx, s->T, s->K, X_dev, s->ldx, Xt_dev, s->ldxt);
   if (st) return st;
+  if (!Y_ref_host) {                             // the batch's frozen target from the X that has just arrived
+    st = faar_layer_ref(ctx, s, X_dev, W, Yref_dev, workspace, workspace_bytes);
+    if (st) return st;
+  }
   st = faar_layer_step(ctx, s, hp, X_dev, Xt_dev, Yref_dev, V, code, scales, s_global, adam_m, adam_u, loss_dev2,
                        workspace, workspace_bytes);
   if (st) return st;
@@ -591,13 +659,22 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
   return cuda_fail(ctx, (int)e);
 }
 
+int faar_silu_mul(faar_ctx* ctx, int rows, int cols, const void* gate, int64_t ldg, const void* up, int64_t ldu,
+                  void* out, int64_t ldo) {
+  if (!ctx || !gate || !up || !out) return FAAR_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || cols % 8 || ldg < cols || ldu < cols || ldo < cols) return FAAR_ERR_SHAPE;
+  if (ldg % 8 || ldu % 8 || ldo % 8 || !aligned16(gate) || !aligned16(up) || !aligned16(out)) return FAAR_ERR_ALIGN;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_silu_mul(ctx, rows, cols, gate, ldg, up, ldu, out, ldo));
+}
+
 int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales, uint8_t* scales_tiled,
                         size_t tiled_bytes) {
   if (!ctx || !scales || !scales_tiled) return FAAR_ERR_INVALID_ARG;
   if (rows <= 0 || cols <= 0) return FAAR_ERR_SHAPE;
   if (tiled_bytes < (size_t)((rows + 127) / 128) * (size_t)((cols + 3) / 4) * 512) return FAAR_ERR_SHAPE;
   if (reinterpret_cast<uintptr_t>(scales_tiled) & 3u) return FAAR_ERR_ALIGN;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, faar_launch_swizzle_scales(ctx, rows, cols, scales, scales_tiled));
 }
 
@@ -623,7 +700,7 @@ int faar_align_loss(faar_ctx* ctx, int T, int vocab, int hidden, const void* Z_f
   int st = faar_align_loss_workspace_size(T, vocab, &need);
   if (st) return st;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need) return FAAR_ERR_WORKSPACE;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   float* kl_p = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + FAAR_WS_HEADER);
   float* mse_p = kl_p + (size_t)T;
   int np = 0;
@@ -644,7 +721,7 @@ int faar_harden_pack(faar_ctx* ctx, const faar_shape* s, const float* V, const u
   if (W_final && wfinal_dtype != FAAR_BF16 && wfinal_dtype != FAAR_F32) return FAAR_ERR_DTYPE;
   if (!aligned16(V) || !aligned16(code) || !aligned16(packed) || (W_final && !aligned16(W_final)))
     return FAAR_ERR_ALIGN;
-  DeviceGuard g(ctx->device);
+  FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, faar_launch_harden_pack(ctx, s, V, code, scales, s_global, packed, scales_out, decisions,
                                                 W_final, wfinal_dtype));
 }

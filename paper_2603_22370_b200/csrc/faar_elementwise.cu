@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(EW_THREADS)
 softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ code,
                       const uint8_t* __restrict__ scales, const float* __restrict__ s_global_p,
                       float beta, int64_t n_groups, float* __restrict__ W_soft, float* __restrict__ H,
-                      __nv_bfloat16* __restrict__ W_bf16) {
+                      __nv_bfloat16* __restrict__ W_bf16, float* __restrict__ W_operand_f32) {
   __shared__ float2 lut[16];
   if (threadIdx.x < 16) {
     const int k = threadIdx.x & 7;
@@ -258,13 +258,19 @@ softquant_eval_kernel(const float* __restrict__ V, const uint8_t* __restrict__ c
         p[1] = make_float4(h[4], h[5], h[6], h[7]);
       }
     }
-    if (W_bf16) {
+    if (W_bf16 || W_operand_f32) {
       float wf[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const float2 nw = lut[(cw >> (4 * i)) & 0xF];
         wf[i] = faar_operand_weight(faar_sigmoid_operand(nbl, hbl, v[i]), nw.x, nw.y, s);
       }
+      if (W_operand_f32) {                              // debug view: the operand before its rounding to BF16
+        float4* p = reinterpret_cast<float4*>(W_operand_f32 + e);
+        p[0] = make_float4(wf[0], wf[1], wf[2], wf[3]);
+        p[1] = make_float4(wf[4], wf[5], wf[6], wf[7]);
+      }
+      if (!W_bf16) continue;
       uint32_t o[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -499,7 +505,7 @@ int faar_launch_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_
 
 int faar_launch_softquant_eval(faar_ctx* ctx, const faar_shape* s, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta, float* W_soft,
-                               float* h, __nv_bfloat16* W_bf16) {
+                               float* h, __nv_bfloat16* W_bf16, float* W_operand_f32) {
   const int64_t groups = (int64_t)s->O * (s->K / 8);
   faar_prof_scope ps(ctx, FAAR_K_SOFT_WEIGHTS);
   cudaLaunchConfig_t cfg = {};
@@ -512,7 +518,7 @@ int faar_launch_softquant_eval(faar_ctx* ctx, const faar_shape* s, const float* 
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, softquant_eval_kernel, V, code, scales, s_global, beta, (int64_t)groups, W_soft,
-                                     h, W_bf16);
+                                     h, W_bf16, W_operand_f32);
   if (e != cudaSuccess) return (int)e;
   return (int)cudaGetLastError();
 }

@@ -788,9 +788,14 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 256 * sizeof(double));
       if (threadIdx.x == 0) {
         __threadfence();                                     // this CTA's partials, ordered by the barrier above
-        const uint32_t prev = atomicAdd(p.fin_counter, 1u);
-        const int last = prev == gridDim.x - 1;
-        if (last) *p.fin_counter = 0u;                       // ready for the next launch
+        int last = 0;
+        // after a wait that gave up the partials are incomplete: no final sums (the caller re-initialises
+        // the workspace, which also clears this counter)
+        if (*reinterpret_cast<volatile uint32_t*>(p.status) == 0u) {
+          const uint32_t prev = atomicAdd(p.fin_counter, 1u);
+          last = prev == gridDim.x - 1;
+          if (last) *p.fin_counter = 0u;                     // ready for the next launch
+        }
         __threadfence();
         *last_flag = last;
       }
@@ -920,8 +925,9 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
   cfg.stream = ctx->stream;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  // how many CTA pairs the device can hold at once (a GPC with an odd SM count strands one SM)
-  static int max_pairs = 0;                      // per kernel instantiation
+  // how many CTA pairs the device can hold at once (a GPC with an odd SM count strands one SM); asked once
+  // per context and kernel instantiation, with the context's device current
+  int& max_pairs = ctx->gemm_max_pairs[MODE == FAAR_GEMM_BWD ? 2 + OPT : MODE];
   if (max_pairs == 0) {
     cfg.gridDim = dim3(2 * (ctx->num_sms / 2), 1, 1);
     int n = 0;
@@ -977,7 +983,8 @@ int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out
   kp.wsoft_next = a->wsoft_next; kp.beta_next = a->beta_next;
   kp.fin_counter = a->fin_counter; kp.fin_mse_partials = a->fin_mse_partials; kp.fin_n_mse = a->fin_n_mse;
   kp.fin_scale_mse = a->fin_scale_mse; kp.fin_scale_round = a->fin_scale_round; kp.fin_out2 = a->fin_out2;
-  // the BWD epilogue forms row offsets of up to 7 rows in 32-bit element counts
+  // the BWD epilogue forms row offsets of up to 7 rows in 32-bit element counts (the entry points refuse
+  // such a K with FAAR_ERR_SHAPE before they get here)
   if (a->mode == FAAR_GEMM_BWD && (long long)a->N * 8 > 0x7FFFFFFFll) return (int)cudaErrorInvalidValue;
 
   switch (a->mode) {

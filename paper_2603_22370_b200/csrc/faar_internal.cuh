@@ -9,6 +9,8 @@
 
 #include <vector>
 
+constexpr int FAAR_GEMM_VARIANTS = 8;     // REF, FWD, BWD x 4 optimiser / chaining variants
+
 struct faar_ctx {
   int device;
   int num_sms;
@@ -18,6 +20,11 @@ struct faar_ctx {
   int tune_bn;                            // 0 = choose the GEMM tile width automatically
   int tune_tail;                          // -1 = choose the tail split automatically, else columns to split
   int last_gemm_bn, last_gemm_pairs, last_gemm_split;   // what the last GEMM launch used
+  // CTA pairs this context's device can hold at once, per GEMM kernel instantiation (0 = not asked yet)
+  int gemm_max_pairs[FAAR_GEMM_VARIANTS];
+  // chained steps: the workspace and the beta of the forward operand that the last backward call wrote
+  const void* wsoft_ws;
+  float wsoft_beta;
   // host-batch path (faar_layer_step_host): copies run on their own stream, ordered by events
   cudaStream_t copy_stream;
   cudaEvent_t ev_copied, ev_done[2];
@@ -78,7 +85,8 @@ int faar_launch_softquant_init(faar_ctx*, const faar_shape*, const void* W, floa
                                uint32_t* amax_word);
 int faar_launch_softquant_eval(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta,
-                               float* W_soft, float* h, __nv_bfloat16* W_soft_bf16);
+                               float* W_soft, float* h, __nv_bfloat16* W_soft_bf16,
+                               float* W_operand_f32 = nullptr);
 int faar_launch_act_fakequant(faar_ctx*, int T, int K, const void* X, int64_t ldx, float s_global_in, void* Xq,
                               int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales, uint32_t* amax_word);
 int faar_launch_transpose_bf16(faar_ctx*, int rows, int cols, const void* in, int64_t ld_in, void* out,
@@ -88,6 +96,8 @@ int faar_launch_swizzle_scales(faar_ctx*, int rows, int cols, const uint8_t* in,
 int faar_launch_align_loss(faar_ctx*, int T, int vocab, int hidden, const void* Z_fp, const void* Z_q, int64_t ldz,
                            const void* H_fp, const void* H_q, int64_t ldh, float tau, float lambda_kl, void* dZ_q,
                            void* dH_q, float* kl_partials, float* mse_partials, int* n_partials);
+int faar_launch_silu_mul(faar_ctx*, int rows, int cols, const void* gate, int64_t ldg, const void* up, int64_t ldu,
+                         void* out, int64_t ldo);
 int faar_launch_round_partials(faar_ctx*, const float* V, int64_t N, float* partials, int* n_partials);
 // out[0] = scale0 * sum(p0[0..n0)), out[1] = scale1 * sum(p1[0..n1)) (either may have n = 0 -> skipped)
 int faar_launch_finalize(faar_ctx*, const float* p0, int n0, float scale0, float* out0, const float* p1,

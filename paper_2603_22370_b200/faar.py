@@ -16,14 +16,47 @@ LIB_PATH = os.path.join(_HERE, "libfaar.so")
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(9)
 BF16, F32 = 0, 1
 
-EXPORTS = ["faar_create", "faar_destroy", "faar_set_stream", "faar_status_string", "faar_last_cuda_error",
-           "faar_workspace_size", "faar_workspace_init", "faar_check_status", "faar_softquant_init",
-           "faar_softquant_eval", "faar_transpose_bf16", "faar_layer_ref", "faar_layer_fwd", "faar_round_loss",
-           "faar_layer_bwd", "faar_layer_step", "faar_layer_step_host", "faar_harden_pack", "faar_profile_begin",
-           "faar_profile_end", "faar_kernel_name", "faar_round_loss_static", "faar_round_loss_static_max_n", "faar_tune_tile_n",
-           "faar_last_gemm_config", "faar_act_fakequant", "faar_swizzle_scales", "faar_tune_tail_split",
-           "faar_last_tail_split", "faar_selftest_wait_timeout", "faar_layer_dx", "faar_align_loss",
-           "faar_align_loss_workspace_size"]
+_P, _I, _L, _F, _Z, _U = C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_size_t, C.c_uint
+
+#: every exported function: (result type, argument types), as declared in include/faar.h
+SIGNATURES = {
+    "faar_create": (_I, [_P, _I, _P]),
+    "faar_destroy": (_I, [_P]),
+    "faar_set_stream": (_I, [_P, _P]),
+    "faar_status_string": (C.c_char_p, [_I]),
+    "faar_last_cuda_error": (_I, [_P]),
+    "faar_tune_tile_n": (_I, [_P, _I]),
+    "faar_tune_tail_split": (_I, [_P, _I]),
+    "faar_last_tail_split": (_I, [_P, _P]),
+    "faar_last_gemm_config": (_I, [_P, _P, _P]),
+    "faar_workspace_size": (_I, [_P, _P]),
+    "faar_workspace_init": (_I, [_P, _P, _Z]),
+    "faar_check_status": (_I, [_P, _P, _P]),
+    "faar_selftest_wait_timeout": (_I, [_P, _P, _Z, _U]),
+    "faar_profile_begin": (_I, [_P]),
+    "faar_profile_end": (_I, [_P, _P, _I, _P]),
+    "faar_kernel_name": (C.c_char_p, [_I]),
+    "faar_softquant_init": (_I, [_P, _P, _P, _F, _P, _P, _P, _P, _P, _Z]),
+    "faar_softquant_eval": (_I, [_P, _P, _P, _P, _P, _P, _F, _P, _P, _P]),
+    "faar_softquant_operand_f32": (_I, [_P, _P, _P, _P, _P, _P, _F, _P]),
+    "faar_transpose_bf16": (_I, [_P, _I, _I, _P, _L, _P, _L]),
+    "faar_act_fakequant": (_I, [_P, _I, _I, _P, _L, _F, _P, _L, _P, _P, _P, _P, _Z]),
+    "faar_layer_ref": (_I, [_P, _P, _P, _P, _P, _P, _Z]),
+    "faar_layer_fwd": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
+    "faar_layer_dx": (_I, [_P, _P, _F, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
+    "faar_round_loss": (_I, [_P, _P, _L, _P, _P, _Z]),
+    "faar_round_loss_static": (_I, [_P, _P, _L, _P]),
+    "faar_round_loss_static_max_n": (_L, []),
+    "faar_layer_bwd": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
+    "faar_layer_step": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
+    "faar_layer_step_host": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
+    "faar_harden_pack": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I]),
+    "faar_align_loss_workspace_size": (_I, [_I, _I, _P]),
+    "faar_align_loss": (_I, [_P, _I, _I, _I, _P, _P, _L, _P, _P, _L, _F, _F, _P, _P, _P, _P, _Z]),
+    "faar_swizzle_scales": (_I, [_P, _I, _I, _P, _P, _Z]),
+    "faar_silu_mul": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L]),
+}
+EXPORTS = list(SIGNATURES)
 
 
 class HParams(C.Structure):
@@ -54,10 +87,9 @@ def lib() -> C.CDLL:
         if not os.path.exists(LIB_PATH):
             raise FileNotFoundError(f"{LIB_PATH} is missing; run `python -m paper_2603_22370_b200.build`")
         l = C.CDLL(LIB_PATH)
-        for name in EXPORTS:
-            getattr(l, name).restype = C.c_int
-        l.faar_status_string.restype = C.c_char_p
-        l.faar_status_string.argtypes = [C.c_int]
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype, fn.argtypes = res, args
         _lib = l
     return _lib
 
@@ -187,6 +219,11 @@ def softquant_eval(ctx, shape, V, code, scales, s_global, beta, W_soft, h, W_sof
                                      C.c_float(beta), _p(W_soft), _p(h), _p(W_soft_bf16)), "faar_softquant_eval")
 
 
+def softquant_operand_f32(ctx, shape, V, code, scales, s_global, beta, W_operand):
+    _check(lib().faar_softquant_operand_f32(ctx._h, C.byref(shape), _p(V), _p(code), _p(scales), _p(s_global),
+                                            C.c_float(beta), _p(W_operand)), "faar_softquant_operand_f32")
+
+
 def act_fakequant(ctx, T, K, X, ldx, s_global_in, Xq_units, ldq, s_global_out, packed, scales, ws):
     _check(lib().faar_act_fakequant(ctx._h, T, K, _p(X), C.c_int64(ldx), C.c_float(s_global_in), _p(Xq_units),
                                     C.c_int64(ldq), _p(s_global_out), _p(packed), _p(scales), _p(ws),
@@ -208,6 +245,10 @@ def align_loss(ctx, T, vocab, hidden, Z_fp, Z_q, ldz, H_fp, H_q, ldh, tau, lambd
 def swizzle_scales(ctx, rows, cols, scales, scales_tiled):
     _check(lib().faar_swizzle_scales(ctx._h, rows, cols, _p(scales), _p(scales_tiled), C.c_size_t(scales_tiled.numel())),
            "faar_swizzle_scales")
+
+
+def silu_mul(ctx, rows, cols, gate, ldg, up, ldu, out, ldo):
+    _check(lib().faar_silu_mul(ctx._h, rows, cols, _p(gate), ldg, _p(up), ldu, _p(out), ldo), "faar_silu_mul")
 
 
 def transpose_bf16(ctx, rows, cols, inp, ld_in, out, ld_out):
@@ -243,9 +284,7 @@ def round_loss_static(ctx, V, N, loss_round):
 
 
 def round_loss_static_max_n() -> int:
-    f = lib().faar_round_loss_static_max_n
-    f.restype = C.c_int64
-    return int(f())
+    return int(lib().faar_round_loss_static_max_n())
 
 
 def layer_bwd(ctx, shape, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, dV, ws):
@@ -266,11 +305,13 @@ def harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, decis
            "faar_harden_pack")
 
 
-def layer_step_host(ctx, shape, hp, X_host, Y_ref_host, X_dev, Xt_dev, Yref_dev, V, code, scales, s_global, adam_m,
+def layer_step_host(ctx, shape, hp, X_host, Y_ref_host, W, X_dev, Xt_dev, Yref_dev, V, code, scales, s_global, adam_m,
                     adam_u, loss_dev2, loss_host2, ws):
-    """X_host, Y_ref_host, loss_host2 are (pinned) CPU tensors; the rest are device tensors."""
+    """X_host, Y_ref_host, loss_host2 are (pinned) CPU tensors; the rest are device tensors.  Y_ref_host None:
+    the target is computed on the device from the copied X and W."""
     _check(lib().faar_layer_step_host(ctx._h, C.byref(shape), C.byref(hp), C.c_void_p(X_host.data_ptr()),
-                                      C.c_void_p(Y_ref_host.data_ptr()), _p(X_dev), _p(Xt_dev), _p(Yref_dev), _p(V),
+                                      C.c_void_p(Y_ref_host.data_ptr() if Y_ref_host is not None else 0), _p(W),
+                                      _p(X_dev), _p(Xt_dev), _p(Yref_dev), _p(V),
                                       _p(code), _p(scales), _p(s_global), _p(adam_m), _p(adam_u), _p(loss_dev2),
                                       C.c_void_p(loss_host2.data_ptr()), _p(ws), C.c_size_t(ws.numel())),
            "faar_layer_step_host")
@@ -286,9 +327,8 @@ def profile_begin(ctx):
 
 def profile_end(ctx) -> dict:
     """{kernel name: (launches, total_ms)} for the kernels launched since profile_begin."""
-    arr = (KernelTime * 16)()
+    arr = (KernelTime * 32)()
     n = C.c_int(0)
-    _check(lib().faar_profile_end(ctx._h, arr, 16, C.byref(n)), "faar_profile_end")
+    _check(lib().faar_profile_end(ctx._h, arr, 32, C.byref(n)), "faar_profile_end")
     l = lib()
-    l.faar_kernel_name.restype = C.c_char_p
     return {l.faar_kernel_name(arr[i].kernel).decode(): (arr[i].launches, arr[i].total_ms) for i in range(n.value)}

@@ -66,3 +66,17 @@ def test_null_context_is_rejected_without_touching_a_device(lib):
     assert lib.faar_harden_pack(z, C.byref(s), z, z, z, z, z, z, z, z, 0) == faar.ERR_INVALID_ARG
     assert lib.faar_create(None, 0, z) == faar.ERR_INVALID_ARG
     assert lib.faar_last_cuda_error(z) == 0
+
+
+def test_binding_declares_argument_types_for_every_export(lib):
+    """Every export has its result and argument types set in the binding, with as many arguments as the
+    header's declaration (so no call relies on ctypes' default int promotion)."""
+    text = open(os.path.join(ROOT, "include", "faar.h")).read()
+    for name in declared_symbols():
+        m = re.search(r"FAAR_API\s+[\w\s\*]+?\b" + name + r"\s*\(([^;]*?)\)\s*;", text, re.S)
+        assert m, name
+        params = m.group(1).strip()
+        n_params = 0 if params in ("", "void") else params.count(",") + 1
+        fn = getattr(lib, name)
+        assert fn.argtypes is not None and len(fn.argtypes) == n_params, (name, n_params, fn.argtypes)
+        assert fn.restype is not None

@@ -211,6 +211,32 @@ def test_harden_vinit_is_rtn_and_pack_roundtrip(seed):
     assert d.shape == (32, 16) and ((d[0, 0] >> 3) & 1) == int(vh[0, 3])
 
 
+def test_pack_decisions_every_bit_against_a_per_element_loop():
+    """Element 8j+i of a row sits in bit i of byte j.  Checked on patterns whose neighbouring decisions
+    differ (a single set element per byte position, an alternating row, a random matrix), element by
+    element, so that a reversed bit order or a shifted byte index fails."""
+    rng = np.random.default_rng(7)
+    O, K = 5, 48
+    pats = [rng.integers(0, 2, (O, K)).astype(bool), (np.arange(O * K).reshape(O, K) % 2 == 0),
+            (np.arange(O * K).reshape(O, K) % 3 == 0)]
+    for e in range(16):                                    # one decision alone, at every position of two bytes
+        one = np.zeros((O, K), bool)
+        one[e % O, e] = True
+        pats.append(one)
+    for vh in pats:
+        d = fo.pack_decisions(vh)
+        assert d.dtype == np.uint8 and d.shape == (O, K // 8)
+        for o in range(O):
+            for e in range(K):
+                assert (int(d[o, e // 8]) >> (e % 8)) & 1 == int(vh[o, e]), (o, e)
+    lone = np.zeros((1, 16), bool)
+    lone[0, 1] = True                                      # element 1 -> bit 1 of byte 0: value 2, not 64
+    assert fo.pack_decisions(lone).tolist() == [[2, 0]]
+    lone[:] = False
+    lone[0, 15] = True                                     # element 15 -> bit 7 of byte 1
+    assert fo.pack_decisions(lone).tolist() == [[0, 128]]
+
+
 # ---- I8: finite differences of Eq. 5 ---------------------------------------
 
 @pytest.mark.parametrize("opt_beta,lam,c", [(4.0, 1.0, 1.0), (11.0, 0.3, 0.01), (32.0, 5.0, 1.0)])
@@ -273,6 +299,21 @@ def test_adam_first_step_and_clip():
         Vc, m, u = fo.adam_update(Vc, np.array([2.0]), m, u, 1e-2, 0.9, 0.999, 0.0, t)
     assert np.allclose(Vc, 0.85)
     assert fo.sgd_update(np.array([0.1, 0.9]), np.array([50.0, -50.0]), 0.01).tolist() == [0.0, 1.0]
+
+
+def test_sgd_step_is_v_minus_lr_times_g_then_clip():
+    """Plain gradient descent on values the clip does not touch: the step is exactly lr * g, downhill;
+    halving lr halves it; a quadratic's minimiser is reached in one step of lr = 1 / curvature."""
+    V = np.array([[0.25, 0.5, 0.75, 0.4]])
+    g = np.array([[2.0, -3.0, 0.5, 0.0]])
+    out = fo.sgd_update(V, g, 0.0625)                      # power-of-two lr: the products are exact
+    assert out.tolist() == [[0.125, 0.6875, 0.71875, 0.4]]
+    assert np.array_equal(V - fo.sgd_update(V, g, 0.03125), 0.5 * (V - out))
+    # f(v) = 2 (v - 0.3)^2 has f' = 4 (v - 0.3): lr = 1/4 lands on the minimiser from anywhere inside [0, 1]
+    v0 = np.array([0.9, 0.1, 0.3])
+    assert np.allclose(fo.sgd_update(v0, 4.0 * (v0 - 0.3), 0.25), 0.3, rtol=0, atol=1e-16)
+    # clip at both ends, and only there
+    assert fo.sgd_update(np.array([0.02, 0.98, 0.5]), np.array([1.0, -1.0, 1.0]), 0.05).tolist() == [0.0, 1.0, 0.45]
 
 
 # ---- I11: exhaustive search on a tiny layer (Eq. 1) -------------------------
@@ -505,3 +546,19 @@ def test_align_loss_gradients_match_finite_differences():
         Hp[t, d] += eps; Hm[t, d] -= eps
         fd = (fo.align_loss(Zf, Zq, Hf, Hp, tau, lam)[1] - fo.align_loss(Zf, Zq, Hf, Hm, tau, lam)[1]) / (2 * eps)
         assert abs(fd - dH[t, d]) <= 1e-7
+
+
+def test_silu_mul_closed_forms_and_library_routine():
+    x = np.array([-30.0, -2.0, -0.5, 0.0, 0.5, 2.0, 30.0, 800.0, -800.0])
+    one = np.ones_like(x)
+    y = fo.silu_mul(x, one)
+    assert y[3] == 0.0 and abs(y[6] - 30.0) < 1e-11 and y[7] == 800.0 and y[8] == 0.0
+    assert np.allclose(y[:7] - fo.silu_mul(-x[:7], one[:7]), x[:7], rtol=0, atol=1e-14)      # silu(x) - silu(-x) = x
+    assert abs(fo.silu_mul(np.array([1.0]), np.array([1.0]))[0] - 1.0 / (1.0 + np.exp(-1.0))) < 1e-16
+    rng = np.random.default_rng(3)
+    g, u = rng.standard_normal((17, 33)) * 4, rng.standard_normal((17, 33))
+    ref = torch.nn.functional.silu(torch.from_numpy(g)) * torch.from_numpy(u)
+    assert np.allclose(fo.silu_mul(g, u), ref.numpy(), rtol=1e-14, atol=1e-300)
+    # the second argument multiplies, the first is gated (not the other way round)
+    assert fo.silu_mul(np.array([0.0]), np.array([5.0]))[0] == 0.0 and fo.silu_mul(np.array([5.0]), np.array([0.0]))[0] == 0.0
+    assert abs(fo.silu_mul(np.array([2.0]), np.array([3.0]))[0] - 3.0 * 2.0 / (1.0 + np.exp(-2.0))) < 1e-15
