@@ -138,32 +138,24 @@ FAAR_API int faar_last_cuda_error(const faar_ctx* ctx);
 
 /* ---- GEMM tiling (no counterpart in the paper: tuning and introspection of this library) -------
  * The tensor-core kernels cover the output with 256-row tiles whose width is chosen per launch (a
- * multiple of 16 in [128, 256]): 256 unless the output is narrower.  faar_tune_tile_n forces a width for the following launches on this context
+ * multiple of 16 in [128, 256]): the widest unless the problem is too small to give every CTA pair a
+ * tile.  faar_tune_tile_n forces a width for the following launches on this context
  * (0 = automatic again).  faar_last_gemm_config reports the width and the number of CTA pairs of the
  * most recent GEMM launch (host out-pointers). */
 FAAR_API int faar_tune_tile_n(faar_ctx* ctx, int bn);
-/* Work distribution of the tensor-core kernels.  By default a launch deals the k blocks (64 elements of the
- * contraction) of all its tiles to the CTA pairs in equal contiguous shares, so that every pair is busy for
- * the same time whatever the ratio of tiles to pairs; a tile whose k blocks fall into two or more shares is
- * finished by the pair that holds its first k block, which adds the other pairs' FP32 partial accumulators
- * (exchanged through the workspace) in k order.  The result of a launch is reproducible run to run, but its
- * FP32 sums are grouped differently from those of a launch with whole tiles.  faar_tune_split(ctx, 0) makes
- * the following launches hand out whole tiles round-robin instead (-1 = default again); faar_last_split
- * reports how many tiles of the most recent GEMM launch were shared between pairs. */
-FAAR_API int faar_tune_split(faar_ctx* ctx, int mode);
-FAAR_API int faar_last_split(const faar_ctx* ctx, int* shared_tiles);
+/* The last, partly empty wave of tiles: the trailing tile columns can be cut into half-width tiles so
+ * that more CTA pairs share it and the final, un-overlapped epilogue is half as long.  The number of
+ * columns cut is chosen per launch from a cost model; faar_tune_tail_split forces it (-1 = automatic,
+ * 0 = none).  faar_last_tail_split reports what the most recent GEMM launch used. */
+FAAR_API int faar_tune_tail_split(faar_ctx* ctx, int columns);
+FAAR_API int faar_last_tail_split(const faar_ctx* ctx, int* columns);
 FAAR_API int faar_last_gemm_config(const faar_ctx* ctx, int* bn, int* cta_pairs);
 
 /* Bytes of workspace that any call on this shape needs (host out-pointer).
- * The workspace must be 256-byte aligned.  Its first 16 KB hold the status
- * word, counters and the flags of split tiles; the caller zeroes them once
- * (faar_workspace_init) before first use.  About 20 MB of it are the partial-
- * accumulator slots of split tiles.  Calls that say they need the header only
- * (faar_softquant_init, faar_act_fakequant, faar_layer_ref) accept a workspace of
- * 256 bytes or more; faar_layer_ref then runs whole tiles. */
+ * The workspace must be 256-byte aligned.  Its first 256 bytes hold the status
+ * word; the caller zeroes them once (faar_workspace_init) before first use. */
 FAAR_API int faar_workspace_size(const faar_shape* shape, size_t* bytes);
-/* Enqueues the zeroing of the workspace's first 16 KB (status word, counters, flags), or of all of it if
- * it is smaller. */
+/* Enqueues the zeroing of the workspace header (status word, counters). */
 FAAR_API int faar_workspace_init(faar_ctx* ctx, void* workspace, size_t workspace_bytes);
 /* Synchronises the context's stream and returns FAAR_ERR_TIMEOUT if a kernel
  * recorded a wait that gave up (detail_out, host, nullable: the raw code),

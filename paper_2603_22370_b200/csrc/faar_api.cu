@@ -84,13 +84,6 @@ struct DeviceGuard {
   DeviceGuard g((ctx)->device);       \
   if (g.err) return cuda_fail((ctx), g.err)
 
-// Hands a GEMM launch the workspace regions that tiles split along the contraction use.
-void give_split_regions(faar_gemm_args* a, uint8_t* ws, const faar_ws_layout& l) {
-  a->slots = reinterpret_cast<float*>(ws + l.off_slots);
-  a->flags = reinterpret_cast<uint32_t*>(ws + FAAR_WS_FLAGS_OFF);
-  a->n_slots = FAAR_SPLIT_SLOTS;
-}
-
 int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Y_ref,
              const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
              void* Y_q, uint8_t* ws, const faar_ws_layout& l, int* n_partials) {
@@ -112,7 +105,6 @@ int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
   a.mse2c = 2.0f * hp->mse_scale;
   a.act_scale = hp->act_scale > 0.f ? hp->act_scale : 1.0f;
   a.partials = reinterpret_cast<float*>(ws + l.off_mse_partials);
-  give_split_regions(&a, ws, l);
   return faar_launch_gemm(ctx, &a, n_partials);
 }
 
@@ -154,7 +146,6 @@ int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
     a.inv_bc1 = (float)(1.0 / (1.0 - pow((double)hp->beta1, (double)hp->step)));
     a.inv_bc2 = (float)(1.0 / (1.0 - pow((double)hp->beta2, (double)hp->step)));
   }
-  give_split_regions(&a, ws, l);
   return faar_launch_gemm(ctx, &a, n_partials);
 }
 
@@ -238,7 +229,7 @@ int faar_create(faar_ctx** out, int device, void* stream) {
   c->last_cuda_error = 0;
   c->encode_tiled = nullptr;
   c->tune_bn = 0;
-  c->tune_split = -1;
+  c->tune_tail = -1;
   c->last_gemm_split = 0;
   for (int i = 0; i < FAAR_GEMM_VARIANTS; ++i) c->gemm_max_pairs[i] = 0;
   c->wsoft_ws = nullptr;
@@ -344,15 +335,15 @@ int faar_tune_tile_n(faar_ctx* ctx, int bn) {
   return FAAR_OK;
 }
 
-int faar_tune_split(faar_ctx* ctx, int mode) {
-  if (!ctx || (mode != -1 && mode != 0)) return FAAR_ERR_INVALID_ARG;
-  ctx->tune_split = mode;
+int faar_tune_tail_split(faar_ctx* ctx, int columns) {
+  if (!ctx || columns < -1) return FAAR_ERR_INVALID_ARG;
+  ctx->tune_tail = columns;
   return FAAR_OK;
 }
 
-int faar_last_split(const faar_ctx* ctx, int* shared_tiles) {
-  if (!ctx || !shared_tiles) return FAAR_ERR_INVALID_ARG;
-  *shared_tiles = ctx->last_gemm_split;
+int faar_last_tail_split(const faar_ctx* ctx, int* columns) {
+  if (!ctx || !columns) return FAAR_ERR_INVALID_ARG;
+  *columns = ctx->last_gemm_split;
   return FAAR_OK;
 }
 
@@ -376,8 +367,7 @@ int faar_workspace_init(faar_ctx* ctx, void* workspace, size_t workspace_bytes) 
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
     return FAAR_ERR_WORKSPACE;
   FAAR_DEVICE_GUARD(ctx);
-  const size_t n = workspace_bytes < FAAR_WS_ZEROED ? workspace_bytes : FAAR_WS_ZEROED;
-  return cuda_fail(ctx, (int)cudaMemsetAsync(workspace, 0, n, ctx->stream));
+  return cuda_fail(ctx, (int)cudaMemsetAsync(workspace, 0, FAAR_WS_HEADER, ctx->stream));
 }
 
 int faar_check_status(faar_ctx* ctx, const void* workspace, uint32_t* detail_out) {
@@ -492,9 +482,6 @@ int faar_layer_ref(faar_ctx* ctx, const faar_shape* s, const void* X, const void
   a.B = X; a.ldb = s->ldx;
   a.status = reinterpret_cast<uint32_t*>(workspace);
   a.Yout = Y_ref; a.yout_dtype = s->yref_dtype; a.ldy = s->ldy; a.yref_t = s->yref_transposed;
-  const faar_ws_layout l = faar_ws_plan(s);
-  if (workspace_bytes >= l.total)                  // a header-only workspace runs whole tiles
-    give_split_regions(&a, reinterpret_cast<uint8_t*>(workspace), l);
   return cuda_fail(ctx, faar_launch_gemm(ctx, &a, nullptr));
 }
 
@@ -528,7 +515,6 @@ int faar_layer_dx(faar_ctx* ctx, const faar_shape* s, float beta, const void* dY
   a.B = dY; a.ldb = s->ldy;
   a.status = reinterpret_cast<uint32_t*>(ws);
   a.Yout = dX; a.yout_dtype = FAAR_BF16; a.ldy = s->ldx;
-  give_split_regions(&a, ws, l);
   return cuda_fail(ctx, faar_launch_gemm(ctx, &a, nullptr));
 }
 
@@ -562,10 +548,10 @@ int faar_round_loss(faar_ctx* ctx, const float* V, int64_t N, float* loss_round,
   if (N <= 0) return FAAR_ERR_SHAPE;
   if (!aligned16(V)) return FAAR_ERR_ALIGN;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
-      workspace_bytes < FAAR_WS_PARTIALS_OFF + 2 * sizeof(float) * FAAR_MAX_PARTIALS)
+      workspace_bytes < FAAR_WS_HEADER + 2 * sizeof(float) * FAAR_MAX_PARTIALS)
     return FAAR_ERR_WORKSPACE;
   FAAR_DEVICE_GUARD(ctx);
-  float* partials = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + FAAR_WS_PARTIALS_OFF +
+  float* partials = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace) + FAAR_WS_HEADER +
                                              sizeof(float) * FAAR_MAX_PARTIALS);
   int np = 0;
   int e = faar_launch_round_partials(ctx, V, N, partials, &np);

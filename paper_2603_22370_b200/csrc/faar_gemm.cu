@@ -19,18 +19,7 @@
 //   BWD : G = dY^T X -> dV -> optimiser update + clip     (step 13, Eq. 5, with Eq. 2/3 chain rule)
 // In all of them the accumulator row (TMEM lane) is the output feature o.
 //
-// Work distribution.  A tile's main loop is `k_blocks` steps of 64 along the contraction; the launch's
-// work is tiles x k_blocks such units.  With `split` on, the units are dealt to the CTA pairs in equal
-// contiguous shares (tile after tile, a tile's k blocks in order), so every pair is busy for the same time
-// whatever the ratio of tiles to pairs.  A share that ends inside a tile leaves that tile to be finished by
-// the next pair(s): the pair that holds a tile's first k block owns the tile and runs its epilogue; every
-// other pair that worked on it -- always as the FIRST item of its own share -- writes its FP32 partial
-// accumulator to its slot in the workspace and raises one flag per epilogue warp; the owner, which reaches
-// the tile as the LAST item of its share, adds the partials in k order (a fixed order: results are
-// reproducible run to run) before its epilogue.  Contributors never wait for anyone before they signal,
-// so an owner's wait always ends.  With `split` off whole tiles go round-robin to the pairs.
-//
-// Every wait on an mbarrier or a flag is bounded: after about two seconds the waiting thread records a code in
+// Every wait on an mbarrier is bounded: after about two seconds the waiting thread records a code in
 // the status word, raises a CTA-wide abort flag and every role leaves its loop; both CTAs then meet at
 // the closing cluster barrier, free their tensor memory and exit.
 #include <cuda.h>
@@ -138,31 +127,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
   return mbar_wait_slow(bar, parity, ac, code);
 }
 
-// "Partial written" flags of split tiles (global memory).  Raised by lane 0 of a contributing warp after the
-// whole warp's stores (each lane fences its own stores first); awaited by lane 0 of the owner's warp.
-__device__ __forceinline__ void flag_raise(uint32_t* f) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(f), "r"(1u) : "memory");
-}
-__device__ __forceinline__ uint32_t flag_read(const uint32_t* f) {
-  uint32_t v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
-  return v;
-}
-__device__ __noinline__ bool flag_wait(const uint32_t* f, const AbortCtl& ac, uint32_t code) {
-  unsigned long long t0 = global_ns();
-  for (uint32_t spin = 1;; ++spin) {
-    if (flag_read(f)) return true;
-    if ((spin & 0x3F) == 0) {
-      if (*ac.flag) return false;
-      if (global_ns() - t0 > ac.limit_ns) {
-        atomicCAS(ac.status, 0u, code);
-        *ac.flag = 1;
-        return false;
-      }
-    }
-  }
-}
-
 // 2-D tiled TMA load into this CTA's shared memory; the byte count is credited to `bar`, which may be
 // a barrier of either CTA of the pair (shared::cluster address).  No multicast.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
@@ -255,9 +219,7 @@ __device__ __forceinline__ uint32_t make_idesc(int bn) {
 struct KParams {
   int M, N, Kc;
   int bn;                 // tile width
-  int split;              // 1: k blocks of all tiles dealt in equal contiguous shares; 0: whole tiles round-robin
-  float* slots;           // split: one FP32 partial-accumulator slot [256][BN_MAX] per CTA pair
-  uint32_t* flags;        // split: [pair][2 * MAX_EPI_WARPS] "partial written" flags, zero between launches
+  int n_full_cols;        // tile columns of full width; the columns after them are bn/2 wide (tail split)
   uint32_t* status;
   // REF / FWD
   void* Yout; int yout_dtype; long long ldy;
@@ -279,84 +241,29 @@ struct KParams {
   float fin_scale_round; float* fin_out2;   // {L_MSE, L_round}; null = no final sums here
 };
 
-// Tile t of the launch: row block fastest.
+// Tile t of the launch: the first n_full_cols tile columns are bn wide, the remaining columns bn/2
+// (half-width tiles fill the last, partly empty wave of the CTA pairs and halve the epilogue that
+// nothing overlaps).  Tiles are numbered row block fastest, all full-width tiles first.
 struct TileCoord { int m0, n0, w; };
 __device__ __forceinline__ TileCoord tile_coord(const KParams& p, int t, int m_tiles) {
+  const int full_tiles = m_tiles * p.n_full_cols;
   TileCoord c;
-  c.m0 = (t % m_tiles) * (2 * BM);
-  c.n0 = (t / m_tiles) * p.bn;
-  c.w = p.bn;
+  if (t < full_tiles) {
+    c.m0 = (t % m_tiles) * (2 * BM);
+    c.n0 = (t / m_tiles) * p.bn;
+    c.w = p.bn;
+  } else {
+    const int u = t - full_tiles;
+    c.m0 = (u % m_tiles) * (2 * BM);
+    c.n0 = p.n_full_cols * p.bn + (u / m_tiles) * (p.bn / 2);
+    c.w = p.bn / 2;
+  }
   return c;
 }
-__device__ __forceinline__ int tile_count(const KParams& p, int m_tiles) { return m_tiles * ((p.N + p.bn - 1) / p.bn); }
-
-// One item of a CTA pair's work: k blocks [kb0, kb1) of one tile.  kb0 == 0: this pair owns the tile (runs
-// its epilogue; if kb1 < k_blocks it first adds the partials of the pairs that hold the rest).  kb0 > 0:
-// this pair contributes a partial accumulator.
-struct Item { int tile, kb0, kb1; };
-struct ItemIter {
-  long long u, u_end;     // split: this pair's units
-  int tile, stride, tiles, k_blocks, split;
-  __device__ __forceinline__ ItemIter(const KParams& p, int pair, int n_pairs, int total_tiles, int kbs)
-      : u(0), u_end(0), tile(pair), stride(n_pairs), tiles(total_tiles), k_blocks(kbs), split(p.split) {
-    if (split) {
-      const long long units = (long long)total_tiles * kbs;
-      u = units * pair / n_pairs;
-      u_end = units * (pair + 1) / n_pairs;
-    }
-  }
-  __device__ __forceinline__ bool next(Item& it) {
-    if (split) {
-      if (u >= u_end) return false;
-      it.tile = (int)(u / k_blocks);
-      it.kb0 = (int)(u - (long long)it.tile * k_blocks);
-      const long long rem = u_end - u;
-      it.kb1 = rem < (long long)(k_blocks - it.kb0) ? it.kb0 + (int)rem : k_blocks;
-      u += it.kb1 - it.kb0;
-      return true;
-    }
-    if (tile >= tiles) return false;
-    it.tile = tile; it.kb0 = 0; it.kb1 = k_blocks;
-    tile += stride;
-    return true;
-  }
-};
-// First unit of pair q's share (split mode).
-__device__ __forceinline__ long long share_begin(int q, int n_pairs, int total_tiles, int k_blocks) {
-  return (long long)total_tiles * k_blocks * q / n_pairs;
-}
-
-// ---- partial accumulators of split tiles ------------------------------------------------------------
-// Slot of pair q: rows 0..255 of the pair's tile (CTA rank r holds rows 128 r ..), BN_MAX floats per row.
-// A lane moves the 16 columns of one tcgen05.ld as four 16-byte vectors; L2 is the point of exchange
-// (.cg: no L1 copy that could be stale).
-constexpr int SLOT_FLOATS = 2 * BM * BN_MAX;
-__device__ __forceinline__ void slot_store16(float* slot_row, int c, const uint32_t (&r)[16]) {
-#pragma unroll
-  for (int q = 0; q < 4; ++q)
-    asm volatile("st.global.cg.v4.b32 [%0], {%1,%2,%3,%4};" ::"l"(slot_row + c + 4 * q), "r"(r[4 * q]), "r"(r[4 * q + 1]),
-                 "r"(r[4 * q + 2]), "r"(r[4 * q + 3]) : "memory");
-}
-__device__ __forceinline__ void slot_add16(const float* slot_row, int c, uint32_t (&r)[16]) {
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    float4 v;
-    asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "l"(slot_row + c + 4 * q) : "memory");
-    r[4 * q] = __float_as_uint(__uint_as_float(r[4 * q]) + v.x);
-    r[4 * q + 1] = __float_as_uint(__uint_as_float(r[4 * q + 1]) + v.y);
-    r[4 * q + 2] = __float_as_uint(__uint_as_float(r[4 * q + 2]) + v.z);
-    r[4 * q + 3] = __float_as_uint(__uint_as_float(r[4 * q + 3]) + v.w);
-  }
-}
-// The contributing pairs of an owned, incomplete tile: pairs first .. first + count - 1 (in k order).
-struct Contrib { int first, count; };
-__device__ __forceinline__ Contrib contributors(const Item& it, int pair, int n_pairs, int total_tiles, int k_blocks) {
-  Contrib c{pair + 1, 0};
-  if (it.kb1 >= k_blocks) return c;
-  const long long tile_end = (long long)(it.tile + 1) * k_blocks;
-  for (int q = pair + 1; q < n_pairs && share_begin(q, n_pairs, total_tiles, k_blocks) < tile_end; ++q) ++c.count;
-  return c;
+__device__ __forceinline__ int tile_count(const KParams& p, int m_tiles) {
+  const int rest = p.N - p.n_full_cols * p.bn;                    // columns covered by half-width tiles
+  const int half_cols = rest > 0 ? (rest + p.bn / 2 - 1) / (p.bn / 2) : 0;
+  return m_tiles * (p.n_full_cols + half_cols);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
@@ -620,7 +527,8 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
 // Launched as clusters of two CTAs along x: CTAs 2c and 2c+1 form pair c.
 template <int MODE, int OPT>
 __global__ void __launch_bounds__(Cfg<MODE>::THREADS, 1)
-faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const KParams p) {
+faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmBh, const KParams p) {
   using C = Cfg<MODE>;
   const int BN = p.bn;
   extern __shared__ uint8_t smem_raw[];
@@ -671,13 +579,12 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const uint64_t keep = l2_policy_keep();
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      ItemIter items(p, pair, n_pairs, total_tiles, k_blocks);
-      Item it;
-      while (ok && items.next(it)) {
-        const TileCoord tc = tile_coord(p, it.tile, m_tiles);
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+        const TileCoord tc = tile_coord(p, tile, m_tiles);
         const int m0 = tc.m0 + (int)rank * BM;
         const int n0 = tc.n0 + (int)rank * (tc.w / 2);
-        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+        const CUtensorMap* mapB = tc.w == BN ? &tmB : &tmBh;      // box of w/2 rows
+        for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(empty_bar(stage), phase ^ 1u, ac, 0x100u | stage);
           if (!ok) break;
           const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
@@ -685,7 +592,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * (uint32_t)(C::A_BYTES + (tc.w / 2) * BK * 2));
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
           tma_load_2d(sa, &tmA, kb * BK, m0, leader_full, keep);
-          tma_load_2d(sb, &tmB, kb * BK, n0, leader_full, keep);
+          tma_load_2d(sb, mapB, kb * BK, n0, leader_full, keep);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -699,19 +606,17 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // ---------------- MMA issuer (leader CTA only) ----------------
     if (lane == 0 && rank == 0) {
       int stage = 0; uint32_t phase = 0;
-      int n_it = 0;
+      int it = 0;
       bool ok = true;
-      ItemIter items(p, pair, n_pairs, total_tiles, k_blocks);
-      Item it;
-      const uint32_t idesc = make_idesc(BN);
-      for (; ok && items.next(it); ++n_it) {
-        const int acc = n_it & 1;
-        const uint32_t acc_phase = (n_it >> 1) & 1;
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
         ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, ac, 0x200u | acc);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN_MAX;
-        for (int kb = it.kb0; kb < it.kb1; ++kb) {
+        const uint32_t idesc = make_idesc(tile_coord(p, tile, m_tiles).w);
+        for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(full_bar(stage), phase, ac, 0x300u | stage);
           if (!ok) break;
           tc_fence_after();
@@ -720,7 +625,7 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 bf16 = 32 bytes inside the swizzled row: +2 in the 16-byte address field
-            tc_mma_bf16(tmem_d, da + 2u * k, db + 2u * k, idesc, (kb > it.kb0 || k != 0) ? 1u : 0u);
+            tc_mma_bf16(tmem_d, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
           tc_commit_pair(empty_bar(stage));            // frees this stage in both CTAs
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -739,79 +644,21 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (MODE == FAAR_GEMM_BWD) s_global = *p.s_global;
     uint32_t pn = 0;                                   // panels this quarter has staged so far
     bool dead = false;
-    int n_it = 0;
-    ItemIter items(p, pair, n_pairs, total_tiles, k_blocks);
-    Item it;
-    // split tiles: this warp's flag in a pair's flag row, and this lane's row in a pair's slot (both recomputed
-    // where they are needed: the BWD epilogue has no registers to spare)
-    auto flag_of = [&](int q) { return p.flags + q * (2 * MAX_EPI_WARPS) + (int)rank * MAX_EPI_WARPS + ew; };
-    auto slot_row_of = [&](int q) {
-      return p.slots + (long long)q * SLOT_FLOATS + ((int)rank * BM + quarter * 32 + lane) * BN_MAX;
-    };
-    for (; items.next(it); ++n_it) {
-      const int acc = n_it & 1;
-      const uint32_t acc_phase = (n_it >> 1) & 1;
+    int it = 0;
+    for (int tile = pair; tile < total_tiles; tile += n_pairs, ++it) {
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, ac, 0x400u | acc);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const TileCoord tc = tile_coord(p, it.tile, m_tiles);
+      const TileCoord tc = tile_coord(p, tile, m_tiles);
       const int m0 = tc.m0 + (int)rank * BM, n0 = tc.n0, TW = tc.w;
       const int cols_per_warp = ((TW / C::COL_GROUPS + 15) / 16) * 16;
       const int col_begin = cg * cols_per_warp;
       const int col_end = min(col_begin + cols_per_warp, TW);
       const int o = m0 + quarter * 32 + lane;
       const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN_MAX);
-
-      if (it.kb0 > 0) {
-        // ---- contributor: this pair's partial accumulator goes to its slot; one flag per warp.  The columns
-        // a warp writes are the ones the same warp of the owner reads (same tile, same mapping).
-        float* const srow = slot_row_of(pair);
-        if constexpr (MODE == FAAR_GEMM_BWD) {
-          const int sub = ew >> 2;
-          for (int pc = 0; pc < TW; pc += PW) {
-            const int c = pc + 16 * sub;
-            if (c < TW && n0 + c < p.N) {
-              uint32_t r[16];
-              tmem_ld16(trow + (uint32_t)c, r);
-              tmem_ld_wait();
-              slot_store16(srow, c, r);
-            }
-          }
-        } else {
-          for (int c = col_begin; c < col_end; c += 16) {
-            if (n0 + c >= p.N) break;
-            uint32_t r[16];
-            tmem_ld16(trow + (uint32_t)c, r);
-            tmem_ld_wait();
-            slot_store16(srow, c, r);
-          }
-        }
-        __threadfence();                               // every lane: its stores before the flag
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) {
-          flag_raise(flag_of(pair));
-          mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
-        }
-        continue;
-      }
-
-      // ---- owner.  An incomplete tile first waits for the partials of the pairs that hold the rest.
-      const int n_contrib = contributors(it, pair, n_pairs, total_tiles, k_blocks).count;   // pairs pair+1 .. pair+n_contrib
-      if (n_contrib > 0) {
-        bool okf = true;
-        if (lane == 0)
-          for (int q = 1; q <= n_contrib && okf; ++q)
-            okf = flag_wait(flag_of(pair + q), ac, 0x800u | (uint32_t)ew);
-        if (!__all_sync(0xffffffffu, okf)) { dead = true; break; }
-        __threadfence();
-      }
-      // adds, in k order, the partials for the 16 columns from c on
-      auto add_partials = [&](int c, uint32_t (&r)[16]) {
-        for (int q = 1; q <= n_contrib; ++q) slot_add16(slot_row_of(pair + q), c, r);
-      };
-
       if constexpr (MODE == FAAR_GEMM_BWD) {
         // PW-column panels, staged by the four warps of this lane quarter together (see epi_bwd_rows)
         const int sub = ew >> 2;
@@ -831,7 +678,6 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t r[16];
             tmem_ld16(trow + (uint32_t)c, r);
             tmem_ld_wait();
-            if (n_contrib > 0) add_partials(c, r);
 #pragma unroll
             for (int u = 0; u < 4; ++u)
               sts128(panel + (uint32_t)lane * (4u * PW) + (uint32_t)(((4 * sub + u) ^ (lane & 7)) << 4), r[4 * u],
@@ -862,12 +708,6 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
         }
-        // the partials have been consumed: the flags go back to zero for the next launch
-        if (n_contrib > 0) {
-          __syncwarp();
-          if (lane == 0)
-            for (int q = 1; q <= n_contrib; ++q) *flag_of(pair + q) = 0u;
-        }
         continue;
       } else {
         if (MODE == FAAR_GEMM_FWD && p.yref_t && p.yref_dtype == FAAR_BF16) {
@@ -891,7 +731,6 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 uint32_t r[16];
                 tmem_ld16(trow + (uint32_t)c, r);
                 tmem_ld_wait();
-                if (n_contrib > 0) add_partials(c, r);
                 const uint32_t w[8] = {yraw[2 * q].x, yraw[2 * q].y, yraw[2 * q].z, yraw[2 * q].w,
                                        yraw[2 * q + 1].x, yraw[2 * q + 1].y, yraw[2 * q + 1].z, yraw[2 * q + 1].w};
                 float yr[16];
@@ -911,7 +750,6 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t r[16];
             tmem_ld16(trow + (uint32_t)c, r);
             tmem_ld_wait();
-            if (n_contrib > 0) add_partials(c, r);
             if (MODE == FAAR_GEMM_REF) {
               epi_ref(p, o, n0 + c, r);
             } else {
@@ -924,12 +762,8 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
-        for (int q = 1; q <= n_contrib; ++q) *flag_of(pair + q) = 0u;
-      }
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
     }
-    (void)dead;
     if (MODE != FAAR_GEMM_REF) {
       warp_acc = faar_warp_sum(warp_acc);
       if (lane == 0) p.partials[blockIdx.x * C::EPI_WARPS + ew] = warp_acc;
@@ -1025,25 +859,47 @@ int make_map(faar_ctx* ctx, CUtensorMap* map, const void* ptr, int rows, int col
 }
 
 // Tile width for an M x N output.  A tile's time is set by the operand bytes it pulls through the SM (A rows
-// are not shared between tiles), not by its columns, so the widest tile wins; a tile is never wider than the
-// output rounded up to 32 columns.
-int pick_bn(const faar_ctx* ctx, int N) {
+// are not shared between tiles), not by its columns, so 256-wide tiles win wherever they were measured
+// against narrower ones that fill more CTA pairs (down_proj-, gate-, q- and k_proj-shaped layers), with one
+// exception: the dW GEMM of a small layer, whose per-weight epilogue is heavy, gains from spreading 128-wide
+// tiles over twice as many pairs while fewer than half of the pairs would have a 256-wide tile.  A tile is
+// never wider than the output rounded up to 32 columns.
+int pick_bn(const faar_ctx* ctx, int mode, int M, int N, int pairs) {
   if (ctx->tune_bn >= 128 && ctx->tune_bn <= BN_MAX && ctx->tune_bn % 16 == 0) return ctx->tune_bn;
-  if (N >= BN_MAX) return BN_MAX;
-  return N <= 128 ? 128 : (N + 31) / 32 * 32;
+  const long long m_tiles = (M + 2 * BM - 1) / (2 * BM);
+  int bn = BN_MAX;
+  if (N < BN_MAX) bn = N <= 128 ? 128 : (N + 31) / 32 * 32;
+  if (mode == FAAR_GEMM_BWD && 2 * m_tiles * ((N + BN_MAX - 1) / BN_MAX) < pairs) bn = 128;
+  return bn;
 }
 
-// CTA pairs for a launch.  Split mode deals k blocks, so any number of pairs up to the device's is busy for
-// the same time; a pair should still have at least MIN_KB k blocks, or the exchange of a partial accumulator
-// (256 KB through L2, about five k blocks' worth of time) costs more than the work it spreads.
-constexpr int MIN_KB = 8;
-int pick_pairs(long long tiles, int k_blocks, int max_pairs, bool split) {
-  long long pairs = tiles < max_pairs ? tiles : max_pairs;
-  if (split) {
-    const long long by_work = tiles * k_blocks / MIN_KB;
-    if (by_work > pairs) pairs = by_work < max_pairs ? by_work : max_pairs;
+// How many trailing tile columns to cut into half-width tiles.  Tiles go to CTA pairs round-robin, all
+// full-width tiles first.  A half tile costs 0.75 of a full one (its A rows are loaded all the same), and
+// the epilogue of a pair's last tile is not overlapped by anything (0.4 of that tile's cost).  Returns the
+// number of full-width columns that minimises the busiest pair's time (ties: fewer half tiles).
+int pick_full_cols(const faar_ctx* ctx, int M, int N, int bn, int pairs) {
+  const int m_tiles = (M + 2 * BM - 1) / (2 * BM);
+  const int n_cols = (N + bn - 1) / bn;
+  if (bn % 32 != 0) return n_cols;
+  if (ctx->tune_tail >= 0) return ctx->tune_tail < n_cols ? n_cols - ctx->tune_tail : 0;
+  double best = -1.0;
+  int best_full = n_cols;
+  for (int split = 0; split <= n_cols && split <= 16; ++split) {
+    const int full_cols = n_cols - split;
+    const long long full_tiles = (long long)m_tiles * full_cols;
+    const int rest = N - full_cols * bn;
+    const long long half_tiles = rest > 0 ? (long long)m_tiles * ((rest + bn / 2 - 1) / (bn / 2)) : 0;
+    const long long total = full_tiles + half_tiles;
+    double worst = 0.0;
+    for (int p = 0; p < pairs && p < total; ++p) {
+      double load = 0.0, last = 0.0;
+      for (long long t = p; t < total; t += pairs) { last = t < full_tiles ? 1.0 : 0.75; load += last; }
+      load += 0.4 * last;
+      if (load > worst) worst = load;
+    }
+    if (best < 0.0 || worst < best - 1e-9) { best = worst; best_full = full_cols; }
   }
-  return (int)(pairs < 1 ? 1 : pairs);
+  return best_full;
 }
 
 template <int MODE, int OPT = 0>
@@ -1080,31 +936,27 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
     if (n > ctx->num_sms / 2) n = ctx->num_sms / 2;
     max_pairs = n;
   }
-  const int bn = pick_bn(ctx, a->N);
+  const int bn = pick_bn(ctx, MODE, a->M, a->N, max_pairs);
   kp.bn = bn;
-  CUtensorMap tmA, tmB;
+  kp.n_full_cols = pick_full_cols(ctx, a->M, a->N, bn, max_pairs);
+  CUtensorMap tmA, tmB, tmBh;
   int e = make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
   if (e) return e;
   e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, bn / 2);
   if (e) return e;
-  const long long tiles = (long long)((a->M + 2 * BM - 1) / (2 * BM)) * ((a->N + bn - 1) / bn);
-  const int k_blocks = (a->Kc + BK - 1) / BK;
-  bool split = ctx->tune_split != 0 && a->slots != nullptr && a->flags != nullptr;
-  int pairs = pick_pairs(tiles, k_blocks, max_pairs, split);
-  if (split && pairs > a->n_slots) { split = false; pairs = pick_pairs(tiles, k_blocks, max_pairs, false); }
-  if (tiles * k_blocks % pairs == 0 && (tiles * k_blocks / pairs) % k_blocks == 0) split = false;   // shares are whole tiles
-  kp.split = split ? 1 : 0;
-  kp.slots = a->slots;
-  kp.flags = a->flags;
+  e = make_map(ctx, &tmBh, a->B, a->N, a->Kc, a->ldb, bn % 32 == 0 ? bn / 4 : bn / 2);   // half-width tiles
+  if (e) return e;
+  const int rest_cols = a->N - kp.n_full_cols * bn;
+  const long long tiles = (long long)((a->M + 2 * BM - 1) / (2 * BM)) *
+                          (kp.n_full_cols + (rest_cols > 0 ? (rest_cols + bn / 2 - 1) / (bn / 2) : 0));
+  const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
   cfg.gridDim = dim3(2 * pairs, 1, 1);
   if (n_partials_out) *n_partials_out = 2 * pairs * C::EPI_WARPS;
   ctx->last_gemm_bn = bn;
   ctx->last_gemm_pairs = pairs;
-  ctx->last_gemm_split = 0;
-  if (split)                                        // tiles whose k blocks are shared by two or more pairs
-    for (int q = 1; q < pairs; ++q) ctx->last_gemm_split += (tiles * k_blocks * q / pairs) % k_blocks != 0;
+  ctx->last_gemm_split = (a->N + bn - 1) / bn - kp.n_full_cols;
   faar_prof_scope ps(ctx, MODE == FAAR_GEMM_REF ? FAAR_K_GEMM_REF : (MODE == FAAR_GEMM_FWD ? FAAR_K_GEMM_FWD : FAAR_K_GEMM_BWD));
-  ce = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, kp);
+  ce = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmBh, kp);
   if (ce != cudaSuccess) return (int)ce;
   return (int)cudaGetLastError();
 }
@@ -1120,8 +972,7 @@ int faar_gemm_max_partials(const faar_ctx* ctx, int, int) { return ctx->num_sms 
 
 int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out) {
   KParams kp;
-  kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.bn = BN_MAX; kp.split = 0; kp.slots = nullptr; kp.flags = nullptr;
-  kp.status = a->status;
+  kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.bn = BN_MAX; kp.n_full_cols = 0; kp.status = a->status;
   kp.Yout = a->Yout; kp.yout_dtype = a->yout_dtype; kp.ldy = a->ldy;
   kp.Yref = a->Yref; kp.yref_dtype = a->yref_dtype; kp.yref_t = a->yref_t;
   kp.dYt = a->dYt; kp.ld_dyt = a->ld_dyt; kp.mse2c = a->mse2c; kp.act_scale = a->act_scale; kp.partials = a->partials;

@@ -18,8 +18,8 @@ struct faar_ctx {
   int last_cuda_error;
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
   int tune_bn;                            // 0 = choose the GEMM tile width automatically
-  int tune_split;                         // -1 = split tiles along the contraction whenever slots are given, 0 = never
-  int last_gemm_bn, last_gemm_pairs, last_gemm_split;   // what the last GEMM launch used (split: tiles shared by pairs)
+  int tune_tail;                          // -1 = choose the tail split automatically, else columns to split
+  int last_gemm_bn, last_gemm_pairs, last_gemm_split;   // what the last GEMM launch used
   // CTA pairs this context's device can hold at once, per GEMM kernel instantiation (0 = not asked yet)
   int gemm_max_pairs[FAAR_GEMM_VARIANTS];
   // chained steps: the workspace and the beta of the forward operand that the last backward call wrote
@@ -48,23 +48,14 @@ struct faar_prof_scope {
 // ---- workspace layout -------------------------------------------------------
 // [0, 256)            header: word 0 = status (0 = ok), word 1 = |W| max bits, word 2 = count of dW-GEMM
 //                     CTAs that have finished (zero between launches)
-// [256, 16384)        "partial written" flags of split GEMM tiles: [pair][32] words, zero between launches
-// [16384, ..)         loss partials (float): MSE region then Round region
+// [256, 256+P)        loss partials (float): MSE region then Round region
 // [..]                W_soft bf16 [O,K]
 // [..]                dYt bf16 [O, ceil8(T)]
-// [..]                FP32 partial-accumulator slots of split GEMM tiles, one 256 x 256 slot per CTA pair
-// faar_workspace_init zeroes the first 16384 bytes (or the whole workspace if it is smaller).
 constexpr size_t FAAR_WS_HEADER = 256;
-constexpr size_t FAAR_WS_FLAGS_OFF = 256;
-constexpr size_t FAAR_WS_ZEROED = 16384;
-constexpr size_t FAAR_WS_PARTIALS_OFF = 16384;
 constexpr int FAAR_MAX_PARTIALS = 16384;  // per loss term
-constexpr int FAAR_SPLIT_SLOTS = 80;      // CTA pairs that can take part in split tiles (B200: 74)
-constexpr size_t FAAR_SLOT_BYTES = 256 * 256 * 4;
-static_assert(FAAR_WS_FLAGS_OFF + (size_t)FAAR_SPLIT_SLOTS * 32 * 4 <= FAAR_WS_ZEROED, "flags fit the zeroed prefix");
 
 struct faar_ws_layout {
-  size_t off_mse_partials, off_round_partials, off_wsoft, off_dyt, off_slots, total;
+  size_t off_mse_partials, off_round_partials, off_wsoft, off_dyt, total;
   int64_t ld_dyt;
 };
 
@@ -73,7 +64,7 @@ static inline size_t faar_align_up(size_t x, size_t a) { return (x + a - 1) / a 
 static inline faar_ws_layout faar_ws_plan(const faar_shape* s) {
   faar_ws_layout l;
   l.ld_dyt = ((int64_t)s->T + 7) / 8 * 8;
-  size_t off = FAAR_WS_PARTIALS_OFF;
+  size_t off = FAAR_WS_HEADER;
   l.off_mse_partials = off;
   off += sizeof(float) * FAAR_MAX_PARTIALS;
   l.off_round_partials = off;
@@ -84,9 +75,6 @@ static inline faar_ws_layout faar_ws_plan(const faar_shape* s) {
   off = faar_align_up(off, 1024);
   l.off_dyt = off;
   off += (size_t)s->O * (size_t)l.ld_dyt * 2;
-  off = faar_align_up(off, 1024);
-  l.off_slots = off;
-  off += (size_t)FAAR_SPLIT_SLOTS * FAAR_SLOT_BYTES;
   l.total = faar_align_up(off, 1024);
   return l;
 }
@@ -140,8 +128,6 @@ struct faar_gemm_args {
   float beta, lam_over_n, lr, b1, b2, eps, inv_bc1, inv_bc2; int opt;
   // BWD, optional: also write the next step's BF16 operand W_soft(V', beta_next) (null = not wanted)
   __nv_bfloat16* wsoft_next; float beta_next;
-  // tiles split along the contraction: partial-accumulator slots and flags in the workspace (null = whole tiles only)
-  float* slots; uint32_t* flags; int n_slots;
   // BWD, optional: final loss sums by the last CTA (fin_out2 null = not wanted)
   uint32_t* fin_counter; const float* fin_mse_partials; int fin_n_mse; float fin_scale_mse, fin_scale_round;
   float* fin_out2;

@@ -26,8 +26,8 @@ SIGNATURES = {
     "faar_status_string": (C.c_char_p, [_I]),
     "faar_last_cuda_error": (_I, [_P]),
     "faar_tune_tile_n": (_I, [_P, _I]),
-    "faar_tune_split": (_I, [_P, _I]),
-    "faar_last_split": (_I, [_P, _P]),
+    "faar_tune_tail_split": (_I, [_P, _I]),
+    "faar_last_tail_split": (_I, [_P, _P]),
     "faar_last_gemm_config": (_I, [_P, _P, _P]),
     "faar_workspace_size": (_I, [_P, _P]),
     "faar_workspace_init": (_I, [_P, _P, _Z]),
@@ -167,15 +167,14 @@ def tune_tile_n(ctx: Context, bn: int):
     _check(lib().faar_tune_tile_n(ctx._h, C.c_int(bn)), "faar_tune_tile_n")
 
 
-def tune_split(ctx: Context, mode: int):
-    """0: the GEMM launches hand out whole tiles round-robin; -1: k blocks in equal shares (the default)."""
-    _check(lib().faar_tune_split(ctx._h, C.c_int(mode)), "faar_tune_split")
+def tune_tail_split(ctx: Context, columns: int):
+    """Forces how many trailing tile columns are cut into half-width tiles (-1 = automatic, 0 = none)."""
+    _check(lib().faar_tune_tail_split(ctx._h, C.c_int(columns)), "faar_tune_tail_split")
 
 
-def last_split(ctx: Context) -> int:
-    """Tiles of the most recent GEMM launch whose k blocks were shared between CTA pairs."""
+def last_tail_split(ctx: Context) -> int:
     n = C.c_int(0)
-    _check(lib().faar_last_split(ctx._h, C.byref(n)), "faar_last_split")
+    _check(lib().faar_last_tail_split(ctx._h, C.byref(n)), "faar_last_tail_split")
     return n.value
 
 

@@ -567,9 +567,9 @@ def test_error_statuses(ctx):
 @pytest.mark.parametrize("bn", [128, 144, 176, 224, 240])
 @pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (520, 272, 1300)])
 def test_forced_tile_widths_give_the_same_step(ctx, O, K, T, bn):
-    """With whole tiles handed out (no tile split along the contraction), the tile width only changes how the
-    output is cut up: every forced width must reproduce the automatic choice bit for bit (each output element
-    is the same sum in the same order); the loss is a sum of differently grouped partials."""
+    """The tile width only changes how the output is cut up: every forced width must reproduce the
+    automatic choice bit for bit (each output element is the same sum in the same order); the loss is a
+    sum of differently grouped partials."""
     W, X, Yref = _problem(O, K, T, seed=5)
     hp, _ = f32hp(beta=6.0, step=2)
     rng = np.random.default_rng(3)
@@ -578,7 +578,6 @@ def test_forced_tile_widths_give_the_same_step(ctx, O, K, T, bn):
     u0 = (1e-6 * rng.uniform(0, 1, W.shape)).astype(np.float32)
     out = []
     try:
-        faar.tune_split(ctx, 0)
         for width in (0, bn):
             faar.tune_tile_n(ctx, width)
             lay = GpuLayer(ctx, W, X)
@@ -594,7 +593,6 @@ def test_forced_tile_widths_give_the_same_step(ctx, O, K, T, bn):
             out.append((dYt, dV, host(lay.V).copy(), host(lay.m).copy(), host(lay.u).copy(), host(lay.loss)[0]))
     finally:
         faar.tune_tile_n(ctx, 0)
-        faar.tune_split(ctx, -1)
     for a, b in zip(out[0][:5], out[1][:5]):
         assert np.array_equal(a, b)
     assert abs(out[0][5] - out[1][5]) <= 1e-5 * abs(out[0][5])
@@ -647,79 +645,38 @@ def test_layer_step_host_matches_device_steps(ctx, two_sets):
     assert rel_l2(out[3][0], out[0][0]) <= 2e-3 and abs(out[3][2][0] - out[0][2][0]) <= 1e-2 * out[0][2][0]
 
 
-# (O, K, T): tiles shared by two pairs in both GEMMs; a dW tile shared by about six pairs and more forward
-# tiles than pairs; a single tile cut into many shares; a contraction too short to be worth sharing.
-SPLIT_SHAPES = [(300, 1040, 600), (1500, 272, 3300), (200, 2100, 256), (520, 784, 130)]
-
-
-@pytest.mark.parametrize("O,K,T", SPLIT_SHAPES)
-def test_tiles_split_along_the_contraction_agree_with_whole_tiles(ctx, O, K, T):
-    """By default a launch deals k blocks, not tiles, to the CTA pairs, and a tile shared by several pairs is
-    summed from their FP32 partial accumulators.  That regroups each output's FP32 sum and nothing else:
-    against whole tiles the results agree to FP32 summation accuracy; a second launch reproduces the first bit
-    for bit (the partials are added in a fixed order); the flags are back to zero afterwards, so a third
-    launch on the same workspace is correct too."""
+@pytest.mark.parametrize("split", [1, 3, 100])
+@pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (520, 784, 1300)])
+def test_half_width_tail_tiles_give_the_same_step(ctx, O, K, T, split):
+    """Cutting trailing tile columns into half-width tiles only re-partitions the output."""
     W, X, Yref = _problem(O, K, T, seed=6)
     hp, _ = f32hp(beta=6.0, step=2)
     rng = np.random.default_rng(4)
     V0 = rng.uniform(0, 1, W.shape).astype(np.float32)
     m0 = (1e-3 * rng.standard_normal(W.shape)).astype(np.float32)
     u0 = (1e-6 * rng.uniform(0, 1, W.shape)).astype(np.float32)
-    out, shared = [], []
+    out = []
     try:
-        for mode in (0, -1, -1, -1):
-            faar.tune_split(ctx, mode)
+        faar.tune_tile_n(ctx, 256)
+        for cols in (0, split):
+            faar.tune_tail_split(ctx, cols)
             lay = GpuLayer(ctx, W, X)
             lay.init()
             lay.set_yref(Yref)
             lay.set_state(V=V0, m=m0, u=u0)
-            Yq = host(lay.fwd(hp, want_yq=True)).copy()
-            n_fwd = faar.last_split(ctx)
+            lay.fwd(hp)
             dYt = host(lay.dYt).copy()
             dV = host(lay.bwd(hp, want_dv=True)).copy()
-            shared.append((n_fwd, faar.last_split(ctx)))
+            if cols:
+                assert faar.last_tail_split(ctx) == min(cols, -(-K // 256))
             lay.check()
-            out.append((dYt, dV, host(lay.V).copy(), host(lay.m).copy(), host(lay.u).copy(), Yq, host(lay.loss)[0]))
+            out.append((dYt, dV, host(lay.V).copy(), host(lay.m).copy(), host(lay.u).copy(), host(lay.loss)[0]))
     finally:
-        faar.tune_split(ctx, -1)
-    assert shared[0] == (0, 0)
-    if K > 512 or T > 512:
-        assert shared[1][0] > 0 or shared[1][1] > 0
-    for a, b, c in zip(out[1][:6], out[2][:6], out[3][:6]):
-        assert np.array_equal(a, b) and np.array_equal(a, c)
-    assert out[1][6] == out[2][6]
-    whole, split = out[0], out[1]
-    assert max_rel_to_peak(split[5], whole[5]) <= 2.0 ** -7          # BF16 outputs: at most one rounding step apart
-    assert rel_l2(split[0], whole[0]) <= 1e-3 and max_rel_to_peak(split[0], whole[0]) <= 2.0 ** -7     # dY^T is BF16 too
-    # dV: the same dY^T would give FP32-accurate agreement; here dY^T itself may differ by BF16 steps
-    assert rel_l2(split[1], whole[1]) <= 2e-3
-    assert abs(split[6] - whole[6]) <= 1e-5 * abs(whole[6])
-
-
-@pytest.mark.parametrize("O,K,T", SPLIT_SHAPES[:2])
-def test_split_backward_alone_matches_whole_tiles_to_fp32_accuracy(ctx, O, K, T):
-    """The backward GEMM given the very same dY^T: split and whole-tile launches may differ only by the
-    grouping of FP32 sums."""
-    W, X, Yref = _problem(O, K, T, seed=6)
-    hp, _ = f32hp(beta=6.0, step=2, opt=0, lr=1e-4)
-    rng = np.random.default_rng(4)
-    V0 = rng.uniform(0, 1, W.shape).astype(np.float32)
-    res = []
-    try:
-        for mode in (0, -1):
-            faar.tune_split(ctx, 0)
-            lay = GpuLayer(ctx, W, X)
-            lay.init()
-            lay.set_yref(Yref)
-            lay.set_state(V=V0)
-            lay.fwd(hp)
-            faar.tune_split(ctx, mode)
-            res.append(host(lay.bwd(hp, want_dv=True)).copy())
-            assert (faar.last_split(ctx) > 0) == (mode == -1)
-            lay.check()
-    finally:
-        faar.tune_split(ctx, -1)
-    assert max_rel_to_peak(res[1], res[0]) <= 1e-5 and rel_l2(res[1], res[0]) <= 1e-5
+        faar.tune_tail_split(ctx, -1)
+        faar.tune_tile_n(ctx, 0)
+    for a, b in zip(out[0][:5], out[1][:5]):
+        assert np.array_equal(a, b)
+    assert abs(out[0][5] - out[1][5]) <= 1e-5 * abs(out[0][5])
 
 
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives(ctx):
