@@ -34,23 +34,34 @@ def problem():
     return W, X
 
 
-def assert_dv_elementwise(X, V, code, scales, sg, hpo, dV_g, dV_o):
-    """Element by element where the gradient is not small against the tensor's largest entry (there the dW
-    dot product has not cancelled): 2e-3 of the entry itself, plus what re-rounding the BF16-boundary
-    weights of the same output row can move it -- weight (o, k) moving by one BF16 step changes G[o, j] by
-    2 c step (X[:, k] . X[:, j]), and dV[o, j] by that times the chain factor of (o, j)."""
+def assert_dv_elementwise(X, Yref, V, code, scales, sg, hpo, dV_g, dV_o):
+    """Element by element, on every entry that is not small against the tensor's largest.  The gradient is a
+    dot product over T tokens that cancels to about 1/sqrt(K) of its summands, so an entry's error is measured
+    against what can legitimately move it:
+      * 2e-3 of the entry itself;
+      * dY is stored in BF16: where the FP32 accumulator and the float64 product leave r = Y_q - Y_ref on
+        different sides of a BF16 boundary (the accumulator's ~1e-5 relative error of r against the spacing
+        2^-8: under 1 % of the entries) the two sides' dY differ by one step, and G[o, j] by a random sum of
+        about sqrt(0.01 T) terms 2^-8 |dY[t, o] X[t, j]|: allowed 6 sigma = 6 * 0.1 * 2^-8 * Q,
+        Q[o, j] = sqrt(sum_t dY[t, o]^2 X[t, j]^2);
+      * re-rounding the BF16-boundary weights of the same output row: weight (o, k) moving by one BF16 step
+        changes G[o, j] by 2 c step (X[:, k] . X[:, j]).
+    The last two enter through the chain factor of (o, j)."""
     import scipy.sparse as sp
-    Xd = X.astype(np.float64)
-    gram = np.abs(Xd.T @ Xd)                                      # |X[:, k] . X[:, j]|
+    Xf = X.astype(np.float32)
+    gram = np.abs(Xf.T @ Xf).astype(np.float64)                  # |X[:, k] . X[:, j]| (a bound: float32 is enough)
     Wo, _ = fo.soft_weights(V, code, scales, sg, hpo.beta)
     tie, step = bf16_tie_elements(Wo)
     chain = np.abs(fo.chain_factor(V, code, scales, sg, hpo.beta))
-    allow = 2.0 * hpo.mse_scale * chain * (sp.csr_matrix(np.where(tie, step, 0.0)) @ gram)
+    _, dY, _ = fo.layer_fwd(X, Yref, V, code, scales, sg, hpo.beta, hpo.mse_scale, "bf16")
+    Q = np.sqrt(((dY.astype(np.float32) ** 2).T @ (Xf ** 2)).astype(np.float64))
+    allow = chain * (2.0 * hpo.mse_scale * (sp.csr_matrix(np.where(tie, step, 0.0)) @ gram) + 6.0 * 0.1 * 2.0 ** -8 * Q)
     sure = np.abs(dV_o) > 1e-3 * np.abs(dV_o).max()
     err = np.abs(dV_g - dV_o)
     bad = sure & (err > 2e-3 * np.abs(dV_o) + allow)
     assert not bad.any(), (int(bad.sum()), float((err / np.abs(dV_o))[bad].max()))
-    # the allowance is the exception, not the rule: most checked entries pass on the 2e-3 alone
+    # the allowances are small against the entries they protect: a typical checked entry is held to a few 1e-3
+    assert np.median((allow / np.abs(dV_o))[sure]) <= 5e-3
     assert (sure & (err > 2e-3 * np.abs(dV_o))).sum() <= 1e-2 * sure.sum()
     return int(sure.sum())
 
@@ -95,7 +106,7 @@ def test_init_step_and_pack_at_full_size(ctx, problem):
     assert abs(host(l_round)[0] - l_round_o) <= 1e-5 * l_round_o
     dV_g = host(dV_g)
     assert rel_l2(dV_g, dV_o) <= 2e-3 and max_rel_to_peak(dV_g, dV_o) <= 2e-3
-    assert_dv_elementwise(X, V0, code, scales, sg, hpo, dV_g, dV_o)
+    assert_dv_elementwise(X, Yref, V0, code, scales, sg, hpo, dV_g, dV_o)
     Vg = host(lay.V)
     assert Vg.min() >= 0.0 and Vg.max() <= 1.0
     # the first Adam step moves every v by lr * g / (|g| + eps): where the gradient's sign is
@@ -161,7 +172,7 @@ def test_benchmarked_launch_configuration_against_the_oracle(ctx, problem):
         sure = np.abs(dV_o) > 1e-3 * np.abs(dV_o).max()
         if t == 0:
             assert np.all(np.abs(Vg - Vo)[sure] <= 1e-6)
-            assert_dv_elementwise(X, state[0], code, scales, sg, hpo, dV_g, dV_o)
+            assert_dv_elementwise(X, Yref, state[0], code, scales, sg, hpo, dV_g, dV_o)
         else:
             assert rel_l2(ug, uo) <= 4e-3
         state = (Vg, mg, ug)
