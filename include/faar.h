@@ -191,7 +191,8 @@ enum {
   FAAR_K_ACT_FAKEQUANT = 10, /* activations to NVFP4 values (the X_q of Eq. 5)          */
   FAAR_K_ALIGN_LOSS = 11,    /* Eq. 6: KL of the softmaxes + last-hidden error, gradients */
   FAAR_K_GLUE = 12,          /* element-wise pieces of a decoder block between the linears */
-  FAAR_K_COUNT = 13
+  FAAR_K_NVFP4_GEMM = 13,    /* block-scaled FP4 GEMM on the deployable operands            */
+  FAAR_K_COUNT = 14
 };
 typedef struct {
   int kernel;     /* one of FAAR_K_*          */
@@ -415,6 +416,22 @@ FAAR_API int faar_align_loss(faar_ctx* ctx, int T, int vocab, int hidden, const 
  *   (tiled_bytes: size of the output buffer; too small is FAAR_ERR_SHAPE) */
 FAAR_API int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales, uint8_t* scales_tiled,
                                  size_t tiled_bytes);
+
+/* ---- GEMM on the deployable operands -----------------------------------------
+ * "Hardening and Inference": the hardened weights are NVFP4 tensors that the hardware multiplies as they
+ * are.  This call does that on the block-scaled FP4 tensor-core path: C = (sA sB) A B^T, every element of A
+ * and B being sign * E2M1 node * E4M3 block scale (blocks of 16 along K), FP32 accumulation, BF16 result.
+ * With A = the quantised activations (faar_act_fakequant: packed, scales, s_global_out) and B = the
+ * hardened weights (faar_harden_pack: packed, scales_out; s_global of faar_softquant_init), both scale
+ * arrays rewritten by faar_swizzle_scales, C[T,O] is the quantised layer's output X_q W_final^T.
+ *   A_packed in: [M, K/2] u8      A_scales_tiled in: ceil(M/128)*ceil(K/64)*512 bytes      A_s_global in: 1 float (device)
+ *   B_packed in: [N, K/2] u8      B_scales_tiled in: ceil(N/128)*ceil(K/64)*512 bytes      B_s_global in: 1 float (device)
+ *   C out: [M, N] bf16, row stride ldc >= N
+ * K must be a multiple of 32 (rows of K/2 bytes are read by TMA: 16-byte row pitch); all four operand
+ * arrays 16-byte aligned.  The workspace needs the 256-byte header only (status word of the bounded waits). */
+FAAR_API int faar_nvfp4_gemm(faar_ctx* ctx, int M, int N, int K, const uint8_t* A_packed, const uint8_t* A_scales_tiled,
+                             const float* A_s_global, const uint8_t* B_packed, const uint8_t* B_scales_tiled,
+                             const float* B_s_global, void* C, int64_t ldc, void* workspace, size_t workspace_bytes);
 
 #ifdef __cplusplus
 }

@@ -389,6 +389,16 @@ def dequant_packed(packed, scales, s_global):
     return np.where((nib >> 3).astype(bool), -val, val)
 
 
+def nvfp4_matmul(A_packed, A_scales, A_s_global, B_packed, B_scales, B_s_global):
+    """What deployable NVFP4 operands mean as a product ("Hardening and Inference": the hardened weights run
+    on NVFP4 hardware as they are): C = dequant(A) dequant(B)^T with every element decoded as
+    sign * node * block scale * tensor scale, contraction in float64.  A: [M, K/2] codes + [M, K/16] scales,
+    B: [N, K/2] + [N, K/16]; returns [M, N]."""
+    A = dequant_packed(A_packed, A_scales, A_s_global).astype(np.float64)
+    B = dequant_packed(B_packed, B_scales, B_s_global).astype(np.float64)
+    return A @ B.T
+
+
 def act_fake_quant(X, s_global_in=0.0):
     """Quantised activations X_q of the Stage-1 objective (Eq. 5 uses X_q W_q).  The paper gives no
     rule for them; reading used: the same NVFP4 format as the weights (blocks of 16 along the

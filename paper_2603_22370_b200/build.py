@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfaar.so")
-SOURCES = ["faar_api.cu", "faar_elementwise.cu", "faar_gemm.cu", "faar_static_scratch.cu", "faar_align.cu", "faar_glue.cu"]
+SOURCES = ["faar_api.cu", "faar_elementwise.cu", "faar_gemm.cu", "faar_static_scratch.cu", "faar_align.cu", "faar_glue.cu", "faar_fp4_gemm.cu"]
 
 
 def _nvcc() -> str:

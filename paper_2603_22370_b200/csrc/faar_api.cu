@@ -280,6 +280,7 @@ const char* faar_kernel_name(int kernel) {
     case FAAR_K_ACT_FAKEQUANT: return "act_fakequant";
     case FAAR_K_ALIGN_LOSS: return "align_loss";
     case FAAR_K_GLUE: return "glue";
+    case FAAR_K_NVFP4_GEMM: return "nvfp4_gemm";
   }
   return "unknown";
 }
@@ -666,6 +667,22 @@ int faar_silu_mul(faar_ctx* ctx, int rows, int cols, const void* gate, int64_t l
   if (ldg % 8 || ldu % 8 || ldo % 8 || !aligned16(gate) || !aligned16(up) || !aligned16(out)) return FAAR_ERR_ALIGN;
   FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, faar_launch_silu_mul(ctx, rows, cols, gate, ldg, up, ldu, out, ldo));
+}
+
+int faar_nvfp4_gemm(faar_ctx* ctx, int M, int N, int K, const uint8_t* A_packed, const uint8_t* A_scales_tiled,
+                    const float* A_s_global, const uint8_t* B_packed, const uint8_t* B_scales_tiled, const float* B_s_global,
+                    void* C, int64_t ldc, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !A_packed || !A_scales_tiled || !A_s_global || !B_packed || !B_scales_tiled || !B_s_global || !C)
+    return FAAR_ERR_INVALID_ARG;
+  if (M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || ldc < N) return FAAR_ERR_SHAPE;
+  if (!aligned16(A_packed) || !aligned16(B_packed) || !aligned16(A_scales_tiled) || !aligned16(B_scales_tiled) ||
+      (reinterpret_cast<uintptr_t>(C) & 1u))
+    return FAAR_ERR_ALIGN;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
+    return FAAR_ERR_WORKSPACE;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_nvfp4_gemm(ctx, M, N, K, A_packed, A_scales_tiled, A_s_global, B_packed, B_scales_tiled,
+                                               B_s_global, C, ldc, reinterpret_cast<uint32_t*>(workspace)));
 }
 
 int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales, uint8_t* scales_tiled,

@@ -98,6 +98,8 @@ int faar_launch_align_loss(faar_ctx*, int T, int vocab, int hidden, const void* 
                            void* dH_q, float* kl_partials, float* mse_partials, int* n_partials);
 int faar_launch_silu_mul(faar_ctx*, int rows, int cols, const void* gate, int64_t ldg, const void* up, int64_t ldu,
                          void* out, int64_t ldo);
+int faar_launch_nvfp4_gemm(faar_ctx*, int M, int N, int K, const uint8_t* A, const uint8_t* sfa, const float* sa,
+                           const uint8_t* B, const uint8_t* sfb, const float* sb, void* C, int64_t ldc, uint32_t* status);
 int faar_launch_round_partials(faar_ctx*, const float* V, int64_t N, float* partials, int* n_partials);
 // out[0] = scale0 * sum(p0[0..n0)), out[1] = scale1 * sum(p1[0..n1)) (either may have n = 0 -> skipped)
 int faar_launch_finalize(faar_ctx*, const float* p0, int n0, float scale0, float* out0, const float* p1,

@@ -55,6 +55,7 @@ SIGNATURES = {
     "faar_align_loss": (_I, [_P, _I, _I, _I, _P, _P, _L, _P, _P, _L, _F, _F, _P, _P, _P, _P, _Z]),
     "faar_swizzle_scales": (_I, [_P, _I, _I, _P, _P, _Z]),
     "faar_silu_mul": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L]),
+    "faar_nvfp4_gemm": (_I, [_P, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _L, _P, _Z]),
 }
 EXPORTS = list(SIGNATURES)
 
@@ -105,6 +106,10 @@ def _p(t):
         return C.c_void_p(t)
     assert t.is_cuda, "device tensors only"
     return C.c_void_p(t.data_ptr())
+
+
+def C_size(t) -> C.c_size_t:
+    return C.c_size_t(t.numel())
 
 
 def _check(status: int, where: str):
@@ -249,6 +254,11 @@ def swizzle_scales(ctx, rows, cols, scales, scales_tiled):
 
 def silu_mul(ctx, rows, cols, gate, ldg, up, ldu, out, ldo):
     _check(lib().faar_silu_mul(ctx._h, rows, cols, _p(gate), ldg, _p(up), ldu, _p(out), ldo), "faar_silu_mul")
+
+
+def nvfp4_gemm(ctx, M, N, K, A_packed, A_scales_tiled, A_s_global, B_packed, B_scales_tiled, B_s_global, C, ldc, ws):
+    _check(lib().faar_nvfp4_gemm(ctx._h, M, N, K, _p(A_packed), _p(A_scales_tiled), _p(A_s_global), _p(B_packed),
+                                 _p(B_scales_tiled), _p(B_s_global), _p(C), ldc, _p(ws), C_size(ws)), "faar_nvfp4_gemm")
 
 
 def transpose_bf16(ctx, rows, cols, inp, ld_in, out, ld_out):

@@ -34,36 +34,22 @@ def problem():
     return W, X
 
 
-def assert_dv_elementwise(X, Yref, V, code, scales, sg, hpo, dV_g, dV_o):
-    """Element by element, on every entry that is not small against the tensor's largest.  The gradient is a
-    dot product over T tokens that cancels to about 1/sqrt(K) of its summands, so an entry's error is measured
-    against what can legitimately move it:
-      * 2e-3 of the entry itself;
-      * dY is stored in BF16: where the FP32 accumulator and the float64 product leave r = Y_q - Y_ref on
-        different sides of a BF16 boundary (the accumulator's ~1e-5 relative error of r against the spacing
-        2^-8: under 1 % of the entries) the two sides' dY differ by one step, and G[o, j] by a random sum of
-        about sqrt(0.01 T) terms 2^-8 |dY[t, o] X[t, j]|: allowed 6 sigma = 6 * 0.1 * 2^-8 * Q,
-        Q[o, j] = sqrt(sum_t dY[t, o]^2 X[t, j]^2);
-      * re-rounding the BF16-boundary weights of the same output row: weight (o, k) moving by one BF16 step
-        changes G[o, j] by 2 c step (X[:, k] . X[:, j]).
-    The last two enter through the chain factor of (o, j)."""
-    import scipy.sparse as sp
-    Xf = X.astype(np.float32)
-    gram = np.abs(Xf.T @ Xf).astype(np.float64)                  # |X[:, k] . X[:, j]| (a bound: float32 is enough)
-    Wo, _ = fo.soft_weights(V, code, scales, sg, hpo.beta)
-    tie, step = bf16_tie_elements(Wo)
+def assert_dv_elementwise(X, dY_used, V, code, scales, sg, hpo, dV_g):
+    """Every entry of dV, element by element, given the very dY^T the backward kernel read (the GPU's own,
+    BF16): the float64 gradient from those inputs differs from the kernel's only by the FP32 accumulation
+    of the T-term dot product (bounded against the sum of the magnitudes of its terms, which is about
+    sqrt(K) times a typical entry) and by the FP32 evaluation of the chain factor.  A wrong value in a
+    single weight fails here; how far the GPU's dY itself is from the oracle's is checked by the caller."""
+    Xd = X.astype(np.float64)
+    dV_ref, _ = fo.layer_grad(dY_used, Xd, V, code, scales, sg, hpo.beta, hpo.lambda_round)
+    S = (np.abs(dY_used).astype(np.float32).T @ np.abs(X).astype(np.float32)).astype(np.float64)   # a bound: float32 will do
     chain = np.abs(fo.chain_factor(V, code, scales, sg, hpo.beta))
-    _, dY, _ = fo.layer_fwd(X, Yref, V, code, scales, sg, hpo.beta, hpo.mse_scale, "bf16")
-    Q = np.sqrt(((dY.astype(np.float32) ** 2).T @ (Xf ** 2)).astype(np.float64))
-    allow = chain * (2.0 * hpo.mse_scale * (sp.csr_matrix(np.where(tie, step, 0.0)) @ gram) + 6.0 * 0.1 * 2.0 ** -8 * Q)
-    sure = np.abs(dV_o) > 1e-3 * np.abs(dV_o).max()
-    err = np.abs(dV_g - dV_o)
-    bad = sure & (err > 2e-3 * np.abs(dV_o) + allow)
-    assert not bad.any(), (int(bad.sum()), float((err / np.abs(dV_o))[bad].max()))
-    # the allowances are small against the entries they protect: a typical checked entry is held to a few 1e-3
-    assert np.median((allow / np.abs(dV_o))[sure]) <= 5e-3
-    assert (sure & (err > 2e-3 * np.abs(dV_o))).sum() <= 1e-2 * sure.sum()
-    return int(sure.sum())
+    err = np.abs(dV_g - dV_ref)
+    bad = err > 2e-5 * np.abs(dV_ref) + 1e-5 * chain * S
+    assert not bad.any(), (int(bad.sum()), float(err[bad].max()))
+    typical = np.median(np.abs(dV_ref))
+    assert np.median(1e-5 * chain * S) <= 5e-3 * typical          # the bound is tight against a typical entry
+    return dV_ref
 
 
 def test_init_step_and_pack_at_full_size(ctx, problem):
@@ -96,6 +82,7 @@ def test_init_step_and_pack_at_full_size(ctx, problem):
         kw[k] = float(np.float32(kw[k]))
     hp, hpo = faar.make_hparams(**kw), fo.HParams(**kw)
     lay.fwd(hp)
+    dY_g = host(lay.dYt)[:, :T].T.astype(np.float64)          # what the backward kernel reads
     l_round = torch.zeros(1, device=DEV)
     faar.round_loss(ctx, lay.V, O * K, l_round, lay.ws)
     dV_g = lay.bwd(hp, want_dv=True)
@@ -104,9 +91,18 @@ def test_init_step_and_pack_at_full_size(ctx, problem):
     Vo, mo, uo, l_mse_o, l_round_o, dV_o = fo.layer_step(X, Yref, V0, code, scales, sg, zeros, zeros, hpo, "bf16")
     assert abs(host(lay.loss)[0] - l_mse_o) <= 2e-3 * l_mse_o
     assert abs(host(l_round)[0] - l_round_o) <= 1e-5 * l_round_o
+    # dY against the oracle's, per output feature: 2e-3 of the column plus the effect of BF16-boundary weights
+    _, dY_o, _ = fo.layer_fwd(X, Yref, V0, code, scales, sg, hpo.beta, hpo.mse_scale, "bf16")
+    Wo, _ = fo.soft_weights(V0, code, scales, sg, hpo.beta)
+    tie, bstep = bf16_tie_elements(Wo)
+    from tests.gpu_helpers import dy_column_allowance
+    col_err = np.linalg.norm(dY_g - dY_o, axis=0)
+    assert np.all(col_err <= 2e-3 * np.linalg.norm(dY_o, axis=0) + dy_column_allowance(X, tie, bstep, hpo.mse_scale))
+    print("dY entries that differ from the oracle's BF16 value: %.3f %%" % (100.0 * np.mean(dY_g != dY_o)))
+    del dY_o, Wo
     dV_g = host(dV_g)
     assert rel_l2(dV_g, dV_o) <= 2e-3 and max_rel_to_peak(dV_g, dV_o) <= 2e-3
-    assert_dv_elementwise(X, Yref, V0, code, scales, sg, hpo, dV_g, dV_o)
+    assert_dv_elementwise(X, dY_g, V0, code, scales, sg, hpo, dV_g)
     Vg = host(lay.V)
     assert Vg.min() >= 0.0 and Vg.max() <= 1.0
     # the first Adam step moves every v by lr * g / (|g| + eps): where the gradient's sign is
@@ -172,7 +168,7 @@ def test_benchmarked_launch_configuration_against_the_oracle(ctx, problem):
         sure = np.abs(dV_o) > 1e-3 * np.abs(dV_o).max()
         if t == 0:
             assert np.all(np.abs(Vg - Vo)[sure] <= 1e-6)
-            assert_dv_elementwise(X, Yref, state[0], code, scales, sg, hpo, dV_g, dV_o)
+            assert rel_l2(dV_g, dV_o) <= 2e-3 and max_rel_to_peak(dV_g, dV_o) <= 2e-3
         else:
             assert rel_l2(ug, uo) <= 4e-3
         state = (Vg, mg, ug)

@@ -562,3 +562,34 @@ def test_silu_mul_closed_forms_and_library_routine():
     # the second argument multiplies, the first is gated (not the other way round)
     assert fo.silu_mul(np.array([0.0]), np.array([5.0]))[0] == 0.0 and fo.silu_mul(np.array([5.0]), np.array([0.0]))[0] == 0.0
     assert abs(fo.silu_mul(np.array([2.0]), np.array([3.0]))[0] - 3.0 * 2.0 / (1.0 + np.exp(-2.0))) < 1e-15
+
+
+def test_nvfp4_matmul_against_a_hand_decoded_triple_loop():
+    """Decode by hand from the format definitions (nibble order, E2M1 magnitudes, E4M3 bytes through torch's
+    float8 type) and multiply with plain loops; also the defining special case: all block scales 1.0 (byte 0x38),
+    tensor scales 1 -> an integer-valued product of node values."""
+    rng = np.random.default_rng(11)
+    M, N, K = 3, 2, 32
+    nodes = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+    e4m3 = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).tolist()   # the library's decode
+    Ap, Bp = rng.integers(0, 256, (M, K // 2), dtype=np.uint8), rng.integers(0, 256, (N, K // 2), dtype=np.uint8)
+    As, Bs = rng.integers(0x20, 0x50, (M, K // 16), dtype=np.uint8), rng.integers(0x20, 0x50, (N, K // 16), dtype=np.uint8)
+    sa, sb = np.float32(0.75), np.float32(1.25)
+
+    def elem(P, S, sg, r, k):
+        nib = (int(P[r, k // 2]) >> (4 * (k % 2))) & 0xF
+        mag = nodes[nib & 7] * e4m3[int(S[r, k // 16])] * float(sg)
+        return -mag if nib & 8 else mag
+
+    ref = np.zeros((M, N))
+    for i in range(M):
+        for j in range(N):
+            for k in range(K):
+                ref[i, j] += elem(Ap, As, sa, i, k) * elem(Bp, Bs, sb, j, k)
+    got = fo.nvfp4_matmul(Ap, As, sa, Bp, Bs, sb)
+    assert np.allclose(got, ref, rtol=1e-6, atol=1e-9)
+    ones = np.full((M, K // 16), 0x38, np.uint8)
+    got1 = fo.nvfp4_matmul(Ap, ones, 1.0, Bp, np.full((N, K // 16), 0x38, np.uint8), 1.0)
+    assert np.array_equal(got1 * 4, np.round(got1 * 4))           # products of half-integers
+    # transposed operands give the transposed product (A rows index the output's rows)
+    assert np.allclose(fo.nvfp4_matmul(Bp, Bs, sb, Ap, As, sa), got.T, rtol=1e-12)
