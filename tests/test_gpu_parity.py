@@ -417,9 +417,14 @@ def test_layer_step_is_fwd_then_bwd_and_matches_oracle(ctx, O, K, T):
     assert rel_l2(V_step, Vo) <= 2e-3 and np.max(np.abs(V_step - Vo)) <= 2.0 * hpo.lr + 1e-6
 
 
-#: Largest fraction of the final rounding decisions in which a free-running GPU run may differ from a
-#: free-running oracle run of config 1 (100 Adam steps amplify each BF16-boundary difference into +-lr moves).
-FREE_RUN_FLIP_FRACTION = 2e-2
+#: A step taken from the oracle's own state may flip a rounding decision only where the oracle's v is this
+#: close to the threshold 0.5 (measured: 4 such decisions in 100 steps x 32768 weights, the farthest at 1.4e-4).
+FLIP_DISTANCE = 5e-3
+#: Two free-running runs (GPU, oracle) of config 1: 100 Adam steps amplify each BF16-boundary difference into
+#: +-lr moves, so their final decisions differ in a small fraction of the weights (measured 1.6 %), all of them
+#: weights that both runs left near the threshold (measured: oracle |v - 0.5| <= 9.2e-3, median 1.3e-3).
+FREE_RUN_FLIP_FRACTION = 4e-2
+FREE_RUN_FLIP_DISTANCE = 3e-2
 
 
 def _config1():
@@ -453,11 +458,10 @@ def test_config1_100_steps_each_step_from_the_oracle_state(ctx):
         Vg = host(lay.V)
         # norm-wise 2e-3; a single entry may differ by up to the Adam step when its gradient is ~0
         assert rel_l2(Vg, V) <= 2e-3 and np.max(np.abs(Vg - V)) <= 2.0 * hpo.lr + 1e-6, t
-        # rounding decisions: a decision may differ from the oracle's only where the oracle's v sits within
-        # one optimiser move of the threshold (the two sides can step by up to lr in opposite directions
-        # where the gradient is ~0), and only in a handful of entries
+        # rounding decisions: from the same state, a decision may differ from the oracle's only where the
+        # oracle's v sits within 5e-3 of the threshold, and only in a handful of entries
         flips = fo.harden(Vg) != fo.harden(V)
-        assert flips.sum() <= 1e-4 * V.size + 1 and np.all(np.abs(V[flips] - 0.5) <= 2.0 * hpo.lr), t
+        assert flips.sum() <= 1e-4 * V.size + 1 and np.all(np.abs(V[flips] - 0.5) < FLIP_DISTANCE), t
         worst_flip = max(worst_flip, float(np.abs(V[flips] - 0.5).max()) if flips.any() else 0.0)
         n_flips += int(flips.sum())
         # Adam moments: near a stationary point the data term and the Round Loss term of dV cancel, so
@@ -511,6 +515,7 @@ def test_config1_free_running_100_steps_then_harden_pack(ctx):
           f"median {np.median(np.abs(res['V'][flips] - 0.5)) if flips.any() else 0:.2e}, "
           f"max {np.abs(res['V'][flips] - 0.5).max() if flips.any() else 0:.2e}")
     assert flips.mean() <= FREE_RUN_FLIP_FRACTION
+    assert np.all(np.abs(res["V"][flips] - 0.5) <= FREE_RUN_FLIP_DISTANCE)
     code, scales, sg = res["code"], res["scales"], res["s_global"]
 
     def hard_loss(V):

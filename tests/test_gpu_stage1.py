@@ -111,8 +111,8 @@ def test_silu_mul_matches_oracle(ctx):
     torch.cuda.synchronize()
     ref = fo.silu_mul(g, u)
     got = host(out[:, :cols]).astype(np.float64)
-    # BF16 output of an FP32 evaluation: half a BF16 step (2^-9) plus the FP32 evaluation's 1e-6
-    assert np.all(np.abs(got - ref) <= (2.0 ** -9 + 2e-6) * np.abs(ref) + 1e-38)
+    # BF16 output of an FP32 evaluation: half a BF16 step (at most 2^-8 of the value) plus the FP32 evaluation's 1e-6
+    assert np.all(np.abs(got - ref) <= (2.0 ** -8 + 2e-6) * np.abs(ref) + 1e-38)
     assert torch.all(out[:, cols:] == 5.0)
     faar.silu_mul(ctx, rows, cols, G, ld, U, ld, U, ld)            # in place on the second operand
     torch.cuda.synchronize()
