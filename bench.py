@@ -591,6 +591,30 @@ def run_ours(args):
 
     dx_us = layer_dx_us()
 
+    # ---- the deployable operands through the library's own NVFP4 GEMM: X_q W_final^T, alone
+    def nvfp4_gemm_us(rounds=20):
+        pw = torch.empty((O, K // 2), dtype=torch.uint8, device=device)
+        sw = torch.empty((O, K // 16), dtype=torch.uint8, device=device)
+        faar.harden_pack(ctx, shape, V, code, scales, s_global, pw, sw, None, None)
+        Xq = torch.empty_like(X)
+        sx = torch.empty(1, dtype=torch.float32, device=device)
+        px = torch.empty((T, K // 2), dtype=torch.uint8, device=device)
+        scx = torch.empty((T, K // 16), dtype=torch.uint8, device=device)
+        faar.act_fakequant(ctx, T, K, X, K, 0.0, Xq, K, sx, px, scx, ws)
+        tw = torch.empty(-(-O // 128) * -(-(K // 16) // 4) * 512, dtype=torch.uint8, device=device)
+        tx = torch.empty(-(-T // 128) * -(-(K // 16) // 4) * 512, dtype=torch.uint8, device=device)
+        faar.swizzle_scales(ctx, O, K // 16, sw, tw)
+        faar.swizzle_scales(ctx, T, K // 16, scx, tx)
+        Y = torch.empty((T, O), dtype=torch.bfloat16, device=device)
+        fn = lambda: faar.nvfp4_gemm(ctx, T, O, K, px, tx, sx, pw, tw, s_global, Y, O, ws)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                fn()
+        stream.synchronize()
+        return 1e3 * timed(lambda: [fn() for _ in range(rounds)]) / rounds
+
+    fp4_us = nvfp4_gemm_us()
+
     # ---- Eq. 6's alignment loss alone: 4096 tokens x 128 256 logits (3.2 GB moved per call, far above L2)
     AL_T, AL_V, AL_D = args.align_tokens, 128256, 2048
 
@@ -620,7 +644,8 @@ def run_ours(args):
             print(json.dumps({"quick": True, "steps": steps, "ms_per_step": ms_job / steps,
                               "kernels_avg_us": {k: round(1e3 * v[1] / v[0], 2) for k, v in prof.items()},
                               "elementwise_alone_us": {k: round(v, 2) for k, v in ew_us.items()},
-                              "layer_dx_us": round(dx_us, 2), "align_loss_us": round(al_us, 2)}))
+                              "layer_dx_us": round(dx_us, 2), "nvfp4_gemm_us": round(fp4_us, 2),
+                              "align_loss_us": round(al_us, 2)}))
         if sampler:
             sampler.stop()
         if world > 1:
@@ -698,6 +723,14 @@ def run_ours(args):
                            **tensor_fracs(dx_tf, pk),
                            "timed": "20 back-to-back calls (soft weights, transpose and GEMM each), one event pair",
                            "note": "input gradient dX = dY W_soft, not part of a Stage-1 step"}
+    fp4_tf = flops / (fp4_us * 1e-6) / 1e12
+    kernels["nvfp4_gemm"] = {"avg_us": round(fp4_us, 2), "bound": "tensor", "achieved": round(fp4_tf, 1),
+                             "peak": 4.0 * pk["bf16_tflops"], "unit": "TFLOP/s", "frac": round(fp4_tf / (4.0 * pk["bf16_tflops"]), 4),
+                             "frac_nominal": round(fp4_tf / 9000.0, 4),
+                             "peak_note": "measured BF16 burst rate x 4 (the nominal FP4 : BF16 ratio)",
+                             "timed": "20 back-to-back calls, one event pair",
+                             "note": "X_q W_final^T on the packed NVFP4 operands (block-scaled FP4 tensor-core path); a check "
+                                     "of the deployable output, not part of a Stage-1 step"}
     al_bytes = 3.0 * AL_T * AL_V * 2 + 3.0 * AL_T * AL_D * 2          # both logit / hidden tensors read, one gradient written
     kernels["align_loss"] = {"avg_us": round(al_us, 2), "bound": "hbm", "achieved": round(al_bytes / (al_us * 1e-6) / 1e9, 1),
                              "peak": pk["hbm_gbs"], "unit": "GB/s",
