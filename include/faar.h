@@ -417,6 +417,36 @@ FAAR_API int faar_align_loss(faar_ctx* ctx, int T, int vocab, int hidden, const 
 FAAR_API int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales, uint8_t* scales_tiled,
                                  size_t tiled_bytes);
 
+/* ---- element-wise pieces of a decoder block --------------------------------------
+ * Procedure steps 16-23 run the whole quantised model forward and backward; between its linears sit the
+ * block's own operations, which the paper takes from the model family (Llama 3 / Qwen 3).  These calls are
+ * the ones that are not matrix products.  BF16 in and out, FP32 arithmetic; cols (and every leading
+ * dimension) a multiple of 8, bases 16-byte aligned.
+ *
+ * faar_rmsnorm: y = x / sqrt(mean(x^2) + eps) * g over each row.
+ *   x in: [rows, cols] bf16 (ldx)    g in: [cols] float    y out: [rows, cols] bf16 (ldy)
+ *   rstd out: [rows] float = 1 / sqrt(mean(x^2) + eps), kept for the backward call (nullable)
+ * faar_rmsnorm_bwd: gradient towards x (g is frozen): dx = rstd * (g dy - xh * mean(g dy xh)), xh = x rstd;
+ *   `add` ([rows, cols] bf16, ldadd; nullable) is added to it: the gradient that reaches x past the norm, along
+ *   the residual connection.  dx may alias add.
+ * faar_rope: rotary position embedding, half-split pairing: in every head, element i < head_dim/2 pairs with
+ *   element i + head_dim/2 and the pair of row t turns by positions[t] * theta^(-2 i / head_dim); inverse != 0
+ *   turns the other way (the backward pass).  x, y: [rows, n_heads * head_dim]; y may alias x; head_dim % 16 == 0.
+ * faar_silu_mul_bwd: gradients of faar_silu_mul: with s = sigmoid(gate), dgate = dout * up * s * (1 + gate (1 - s)),
+ *   dup = dout * gate * s.  dgate may alias gate and dup may alias up.
+ * faar_embedding: out[t, :] = table[tokens[t], :]; tokens are 32-bit ints on the device; a token outside
+ *   [0, vocab) yields a row of zeros. */
+FAAR_API int faar_rmsnorm(faar_ctx* ctx, int rows, int cols, const void* x, int64_t ldx, const float* g, float eps, void* y,
+                          int64_t ldy, float* rstd);
+FAAR_API int faar_rmsnorm_bwd(faar_ctx* ctx, int rows, int cols, const void* dy, int64_t lddy, const void* x, int64_t ldx,
+                              const float* g, const float* rstd, const void* add, int64_t ldadd, void* dx, int64_t lddx);
+FAAR_API int faar_rope(faar_ctx* ctx, int rows, int n_heads, int head_dim, const void* x, int64_t ldx, const int* positions,
+                       float theta, int inverse, void* y, int64_t ldy);
+FAAR_API int faar_silu_mul_bwd(faar_ctx* ctx, int rows, int cols, const void* dout, int64_t ldd, const void* gate,
+                               int64_t ldg, const void* up, int64_t ldu, void* dgate, int64_t lddg, void* dup, int64_t lddu);
+FAAR_API int faar_embedding(faar_ctx* ctx, int rows, int cols, int vocab, const void* table, int64_t ldt, const int* tokens,
+                            void* out, int64_t ldo);
+
 /* ---- GEMM on the deployable operands -----------------------------------------
  * "Hardening and Inference": the hardened weights are NVFP4 tensors that the hardware multiplies as they
  * are.  This call does that on the block-scaled FP4 tensor-core path: C = (sA sB) A B^T, every element of A

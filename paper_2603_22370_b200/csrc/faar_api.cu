@@ -1,6 +1,7 @@
 // extern "C" entry points of libfaar.so: argument validation, workspace carving,
 // kernel sequencing.  No device memory is allocated here.
 #include <math.h>
+#include <initializer_list>
 #include <new>
 
 #include "faar_internal.cuh"
@@ -80,9 +81,9 @@ struct DeviceGuard {
   }
   ~DeviceGuard() { if (prev >= 0) (void)cudaSetDevice(prev); }
 };
-#define FAAR_DEVICE_GUARD(ctx)        \
-  DeviceGuard g((ctx)->device);       \
-  if (g.err) return cuda_fail((ctx), g.err)
+#define FAAR_DEVICE_GUARD(ctx)                  \
+  DeviceGuard device_guard_((ctx)->device);     \
+  if (device_guard_.err) return cuda_fail((ctx), device_guard_.err)
 
 int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Y_ref,
              const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
@@ -196,6 +197,19 @@ faar_prof_scope::faar_prof_scope(faar_ctx* ctx, int kernel_id) : c(ctx), pair(-1
 faar_prof_scope::~faar_prof_scope() {
   if (pair >= 0) cudaEventRecord(c->prof_events[2 * pair + 1], c->stream);
 }
+
+namespace {
+int check_rows_cols(int rows, int cols, std::initializer_list<int64_t> lds, std::initializer_list<const void*> ptrs) {
+  if (rows <= 0 || cols <= 0 || cols % 8) return FAAR_ERR_SHAPE;
+  for (int64_t ld : lds) {
+    if (ld < cols) return FAAR_ERR_SHAPE;
+    if (ld % 8) return FAAR_ERR_ALIGN;
+  }
+  for (const void* q : ptrs)
+    if (q && !aligned16(q)) return FAAR_ERR_ALIGN;
+  return FAAR_OK;
+}
+}  // namespace
 
 extern "C" {
 
@@ -683,6 +697,57 @@ int faar_nvfp4_gemm(faar_ctx* ctx, int M, int N, int K, const uint8_t* A_packed,
   FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, faar_launch_nvfp4_gemm(ctx, M, N, K, A_packed, A_scales_tiled, A_s_global, B_packed, B_scales_tiled,
                                                B_s_global, C, ldc, reinterpret_cast<uint32_t*>(workspace)));
+}
+
+// ---- element-wise pieces of a decoder block (full-model alignment) -----------------------------------
+int faar_rmsnorm(faar_ctx* ctx, int rows, int cols, const void* x, int64_t ldx, const float* g, float eps, void* y,
+                 int64_t ldy, float* rstd) {
+  if (!ctx || !x || !g || !y) return FAAR_ERR_INVALID_ARG;
+  if (!(eps >= 0.f) || !isfinite(eps)) return FAAR_ERR_INVALID_ARG;
+  int st = check_rows_cols(rows, cols, {ldx, ldy}, {x, g, y});
+  if (st) return st;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_rmsnorm(ctx, rows, cols, x, ldx, g, eps, y, ldy, rstd));
+}
+
+int faar_rmsnorm_bwd(faar_ctx* ctx, int rows, int cols, const void* dy, int64_t lddy, const void* x, int64_t ldx,
+                     const float* g, const float* rstd, const void* add, int64_t ldadd, void* dx, int64_t lddx) {
+  if (!ctx || !dy || !x || !g || !rstd || !dx) return FAAR_ERR_INVALID_ARG;
+  int st = check_rows_cols(rows, cols, {lddy, ldx, lddx}, {dy, x, g, dx, add});
+  if (st) return st;
+  if (add && (ldadd < cols || ldadd % 8)) return ldadd < cols ? FAAR_ERR_SHAPE : FAAR_ERR_ALIGN;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_rmsnorm_bwd(ctx, rows, cols, dy, lddy, x, ldx, g, rstd, add, ldadd, dx, lddx));
+}
+
+int faar_rope(faar_ctx* ctx, int rows, int n_heads, int head_dim, const void* x, int64_t ldx, const int* positions,
+              float theta, int inverse, void* y, int64_t ldy) {
+  if (!ctx || !x || !positions || !y) return FAAR_ERR_INVALID_ARG;
+  if (n_heads <= 0 || head_dim <= 0 || head_dim % 16) return FAAR_ERR_SHAPE;
+  if (!(theta > 1.f) || !isfinite(theta)) return FAAR_ERR_INVALID_ARG;
+  int st = check_rows_cols(rows, n_heads * head_dim, {ldx, ldy}, {x, y});
+  if (st) return st;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_rope(ctx, rows, n_heads, head_dim, x, ldx, positions, theta, inverse, y, ldy));
+}
+
+int faar_silu_mul_bwd(faar_ctx* ctx, int rows, int cols, const void* dout, int64_t ldd, const void* gate, int64_t ldg,
+                      const void* up, int64_t ldu, void* dgate, int64_t lddg, void* dup, int64_t lddu) {
+  if (!ctx || !dout || !gate || !up || !dgate || !dup) return FAAR_ERR_INVALID_ARG;
+  int st = check_rows_cols(rows, cols, {ldd, ldg, ldu, lddg, lddu}, {dout, gate, up, dgate, dup});
+  if (st) return st;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_silu_mul_bwd(ctx, rows, cols, dout, ldd, gate, ldg, up, ldu, dgate, lddg, dup, lddu));
+}
+
+int faar_embedding(faar_ctx* ctx, int rows, int cols, int vocab, const void* table, int64_t ldt, const int* tokens,
+                   void* out, int64_t ldo) {
+  if (!ctx || !table || !tokens || !out) return FAAR_ERR_INVALID_ARG;
+  if (vocab <= 0) return FAAR_ERR_SHAPE;
+  int st = check_rows_cols(rows, cols, {ldt, ldo}, {table, out});
+  if (st) return st;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_embedding(ctx, rows, cols, vocab, table, ldt, tokens, out, ldo));
 }
 
 int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_t* scales, uint8_t* scales_tiled,

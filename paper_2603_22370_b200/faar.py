@@ -55,6 +55,11 @@ SIGNATURES = {
     "faar_align_loss": (_I, [_P, _I, _I, _I, _P, _P, _L, _P, _P, _L, _F, _F, _P, _P, _P, _P, _Z]),
     "faar_swizzle_scales": (_I, [_P, _I, _I, _P, _P, _Z]),
     "faar_silu_mul": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L]),
+    "faar_rmsnorm": (_I, [_P, _I, _I, _P, _L, _P, _F, _P, _L, _P]),
+    "faar_rmsnorm_bwd": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _P, _P, _L, _P, _L]),
+    "faar_rope": (_I, [_P, _I, _I, _I, _P, _L, _P, _F, _I, _P, _L]),
+    "faar_silu_mul_bwd": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L, _P, _L, _P, _L]),
+    "faar_embedding": (_I, [_P, _I, _I, _I, _P, _L, _P, _P, _L]),
     "faar_nvfp4_gemm": (_I, [_P, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _L, _P, _Z]),
 }
 EXPORTS = list(SIGNATURES)
@@ -254,6 +259,29 @@ def swizzle_scales(ctx, rows, cols, scales, scales_tiled):
 
 def silu_mul(ctx, rows, cols, gate, ldg, up, ldu, out, ldo):
     _check(lib().faar_silu_mul(ctx._h, rows, cols, _p(gate), ldg, _p(up), ldu, _p(out), ldo), "faar_silu_mul")
+
+
+def rmsnorm(ctx, rows, cols, x, ldx, g, eps, y, ldy, rstd=None):
+    _check(lib().faar_rmsnorm(ctx._h, rows, cols, _p(x), ldx, _p(g), eps, _p(y), ldy, _p(rstd)), "faar_rmsnorm")
+
+
+def rmsnorm_bwd(ctx, rows, cols, dy, lddy, x, ldx, g, rstd, add, ldadd, dx, lddx):
+    _check(lib().faar_rmsnorm_bwd(ctx._h, rows, cols, _p(dy), lddy, _p(x), ldx, _p(g), _p(rstd), _p(add), ldadd, _p(dx), lddx),
+           "faar_rmsnorm_bwd")
+
+
+def rope(ctx, rows, n_heads, head_dim, x, ldx, positions, theta, inverse, y, ldy):
+    _check(lib().faar_rope(ctx._h, rows, n_heads, head_dim, _p(x), ldx, _p(positions), theta, int(inverse), _p(y), ldy),
+           "faar_rope")
+
+
+def silu_mul_bwd(ctx, rows, cols, dout, ldd, gate, ldg, up, ldu, dgate, lddg, dup, lddu):
+    _check(lib().faar_silu_mul_bwd(ctx._h, rows, cols, _p(dout), ldd, _p(gate), ldg, _p(up), ldu, _p(dgate), lddg, _p(dup),
+                                   lddu), "faar_silu_mul_bwd")
+
+
+def embedding(ctx, rows, cols, vocab, table, ldt, tokens, out, ldo):
+    _check(lib().faar_embedding(ctx._h, rows, cols, vocab, _p(table), ldt, _p(tokens), _p(out), ldo), "faar_embedding")
 
 
 def nvfp4_gemm(ctx, M, N, K, A_packed, A_scales_tiled, A_s_global, B_packed, B_scales_tiled, B_s_global, C, ldc, ws):
