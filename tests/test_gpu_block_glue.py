@@ -39,7 +39,7 @@ def close_bf16(got, ref, extra_abs=0.0):
 def test_rmsnorm_forward_and_backward(ctx, rows, cols, ld):
     rng = np.random.default_rng(rows)
     x = inputs.to_bf16_f32(rng.standard_normal((rows, cols)) * 2)
-    x[0, :] *= 30.0                                                    # a row with a large norm
+    x[0, :] *= 32.0                                                    # a row with a large norm (still BF16 values)
     g = inputs.to_bf16_f32(rng.uniform(0.5, 1.5, cols)).astype(np.float32)
     dy = inputs.to_bf16_f32(rng.standard_normal((rows, cols)))
     res = inputs.to_bf16_f32(rng.standard_normal((rows, cols)))
