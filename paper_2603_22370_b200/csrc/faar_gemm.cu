@@ -221,6 +221,7 @@ struct KParams {
   int bn;                 // tile width
   int n_full_cols;        // tile columns of full width; the columns after them are bn/2 wide (tail split)
   uint32_t* status;
+  long long ext_yout, ext_dyt, ext_state, ext_wsoft;   // bytes of Yout, dYt, each of V / m / u / dV, wsoft_next (debug checks)
   // REF / FWD
   void* Yout; int yout_dtype; long long ldy;
   const void* Yref; int yref_dtype;
@@ -271,6 +272,22 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&p);
 }
 
+// Debug build (-DFAAR_DEBUG): every epilogue store is checked against the extent of the tensor it writes; a
+// store that would leave it is skipped and recorded in the status word (0xD00 | tensor id), which
+// faar_check_status reports.  No trap, no assert: the kernel runs on.  In the normal build the check is gone.
+#ifdef FAAR_DEBUG
+__device__ __forceinline__ bool dbg_in_range(const KParams& p, const void* ptr, long long bytes, const void* base,
+                                             long long extent, uint32_t id) {
+  const long long off = reinterpret_cast<const char*>(ptr) - reinterpret_cast<const char*>(base);
+  if (off >= 0 && off + bytes <= extent) return true;
+  atomicCAS(p.status, 0u, 0xD00u | id);
+  return false;
+}
+#define FAAR_DBG_OK(p, ptr, bytes, base, extent, id) dbg_in_range(p, ptr, bytes, base, extent, id)
+#else
+#define FAAR_DBG_OK(p, ptr, bytes, base, extent, id) true
+#endif
+
 // ---- epilogues: one call handles 16 accumulator columns of one row ---------------------------
 // REF: write acc to Y[t, o].
 __device__ __forceinline__ void epi_ref(const KParams& p, int o, int t0, const uint32_t (&acc)[16]) {
@@ -282,10 +299,12 @@ __device__ __forceinline__ void epi_ref(const KParams& p, int o, int t0, const u
       float a[16];
 #pragma unroll
       for (int j = 0; j < 16; ++j) a[j] = (t0 + j < p.N) ? __uint_as_float(acc[j]) : 0.f;
+      if (!FAAR_DBG_OK(p, d4, 32, p.Yout, p.ext_yout, 1u)) return;
       d4[0] = make_uint4(pack_bf16x2(a[0], a[1]), pack_bf16x2(a[2], a[3]), pack_bf16x2(a[4], a[5]), pack_bf16x2(a[6], a[7]));
       d4[1] = make_uint4(pack_bf16x2(a[8], a[9]), pack_bf16x2(a[10], a[11]), pack_bf16x2(a[12], a[13]), pack_bf16x2(a[14], a[15]));
     } else {
       float4* d4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.Yout) + (long long)o * p.ldy + t0);
+      if (!FAAR_DBG_OK(p, d4, 64, p.Yout, p.ext_yout, 1u)) return;
 #pragma unroll
       for (int q = 0; q < 4; ++q)
         d4[q] = make_float4((t0 + 4 * q < p.N) ? __uint_as_float(acc[4 * q]) : 0.f,
@@ -300,10 +319,13 @@ __device__ __forceinline__ void epi_ref(const KParams& p, int o, int t0, const u
     int t = t0 + j;
     if (t < p.N) {
       float a = __uint_as_float(acc[j]);
-      if (p.yout_dtype == FAAR_BF16)
-        reinterpret_cast<__nv_bfloat16*>(p.Yout)[(long long)t * p.ldy + o] = __float2bfloat16_rn(a);
-      else
-        reinterpret_cast<float*>(p.Yout)[(long long)t * p.ldy + o] = a;
+      if (p.yout_dtype == FAAR_BF16) {
+        __nv_bfloat16* q = reinterpret_cast<__nv_bfloat16*>(p.Yout) + (long long)t * p.ldy + o;
+        if (FAAR_DBG_OK(p, q, 2, p.Yout, p.ext_yout, 1u)) *q = __float2bfloat16_rn(a);
+      } else {
+        float* q = reinterpret_cast<float*>(p.Yout) + (long long)t * p.ldy + o;
+        if (FAAR_DBG_OK(p, q, 4, p.Yout, p.ext_yout, 1u)) *q = a;
+      }
     }
   }
 }
@@ -352,6 +374,7 @@ __device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const 
     dy[j] = p.mse2c * r;
   }
   __nv_bfloat16* drow = p.dYt + (long long)o * p.ld_dyt + t0;
+  if (!FAAR_DBG_OK(p, drow, 2 * (t0 + 16 <= p.N ? 16 : p.N - t0), p.dYt, p.ext_dyt, 2u)) return ss;
   if (t0 + 16 <= p.N) {
     uint4* d4 = reinterpret_cast<uint4*>(drow);
     d4[0] = make_uint4(pack_bf16x2(dy[0], dy[1]), pack_bf16x2(dy[2], dy[3]), pack_bf16x2(dy[4], dy[5]), pack_bf16x2(dy[6], dy[7]));
@@ -365,9 +388,10 @@ __device__ __forceinline__ float epi_fwd(const KParams& p, int o, int t0, const 
     __nv_bfloat16* yq = reinterpret_cast<__nv_bfloat16*>(p.Yout);
 #pragma unroll
     for (int j = 0; j < 16; ++j)
-      if (t0 + j < p.N)
-        yq[p.yref_t ? (long long)o * p.ldy + t0 + j : (long long)(t0 + j) * p.ldy + o] =
-            __float2bfloat16_rn(__uint_as_float(acc[j]) * p.act_scale);
+      if (t0 + j < p.N) {
+        __nv_bfloat16* q = yq + (p.yref_t ? (long long)o * p.ldy + t0 + j : (long long)(t0 + j) * p.ldy + o);
+        if (FAAR_DBG_OK(p, q, 2, p.Yout, p.ext_yout, 1u)) *q = __float2bfloat16_rn(__uint_as_float(acc[j]) * p.act_scale);
+      }
   }
   return ss;
 }
@@ -508,6 +532,9 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
             wn[j] = __uint_as_float(__float_as_uint(mag) ^ sgn);
           }
         }
+        // one check covers the five stores below: they share the element offset e0 + off
+        if (!FAAR_DBG_OK(p, Vp + off, 16, p.V, p.ext_state, 3u)) continue;
+        if ((OPT & 2) && !FAAR_DBG_OK(p, p.wsoft_next + e0 + off, 8, p.wsoft_next, p.ext_wsoft, 4u)) continue;
         if (OPT & 2)
           *reinterpret_cast<uint2*>(p.wsoft_next + e0 + off) = make_uint2(pack_bf16x2(wn[0], wn[1]), pack_bf16x2(wn[2], wn[3]));
         if (p.dV) stg128_stream(p.dV + e0 + off, g[0], g[1], g[2], g[3], stream);
@@ -973,6 +1000,15 @@ int faar_gemm_max_partials(const faar_ctx* ctx, int, int) { return ctx->num_sms 
 int faar_launch_gemm(faar_ctx* ctx, const faar_gemm_args* a, int* n_partials_out) {
   KParams kp;
   kp.M = a->M; kp.N = a->N; kp.Kc = a->Kc; kp.bn = BN_MAX; kp.n_full_cols = 0; kp.status = a->status;
+  {
+    const long long ysz = a->yout_dtype == FAAR_BF16 ? 2 : 4;
+    // Y is [N(T), ldy] or, transposed, [M(O), ldy]; the last row ends after its last valid (or padded) column
+    kp.ext_yout = a->Yout ? (a->yref_t ? ((long long)(a->M - 1) * a->ldy + (a->N + 15) / 16 * 16)
+                                       : ((long long)(a->N - 1) * a->ldy + a->M)) * ysz : 0;
+    kp.ext_dyt = a->dYt ? ((long long)(a->M - 1) * a->ld_dyt + a->N) * 2 : 0;
+    kp.ext_state = (long long)a->M * a->N * 4;
+    kp.ext_wsoft = (long long)a->M * a->N * 2;
+  }
   kp.Yout = a->Yout; kp.yout_dtype = a->yout_dtype; kp.ldy = a->ldy;
   kp.Yref = a->Yref; kp.yref_dtype = a->yref_dtype; kp.yref_t = a->yref_t;
   kp.dYt = a->dYt; kp.ld_dyt = a->ld_dyt; kp.mse2c = a->mse2c; kp.act_scale = a->act_scale; kp.partials = a->partials;

@@ -11,7 +11,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libfaar.so")
+#: the library this process binds: libfaar.so next to this file, or the file FAAR_LIB names (the debug build)
+LIB_PATH = os.environ.get("FAAR_LIB") or os.path.join(_HERE, "libfaar.so")
 
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_DTYPE, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(9)
 BF16, F32 = 0, 1

@@ -80,3 +80,11 @@ def test_binding_declares_argument_types_for_every_export(lib):
         fn = getattr(lib, name)
         assert fn.argtypes is not None and len(fn.argtypes) == n_params, (name, n_params, fn.argtypes)
         assert fn.restype is not None
+
+
+def test_debug_build_exports_the_same_symbols():
+    """The bounds-checking build (-DFAAR_DEBUG) is the same library with checked epilogue stores."""
+    path = faar_build.build(debug=True)
+    dbg = C.CDLL(path)
+    for n in declared_symbols():
+        assert hasattr(dbg, n), n
