@@ -192,7 +192,8 @@ enum {
   FAAR_K_ALIGN_LOSS = 11,    /* Eq. 6: KL of the softmaxes + last-hidden error, gradients */
   FAAR_K_GLUE = 12,          /* element-wise pieces of a decoder block between the linears */
   FAAR_K_NVFP4_GEMM = 13,    /* block-scaled FP4 GEMM on the deployable operands            */
-  FAAR_K_COUNT = 14
+  FAAR_K_ATTENTION = 14,     /* causal attention, forward or backward                       */
+  FAAR_K_COUNT = 15
 };
 typedef struct {
   int kernel;     /* one of FAAR_K_*          */
@@ -446,6 +447,28 @@ FAAR_API int faar_silu_mul_bwd(faar_ctx* ctx, int rows, int cols, const void* do
                                int64_t ldg, const void* up, int64_t ldu, void* dgate, int64_t lddg, void* dup, int64_t lddu);
 FAAR_API int faar_embedding(faar_ctx* ctx, int rows, int cols, int vocab, const void* table, int64_t ldt, const int* tokens,
                             void* out, int64_t ldo);
+
+/* faar_add: out = a + b, element-wise on [rows, cols] BF16 matrices (residual connections; gradients that meet
+ * at one tensor).  out may alias a or b. */
+FAAR_API int faar_add(faar_ctx* ctx, int rows, int cols, const void* a, int64_t lda, const void* b, int64_t ldb, void* out,
+                      int64_t ldo);
+
+/* ---- attention of a decoder block -------------------------------------------------
+ * Procedure steps 16-23 again: the model family's causal softmax attention with grouped key/value heads sits
+ * between a block's q/k/v projections and its output projection, and Eq. 6's gradient passes through it.
+ *   out[t, h, :] = sum over u <= t of the same sequence of softmax_u(q[t, h, :] . k[u, g, :] / sqrt(head_dim)) v[u, g, :]
+ * with g = h / (n_heads / n_kv_heads).  Tokens of a sequence are contiguous rows: row = sequence * seq + position.
+ *   q in: [batch*seq, n_heads*head_dim] bf16 (ldq)     k, v in: [batch*seq, n_kv_heads*head_dim] bf16 (ldkv)
+ *   out: [batch*seq, n_heads*head_dim] bf16 (ldo)      lse out: [batch, n_heads, seq] float, log2 of each row's
+ *   sum of 2^(score log2 e / sqrt(head_dim)): what the backward call recomputes the probabilities from.
+ * faar_attention_bwd: from dout (layout of out) to dq (layout of q), dk, dv (layout of k, v); out and lse are the
+ * forward call's; dsum is scratch, [batch, n_heads, seq] floats.  No matrix of seq x seq values is stored; results
+ * are reproducible (no atomics).  head_dim is 64 or 128; leading dimensions multiples of 8, bases 16-byte aligned. */
+FAAR_API int faar_attention_fwd(faar_ctx* ctx, int batch, int seq, int n_heads, int n_kv_heads, int head_dim, const void* q,
+                                int64_t ldq, const void* k, const void* v, int64_t ldkv, void* out, int64_t ldo, float* lse);
+FAAR_API int faar_attention_bwd(faar_ctx* ctx, int batch, int seq, int n_heads, int n_kv_heads, int head_dim, const void* q,
+                                int64_t ldq, const void* k, const void* v, int64_t ldkv, const void* out, const void* dout,
+                                int64_t ldo, const float* lse, float* dsum, void* dq, void* dk, void* dv);
 
 /* ---- GEMM on the deployable operands -----------------------------------------
  * "Hardening and Inference": the hardened weights are NVFP4 tensors that the hardware multiplies as they

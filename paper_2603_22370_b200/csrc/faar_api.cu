@@ -209,6 +209,15 @@ int check_rows_cols(int rows, int cols, std::initializer_list<int64_t> lds, std:
     if (q && !aligned16(q)) return FAAR_ERR_ALIGN;
   return FAAR_OK;
 }
+int check_attention(int batch, int seq, int n_heads, int n_kv_heads, int head_dim, int64_t ldq, int64_t ldkv, int64_t ldo) {
+  if (batch <= 0 || seq <= 0 || n_heads <= 0 || n_kv_heads <= 0 || n_heads % n_kv_heads) return FAAR_ERR_SHAPE;
+  if (head_dim != 64 && head_dim != 128) return FAAR_ERR_SHAPE;
+  if ((long long)batch * seq > 0x7FFFFFFFll) return FAAR_ERR_SHAPE;
+  if (ldq < (int64_t)n_heads * head_dim || ldo < (int64_t)n_heads * head_dim || ldkv < (int64_t)n_kv_heads * head_dim)
+    return FAAR_ERR_SHAPE;
+  if (ldq % 8 || ldkv % 8 || ldo % 8) return FAAR_ERR_ALIGN;
+  return FAAR_OK;
+}
 }  // namespace
 
 extern "C" {
@@ -295,6 +304,7 @@ const char* faar_kernel_name(int kernel) {
     case FAAR_K_ALIGN_LOSS: return "align_loss";
     case FAAR_K_GLUE: return "glue";
     case FAAR_K_NVFP4_GEMM: return "nvfp4_gemm";
+    case FAAR_K_ATTENTION: return "attention";
   }
   return "unknown";
 }
@@ -738,6 +748,39 @@ int faar_silu_mul_bwd(faar_ctx* ctx, int rows, int cols, const void* dout, int64
   if (st) return st;
   FAAR_DEVICE_GUARD(ctx);
   return cuda_fail(ctx, faar_launch_silu_mul_bwd(ctx, rows, cols, dout, ldd, gate, ldg, up, ldu, dgate, lddg, dup, lddu));
+}
+
+int faar_add(faar_ctx* ctx, int rows, int cols, const void* a, int64_t lda, const void* b, int64_t ldb, void* out,
+             int64_t ldo) {
+  if (!ctx || !a || !b || !out) return FAAR_ERR_INVALID_ARG;
+  int st = check_rows_cols(rows, cols, {lda, ldb, ldo}, {a, b, out});
+  if (st) return st;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_add(ctx, rows, cols, a, lda, b, ldb, out, ldo));
+}
+
+int faar_attention_fwd(faar_ctx* ctx, int batch, int seq, int n_heads, int n_kv_heads, int head_dim, const void* q,
+                       int64_t ldq, const void* k, const void* v, int64_t ldkv, void* out, int64_t ldo, float* lse) {
+  if (!ctx || !q || !k || !v || !out || !lse) return FAAR_ERR_INVALID_ARG;
+  int st = check_attention(batch, seq, n_heads, n_kv_heads, head_dim, ldq, ldkv, ldo);
+  if (st) return st;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return FAAR_ERR_ALIGN;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_attention_fwd(ctx, batch, seq, n_heads, n_kv_heads, head_dim, q, ldq, k, v, ldkv, out, ldo, lse));
+}
+
+int faar_attention_bwd(faar_ctx* ctx, int batch, int seq, int n_heads, int n_kv_heads, int head_dim, const void* q,
+                       int64_t ldq, const void* k, const void* v, int64_t ldkv, const void* out, const void* dout,
+                       int64_t ldo, const float* lse, float* dsum, void* dq, void* dk, void* dv) {
+  if (!ctx || !q || !k || !v || !out || !dout || !lse || !dsum || !dq || !dk || !dv) return FAAR_ERR_INVALID_ARG;
+  int st = check_attention(batch, seq, n_heads, n_kv_heads, head_dim, ldq, ldkv, ldo);
+  if (st) return st;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(dout) || !aligned16(dq) ||
+      !aligned16(dk) || !aligned16(dv))
+    return FAAR_ERR_ALIGN;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_attention_bwd(ctx, batch, seq, n_heads, n_kv_heads, head_dim, q, ldq, k, v, ldkv, out,
+                                                  dout, ldo, lse, dsum, dq, dk, dv));
 }
 
 int faar_embedding(faar_ctx* ctx, int rows, int cols, int vocab, const void* table, int64_t ldt, const int* tokens,

@@ -197,6 +197,24 @@ embedding_kernel(const __nv_bfloat16* __restrict__ table, int64_t ldt, const int
   }
 }
 
+// ---- out = a + b (residual connections and the sums of gradients that meet at one tensor) -----------
+__global__ void __launch_bounds__(GL_THREADS)
+add_kernel(const __nv_bfloat16* __restrict__ a, int64_t lda, const __nv_bfloat16* __restrict__ b, int64_t ldb,
+           __nv_bfloat16* __restrict__ out, int64_t ldo, int rows, int cols) {
+  const uint32_t groups_per_row = cols / 8;
+  const int64_t total = (int64_t)rows * groups_per_row;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t row = t / groups_per_row;
+    const int col = (int)(t - row * groups_per_row) * 8;
+    float x[8], y[8], o[8];
+    unpack8(*reinterpret_cast<const uint4*>(a + row * lda + col), x);
+    unpack8(*reinterpret_cast<const uint4*>(b + row * ldb + col), y);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] = x[i] + y[i];
+    *reinterpret_cast<uint4*>(out + row * ldo + col) = pack8(o);
+  }
+}
+
 int glue_grid(const faar_ctx* ctx, int64_t items) {
   int64_t blocks = (items + GL_THREADS - 1) / GL_THREADS;
   const int64_t cap = (int64_t)ctx->num_sms * 8;
@@ -256,5 +274,14 @@ int faar_launch_embedding(faar_ctx* ctx, int rows, int cols, int vocab, const vo
   faar_prof_scope ps(ctx, FAAR_K_GLUE);
   embedding_kernel<<<glue_grid(ctx, (int64_t)rows * (cols / 8)), GL_THREADS, 0, ctx->stream>>>(
       reinterpret_cast<const __nv_bfloat16*>(table), ldt, tokens, vocab, reinterpret_cast<__nv_bfloat16*>(out), ldo, rows, cols);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_add(faar_ctx* ctx, int rows, int cols, const void* a, int64_t lda, const void* b, int64_t ldb, void* out,
+                    int64_t ldo) {
+  faar_prof_scope ps(ctx, FAAR_K_GLUE);
+  add_kernel<<<glue_grid(ctx, (int64_t)rows * (cols / 8)), GL_THREADS, 0, ctx->stream>>>(
+      reinterpret_cast<const __nv_bfloat16*>(a), lda, reinterpret_cast<const __nv_bfloat16*>(b), ldb,
+      reinterpret_cast<__nv_bfloat16*>(out), ldo, rows, cols);
   return (int)cudaGetLastError();
 }

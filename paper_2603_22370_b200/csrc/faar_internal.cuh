@@ -108,6 +108,13 @@ int faar_launch_silu_mul_bwd(faar_ctx*, int rows, int cols, const void* dout, in
                              const void* up, int64_t ldu, void* dgate, int64_t lddg, void* dup, int64_t lddu);
 int faar_launch_embedding(faar_ctx*, int rows, int cols, int vocab, const void* table, int64_t ldt, const int* tokens,
                           void* out, int64_t ldo);
+int faar_launch_add(faar_ctx*, int rows, int cols, const void* a, int64_t lda, const void* b, int64_t ldb, void* out,
+                    int64_t ldo);
+int faar_launch_attention_fwd(faar_ctx*, int B, int S, int H, int Hkv, int D, const void* q, int64_t ldq, const void* k,
+                              const void* v, int64_t ldk, void* out, int64_t ldo, float* lse);
+int faar_launch_attention_bwd(faar_ctx*, int B, int S, int H, int Hkv, int D, const void* q, int64_t ldq, const void* k,
+                              const void* v, int64_t ldk, const void* out, const void* dout, int64_t ldo, const float* lse,
+                              float* dsum, void* dq, void* dk, void* dv);
 int faar_launch_nvfp4_gemm(faar_ctx*, int M, int N, int K, const uint8_t* A, const uint8_t* sfa, const float* sa,
                            const uint8_t* B, const uint8_t* sfb, const float* sb, void* C, int64_t ldc, uint32_t* status);
 int faar_launch_round_partials(faar_ctx*, const float* V, int64_t N, float* partials, int* n_partials);

@@ -61,6 +61,9 @@ SIGNATURES = {
     "faar_rope": (_I, [_P, _I, _I, _I, _P, _L, _P, _F, _I, _P, _L]),
     "faar_silu_mul_bwd": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L, _P, _L, _P, _L]),
     "faar_embedding": (_I, [_P, _I, _I, _I, _P, _L, _P, _P, _L]),
+    "faar_add": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L]),
+    "faar_attention_fwd": (_I, [_P, _I, _I, _I, _I, _I, _P, _L, _P, _P, _L, _P, _L, _P]),
+    "faar_attention_bwd": (_I, [_P, _I, _I, _I, _I, _I, _P, _L, _P, _P, _L, _P, _P, _L, _P, _P, _P, _P, _P]),
     "faar_nvfp4_gemm": (_I, [_P, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _L, _P, _Z]),
 }
 EXPORTS = list(SIGNATURES)
@@ -283,6 +286,20 @@ def silu_mul_bwd(ctx, rows, cols, dout, ldd, gate, ldg, up, ldu, dgate, lddg, du
 
 def embedding(ctx, rows, cols, vocab, table, ldt, tokens, out, ldo):
     _check(lib().faar_embedding(ctx._h, rows, cols, vocab, _p(table), ldt, _p(tokens), _p(out), ldo), "faar_embedding")
+
+
+def add(ctx, rows, cols, a, lda, b, ldb, out, ldo):
+    _check(lib().faar_add(ctx._h, rows, cols, _p(a), lda, _p(b), ldb, _p(out), ldo), "faar_add")
+
+
+def attention_fwd(ctx, batch, seq, n_heads, n_kv_heads, head_dim, q, ldq, k, v, ldkv, out, ldo, lse):
+    _check(lib().faar_attention_fwd(ctx._h, batch, seq, n_heads, n_kv_heads, head_dim, _p(q), ldq, _p(k), _p(v), ldkv,
+                                    _p(out), ldo, _p(lse)), "faar_attention_fwd")
+
+
+def attention_bwd(ctx, batch, seq, n_heads, n_kv_heads, head_dim, q, ldq, k, v, ldkv, out, dout, ldo, lse, dsum, dq, dk, dv):
+    _check(lib().faar_attention_bwd(ctx._h, batch, seq, n_heads, n_kv_heads, head_dim, _p(q), ldq, _p(k), _p(v), ldkv,
+                                    _p(out), _p(dout), ldo, _p(lse), _p(dsum), _p(dq), _p(dk), _p(dv)), "faar_attention_bwd")
 
 
 def nvfp4_gemm(ctx, M, N, K, A_packed, A_scales_tiled, A_s_global, B_packed, B_scales_tiled, B_s_global, C, ldc, ws):
