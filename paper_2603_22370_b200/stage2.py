@@ -1,0 +1,242 @@
+"""Stage-2 driver: full-model alignment (Eq. 6, Procedure steps 15-24) of a Llama-style decoder model whose
+linears all carry their own rounding tensor V.  Host loop and buffer management only: every arithmetic step --
+embedding, norms, rotary embedding, attention, the gated MLP, every matrix product, the loss with its gradients,
+the chain rule into V, the optimiser update -- is a call into the CUDA library through `faar`.
+
+One step (`Stage2Model.step`):
+  frozen model forward (BF16 weights)                      -> Z_fp, H_fp            Procedure 16
+  quantised model forward (Eq. 2 soft weights of every V)  -> Z_q, H_q, activations Procedure 17
+  faar_align_loss                                          -> L_KL, L_MSE, dZ_q, dH_q   Procedure 18-20, Eq. 6
+  backward through the quantised model; per linear: input gradient dX = dY W_soft (faar_layer_dx, at the
+  pre-update V), then dW GEMM + chain rule + Round Loss gradient + optimiser update + clip (faar_layer_bwd)
+                                                                                     Procedure 21-23
+Embedding, norms and LM head are frozen and stay in BF16 / FP32; the seven linears of every block are quantised.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import torch
+
+from . import faar
+
+LINEARS = ("q_proj", "k_proj", "v_proj", "o_proj", "gate_proj", "up_proj", "down_proj")
+
+
+@dataclass
+class ModelConfig:
+    vocab: int
+    hidden: int
+    n_layers: int
+    n_heads: int
+    n_kv_heads: int
+    head_dim: int
+    ffn: int
+    eps: float = 1e-5
+    theta: float = 10000.0
+
+    def linear_shapes(self) -> dict:
+        d, q, kv, f = self.hidden, self.n_heads * self.head_dim, self.n_kv_heads * self.head_dim, self.ffn
+        return {"q_proj": (q, d), "k_proj": (kv, d), "v_proj": (kv, d), "o_proj": (d, q),
+                "gate_proj": (f, d), "up_proj": (f, d), "down_proj": (d, f)}
+
+
+class QuantLinear:
+    """Device state of one quantised linear: frozen W, its NVFP4 bracket (scales, code, tensor scale), the
+    rounding tensor V with its Adam moments, and a BF16 buffer for the soft weights of the current step."""
+
+    def __init__(self, ctx: faar.Context, W: torch.Tensor, ws: torch.Tensor, opt: int = 1):
+        O, K = W.shape
+        dev = W.device
+        self.W, self.O, self.K = W, O, K
+        self.scales = torch.empty((O, K // 16), dtype=torch.uint8, device=dev)
+        self.code = torch.empty((O, K // 2), dtype=torch.uint8, device=dev)
+        self.s_global = torch.empty(1, dtype=torch.float32, device=dev)
+        self.V = torch.empty((O, K), dtype=torch.float32, device=dev)
+        self.m = torch.zeros((O, K), dtype=torch.float32, device=dev) if opt == 1 else None
+        self.u = torch.zeros((O, K), dtype=torch.float32, device=dev) if opt == 1 else None
+        self.Wsoft = torch.empty((O, K), dtype=torch.bfloat16, device=dev)
+        faar.softquant_init(ctx, faar.make_shape(O, K, 8), W, 0.0, self.scales, self.s_global, self.code, self.V, ws)
+
+
+class Stage2Model:
+    """A decoder model on one GPU.  params: "embed" [vocab, hidden] bf16, "lm_head" [vocab, hidden] bf16,
+    "final_norm", "attn_norm.l", "mlp_norm.l" [hidden] float32; weights[l][name]: [O, K] bf16 (frozen)."""
+
+    def __init__(self, ctx: faar.Context, cfg: ModelConfig, params: dict, weights: list, batch: int, seq: int, opt: int = 1):
+        self.ctx, self.cfg, self.params, self.opt = ctx, cfg, params, opt
+        self.batch, self.seq, self.T = batch, seq, batch * seq
+        assert cfg.vocab % 16 == 0 and cfg.hidden % 16 == 0 and cfg.ffn % 16 == 0 and cfg.head_dim in (64, 128)
+        dev = params["embed"].device
+        self.dev = dev
+        T, c = self.T, cfg
+        big = max(o * k for o, k in c.linear_shapes().values())
+        self.ws = torch.empty(max(faar.workspace_size(faar.make_shape(o, k, T)) for o, k in c.linear_shapes().values()),
+                              dtype=torch.uint8, device=dev)
+        faar.workspace_init(ctx, self.ws)
+        self.lin = [{n: QuantLinear(ctx, weights[l][n], self.ws, opt) for n in LINEARS} for l in range(c.n_layers)]
+        self.pos = torch.arange(seq, dtype=torch.int32, device=dev).repeat(batch)
+        self.lm_head_t = torch.empty((c.hidden, (c.vocab + 7) // 8 * 8), dtype=torch.bfloat16, device=dev)
+        faar.transpose_bf16(ctx, c.vocab, c.hidden, params["lm_head"], c.hidden, self.lm_head_t, self.lm_head_t.shape[1])
+        self.aws = torch.empty(faar.align_loss_workspace_size(T, c.vocab), dtype=torch.uint8, device=dev)
+        faar.workspace_init(ctx, self.aws)
+        self.loss = torch.zeros(2, dtype=torch.float32, device=dev)
+        # scratch shared by all linears' backward passes
+        k_max = max(k for _, k in c.linear_shapes().values())
+        o_max = max(o for o, _ in c.linear_shapes().values())
+        self.ldt = (T + 7) // 8 * 8
+        self.Xt = torch.empty(k_max * self.ldt, dtype=torch.bfloat16, device=dev)
+        self.dYt = torch.empty(o_max * self.ldt, dtype=torch.bfloat16, device=dev)
+        self.WsT = torch.empty(big + 8 * k_max, dtype=torch.bfloat16, device=dev)
+        self.dsum = torch.empty((batch, c.n_heads, seq), dtype=torch.float32, device=dev)
+        self.step_count = 0
+
+    # ---- helpers ------------------------------------------------------------------------------------
+    def _new(self, cols, dtype=torch.bfloat16):
+        return torch.empty((self.T, cols), dtype=dtype, device=self.dev)
+
+    def _matmul(self, X, W):
+        """Y[T, O] = X[T, K] W[O, K]^T on the tensor cores (the frozen-target GEMM)."""
+        O, K = W.shape
+        Y = self._new(O)
+        faar.layer_ref(self.ctx, faar.make_shape(O, K, self.T), X, W, Y, self.ws)
+        return Y
+
+    def _linear(self, l, name, X, quantised, beta):
+        lin = self.lin[l][name]
+        if not quantised:
+            return self._matmul(X, lin.W)
+        faar.softquant_eval(self.ctx, faar.make_shape(lin.O, lin.K, self.T), lin.V, lin.code, lin.scales, lin.s_global, beta,
+                            None, None, lin.Wsoft)
+        return self._matmul(X, lin.Wsoft)
+
+    # ---- forward -------------------------------------------------------------------------------------
+    def forward(self, tokens: torch.Tensor, quantised: bool, beta: float = 4.0, keep: bool = False):
+        """tokens: [batch*seq] int32 on the device.  Returns (Z [T, vocab], H [T, hidden], cache or None)."""
+        c, ctx, T = self.cfg, self.ctx, self.T
+        d, qd, kvd, f = c.hidden, c.n_heads * c.head_dim, c.n_kv_heads * c.head_dim, c.ffn
+        x = self._new(d)
+        faar.embedding(ctx, T, d, c.vocab, self.params["embed"], d, tokens, x, d)
+        cache = []
+        for l in range(c.n_layers):
+            s = {"x_in": x}
+            hn, s["rstd1"] = self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
+            faar.rmsnorm(ctx, T, d, x, d, self.params[f"attn_norm.{l}"], c.eps, hn, d, s["rstd1"])
+            q, k, v = (self._linear(l, n, hn, quantised, beta) for n in ("q_proj", "k_proj", "v_proj"))
+            faar.rope(ctx, T, c.n_heads, c.head_dim, q, qd, self.pos, c.theta, 0, q, qd)
+            faar.rope(ctx, T, c.n_kv_heads, c.head_dim, k, kvd, self.pos, c.theta, 0, k, kvd)
+            a = self._new(qd)
+            lse = torch.empty((self.batch, c.n_heads, self.seq), dtype=torch.float32, device=self.dev)
+            faar.attention_fwd(ctx, self.batch, self.seq, c.n_heads, c.n_kv_heads, c.head_dim, q, qd, k, v, kvd, a, qd, lse)
+            o = self._linear(l, "o_proj", a, quantised, beta)
+            x_mid = self._new(d)
+            faar.add(ctx, T, d, x, d, o, d, x_mid, d)
+            mn, s["rstd2"] = self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
+            faar.rmsnorm(ctx, T, d, x_mid, d, self.params[f"mlp_norm.{l}"], c.eps, mn, d, s["rstd2"])
+            g, u = self._linear(l, "gate_proj", mn, quantised, beta), self._linear(l, "up_proj", mn, quantised, beta)
+            act = self._new(f)
+            faar.silu_mul(ctx, T, f, g, f, u, f, act, f)
+            dn = self._linear(l, "down_proj", act, quantised, beta)
+            x = self._new(d)
+            faar.add(ctx, T, d, x_mid, d, dn, d, x, d)
+            if keep:
+                s.update(hn=hn, q=q, k=k, v=v, a=a, lse=lse, x_mid=x_mid, mn=mn, g=g, u=u, act=act)
+                cache.append(s)
+        H, rstd_f = self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
+        faar.rmsnorm(ctx, T, d, x, d, self.params["final_norm"], c.eps, H, d, rstd_f)
+        Z = self._matmul(H, self.params["lm_head"])
+        return Z, H, ((cache, x, rstd_f) if keep else None)
+
+    # ---- backward ------------------------------------------------------------------------------------
+    def _linear_bwd(self, l, name, dY, X, hp, want_dv):
+        """One quantised linear: dX = dY W_soft at the pre-update V, then the dW GEMM with the chain rule into V,
+        the Round Loss gradient, the optimiser update and the clip.  Returns (dX, dV or None)."""
+        lin, T, ctx = self.lin[l][name], self.T, self.ctx
+        O, K = lin.O, lin.K
+        shape = faar.make_shape(O, K, T, ldxt=self.ldt)
+        dX = self._new(K)
+        faar.layer_dx(ctx, shape, hp.beta, dY, lin.V, lin.code, lin.scales, lin.s_global, self.WsT, dX, self.ws)
+        faar.transpose_bf16(ctx, T, O, dY, O, self.dYt, self.ldt)
+        faar.transpose_bf16(ctx, T, K, X, K, self.Xt, self.ldt)
+        dV = torch.empty((O, K), dtype=torch.float32, device=self.dev) if want_dv else None
+        faar.layer_bwd(ctx, shape, hp, self.dYt, self.Xt, lin.V, lin.code, lin.scales, lin.s_global, lin.m, lin.u, dV, self.ws)
+        return dX, dV
+
+    def backward(self, dZ, dH, saved, hp, want_dv=False):
+        """From the loss gradients at the logits and at the last hidden state back to every V (updated in place).
+        Returns {(l, name): dV} if want_dv."""
+        c, ctx, T = self.cfg, self.ctx, self.T
+        d, qd, kvd, f = c.hidden, c.n_heads * c.head_dim, c.n_kv_heads * c.head_dim, c.ffn
+        cache, x_last, rstd_f = saved
+        grads = {}
+        # LM head (frozen): dH += dZ W_lm, then the final norm
+        dHz = self._new(d)
+        faar.layer_ref(ctx, faar.make_shape(d, self.lm_head_t.shape[1], T, ldw=self.lm_head_t.shape[1], ldx=dZ.shape[1]), dZ,
+                       self.lm_head_t, dHz, self.ws)
+        faar.add(ctx, T, d, dHz, d, dH, d, dHz, d)
+        dx = self._new(d)
+        faar.rmsnorm_bwd(ctx, T, d, dHz, d, x_last, d, self.params["final_norm"], rstd_f, None, d, dx, d)
+        for l in reversed(range(c.n_layers)):
+            s = cache[l]
+            # MLP branch: x = x_mid + act W_down^T
+            dact, grads[(l, "down_proj")] = self._linear_bwd(l, "down_proj", dx, s["act"], hp, want_dv)
+            dg, du = self._new(f), self._new(f)
+            faar.silu_mul_bwd(ctx, T, f, dact, f, s["g"], f, s["u"], f, dg, f, du, f)
+            dmn, grads[(l, "gate_proj")] = self._linear_bwd(l, "gate_proj", dg, s["mn"], hp, want_dv)
+            dmn2, grads[(l, "up_proj")] = self._linear_bwd(l, "up_proj", du, s["mn"], hp, want_dv)
+            faar.add(ctx, T, d, dmn, d, dmn2, d, dmn, d)
+            faar.rmsnorm_bwd(ctx, T, d, dmn, d, s["x_mid"], d, self.params[f"mlp_norm.{l}"], s["rstd2"], dx, d, dx, d)
+            # attention branch: x_mid = x_in + a W_o^T
+            da, grads[(l, "o_proj")] = self._linear_bwd(l, "o_proj", dx, s["a"], hp, want_dv)
+            dq, dk, dv = self._new(qd), self._new(kvd), self._new(kvd)
+            faar.attention_bwd(ctx, self.batch, self.seq, c.n_heads, c.n_kv_heads, c.head_dim, s["q"], qd, s["k"], s["v"], kvd,
+                               s["a"], da, qd, s["lse"], self.dsum, dq, dk, dv)
+            faar.rope(ctx, T, c.n_heads, c.head_dim, dq, qd, self.pos, c.theta, 1, dq, qd)
+            faar.rope(ctx, T, c.n_kv_heads, c.head_dim, dk, kvd, self.pos, c.theta, 1, dk, kvd)
+            dhn, grads[(l, "q_proj")] = self._linear_bwd(l, "q_proj", dq, s["hn"], hp, want_dv)
+            dhk, grads[(l, "k_proj")] = self._linear_bwd(l, "k_proj", dk, s["hn"], hp, want_dv)
+            dhv, grads[(l, "v_proj")] = self._linear_bwd(l, "v_proj", dv, s["hn"], hp, want_dv)
+            faar.add(ctx, T, d, dhn, d, dhk, d, dhn, d)
+            faar.add(ctx, T, d, dhn, d, dhv, d, dhn, d)
+            faar.rmsnorm_bwd(ctx, T, d, dhn, d, s["x_in"], d, self.params[f"attn_norm.{l}"], s["rstd1"], dx, d, dx, d)
+        return grads if want_dv else None
+
+    # ---- one step of Eq. 6 -----------------------------------------------------------------------------
+    def step(self, tokens: torch.Tensor, beta: float, tau: float = 1.0, lambda_kl: float = 1.0, lambda_round: float = 1.0,
+             lr: float = 5e-4, want_dv: bool = False, fp_outputs=None):
+        """One alignment step on a batch of token ids ([batch*seq] int32, device).  Losses {L_KL, L_MSE} are left in
+        self.loss (device).  fp_outputs = (Z_fp, H_fp) reuses a frozen-model forward of the same batch."""
+        self.step_count += 1
+        Z_fp, H_fp = fp_outputs if fp_outputs is not None else self.forward(tokens, quantised=False)[:2]
+        Z_q, H_q, saved = self.forward(tokens, quantised=True, beta=beta, keep=True)
+        c, T = self.cfg, self.T
+        dZ, dH = torch.empty_like(Z_q), torch.empty_like(H_q)
+        faar.align_loss(self.ctx, T, c.vocab, c.hidden, Z_fp, Z_q, Z_q.shape[1], H_fp, H_q, c.hidden, tau, lambda_kl, dZ, dH,
+                        self.loss, self.aws)
+        hp = faar.make_hparams(beta=beta, lambda_round=lambda_round, opt=self.opt, lr=lr, step=self.step_count)
+        grads = self.backward(dZ, dH, saved, hp, want_dv)
+        return (Z_q, H_q, grads) if want_dv else None
+
+    def round_loss_sum(self) -> float:
+        """Sum over all linears of the Round Loss (Eq. 6's third term without lambda); reads back one float each."""
+        out = torch.zeros(1, dtype=torch.float32, device=self.dev)
+        total = 0.0
+        for layer in self.lin:
+            for lin in layer.values():
+                faar.round_loss(self.ctx, lin.V, lin.O * lin.K, out, self.ws)
+                total += float(out.item())
+        return total
+
+    def harden(self) -> list:
+        """Eq. 7 for every linear: packed NVFP4 codes (the scales and tensor scale are the set-up's)."""
+        res = []
+        for layer in self.lin:
+            d = {}
+            for n, lin in layer.items():
+                packed = torch.empty((lin.O, lin.K // 2), dtype=torch.uint8, device=self.dev)
+                faar.harden_pack(self.ctx, faar.make_shape(lin.O, lin.K, 8), lin.V, lin.code, lin.scales, lin.s_global, packed,
+                                 None, None, None)
+                d[n] = packed
+            res.append(d)
+        faar.check_status(self.ctx, self.ws)
+        return res
