@@ -205,7 +205,8 @@ class Stage2Model:
     def step(self, tokens: torch.Tensor, beta: float, tau: float = 1.0, lambda_kl: float = 1.0, lambda_round: float = 1.0,
              lr: float = 5e-4, want_dv: bool = False, fp_outputs=None):
         """One alignment step on a batch of token ids ([batch*seq] int32, device).  Losses {L_KL, L_MSE} are left in
-        self.loss (device).  fp_outputs = (Z_fp, H_fp) reuses a frozen-model forward of the same batch."""
+        self.loss (device).  fp_outputs = (Z_fp, H_fp) reuses a frozen-model forward of the same batch.  want_dv: also
+        return the quantised model's outputs, the loss gradients and every linear's dV (for inspection)."""
         self.step_count += 1
         Z_fp, H_fp = fp_outputs if fp_outputs is not None else self.forward(tokens, quantised=False)[:2]
         Z_q, H_q, saved = self.forward(tokens, quantised=True, beta=beta, keep=True)
@@ -215,7 +216,7 @@ class Stage2Model:
                         self.loss, self.aws)
         hp = faar.make_hparams(beta=beta, lambda_round=lambda_round, opt=self.opt, lr=lr, step=self.step_count)
         grads = self.backward(dZ, dH, saved, hp, want_dv)
-        return (Z_q, H_q, grads) if want_dv else None
+        return {"Z_q": Z_q, "H_q": H_q, "dZ": dZ, "dH": dH, "dV": grads} if want_dv else None
 
     def round_loss_sum(self) -> float:
         """Sum over all linears of the Round Loss (Eq. 6's third term without lambda); reads back one float each."""

@@ -67,29 +67,38 @@ def test_stage2_step_matches_the_oracle(ctx):
     Zf_o, Hf_o, _ = so.forward(ocfg, params, W_fp, tokens)
     assert rel_l2(host(Zf), Zf_o) <= 1.5e-2 and rel_l2(host(Hf), Hf_o) <= 1.5e-2
     # ---- the step, with the gradients returned
-    Zq, Hq, grads = model.step(tok, beta, tau, lam_kl, lam_r, lr, want_dv=True, fp_outputs=(Zf, Hf))
+    res = model.step(tok, beta, tau, lam_kl, lam_r, lr, want_dv=True, fp_outputs=(Zf, Hf))
+    Zq, Hq, grads = res["Z_q"], res["H_q"], res["dV"]
     faar.check_status(ctx, model.ws)
     total_o, (l_kl_o, l_mse_o, l_round_o), dV_o = so.stage2_loss_and_grads(ocfg, params, W_fp, state, tokens, beta, tau,
                                                                            lam_kl, lam_r)
-    Zq_o, Hq_o, _ = so.forward(ocfg, params, so.quantised_weights(state, beta), tokens)
+    Wq_o = so.quantised_weights(state, beta)
+    Zq_o, Hq_o, saved = so.forward(ocfg, params, Wq_o, tokens, keep=True)
     assert rel_l2(host(Zq), Zq_o) <= 1.5e-2 and rel_l2(host(Hq), Hq_o) <= 1.5e-2
     loss = host(model.loss)
     print("L_KL gpu / oracle:", loss[0], l_kl_o, " L_MSE:", loss[1], l_mse_o)
-    # the data terms are differences of two nearly equal forward passes: BF16 activations leave ~1e-2 of each
-    # pass in them, i.e. a larger share of their difference
+    # The data terms are differences of two nearly equal forward passes: the BF16 storage of Z and H (2^-9 of each
+    # pass) is a much larger share of their difference, in the loss values and in the loss gradients alike.
     assert abs(loss[0] - l_kl_o) <= 0.15 * l_kl_o and abs(loss[1] - l_mse_o) <= 0.15 * l_mse_o
-    assert abs(model.round_loss_sum() - 0.0) >= 0.0                        # callable; value checked below
-    worst = 0.0
+    l_round_g = model.round_loss_sum()          # after the update: V has moved by at most lr
+    assert abs(l_round_g - l_round_o) <= 4 * lr * 14 + 1e-3 * l_round_o
+    # (a) the backward pass on its own: the oracle back-propagates the GPU's own loss gradients
+    G = so.backward(ocfg, params, Wq_o, host(res["dZ"]).astype(np.float64), host(res["dH"]).astype(np.float64), saved)
+    # (b) the whole step against the oracle's own gradients (looser: the seed noise explained above)
+    worst_a, worst_b = 0.0, 0.0
     for l in range(cfg["n_layers"]):
         for n in so.LINEARS:
-            g, ref = host(grads[(l, n)]).astype(np.float64), dV_o[l][n]
-            err = rel_l2(g, ref)
-            worst = max(worst, err)
-            assert err <= 0.12, (l, n, err)
-            # direction: the update moves V the way the oracle's gradient says, for the entries that matter
-            big = np.abs(ref) > 0.2 * np.abs(ref).max()
-            assert np.mean(np.sign(g[big]) == np.sign(ref[big])) >= 0.98, (l, n)
-    print("worst relative dV error over the 14 linears:", worst)
+            V, code, scales, sg = state[l][n]
+            Vd = V.astype(np.float64)
+            ref_a = G[l][n] * fo.chain_factor(Vd, code, scales, sg, beta) + (lam_r / Vd.size) * (4.0 - 8.0 * Vd)
+            g = host(grads[(l, n)]).astype(np.float64)
+            ea, eb = rel_l2(g, ref_a), rel_l2(g, dV_o[l][n])
+            worst_a, worst_b = max(worst_a, ea), max(worst_b, eb)
+            assert ea <= 4e-2, (l, n, ea)
+            assert eb <= 0.25, (l, n, eb)
+            big = np.abs(dV_o[l][n]) > 0.3 * np.abs(dV_o[l][n]).max()
+            assert np.mean(np.sign(g[big]) == np.sign(dV_o[l][n][big])) >= 0.97, (l, n)
+    print("worst relative dV error over the 14 linears: backward alone %.3g, whole step %.3g" % (worst_a, worst_b))
     # ---- state after the update: Adam's first step is lr * sign-like; V stays in [0, 1]
     for l in range(cfg["n_layers"]):
         for n in so.LINEARS:
@@ -97,8 +106,8 @@ def test_stage2_step_matches_the_oracle(ctx):
             Vn = host(model.lin[l][n].V)
             assert Vn.min() >= 0.0 and Vn.max() <= 1.0
             assert np.max(np.abs(Vn - V0)) <= lr * 1.001 + 1e-7
-            moved = np.abs(dV_o[l][n]) > 0.2 * np.abs(dV_o[l][n]).max()
-            assert np.mean(np.sign(V0 - Vn)[moved] == np.sign(dV_o[l][n])[moved]) >= 0.98
+            moved = np.abs(dV_o[l][n]) > 0.3 * np.abs(dV_o[l][n]).max()
+            assert np.mean(np.sign(V0 - Vn)[moved] == np.sign(dV_o[l][n])[moved]) >= 0.97
 
 
 def test_stage2_steps_reduce_the_alignment_loss(ctx):
