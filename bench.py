@@ -44,7 +44,24 @@ BLOCK_WORKLOADS = {
        "down 2048x6144, W bf16 0.02*N(0,1); calibration hidden states N(0,1) + 8 channels x30, RMS-normalised, "
        "4096-row minibatches; Adam lr 1e-2, beta 4->32 geometric",
 }
+STAGE2_MODEL = dict(vocab=128256, hidden=2048, n_layers=16, n_heads=32, n_kv_heads=8, head_dim=64, ffn=8192)
+STAGE2_BATCH, STAGE2_SEQ = 4, 2048
+STAGE2_WORKLOAD = "Stage-2 full-model alignment step (Eq. 6) on a 16-layer Llama-3.2-1B-shaped model (hidden 2048, 32 heads / " \
+                  "8 KV heads, head_dim 64, MLP 8192, vocab 128256, random-init bf16 0.02*N(0,1)), all 112 linears " \
+                  "soft-quantised with their own V, batch 4 x 2048 token ids uniform over the vocabulary, loss = KL(logits) + " \
+                  "MSE(last hidden state) + Round Loss, Adam lr 5e-4"
 METRIC, UNIT = "faar_layer_steps_per_s", "steps/s"
+
+
+def stage2_flops(m=STAGE2_MODEL, batch=STAGE2_BATCH, seq=STAGE2_SEQ):
+    """Algorithmic flop of one alignment step (no recomputation counted): per quantised linear the frozen forward,
+    the quantised forward, the input gradient and the dW GEMM (8 T O K); the LM head twice forward and once
+    backward; causal attention forward in both models (2 products) and backward (4 products)."""
+    T = batch * seq
+    q, kv = m["n_heads"] * m["head_dim"], m["n_kv_heads"] * m["head_dim"]
+    p_lin = m["n_layers"] * (2 * q * m["hidden"] + 2 * kv * m["hidden"] + 3 * m["ffn"] * m["hidden"])
+    att_unit = 2.0 * batch * m["n_heads"] * seq * seq * m["head_dim"] / 2.0
+    return 8.0 * T * p_lin + 3.0 * 2.0 * T * m["vocab"] * m["hidden"] + m["n_layers"] * 8.0 * att_unit
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0
 
@@ -237,6 +254,18 @@ def run_reference(args):
         return rate, dt, th, f"each step = {r} of {O} output rows (exact sub-problem: the loss separates over rows) on " \
                              f"{tk} of {T} tokens, K={K}; rate scaled by the work ratio {O}/{r} x {T}/{tk}"
 
+    if args.config == 5:
+        # each step of the run = the bounded sample of one alignment step (see oracle_stage2_rate)
+        n = max(1, min(args.steps, 3))
+        res = [oracle_stage2_rate() for _ in range(n)]
+        rate, threads, sample = sum(r[0] for r in res) / n, res[0][2], res[0][3]
+        line = {"impl": "reference", "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": 1e3 / rate, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_config(5),
+                "cpu_baseline": {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+                "e2e": {"value": rate, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+        print(json.dumps(line))
+        return 0
     while True:
         _, dt_probe, _, _ = probe(rows, tokens, 1, 1)
         if dt_probe <= budget or (rows <= 16 and tokens <= 128):
@@ -260,6 +289,11 @@ def run_reference(args):
 def workload_config(config: int):
     """The `config` object both arms print: the workload and its sizes, nothing else."""
     l2 = "no flush: one step touches about 410 MB (X, X^T, V, m, u, W_soft, Y_ref, dY^T, codes), more than the 126 MB L2"
+    if config == 5:
+        return {"workload": STAGE2_WORKLOAD, "batch": STAGE2_BATCH, "seq_len": STAGE2_SEQ, **STAGE2_MODEL,
+                "l2": "no flush: one step touches tens of GB (weights, V and Adam moments of 973 M parameters, activations)",
+                "timed_region": "K x (frozen forward, quantised forward, loss, backward with the update of all 112 V); "
+                                "weights, V, Adam moments and the token batch resident in HBM"}
     if config == 2:
         return {"workload": WORKLOAD, "O": O, "K": K, "T": T, "l2": l2,
                 "timed_region": "softquant_init + K x layer_step + harden_pack, inputs resident in HBM"}
@@ -467,6 +501,141 @@ def run_block(args, rt):
     return 0
 
 
+def oracle_stage2_rate(seq=128, warm=0):
+    """Steps/s of the Stage-2 oracle (numpy, float64) for the full workload, from ONE alignment step on a bounded
+    sample -- one decoder block of the sixteen, one sequence of `seq` tokens, the full vocabulary -- scaled by the
+    algorithmic flop count.  Returns (rate, seconds of the sampled step, threads, description)."""
+    import numpy as np
+
+    from oracle import faar_oracle as fo
+    from oracle import stage2_oracle as so
+    from paper_2603_22370_b200 import inputs
+    m = dict(STAGE2_MODEL, n_layers=1)
+    cfg = so.ModelCfg(**m)
+    rng = np.random.default_rng(0)
+    params = {"embed": 0.02 * rng.standard_normal((cfg.vocab, cfg.hidden), dtype=np.float32),
+              "lm_head": 0.02 * rng.standard_normal((cfg.vocab, cfg.hidden), dtype=np.float32),
+              "final_norm": np.ones(cfg.hidden), "attn_norm.0": np.ones(cfg.hidden), "mlp_norm.0": np.ones(cfg.hidden)}
+    W_fp, state = [{}], [{}]
+    for name, (o, k) in cfg.linear_shapes().items():
+        W = inputs.to_bf16_f32(inputs.weights(rng, o, k, 0.02))
+        scales, sg, code, V = fo.softquant_init(W)
+        W_fp[0][name], state[0][name] = W, (V, code, scales, sg)
+    tokens = rng.integers(0, cfg.vocab, (1, seq))
+    t0 = time.perf_counter()
+    so.stage2_loss_and_grads(cfg, params, W_fp, state, tokens, beta=4.0)
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = len(os.sched_getaffinity(0))
+    ratio = stage2_flops() / stage2_flops(m, 1, seq)
+    sample = f"one alignment step of the oracle on 1 of 16 decoder blocks and 1 x {seq} of {STAGE2_BATCH} x {STAGE2_SEQ} tokens " \
+             f"(full vocabulary); time scaled by the flop ratio x{ratio:.0f}"
+    return 1.0 / (dt * ratio), dt, threads, sample
+
+
+def run_stage2(args, rt):
+    """--config 5: full-model alignment steps through the package's Stage-2 driver."""
+    from paper_2603_22370_b200 import stage2
+    torch, faar, ctx, stream, device = rt.torch, rt.faar, rt.ctx, rt.stream, rt.device
+    steps, warmup = args.steps, max(args.warmup, 3)
+    m = dict(STAGE2_MODEL)
+    if args.layers:
+        m["n_layers"] = args.layers
+    cfg = stage2.ModelConfig(**m)
+    B, S = STAGE2_BATCH, STAGE2_SEQ
+    gen = torch.Generator(device=device).manual_seed(1234 + rt.rank)
+
+    def normal(*shape, sigma=0.02):
+        return (sigma * torch.randn(shape, device=device, generator=gen, dtype=torch.float32)).to(torch.bfloat16)
+
+    with torch.cuda.stream(stream):
+        params = {"embed": normal(cfg.vocab, cfg.hidden, sigma=1.0), "lm_head": normal(cfg.vocab, cfg.hidden),
+                  "final_norm": torch.ones(cfg.hidden, dtype=torch.float32, device=device)}
+        weights = []
+        for l in range(cfg.n_layers):
+            params[f"attn_norm.{l}"] = torch.ones(cfg.hidden, dtype=torch.float32, device=device)
+            params[f"mlp_norm.{l}"] = torch.ones(cfg.hidden, dtype=torch.float32, device=device)
+            weights.append({n: normal(o, k) for n, (o, k) in cfg.linear_shapes().items()})
+        model = stage2.Stage2Model(ctx, cfg, params, weights, B, S)
+        tok_h = torch.randint(0, cfg.vocab, (B * S,), dtype=torch.int32).pin_memory()
+        tok = tok_h.to(device, non_blocking=True)
+    stream.synchronize()
+
+    def job(n, t0=0):
+        for t in range(n):
+            model.step(tok, beta=beta_at(t0 + t, max(steps, 2)), lr=5e-4)
+
+    with torch.cuda.stream(stream):
+        job(warmup)
+    stream.synchronize()
+    faar.check_status(ctx, model.ws)
+    ms_job = rt.timed(lambda: job(steps))
+    faar.check_status(ctx, model.ws)
+    loss_final = model.loss.cpu().tolist()
+
+    def profiled():
+        faar.profile_begin(ctx)
+        job(1)
+
+    rt.timed(profiled)
+    prof = faar.profile_end(ctx)
+
+    # end to end: the token batch comes from pinned host memory and the two loss values go back, every step
+    loss_h = torch.zeros(2, dtype=torch.float32).pin_memory()
+
+    def e2e_job(n):
+        for t in range(n):
+            tok.copy_(tok_h, non_blocking=True)
+            model.step(tok, beta=beta_at(t, max(steps, 2)), lr=5e-4)
+            loss_h.copy_(model.loss, non_blocking=True)
+            stream.synchronize()
+
+    ms_e2e = rt.timed(lambda: e2e_job(steps))
+    clocks = rt.sampler.stop() if rt.sampler else None
+    if rt.rank != 0:
+        rt.finish()
+        return 0
+    pk, pk_kind = peaks()
+    flop = stage2_flops(m)
+    peak_key, frac_key, peak_why = applicable_peak(ms_job, clocks)
+    value = rt.world * steps / (ms_job * 1e-3)
+    tf = flop * steps / (ms_job * 1e-3) / 1e12
+    kern = {k: {"launches": v[0], "total_ms": round(v[1], 3)} for k, v in prof.items()}
+    step_ms = sum(v[1] for v in prof.values())
+    for k in kern:
+        kern[k]["share"] = round(prof[k][1] / step_ms, 4)
+    gemm_ms = prof.get("gemm_ref", (0, 0.0))[1] + prof.get("gemm_bwd", (0, 0.0))[1]
+    T = B * S
+    q, kv = cfg.n_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim
+    p_lin = cfg.n_layers * (2 * q * cfg.hidden + 2 * kv * cfg.hidden + 3 * cfg.ffn * cfg.hidden)
+    gemm_flop = 8.0 * T * p_lin + 6.0 * T * cfg.vocab * cfg.hidden
+    gemm_tf = gemm_flop / (gemm_ms * 1e-3) / 1e12 if gemm_ms else 0.0
+    roofline = {"kernel": "the tensor-core GEMM launches of one step (forward products, input gradients, dW + update)",
+                "bound": "tensor", "achieved": round(gemm_tf, 1), "peak": pk[peak_key], "unit": "TFLOP/s",
+                "frac": tensor_fracs(gemm_tf, pk)[frac_key], **tensor_fracs(gemm_tf, pk), "traffic": None,
+                "peak_source": f"{pk_kind} {peak_key}: {peak_why}",
+                "timed": "per-kernel CUDA events on the launching stream, one profiled step after the timed job"}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_job / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": workload_config(5) if not args.layers else
+            dict(workload_config(5), n_layers=cfg.n_layers, note="reduced layer count (--layers)"),
+            "clocks": clocks, "step_tflops": round(tf, 1), "step_frac": tensor_fracs(tf, pk),
+            "e2e": {"value": rt.world * steps / (ms_e2e * 1e-3), "unit": UNIT, "steps": steps, "h2d_bytes_per_step": T * 4,
+                    "d2h_bytes_per_step": 8, "path": "Stage2Model.step: token ids copied in from pinned memory, losses copied out and "
+                                                     "the stream synchronised every step"},
+            "gpu_launches": steps * sum(v[0] for v in prof.values()), "roofline": roofline, "kernels": kern,
+            "final_loss": loss_final}
+    if not args.quick:
+        rate, dt, threads, sample = oracle_stage2_rate()
+        line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+    print(json.dumps(line))
+    rt.finish()
+    return 0
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -476,6 +645,8 @@ def run_ours(args):
     rt = Runtime(args)
     if args.config in (3, 4):
         return run_block(args, rt)
+    if args.config == 5:
+        return run_stage2(args, rt)
     rank, world, dev, device, dist = rt.rank, rt.world, rt.dev, rt.device, rt.dist
     n_gpus = args.gpus
     steps, warmup = args.steps, max(args.warmup, 3)
@@ -780,9 +951,11 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5],
                     help="2: the down_proj-shaped layer (the headline); 3 / 4: the seven linears of a Llama-3.2-1B- / "
                          "Qwen3-1.7B-shaped decoder block")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="--config 5 only: decoder blocks of the model (0 = the workload's 16); smaller for profiler captures")
     ap.add_argument("--calib-tokens", type=int, default=65536,
                     help="rows of the synthetic calibration set of --config 3 / 4 (4096-row minibatches, round-robin)")
     ap.add_argument("--align-tokens", type=int, default=4096,
