@@ -75,6 +75,11 @@ attn_fwd_kernel(const AttnParams p) {
 #pragma unroll
   for (int n = 0; n < D / 16; ++n) wmma::fill_fragment(oacc[n], 0.f);
 
+  __syncthreads();
+  wmma::fragment<wmma::matrix_a, 16, 16, 16, __nv_bfloat16, wmma::row_major> qf[D / 16];      // this warp's queries, kept
+#pragma unroll
+  for (int kk = 0; kk < D / 16; ++kk) wmma::load_matrix_sync(qf[kk], &Qs[16 * warp][16 * kk], D + 8);
+
   for (int pass = 0; pass < 2; ++pass) {
     for (int kt = 0; kt <= qt; ++kt) {
       const int k0 = kt * AT;
@@ -83,29 +88,33 @@ attn_fwd_kernel(const AttnParams p) {
       if (pass == 1) load_tile<D>(Vs, p.v, p.ldk, seq0 + k0, seq0 + p.S, g * D);
       __syncthreads();
       // scores of this warp's 16 queries against the 64 keys
+      {
+        wmma::fragment<wmma::accumulator, 16, 16, 16, float> sacc[AT / 16];
 #pragma unroll
-      for (int n = 0; n < AT / 16; ++n) {
-        wmma::fragment<wmma::accumulator, 16, 16, 16, float> sacc;
-        wmma::fill_fragment(sacc, 0.f);
+        for (int n = 0; n < AT / 16; ++n) wmma::fill_fragment(sacc[n], 0.f);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          wmma::fragment<wmma::matrix_a, 16, 16, 16, __nv_bfloat16, wmma::row_major> a;
-          wmma::fragment<wmma::matrix_b, 16, 16, 16, __nv_bfloat16, wmma::col_major> bf;
-          wmma::load_matrix_sync(a, &Qs[16 * warp][16 * kk], D + 8);
-          wmma::load_matrix_sync(bf, &Ks[16 * n][16 * kk], D + 8);
-          wmma::mma_sync(sacc, a, bf, sacc);
+#pragma unroll
+          for (int n = 0; n < AT / 16; ++n) {
+            wmma::fragment<wmma::matrix_b, 16, 16, 16, __nv_bfloat16, wmma::col_major> bf;
+            wmma::load_matrix_sync(bf, &Ks[16 * n][16 * kk], D + 8);
+            wmma::mma_sync(sacc[n], qf[kk], bf, sacc[n]);
+          }
         }
-        wmma::store_matrix_sync(Sw + 16 * n, sacc, AT + 4, wmma::mem_row_major);
+#pragma unroll
+        for (int n = 0; n < AT / 16; ++n) wmma::store_matrix_sync(Sw + 16 * n, sacc[n], AT + 4, wmma::mem_row_major);
       }
       __syncwarp();
-      float* srow = Sw + row * (AT + 4) + 32 * half;
+      // element-wise phase: this lane takes the columns half, half + 2, ... of its row (two lanes interleave,
+      // so that a warp's accesses spread over the shared-memory banks)
+      float* srow = Sw + row * (AT + 4) + half;
       if (pass == 0) {
         float mx = -INFINITY;
 #pragma unroll 8
         for (int c = 0; c < 32; ++c) {
-          const int kj = k0 + 32 * half + c;
-          const float s = (kj <= qi && kj < p.S) ? srow[c] * p.scale_log2 : -INFINITY;
-          srow[c] = s;
+          const int kj = k0 + half + 2 * c;
+          const float s = (kj <= qi && kj < p.S) ? srow[2 * c] * p.scale_log2 : -INFINITY;
+          srow[2 * c] = s;
           mx = fmaxf(mx, s);
         }
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
@@ -113,19 +122,19 @@ attn_fwd_kernel(const AttnParams p) {
         float sum = 0.f;
         if (m_new > -INFINITY) {
 #pragma unroll 8
-          for (int c = 0; c < 32; ++c) sum += exp2f(srow[c] - m_new);
+          for (int c = 0; c < 32; ++c) sum += exp2f(srow[2 * c] - m_new);
         }
         sum += __shfl_xor_sync(0xffffffffu, sum, 1);
         l_run = (m_run > -INFINITY ? l_run * exp2f(m_run - m_new) : 0.f) + sum;
         m_run = m_new;
       } else {
         const float inv_l = l_run > 0.f ? 1.0f / l_run : 0.f;
-        __nv_bfloat16* prow = Pw + row * (AT + 8) + 32 * half;
+        __nv_bfloat16* prow = Pw + row * (AT + 8) + half;
 #pragma unroll 8
         for (int c = 0; c < 32; ++c) {
-          const int kj = k0 + 32 * half + c;
-          const float pr = (kj <= qi && kj < p.S) ? exp2f(srow[c] * p.scale_log2 - m_run) * inv_l : 0.f;
-          prow[c] = __float2bfloat16_rn(pr);
+          const int kj = k0 + half + 2 * c;
+          const float pr = (kj <= qi && kj < p.S) ? exp2f(srow[2 * c] * p.scale_log2 - m_run) * inv_l : 0.f;
+          prow[2 * c] = __float2bfloat16_rn(pr);
         }
         __syncwarp();
 #pragma unroll
