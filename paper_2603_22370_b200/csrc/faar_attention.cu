@@ -427,6 +427,303 @@ attn_dq_kernel(const AttnParams p) {
   }
 }
 
+// =====================================================================================================
+// head_dim 64: the same three kernels with every intermediate kept in registers.  The matrix products are
+// mma.sync m16n8k16 (BF16 in, FP32 accumulate) whose accumulator layout is documented: lane l holds, of a
+// 16 x 8 tile, rows l / 4 and l / 4 + 8, columns 2 (l % 4) and 2 (l % 4) + 1.  Two neighbouring accumulator
+// tiles are exactly the A operand of the next product (rows the same, 16 contraction columns), so the scores
+// become probabilities and then the left operand of P V without leaving the register file; row maxima and sums
+// are reduced over the four lanes that share a row.  Operands come from shared memory through ldmatrix (rows
+// of D + 8 elements: 16-byte aligned and conflict-free); the forward pass makes one sweep over the keys with a
+// running maximum (the output accumulators are rescaled in place).
+// =====================================================================================================
+constexpr int HD = 64;                       // head_dim of this path
+constexpr int LDS = HD + 8;                  // shared-memory row stride (elements)
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void* ptr) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(ptr);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const void* ptr) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(ptr);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+// D[16 x 8] += A[16 x 16] B[16 x 8]
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+// A operand (16 rows of `tile` from row0, contraction columns 16 kk ..): a0 rows 0-7 / k 0-7, a1 rows 8-15 / k 0-7,
+// a2 rows 0-7 / k 8-15, a3 rows 8-15 / k 8-15.
+__device__ __forceinline__ void load_a(uint32_t (&a)[4], const __nv_bfloat16 (*tile)[LDS], int row0, int kk, int lane) {
+  ldsm_x4(a, &tile[row0 + (lane & 15)][16 * kk + 8 * (lane >> 4)]);
+}
+// B operands for two neighbouring 8-column tiles when B[k][n] = tile[n][k] (the tile's rows are the output
+// columns: Q K^T style): r0, r1 for columns n0 .. n0 + 7, r2, r3 for n0 + 8 .. n0 + 15; contraction 16 kk ..
+__device__ __forceinline__ void load_b_rows(uint32_t (&r)[4], const __nv_bfloat16 (*tile)[LDS], int n0, int kk, int lane) {
+  ldsm_x4(r, &tile[n0 + (lane & 7) + 8 * (lane >> 4)][16 * kk + 8 * ((lane >> 3) & 1)]);
+}
+// B operands for two neighbouring 8-column tiles when B[k][n] = tile[k][n] (the tile's rows are contracted:
+// P V style): contraction rows k0 .. k0 + 15, r0, r1 for columns n0 .. n0 + 7, r2, r3 for n0 + 8 .. n0 + 15.
+__device__ __forceinline__ void load_b_cols(uint32_t (&r)[4], const __nv_bfloat16 (*tile)[LDS], int k0, int n0, int lane) {
+  ldsm_x4_t(r, &tile[k0 + (lane & 7) + 8 * ((lane >> 3) & 1)][n0 + 8 * (lane >> 4)]);
+}
+
+// S[16 x 64] = A-rows (fragments af[4], contraction over head_dim) times tile^T
+__device__ __forceinline__ void scores_16x64(float (&acc)[8][4], const uint32_t (&af)[HD / 16][4], const __nv_bfloat16 (*tile)[LDS],
+                                             int lane) {
+#pragma unroll
+  for (int n = 0; n < 8; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
+#pragma unroll
+  for (int kk = 0; kk < HD / 16; ++kk) {
+#pragma unroll
+    for (int n2 = 0; n2 < 4; ++n2) {
+      uint32_t b[4];
+      load_b_rows(b, tile, 16 * n2, kk, lane);
+      mma16816(acc[2 * n2], af[kk], b[0], b[1]);
+      mma16816(acc[2 * n2 + 1], af[kk], b[2], b[3]);
+    }
+  }
+}
+// out[16 x 64] += P[16 x 64] (as A fragments pf[4]) times tile (rows contracted)
+__device__ __forceinline__ void accumulate_16x64(float (&out)[8][4], const uint32_t (&pf)[4][4], const __nv_bfloat16 (*tile)[LDS], int lane) {
+#pragma unroll
+  for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+    for (int n2 = 0; n2 < 4; ++n2) {
+      uint32_t b[4];
+      load_b_cols(b, tile, 16 * kk, 16 * n2, lane);
+      mma16816(out[2 * n2], pf[kk], b[0], b[1]);
+      mma16816(out[2 * n2 + 1], pf[kk], b[2], b[3]);
+    }
+  }
+}
+// accumulator tiles -> A fragments of the next product
+__device__ __forceinline__ void to_a_frags(uint32_t (&pf)[4][4], const float (&acc)[8][4]) {
+#pragma unroll
+  for (int kk = 0; kk < 4; ++kk) {
+    pf[kk][0] = pack2(acc[2 * kk][0], acc[2 * kk][1]);
+    pf[kk][1] = pack2(acc[2 * kk][2], acc[2 * kk][3]);
+    pf[kk][2] = pack2(acc[2 * kk + 1][0], acc[2 * kk + 1][1]);
+    pf[kk][3] = pack2(acc[2 * kk + 1][2], acc[2 * kk + 1][3]);
+  }
+}
+// a warp's 16 x 64 accumulator as BF16 rows of a [.., ld] matrix (rows row0 + l/4 and + 8, valid below row_end)
+__device__ __forceinline__ void store_16x64(__nv_bfloat16* base, long long ld, long long row0, long long row_end, int col0,
+                                            const float (&acc)[8][4], float s0, float s1, int lane) {
+  const long long r0 = row0 + (lane >> 2), r1 = r0 + 8;
+#pragma unroll
+  for (int n = 0; n < 8; ++n) {
+    const int c = col0 + 8 * n + 2 * (lane & 3);
+    if (r0 < row_end) *reinterpret_cast<uint32_t*>(base + r0 * ld + c) = pack2(acc[n][0] * s0, acc[n][1] * s0);
+    if (r1 < row_end) *reinterpret_cast<uint32_t*>(base + r1 * ld + c) = pack2(acc[n][2] * s1, acc[n][3] * s1);
+  }
+}
+
+// ---- forward, head_dim 64: grid (query tiles, H, B); warp w owns queries 16 w .. 16 w + 15 ------------------
+__global__ void __launch_bounds__(ATT_THREADS)
+attn_fwd64_kernel(const AttnParams p) {
+  __shared__ __align__(128) __nv_bfloat16 Qs[AT][LDS];
+  __shared__ __align__(128) __nv_bfloat16 Ks[AT][LDS];
+  __shared__ __align__(128) __nv_bfloat16 Vs[AT][LDS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;      // longest tiles first
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.H / p.Hkv);
+  const long long seq0 = (long long)b * p.S;
+  const int q0 = qt * AT;
+  load_tile<HD>(Qs, p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
+  __syncthreads();
+  uint32_t qf[HD / 16][4];
+#pragma unroll
+  for (int kk = 0; kk < HD / 16; ++kk) load_a(qf[kk], Qs, 16 * warp, kk, lane);
+  const int qi0 = q0 + 16 * warp + (lane >> 2), qi1 = qi0 + 8;          // this lane's two query rows
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  float o[8][4];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+
+  for (int kt = 0; kt <= qt; ++kt) {
+    const int k0 = kt * AT;
+    __syncthreads();
+    load_tile<HD>(Ks, p.k, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+    load_tile<HD>(Vs, p.v, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+    __syncthreads();
+    float s[8][4];
+    scores_16x64(s, qf, Ks, lane);
+    // scale to log2 units, causal mask, row maxima
+    float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int kj = k0 + 8 * n + 2 * (lane & 3) + j;
+        s[n][j] = (kj <= qi0 && kj < p.S) ? s[n][j] * p.scale_log2 : -INFINITY;
+        s[n][2 + j] = (kj <= qi1 && kj < p.S) ? s[n][2 + j] * p.scale_log2 : -INFINITY;
+        mx0 = fmaxf(mx0, s[n][j]);
+        mx1 = fmaxf(mx1, s[n][2 + j]);
+      }
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+    // a row that has seen no key yet keeps maximum -inf: use 0 as the reference so that nothing is NaN
+    const float ref0 = mn0 == -INFINITY ? 0.f : mn0, ref1 = mn1 == -INFINITY ? 0.f : mn1;
+    const float a0 = exp2f(m0 - ref0), a1 = exp2f(m1 - ref1);            // exp2f(-inf) = 0
+    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      s[n][0] = exp2f(s[n][0] - ref0); s[n][1] = exp2f(s[n][1] - ref0);
+      s[n][2] = exp2f(s[n][2] - ref1); s[n][3] = exp2f(s[n][3] - ref1);
+      sum0 += s[n][0] + s[n][1];
+      sum1 += s[n][2] + s[n][3];
+      o[n][0] *= a0; o[n][1] *= a0; o[n][2] *= a1; o[n][3] *= a1;
+    }
+    sum0 += __shfl_xor_sync(0xffffffffu, sum0, 1); sum0 += __shfl_xor_sync(0xffffffffu, sum0, 2);
+    sum1 += __shfl_xor_sync(0xffffffffu, sum1, 1); sum1 += __shfl_xor_sync(0xffffffffu, sum1, 2);
+    l0 = l0 * a0 + sum0; l1 = l1 * a1 + sum1;
+    m0 = mn0; m1 = mn1;
+    uint32_t pf[4][4];
+    to_a_frags(pf, s);
+    accumulate_16x64(o, pf, Vs, lane);
+  }
+  const float i0 = l0 > 0.f ? 1.0f / l0 : 0.f, i1 = l1 > 0.f ? 1.0f / l1 : 0.f;
+  store_16x64(p.out, p.ldo, seq0 + q0 + 16 * warp, seq0 + p.S, h * HD, o, i0, i1, lane);
+  if ((lane & 3) == 0) {
+    float* lse = p.lse + ((long long)b * p.H + h) * p.S;
+    if (qi0 < p.S) lse[qi0] = m0 + log2f(l0);
+    if (qi1 < p.S) lse[qi1] = m1 + log2f(l1);
+  }
+}
+
+// ---- backward, head_dim 64, dQ: grid (query tiles, H, B); warp w owns queries 16 w .. 16 w + 15 ------------------
+__global__ void __launch_bounds__(ATT_THREADS)
+attn_dq64_kernel(const AttnParams p) {
+  __shared__ __align__(128) __nv_bfloat16 Qs[AT][LDS];
+  __shared__ __align__(128) __nv_bfloat16 Ds[AT][LDS];
+  __shared__ __align__(128) __nv_bfloat16 Ks[AT][LDS];
+  __shared__ __align__(128) __nv_bfloat16 Vs[AT][LDS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.H / p.Hkv);
+  const long long seq0 = (long long)b * p.S;
+  const int q0 = qt * AT;
+  load_tile<HD>(Qs, p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
+  load_tile<HD>(Ds, p.dout, p.ldo, seq0 + q0, seq0 + p.S, h * HD);
+  __syncthreads();
+  uint32_t qf[HD / 16][4], df[HD / 16][4];
+#pragma unroll
+  for (int kk = 0; kk < HD / 16; ++kk) { load_a(qf[kk], Qs, 16 * warp, kk, lane); load_a(df[kk], Ds, 16 * warp, kk, lane); }
+  const int qi0 = q0 + 16 * warp + (lane >> 2), qi1 = qi0 + 8;
+  const long long ro = ((long long)b * p.H + h) * p.S;
+  const float lse0 = qi0 < p.S ? p.lse[ro + qi0] : 0.f, lse1 = qi1 < p.S ? p.lse[ro + qi1] : 0.f;
+  const float dsm0 = qi0 < p.S ? p.dsum[ro + qi0] : 0.f, dsm1 = qi1 < p.S ? p.dsum[ro + qi1] : 0.f;
+  const float inv_sqrt_d = p.scale_log2 / LOG2E;
+  float dq[8][4];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) { dq[n][0] = dq[n][1] = dq[n][2] = dq[n][3] = 0.f; }
+
+  for (int kt = 0; kt <= qt; ++kt) {
+    const int k0 = kt * AT;
+    __syncthreads();
+    load_tile<HD>(Ks, p.k, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+    load_tile<HD>(Vs, p.v, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+    __syncthreads();
+    float s[8][4], dp[8][4];
+    scores_16x64(s, qf, Ks, lane);
+    scores_16x64(dp, df, Vs, lane);
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int kj = k0 + 8 * n + 2 * (lane & 3) + j;
+        const float p0 = (kj <= qi0 && qi0 < p.S) ? exp2f(s[n][j] * p.scale_log2 - lse0) : 0.f;
+        const float p1 = (kj <= qi1 && qi1 < p.S) ? exp2f(s[n][2 + j] * p.scale_log2 - lse1) : 0.f;
+        s[n][j] = p0 * (dp[n][j] - dsm0) * inv_sqrt_d;              // dS
+        s[n][2 + j] = p1 * (dp[n][2 + j] - dsm1) * inv_sqrt_d;
+      }
+    }
+    uint32_t sf[4][4];
+    to_a_frags(sf, s);
+    accumulate_16x64(dq, sf, Ks, lane);                             // dQ += dS K
+  }
+  store_16x64(p.dq, p.ldq, seq0 + q0 + 16 * warp, seq0 + p.S, h * HD, dq, 1.f, 1.f, lane);
+}
+
+// ---- backward, head_dim 64, dK and dV: grid (key tiles, Hkv, B); warp w owns keys 16 w .. 16 w + 15 ---------------
+// The products are formed transposed (keys on the accumulator rows): S^T = K Q^T, dP^T = V dO^T; then
+// dV += P^T dO and dK += dS^T Q contract over the 64 queries of the tile.
+__global__ void __launch_bounds__(ATT_THREADS)
+attn_dkv64_kernel(const AttnParams p) {
+  __shared__ __align__(128) __nv_bfloat16 Ks[AT][LDS];
+  __shared__ __align__(128) __nv_bfloat16 Vs[AT][LDS];
+  __shared__ __align__(128) __nv_bfloat16 Qs[AT][LDS];
+  __shared__ __align__(128) __nv_bfloat16 Ds[AT][LDS];
+  __shared__ __align__(16) float rowv[2 * AT];                     // lse and dsum of the tile's 64 queries
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kt = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int rep = p.H / p.Hkv;
+  const long long seq0 = (long long)b * p.S;
+  const int k0 = kt * AT;
+  const int n_qt = (p.S + AT - 1) / AT;
+  load_tile<HD>(Ks, p.k, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+  load_tile<HD>(Vs, p.v, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+  __syncthreads();
+  uint32_t kf[HD / 16][4], vf[HD / 16][4];
+#pragma unroll
+  for (int kk = 0; kk < HD / 16; ++kk) { load_a(kf[kk], Ks, 16 * warp, kk, lane); load_a(vf[kk], Vs, 16 * warp, kk, lane); }
+  const int kj0 = k0 + 16 * warp + (lane >> 2), kj1 = kj0 + 8;          // this lane's two key rows
+  const float inv_sqrt_d = p.scale_log2 / LOG2E;
+  float dk[8][4], dv[8][4];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) { dk[n][0] = dk[n][1] = dk[n][2] = dk[n][3] = 0.f; dv[n][0] = dv[n][1] = dv[n][2] = dv[n][3] = 0.f; }
+
+  for (int hh = 0; hh < rep; ++hh) {
+    const int h = g * rep + hh;
+    const long long ro = ((long long)b * p.H + h) * p.S;
+    for (int qt = kt; qt < n_qt; ++qt) {
+      const int q0 = qt * AT;
+      __syncthreads();
+      load_tile<HD>(Qs, p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
+      load_tile<HD>(Ds, p.dout, p.ldo, seq0 + q0, seq0 + p.S, h * HD);
+      if (threadIdx.x < AT) {
+        const int qi = q0 + threadIdx.x;
+        rowv[threadIdx.x] = qi < p.S ? p.lse[ro + qi] : 0.f;
+        rowv[AT + threadIdx.x] = qi < p.S ? p.dsum[ro + qi] : 0.f;
+      }
+      __syncthreads();
+      float st[8][4], dpt[8][4];
+      scores_16x64(st, kf, Qs, lane);                               // S^T[key][query]
+      scores_16x64(dpt, vf, Ds, lane);                              // dP^T[key][query]
+      uint32_t pf[4][4];
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int c = 8 * n + 2 * (lane & 3) + j, qi = q0 + c;
+          const float lse = rowv[c], dsm = rowv[AT + c];
+          const float p0 = (kj0 <= qi && qi < p.S) ? exp2f(st[n][j] * p.scale_log2 - lse) : 0.f;
+          const float p1 = (kj1 <= qi && qi < p.S) ? exp2f(st[n][2 + j] * p.scale_log2 - lse) : 0.f;
+          st[n][j] = p0; st[n][2 + j] = p1;
+          dpt[n][j] = p0 * (dpt[n][j] - dsm) * inv_sqrt_d;          // dS^T
+          dpt[n][2 + j] = p1 * (dpt[n][2 + j] - dsm) * inv_sqrt_d;
+        }
+      }
+      to_a_frags(pf, st);
+      accumulate_16x64(dv, pf, Ds, lane);                           // dV += P^T dO
+      to_a_frags(pf, dpt);
+      accumulate_16x64(dk, pf, Qs, lane);                           // dK += dS^T Q
+    }
+  }
+  store_16x64(p.dv, p.ldk, seq0 + k0 + 16 * warp, seq0 + p.S, g * HD, dv, 1.f, 1.f, lane);
+  store_16x64(p.dk, p.ldk, seq0 + k0 + 16 * warp, seq0 + p.S, g * HD, dk, 1.f, 1.f, lane);
+}
+
 template <int D> constexpr int fwd_smem() { return 3 * AT * (D + 8) * 2 + 4 * 16 * (AT + 4) * 4 + 4 * 16 * (AT + 8) * 2; }
 template <int D> constexpr int dkv_smem() { return 4 * AT * (D + 8) * 2 + 2 * 4 * AT * 20 * 4 + 4 * AT * 24 * 2 + 2 * AT * 4; }
 template <int D> constexpr int dq_smem() { return 4 * AT * (D + 8) * 2 + 2 * 4 * 16 * (AT + 4) * 4 + 4 * 16 * (AT + 8) * 2; }
@@ -437,7 +734,10 @@ int launch_fwd(faar_ctx* ctx, const AttnParams& p) {
   if (e != cudaSuccess) return (int)e;
   dim3 grid((p.S + AT - 1) / AT, p.H, p.B);
   faar_prof_scope ps(ctx, FAAR_K_ATTENTION);
-  attn_fwd_kernel<D><<<grid, ATT_THREADS, fwd_smem<D>(), ctx->stream>>>(p);
+  if (D == HD && !ctx->tune_attention_fragments)
+    attn_fwd64_kernel<<<grid, ATT_THREADS, 0, ctx->stream>>>(p);
+  else
+    attn_fwd_kernel<D><<<grid, ATT_THREADS, fwd_smem<D>(), ctx->stream>>>(p);
   return (int)cudaGetLastError();
 }
 
@@ -452,6 +752,11 @@ int launch_bwd(faar_ctx* ctx, const AttnParams& p, float* dsum) {
   if (blocks > (long long)ctx->num_sms * 16) blocks = (long long)ctx->num_sms * 16;
   attn_dsum_kernel<D><<<(int)blocks, ATT_THREADS, 0, ctx->stream>>>(p, dsum);
   const int tiles = (p.S + AT - 1) / AT;
+  if (D == HD && !ctx->tune_attention_fragments) {
+    attn_dkv64_kernel<<<dim3(tiles, p.Hkv, p.B), ATT_THREADS, 0, ctx->stream>>>(p);
+    attn_dq64_kernel<<<dim3(tiles, p.H, p.B), ATT_THREADS, 0, ctx->stream>>>(p);
+    return (int)cudaGetLastError();
+  }
   attn_dkv_kernel<D><<<dim3(tiles, p.Hkv, p.B), ATT_THREADS, dkv_smem<D>(), ctx->stream>>>(p);
   attn_dq_kernel<D><<<dim3(tiles, p.H, p.B), ATT_THREADS, dq_smem<D>(), ctx->stream>>>(p);
   return (int)cudaGetLastError();

@@ -62,6 +62,7 @@ SIGNATURES = {
     "faar_silu_mul_bwd": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L, _P, _L, _P, _L]),
     "faar_embedding": (_I, [_P, _I, _I, _I, _P, _L, _P, _P, _L]),
     "faar_add": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L]),
+    "faar_tune_attention": (_I, [_P, _I]),
     "faar_attention_fwd": (_I, [_P, _I, _I, _I, _I, _I, _P, _L, _P, _P, _L, _P, _L, _P]),
     "faar_attention_bwd": (_I, [_P, _I, _I, _I, _I, _I, _P, _L, _P, _P, _L, _P, _P, _L, _P, _P, _P, _P, _P]),
     "faar_nvfp4_gemm": (_I, [_P, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _L, _P, _Z]),
@@ -290,6 +291,11 @@ def embedding(ctx, rows, cols, vocab, table, ldt, tokens, out, ldo):
 
 def add(ctx, rows, cols, a, lda, b, ldb, out, ldo):
     _check(lib().faar_add(ctx._h, rows, cols, _p(a), lda, _p(b), ldb, _p(out), ldo), "faar_add")
+
+
+def tune_attention(ctx, mode: int):
+    """1: head_dim 64 also runs the shared-memory fragment kernels (as head_dim 128 does); 0: the default."""
+    _check(lib().faar_tune_attention(ctx._h, mode), "faar_tune_attention")
 
 
 def attention_fwd(ctx, batch, seq, n_heads, n_kv_heads, head_dim, q, ldq, k, v, ldkv, out, ldo, lse):

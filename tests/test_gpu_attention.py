@@ -29,9 +29,22 @@ def padded(a, ld, fill=9.0):
     return t
 
 
+@pytest.mark.parametrize("fragments", [0, 1])
 @pytest.mark.parametrize("B,S,H,HKV,D", [(2, 100, 4, 2, 64), (1, 64, 2, 2, 64), (3, 7, 2, 1, 64), (1, 200, 4, 1, 128),
-                                         (2, 129, 8, 2, 64)])
-def test_attention_forward_and_backward_match_the_oracle(ctx, B, S, H, HKV, D):
+                                         (2, 129, 8, 2, 64), (1, 321, 4, 4, 64)])
+def test_attention_forward_and_backward_match_the_oracle(ctx, B, S, H, HKV, D, fragments):
+    """fragments = 0: the default kernels (head_dim 64 keeps scores in registers); 1: head_dim 64 through the
+    shared-memory fragment kernels that head_dim 128 always uses."""
+    if fragments and D != 64:
+        pytest.skip("head_dim 128 has one kind of kernel")
+    faar.tune_attention(ctx, fragments)
+    try:
+        _attention_case(ctx, B, S, H, HKV, D)
+    finally:
+        faar.tune_attention(ctx, 0)
+
+
+def _attention_case(ctx, B, S, H, HKV, D):
     rng = np.random.default_rng(S + D)
     T = B * S
     q = inputs.to_bf16_f32(rng.standard_normal((T, H * D)))
