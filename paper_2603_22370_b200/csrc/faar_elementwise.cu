@@ -40,6 +40,7 @@ __device__ __forceinline__ int64_t w_offset(int64_t g, uint32_t groups_per_row, 
 // ---- pass 1: max |W| over the tensor -----------------------------------------
 __global__ void __launch_bounds__(EW_THREADS)
 amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, uint32_t* amax_word) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel waits for this one's end itself
   const uint32_t groups_per_row = K / 8;
   const int64_t total = (int64_t)O * groups_per_row;
   const bool dense = ldw == K;
@@ -76,66 +77,219 @@ amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, 
   }
 }
 
+// ---- one thread, one 16-element scale block -----------------------------------------------------
+// The set-up and activation kernels give each thread a whole scale block: the block maximum needs no
+// exchange, the E4M3 scale is formed once per 16 values, and all 16 quotients w / s share one
+// reciprocal.  Outputs wider than the input (V: 64 bytes per thread) pass through shared memory so that
+// every global store instruction of a warp covers one contiguous run.
+//
+// These kernels are bound by the SM's integer/logic pipe (compares, selects, min/max, shifts and
+// bit operations issue at half the rate of FP32 multiply-add), so the per-value work is phrased in
+// exact FP32 arithmetic wherever that is possible: the region of the node grid comes from two
+// saturating multiply-adds, floor() from an addition that rounds down, the nibbles of eight values
+// are summed as small integers in FP32.  Every such operation is exact, so the results equal those
+// of the compare-and-select formulation bit for bit.
+
+// 16 consecutive values as binary32.
+__device__ __forceinline__ void load16(const void* W, int w_dtype, int64_t idx, float (&w)[16]) {
+  if (w_dtype == FAAR_BF16) {
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W) + idx);
+    const uint4 r0 = p[0], r1 = p[1];
+    const uint32_t r[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      w[2 * i] = __uint_as_float(r[i] << 16);
+      w[2 * i + 1] = __uint_as_float(r[i] & 0xFFFF0000u);
+    }
+  } else {
+    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(W) + idx);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 r = p[j];
+      w[4 * j] = r.x; w[4 * j + 1] = r.y; w[4 * j + 2] = r.z; w[4 * j + 3] = r.w;
+    }
+  }
+}
+
+// q[i] = w[i] / s, correctly rounded (the result of a binary32 division; rounding to nearest is
+// symmetric, so the sign rides along), for the 16 values of a block.
+// FAST: r = RN(1/s) once, then per value q0 = RN(w r) and two residual corrections
+// e = w - q s (one FMA), q <- RN(q + e r).  After the first correction q is within half a unit of
+// w / s plus 2^-47 relative, hence a faithful rounding; the residual of a faithful quotient is exact in
+// one FMA, and a faithful quotient corrected once more with the correctly rounded reciprocal is the
+// correctly rounded quotient (Markstein's theorem), provided nothing under- or overflows.  The caller
+// secures that proviso: s and the block maximum within [2^-40, 2^40] and no magnitude below 2^-80
+// keep every quotient, product and residual a normal number.  The corrections run as packed pairs
+// (two binary32 lanes per instruction).
+// Otherwise (a zero or minute value, an extreme scale): the division instruction sequence.
+template <bool FAST>
+__device__ __forceinline__ void block_quotients(const float (&w)[16], float s, float (&q)[16]) {
+  if (FAST) {
+    const float r = __frcp_rn(s);
+    const float2 r2 = make_float2(r, r), ns2 = make_float2(-s, -s);
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+      const float2 w2 = make_float2(w[i], w[i + 1]);
+      float2 qq = __fmul2_rn(w2, r2);
+      float2 e = __ffma2_rn(qq, ns2, w2);
+      qq = __ffma2_rn(e, r2, qq);
+      e = __ffma2_rn(qq, ns2, w2);
+      qq = __ffma2_rn(e, r2, qq);
+      q[i] = qq.x;
+      q[i + 1] = qq.y;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) q[i] = s > 0.f ? __fdiv_rn(w[i], s) : 0.f;
+  }
+}
+
+// Position of one scaled magnitude q = min(|w| / s, 6) on the node grid {0, .5, 1, 1.5, 2, 3, 4, 6}.
+// The grid has three regions of constant spacing: [0, 2] by 0.5, [2, 4] by 1, [4, 6] by 2 (a value on
+// a shared end point gets the same answer from either side).  With t1 = [q > 2], t2 = [q > 4] as 0 / 1
+// (q - 2 and q - 4 are multiples of 2^-22 there, so a saturating FMA by 2^22 gives exactly 0 or 1),
+//   m = 1 / spacing = 2 - t1 - t2 / 2,  u = q m,  j = floor(u)  (j = 2 throughout the last region:
+//   it is a single interval that includes its upper end 6),
+//   interval index k = j + 2 t1 + 2 t2,   v = u - j = (q - lower node) / spacing, in [0, 1].
+struct grid_pos {
+  float k, j, v, t1, t2;
+};
+__device__ __forceinline__ grid_pos locate(float q_signed) {
+  grid_pos g;
+  const float q = fminf(fabsf(q_signed), 6.0f);
+  g.t1 = __saturatef(__fmaf_rn(q, 0x1p22f, -0x1p23f));
+  g.t2 = __saturatef(__fmaf_rn(q, 0x1p22f, -0x1p24f));
+  const float m = __fmaf_rn(-0.5f, g.t2, __fsub_rn(2.0f, g.t1));
+  const float u = __fmul_rn(q, m);
+  const float fl = __fsub_rn(__fadd_rd(u, 0x1p23f), 0x1p23f);      // floor(u): the sum has unit spacing, rounded down
+  g.j = __fmaf_rn(g.t2, __fsub_rn(2.0f, fl), fl);
+  g.v = __fsub_rn(u, g.j);
+  g.k = __fmaf_rn(2.0f, g.t2, __fmaf_rn(2.0f, g.t1, g.j));
+  return g;
+}
+
+// 1 for a negative value, 0 otherwise (-0.0 counts as positive).  FAST: the quotient is a normal number
+// of magnitude at least 2^-120, so its product with -2^126 saturates to 0 or 1.
+template <bool FAST>
+__device__ __forceinline__ float negative_flag(float w, float q_signed) {
+  return FAST ? __saturatef(__fmul_rn(q_signed, -0x1p126f)) : (w < 0.f ? 1.0f : 0.0f);
+}
+
+// Eight nibbles given as FP32 integers 0..15 -> one 32-bit word, nibble i at bits 4i.  Four nibbles sum
+// exactly in FP32 (below 2^16); adding 2^23 leaves that integer in the low mantissa bits.
+__device__ __forceinline__ uint32_t pack_nibbles(const float (&n)[8]) {
+  const float lo = __fmaf_rn(n[3], 4096.f, __fmaf_rn(n[2], 256.f, __fmaf_rn(n[1], 16.f, n[0])));
+  const float hi = __fmaf_rn(n[7], 4096.f, __fmaf_rn(n[6], 256.f, __fmaf_rn(n[5], 16.f, n[4])));
+  return __byte_perm(__float_as_uint(__fadd_rn(lo, 0x1p23f)), __float_as_uint(__fadd_rn(hi, 0x1p23f)), 0x5410);
+}
+
+// A warp's threads each hold CH 16-byte chunks that are consecutive in the output (thread t: chunks
+// t*CH .. t*CH+CH-1 of the warp's run).  Pass them through the warp's slice of shared memory so that
+// store instruction i writes chunks 32 i .. 32 i + 31.  The chunk position inside a thread's group is
+// XOR-ed with a few bits of the thread index: without it the 8 threads of a quarter-warp, CH chunks
+// apart, would fall on the same banks.
+template <int CH>
+__device__ __forceinline__ void warp_store_chunks(uint4* stage_warp, const uint4 (&mine)[CH], uint4* out_warp,
+                                                  int valid_threads) {
+  const int lane = threadIdx.x & 31;
+  constexpr int G = 8 / CH;
+#pragma unroll
+  for (int j = 0; j < CH; ++j) stage_warp[lane * CH + (j ^ ((lane / G) & (CH - 1)))] = mine[j];
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < CH; ++i) {
+    const int c = i * 32 + lane, t = c / CH, j = c % CH;
+    const uint4 x = stage_warp[t * CH + (j ^ ((t / G) & (CH - 1)))];
+    if (t < valid_threads) out_warp[c] = x;
+  }
+  __syncwarp();
+}
+
+// Element offset in a row-major tensor of 16-element block b.
+__device__ __forceinline__ int64_t block_offset(int64_t b, uint32_t blocks_per_row, int64_t ld, bool dense) {
+  if (dense) return b * 16;
+  const uint32_t row = (uint32_t)b / blocks_per_row;
+  return (int64_t)row * ld + (int64_t)((uint32_t)b - row * blocks_per_row) * 16;
+}
+
+__device__ __forceinline__ float tensor_scale(float s_global_in, const uint32_t* amax_word) {
+  if (s_global_in > 0.f) return s_global_in;
+  const float amax_t = __uint_as_float(*amax_word);
+  return amax_t == 0.f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);
+}
+
+// Block maximum of |w| and whether the packed division may be used (see block_quotients).
+__device__ __forceinline__ float block_amax(const float (&w)[16], bool* has_minute) {
+  float amax = 0.f;
+  bool minute = false;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    amax = fmaxf(amax, fabsf(w[i]));
+    minute |= fabsf(w[i]) < 0x1p-80f;
+  }
+  *has_minute = minute;
+  return amax;
+}
+__device__ __forceinline__ bool fast_division_ok(float s, float amax, bool has_minute) {
+  return s >= 0x1p-40f && s <= 0x1p40f && amax <= 0x1p40f && !has_minute;
+}
+
 // ---- pass 2: block scales, bracket, V_init -------------------------------------
-__global__ void __launch_bounds__(EW_THREADS)
+// Bracket of w~ = min(|w| / s, 6): interval index k (lower node = node k) and V_init = (w~ - lower node) / width.
+template <bool FAST>
+__device__ __forceinline__ void bracket_block(const float (&w)[16], float s, float (&v)[16], uint32_t (&cw)[2]) {
+  float q[16];
+  block_quotients<FAST>(w, s, q);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float n[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const grid_pos g = locate(q[8 * h + i]);
+      v[8 * h + i] = g.v;
+      n[i] = __fmaf_rn(8.0f, negative_flag<FAST>(w[8 * h + i], q[8 * h + i]), g.k);
+    }
+    cw[h] = pack_nibbles(n);
+  }
+}
+
+__global__ void __launch_bounds__(EW_THREADS, 4)
 softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw,
                       float s_global_in, const uint32_t* __restrict__ amax_word,
                       uint8_t* __restrict__ scales, float* __restrict__ s_global_out,
                       uint8_t* __restrict__ code, float* __restrict__ V) {
-  float s_global;
-  if (s_global_in > 0.f) {
-    s_global = s_global_in;
-  } else {
-    float amax_t = __uint_as_float(*amax_word);
-    s_global = amax_t == 0.f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);
-  }
+  __shared__ uint4 stage[EW_THREADS * 4];
+  asm volatile("griddepcontrol.wait;" ::: "memory");      // the maximum (and W itself) may come from the kernel before
+  const float s_global = tensor_scale(s_global_in, amax_word);
   if (blockIdx.x == 0 && threadIdx.x == 0) *s_global_out = s_global;
   const float d = __fmul_rn(s_global, 6.0f);
 
-  const uint32_t groups_per_row = K / 8;
-  const int64_t total = (int64_t)O * groups_per_row;
+  const uint32_t blocks_per_row = K / 16;
+  const int64_t total = (int64_t)O * blocks_per_row;
   const bool dense = ldw == K;
-  // the grid is sized so that every warp is either fully inside or the tail is padded with idle lanes
-  for (int64_t g0 = (int64_t)blockIdx.x * blockDim.x; g0 < total; g0 += (int64_t)gridDim.x * blockDim.x) {
-    int64_t g = g0 + threadIdx.x;
-    bool valid = g < total;
-    int64_t gc = valid ? g : total - 1;
-    float w[8];
-    load8(W, w_dtype, w_offset(gc, groups_per_row, ldw, dense), w);
-    float amax = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[i]));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));   // partner holds the other half-block
+  uint4* stage_warp = stage + (threadIdx.x & ~31) * 4;
+  for (int64_t b0 = (int64_t)blockIdx.x * blockDim.x; b0 < total; b0 += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t b = b0 + threadIdx.x;
+    const bool valid = b < total;
+    float w[16];
+    load16(W, w_dtype, block_offset(valid ? b : total - 1, blocks_per_row, ldw, dense), w);
+    bool has_minute;
+    const float amax = block_amax(w, &has_minute);
     const uint32_t sb = faar_float_to_e4m3(__fdiv_rn(amax, d));
     const float s = __fmul_rn(faar_e4m3_to_float(sb), s_global);
-    uint32_t cw = 0;
-    float v[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      float wt = s > 0.f ? __fdiv_rn(fabsf(w[i]), s) : 0.f;
-      wt = fminf(wt, 6.0f);
-      // From 1 upwards the nodes are the floats with a one-bit mantissa, so the bits of w~ give the bracket:
-      // lower node = w~ with the mantissa cut to its top bit, interval index = (bits >> 22) - 252
-      // ([1,1.5) -> 2, [1.5,2) -> 3, [2,3) -> 4, [3,4) -> 5, [4,6) -> 6), 1 / width = 2^(1 - exponent).
-      // Below 1 the nodes 0, 0.5, 1 are 0.5 apart.  w~ = 6 (the clamp) closes the last interval: k = 6, v = 1.
-      const uint32_t wb = __float_as_uint(wt);
-      const bool ge1 = wt >= 1.0f, geh = wt >= 0.5f;
-      const float lo = ge1 ? __uint_as_float(wb & 0xFFC00000u) : (geh ? 0.5f : 0.0f);
-      const float inv_w = ge1 ? __uint_as_float(0x7F800000u - (wb & 0x7F800000u)) : 2.0f;      // 2, 1, 0.5
-      uint32_t k = ge1 ? (wb >> 22) - 252u : (geh ? 1u : 0u);
-      float vi = __fmul_rn(__fsub_rn(wt, lo), inv_w);
-      if (wt >= 6.0f) { k = 6u; vi = 1.0f; }
-      v[i] = vi;
-      cw |= (k | (w[i] < 0.f ? 8u : 0u)) << (4 * i);                  // -0.0 counts as positive
+    uint32_t cw[2];
+    uint4 vq[4];
+    float(&v)[16] = *reinterpret_cast<float(*)[16]>(vq);
+    if (fast_division_ok(s, amax, has_minute)) bracket_block<true>(w, s, v, cw);
+    else bracket_block<false>(w, s, v, cw);
+    const int64_t warp_first = b0 + (threadIdx.x & ~31);
+    if (warp_first < total) {
+      const int64_t left = total - warp_first;
+      warp_store_chunks<4>(stage_warp, vq, reinterpret_cast<uint4*>(V + warp_first * 16), left < 32 ? (int)left : 32);
     }
     if (valid) {
-      const int64_t e = g * 8;                 // V, code, scales are dense
-      const bool first_half = (g & 1) == 0;    // K % 16 == 0: even groups start a scale block
-      float4* vp = reinterpret_cast<float4*>(V + e);
-      vp[0] = make_float4(v[0], v[1], v[2], v[3]);
-      vp[1] = make_float4(v[4], v[5], v[6], v[7]);
-      *reinterpret_cast<uint32_t*>(code + e / 2) = cw;
-      if (first_half) scales[e / 16] = (uint8_t)sb;
+      *reinterpret_cast<uint2*>(code + b * 8) = make_uint2(cw[0], cw[1]);
+      scales[b] = (uint8_t)sb;
     }
   }
 }
@@ -145,64 +299,78 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
 // magnitude (Eq. 7 applied to the initial position).  The output holds sign * node * block scale, which
 // needs at most 7 significant bits and is therefore exact in BF16; the FP32 tensor scale stays outside
 // (X_q = Xq_units * s_global) and is applied by the GEMM epilogues.
-__global__ void __launch_bounds__(EW_THREADS)
+// From the bracket: t = [v >= 0.5] (v - 0.5 is a multiple of 2^-25, so a saturating FMA by 2^25 gives 0 or 1),
+// node = (j + t) * spacing, magnitude code = k + t.
+template <bool FAST>
+__device__ __forceinline__ void nearest_block(const float (&w)[16], float s, float sg, uint32_t (&o)[8], uint32_t (&cw)[2]) {
+  float q[16];
+  block_quotients<FAST>(w, s, q);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float n[8];
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) {
+      float out[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int x = 8 * h + i + e;
+        const grid_pos g = locate(q[x]);
+        const float t = __saturatef(__fmaf_rn(g.v, 0x1p25f, 1.0f - 0x1p24f));
+        const float neg = negative_flag<FAST>(w[x], q[x]);
+        n[i + e] = __fmaf_rn(8.0f, neg, __fadd_rn(g.k, t));
+        const float spacing_sg = __fmul_rn(__fmaf_rn(0.5f, g.t1, __fadd_rn(0.5f, g.t2)), sg);   // {.5, 1, 2} * sg
+        const float mag = __fmul_rn(__fadd_rn(g.j, t), spacing_sg);                          // exact: 3 x 4 bits at most
+        out[e] = __fmul_rn(mag, __fmaf_rn(-2.0f, neg, 1.0f));
+      }
+      // both values have zero low halves: the BF16 pair is the two high halves
+      o[(8 * h + i) >> 1] = __byte_perm(__float_as_uint(out[0]), __float_as_uint(out[1]), 0x7632);
+    }
+    cw[h] = pack_nibbles(n);
+  }
+}
+
+__global__ void __launch_bounds__(EW_THREADS, 3)
 act_fakequant_kernel(const __nv_bfloat16* __restrict__ X, int T, int K, int64_t ldx, float s_global_in,
                      const uint32_t* __restrict__ amax_word, __nv_bfloat16* __restrict__ Xq, int64_t ldq,
                      float* __restrict__ s_global_out, uint8_t* __restrict__ packed, uint8_t* __restrict__ scales) {
-  float s_global;
-  if (s_global_in > 0.f) {
-    s_global = s_global_in;
-  } else {
-    float amax_t = __uint_as_float(*amax_word);
-    s_global = amax_t == 0.f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);
-  }
+  __shared__ uint4 stage[EW_THREADS * 2];
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const float s_global = tensor_scale(s_global_in, amax_word);
   if (blockIdx.x == 0 && threadIdx.x == 0) *s_global_out = s_global;
   const float d = __fmul_rn(s_global, 6.0f);
-  const uint32_t groups_per_row = K / 8;
-  const int64_t total = (int64_t)T * groups_per_row;
-  for (int64_t g0 = (int64_t)blockIdx.x * blockDim.x; g0 < total; g0 += (int64_t)gridDim.x * blockDim.x) {
-    int64_t g = g0 + threadIdx.x;
-    bool valid = g < total;
-    int64_t gc = valid ? g : total - 1;
-    const uint32_t row = (uint32_t)gc / groups_per_row, col = ((uint32_t)gc - row * groups_per_row) * 8;
-    float w[8];
-    load8(X, FAAR_BF16, (int64_t)row * ldx + col, w);
-    float amax = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[i]));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));   // partner holds the other half-block
+  const uint32_t blocks_per_row = K / 16;
+  const int64_t total = (int64_t)T * blocks_per_row;
+  const bool dense_in = ldx == K, dense_out = ldq == K;
+  uint4* stage_warp = stage + (threadIdx.x & ~31) * 2;
+  for (int64_t b0 = (int64_t)blockIdx.x * blockDim.x; b0 < total; b0 += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t b = b0 + threadIdx.x;
+    const bool valid = b < total;
+    float w[16];
+    load16(X, FAAR_BF16, block_offset(valid ? b : total - 1, blocks_per_row, ldx, dense_in), w);
+    bool has_minute;
+    const float amax = block_amax(w, &has_minute);
     const uint32_t sb = faar_float_to_e4m3(__fdiv_rn(amax, d));
     const float sg = faar_e4m3_to_float(sb);
     const float s = __fmul_rn(sg, s_global);
-    uint32_t cw = 0;
-    float q[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      float wt = s > 0.f ? __fdiv_rn(fabsf(w[i]), s) : 0.f;
-      wt = fminf(wt, 6.0f);
-      // Nearest node, a tie to the larger one.  From 1 upwards the nodes are the floats with a one-bit
-      // mantissa: add a quarter of the binade and cut the mantissa to its top bit (5 -> 6, 3.5 -> 4,
-      // 1.25 -> 1.5; 6 stays 6).  Below 1 the nodes 0, 0.5, 1 are 0.5 apart.
-      const uint32_t rb = (__float_as_uint(wt) + 0x00200000u) & 0xFFC00000u;
-      const float node = wt >= 1.0f ? __uint_as_float(rb) : (wt >= 0.75f ? 1.0f : (wt >= 0.25f ? 0.5f : 0.0f));
-      // E2M1 magnitude code of the node: 0, 0.5 -> 0, 1; from 1 upwards exponent and mantissa bit count on
-      const int c = node >= 1.0f ? (int)(__float_as_uint(node) >> 22) - 252 : (node > 0.0f ? 1 : 0);
-      const float mag = __fmul_rn(node, sg);                      // exact: 2 x 4 significant bits
-      const bool neg = w[i] < 0.f;
-      q[i] = neg ? -mag : mag;
-      cw |= ((uint32_t)c | (neg ? 8u : 0u)) << (4 * i);
+    uint32_t cw[2];
+    uint4 oq[2];
+    uint32_t(&o)[8] = *reinterpret_cast<uint32_t(*)[8]>(oq);
+    if (fast_division_ok(s, amax, has_minute)) nearest_block<true>(w, s, sg, o, cw);
+    else nearest_block<false>(w, s, sg, o, cw);
+    if (dense_out) {
+      const int64_t warp_first = b0 + (threadIdx.x & ~31);
+      if (warp_first < total) {
+        const int64_t left = total - warp_first;
+        warp_store_chunks<2>(stage_warp, oq, reinterpret_cast<uint4*>(Xq + warp_first * 16), left < 32 ? (int)left : 32);
+      }
+    } else if (valid) {
+      uint4* p = reinterpret_cast<uint4*>(Xq + block_offset(b, blocks_per_row, ldq, false));
+      p[0] = oq[0];
+      p[1] = oq[1];
     }
     if (valid) {
-      uint32_t o[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 p2 = __floats2bfloat162_rn(q[2 * i], q[2 * i + 1]);
-        o[i] = *reinterpret_cast<uint32_t*>(&p2);
-      }
-      *reinterpret_cast<uint4*>(Xq + (int64_t)row * ldq + col) = make_uint4(o[0], o[1], o[2], o[3]);
-      const int64_t e = g * 8;                 // packed and scales are dense
-      if (packed) *reinterpret_cast<uint32_t*>(packed + e / 2) = cw;
-      if (scales && (g & 1) == 0) scales[e / 16] = (uint8_t)sb;
+      if (packed) *reinterpret_cast<uint2*>(packed + b * 8) = make_uint2(cw[0], cw[1]);
+      if (scales) scales[b] = (uint8_t)sb;
     }
   }
 }
@@ -469,37 +637,54 @@ int grid_for(const faar_ctx* ctx, int64_t work_items, int per_sm) {
 
 }  // namespace
 
+// Launch with stream serialisation relaxed: the kernel's CTAs may be scheduled while the kernel before
+// it drains; the kernel itself waits (griddepcontrol.wait) before it touches global memory.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_relaxed(faar_ctx* ctx, void (*kernel)(KArgs...), int grid, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(EW_THREADS, 1, 1);
+  cfg.stream = ctx->stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 int faar_launch_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float s_global_in,
                                uint8_t* scales, float* s_global_out, uint8_t* code, float* V,
                                uint32_t* amax_word) {
   const int64_t groups = (int64_t)s->O * (s->K / 8);
-  const int grid = grid_for(ctx, groups, 8);
   if (!(s_global_in > 0.f)) {
     cudaError_t e = cudaMemsetAsync(amax_word, 0, sizeof(uint32_t), ctx->stream);
     if (e != cudaSuccess) return (int)e;
     faar_prof_scope ps(ctx, FAAR_K_AMAX);
-    amax_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, amax_word);
+    amax_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, amax_word);
   }
   faar_prof_scope ps(ctx, FAAR_K_SOFTQUANT_INIT);
-  softquant_init_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, s_global_in,
-                                                               amax_word, scales, s_global_out, code, V);
+  cudaError_t e = launch_relaxed(ctx, softquant_init_kernel, grid_for(ctx, groups / 2, 4), W, s->w_dtype, s->O, s->K,
+                                 s->ldw, s_global_in, (const uint32_t*)amax_word, scales, s_global_out, code, V);
+  if (e != cudaSuccess) return (int)e;
   return (int)cudaGetLastError();
 }
 
 int faar_launch_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_t ldx, float s_global_in, void* Xq,
                               int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales, uint32_t* amax_word) {
   const int64_t groups = (int64_t)T * (K / 8);
-  const int grid = grid_for(ctx, groups, 8);
   if (!(s_global_in > 0.f)) {
     cudaError_t e = cudaMemsetAsync(amax_word, 0, sizeof(uint32_t), ctx->stream);
     if (e != cudaSuccess) return (int)e;
     faar_prof_scope ps(ctx, FAAR_K_AMAX);
-    amax_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(X, FAAR_BF16, T, K, ldx, amax_word);
+    amax_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(X, FAAR_BF16, T, K, ldx, amax_word);
   }
   faar_prof_scope ps(ctx, FAAR_K_ACT_FAKEQUANT);
-  act_fakequant_kernel<<<grid, EW_THREADS, 0, ctx->stream>>>(reinterpret_cast<const __nv_bfloat16*>(X), T, K, ldx,
-                                                            s_global_in, amax_word, reinterpret_cast<__nv_bfloat16*>(Xq),
-                                                            ldq, s_global_out, packed, scales);
+  cudaError_t e = launch_relaxed(ctx, act_fakequant_kernel, grid_for(ctx, groups / 2, 3),
+                                 reinterpret_cast<const __nv_bfloat16*>(X), T, K, ldx, s_global_in,
+                                 (const uint32_t*)amax_word, reinterpret_cast<__nv_bfloat16*>(Xq), ldq, s_global_out,
+                                 packed, scales);
+  if (e != cudaSuccess) return (int)e;
   return (int)cudaGetLastError();
 }
 
