@@ -436,7 +436,7 @@ int faar_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
     return FAAR_ERR_WORKSPACE;
   FAAR_DEVICE_GUARD(ctx);
-  uint32_t* amax_word = reinterpret_cast<uint32_t*>(workspace) + 1;
+  unsigned long long* amax_word = reinterpret_cast<unsigned long long*>(workspace) + 2;
   return cuda_fail(ctx, faar_launch_softquant_init(ctx, s, W, s_global_in, scales, s_global_out, code, V_init,
                                                    amax_word));
 }
@@ -488,7 +488,7 @@ int faar_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_t ldx, 
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < FAAR_WS_HEADER)
     return FAAR_ERR_WORKSPACE;
   FAAR_DEVICE_GUARD(ctx);
-  uint32_t* amax_word = reinterpret_cast<uint32_t*>(workspace) + 1;
+  unsigned long long* amax_word = reinterpret_cast<unsigned long long*>(workspace) + 2;
   return cuda_fail(ctx, faar_launch_act_fakequant(ctx, T, K, X, ldx, s_global_in, Xq_units, ldq, s_global_out, packed,
                                                   scales, amax_word));
 }

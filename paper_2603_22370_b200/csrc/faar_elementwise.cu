@@ -8,26 +8,11 @@
 // threads of a block exchange their maxima with one shuffle.
 #include "faar_internal.cuh"
 
+#include <atomic>
+
 namespace {
 
 constexpr int EW_THREADS = 256;
-
-__device__ __forceinline__ void load8(const void* W, int w_dtype, int64_t idx, float (&w)[8]) {
-  if (w_dtype == FAAR_BF16) {
-    uint4 raw = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W) + idx);
-    const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      w[2 * i] = __uint_as_float(r[i] << 16);
-      w[2 * i + 1] = __uint_as_float(r[i] & 0xFFFF0000u);
-    }
-  } else {
-    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(W) + idx);
-    float4 a = p[0], b = p[1];
-    w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
-    w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
-  }
-}
 
 // Element offset in W of 8-element group g.  Dense rows (ldw == K) need no division; otherwise the
 // row comes from a 32-bit division (the host checks that the group count fits).
@@ -38,33 +23,54 @@ __device__ __forceinline__ int64_t w_offset(int64_t g, uint32_t groups_per_row, 
 }
 
 // ---- pass 1: max |W| over the tensor -----------------------------------------
+// One thread takes 8-value groups g, g + stride, ...; eight 16-byte loads (FP32: sixteen) are in flight per
+// thread and iteration, the ragged end re-reads the last group instead of branching.  BF16 values are
+// compared as packed pairs.
+template <bool BF16IN>
 __global__ void __launch_bounds__(EW_THREADS)
-amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, uint32_t* amax_word) {
+amax_kernel(const void* __restrict__ W, int O, int K, int64_t ldw, unsigned long long* amax_word, uint32_t epoch) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel waits for this one's end itself
   const uint32_t groups_per_row = K / 8;
   const int64_t total = (int64_t)O * groups_per_row;
   const bool dense = ldw == K;
-  float amax = 0.f;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  // four independent 16-byte (32-byte for FP32) loads in flight per thread
-  for (; g + 3 * stride < total; g += 4 * stride) {
-    float w[4][8];
+  constexpr int DEPTH = 8;
+  float amax = 0.f;
+  __nv_bfloat162 mx2 = __float2bfloat162_rn(0.f);
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += DEPTH * stride) {
+    if (BF16IN) {
+      uint4 raw[DEPTH];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      load8(W, w_dtype, w_offset(g + j * stride, groups_per_row, ldw, dense), w[j]);
+      for (int j = 0; j < DEPTH; ++j) {
+        const int64_t gj = min(g + j * stride, total - 1);
+        raw[j] = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W) +
+                                                 w_offset(gj, groups_per_row, ldw, dense));
+      }
+#pragma unroll
+      for (int j = 0; j < DEPTH; ++j) {
+        const uint32_t r[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) mx2 = __hmax2(mx2, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&r[i])));
+      }
+    } else {
+      float4 raw[DEPTH][2];
+#pragma unroll
+      for (int j = 0; j < DEPTH; ++j) {
+        const int64_t gj = min(g + j * stride, total - 1);
+        const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(W) +
+                                                          w_offset(gj, groups_per_row, ldw, dense));
+        raw[j][0] = p[0];
+        raw[j][1] = p[1];
+      }
+#pragma unroll
+      for (int j = 0; j < DEPTH; ++j)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          amax = fmaxf(fmaxf(amax, fabsf(raw[j][h].x)),
+                       fmaxf(fmaxf(fabsf(raw[j][h].y), fabsf(raw[j][h].z)), fabsf(raw[j][h].w)));
     }
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-#pragma unroll
-      for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[j][i]));
   }
-  for (; g < total; g += stride) {
-    float w[8];
-    load8(W, w_dtype, w_offset(g, groups_per_row, ldw, dense), w);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(w[i]));
-  }
+  if (BF16IN) amax = fmaxf(__low2float(mx2), __high2float(mx2));
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
   __shared__ float s_max[EW_THREADS / 32];
@@ -73,7 +79,9 @@ amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, 
   if (threadIdx.x == 0) {
     float m = 0.f;
     for (int i = 0; i < EW_THREADS / 32; ++i) m = fmaxf(m, s_max[i]);
-    atomicMax(amax_word, __float_as_uint(m));   // non-negative floats order like their bit patterns
+    // non-negative floats order like their bit patterns; the call's serial number on top makes a value left
+    // by an earlier call lose against any value of this one, so the word is never cleared between calls
+    atomicMax(amax_word, ((unsigned long long)epoch << 32) | __float_as_uint(m));
   }
 }
 
@@ -90,24 +98,61 @@ amax_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw, 
 // are summed as small integers in FP32.  Every such operation is exact, so the results equal those
 // of the compare-and-select formulation bit for bit.
 
-// 16 consecutive values as binary32.
-__device__ __forceinline__ void load16(const void* W, int w_dtype, int64_t idx, float (&w)[16]) {
-  if (w_dtype == FAAR_BF16) {
+// The 16 values of a block as loaded: 32 bytes of BF16 (in r[0..7]) or 64 bytes of FP32.
+struct block_raw {
+  uint32_t r[16];
+};
+template <bool BF16IN>
+__device__ __forceinline__ block_raw load_block(const void* W, int64_t idx) {
+  block_raw raw;
+  if (BF16IN) {
     const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W) + idx);
     const uint4 r0 = p[0], r1 = p[1];
-    const uint32_t r[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      w[2 * i] = __uint_as_float(r[i] << 16);
-      w[2 * i + 1] = __uint_as_float(r[i] & 0xFFFF0000u);
-    }
+    raw.r[0] = r0.x; raw.r[1] = r0.y; raw.r[2] = r0.z; raw.r[3] = r0.w;
+    raw.r[4] = r1.x; raw.r[5] = r1.y; raw.r[6] = r1.z; raw.r[7] = r1.w;
   } else {
-    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(W) + idx);
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(W) + idx);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const float4 r = p[j];
-      w[4 * j] = r.x; w[4 * j + 1] = r.y; w[4 * j + 2] = r.z; w[4 * j + 3] = r.w;
+      const uint4 r = p[j];
+      raw.r[4 * j] = r.x; raw.r[4 * j + 1] = r.y; raw.r[4 * j + 2] = r.z; raw.r[4 * j + 3] = r.w;
     }
+  }
+  return raw;
+}
+
+// Values as binary32, the block maximum of |w|, and whether some magnitude is below 2^-80 (zero included):
+// such a block takes the division instruction instead of the shared reciprocal (see block_quotients).
+// BF16 input: maximum and minimum run on the packed pairs, two values per instruction.
+template <bool BF16IN>
+__device__ __forceinline__ float unpack_block(const block_raw& raw, float (&w)[16], bool* has_minute) {
+  if (BF16IN) {
+    __nv_bfloat162 mx = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&raw.r[0]));
+    __nv_bfloat162 mn = mx;
+#pragma unroll
+    for (int i = 1; i < 8; ++i) {
+      const __nv_bfloat162 a = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&raw.r[i]));
+      mx = __hmax2(mx, a);
+      mn = __hmin2(mn, a);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      w[2 * i] = __uint_as_float(raw.r[i] << 16);
+      w[2 * i + 1] = __uint_as_float(raw.r[i] & 0xFFFF0000u);
+    }
+    *has_minute = fminf(__low2float(mn), __high2float(mn)) < 0x1p-80f;
+    return fmaxf(__low2float(mx), __high2float(mx));
+  } else {
+    float amax = 0.f;
+    bool minute = false;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      w[i] = __uint_as_float(raw.r[i]);
+      amax = fmaxf(amax, fabsf(w[i]));
+      minute |= fabsf(w[i]) < 0x1p-80f;
+    }
+    *has_minute = minute;
+    return amax;
   }
 }
 
@@ -164,7 +209,7 @@ __device__ __forceinline__ grid_pos locate(float q_signed) {
   const float fl = __fsub_rn(__fadd_rd(u, 0x1p23f), 0x1p23f);      // floor(u): the sum has unit spacing, rounded down
   g.j = __fmaf_rn(g.t2, __fsub_rn(2.0f, fl), fl);
   g.v = __fsub_rn(u, g.j);
-  g.k = __fmaf_rn(2.0f, g.t2, __fmaf_rn(2.0f, g.t1, g.j));
+  g.k = __fmaf_rn(2.0f, __fadd_rn(g.t1, g.t2), g.j);
   return g;
 }
 
@@ -212,24 +257,12 @@ __device__ __forceinline__ int64_t block_offset(int64_t b, uint32_t blocks_per_r
   return (int64_t)row * ld + (int64_t)((uint32_t)b - row * blocks_per_row) * 16;
 }
 
-__device__ __forceinline__ float tensor_scale(float s_global_in, const uint32_t* amax_word) {
+__device__ __forceinline__ float tensor_scale(float s_global_in, const unsigned long long* amax_word) {
   if (s_global_in > 0.f) return s_global_in;
-  const float amax_t = __uint_as_float(*amax_word);
+  const float amax_t = __uint_as_float((uint32_t)*amax_word);      // low half: the maximum's bits
   return amax_t == 0.f ? 1.0f : __fdiv_rn(amax_t, 2688.0f);
 }
 
-// Block maximum of |w| and whether the packed division may be used (see block_quotients).
-__device__ __forceinline__ float block_amax(const float (&w)[16], bool* has_minute) {
-  float amax = 0.f;
-  bool minute = false;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    amax = fmaxf(amax, fabsf(w[i]));
-    minute |= fabsf(w[i]) < 0x1p-80f;
-  }
-  *has_minute = minute;
-  return amax;
-}
 __device__ __forceinline__ bool fast_division_ok(float s, float amax, bool has_minute) {
   return s >= 0x1p-40f && s <= 0x1p40f && amax <= 0x1p40f && !has_minute;
 }
@@ -253,9 +286,10 @@ __device__ __forceinline__ void bracket_block(const float (&w)[16], float s, flo
   }
 }
 
-__global__ void __launch_bounds__(EW_THREADS, 4)
-softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int64_t ldw,
-                      float s_global_in, const uint32_t* __restrict__ amax_word,
+template <bool BF16IN>
+__global__ void __launch_bounds__(EW_THREADS, 3)
+softquant_init_kernel(const void* __restrict__ W, int O, int K, int64_t ldw,
+                      float s_global_in, const unsigned long long* __restrict__ amax_word,
                       uint8_t* __restrict__ scales, float* __restrict__ s_global_out,
                       uint8_t* __restrict__ code, float* __restrict__ V) {
   __shared__ uint4 stage[EW_THREADS * 4];
@@ -267,14 +301,21 @@ softquant_init_kernel(const void* __restrict__ W, int w_dtype, int O, int K, int
   const uint32_t blocks_per_row = K / 16;
   const int64_t total = (int64_t)O * blocks_per_row;
   const bool dense = ldw == K;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   uint4* stage_warp = stage + (threadIdx.x & ~31) * 4;
-  for (int64_t b0 = (int64_t)blockIdx.x * blockDim.x; b0 < total; b0 += (int64_t)gridDim.x * blockDim.x) {
+  int64_t b0 = (int64_t)blockIdx.x * blockDim.x;
+  if (b0 >= total) return;
+  // the next block's values are requested before this block's arithmetic starts
+  block_raw next = load_block<BF16IN>(W, block_offset(min(b0 + threadIdx.x, total - 1), blocks_per_row, ldw, dense));
+  for (; b0 < total; b0 += stride) {
     const int64_t b = b0 + threadIdx.x;
     const bool valid = b < total;
+    const block_raw raw = next;
+    if (b0 + stride < total)
+      next = load_block<BF16IN>(W, block_offset(min(b + stride, total - 1), blocks_per_row, ldw, dense));
     float w[16];
-    load16(W, w_dtype, block_offset(valid ? b : total - 1, blocks_per_row, ldw, dense), w);
     bool has_minute;
-    const float amax = block_amax(w, &has_minute);
+    const float amax = unpack_block<BF16IN>(raw, w, &has_minute);
     const uint32_t sb = faar_float_to_e4m3(__fdiv_rn(amax, d));
     const float s = __fmul_rn(faar_e4m3_to_float(sb), s_global);
     uint32_t cw[2];
@@ -331,7 +372,7 @@ __device__ __forceinline__ void nearest_block(const float (&w)[16], float s, flo
 
 __global__ void __launch_bounds__(EW_THREADS, 3)
 act_fakequant_kernel(const __nv_bfloat16* __restrict__ X, int T, int K, int64_t ldx, float s_global_in,
-                     const uint32_t* __restrict__ amax_word, __nv_bfloat16* __restrict__ Xq, int64_t ldq,
+                     const unsigned long long* __restrict__ amax_word, __nv_bfloat16* __restrict__ Xq, int64_t ldq,
                      float* __restrict__ s_global_out, uint8_t* __restrict__ packed, uint8_t* __restrict__ scales) {
   __shared__ uint4 stage[EW_THREADS * 2];
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -342,13 +383,19 @@ act_fakequant_kernel(const __nv_bfloat16* __restrict__ X, int T, int K, int64_t 
   const int64_t total = (int64_t)T * blocks_per_row;
   const bool dense_in = ldx == K, dense_out = ldq == K;
   uint4* stage_warp = stage + (threadIdx.x & ~31) * 2;
-  for (int64_t b0 = (int64_t)blockIdx.x * blockDim.x; b0 < total; b0 += (int64_t)gridDim.x * blockDim.x) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int64_t b0 = (int64_t)blockIdx.x * blockDim.x;
+  if (b0 >= total) return;
+  block_raw next = load_block<true>(X, block_offset(min(b0 + threadIdx.x, total - 1), blocks_per_row, ldx, dense_in));
+  for (; b0 < total; b0 += stride) {
     const int64_t b = b0 + threadIdx.x;
     const bool valid = b < total;
+    const block_raw raw = next;
+    if (b0 + stride < total)
+      next = load_block<true>(X, block_offset(min(b + stride, total - 1), blocks_per_row, ldx, dense_in));
     float w[16];
-    load16(X, FAAR_BF16, block_offset(valid ? b : total - 1, blocks_per_row, ldx, dense_in), w);
     bool has_minute;
-    const float amax = block_amax(w, &has_minute);
+    const float amax = unpack_block<true>(raw, w, &has_minute);
     const uint32_t sb = faar_float_to_e4m3(__fdiv_rn(amax, d));
     const float sg = faar_e4m3_to_float(sb);
     const float s = __fmul_rn(sg, s_global);
@@ -653,37 +700,55 @@ static cudaError_t launch_relaxed(faar_ctx* ctx, void (*kernel)(KArgs...), int g
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Serial number of a tensor-maximum pass, shared by all contexts of the process (a workspace may pass from one
+// context to another).  0 is what a freshly initialised workspace header holds and is skipped.
+static std::atomic<uint32_t> g_amax_epoch{0};
+
+static int launch_amax(faar_ctx* ctx, bool bf16, const void* W, int rows, int K, int64_t ld,
+                       unsigned long long* amax_word) {
+  uint32_t epoch = ++g_amax_epoch;
+  if (epoch == 0) {                                        // the counter wrapped: start over from a cleared word
+    cudaError_t e = cudaMemsetAsync(amax_word, 0, sizeof(unsigned long long), ctx->stream);
+    if (e != cudaSuccess) return (int)e;
+    epoch = ++g_amax_epoch;
+  }
+  const int64_t groups = (int64_t)rows * (K / 8);
+  faar_prof_scope ps(ctx, FAAR_K_AMAX);
+  const int grid = grid_for(ctx, (groups + 7) / 8, 8);
+  if (bf16) amax_kernel<true><<<grid, EW_THREADS, 0, ctx->stream>>>(W, rows, K, ld, amax_word, epoch);
+  else amax_kernel<false><<<grid, EW_THREADS, 0, ctx->stream>>>(W, rows, K, ld, amax_word, epoch);
+  return (int)cudaGetLastError();
+}
+
 int faar_launch_softquant_init(faar_ctx* ctx, const faar_shape* s, const void* W, float s_global_in,
                                uint8_t* scales, float* s_global_out, uint8_t* code, float* V,
-                               uint32_t* amax_word) {
-  const int64_t groups = (int64_t)s->O * (s->K / 8);
+                               unsigned long long* amax_word) {
+  const int64_t blocks = (int64_t)s->O * (s->K / 16);
   if (!(s_global_in > 0.f)) {
-    cudaError_t e = cudaMemsetAsync(amax_word, 0, sizeof(uint32_t), ctx->stream);
-    if (e != cudaSuccess) return (int)e;
-    faar_prof_scope ps(ctx, FAAR_K_AMAX);
-    amax_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(W, s->w_dtype, s->O, s->K, s->ldw, amax_word);
+    int e = launch_amax(ctx, s->w_dtype == FAAR_BF16, W, s->O, s->K, s->ldw, amax_word);
+    if (e) return e;
   }
   faar_prof_scope ps(ctx, FAAR_K_SOFTQUANT_INIT);
-  cudaError_t e = launch_relaxed(ctx, softquant_init_kernel, grid_for(ctx, groups / 2, 4), W, s->w_dtype, s->O, s->K,
-                                 s->ldw, s_global_in, (const uint32_t*)amax_word, scales, s_global_out, code, V);
+  cudaError_t e = launch_relaxed(ctx, s->w_dtype == FAAR_BF16 ? softquant_init_kernel<true> : softquant_init_kernel<false>,
+                                 grid_for(ctx, blocks, 3), W, s->O, s->K, s->ldw, s_global_in,
+                                 (const unsigned long long*)amax_word, scales, s_global_out, code, V);
   if (e != cudaSuccess) return (int)e;
   return (int)cudaGetLastError();
 }
 
 int faar_launch_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_t ldx, float s_global_in, void* Xq,
-                              int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales, uint32_t* amax_word) {
-  const int64_t groups = (int64_t)T * (K / 8);
+                              int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales,
+                              unsigned long long* amax_word) {
+  const int64_t blocks = (int64_t)T * (K / 16);
   if (!(s_global_in > 0.f)) {
-    cudaError_t e = cudaMemsetAsync(amax_word, 0, sizeof(uint32_t), ctx->stream);
-    if (e != cudaSuccess) return (int)e;
-    faar_prof_scope ps(ctx, FAAR_K_AMAX);
-    amax_kernel<<<grid_for(ctx, groups, 8), EW_THREADS, 0, ctx->stream>>>(X, FAAR_BF16, T, K, ldx, amax_word);
+    int e = launch_amax(ctx, true, X, T, K, ldx, amax_word);
+    if (e) return e;
   }
   faar_prof_scope ps(ctx, FAAR_K_ACT_FAKEQUANT);
-  cudaError_t e = launch_relaxed(ctx, act_fakequant_kernel, grid_for(ctx, groups / 2, 3),
+  cudaError_t e = launch_relaxed(ctx, act_fakequant_kernel, grid_for(ctx, blocks, 3),
                                  reinterpret_cast<const __nv_bfloat16*>(X), T, K, ldx, s_global_in,
-                                 (const uint32_t*)amax_word, reinterpret_cast<__nv_bfloat16*>(Xq), ldq, s_global_out,
-                                 packed, scales);
+                                 (const unsigned long long*)amax_word, reinterpret_cast<__nv_bfloat16*>(Xq), ldq,
+                                 s_global_out, packed, scales);
   if (e != cudaSuccess) return (int)e;
   return (int)cudaGetLastError();
 }

@@ -47,8 +47,9 @@ struct faar_prof_scope {
 };
 
 // ---- workspace layout -------------------------------------------------------
-// [0, 256)            header: word 0 = status (0 = ok), word 1 = |W| max bits, word 2 = count of dW-GEMM
-//                     CTAs that have finished (zero between launches)
+// [0, 256)            header: word 0 = status (0 = ok), word 2 = count of dW-GEMM
+//                     CTAs that have finished (zero between launches), bytes 16..23 = tensor maximum of
+//                     the last set-up pass (high word: the pass's serial number, low word: max |W| bits)
 // [256, 256+P)        loss partials (float): MSE region then Round region
 // [..]                W_soft bf16 [O,K]
 // [..]                dYt bf16 [O, ceil8(T)]
@@ -83,13 +84,14 @@ static inline faar_ws_layout faar_ws_plan(const faar_shape* s) {
 // ---- launchers (each returns a cudaError_t as int) ---------------------------
 int faar_launch_softquant_init(faar_ctx*, const faar_shape*, const void* W, float s_global_in,
                                uint8_t* scales, float* s_global_out, uint8_t* code, float* V,
-                               uint32_t* amax_word);
+                               unsigned long long* amax_word);
 int faar_launch_softquant_eval(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta,
                                float* W_soft, float* h, __nv_bfloat16* W_soft_bf16,
                                float* W_operand_f32 = nullptr);
 int faar_launch_act_fakequant(faar_ctx*, int T, int K, const void* X, int64_t ldx, float s_global_in, void* Xq,
-                              int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales, uint32_t* amax_word);
+                              int64_t ldq, float* s_global_out, uint8_t* packed, uint8_t* scales,
+                              unsigned long long* amax_word);
 int faar_launch_transpose_bf16(faar_ctx*, int rows, int cols, const void* in, int64_t ld_in, void* out,
                                int64_t ld_out);
 int faar_launch_swizzle_scales(faar_ctx*, int rows, int cols, const uint8_t* in, uint8_t* out);
