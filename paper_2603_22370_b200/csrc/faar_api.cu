@@ -254,6 +254,7 @@ int faar_create(faar_ctx** out, int device, void* stream) {
   c->tune_bn = 0;
   c->tune_tail = -1;
   c->tune_attention_fragments = 0;
+  c->tune_wide = -1;
   c->last_gemm_split = 0;
   for (int i = 0; i < FAAR_GEMM_VARIANTS; ++i) c->gemm_max_pairs[i] = 0;
   c->wsoft_ws = nullptr;
@@ -370,6 +371,12 @@ int faar_tune_tail_split(faar_ctx* ctx, int columns) {
 int faar_last_tail_split(const faar_ctx* ctx, int* columns) {
   if (!ctx || !columns) return FAAR_ERR_INVALID_ARG;
   *columns = ctx->last_gemm_split;
+  return FAAR_OK;
+}
+
+int faar_tune_wide_tiles(faar_ctx* ctx, int mode) {
+  if (!ctx || mode < -1 || mode > 1) return FAAR_ERR_INVALID_ARG;
+  ctx->tune_wide = mode;
   return FAAR_OK;
 }
 

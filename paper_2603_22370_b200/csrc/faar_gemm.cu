@@ -41,11 +41,18 @@ constexpr int MAX_EPI_WARPS = 16;
 // The tile width bn (accumulator columns, a multiple of 16 up to 256) is a launch parameter chosen by
 // the host (pick_bn).  Shared memory and tensor memory are laid out for the widest tile.
 constexpr int BN_MAX = 256;
-template <int MODE> struct Cfg {
+// WIDE: the pair's tile is 256 x 512, the whole of tensor memory as ONE accumulator (two column halves of 256,
+// each fed by its own MMA from the same A stage).  A stage then holds this CTA's 128 rows of both B halves.
+// Per flop the tile pulls a quarter less operand data through the SM than a 256 x 256 tile, which is what
+// bounds these kernels; the price is that the epilogue of a tile no longer overlaps the next tile's main loop
+// (the two halves drain one after the other while the issuer waits).
+constexpr int WIDE_BN = 2 * BN_MAX;
+template <int MODE, bool WIDE = false> struct Cfg {
   static constexpr int EPI_WARPS = MODE == FAAR_GEMM_BWD ? 16 : 8;
   static constexpr int THREADS = 32 * (2 + EPI_WARPS);
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = (BN_MAX / 2) * BK * 2;        // this CTA's half of the B tile (slot size)
+  static constexpr int BH_BYTES = (BN_MAX / 2) * BK * 2;       // this CTA's 128 rows of one 256-column B tile
+  static constexpr int B_BYTES = WIDE ? 2 * BH_BYTES : BH_BYTES;   // slot size
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int EPI_BYTES = MODE == FAAR_GEMM_BWD ? 4 * PANEL_BYTES : 0;
   static constexpr int FIT = (SMEM_LIMIT - 1024 - CTL_BYTES - EPI_BYTES) / STAGE_BYTES;
@@ -552,11 +559,11 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
 
 // ---- the kernel ------------------------------------------------------------------------------
 // Launched as clusters of two CTAs along x: CTAs 2c and 2c+1 form pair c.
-template <int MODE, int OPT>
-__global__ void __launch_bounds__(Cfg<MODE>::THREADS, 1)
+template <int MODE, int OPT, bool WIDE>
+__global__ void __launch_bounds__(Cfg<MODE, WIDE>::THREADS, 1)
 faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmBh, const KParams p) {
-  using C = Cfg<MODE>;
+  using C = Cfg<MODE, WIDE>;
   const int BN = p.bn;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -578,7 +585,8 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const uint32_t rank = cluster_ctarank();             // 0 = leader of the pair
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int m_tiles = (p.M + 2 * BM - 1) / (2 * BM);
-  const int total_tiles = tile_count(p, m_tiles);
+  // WIDE: tiles of 512 columns, numbered row block fastest; no tail split
+  const int total_tiles = WIDE ? m_tiles * ((p.N + WIDE_BN - 1) / WIDE_BN) : tile_count(p, m_tiles);
   const int k_blocks = (p.Kc + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -606,8 +614,14 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const uint64_t keep = l2_policy_keep();
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
+      auto coords = [&](int tile) {
+        TileCoord tc;
+        if (WIDE) { tc.m0 = (tile % m_tiles) * (2 * BM); tc.n0 = (tile / m_tiles) * WIDE_BN; tc.w = BN_MAX; }
+        else tc = tile_coord(p, tile, m_tiles);
+        return tc;
+      };
       for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
-        const TileCoord tc = tile_coord(p, tile, m_tiles);
+        const TileCoord tc = coords(tile);
         const int m0 = tc.m0 + (int)rank * BM;
         const int n0 = tc.n0 + (int)rank * (tc.w / 2);
         const CUtensorMap* mapB = tc.w == BN ? &tmB : &tmBh;      // box of w/2 rows
@@ -616,10 +630,14 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (!ok) break;
           const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
           // the leader's barrier collects the bytes of both CTAs' copies
-          if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * (uint32_t)(C::A_BYTES + (tc.w / 2) * BK * 2));
+          if (rank == 0)
+            mbar_expect_tx(full_bar(stage), WIDE ? 2u * (uint32_t)(C::A_BYTES + C::B_BYTES)
+                                                 : 2u * (uint32_t)(C::A_BYTES + (tc.w / 2) * BK * 2));
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
           tma_load_2d(sa, &tmA, kb * BK, m0, leader_full, keep);
           tma_load_2d(sb, mapB, kb * BK, n0, leader_full, keep);
+          // second column half (rows beyond the matrix arrive as zeros)
+          if (WIDE) tma_load_2d(sb + C::BH_BYTES, &tmB, kb * BK, n0 + BN_MAX, leader_full, keep);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -636,13 +654,15 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int it = 0;
       bool ok = true;
       for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
-        const int acc = it & 1;
-        const uint32_t acc_phase = (it >> 1) & 1;
+        // WIDE: the two column halves take the place of the two accumulator buffers; both must be drained
+        const int acc = WIDE ? 0 : it & 1;
+        const uint32_t acc_phase = WIDE ? it & 1 : (it >> 1) & 1;
         ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, ac, 0x200u | acc);
+        if (ok && WIDE) ok = mbar_wait(tempty_bar(1), acc_phase ^ 1u, ac, 0x201u);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN_MAX;
-        const uint32_t idesc = make_idesc(tile_coord(p, tile, m_tiles).w);
+        const uint32_t idesc = make_idesc(WIDE ? BN_MAX : tile_coord(p, tile, m_tiles).w);
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(full_bar(stage), phase, ac, 0x300u | stage);
           if (!ok) break;
@@ -653,11 +673,17 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 bf16 = 32 bytes inside the swizzled row: +2 in the 16-byte address field
             tc_mma_bf16(tmem_d, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            if (WIDE)
+              tc_mma_bf16(tmem_d + BN_MAX, da + 2u * k, make_smem_desc(sb + C::BH_BYTES) + 2u * k, idesc,
+                          (kb | k) != 0 ? 1u : 0u);
           }
           tc_commit_pair(empty_bar(stage));            // frees this stage in both CTAs
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (ok) tc_commit_pair(tfull_bar(acc));        // accumulator ready in both CTAs
+        if (ok) {
+          tc_commit_pair(tfull_bar(acc));              // accumulator ready in both CTAs
+          if (WIDE) tc_commit_pair(tfull_bar(1));
+        }
       }
     }
   } else {
@@ -671,15 +697,20 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (MODE == FAAR_GEMM_BWD) s_global = *p.s_global;
     uint32_t pn = 0;                                   // panels this quarter has staged so far
     bool dead = false;
-    int it = 0;
-    for (int tile = pair; tile < total_tiles; tile += n_pairs, ++it) {
-      const int acc = it & 1;
-      const uint32_t acc_phase = (it >> 1) & 1;
+    // One pass per accumulator buffer that fills: a tile, or (WIDE) a 256-column half of a tile.
+    for (int vt = 0;; ++vt) {
+      const int it = WIDE ? vt >> 1 : vt;
+      const int tile = pair + it * n_pairs;
+      if (tile >= total_tiles) break;
+      const int acc = WIDE ? vt & 1 : it & 1;
+      const uint32_t acc_phase = WIDE ? it & 1 : (it >> 1) & 1;
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, ac, 0x400u | acc);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const TileCoord tc = tile_coord(p, tile, m_tiles);
+      TileCoord tc;
+      if (WIDE) { tc.m0 = (tile % m_tiles) * (2 * BM); tc.n0 = (tile / m_tiles) * WIDE_BN + acc * BN_MAX; tc.w = BN_MAX; }
+      else tc = tile_coord(p, tile, m_tiles);
       const int m0 = tc.m0 + (int)rank * BM, n0 = tc.n0, TW = tc.w;
       const int cols_per_warp = ((TW / C::COL_GROUPS + 15) / 16) * 16;
       const int col_begin = cg * cols_per_warp;
@@ -929,16 +960,62 @@ int pick_full_cols(const faar_ctx* ctx, int M, int N, int bn, int pairs) {
   return best_full;
 }
 
-template <int MODE, int OPT = 0>
-int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_out) {
-  using C = Cfg<MODE>;
+// Whether a launch takes 256 x 512 tiles (see Cfg).  Measured on a down_proj-shaped layer (2048 x 8192, 4096
+// tokens): the forward GEMM gains 4 % (64 tiles in one wave instead of 128 in two unequal ones), the dW GEMM
+// loses 29 % (its long epilogue is no longer hidden) and the plain product loses as well when it needs more
+// than one wave.  So the rule takes them for the forward GEMM only, where 256-wide tiles were chosen anyway,
+// the output cuts into 512-column tiles without a mostly empty last one, and those tiles fill one wave of the
+// CTA pairs to at least three quarters.  ctx->tune_wide: -1 = this rule, 0 = never, 1 = whenever the shape allows.
+bool pick_wide(const faar_ctx* ctx, int mode, int M, int N, int bn, int pairs) {
+  if (bn != BN_MAX || N <= BN_MAX || ctx->tune_wide == 0) return false;
+  if (ctx->tune_wide == 1) return true;
+  if (ctx->tune_tail >= 0 || mode != FAAR_GEMM_FWD) return false;    // a forced tail split asks for 256-wide tiles
+  const long long m_tiles = (M + 2 * BM - 1) / (2 * BM);
+  const long long tiles = m_tiles * ((N + WIDE_BN - 1) / WIDE_BN);
+  const int rest = N % WIDE_BN;
+  return (rest == 0 || rest > BN_MAX) && tiles <= pairs && 4 * tiles >= 3 * (long long)pairs;
+}
+
+template <int MODE, int OPT, bool WIDE>
+int launch_variant(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_out, int bn, int max_pairs,
+                   const cudaLaunchConfig_t& base_cfg) {
+  using C = Cfg<MODE, WIDE>;
   static_assert(C::STAGES >= 3, "ring too short");
   static_assert(C::SMEM_BYTES <= SMEM_LIMIT, "shared memory budget");
   static_assert(C::EPI_WARPS <= MAX_EPI_WARPS, "partials budget");
-  auto kern = faar_gemm_kernel<MODE, OPT>;
+  auto kern = faar_gemm_kernel<MODE, OPT, WIDE>;
   cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (ce != cudaSuccess) return (int)ce;
+  cudaLaunchConfig_t cfg = base_cfg;
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  kp.bn = bn;
+  kp.n_full_cols = WIDE ? 0 : pick_full_cols(ctx, a->M, a->N, bn, max_pairs);
+  CUtensorMap tmA, tmB, tmBh;
+  int e = make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
+  if (e) return e;
+  e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, bn / 2);
+  if (e) return e;
+  e = make_map(ctx, &tmBh, a->B, a->N, a->Kc, a->ldb, bn % 32 == 0 ? bn / 4 : bn / 2);   // half-width tiles
+  if (e) return e;
+  const long long m_tiles = (a->M + 2 * BM - 1) / (2 * BM);
+  const int rest_cols = a->N - kp.n_full_cols * bn;
+  const long long tiles = WIDE ? m_tiles * ((a->N + WIDE_BN - 1) / WIDE_BN)
+                               : m_tiles * (kp.n_full_cols + (rest_cols > 0 ? (rest_cols + bn / 2 - 1) / (bn / 2) : 0));
+  const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  if (n_partials_out) *n_partials_out = 2 * pairs * C::EPI_WARPS;
+  ctx->last_gemm_bn = WIDE ? WIDE_BN : bn;
+  ctx->last_gemm_pairs = pairs;
+  ctx->last_gemm_split = WIDE ? 0 : (a->N + bn - 1) / bn - kp.n_full_cols;
+  faar_prof_scope ps(ctx, MODE == FAAR_GEMM_REF ? FAAR_K_GEMM_REF : (MODE == FAAR_GEMM_FWD ? FAAR_K_GEMM_FWD : FAAR_K_GEMM_BWD));
+  ce = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmBh, kp);
+  if (ce != cudaSuccess) return (int)ce;
+  return (int)cudaGetLastError();
+}
 
+template <int MODE, int OPT = 0>
+int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_out) {
+  using C = Cfg<MODE>;
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -953,9 +1030,12 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   // how many CTA pairs the device can hold at once (a GPC with an odd SM count strands one SM); asked once
-  // per context and kernel instantiation, with the context's device current
+  // per context and kernel mode, with the context's device current (every variant takes one CTA per SM)
   int& max_pairs = ctx->gemm_max_pairs[MODE == FAAR_GEMM_BWD ? 2 + OPT : MODE];
   if (max_pairs == 0) {
+    auto kern = faar_gemm_kernel<MODE, OPT, false>;
+    cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
+    if (ce != cudaSuccess) return (int)ce;
     cfg.gridDim = dim3(2 * (ctx->num_sms / 2), 1, 1);
     int n = 0;
     ce = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
@@ -964,28 +1044,9 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
     max_pairs = n;
   }
   const int bn = pick_bn(ctx, MODE, a->M, a->N, max_pairs);
-  kp.bn = bn;
-  kp.n_full_cols = pick_full_cols(ctx, a->M, a->N, bn, max_pairs);
-  CUtensorMap tmA, tmB, tmBh;
-  int e = make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
-  if (e) return e;
-  e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, bn / 2);
-  if (e) return e;
-  e = make_map(ctx, &tmBh, a->B, a->N, a->Kc, a->ldb, bn % 32 == 0 ? bn / 4 : bn / 2);   // half-width tiles
-  if (e) return e;
-  const int rest_cols = a->N - kp.n_full_cols * bn;
-  const long long tiles = (long long)((a->M + 2 * BM - 1) / (2 * BM)) *
-                          (kp.n_full_cols + (rest_cols > 0 ? (rest_cols + bn / 2 - 1) / (bn / 2) : 0));
-  const int pairs = (int)(tiles < max_pairs ? tiles : max_pairs);
-  cfg.gridDim = dim3(2 * pairs, 1, 1);
-  if (n_partials_out) *n_partials_out = 2 * pairs * C::EPI_WARPS;
-  ctx->last_gemm_bn = bn;
-  ctx->last_gemm_pairs = pairs;
-  ctx->last_gemm_split = (a->N + bn - 1) / bn - kp.n_full_cols;
-  faar_prof_scope ps(ctx, MODE == FAAR_GEMM_REF ? FAAR_K_GEMM_REF : (MODE == FAAR_GEMM_FWD ? FAAR_K_GEMM_FWD : FAAR_K_GEMM_BWD));
-  ce = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmBh, kp);
-  if (ce != cudaSuccess) return (int)ce;
-  return (int)cudaGetLastError();
+  if (pick_wide(ctx, MODE, a->M, a->N, bn, max_pairs))
+    return launch_variant<MODE, OPT, true>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
+  return launch_variant<MODE, OPT, false>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
 }
 
 }  // namespace

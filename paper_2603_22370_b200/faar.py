@@ -63,6 +63,7 @@ SIGNATURES = {
     "faar_embedding": (_I, [_P, _I, _I, _I, _P, _L, _P, _P, _L]),
     "faar_add": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L]),
     "faar_tune_attention": (_I, [_P, _I]),
+    "faar_tune_wide_tiles": (_I, [_P, _I]),
     "faar_attention_fwd": (_I, [_P, _I, _I, _I, _I, _I, _P, _L, _P, _P, _L, _P, _L, _P]),
     "faar_attention_bwd": (_I, [_P, _I, _I, _I, _I, _I, _P, _L, _P, _P, _L, _P, _P, _L, _P, _P, _P, _P, _P]),
     "faar_nvfp4_gemm": (_I, [_P, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _L, _P, _Z]),
@@ -291,6 +292,11 @@ def embedding(ctx, rows, cols, vocab, table, ldt, tokens, out, ldo):
 
 def add(ctx, rows, cols, a, lda, b, ldb, out, ldo):
     _check(lib().faar_add(ctx._h, rows, cols, _p(a), lda, _p(b), ldb, _p(out), ldo), "faar_add")
+
+
+def tune_wide_tiles(ctx, mode: int):
+    """-1: 256 x 512 GEMM tiles where the library's rule picks them; 0: never; 1: whenever the shape allows."""
+    _check(lib().faar_tune_wide_tiles(ctx._h, mode), "faar_tune_wide_tiles")
 
 
 def tune_attention(ctx, mode: int):

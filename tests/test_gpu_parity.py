@@ -684,6 +684,46 @@ def test_half_width_tail_tiles_give_the_same_step(ctx, O, K, T, split):
     assert abs(out[0][5] - out[1][5]) <= 1e-5 * abs(out[0][5])
 
 
+@pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (520, 784, 1300), (256, 512, 1024)])
+def test_wide_tiles_give_the_same_step(ctx, O, K, T):
+    """256 x 512 tiles (one accumulator of two column halves, no overlap of epilogue and main loop) only
+    re-partition the output: forward residuals, gradient, updated state and the frozen target must equal the
+    256-wide launch bit for bit.  The shapes leave a last tile whose second half is partly or wholly outside
+    the matrix."""
+    W, X, Yref = _problem(O, K, T, seed=8)
+    hp, _ = f32hp(beta=6.0, step=2)
+    rng = np.random.default_rng(5)
+    V0 = rng.uniform(0, 1, W.shape).astype(np.float32)
+    m0 = (1e-3 * rng.standard_normal(W.shape)).astype(np.float32)
+    u0 = (1e-6 * rng.uniform(0, 1, W.shape)).astype(np.float32)
+    out = []
+    try:
+        faar.tune_tile_n(ctx, 256)
+        for wide in (0, 1):
+            faar.tune_wide_tiles(ctx, wide)
+            lay = GpuLayer(ctx, W, X)
+            lay.init()
+            yr = torch.empty((T, O), dtype=torch.bfloat16, device=DEV)
+            faar.layer_ref(ctx, lay.shape, lay.X, lay.W, yr, lay.ws)
+            assert faar.last_gemm_config(ctx)[0] == (512 if wide else 256)
+            lay.set_yref(Yref)
+            lay.set_state(V=V0, m=m0, u=u0)
+            lay.fwd(hp)
+            assert faar.last_gemm_config(ctx)[0] == (512 if wide else 256)
+            dYt = host(lay.dYt).copy()
+            dV = host(lay.bwd(hp, want_dv=True)).copy()
+            assert faar.last_gemm_config(ctx)[0] == (512 if wide else 256)
+            lay.check()
+            out.append((dYt, dV, host(lay.V).copy(), host(lay.m).copy(), host(lay.u).copy(), host(yr).copy(),
+                        host(lay.loss).copy()))
+    finally:
+        faar.tune_wide_tiles(ctx, -1)
+        faar.tune_tile_n(ctx, 0)
+    for a, b in zip(out[0][:6], out[1][:6]):
+        assert np.array_equal(a, b)
+    assert np.all(np.abs(out[0][6] - out[1][6]) <= 1e-5 * np.abs(out[0][6]))
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives(ctx):
     """The tensor-core kernels bound every barrier wait.  The self-test kernel waits (1 ms limit) on a
     barrier that nothing arrives at: it must exit by itself and leave its code in the status word of the
