@@ -524,61 +524,110 @@ __device__ __forceinline__ void store_16x64(__nv_bfloat16* base, long long ld, l
   }
 }
 
-// ---- forward, head_dim 64: grid (query tiles, H, B); warp w owns queries 16 w .. 16 w + 15 ------------------
-__global__ void __launch_bounds__(ATT_THREADS)
+// ---- asynchronous tile copies (cp.async, 16 bytes each; rows at or beyond row_end arrive as zeros) ------------
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
+  const int n = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// ROWS x 64 BF16 tile of `src` (rows row0 .., columns col0 ..) into tile[ROWS][LDS], by NT threads
+template <int ROWS, int NT>
+__device__ __forceinline__ void tile_async(__nv_bfloat16 (*tile)[LDS], const __nv_bfloat16* src, long long ld, long long row0,
+                                           long long row_end, int col0) {
+  for (int i = threadIdx.x; i < ROWS * (HD / 8); i += NT) {
+    const int r = i >> 3, c = (i & 7) * 8;
+    const bool valid = row0 + r < row_end;
+    cp_async16(&tile[r][c], src + (valid ? row0 + r : row0) * ld + col0 + c, valid);
+  }
+}
+
+// ---- forward, head_dim 64: grid (128-query tiles, H, B); 8 warps, warp w owns queries 16 w .. 16 w + 15 ----------
+// Key / value tiles of 64 keys run through a three-stage cp.async ring (the copy of tile t + 2 is issued before
+// the products of tile t), one block-wide barrier per tile.  The query tile first sits in the ring's third
+// stage; once every warp holds its query fragments the stage joins the ring.  A warp skips key tiles that lie
+// wholly above its rows' diagonal and masks only where a tile crosses it (or the sequence end).
+constexpr int FQ = 128;
+constexpr int FWD_THREADS = 256;
+constexpr int STAGE_ELEMS = 2 * AT * LDS;            // a K tile and a V tile; equals one 128-row query tile
+constexpr int FWD64_SMEM = 3 * STAGE_ELEMS * 2;
+__global__ void __launch_bounds__(FWD_THREADS, 2)
 attn_fwd64_kernel(const AttnParams p) {
-  __shared__ __align__(128) __nv_bfloat16 Qs[AT][LDS];
-  __shared__ __align__(128) __nv_bfloat16 Ks[AT][LDS];
-  __shared__ __align__(128) __nv_bfloat16 Vs[AT][LDS];
+  extern __shared__ __align__(128) uint8_t att_smem[];
+  auto stage_k = [&](int s) { return reinterpret_cast<__nv_bfloat16(*)[LDS]>(att_smem) + (size_t)s * 2 * AT; };
+  auto stage_v = [&](int s) { return stage_k(s) + AT; };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;      // longest tiles first
   const int h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.H / p.Hkv);
   const long long seq0 = (long long)b * p.S;
-  const int q0 = qt * AT;
-  load_tile<HD>(Qs, p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
+  const int q0 = qt * FQ;
+  const int last_q = min(q0 + FQ, p.S) - 1;
+  const int n_kt = last_q / AT + 1;                          // key tiles that some query of this tile sees
+  auto load_kv = [&](int kt) {
+    if (kt < n_kt) {
+      tile_async<AT, FWD_THREADS>(stage_k(kt % 3), p.k, p.ldk, seq0 + kt * AT, seq0 + p.S, g * HD);
+      tile_async<AT, FWD_THREADS>(stage_v(kt % 3), p.v, p.ldk, seq0 + kt * AT, seq0 + p.S, g * HD);
+    }
+    cp_async_commit();
+  };
+  auto Qs = stage_k(2);                                      // 128 rows
+  tile_async<FQ, FWD_THREADS>(Qs, p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
+  cp_async_commit();
+  load_kv(0);
+  load_kv(1);
+  cp_async_wait<2>();                                        // the query tile has landed
   __syncthreads();
   uint32_t qf[HD / 16][4];
 #pragma unroll
   for (int kk = 0; kk < HD / 16; ++kk) load_a(qf[kk], Qs, 16 * warp, kk, lane);
-  const int qi0 = q0 + 16 * warp + (lane >> 2), qi1 = qi0 + 8;          // this lane's two query rows
+  const int r_first = q0 + 16 * warp;                        // this warp's first query
+  const int qi0 = r_first + (lane >> 2), qi1 = qi0 + 8;      // this lane's two query rows
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
   float o[8][4];
 #pragma unroll
   for (int n = 0; n < 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
 
-  for (int kt = 0; kt <= qt; ++kt) {
+  for (int kt = 0; kt < n_kt; ++kt) {
     const int k0 = kt * AT;
-    __syncthreads();
-    load_tile<HD>(Ks, p.k, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
-    load_tile<HD>(Vs, p.v, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
-    __syncthreads();
+    cp_async_wait<1>();                                      // tile kt has landed (tile kt + 1 may be in flight)
+    __syncthreads();                                         // ... for every thread; stage (kt + 2) % 3 is free
+    load_kv(kt + 2);
+    if (k0 > r_first + 15) continue;                         // wholly masked for this warp
+    const __nv_bfloat16(*Ks)[LDS] = stage_k(kt % 3);
+    const __nv_bfloat16(*Vs)[LDS] = stage_v(kt % 3);
     float s[8][4];
     scores_16x64(s, qf, Ks, lane);
-    // scale to log2 units, causal mask, row maxima
+    if (k0 + AT - 1 > r_first || k0 + AT > p.S) {            // the tile crosses the diagonal or the sequence end
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int kj = k0 + 8 * n + 2 * (lane & 3) + j;
+          if (!(kj <= qi0 && kj < p.S)) s[n][j] = -INFINITY;
+          if (!(kj <= qi1 && kj < p.S)) s[n][2 + j] = -INFINITY;
+        }
+      }
+    }
     float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const int kj = k0 + 8 * n + 2 * (lane & 3) + j;
-        s[n][j] = (kj <= qi0 && kj < p.S) ? s[n][j] * p.scale_log2 : -INFINITY;
-        s[n][2 + j] = (kj <= qi1 && kj < p.S) ? s[n][2 + j] * p.scale_log2 : -INFINITY;
-        mx0 = fmaxf(mx0, s[n][j]);
-        mx1 = fmaxf(mx1, s[n][2 + j]);
-      }
+      mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
+      mx1 = fmaxf(mx1, fmaxf(s[n][2], s[n][3]));
     }
     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+    // running maxima in log2 units (the raw scores times scale_log2, a positive factor)
+    const float mn0 = fmaxf(m0, mx0 * p.scale_log2), mn1 = fmaxf(m1, mx1 * p.scale_log2);
     // a row that has seen no key yet keeps maximum -inf: use 0 as the reference so that nothing is NaN
     const float ref0 = mn0 == -INFINITY ? 0.f : mn0, ref1 = mn1 == -INFINITY ? 0.f : mn1;
     const float a0 = exp2f(m0 - ref0), a1 = exp2f(m1 - ref1);            // exp2f(-inf) = 0
     float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
-      s[n][0] = exp2f(s[n][0] - ref0); s[n][1] = exp2f(s[n][1] - ref0);
-      s[n][2] = exp2f(s[n][2] - ref1); s[n][3] = exp2f(s[n][3] - ref1);
+      s[n][0] = exp2f(fmaf(s[n][0], p.scale_log2, -ref0)); s[n][1] = exp2f(fmaf(s[n][1], p.scale_log2, -ref0));
+      s[n][2] = exp2f(fmaf(s[n][2], p.scale_log2, -ref1)); s[n][3] = exp2f(fmaf(s[n][3], p.scale_log2, -ref1));
       sum0 += s[n][0] + s[n][1];
       sum1 += s[n][2] + s[n][3];
       o[n][0] *= a0; o[n][1] *= a0; o[n][2] *= a1; o[n][3] *= a1;
@@ -591,8 +640,9 @@ attn_fwd64_kernel(const AttnParams p) {
     to_a_frags(pf, s);
     accumulate_16x64(o, pf, Vs, lane);
   }
+  cp_async_wait<0>();
   const float i0 = l0 > 0.f ? 1.0f / l0 : 0.f, i1 = l1 > 0.f ? 1.0f / l1 : 0.f;
-  store_16x64(p.out, p.ldo, seq0 + q0 + 16 * warp, seq0 + p.S, h * HD, o, i0, i1, lane);
+  store_16x64(p.out, p.ldo, seq0 + r_first, seq0 + p.S, h * HD, o, i0, i1, lane);
   if ((lane & 3) == 0) {
     float* lse = p.lse + ((long long)b * p.H + h) * p.S;
     if (qi0 < p.S) lse[qi0] = m0 + log2f(l0);
@@ -733,9 +783,13 @@ int launch_fwd(faar_ctx* ctx, const AttnParams& p) {
   cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, fwd_smem<D>());
   if (e != cudaSuccess) return (int)e;
   dim3 grid((p.S + AT - 1) / AT, p.H, p.B);
+  if (D == HD && !ctx->tune_attention_fragments) {
+    e = cudaFuncSetAttribute(attn_fwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD64_SMEM);
+    if (e != cudaSuccess) return (int)e;
+  }
   faar_prof_scope ps(ctx, FAAR_K_ATTENTION);
   if (D == HD && !ctx->tune_attention_fragments)
-    attn_fwd64_kernel<<<grid, ATT_THREADS, 0, ctx->stream>>>(p);
+    attn_fwd64_kernel<<<dim3((p.S + FQ - 1) / FQ, p.H, p.B), FWD_THREADS, FWD64_SMEM, ctx->stream>>>(p);
   else
     attn_fwd_kernel<D><<<grid, ATT_THREADS, fwd_smem<D>(), ctx->stream>>>(p);
   return (int)cudaGetLastError();
