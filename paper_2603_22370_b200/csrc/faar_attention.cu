@@ -651,125 +651,168 @@ attn_fwd64_kernel(const AttnParams p) {
 }
 
 // ---- backward, head_dim 64, dQ: grid (query tiles, H, B); warp w owns queries 16 w .. 16 w + 15 ------------------
-__global__ void __launch_bounds__(ATT_THREADS)
+// Same ring as the forward kernel: the query and dO tiles sit in the third stage until their fragments are in
+// registers.  Only the last key tile crosses the diagonal.  Keys beyond the sequence end need no mask of
+// their own: their K rows are zero, so whatever dS they get adds nothing to dQ.
+constexpr int BWD_THREADS = 128;
+constexpr int BWD64_SMEM = 3 * STAGE_ELEMS * 2 + 3 * 2 * AT * 4;      // three stages + their lse / dsum rows (dK, dV kernel)
+__global__ void __launch_bounds__(BWD_THREADS, 3)
 attn_dq64_kernel(const AttnParams p) {
-  __shared__ __align__(128) __nv_bfloat16 Qs[AT][LDS];
-  __shared__ __align__(128) __nv_bfloat16 Ds[AT][LDS];
-  __shared__ __align__(128) __nv_bfloat16 Ks[AT][LDS];
-  __shared__ __align__(128) __nv_bfloat16 Vs[AT][LDS];
+  extern __shared__ __align__(128) uint8_t att_smem[];
+  auto stage_k = [&](int s) { return reinterpret_cast<__nv_bfloat16(*)[LDS]>(att_smem) + (size_t)s * 2 * AT; };
+  auto stage_v = [&](int s) { return stage_k(s) + AT; };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
   const int h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.H / p.Hkv);
   const long long seq0 = (long long)b * p.S;
   const int q0 = qt * AT;
-  load_tile<HD>(Qs, p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
-  load_tile<HD>(Ds, p.dout, p.ldo, seq0 + q0, seq0 + p.S, h * HD);
+  const int n_kt = qt + 1;
+  auto load_kv = [&](int kt) {
+    if (kt < n_kt) {
+      tile_async<AT, BWD_THREADS>(stage_k(kt % 3), p.k, p.ldk, seq0 + kt * AT, seq0 + p.S, g * HD);
+      tile_async<AT, BWD_THREADS>(stage_v(kt % 3), p.v, p.ldk, seq0 + kt * AT, seq0 + p.S, g * HD);
+    }
+    cp_async_commit();
+  };
+  tile_async<AT, BWD_THREADS>(stage_k(2), p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
+  tile_async<AT, BWD_THREADS>(stage_v(2), p.dout, p.ldo, seq0 + q0, seq0 + p.S, h * HD);
+  cp_async_commit();
+  load_kv(0);
+  load_kv(1);
+  cp_async_wait<2>();
   __syncthreads();
   uint32_t qf[HD / 16][4], df[HD / 16][4];
 #pragma unroll
-  for (int kk = 0; kk < HD / 16; ++kk) { load_a(qf[kk], Qs, 16 * warp, kk, lane); load_a(df[kk], Ds, 16 * warp, kk, lane); }
+  for (int kk = 0; kk < HD / 16; ++kk) { load_a(qf[kk], stage_k(2), 16 * warp, kk, lane); load_a(df[kk], stage_v(2), 16 * warp, kk, lane); }
   const int qi0 = q0 + 16 * warp + (lane >> 2), qi1 = qi0 + 8;
   const long long ro = ((long long)b * p.H + h) * p.S;
   const float lse0 = qi0 < p.S ? p.lse[ro + qi0] : 0.f, lse1 = qi1 < p.S ? p.lse[ro + qi1] : 0.f;
-  const float dsm0 = qi0 < p.S ? p.dsum[ro + qi0] : 0.f, dsm1 = qi1 < p.S ? p.dsum[ro + qi1] : 0.f;
   const float inv_sqrt_d = p.scale_log2 / LOG2E;
+  // dS = P (dP - dsum) / sqrt(d): the subtrahend and the factor are folded into one FMA per element
+  const float nd0 = qi0 < p.S ? -p.dsum[ro + qi0] * inv_sqrt_d : 0.f, nd1 = qi1 < p.S ? -p.dsum[ro + qi1] * inv_sqrt_d : 0.f;
   float dq[8][4];
 #pragma unroll
   for (int n = 0; n < 8; ++n) { dq[n][0] = dq[n][1] = dq[n][2] = dq[n][3] = 0.f; }
 
-  for (int kt = 0; kt <= qt; ++kt) {
+  for (int kt = 0; kt < n_kt; ++kt) {
     const int k0 = kt * AT;
+    cp_async_wait<1>();
     __syncthreads();
-    load_tile<HD>(Ks, p.k, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
-    load_tile<HD>(Vs, p.v, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
-    __syncthreads();
+    load_kv(kt + 2);
+    const __nv_bfloat16(*Ks)[LDS] = stage_k(kt % 3);
+    const __nv_bfloat16(*Vs)[LDS] = stage_v(kt % 3);
     float s[8][4], dp[8][4];
     scores_16x64(s, qf, Ks, lane);
     scores_16x64(dp, df, Vs, lane);
+    const bool diag = kt == qt;
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         const int kj = k0 + 8 * n + 2 * (lane & 3) + j;
-        const float p0 = (kj <= qi0 && qi0 < p.S) ? exp2f(s[n][j] * p.scale_log2 - lse0) : 0.f;
-        const float p1 = (kj <= qi1 && qi1 < p.S) ? exp2f(s[n][2 + j] * p.scale_log2 - lse1) : 0.f;
-        s[n][j] = p0 * (dp[n][j] - dsm0) * inv_sqrt_d;              // dS
-        s[n][2 + j] = p1 * (dp[n][2 + j] - dsm1) * inv_sqrt_d;
+        float p0 = exp2f(fmaf(s[n][j], p.scale_log2, -lse0));
+        float p1 = exp2f(fmaf(s[n][2 + j], p.scale_log2, -lse1));
+        if (diag) { if (kj > qi0) p0 = 0.f; if (kj > qi1) p1 = 0.f; }
+        s[n][j] = p0 * fmaf(dp[n][j], inv_sqrt_d, nd0);             // dS
+        s[n][2 + j] = p1 * fmaf(dp[n][2 + j], inv_sqrt_d, nd1);
       }
     }
     uint32_t sf[4][4];
     to_a_frags(sf, s);
     accumulate_16x64(dq, sf, Ks, lane);                             // dQ += dS K
   }
+  cp_async_wait<0>();
   store_16x64(p.dq, p.ldq, seq0 + q0 + 16 * warp, seq0 + p.S, h * HD, dq, 1.f, 1.f, lane);
 }
 
 // ---- backward, head_dim 64, dK and dV: grid (key tiles, Hkv, B); warp w owns keys 16 w .. 16 w + 15 ---------------
 // The products are formed transposed (keys on the accumulator rows): S^T = K Q^T, dP^T = V dO^T; then
-// dV += P^T dO and dK += dS^T Q contract over the 64 queries of the tile.
-__global__ void __launch_bounds__(ATT_THREADS)
+// dV += P^T dO and dK += dS^T Q contract over the 64 queries of a tile.  The (head, query tile) pairs that see
+// this key tile form one sequence that runs through the ring (a Q tile, a dO tile and the 64 lse / dsum values per
+// stage).  Only the first query tile of a head crosses the diagonal.  Queries beyond the sequence end need no
+// mask: their Q and dO rows are zero, so whatever P and dS they get adds nothing to dV or dK.
+__global__ void __launch_bounds__(BWD_THREADS, 2)
 attn_dkv64_kernel(const AttnParams p) {
-  __shared__ __align__(128) __nv_bfloat16 Ks[AT][LDS];
-  __shared__ __align__(128) __nv_bfloat16 Vs[AT][LDS];
-  __shared__ __align__(128) __nv_bfloat16 Qs[AT][LDS];
-  __shared__ __align__(128) __nv_bfloat16 Ds[AT][LDS];
-  __shared__ __align__(16) float rowv[2 * AT];                     // lse and dsum of the tile's 64 queries
+  extern __shared__ __align__(128) uint8_t att_smem[];
+  auto stage_q = [&](int s) { return reinterpret_cast<__nv_bfloat16(*)[LDS]>(att_smem) + (size_t)s * 2 * AT; };
+  auto stage_d = [&](int s) { return stage_q(s) + AT; };
+  float* rows_all = reinterpret_cast<float*>(att_smem + 3 * STAGE_ELEMS * 2);        // [3][2][AT]: lse, dsum
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kt = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int kt = blockIdx.x;                               // the first key tiles see the most queries: they start first
+  const int g = blockIdx.y, b = blockIdx.z;
   const int rep = p.H / p.Hkv;
   const long long seq0 = (long long)b * p.S;
   const int k0 = kt * AT;
   const int n_qt = (p.S + AT - 1) / AT;
-  load_tile<HD>(Ks, p.k, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
-  load_tile<HD>(Vs, p.v, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+  const int per_head = n_qt - kt;
+  const int n_it = rep * per_head;
+  auto load_qd = [&](int it) {
+    if (it < n_it) {
+      const int h = g * rep + it / per_head, q0 = (kt + it % per_head) * AT;
+      tile_async<AT, BWD_THREADS>(stage_q(it % 3), p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
+      tile_async<AT, BWD_THREADS>(stage_d(it % 3), p.dout, p.ldo, seq0 + q0, seq0 + p.S, h * HD);
+      const long long ro = ((long long)b * p.H + h) * p.S;
+      const int c = threadIdx.x & (AT - 1);
+      const float* src = threadIdx.x < AT ? p.lse : p.dsum;
+      const bool valid = q0 + c < p.S;
+      const uint32_t d = (uint32_t)__cvta_generic_to_shared(rows_all + (it % 3) * 2 * AT + threadIdx.x);
+      const int nb = valid ? 4 : 0;
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(d), "l"(src + ro + (valid ? q0 + c : 0)), "r"(nb) : "memory");
+    }
+    cp_async_commit();
+  };
+  tile_async<AT, BWD_THREADS>(stage_q(2), p.k, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+  tile_async<AT, BWD_THREADS>(stage_d(2), p.v, p.ldk, seq0 + k0, seq0 + p.S, g * HD);
+  cp_async_commit();
+  load_qd(0);
+  load_qd(1);
+  cp_async_wait<2>();
   __syncthreads();
   uint32_t kf[HD / 16][4], vf[HD / 16][4];
 #pragma unroll
-  for (int kk = 0; kk < HD / 16; ++kk) { load_a(kf[kk], Ks, 16 * warp, kk, lane); load_a(vf[kk], Vs, 16 * warp, kk, lane); }
+  for (int kk = 0; kk < HD / 16; ++kk) { load_a(kf[kk], stage_q(2), 16 * warp, kk, lane); load_a(vf[kk], stage_d(2), 16 * warp, kk, lane); }
   const int kj0 = k0 + 16 * warp + (lane >> 2), kj1 = kj0 + 8;          // this lane's two key rows
   const float inv_sqrt_d = p.scale_log2 / LOG2E;
   float dk[8][4], dv[8][4];
 #pragma unroll
   for (int n = 0; n < 8; ++n) { dk[n][0] = dk[n][1] = dk[n][2] = dk[n][3] = 0.f; dv[n][0] = dv[n][1] = dv[n][2] = dv[n][3] = 0.f; }
 
-  for (int hh = 0; hh < rep; ++hh) {
-    const int h = g * rep + hh;
-    const long long ro = ((long long)b * p.H + h) * p.S;
-    for (int qt = kt; qt < n_qt; ++qt) {
-      const int q0 = qt * AT;
-      __syncthreads();
-      load_tile<HD>(Qs, p.q, p.ldq, seq0 + q0, seq0 + p.S, h * HD);
-      load_tile<HD>(Ds, p.dout, p.ldo, seq0 + q0, seq0 + p.S, h * HD);
-      if (threadIdx.x < AT) {
-        const int qi = q0 + threadIdx.x;
-        rowv[threadIdx.x] = qi < p.S ? p.lse[ro + qi] : 0.f;
-        rowv[AT + threadIdx.x] = qi < p.S ? p.dsum[ro + qi] : 0.f;
-      }
-      __syncthreads();
-      float st[8][4], dpt[8][4];
-      scores_16x64(st, kf, Qs, lane);                               // S^T[key][query]
-      scores_16x64(dpt, vf, Ds, lane);                              // dP^T[key][query]
-      uint32_t pf[4][4];
+  for (int it = 0; it < n_it; ++it) {
+    cp_async_wait<1>();
+    __syncthreads();
+    load_qd(it + 2);
+    const __nv_bfloat16(*Qs)[LDS] = stage_q(it % 3);
+    const __nv_bfloat16(*Ds)[LDS] = stage_d(it % 3);
+    const float* rowv = rows_all + (it % 3) * 2 * AT;
+    const int q0 = (kt + it % per_head) * AT;
+    const bool diag = it % per_head == 0;
+    float st[8][4], dpt[8][4];
+    scores_16x64(st, kf, Qs, lane);                               // S^T[key][query]
+    scores_16x64(dpt, vf, Ds, lane);                              // dP^T[key][query]
+    uint32_t pf[4][4];
 #pragma unroll
-      for (int n = 0; n < 8; ++n) {
+    for (int n = 0; n < 8; ++n) {
+      const int c = 8 * n + 2 * (lane & 3);
+      const float2 lse2 = *reinterpret_cast<const float2*>(rowv + c), dsm2 = *reinterpret_cast<const float2*>(rowv + AT + c);
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const int c = 8 * n + 2 * (lane & 3) + j, qi = q0 + c;
-          const float lse = rowv[c], dsm = rowv[AT + c];
-          const float p0 = (kj0 <= qi && qi < p.S) ? exp2f(st[n][j] * p.scale_log2 - lse) : 0.f;
-          const float p1 = (kj1 <= qi && qi < p.S) ? exp2f(st[n][2 + j] * p.scale_log2 - lse) : 0.f;
-          st[n][j] = p0; st[n][2 + j] = p1;
-          dpt[n][j] = p0 * (dpt[n][j] - dsm) * inv_sqrt_d;          // dS^T
-          dpt[n][2 + j] = p1 * (dpt[n][2 + j] - dsm) * inv_sqrt_d;
-        }
+      for (int j = 0; j < 2; ++j) {
+        const int qi = q0 + c + j;
+        const float lse = j ? lse2.y : lse2.x, nd = -(j ? dsm2.y : dsm2.x) * inv_sqrt_d;
+        float p0 = exp2f(fmaf(st[n][j], p.scale_log2, -lse));
+        float p1 = exp2f(fmaf(st[n][2 + j], p.scale_log2, -lse));
+        if (diag) { if (kj0 > qi) p0 = 0.f; if (kj1 > qi) p1 = 0.f; }
+        st[n][j] = p0; st[n][2 + j] = p1;
+        dpt[n][j] = p0 * fmaf(dpt[n][j], inv_sqrt_d, nd);          // dS^T
+        dpt[n][2 + j] = p1 * fmaf(dpt[n][2 + j], inv_sqrt_d, nd);
       }
-      to_a_frags(pf, st);
-      accumulate_16x64(dv, pf, Ds, lane);                           // dV += P^T dO
-      to_a_frags(pf, dpt);
-      accumulate_16x64(dk, pf, Qs, lane);                           // dK += dS^T Q
     }
+    to_a_frags(pf, st);
+    accumulate_16x64(dv, pf, Ds, lane);                           // dV += P^T dO
+    to_a_frags(pf, dpt);
+    accumulate_16x64(dk, pf, Qs, lane);                           // dK += dS^T Q
   }
+  cp_async_wait<0>();
   store_16x64(p.dv, p.ldk, seq0 + k0 + 16 * warp, seq0 + p.S, g * HD, dv, 1.f, 1.f, lane);
   store_16x64(p.dk, p.ldk, seq0 + k0 + 16 * warp, seq0 + p.S, g * HD, dk, 1.f, 1.f, lane);
 }
@@ -799,6 +842,8 @@ template <int D>
 int launch_bwd(faar_ctx* ctx, const AttnParams& p, float* dsum) {
   cudaError_t e = cudaFuncSetAttribute(attn_dkv_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, dkv_smem<D>());
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, dq_smem<D>());
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_dkv64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD64_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_dq64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD64_SMEM);
   if (e != cudaSuccess) return (int)e;
   faar_prof_scope ps(ctx, FAAR_K_ATTENTION);
   long long rows = (long long)p.B * p.S * p.H;
@@ -807,8 +852,8 @@ int launch_bwd(faar_ctx* ctx, const AttnParams& p, float* dsum) {
   attn_dsum_kernel<D><<<(int)blocks, ATT_THREADS, 0, ctx->stream>>>(p, dsum);
   const int tiles = (p.S + AT - 1) / AT;
   if (D == HD && !ctx->tune_attention_fragments) {
-    attn_dkv64_kernel<<<dim3(tiles, p.Hkv, p.B), ATT_THREADS, 0, ctx->stream>>>(p);
-    attn_dq64_kernel<<<dim3(tiles, p.H, p.B), ATT_THREADS, 0, ctx->stream>>>(p);
+    attn_dkv64_kernel<<<dim3(tiles, p.Hkv, p.B), BWD_THREADS, BWD64_SMEM, ctx->stream>>>(p);
+    attn_dq64_kernel<<<dim3(tiles, p.H, p.B), BWD_THREADS, BWD64_SMEM, ctx->stream>>>(p);
     return (int)cudaGetLastError();
   }
   attn_dkv_kernel<D><<<dim3(tiles, p.Hkv, p.B), ATT_THREADS, dkv_smem<D>(), ctx->stream>>>(p);
