@@ -150,12 +150,12 @@ FAAR_API int faar_tune_tile_n(faar_ctx* ctx, int bn);
 FAAR_API int faar_tune_tail_split(faar_ctx* ctx, int columns);
 FAAR_API int faar_last_tail_split(const faar_ctx* ctx, int* columns);
 FAAR_API int faar_last_gemm_config(const faar_ctx* ctx, int* bn, int* cta_pairs);
-/* Where the output is wide enough, a launch may instead take 256 x 512 tiles: the pair's whole tensor memory
- * as one accumulator, a quarter less operand traffic per flop, no overlap of a tile's epilogue with the next
- * tile's main loop, no tail split.  mode: -1 = decided per launch (default: the forward GEMM takes them when
- * they fill one wave of the CTA pairs to at least three quarters), 0 = never, 1 = whenever the
- * output has more than 256 columns and 256-wide tiles would have been used.  faar_last_gemm_config reports
- * bn = 512 for such a launch.  The per-weight results (dW, V, moments) do not depend on the tile shape. */
+/* On request a launch takes 256 x 512 tiles: the pair's whole tensor memory as one accumulator, a quarter less
+ * operand traffic per flop, no overlap of a tile's epilogue with the next tile's main loop, no tail split.
+ * mode: 1 = whenever the output has more than 256 columns and 256-wide tiles would have been used; 0 and -1
+ * (the default) = never: measured, they win by a few per cent only for the forward GEMM of a large layer in a
+ * short job and lose elsewhere.  faar_last_gemm_config reports bn = 512 for such a launch.  The per-weight
+ * results (dW, V, moments) do not depend on the tile shape. */
 FAAR_API int faar_tune_wide_tiles(faar_ctx* ctx, int mode);
 
 /* Bytes of workspace that any call on this shape needs (host out-pointer).

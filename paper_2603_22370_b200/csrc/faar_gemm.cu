@@ -960,20 +960,14 @@ int pick_full_cols(const faar_ctx* ctx, int M, int N, int bn, int pairs) {
   return best_full;
 }
 
-// Whether a launch takes 256 x 512 tiles (see Cfg).  Measured on a down_proj-shaped layer (2048 x 8192, 4096
-// tokens): the forward GEMM gains 4 % (64 tiles in one wave instead of 128 in two unequal ones), the dW GEMM
-// loses 29 % (its long epilogue is no longer hidden) and the plain product loses as well when it needs more
-// than one wave.  So the rule takes them for the forward GEMM only, where 256-wide tiles were chosen anyway,
-// the output cuts into 512-column tiles without a mostly empty last one, and those tiles fill one wave of the
-// CTA pairs to at least three quarters.  ctx->tune_wide: -1 = this rule, 0 = never, 1 = whenever the shape allows.
-bool pick_wide(const faar_ctx* ctx, int mode, int M, int N, int bn, int pairs) {
-  if (bn != BN_MAX || N <= BN_MAX || ctx->tune_wide == 0) return false;
-  if (ctx->tune_wide == 1) return true;
-  if (ctx->tune_tail >= 0 || mode != FAAR_GEMM_FWD) return false;    // a forced tail split asks for 256-wide tiles
-  const long long m_tiles = (M + 2 * BM - 1) / (2 * BM);
-  const long long tiles = m_tiles * ((N + WIDE_BN - 1) / WIDE_BN);
-  const int rest = N % WIDE_BN;
-  return (rest == 0 || rest > BN_MAX) && tiles <= pairs && 4 * tiles >= 3 * (long long)pairs;
+// Whether a launch takes 256 x 512 tiles (see Cfg): only on request (ctx->tune_wide == 1) and where the shape
+// allows.  Measured: on a down_proj-shaped layer (2048 x 8192, 4096 tokens) in a short job at full clocks the
+// forward GEMM gains 1-4 % (64 tiles in one wave instead of 128 in two unequal ones), but in the long,
+// power-capped jobs of whole decoder blocks the same launch and the q / o projections lose 6-10 %; the dW GEMM
+// loses 29 % (its long epilogue is no longer hidden) and the plain product loses whenever it needs more than
+// one wave.  No rule was found that wins consistently, so the default never takes them.
+bool pick_wide(const faar_ctx* ctx, int N, int bn) {
+  return ctx->tune_wide == 1 && bn == BN_MAX && N > BN_MAX;
 }
 
 template <int MODE, int OPT, bool WIDE>
@@ -1044,7 +1038,7 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
     max_pairs = n;
   }
   const int bn = pick_bn(ctx, MODE, a->M, a->N, max_pairs);
-  if (pick_wide(ctx, MODE, a->M, a->N, bn, max_pairs))
+  if (pick_wide(ctx, a->N, bn))
     return launch_variant<MODE, OPT, true>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
   return launch_variant<MODE, OPT, false>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
 }

@@ -19,7 +19,7 @@ struct faar_ctx {
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime
   int tune_bn;                            // 0 = choose the GEMM tile width automatically
   int tune_tail;                          // -1 = choose the tail split automatically, else columns to split
-  int tune_wide;                          // -1 = choose 256 x 512 GEMM tiles automatically, 0 = never, 1 = whenever possible
+  int tune_wide;                          // 1 = 256 x 512 GEMM tiles wherever the shape allows; -1 (default), 0 = never
   int tune_attention_fragments;           // 1 = head_dim 64 attention also runs the shared-memory fragment kernels
   int last_gemm_bn, last_gemm_pairs, last_gemm_split;   // what the last GEMM launch used
   // CTA pairs this context's device can hold at once, per GEMM kernel instantiation (0 = not asked yet)

@@ -295,7 +295,7 @@ def add(ctx, rows, cols, a, lda, b, ldb, out, ldo):
 
 
 def tune_wide_tiles(ctx, mode: int):
-    """-1: 256 x 512 GEMM tiles where the library's rule picks them; 0: never; 1: whenever the shape allows."""
+    """1: 256 x 512 GEMM tiles whenever the shape allows; 0 or -1 (the default): never."""
     _check(lib().faar_tune_wide_tiles(ctx._h, mode), "faar_tune_wide_tiles")
 
 
