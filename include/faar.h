@@ -291,9 +291,10 @@ FAAR_API int faar_layer_fwd(faar_ctx* ctx, const faar_shape* shape, const faar_h
  * Procedure steps 16-23 train the rounding variables of all layers through the
  * whole model; a layer must then also pass the gradient on to its input:
  * dX = dY W_soft (the derivative of Y_q = X W_soft^T, W_soft as in faar_layer_fwd).
- * Soft weights, a transpose into the caller's scratch and one tensor-core GEMM.
+ * Soft weights (into the workspace) and one tensor-core GEMM that reads them untransposed, with the
+ * output-feature index as the contraction row.
  *   dY     in : [T,O] bf16 (ldy, multiple of 8)      dX out: [T,K] bf16 (ldx, multiple of 8)
- *   WsoftT scratch: [K, O rounded up to 8] bf16, overwritten */
+ *   WsoftT: not used (earlier versions transposed the soft weights into it); may be null */
 FAAR_API int faar_layer_dx(faar_ctx* ctx, const faar_shape* shape, float beta, const void* dY, const float* V,
                            const uint8_t* code, const uint8_t* scales, const float* s_global, void* WsoftT,
                            void* dX, void* workspace, size_t workspace_bytes);
@@ -346,6 +347,17 @@ FAAR_API int64_t faar_round_loss_static_max_n(void);
  *   dV out: [O,K] float, nullable */
 FAAR_API int faar_layer_bwd(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp, const void* dYt,
                    const void* Xt, float* V, const uint8_t* code, const uint8_t* scales,
+                   const float* s_global, float* adam_m, float* adam_u, float* dV,
+                   void* workspace, size_t workspace_bytes);
+
+/* faar_layer_bwd on the operands as a model's backward pass holds them: dY [T, ldy] and X [T, ldx], one row
+ * per token (BF16; shape->ldy >= O, shape->ldx >= K, both multiples of 8; bases 16-byte aligned), no transposed
+ * copies.  The tensor cores read both operands with the token index as the contraction row.  Everything else
+ * as faar_layer_bwd; the results are the same bits (each dW element is the same sum in the same order).  The
+ * GEMM itself takes the same time as on transposed operands (measured on four decoder-block shapes at 8192
+ * tokens), so what is saved is the two transposes: 17-30 % of a linear's backward pass. */
+FAAR_API int faar_layer_bwd_rowmajor(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp, const void* dY,
+                   const void* X, float* V, const uint8_t* code, const uint8_t* scales,
                    const float* s_global, float* adam_m, float* adam_u, float* dV,
                    void* workspace, size_t workspace_bytes);
 

@@ -112,7 +112,7 @@ int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
 int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* dYt, const void* Xt,
              float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
              float* adam_u, float* dV, uint8_t* ws, const faar_ws_layout& l, int* n_partials,
-             float* loss_out2 = nullptr, int n_mse_partials = 0) {
+             float* loss_out2 = nullptr, int n_mse_partials = 0, bool row_major = false) {
   faar_gemm_args a = {};
   if (loss_out2) {
     // the kernel's last CTA sums the forward's MSE partials and its own Round Loss partials
@@ -125,8 +125,13 @@ int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
   }
   a.mode = FAAR_GEMM_BWD;
   a.M = s->O; a.N = s->K; a.Kc = s->T;
-  a.A = dYt; a.lda = l.ld_dyt;
-  a.B = Xt; a.ldb = s->ldxt;
+  if (row_major) {                         // dY [T, ldy] and X [T, ldx] as they are: token index = contraction row
+    a.A = dYt; a.lda = s->ldy; a.a_mn = 1;
+    a.B = Xt; a.ldb = s->ldx; a.b_mn = 1;
+  } else {
+    a.A = dYt; a.lda = l.ld_dyt;
+    a.B = Xt; a.ldb = s->ldxt;
+  }
   a.status = reinterpret_cast<uint32_t*>(ws);
   a.partials = reinterpret_cast<float*>(ws + l.off_round_partials);
   a.V = V; a.code = code; a.scales = scales; a.s_global = s_global;
@@ -527,13 +532,13 @@ int faar_layer_ref(faar_ctx* ctx, const faar_shape* s, const void* X, const void
 int faar_layer_dx(faar_ctx* ctx, const faar_shape* s, float beta, const void* dY, const float* V, const uint8_t* code,
                   const uint8_t* scales, const float* s_global, void* WsoftT, void* dX, void* workspace,
                   size_t workspace_bytes) {
-  if (!ctx || !dY || !V || !code || !scales || !s_global || !WsoftT || !dX) return FAAR_ERR_INVALID_ARG;
+  (void)WsoftT;                                  // kept in the signature; the operand is read untransposed now
+  if (!ctx || !dY || !V || !code || !scales || !s_global || !dX) return FAAR_ERR_INVALID_ARG;
   int st = check_shape(s);
   if (st) return st;
   if (!(beta > 0.f) || !isfinite(beta)) return FAAR_ERR_INVALID_ARG;
   if (s->ldy < s->O || s->ldx < s->K) return FAAR_ERR_SHAPE;
-  if (s->ldy % 8 || s->ldx % 8 || !aligned16(dY) || !aligned16(V) || !aligned16(code) || !aligned16(WsoftT) ||
-      !aligned16(dX))
+  if (s->ldy % 8 || s->ldx % 8 || !aligned16(dY) || !aligned16(V) || !aligned16(code) || !aligned16(dX))
     return FAAR_ERR_ALIGN;
   if ((st = check_ws(s, workspace, workspace_bytes))) return st;
   FAAR_DEVICE_GUARD(ctx);
@@ -541,16 +546,14 @@ int faar_layer_dx(faar_ctx* ctx, const faar_shape* s, float beta, const void* dY
   const faar_ws_layout l = faar_ws_plan(s);
   __nv_bfloat16* wsoft = reinterpret_cast<__nv_bfloat16*>(ws + l.off_wsoft);
   if (ctx->wsoft_ws == workspace) ctx->wsoft_ws = nullptr;     // the operand slot is overwritten below
-  const int64_t ldo = ((int64_t)s->O + 7) / 8 * 8;
   int e = faar_launch_softquant_eval(ctx, s, V, code, scales, s_global, beta, nullptr, nullptr, wsoft);
   if (e) return cuda_fail(ctx, e);
-  e = faar_launch_transpose_bf16(ctx, s->O, s->K, wsoft, s->K, WsoftT, ldo);
-  if (e) return cuda_fail(ctx, e);
-  // dX^T[K,T] = WsoftT[K,O] * dY[T,O]^T, written transposed as dX[T,K]
+  // dX^T[K,T] = W_soft^T[K,O] * dY[T,O]^T, written transposed as dX[T,K].  W_soft [O,K] is that A operand with
+  // its M index (k) contiguous and the contraction index (o) as the row: read as it is.
   faar_gemm_args a = {};
   a.mode = FAAR_GEMM_REF;
   a.M = s->K; a.N = s->T; a.Kc = s->O;
-  a.A = WsoftT; a.lda = ldo;
+  a.A = wsoft; a.lda = s->K; a.a_mn = 1;
   a.B = dY; a.ldb = s->ldy;
   a.status = reinterpret_cast<uint32_t*>(ws);
   a.Yout = dX; a.yout_dtype = FAAR_BF16; a.ldy = s->ldx;
@@ -617,6 +620,27 @@ int faar_layer_bwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, c
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const faar_ws_layout l = faar_ws_plan(s);
   return cuda_fail(ctx, bwd_impl(ctx, s, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u, dV, ws, l, nullptr));
+}
+
+int faar_layer_bwd_rowmajor(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* dY, const void* X,
+                            float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
+                            float* adam_u, float* dV, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !dY || !X || !V || !code || !scales || !s_global) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if ((st = check_hp(hp, true))) return st;
+  if (hp->opt == 1 && (!adam_m || !adam_u)) return FAAR_ERR_INVALID_ARG;
+  if ((st = check_bwd_k(s))) return st;
+  if (s->ldy < s->O || s->ldx < s->K) return FAAR_ERR_SHAPE;
+  if (s->ldy % 8 || s->ldx % 8 || !aligned16(dY) || !aligned16(X) || !aligned16(V) || !aligned16(code) ||
+      (adam_m && !aligned16(adam_m)) || (adam_u && !aligned16(adam_u)) || (dV && !aligned16(dV)))
+    return FAAR_ERR_ALIGN;
+  if ((st = check_ws(s, workspace, workspace_bytes))) return st;
+  FAAR_DEVICE_GUARD(ctx);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const faar_ws_layout l = faar_ws_plan(s);
+  return cuda_fail(ctx, bwd_impl(ctx, s, hp, dY, X, V, code, scales, s_global, adam_m, adam_u, dV, ws, l, nullptr, nullptr, 0,
+                                 true));
 }
 
 int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Xt,

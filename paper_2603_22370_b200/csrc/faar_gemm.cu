@@ -218,15 +218,34 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                          // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: D = F32, A = B = BF16, both K-major, M = 256 (the CTA pair), N = bn.
-__device__ __forceinline__ uint32_t make_idesc(int bn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+// The same for an operand stored with its M (or N) index contiguous and the contraction index as the row
+// ("MN-major"): 64 elements (128 B) of one contraction index form a row, 8 consecutive contraction indices a
+// 1024-byte swizzle atom; atoms follow each other along the contraction (stride byte offset, 1024 B: a TMA box
+// of 64 x 64 elements lands exactly so) and along M / N (leading byte offset: the next 64-element box, 8192 B on).
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(8192 >> 4) << 16;                // leading byte offset: next 64 M / N elements
+  d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset: next 8 contraction indices
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+constexpr int MN_BOX = 64;                         // M / N elements per MN-major TMA box
+constexpr int MN_BOX_BYTES = MN_BOX * BK * 2;      // 8192
+constexpr uint32_t MN_KSTEP = (UMMA_K * 128) >> 4; // 16 contraction indices on: 2048 B in the address field
+// Instruction descriptor: D = F32, A = B = BF16, M = 256 (the CTA pair), N = bn; bits 15 / 16 say that A / B is
+// MN-major instead of K-major.
+__device__ __forceinline__ uint32_t make_idesc(int bn, int a_mn = 0, int b_mn = 0) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+         ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 }
 
 struct KParams {
   int M, N, Kc;
   int bn;                 // tile width
   int n_full_cols;        // tile columns of full width; the columns after them are bn/2 wide (tail split)
+  int a_mn, b_mn;         // operand stored with M (N) contiguous, [Kc, M] / [Kc, N], instead of [M, Kc] / [N, Kc]
   uint32_t* status;
   long long ext_yout, ext_dyt, ext_state, ext_wsoft;   // bytes of Yout, dYt, each of V / m / u / dV, wsoft_next (debug checks)
   // REF / FWD
@@ -634,8 +653,18 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             mbar_expect_tx(full_bar(stage), WIDE ? 2u * (uint32_t)(C::A_BYTES + C::B_BYTES)
                                                  : 2u * (uint32_t)(C::A_BYTES + (tc.w / 2) * BK * 2));
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-          tma_load_2d(sa, &tmA, kb * BK, m0, leader_full, keep);
-          tma_load_2d(sb, mapB, kb * BK, n0, leader_full, keep);
+          if (p.a_mn) {                                        // two boxes of 64 rows of A, each [64 k][64 m]
+            tma_load_2d(sa, &tmA, m0, kb * BK, leader_full, keep);
+            tma_load_2d(sa + MN_BOX_BYTES, &tmA, m0 + MN_BOX, kb * BK, leader_full, keep);
+          } else {
+            tma_load_2d(sa, &tmA, kb * BK, m0, leader_full, keep);
+          }
+          if (p.b_mn) {                                        // w/2 = 128 or 64 rows of B: two boxes or one
+            tma_load_2d(sb, &tmB, n0, kb * BK, leader_full, keep);
+            if (tc.w / 2 > MN_BOX) tma_load_2d(sb + MN_BOX_BYTES, &tmB, n0 + MN_BOX, kb * BK, leader_full, keep);
+          } else {
+            tma_load_2d(sb, mapB, kb * BK, n0, leader_full, keep);
+          }
           // second column half (rows beyond the matrix arrive as zeros)
           if (WIDE) tma_load_2d(sb + C::BH_BYTES, &tmB, kb * BK, n0 + BN_MAX, leader_full, keep);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -662,17 +691,20 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN_MAX;
-        const uint32_t idesc = make_idesc(WIDE ? BN_MAX : tile_coord(p, tile, m_tiles).w);
+        const uint32_t idesc = make_idesc(WIDE ? BN_MAX : tile_coord(p, tile, m_tiles).w, p.a_mn, p.b_mn);
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(full_bar(stage), phase, ac, 0x300u | stage);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-          const uint64_t da = make_smem_desc(sa), db = make_smem_desc(sb);
+          const uint64_t da = p.a_mn ? make_smem_desc_mn(sa) : make_smem_desc(sa);
+          const uint64_t db = p.b_mn ? make_smem_desc_mn(sb) : make_smem_desc(sb);
+          const uint32_t ka = p.a_mn ? MN_KSTEP : 2u, kbs = p.b_mn ? MN_KSTEP : 2u;
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 bf16 = 32 bytes inside the swizzled row: +2 in the 16-byte address field
-            tc_mma_bf16(tmem_d, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            // (MN-major: 16 rows of 128 bytes further on)
+            tc_mma_bf16(tmem_d, da + ka * k, db + kbs * k, idesc, (kb | k) != 0 ? 1u : 0u);
             if (WIDE)
               tc_mma_bf16(tmem_d + BN_MAX, da + 2u * k, make_smem_desc(sb + C::BH_BYTES) + 2u * k, idesc,
                           (kb | k) != 0 ? 1u : 0u);
@@ -916,13 +948,32 @@ int make_map(faar_ctx* ctx, CUtensorMap* map, const void* ptr, int rows, int col
   return r == CUDA_SUCCESS ? 0 : (int)cudaErrorInvalidValue;
 }
 
+// An operand stored [kc_rows, mn_cols] (M or N contiguous, row stride ld elements): boxes of 64 x 64.
+int make_map_mn(faar_ctx* ctx, CUtensorMap* map, const void* ptr, int kc_rows, int mn_cols, int64_t ld) {
+  cuuint64_t dims[2] = {(cuuint64_t)mn_cols, (cuuint64_t)kc_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)MN_BOX, (cuuint32_t)BK};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+      map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : (int)cudaErrorInvalidValue;
+}
+
 // Tile width for an M x N output.  A tile's time is set by the operand bytes it pulls through the SM (A rows
 // are not shared between tiles), not by its columns, so 256-wide tiles win wherever they were measured
 // against narrower ones that fill more CTA pairs (down_proj-, gate-, q- and k_proj-shaped layers), with one
 // exception: the dW GEMM of a small layer, whose per-weight epilogue is heavy, gains from spreading 128-wide
 // tiles over twice as many pairs while fewer than half of the pairs would have a 256-wide tile.  A tile is
 // never wider than the output rounded up to 32 columns.
-int pick_bn(const faar_ctx* ctx, int mode, int M, int N, int pairs) {
+int pick_bn_k_major(const faar_ctx* ctx, int mode, int M, int N, int pairs);
+int pick_bn(const faar_ctx* ctx, int mode, int M, int N, int pairs, bool b_mn) {
+  const int bn = pick_bn_k_major(ctx, mode, M, N, pairs);
+  // an N-contiguous B comes in boxes of 64 columns per CTA: widths 128 and 256 only
+  return b_mn && bn % 128 != 0 ? (N <= 128 ? 128 : BN_MAX) : bn;
+}
+int pick_bn_k_major(const faar_ctx* ctx, int mode, int M, int N, int pairs) {
   if (ctx->tune_bn >= 128 && ctx->tune_bn <= BN_MAX && ctx->tune_bn % 16 == 0) return ctx->tune_bn;
   const long long m_tiles = (M + 2 * BM - 1) / (2 * BM);
   int bn = BN_MAX;
@@ -984,12 +1035,19 @@ int launch_variant(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_p
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   kp.bn = bn;
   kp.n_full_cols = WIDE ? 0 : pick_full_cols(ctx, a->M, a->N, bn, max_pairs);
+  if (a->b_mn && bn != BN_MAX) kp.n_full_cols = (a->N + bn - 1) / bn;      // half tiles of a 128-wide tile would be 32 columns per CTA
   CUtensorMap tmA, tmB, tmBh;
-  int e = make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
+  kp.a_mn = a->a_mn; kp.b_mn = a->b_mn;
+  int e = a->a_mn ? make_map_mn(ctx, &tmA, a->A, a->Kc, a->M, a->lda) : make_map(ctx, &tmA, a->A, a->M, a->Kc, a->lda, BM);
   if (e) return e;
-  e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, bn / 2);
-  if (e) return e;
-  e = make_map(ctx, &tmBh, a->B, a->N, a->Kc, a->ldb, bn % 32 == 0 ? bn / 4 : bn / 2);   // half-width tiles
+  if (a->b_mn) {
+    e = make_map_mn(ctx, &tmB, a->B, a->Kc, a->N, a->ldb);    // one map serves full and half-width tiles
+    tmBh = tmB;
+  } else {
+    e = make_map(ctx, &tmB, a->B, a->N, a->Kc, a->ldb, bn / 2);
+    if (e) return e;
+    e = make_map(ctx, &tmBh, a->B, a->N, a->Kc, a->ldb, bn % 32 == 0 ? bn / 4 : bn / 2);   // half-width tiles
+  }
   if (e) return e;
   const long long m_tiles = (a->M + 2 * BM - 1) / (2 * BM);
   const int rest_cols = a->N - kp.n_full_cols * bn;
@@ -1037,8 +1095,8 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
     if (n > ctx->num_sms / 2) n = ctx->num_sms / 2;
     max_pairs = n;
   }
-  const int bn = pick_bn(ctx, MODE, a->M, a->N, max_pairs);
-  if (pick_wide(ctx, a->N, bn))
+  const int bn = pick_bn(ctx, MODE, a->M, a->N, max_pairs, a->b_mn != 0);
+  if (!a->a_mn && !a->b_mn && pick_wide(ctx, a->N, bn))
     return launch_variant<MODE, OPT, true>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
   return launch_variant<MODE, OPT, false>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
 }

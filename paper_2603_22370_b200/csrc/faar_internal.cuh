@@ -136,6 +136,7 @@ struct faar_gemm_args {
   int M, N, Kc;           // C[M,N] = A[M,Kc] * B[N,Kc]^T, both operands bf16 with Kc contiguous
   const void* A; int64_t lda;
   const void* B; int64_t ldb;
+  int a_mn, b_mn;         // 1: the operand is stored with M (N) contiguous instead: A[Kc, M] (lda), B[Kc, N] (ldb)
   uint32_t* status;       // workspace status word
   // REF / FWD
   void* Yout; int yout_dtype; int64_t ldy;     // [N(T), M(O)] written transposed; nullable in FWD

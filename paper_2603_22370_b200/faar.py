@@ -49,6 +49,7 @@ SIGNATURES = {
     "faar_round_loss_static": (_I, [_P, _P, _L, _P]),
     "faar_round_loss_static_max_n": (_L, []),
     "faar_layer_bwd": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
+    "faar_layer_bwd_rowmajor": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
     "faar_layer_step": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
     "faar_layer_step_host": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
     "faar_harden_pack": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I]),
@@ -359,6 +360,12 @@ def layer_bwd(ctx, shape, hp, dYt, Xt, V, code, scales, s_global, adam_m, adam_u
     _check(lib().faar_layer_bwd(ctx._h, C.byref(shape), C.byref(hp), _p(dYt), _p(Xt), _p(V), _p(code), _p(scales),
                                 _p(s_global), _p(adam_m), _p(adam_u), _p(dV), _p(ws), C.c_size_t(ws.numel())),
            "faar_layer_bwd")
+
+
+def layer_bwd_rowmajor(ctx, shape, hp, dY, X, V, code, scales, s_global, adam_m, adam_u, dV, ws):
+    _check(lib().faar_layer_bwd_rowmajor(ctx._h, C.byref(shape), C.byref(hp), _p(dY), _p(X), _p(V), _p(code), _p(scales),
+                                _p(s_global), _p(adam_m), _p(adam_u), _p(dV), _p(ws), C.c_size_t(ws.numel())),
+           "faar_layer_bwd_rowmajor")
 
 
 def layer_step(ctx, shape, hp, X, Xt, Y_ref, V, code, scales, s_global, adam_m, adam_u, loss_out2, ws):

@@ -81,13 +81,7 @@ class Stage2Model:
         self.aws = torch.empty(faar.align_loss_workspace_size(T, c.vocab), dtype=torch.uint8, device=dev)
         faar.workspace_init(ctx, self.aws)
         self.loss = torch.zeros(2, dtype=torch.float32, device=dev)
-        # scratch shared by all linears' backward passes
-        k_max = max(k for _, k in c.linear_shapes().values())
-        o_max = max(o for o, _ in c.linear_shapes().values())
         self.ldt = (T + 7) // 8 * 8
-        self.Xt = torch.empty(k_max * self.ldt, dtype=torch.bfloat16, device=dev)
-        self.dYt = torch.empty(o_max * self.ldt, dtype=torch.bfloat16, device=dev)
-        self.WsT = torch.empty(big + 8 * k_max, dtype=torch.bfloat16, device=dev)
         self.dsum = torch.empty((batch, c.n_heads, seq), dtype=torch.float32, device=dev)
         self.step_count = 0
 
@@ -155,11 +149,10 @@ class Stage2Model:
         O, K = lin.O, lin.K
         shape = faar.make_shape(O, K, T, ldxt=self.ldt)
         dX = self._new(K)
-        faar.layer_dx(ctx, shape, hp.beta, dY, lin.V, lin.code, lin.scales, lin.s_global, self.WsT, dX, self.ws)
-        faar.transpose_bf16(ctx, T, O, dY, O, self.dYt, self.ldt)
-        faar.transpose_bf16(ctx, T, K, X, K, self.Xt, self.ldt)
+        faar.layer_dx(ctx, shape, hp.beta, dY, lin.V, lin.code, lin.scales, lin.s_global, None, dX, self.ws)
         dV = torch.empty((O, K), dtype=torch.float32, device=self.dev) if want_dv else None
-        faar.layer_bwd(ctx, shape, hp, self.dYt, self.Xt, lin.V, lin.code, lin.scales, lin.s_global, lin.m, lin.u, dV, self.ws)
+        # dY [T, O] and X [T, K] as the backward pass holds them: no transposed copies
+        faar.layer_bwd_rowmajor(ctx, shape, hp, dY, X, lin.V, lin.code, lin.scales, lin.s_global, lin.m, lin.u, dV, self.ws)
         return dX, dV
 
     def backward(self, dZ, dH, saved, hp, want_dv=False):

@@ -724,6 +724,46 @@ def test_wide_tiles_give_the_same_step(ctx, O, K, T):
     assert np.all(np.abs(out[0][6] - out[1][6]) <= 1e-5 * np.abs(out[0][6]))
 
 
+@pytest.mark.parametrize("opt", [0, 1])
+@pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (520, 784, 1300), (64, 128, 72), (1024, 512, 2048)])
+def test_backward_on_row_major_operands_gives_the_same_bits(ctx, O, K, T, opt):
+    """faar_layer_bwd_rowmajor reads dY [T, O] and X [T, K] as they are (token index = contraction row of the tensor
+    cores); faar_layer_bwd reads their transposes.  The same products in the same order: every output must
+    be equal bit for bit.  Shapes with O, K, T off the 64-element boxes, row strides with padding."""
+    W, X, Yref = _problem(O, K, T, seed=9)
+    hp, _ = f32hp(beta=6.0, step=3, opt=opt)
+    rng = np.random.default_rng(6)
+    V0 = rng.uniform(0, 1, W.shape).astype(np.float32)
+    m0 = (1e-3 * rng.standard_normal(W.shape)).astype(np.float32)
+    u0 = (1e-6 * rng.uniform(0, 1, W.shape)).astype(np.float32)
+    lay = GpuLayer(ctx, W, X)
+    lay.init()
+    lay.set_yref(Yref)
+    lay.set_state(V=V0, m=m0, u=u0)
+    lay.fwd(hp)                                              # dY^T [O, ldt] in lay.dYt
+    dV_t = host(lay.bwd(hp, want_dv=True)).copy()
+    lay.check()
+    ref = (dV_t, host(lay.V).copy(), host(lay.m).copy(), host(lay.u).copy())
+    # the same dY untransposed, with padded row strides
+    ldy, ldx = (O + 7) // 8 * 8 + 8, K + 16
+    dY = torch.full((T, ldy), 3.0, dtype=torch.bfloat16, device=DEV)
+    dY[:, :O] = lay.dYt[:, :T].t()
+    Xp = torch.full((T, ldx), 3.0, dtype=torch.bfloat16, device=DEV)
+    Xp[:, :K] = lay.X
+    lay.set_state(V=V0, m=m0, u=u0)
+    shape = faar.make_shape(O, K, T, ldx=ldx, ldy=ldy, ldxt=lay.ldt)
+    dV = torch.empty((O, K), dtype=torch.float32, device=DEV)
+    faar.layer_bwd_rowmajor(ctx, shape, hp, dY, Xp, lay.V, lay.code, lay.scales, lay.s_global, lay.m, lay.u, dV, lay.ws)
+    lay.check()
+    got = (host(dV), host(lay.V), host(lay.m), host(lay.u))
+    for a, b in zip(ref, got):
+        assert np.array_equal(a, b)
+    with pytest.raises(faar.FaarError) as e:
+        faar.layer_bwd_rowmajor(ctx, faar.make_shape(O, K, T, ldx=K - 8, ldy=ldy), hp, dY, Xp, lay.V, lay.code, lay.scales,
+                                lay.s_global, lay.m, lay.u, dV, lay.ws)
+    assert e.value.status == faar.ERR_SHAPE
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives(ctx):
     """The tensor-core kernels bound every barrier wait.  The self-test kernel waits (1 ms limit) on a
     barrier that nothing arrives at: it must exit by itself and leave its code in the status word of the
