@@ -851,6 +851,38 @@ def run_ours(args):
     ms_e2e = timed(lambda: e2e_job(e2e_steps))
     e2e_value = n_gpus * e2e_steps / (ms_e2e * 1e-3)
     faar.check_status(ctx, ws)
+
+    # ---- the same end to end with quantised activations (the X_q of Eq. 5): the batch travels as the packed NVFP4
+    # codes and block scales the library's own quantiser produced (4.5 bits per value) plus its frozen target
+    with torch.cuda.stream(stream):
+        Xq_units = torch.empty_like(X)
+        sx = torch.empty(1, dtype=torch.float32, device=device)
+        px = torch.empty((T, K // 2), dtype=torch.uint8, device=device)
+        scx = torch.empty((T, K // 16), dtype=torch.uint8, device=device)
+        faar.act_fakequant(ctx, T, K, X, K, 0.0, Xq_units, K, sx, px, scx, ws)
+    stream.synchronize()
+    act_scale = float(sx.item())
+    px_h, scx_h, yref_h = px.cpu().pin_memory(), scx.cpu().pin_memory(), Yref.cpu().pin_memory()
+    pk_sets = [(torch.empty_like(px), torch.empty_like(scx), torch.empty_like(X), torch.empty_like(Yref)) for _ in range(2)]
+    pk_bytes = px_h.numel() + scx_h.numel() + yref_h.numel() * 2
+    del Xq_units
+
+    def e2e_packed_job(n):
+        m.zero_()
+        u.zero_()
+        faar.softquant_init(ctx, shape, W, 0.0, scales, s_global, code, V, ws)
+        for t in range(n):
+            hp = faar.make_hparams(beta=beta_at(t, n), step=t + 1, act_scale=act_scale)
+            pd, sd, xd, yd = pk_sets[t & 1]
+            faar.layer_step_host_nvfp4(ctx, shape, hp, px_h, scx_h, yref_h, pd, sd, xd, yd, V, code, scales, s_global, m, u,
+                                       loss, loss_h, ws)
+        faar.harden_pack(ctx, shape, V, code, scales, s_global, packed, scales_out, None, None)
+
+    with torch.cuda.stream(stream):
+        e2e_packed_job(3)
+    stream.synchronize()
+    ms_e2e_pk = timed(lambda: e2e_packed_job(e2e_steps))
+    faar.check_status(ctx, ws)
     clocks = sampler.stop() if sampler else None
 
     if rank != 0:
@@ -936,6 +968,12 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "steps": e2e_steps,
                     "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": 8,
                     "path": e2e_path},
+            "e2e_nvfp4_activations": {"value": n_gpus * e2e_steps / (ms_e2e_pk * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                                      "h2d_bytes_per_step": pk_bytes, "d2h_bytes_per_step": 8,
+                                      "path": "faar_layer_step_host_nvfp4: quantised activations (Eq. 5's X_q) as packed NVFP4 "
+                                              "codes + block scales and the frozen target copied in from pinned memory, "
+                                              "expanded on the device, step, losses copied out; a different workload from "
+                                              "`e2e` (which steps on the unquantised BF16 batch)"},
             "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "kernels": kernels, "final_loss": loss_final,
             "step_tflops": round(2 * flops * steps / (ms_job * 1e-3) / 1e12, 1)}

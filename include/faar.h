@@ -395,6 +395,28 @@ FAAR_API int faar_layer_step_host(faar_ctx* ctx, const faar_shape* shape, const 
                                   const float* s_global, float* adam_m, float* adam_u, float* loss_dev2,
                                   float* loss_host2, void* workspace, size_t workspace_bytes);
 
+/* The inverse of faar_act_fakequant's packed output: out[r][c] = sign * E2M1 node * E4M3 block scale as BF16
+ * (exact; the FP32 tensor scale stays outside), from packed [rows, K/2] nibbles (8-byte aligned) and scales
+ * [rows, K/16] bytes, both dense.  out: [rows, ld] bf16, ld >= K, multiple of 8, 16-byte aligned.  K % 16 == 0. */
+FAAR_API int faar_nvfp4_expand(faar_ctx* ctx, int rows, int K, const void* packed, const void* scales, void* out,
+                               int64_t ld);
+
+/* faar_layer_step_host for quantised activations (the X_q of Eq. 5): the batch crosses the bus as the packed
+ * NVFP4 codes and block scales that faar_act_fakequant produced (4.5 bits per value instead of 16), together
+ * with its frozen target Y_ref (computed from the unquantised X, Procedure step 8, so it cannot be rebuilt
+ * from what arrives).  On the device the batch is expanded into Xq_dev [T, ldx] (faar_nvfp4_expand) and the
+ * step runs on it with hp->act_scale = the batch's FP32 tensor scale (required, > 0); the dW GEMM reads
+ * Xq_dev with the token index as its contraction row, so no transposed copy is built.
+ *   Xpacked_host [T, K/2], Xscales_host [T, K/16]: host (ideally pinned), dense
+ *   Xpacked_dev, Xscales_dev, Xq_dev, Yref_dev: the caller's device staging buffers (16-byte aligned)
+ * Bytes moved: T*K*9/16 + T*O*sizeof(yref_dtype) in, 8 out.  Stream order, validation before the first copy
+ * and the alternation of two staging sets are as for faar_layer_step_host. */
+FAAR_API int faar_layer_step_host_nvfp4(faar_ctx* ctx, const faar_shape* shape, const faar_hparams* hp,
+                   const void* Xpacked_host, const void* Xscales_host, const void* Y_ref_host,
+                   void* Xpacked_dev, void* Xscales_dev, void* Xq_dev, void* Yref_dev, float* V,
+                   const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
+                   float* adam_u, float* loss_dev2, float* loss_host2, void* workspace, size_t workspace_bytes);
+
 /* ---- part 5: harden + pack ---------------------------------------------------
  * Procedure steps 25-26, Eq. 7: v_hat = (v >= 0.5); weight code = k + v_hat.
  *   packed     out: [O,K/2] u8           scales_out out: [O,K/16] u8 (copy; nullable)

@@ -112,7 +112,7 @@ int fwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
 int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* dYt, const void* Xt,
              float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
              float* adam_u, float* dV, uint8_t* ws, const faar_ws_layout& l, int* n_partials,
-             float* loss_out2 = nullptr, int n_mse_partials = 0, bool row_major = false) {
+             float* loss_out2 = nullptr, int n_mse_partials = 0, int row_major = 0) {
   faar_gemm_args a = {};
   if (loss_out2) {
     // the kernel's last CTA sums the forward's MSE partials and its own Round Loss partials
@@ -125,8 +125,11 @@ int bwd_impl(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const v
   }
   a.mode = FAAR_GEMM_BWD;
   a.M = s->O; a.N = s->K; a.Kc = s->T;
-  if (row_major) {                         // dY [T, ldy] and X [T, ldx] as they are: token index = contraction row
+  if (row_major == 1) {                    // dY [T, ldy] and X [T, ldx] as they are: token index = contraction row
     a.A = dYt; a.lda = s->ldy; a.a_mn = 1;
+    a.B = Xt; a.ldb = s->ldx; a.b_mn = 1;
+  } else if (row_major == 2) {             // dY^T from the forward kernel, X [T, ldx] as it is
+    a.A = dYt; a.lda = l.ld_dyt;
     a.B = Xt; a.ldb = s->ldx; a.b_mn = 1;
   } else {
     a.A = dYt; a.lda = l.ld_dyt;
@@ -640,7 +643,7 @@ int faar_layer_bwd_rowmajor(faar_ctx* ctx, const faar_shape* s, const faar_hpara
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const faar_ws_layout l = faar_ws_plan(s);
   return cuda_fail(ctx, bwd_impl(ctx, s, hp, dY, X, V, code, scales, s_global, adam_m, adam_u, dV, ws, l, nullptr, nullptr, 0,
-                                 true));
+                                 1));
 }
 
 int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Xt,
@@ -661,6 +664,87 @@ int faar_layer_step(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, 
   return cuda_fail(ctx, e);
 }
 
+int faar_nvfp4_expand(faar_ctx* ctx, int rows, int K, const void* packed, const void* scales, void* out, int64_t ld) {
+  if (!ctx || !packed || !scales || !out) return FAAR_ERR_INVALID_ARG;
+  if (rows <= 0 || K <= 0 || K % 16 || ld < K) return FAAR_ERR_SHAPE;
+  if (ld % 8 || !aligned16(out) || (reinterpret_cast<uintptr_t>(packed) & 7u)) return FAAR_ERR_ALIGN;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_nvfp4_expand(ctx, rows, K, reinterpret_cast<const uint8_t*>(packed),
+                                                 reinterpret_cast<const uint8_t*>(scales), out, ld));
+}
+
+// Copy-stream bookkeeping shared by the host-batch entry points: creates the stream and events on first use and
+// makes the copy stream wait until the staging set `key` is free again.  Returns the event slot of this call.
+static cudaError_t begin_host_copy(faar_ctx* ctx, const void* key, int* slot_out) {
+  cudaError_t e = cudaSuccess;
+  if (!ctx->copy_stream) {                       // host resources of this path, created on first use
+    e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_copied, cudaEventDisableTiming);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming);
+    if (e != cudaSuccess) return e;
+  }
+  // The staging buffers of this call were last read by the step of two calls ago when the caller
+  // alternates between two sets (then this copy overlaps the previous step), by the previous step
+  // when it reuses one set (then the copy waits for it).
+  const unsigned long long n = ctx->host_calls++;
+  const int slot = (int)(n & 1);
+  if (n >= 2) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot], 0);
+  if (e == cudaSuccess && n >= 1 && ctx->last_staging == key)
+    e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot ^ 1], 0);
+  if (e == cudaSuccess && n == 0) {              // order after whatever the caller enqueued before (set-up)
+    e = cudaEventRecord(ctx->ev_done[slot], ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot], 0);
+  }
+  ctx->last_staging = key;
+  *slot_out = slot;
+  return e;
+}
+
+int faar_layer_step_host_nvfp4(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* Xpacked_host,
+                               const void* Xscales_host, const void* Y_ref_host, void* Xpacked_dev, void* Xscales_dev,
+                               void* Xq_dev, void* Yref_dev, float* V, const uint8_t* code, const uint8_t* scales,
+                               const float* s_global, float* adam_m, float* adam_u, float* loss_dev2,
+                               float* loss_host2, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !Xpacked_host || !Xscales_host || !Y_ref_host || !Xpacked_dev || !Xscales_dev || !Xq_dev || !Yref_dev ||
+      !loss_dev2 || !loss_host2)
+    return FAAR_ERR_INVALID_ARG;
+  // every check of the step itself, before the first copy is enqueued (X^T is not needed: the dW GEMM reads
+  // the expanded batch with the token index as its contraction row)
+  int st = validate_step(ctx, s, hp, Xq_dev, Xq_dev, Yref_dev, V, code, scales, s_global, adam_m, adam_u, loss_dev2,
+                         workspace, workspace_bytes);
+  if (st) return st;
+  if (!(hp->act_scale > 0.f)) return FAAR_ERR_INVALID_ARG;      // the tensor scale of the quantised batch
+  if ((reinterpret_cast<uintptr_t>(Xpacked_dev) & 15u) || (reinterpret_cast<uintptr_t>(Xscales_dev) & 15u)) return FAAR_ERR_ALIGN;
+  FAAR_DEVICE_GUARD(ctx);
+  int slot = 0;
+  cudaError_t e = begin_host_copy(ctx, Xq_dev, &slot);
+  const size_t ybytes = s->yref_dtype == FAAR_BF16 ? 2 : 4;
+  const size_t n_val = (size_t)s->T * (size_t)s->K;
+  if (e == cudaSuccess) e = cudaMemcpyAsync(Xpacked_dev, Xpacked_host, n_val / 2, cudaMemcpyHostToDevice, ctx->copy_stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(Xscales_dev, Xscales_host, n_val / 16, cudaMemcpyHostToDevice, ctx->copy_stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(Yref_dev, Y_ref_host, (size_t)(s->yref_transposed ? s->O : s->T) * (size_t)s->ldy * ybytes,
+                        cudaMemcpyHostToDevice, ctx->copy_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_copied, ctx->copy_stream);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->stream, ctx->ev_copied, 0);
+  if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+  int le = faar_launch_nvfp4_expand(ctx, s->T, s->K, reinterpret_cast<const uint8_t*>(Xpacked_dev),
+                                    reinterpret_cast<const uint8_t*>(Xscales_dev), Xq_dev, s->ldx);
+  if (le) return cuda_fail(ctx, le);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const faar_ws_layout l = faar_ws_plan(s);
+  void* dYt = ws + l.off_dyt;
+  int np_mse = 0, np_round = 0;
+  le = fwd_impl(ctx, s, hp, Xq_dev, Yref_dev, V, code, scales, s_global, dYt, nullptr, ws, l, &np_mse);
+  if (le) return cuda_fail(ctx, le);
+  le = bwd_impl(ctx, s, hp, dYt, Xq_dev, V, code, scales, s_global, adam_m, adam_u, nullptr, ws, l, &np_round, loss_dev2,
+                np_mse, 2);
+  if (le) return cuda_fail(ctx, le);
+  e = cudaMemcpyAsync(loss_host2, loss_dev2, 2 * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->ev_done[slot], ctx->stream);
+  return cuda_fail(ctx, (int)e);
+}
+
 int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X_host,
                          const void* Y_ref_host, const void* W, void* X_dev, void* Xt_dev, void* Yref_dev, float* V,
                          const uint8_t* code, const uint8_t* scales, const float* s_global, float* adam_m,
@@ -678,26 +762,8 @@ int faar_layer_step_host(faar_ctx* ctx, const faar_shape* s, const faar_hparams*
     if (s->ldw % 8 || !aligned16(W)) return FAAR_ERR_ALIGN;
   }
   FAAR_DEVICE_GUARD(ctx);
-  cudaError_t e = cudaSuccess;
-  if (!ctx->copy_stream) {                       // host resources of this path, created on first use
-    e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_copied, cudaEventDisableTiming);
-    for (int i = 0; i < 2 && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming);
-    if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
-  }
-  // The staging buffers of this call were last read by the step of two calls ago when the caller
-  // alternates between two sets (then this copy overlaps the previous step), by the previous step
-  // when it reuses one set (then the copy waits for it).
-  const unsigned long long n = ctx->host_calls++;
-  const int slot = (int)(n & 1);
-  if (n >= 2) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot], 0);
-  if (e == cudaSuccess && n >= 1 && ctx->last_staging == X_dev)
-    e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot ^ 1], 0);
-  if (e == cudaSuccess && n == 0) {              // order after whatever the caller enqueued before (set-up)
-    e = cudaEventRecord(ctx->ev_done[slot], ctx->stream);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[slot], 0);
-  }
-  ctx->last_staging = X_dev;
+  int slot = 0;
+  cudaError_t e = begin_host_copy(ctx, X_dev, &slot);
   const size_t ybytes = s->yref_dtype == FAAR_BF16 ? 2 : 4;
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(X_dev, X_host, (size_t)s->T * (size_t)s->ldx * 2, cudaMemcpyHostToDevice, ctx->copy_stream);

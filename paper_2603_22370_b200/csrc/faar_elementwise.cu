@@ -422,6 +422,36 @@ act_fakequant_kernel(const __nv_bfloat16* __restrict__ X, int T, int K, int64_t 
   }
 }
 
+// ---- packed NVFP4 activations back to the BF16 operand: the inverse of the kernel above -------------------
+// out[r][c] = sign * node(code) * block scale (the FP32 tensor scale stays outside, as in act_fakequant's X_q):
+// exactly the values act_fakequant wrote, from 4.5 bits per value instead of 16.  One thread per 16-value block.
+__global__ void __launch_bounds__(EW_THREADS)
+nvfp4_expand_kernel(const uint8_t* __restrict__ packed, const uint8_t* __restrict__ scales, int rows, int K,
+                    __nv_bfloat16* __restrict__ out, int64_t ld) {
+  const uint32_t blocks_per_row = K / 16;
+  const int64_t total = (int64_t)rows * blocks_per_row;
+  for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < total; b += (int64_t)gridDim.x * blockDim.x) {
+    const uint2 cw = *reinterpret_cast<const uint2*>(packed + b * 8);
+    const float sg = faar_e4m3_to_float(scales[b]);
+    const uint32_t w[2] = {cw.x, cw.y};
+    uint32_t o[8];
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+      uint32_t h[2];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const uint32_t nib = (w[(i + e) >> 3] >> (4 * ((i + e) & 7))) & 0xFu;
+        const float mag = __fmul_rn(faar_node(nib & 7), sg);            // exact: 2 x 4 significant bits
+        h[e] = __float_as_uint(mag) | ((nib & 8u) << 28);
+      }
+      o[i >> 1] = __byte_perm(h[0], h[1], 0x7632);                       // the two high halves: a BF16 pair
+    }
+    uint4* dst = reinterpret_cast<uint4*>(out + block_offset(b, blocks_per_row, ld, ld == K));
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+  }
+}
+
 // ---- Eq. 2 / Eq. 3 -----------------------------------------------------------------------------
 // FP32 outputs (W_soft, H): the parity view, relative error below 1e-6.
 // BF16 output: the operand of the forward GEMM.  It is rounded from a cheaper FP32 evaluation whose
@@ -750,6 +780,15 @@ int faar_launch_act_fakequant(faar_ctx* ctx, int T, int K, const void* X, int64_
                                  (const unsigned long long*)amax_word, reinterpret_cast<__nv_bfloat16*>(Xq), ldq,
                                  s_global_out, packed, scales);
   if (e != cudaSuccess) return (int)e;
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_nvfp4_expand(faar_ctx* ctx, int rows, int K, const uint8_t* packed, const uint8_t* scales, void* out,
+                             int64_t ld) {
+  const int64_t blocks = (int64_t)rows * (K / 16);
+  faar_prof_scope ps(ctx, FAAR_K_ACT_FAKEQUANT);
+  nvfp4_expand_kernel<<<grid_for(ctx, blocks, 8), EW_THREADS, 0, ctx->stream>>>(packed, scales, rows, K,
+                                                                               reinterpret_cast<__nv_bfloat16*>(out), ld);
   return (int)cudaGetLastError();
 }
 

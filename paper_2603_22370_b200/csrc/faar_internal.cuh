@@ -86,6 +86,7 @@ static inline faar_ws_layout faar_ws_plan(const faar_shape* s) {
 int faar_launch_softquant_init(faar_ctx*, const faar_shape*, const void* W, float s_global_in,
                                uint8_t* scales, float* s_global_out, uint8_t* code, float* V,
                                unsigned long long* amax_word);
+int faar_launch_nvfp4_expand(faar_ctx*, int rows, int K, const uint8_t* packed, const uint8_t* scales, void* out, int64_t ld);
 int faar_launch_softquant_eval(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta,
                                float* W_soft, float* h, __nv_bfloat16* W_soft_bf16,

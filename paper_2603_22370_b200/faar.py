@@ -52,6 +52,8 @@ SIGNATURES = {
     "faar_layer_bwd_rowmajor": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
     "faar_layer_step": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
     "faar_layer_step_host": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
+    "faar_nvfp4_expand": (_I, [_P, _I, _I, _P, _P, _P, _L]),
+    "faar_layer_step_host_nvfp4": (_I, [_P] * 19 + [_Z]),
     "faar_harden_pack": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _I]),
     "faar_align_loss_workspace_size": (_I, [_I, _I, _P]),
     "faar_align_loss": (_I, [_P, _I, _I, _I, _P, _P, _L, _P, _P, _L, _F, _F, _P, _P, _P, _P, _Z]),
@@ -390,6 +392,20 @@ def layer_step_host(ctx, shape, hp, X_host, Y_ref_host, W, X_dev, Xt_dev, Yref_d
                                       _p(code), _p(scales), _p(s_global), _p(adam_m), _p(adam_u), _p(loss_dev2),
                                       C.c_void_p(loss_host2.data_ptr()), _p(ws), C.c_size_t(ws.numel())),
            "faar_layer_step_host")
+
+
+def nvfp4_expand(ctx, rows, K, packed, scales, out, ld):
+    _check(lib().faar_nvfp4_expand(ctx._h, rows, K, _p(packed), _p(scales), _p(out), C.c_int64(ld)), "faar_nvfp4_expand")
+
+
+def layer_step_host_nvfp4(ctx, shape, hp, Xpacked_host, Xscales_host, Y_ref_host, Xpacked_dev, Xscales_dev, Xq_dev, Yref_dev,
+                          V, code, scales, s_global, adam_m, adam_u, loss_dev2, loss_host2, ws):
+    """Host tensors (pinned): packed codes, block scales, frozen target, the two-float loss."""
+    _check(lib().faar_layer_step_host_nvfp4(
+        ctx._h, C.byref(shape), C.byref(hp), C.c_void_p(Xpacked_host.data_ptr()), C.c_void_p(Xscales_host.data_ptr()),
+        C.c_void_p(Y_ref_host.data_ptr()), _p(Xpacked_dev), _p(Xscales_dev), _p(Xq_dev), _p(Yref_dev), _p(V), _p(code),
+        _p(scales), _p(s_global), _p(adam_m), _p(adam_u), _p(loss_dev2), C.c_void_p(loss_host2.data_ptr()), _p(ws),
+        C.c_size_t(ws.numel())), "faar_layer_step_host_nvfp4")
 
 
 class KernelTime(C.Structure):

@@ -650,6 +650,61 @@ def test_layer_step_host_matches_device_steps(ctx, two_sets):
     assert rel_l2(out[3][0], out[0][0]) <= 2e-3 and abs(out[3][2][0] - out[0][2][0]) <= 1e-2 * out[0][2][0]
 
 
+def test_packed_activation_batches_from_the_host_match_device_steps(ctx):
+    """Quantised-activation steps whose batches arrive as packed NVFP4 codes + block scales (+ the frozen target)
+    and are expanded on the device must give the trajectory of the same steps run on the quantiser's own BF16
+    output, bit for bit; the expansion alone must reproduce that output bit for bit."""
+    O, K, T = 128, 256, 520
+    W, _ = inputs.config2(2, O, K, T)
+    batches = [inputs.config2(30 + i, 8, K, T)[1] for i in range(4)]
+    yrefs = [inputs.to_bf16_f32(fo.layer_ref(Xb, W)) for Xb in batches]
+    lay = GpuLayer(ctx, W, batches[0])
+    q = []                                                    # per batch: Xq units, tensor scale, packed, scales
+    for Xb in batches:
+        Xd = dev_bf16(Xb)
+        Xq = torch.empty_like(Xd)
+        sx = torch.empty(1, dtype=torch.float32, device=DEV)
+        px = torch.empty((T, K // 2), dtype=torch.uint8, device=DEV)
+        sc = torch.empty((T, K // 16), dtype=torch.uint8, device=DEV)
+        faar.act_fakequant(ctx, T, K, Xd, K, 0.0, Xq, K, sx, px, sc, lay.ws)
+        out = torch.full((T, K + 8), 7.0, dtype=torch.bfloat16, device=DEV)
+        faar.nvfp4_expand(ctx, T, K, px, sc, out, K + 8)
+        torch.cuda.synchronize()
+        assert torch.equal(out[:, :K].view(torch.int16), Xq.view(torch.int16)) and torch.all(out[:, K:] == 7.0)
+        q.append((Xq, float(sx.item()), px.cpu().pin_memory(), sc.cpu().pin_memory()))
+    out = []
+    for mode in ("device", "host packed"):
+        lay = GpuLayer(ctx, W, batches[0])
+        lay.init()
+        loss_h = torch.zeros(2).pin_memory()
+        sets = [(torch.empty((T, K // 2), dtype=torch.uint8, device=DEV), torch.empty((T, K // 16), dtype=torch.uint8, device=DEV),
+                 torch.empty((T, K), dtype=torch.bfloat16, device=DEV), torch.empty((T, O), dtype=torch.bfloat16, device=DEV))
+                for _ in range(2)]
+        for t, (Xq, sx, px_h, sc_h) in enumerate(q):
+            hp = faar.make_hparams(beta=4.0 + t, step=t + 1, act_scale=sx)
+            if mode == "device":
+                lay.X.copy_(Xq)
+                faar.transpose_bf16(ctx, T, K, lay.X, K, lay.Xt, lay.ldt)
+                lay.set_yref(yrefs[t])
+                lay.step(hp)
+            else:
+                pd, sd, xd, yd = sets[t % 2]
+                y_h = torch.from_numpy(yrefs[t]).to(torch.bfloat16).pin_memory()
+                faar.layer_step_host_nvfp4(ctx, lay.shape, hp, px_h, sc_h, y_h, pd, sd, xd, yd, lay.V, lay.code, lay.scales,
+                                           lay.s_global, lay.m, lay.u, lay.loss, loss_h, lay.ws)
+            torch.cuda.synchronize()
+        lay.check()
+        out.append((host(lay.V).copy(), host(lay.m).copy(), host(lay.loss).copy(), loss_h.numpy().copy()))
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1])
+    assert np.array_equal(out[0][2], out[1][2]) and np.array_equal(out[1][2], out[1][3])
+    bad = faar.make_hparams(beta=4.0, step=1)                   # no tensor scale of the batch
+    pd, sd, xd, yd = sets[0]
+    with pytest.raises(faar.FaarError) as e:
+        faar.layer_step_host_nvfp4(ctx, lay.shape, bad, q[0][2], q[0][3], y_h, pd, sd, xd, yd, lay.V, lay.code, lay.scales,
+                                   lay.s_global, lay.m, lay.u, lay.loss, loss_h, lay.ws)
+    assert e.value.status == faar.ERR_INVALID_ARG
+
+
 @pytest.mark.parametrize("split", [1, 3, 100])
 @pytest.mark.parametrize("O,K,T", [(300, 1040, 600), (520, 784, 1300)])
 def test_half_width_tail_tiles_give_the_same_step(ctx, O, K, T, split):
