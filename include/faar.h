@@ -505,11 +505,19 @@ FAAR_API int faar_add(faar_ctx* ctx, int rows, int cols, const void* a, int64_t 
  * faar_attention_bwd: from dout (layout of out) to dq (layout of q), dk, dv (layout of k, v); out and lse are the
  * forward call's; dsum is scratch, [batch, n_heads, seq] floats.  No matrix of seq x seq values is stored; results
  * are reproducible (no atomics).  head_dim is 64 or 128; leading dimensions multiples of 8, bases 16-byte aligned. */
-/* head_dim 64 runs kernels that keep scores and probabilities in registers (mma.sync m16n8k16, one sweep over the
- * keys with a running maximum); head_dim 128 runs kernels that pass them through shared memory as 16 x 16 fragments
- * (two sweeps in the forward pass).  faar_tune_attention(ctx, 1) makes head_dim 64 take the second kind too
- * (0 = default again): the same mathematics, used to test both. */
+/* Which kernels head_dim 64 takes (head_dim 128 always takes the third kind):
+ *   0 (default): forward on the tcgen05 tensor cores (128-query tiles, scores and the per-tile output in tensor
+ *      memory, one query row per thread), backward as mode 2;
+ *   2: forward and backward with scores and probabilities in registers (mma.sync m16n8k16, one sweep over the
+ *      keys with a running maximum);
+ *   1: kernels that pass scores and probabilities through shared memory as 16 x 16 fragments (two sweeps in the
+ *      forward pass).
+ * The same mathematics in all three, used to test them against each other and the definition. */
 FAAR_API int faar_tune_attention(faar_ctx* ctx, int mode);
+/* The tcgen05 attention kernel bounds its barrier waits like the GEMM kernels; a wait that gave up is recorded in
+ * a status word of the library, which this call reads and clears (after the caller has synchronised the stream):
+ * FAAR_ERR_TIMEOUT with the raw code in detail_out (host, nullable), else FAAR_OK. */
+FAAR_API int faar_attention_status(faar_ctx* ctx, uint32_t* detail_out);
 FAAR_API int faar_attention_fwd(faar_ctx* ctx, int batch, int seq, int n_heads, int n_kv_heads, int head_dim, const void* q,
                                 int64_t ldq, const void* k, const void* v, int64_t ldkv, void* out, int64_t ldo, float* lse);
 FAAR_API int faar_attention_bwd(faar_ctx* ctx, int batch, int seq, int n_heads, int n_kv_heads, int head_dim, const void* q,

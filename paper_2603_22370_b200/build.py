@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfaar.so")
 LIB_DEBUG = os.path.join(HERE, "libfaar_debug.so")     # -DFAAR_DEBUG: epilogue stores checked against tensor extents
-SOURCES = ["faar_api.cu", "faar_elementwise.cu", "faar_gemm.cu", "faar_static_scratch.cu", "faar_align.cu", "faar_glue.cu", "faar_fp4_gemm.cu", "faar_attention.cu"]
+SOURCES = ["faar_api.cu", "faar_elementwise.cu", "faar_gemm.cu", "faar_static_scratch.cu", "faar_align.cu", "faar_glue.cu", "faar_fp4_gemm.cu", "faar_attention.cu", "faar_attention_tc.cu"]
 
 
 def _nvcc() -> str:

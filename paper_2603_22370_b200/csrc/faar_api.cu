@@ -388,8 +388,18 @@ int faar_tune_wide_tiles(faar_ctx* ctx, int mode) {
   return FAAR_OK;
 }
 
+int faar_attention_status(faar_ctx* ctx, uint32_t* detail_out) {
+  if (!ctx) return FAAR_ERR_INVALID_ARG;
+  FAAR_DEVICE_GUARD(ctx);
+  uint32_t code = 0;
+  int e = faar_attention_tc_status(&code);
+  if (detail_out) *detail_out = code;
+  if (e) return cuda_fail(ctx, e);
+  return code ? FAAR_ERR_TIMEOUT : FAAR_OK;
+}
+
 int faar_tune_attention(faar_ctx* ctx, int mode) {
-  if (!ctx || (mode != 0 && mode != 1)) return FAAR_ERR_INVALID_ARG;
+  if (!ctx || mode < 0 || mode > 2) return FAAR_ERR_INVALID_ARG;
   ctx->tune_attention_fragments = mode;
   return FAAR_OK;
 }

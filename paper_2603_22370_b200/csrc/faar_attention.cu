@@ -826,12 +826,15 @@ int launch_fwd(faar_ctx* ctx, const AttnParams& p) {
   cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, fwd_smem<D>());
   if (e != cudaSuccess) return (int)e;
   dim3 grid((p.S + AT - 1) / AT, p.H, p.B);
-  if (D == HD && !ctx->tune_attention_fragments) {
+  if (D == HD && ctx->tune_attention_fragments != 1) {
     e = cudaFuncSetAttribute(attn_fwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FWD64_SMEM);
     if (e != cudaSuccess) return (int)e;
   }
   faar_prof_scope ps(ctx, FAAR_K_ATTENTION);
-  if (D == HD && !ctx->tune_attention_fragments)
+  if (D == HD && ctx->tune_attention_fragments == 0)
+    return faar_launch_attention_fwd64_tc(ctx, p.B, p.S, p.H, p.Hkv, p.q, p.ldq, p.k, p.v, p.ldk, p.out, p.ldo, p.lse,
+                                          p.scale_log2);
+  if (D == HD && ctx->tune_attention_fragments == 2)
     attn_fwd64_kernel<<<dim3((p.S + FQ - 1) / FQ, p.H, p.B), FWD_THREADS, FWD64_SMEM, ctx->stream>>>(p);
   else
     attn_fwd_kernel<D><<<grid, ATT_THREADS, fwd_smem<D>(), ctx->stream>>>(p);
@@ -851,7 +854,7 @@ int launch_bwd(faar_ctx* ctx, const AttnParams& p, float* dsum) {
   if (blocks > (long long)ctx->num_sms * 16) blocks = (long long)ctx->num_sms * 16;
   attn_dsum_kernel<D><<<(int)blocks, ATT_THREADS, 0, ctx->stream>>>(p, dsum);
   const int tiles = (p.S + AT - 1) / AT;
-  if (D == HD && !ctx->tune_attention_fragments) {
+  if (D == HD && ctx->tune_attention_fragments != 1) {
     attn_dkv64_kernel<<<dim3(tiles, p.Hkv, p.B), BWD_THREADS, BWD64_SMEM, ctx->stream>>>(p);
     attn_dq64_kernel<<<dim3(tiles, p.H, p.B), BWD_THREADS, BWD64_SMEM, ctx->stream>>>(p);
     return (int)cudaGetLastError();

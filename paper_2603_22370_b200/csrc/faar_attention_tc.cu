@@ -1,0 +1,347 @@
+// Causal attention forward for head_dim 64 on the tcgen05 tensor cores (sm_100a).
+//
+// One CTA takes 128 queries of one head and sweeps the keys in tiles of 64 (one sweep, running maximum):
+//   S   = Q K_j^T       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 FP32 columns of tensor memory
+//   P_j = 2^(c S - m)   four warps, one query row per thread (its tensor-memory lane): no shuffles; the row
+//                       goes to shared memory as BF16 in the 128-byte-swizzled layout an A operand has
+//   O_j = P_j V_j       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 more columns; V_j is read as it lies in
+//                       memory (keys as rows: a B operand with its N index contiguous)
+//   O   = O * 2^(m_old - m) + O_j   in registers of the row's thread
+// Q, K_j, V_j arrive by TMA (two stages for K and V).  A fifth warp's lane 0 issues every copy and every MMA.
+// Per tile the chain S -> softmax -> P V -> accumulate is serial within a CTA; two CTAs per SM overlap theirs.
+// Rows of a query tile beyond the sequence end compute on whatever rows follow in memory (or zeros past the
+// tensor) and are not stored; keys beyond the end are masked.
+// Every barrier wait is bounded; a wait that gives up records a code in a status word of this module (read by
+// faar_attention_status), raises the CTA's abort flag and all roles leave.
+#include <cuda.h>
+
+#include "faar_internal.cuh"
+
+namespace {
+
+constexpr int QT = 128, KT = 64, HD = 64;
+constexpr int Q_BYTES = QT * HD * 2, KV_BYTES = KT * HD * 2, P_BYTES = QT * KT * 2;
+constexpr int OFF_K = Q_BYTES, OFF_V = OFF_K + 2 * KV_BYTES, OFF_P = OFF_V + 2 * KV_BYTES, OFF_CTL = OFF_P + P_BYTES;
+constexpr int CTL = 256;
+constexpr int SMEM = OFF_CTL + CTL + 1024;
+constexpr int THREADS = 160;
+constexpr int TMEM_COLS = 128;                     // S: columns 0..63, O_j: 64..127
+constexpr unsigned long long LIMIT_NS = 2000000000ull;
+
+__device__ uint32_t g_attn_status;                 // 0 = no wait has given up since the last read-and-clear
+
+struct TcParams {
+  __nv_bfloat16* out; float* lse;
+  long long ldo;
+  int S, H, Hkv;
+  float scale_log2;
+};
+
+__device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void bar_init(uint32_t b, uint32_t n) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(b), "r"(n)); }
+__device__ __forceinline__ void bar_arrive(uint32_t b) { asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(b) : "memory"); }
+__device__ __forceinline__ void bar_expect(uint32_t b, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t bar_try(uint32_t b, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(b), "r"(parity) : "memory");
+  return ok;
+}
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __noinline__ bool bar_wait_slow(uint32_t b, uint32_t parity, volatile int* abort_flag, uint32_t code) {
+  const unsigned long long t0 = now_ns();
+  for (uint32_t spin = 1;; ++spin) {
+    if (bar_try(b, parity)) return true;
+    if ((spin & 0xFF) == 0) {
+      if (*abort_flag) return false;
+      if (now_ns() - t0 > LIMIT_NS) { atomicCAS(&g_attn_status, 0u, code); *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ bool bar_wait(uint32_t b, uint32_t parity, volatile int* abort_flag, uint32_t code) {
+  return bar_try(b, parity) ? true : bar_wait_slow(b, parity, abort_flag, code);
+}
+__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Operand with the contraction index contiguous: rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t desc_k_major(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+// Operand with its N index contiguous (64 of them = one 128-byte row per contraction index): groups of 8
+// contraction indices 1024 B apart; a single 64-wide group along N, so the leading offset is not used.
+__device__ __forceinline__ uint64_t desc_n_major(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)(8192 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// D = F32, A = B = BF16, M = 128, N = 64; bit 16: B has its N index contiguous.
+__device__ __forceinline__ uint32_t idesc(int b_n_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_n_major << 16) | ((uint32_t)(KT >> 3) << 17) | ((uint32_t)(QT >> 4) << 24);
+}
+__device__ __forceinline__ void mma(uint32_t d, uint64_t da, uint64_t db, uint32_t id, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d), "l"(da), "l"(db), "r"(id), "r"(acc) : "memory");
+}
+// 32 consecutive FP32 columns of this thread's tensor-memory lane
+__device__ __forceinline__ void ld32(uint32_t taddr, float (&r)[32]) {
+  uint32_t u[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,"
+      "%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]), "=r"(u[9]),
+        "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]), "=r"(u[17]), "=r"(u[18]),
+        "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]),
+        "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(THREADS, 2)
+attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                     const __grid_constant__ CUtensorMap tmV, const TcParams p) {
+  extern __shared__ uint8_t raw[];
+  const uint32_t base = (s32(raw) + 1023u) & ~1023u;
+  uint8_t* smem = raw + (base - s32(raw));
+  const uint32_t ctl = base + OFF_CTL;
+  const uint32_t bar_q = ctl, bar_s = ctl + 40, bar_sfree = ctl + 48, bar_p = ctl + 56, bar_o = ctl + 64, bar_ofree = ctl + 72;
+  auto kfull = [&](int s) { return ctl + 8u + 8u * s; };
+  auto vfull = [&](int s) { return ctl + 24u + 8u * s; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_CTL + 80);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_CTL + 84);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;       // longest tiles first
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.H / p.Hkv);
+  const long long seq0 = (long long)b * p.S;
+  const int q0 = qt * QT;
+  const int last_q = min(q0 + QT, p.S) - 1;
+  const int n_kt = last_q / KT + 1;                          // key tiles that some query of this tile sees
+
+  if (threadIdx.x == 0) {
+    bar_init(bar_q, 1);
+    for (int s = 0; s < 2; ++s) { bar_init(kfull(s), 1); bar_init(vfull(s), 1); }
+    bar_init(bar_s, 1); bar_init(bar_o, 1);
+    bar_init(bar_sfree, 128); bar_init(bar_ofree, 128); bar_init(bar_p, 128);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(const_cast<uint32_t*>(tmem_slot))),
+                 "r"((uint32_t)TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t sQ = base, sP = base + OFF_P;
+  auto sK = [&](int s) { return base + OFF_K + (uint32_t)s * KV_BYTES; };
+  auto sV = [&](int s) { return base + OFF_V + (uint32_t)s * KV_BYTES; };
+
+  if (warp == 4) {
+    // ---------------- copies and MMAs: one thread ----------------
+    if (lane == 0) {
+      auto load_k = [&](int j) { bar_expect(kfull(j & 1), KV_BYTES); tma_2d(sK(j & 1), &tmK, g * HD, (int)(seq0 + (long long)j * KT), kfull(j & 1)); };
+      auto load_v = [&](int j) { bar_expect(vfull(j & 1), KV_BYTES); tma_2d(sV(j & 1), &tmV, g * HD, (int)(seq0 + (long long)j * KT), vfull(j & 1)); };
+      bar_expect(bar_q, Q_BYTES);
+      tma_2d(sQ, &tmQ, h * HD, (int)(seq0 + q0), bar_q);
+      load_k(0); load_v(0);
+      if (n_kt > 1) { load_k(1); load_v(1); }
+      bool ok = bar_wait(bar_q, 0u, abort_flag, 0xA01u);
+      const uint32_t id_s = idesc(0), id_pv = idesc(1);
+      for (int j = 0; j < n_kt && ok; ++j) {
+        const int st = j & 1;
+        const uint32_t ph = (uint32_t)((j >> 1) & 1);
+        ok = bar_wait(kfull(st), ph, abort_flag, 0xA10u | st);
+        if (ok && j > 0) ok = bar_wait(bar_sfree, (uint32_t)((j - 1) & 1), abort_flag, 0xA20u);
+        if (!ok) break;
+        fence_after();
+        {
+          const uint64_t da = desc_k_major(sQ), db = desc_k_major(sK(st));
+#pragma unroll
+          for (int k = 0; k < HD / 16; ++k) mma(tmem, da + 2u * k, db + 2u * k, id_s, k != 0 ? 1u : 0u);
+        }
+        commit(bar_s);
+        // P_j written: S_j has been read, so its K stage is free; S_j followed P V_{j-1} on the tensor pipe, so
+        // that product is complete too and its V stage is free
+        ok = bar_wait(bar_p, (uint32_t)(j & 1), abort_flag, 0xA30u);
+        if (!ok) break;
+        if (j + 2 < n_kt) load_k(j + 2);
+        if (j >= 1 && j + 1 < n_kt) load_v(j + 1);
+        ok = bar_wait(vfull(st), ph, abort_flag, 0xA40u | st);
+        if (ok && j > 0) ok = bar_wait(bar_ofree, (uint32_t)((j - 1) & 1), abort_flag, 0xA50u);
+        if (!ok) break;
+        fence_after();
+        {
+          const uint64_t da = desc_k_major(sP), db = desc_n_major(sV(st));
+#pragma unroll
+          for (int k = 0; k < KT / 16; ++k) mma(tmem + 64u, da + 2u * k, db + 128u * k, id_pv, k != 0 ? 1u : 0u);
+        }
+        commit(bar_o);
+      }
+      if (!ok) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) {} }   // copies in flight
+    }
+  } else {
+    // ---------------- softmax and accumulation: thread = query row = tensor-memory lane ----------------
+    const int row = 32 * warp + lane;
+    const int qi = q0 + row;
+    const uint32_t t_s = tmem + ((uint32_t)(32 * warp) << 16), t_o = t_s + 64u;
+    float o_acc[HD];
+#pragma unroll
+    for (int i = 0; i < HD; ++i) o_acc[i] = 0.f;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    auto fold = [&]() {                                       // o_acc += O_j
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float t[32];
+        ld32(t_o + 32u * half, t);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o_acc[32 * half + i] += t[i];
+      }
+    };
+    for (int j = 0; j < n_kt; ++j) {
+      const int k0 = j * KT;
+      ok = bar_wait(bar_s, (uint32_t)(j & 1), abort_flag, 0xB10u);
+      if (ok && j > 0) ok = bar_wait(bar_o, (uint32_t)((j - 1) & 1), abort_flag, 0xB20u);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      fence_after();
+      if (j > 0) {
+        fold();                                               // still relative to the maximum of tile j - 1
+        fence_before();
+        bar_arrive(bar_ofree);
+      }
+      float s[KT];
+      {
+        float t[32];
+        ld32(t_s, t);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) s[i] = t[i];
+        ld32(t_s + 32u, t);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) s[32 + i] = t[i];
+      }
+      fence_before();
+      bar_arrive(bar_sfree);
+      if (k0 + KT - 1 > q0 || k0 + KT > p.S) {                // the tile crosses some row's diagonal, or the sequence end
+#pragma unroll
+        for (int i = 0; i < KT; ++i)
+          if (!(k0 + i <= qi && k0 + i < p.S)) s[i] = -INFINITY;
+      }
+      float mx = s[0];
+#pragma unroll
+      for (int i = 1; i < KT; ++i) mx = fmaxf(mx, s[i]);
+      const float m_new = fmaxf(m, mx * p.scale_log2);
+      const float ref = m_new == -INFINITY ? 0.f : m_new;     // a row beyond the sequence may have seen no key
+      const float alpha = exp2f(m - ref);
+      float sum = 0.f;
+      uint8_t* prow = smem + OFF_P + row * 128;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        float e[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { e[i] = exp2f(fmaf(s[8 * c + i], p.scale_log2, -ref)); sum += e[i]; }
+        *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
+            make_uint4(pack2(e[0], e[1]), pack2(e[2], e[3]), pack2(e[4], e[5]), pack2(e[6], e[7]));
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this row of P, visible to the tensor cores
+      bar_arrive(bar_p);
+      l = l * alpha + sum;
+#pragma unroll
+      for (int i = 0; i < HD; ++i) o_acc[i] *= alpha;
+      m = m_new;
+    }
+    if (ok) {
+      ok = bar_wait(bar_o, (uint32_t)((n_kt - 1) & 1), abort_flag, 0xB30u);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      fence_after();
+      fold();
+      if (qi < p.S) {
+        const float inv = l > 0.f ? 1.0f / l : 0.f;
+        uint4* dst = reinterpret_cast<uint4*>(p.out + (seq0 + qi) * p.ldo + h * HD);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          dst[c] = make_uint4(pack2(o_acc[8 * c] * inv, o_acc[8 * c + 1] * inv), pack2(o_acc[8 * c + 2] * inv, o_acc[8 * c + 3] * inv),
+                              pack2(o_acc[8 * c + 4] * inv, o_acc[8 * c + 5] * inv), pack2(o_acc[8 * c + 6] * inv, o_acc[8 * c + 7] * inv));
+        p.lse[((long long)b * p.H + h) * p.S + qi] = m + log2f(l);
+      }
+    }
+  }
+  __syncwarp();
+  fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// [rows, cols] BF16, row stride ld elements: boxes of 64 columns x box_rows rows, 128-byte swizzle
+int head_map(faar_ctx* ctx, CUtensorMap* map, const void* ptr, long long rows, int cols, long long ld, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)HD, (cuuint32_t)box_rows};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = reinterpret_cast<EncodeFn>(ctx->encode_tiled)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims,
+                                                             strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : (int)cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+int faar_launch_attention_fwd64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, const void* q, int64_t ldq, const void* k,
+                                   const void* v, int64_t ldk, void* out, int64_t ldo, float* lse, float scale_log2) {
+  static_assert(2 * SMEM <= 227 * 1024, "two CTAs per SM");
+  const long long T = (long long)B * S;
+  if (T > 0x7FFFFFFFll) return (int)cudaErrorInvalidValue;
+  CUtensorMap tmQ, tmK, tmV;
+  int e = head_map(ctx, &tmQ, q, T, H * HD, ldq, QT);
+  if (!e) e = head_map(ctx, &tmK, k, T, Hkv * HD, ldk, KT);
+  if (!e) e = head_map(ctx, &tmV, v, T, Hkv * HD, ldk, KT);
+  if (e) return e;
+  cudaError_t ce = cudaFuncSetAttribute(attn_fwd64_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  if (ce != cudaSuccess) return (int)ce;
+  TcParams p;
+  p.out = reinterpret_cast<__nv_bfloat16*>(out); p.lse = lse; p.ldo = ldo; p.S = S; p.H = H; p.Hkv = Hkv;
+  p.scale_log2 = scale_log2;
+  attn_fwd64_tc_kernel<<<dim3((S + QT - 1) / QT, H, B), THREADS, SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
+  return (int)cudaGetLastError();
+}
+
+// Reads and clears the status word of this module (synchronous copy: call after the stream has been synchronised).
+int faar_attention_tc_status(uint32_t* code_out) {
+  uint32_t v = 0, zero = 0;
+  cudaError_t e = cudaMemcpyFromSymbol(&v, g_attn_status, sizeof(v));
+  if (e == cudaSuccess && v) e = cudaMemcpyToSymbol(g_attn_status, &zero, sizeof(zero));
+  *code_out = v;
+  return (int)e;
+}

@@ -20,7 +20,7 @@ struct faar_ctx {
   int tune_bn;                            // 0 = choose the GEMM tile width automatically
   int tune_tail;                          // -1 = choose the tail split automatically, else columns to split
   int tune_wide;                          // 1 = 256 x 512 GEMM tiles wherever the shape allows; -1 (default), 0 = never
-  int tune_attention_fragments;           // 1 = head_dim 64 attention also runs the shared-memory fragment kernels
+  int tune_attention_fragments;           // head_dim 64 attention: 0 = tcgen05 forward + mma.sync backward, 2 = mma.sync both, 1 = the shared-memory fragment kernels
   int last_gemm_bn, last_gemm_pairs, last_gemm_split;   // what the last GEMM launch used
   // CTA pairs this context's device can hold at once, per GEMM kernel instantiation (0 = not asked yet)
   int gemm_max_pairs[FAAR_GEMM_VARIANTS];
@@ -87,6 +87,9 @@ int faar_launch_softquant_init(faar_ctx*, const faar_shape*, const void* W, floa
                                uint8_t* scales, float* s_global_out, uint8_t* code, float* V,
                                unsigned long long* amax_word);
 int faar_launch_nvfp4_expand(faar_ctx*, int rows, int K, const uint8_t* packed, const uint8_t* scales, void* out, int64_t ld);
+int faar_launch_attention_fwd64_tc(faar_ctx*, int B, int S, int H, int Hkv, const void* q, int64_t ldq, const void* k,
+                                   const void* v, int64_t ldk, void* out, int64_t ldo, float* lse, float scale_log2);
+int faar_attention_tc_status(uint32_t* code_out);
 int faar_launch_softquant_eval(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta,
                                float* W_soft, float* h, __nv_bfloat16* W_soft_bf16,

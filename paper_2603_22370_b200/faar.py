@@ -66,6 +66,7 @@ SIGNATURES = {
     "faar_embedding": (_I, [_P, _I, _I, _I, _P, _L, _P, _P, _L]),
     "faar_add": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L]),
     "faar_tune_attention": (_I, [_P, _I]),
+    "faar_attention_status": (_I, [_P, _P]),
     "faar_tune_wide_tiles": (_I, [_P, _I]),
     "faar_attention_fwd": (_I, [_P, _I, _I, _I, _I, _I, _P, _L, _P, _P, _L, _P, _L, _P]),
     "faar_attention_bwd": (_I, [_P, _I, _I, _I, _I, _I, _P, _L, _P, _P, _L, _P, _P, _L, _P, _P, _P, _P, _P]),
@@ -302,8 +303,15 @@ def tune_wide_tiles(ctx, mode: int):
     _check(lib().faar_tune_wide_tiles(ctx._h, mode), "faar_tune_wide_tiles")
 
 
+def attention_status(ctx):
+    """Raises FaarError(TIMEOUT) if a wait of the tcgen05 attention kernel gave up (call after a synchronise)."""
+    code = C.c_uint32(0)
+    _check(lib().faar_attention_status(ctx._h, C.byref(code)), f"faar_attention_status (code {code.value:#x})")
+
+
 def tune_attention(ctx, mode: int):
-    """1: head_dim 64 also runs the shared-memory fragment kernels (as head_dim 128 does); 0: the default."""
+    """head_dim 64: 0 = tcgen05 forward + register-resident backward (default), 2 = register-resident kernels for
+    both, 1 = the shared-memory fragment kernels (as head_dim 128 always takes)."""
     _check(lib().faar_tune_attention(ctx._h, mode), "faar_tune_attention")
 
 

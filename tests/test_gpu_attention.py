@@ -29,12 +29,13 @@ def padded(a, ld, fill=9.0):
     return t
 
 
-@pytest.mark.parametrize("fragments", [0, 1])
+@pytest.mark.parametrize("fragments", [0, 1, 2])
 @pytest.mark.parametrize("B,S,H,HKV,D", [(2, 100, 4, 2, 64), (1, 64, 2, 2, 64), (3, 7, 2, 1, 64), (1, 200, 4, 1, 128),
                                          (2, 129, 8, 2, 64), (1, 321, 4, 4, 64)])
 def test_attention_forward_and_backward_match_the_oracle(ctx, B, S, H, HKV, D, fragments):
-    """fragments = 0: the default kernels (head_dim 64 keeps scores in registers); 1: head_dim 64 through the
-    shared-memory fragment kernels that head_dim 128 always uses."""
+    """fragments = 0: the default kernels (head_dim 64: forward on tcgen05, backward with scores in registers);
+    2: head_dim 64 with scores in registers forward and backward; 1: head_dim 64 through the shared-memory fragment
+    kernels that head_dim 128 always uses."""
     if fragments and D != 64:
         pytest.skip("head_dim 128 has one kind of kernel")
     faar.tune_attention(ctx, fragments)
@@ -57,6 +58,7 @@ def _attention_case(ctx, B, S, H, HKV, D):
     lse = torch.zeros((B, H, S), dtype=torch.float32, device=DEV)
     faar.attention_fwd(ctx, B, S, H, HKV, D, Q, ldq, K, V, ldk, O, ldq, lse)
     torch.cuda.synchronize()
+    faar.attention_status(ctx)
     out_o, P = so.attention(q, k, v, B, S, H, HKV, D)
     got = host(O[:, :H * D]).astype(np.float64)
     assert rel_l2(got, out_o) <= 6e-3 and max_rel_to_peak(got, out_o) <= 1e-2
