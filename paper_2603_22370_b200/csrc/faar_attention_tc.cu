@@ -7,8 +7,9 @@
 //   O_j = P_j V_j       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 more columns; V_j is read as it lies in
 //                       memory (keys as rows: a B operand with its N index contiguous)
 //   O   = O * 2^(m_old - m) + O_j   in registers of the row's thread
-// Q, K_j, V_j arrive by TMA (two stages for K and V).  A fifth warp's lane 0 issues every copy and every MMA.
-// Per tile the chain S -> softmax -> P V -> accumulate is serial within a CTA; two CTAs per SM overlap theirs.
+// Q, K_j, V_j arrive by TMA (two stages for K and V).  A fifth warp's lane 0 issues every copy and every MMA; the
+// scores have two buffers in tensor memory, so S of tile j + 1 is formed while the warps work on tile j, and two
+// CTAs per SM overlap what remains serial (softmax -> P V -> accumulate).
 // Rows of a query tile beyond the sequence end compute on whatever rows follow in memory (or zeros past the
 // tensor) and are not stored; keys beyond the end are masked.
 // Every barrier wait is bounded; a wait that gives up records a code in a status word of this module (read by
@@ -21,11 +22,11 @@ namespace {
 
 constexpr int QT = 128, KT = 64, HD = 64;
 constexpr int Q_BYTES = QT * HD * 2, KV_BYTES = KT * HD * 2, P_BYTES = QT * KT * 2;
-constexpr int OFF_K = Q_BYTES, OFF_V = OFF_K + 2 * KV_BYTES, OFF_P = OFF_V + 2 * KV_BYTES, OFF_CTL = OFF_P + P_BYTES;
+constexpr int OFF_K = Q_BYTES, OFF_V = OFF_K + 2 * KV_BYTES, OFF_P = OFF_V + 2 * KV_BYTES, OFF_CTL = OFF_P + 2 * P_BYTES;
 constexpr int CTL = 256;
 constexpr int SMEM = OFF_CTL + CTL + 1024;
 constexpr int THREADS = 160;
-constexpr int TMEM_COLS = 128;                     // S: columns 0..63, O_j: 64..127
+constexpr int TMEM_COLS = 256;                     // S of even / odd tiles: columns 0..63 / 64..127, O_j: 128..191
 constexpr unsigned long long LIMIT_NS = 2000000000ull;
 
 __device__ uint32_t g_attn_status;                 // 0 = no wait has given up since the last read-and-clear
@@ -122,11 +123,13 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   const uint32_t base = (s32(raw) + 1023u) & ~1023u;
   uint8_t* smem = raw + (base - s32(raw));
   const uint32_t ctl = base + OFF_CTL;
-  const uint32_t bar_q = ctl, bar_s = ctl + 40, bar_sfree = ctl + 48, bar_p = ctl + 56, bar_o = ctl + 64, bar_ofree = ctl + 72;
+  const uint32_t bar_q = ctl, bar_p = ctl + 72, bar_o = ctl + 80, bar_ofree = ctl + 88;
   auto kfull = [&](int s) { return ctl + 8u + 8u * s; };
   auto vfull = [&](int s) { return ctl + 24u + 8u * s; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_CTL + 80);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_CTL + 84);
+  auto bar_s = [&](int s) { return ctl + 40u + 8u * s; };         // scores of a tile in buffer s are complete
+  auto bar_sfree = [&](int s) { return ctl + 56u + 8u * s; };     // ... have been read by all 128 rows
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_CTL + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_CTL + 100);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;       // longest tiles first
@@ -140,8 +143,8 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   if (threadIdx.x == 0) {
     bar_init(bar_q, 1);
     for (int s = 0; s < 2; ++s) { bar_init(kfull(s), 1); bar_init(vfull(s), 1); }
-    bar_init(bar_s, 1); bar_init(bar_o, 1);
-    bar_init(bar_sfree, 128); bar_init(bar_ofree, 128); bar_init(bar_p, 128);
+    for (int s = 0; s < 2; ++s) { bar_init(bar_s(s), 1); bar_init(bar_sfree(s), 128); }
+    bar_init(bar_o, 1); bar_init(bar_ofree, 128); bar_init(bar_p, 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -155,7 +158,8 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   __syncthreads();
   fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t sQ = base, sP = base + OFF_P;
+  const uint32_t sQ = base;
+  auto sP = [&](int s) { return base + OFF_P + (uint32_t)s * P_BYTES; };
   auto sK = [&](int s) { return base + OFF_K + (uint32_t)s * KV_BYTES; };
   auto sV = [&](int s) { return base + OFF_V + (uint32_t)s * KV_BYTES; };
 
@@ -170,33 +174,41 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       if (n_kt > 1) { load_k(1); load_v(1); }
       bool ok = bar_wait(bar_q, 0u, abort_flag, 0xA01u);
       const uint32_t id_s = idesc(0), id_pv = idesc(1);
+      // S of tile j into score buffer j & 1.  The scores of tile j + 1 are issued before this thread waits for the
+      // probabilities of tile j, so the tensor cores form them while the four warps work on tile j.
+      auto issue_s = [&](int j) {
+        const uint64_t da = desc_k_major(sQ), db = desc_k_major(sK(j & 1));
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) mma(tmem + 64u * (uint32_t)(j & 1), da + 2u * k, db + 2u * k, id_s, k != 0 ? 1u : 0u);
+        commit(bar_s(j & 1));
+      };
+      if (ok) ok = bar_wait(kfull(0), 0u, abort_flag, 0xA10u);
+      if (ok) { fence_after(); issue_s(0); }
       for (int j = 0; j < n_kt && ok; ++j) {
         const int st = j & 1;
         const uint32_t ph = (uint32_t)((j >> 1) & 1);
-        ok = bar_wait(kfull(st), ph, abort_flag, 0xA10u | st);
-        if (ok && j > 0) ok = bar_wait(bar_sfree, (uint32_t)((j - 1) & 1), abort_flag, 0xA20u);
-        if (!ok) break;
-        fence_after();
-        {
-          const uint64_t da = desc_k_major(sQ), db = desc_k_major(sK(st));
-#pragma unroll
-          for (int k = 0; k < HD / 16; ++k) mma(tmem, da + 2u * k, db + 2u * k, id_s, k != 0 ? 1u : 0u);
+        if (j + 1 < n_kt) {
+          ok = bar_wait(kfull((j + 1) & 1), (uint32_t)(((j + 1) >> 1) & 1), abort_flag, 0xA10u | ((j + 1) & 1));
+          // its score buffer last held tile j - 1
+          if (ok && j >= 1) ok = bar_wait(bar_sfree((j + 1) & 1), (uint32_t)(((j - 1) >> 1) & 1), abort_flag, 0xA20u);
+          if (!ok) break;
+          fence_after();
+          issue_s(j + 1);
         }
-        commit(bar_s);
-        // P_j written: S_j has been read, so its K stage is free; S_j followed P V_{j-1} on the tensor pipe, so
-        // that product is complete too and its V stage is free
+        // P_j written (into P buffer j & 1): S_j has been read, so its K stage is free
         ok = bar_wait(bar_p, (uint32_t)(j & 1), abort_flag, 0xA30u);
         if (!ok) break;
         if (j + 2 < n_kt) load_k(j + 2);
-        if (j >= 1 && j + 1 < n_kt) load_v(j + 1);
         ok = bar_wait(vfull(st), ph, abort_flag, 0xA40u | st);
+        // O_{j-1} folded by every row: P V_{j-1} is complete, its output columns and its V stage are free
         if (ok && j > 0) ok = bar_wait(bar_ofree, (uint32_t)((j - 1) & 1), abort_flag, 0xA50u);
         if (!ok) break;
+        if (j >= 1 && j + 1 < n_kt) load_v(j + 1);
         fence_after();
         {
-          const uint64_t da = desc_k_major(sP), db = desc_n_major(sV(st));
+          const uint64_t da = desc_k_major(sP(st)), db = desc_n_major(sV(st));
 #pragma unroll
-          for (int k = 0; k < KT / 16; ++k) mma(tmem + 64u, da + 2u * k, db + 128u * k, id_pv, k != 0 ? 1u : 0u);
+          for (int k = 0; k < KT / 16; ++k) mma(tmem + 128u, da + 2u * k, db + 128u * k, id_pv, k != 0 ? 1u : 0u);
         }
         commit(bar_o);
       }
@@ -206,7 +218,7 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     // ---------------- softmax and accumulation: thread = query row = tensor-memory lane ----------------
     const int row = 32 * warp + lane;
     const int qi = q0 + row;
-    const uint32_t t_s = tmem + ((uint32_t)(32 * warp) << 16), t_o = t_s + 64u;
+    const uint32_t t_lane = tmem + ((uint32_t)(32 * warp) << 16), t_o = t_lane + 128u;
     float o_acc[HD];
 #pragma unroll
     for (int i = 0; i < HD; ++i) o_acc[i] = 0.f;
@@ -223,15 +235,10 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     };
     for (int j = 0; j < n_kt; ++j) {
       const int k0 = j * KT;
-      ok = bar_wait(bar_s, (uint32_t)(j & 1), abort_flag, 0xB10u);
-      if (ok && j > 0) ok = bar_wait(bar_o, (uint32_t)((j - 1) & 1), abort_flag, 0xB20u);
+      const uint32_t t_s = t_lane + 64u * (uint32_t)(j & 1);
+      ok = bar_wait(bar_s(j & 1), (uint32_t)((j >> 1) & 1), abort_flag, 0xB10u);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       fence_after();
-      if (j > 0) {
-        fold();                                               // still relative to the maximum of tile j - 1
-        fence_before();
-        bar_arrive(bar_ofree);
-      }
       float s[KT];
       {
         float t[32];
@@ -243,7 +250,7 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         for (int i = 0; i < 32; ++i) s[32 + i] = t[i];
       }
       fence_before();
-      bar_arrive(bar_sfree);
+      bar_arrive(bar_sfree(j & 1));
       if (k0 + KT - 1 > q0 || k0 + KT > p.S) {                // the tile crosses some row's diagonal, or the sequence end
 #pragma unroll
         for (int i = 0; i < KT; ++i)
@@ -256,7 +263,7 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       const float ref = m_new == -INFINITY ? 0.f : m_new;     // a row beyond the sequence may have seen no key
       const float alpha = exp2f(m - ref);
       float sum = 0.f;
-      uint8_t* prow = smem + OFF_P + row * 128;
+      uint8_t* prow = smem + OFF_P + (j & 1) * P_BYTES + row * 128;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         float e[8];
@@ -267,6 +274,16 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this row of P, visible to the tensor cores
       bar_arrive(bar_p);
+      // the previous tile's P V has had the whole of this tile's softmax to finish: fold it in (still relative to
+      // the maximum of tile j - 1), then move everything to the new maximum
+      if (j > 0) {
+        ok = bar_wait(bar_o, (uint32_t)((j - 1) & 1), abort_flag, 0xB20u);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        fence_after();
+        fold();
+        fence_before();
+        bar_arrive(bar_ofree);
+      }
       l = l * alpha + sum;
 #pragma unroll
       for (int i = 0; i < HD; ++i) o_acc[i] *= alpha;
