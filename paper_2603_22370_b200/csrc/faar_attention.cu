@@ -854,6 +854,13 @@ int launch_bwd(faar_ctx* ctx, const AttnParams& p, float* dsum) {
   if (blocks > (long long)ctx->num_sms * 16) blocks = (long long)ctx->num_sms * 16;
   attn_dsum_kernel<D><<<(int)blocks, ATT_THREADS, 0, ctx->stream>>>(p, dsum);
   const int tiles = (p.S + AT - 1) / AT;
+  if (D == HD && ctx->tune_attention_fragments == 0) {
+    int le = faar_launch_attention_dkv64_tc(ctx, p.B, p.S, p.H, p.Hkv, p.q, p.ldq, p.k, p.v, p.ldk, p.dout, p.ldo, p.lse, dsum,
+                                            p.dk, p.dv, p.scale_log2);
+    if (le) return le;
+    return faar_launch_attention_dq64_tc(ctx, p.B, p.S, p.H, p.Hkv, p.q, p.ldq, p.k, p.v, p.ldk, p.dout, p.ldo, p.lse, dsum,
+                                         p.dq, p.scale_log2);
+  }
   if (D == HD && ctx->tune_attention_fragments != 1) {
     attn_dkv64_kernel<<<dim3(tiles, p.Hkv, p.B), BWD_THREADS, BWD64_SMEM, ctx->stream>>>(p);
     attn_dq64_kernel<<<dim3(tiles, p.H, p.B), BWD_THREADS, BWD64_SMEM, ctx->stream>>>(p);

@@ -316,6 +316,402 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   }
 }
 
+// ---- backward, dQ: one CTA per 128 queries of a head, sweeping the key tiles up to the diagonal ---------------
+//   S_j = Q K_j^T, dP_j = dO V_j^T     two MMAs into 64 + 64 columns of tensor memory
+//   dS_j = P_j (dP_j - delta) / sqrt(d), P_j = 2^(c S_j - lse)     one query row per thread, written as a BF16
+//                                                                   A operand into swizzled shared memory
+//   dQ += dS_j K_j                       third MMA, accumulating in 64 more columns over the whole sweep (K_j read
+//                                        as it lies in memory: keys as contraction rows, d contiguous)
+// The dQ product of tile j - 1 is issued after the score products of tile j, so it runs while the rows work on
+// tile j; K / V tiles come through three TMA stages.  Only the final dQ leaves tensor memory.
+constexpr int DQ_OFF_DO = Q_BYTES, DQ_OFF_KV = 2 * Q_BYTES, DQ_STAGE = 2 * KV_BYTES, DQ_STAGES = 3;
+constexpr int DQ_OFF_DS = DQ_OFF_KV + DQ_STAGES * DQ_STAGE, DQ_OFF_CTL = DQ_OFF_DS + P_BYTES;
+constexpr int DQ_SMEM = DQ_OFF_CTL + CTL + 1024;
+
+struct TcBwdParams {
+  const float* lse; const float* dsum;
+  __nv_bfloat16* dq; __nv_bfloat16* dk; __nv_bfloat16* dv;
+  long long ldq, ldk;
+  int S, H, Hkv;
+  float scale_log2, inv_sqrt_d;
+};
+
+__global__ void __launch_bounds__(THREADS, 2)
+attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
+                    const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const TcBwdParams p) {
+  extern __shared__ uint8_t raw[];
+  const uint32_t base = (s32(raw) + 1023u) & ~1023u;
+  uint8_t* smem = raw + (base - s32(raw));
+  const uint32_t ctl = base + DQ_OFF_CTL;
+  const uint32_t bar_qd = ctl, bar_s = ctl + 40, bar_sfree = ctl + 48, bar_ds = ctl + 56, bar_done = ctl + 64;
+  auto kvfull = [&](int s) { return ctl + 8u + 8u * s; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + DQ_OFF_CTL + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + DQ_OFF_CTL + 100);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.H / p.Hkv);
+  const long long seq0 = (long long)b * p.S;
+  const int q0 = qt * QT;
+  const int last_q = min(q0 + QT, p.S) - 1;
+  const int n_kt = last_q / KT + 1;
+
+  if (threadIdx.x == 0) {
+    bar_init(bar_qd, 1);
+    for (int s = 0; s < DQ_STAGES; ++s) bar_init(kvfull(s), 1);
+    bar_init(bar_s, 1); bar_init(bar_done, 1);
+    bar_init(bar_sfree, 128); bar_init(bar_ds, 128);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(const_cast<uint32_t*>(tmem_slot))),
+                 "r"((uint32_t)TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem = *tmem_slot;                         // S: columns 0..63, dP: 64..127, dQ: 128..191
+  const uint32_t sQ = base, sDO = base + DQ_OFF_DO, sDS = base + DQ_OFF_DS;
+  auto sK = [&](int s) { return base + DQ_OFF_KV + (uint32_t)s * DQ_STAGE; };
+  auto sV = [&](int s) { return sK(s) + KV_BYTES; };
+
+  if (warp == 4) {
+    if (lane == 0) {
+      auto load_kv = [&](int j) {
+        const int st = j % DQ_STAGES;
+        bar_expect(kvfull(st), 2 * KV_BYTES);
+        tma_2d(sK(st), &tmK, g * HD, (int)(seq0 + (long long)j * KT), kvfull(st));
+        tma_2d(sV(st), &tmV, g * HD, (int)(seq0 + (long long)j * KT), kvfull(st));
+      };
+      bar_expect(bar_qd, 2 * Q_BYTES);
+      tma_2d(sQ, &tmQ, h * HD, (int)(seq0 + q0), bar_qd);
+      tma_2d(sDO, &tmDO, h * HD, (int)(seq0 + q0), bar_qd);
+      load_kv(0);
+      if (n_kt > 1) load_kv(1);
+      bool ok = bar_wait(bar_qd, 0u, abort_flag, 0xC01u);
+      const uint32_t id_k = idesc(0), id_n = idesc(1);
+      auto issue_dq = [&](int j) {                            // dQ += dS_j K_j
+        const uint64_t da = desc_k_major(sDS), db = desc_n_major(sK(j % DQ_STAGES));
+#pragma unroll
+        for (int k = 0; k < KT / 16; ++k) mma(tmem + 128u, da + 2u * k, db + 128u * k, id_n, (j | k) != 0 ? 1u : 0u);
+        commit(bar_done);
+      };
+      for (int j = 0; j < n_kt && ok; ++j) {
+        const int st = j % DQ_STAGES;
+        if (j >= 1 && j + 1 < n_kt) {                         // stage of tile j + 1 last held tile j - 2
+          if (j >= 2) ok = bar_wait(bar_done, (uint32_t)((j - 2) & 1), abort_flag, 0xC10u);
+          if (!ok) break;
+          load_kv(j + 1);
+        }
+        ok = bar_wait(kvfull(st), (uint32_t)((j / DQ_STAGES) & 1), abort_flag, 0xC20u | st);
+        if (ok && j > 0) ok = bar_wait(bar_sfree, (uint32_t)((j - 1) & 1), abort_flag, 0xC30u);
+        if (!ok) break;
+        fence_after();
+        {
+          const uint64_t dq_ = desc_k_major(sQ), dk_ = desc_k_major(sK(st)), dd = desc_k_major(sDO), dv_ = desc_k_major(sV(st));
+#pragma unroll
+          for (int k = 0; k < HD / 16; ++k) mma(tmem, dq_ + 2u * k, dk_ + 2u * k, id_k, k != 0 ? 1u : 0u);
+#pragma unroll
+          for (int k = 0; k < HD / 16; ++k) mma(tmem + 64u, dd + 2u * k, dv_ + 2u * k, id_k, k != 0 ? 1u : 0u);
+        }
+        commit(bar_s);
+        if (j > 0) {
+          ok = bar_wait(bar_ds, (uint32_t)((j - 1) & 1), abort_flag, 0xC40u);
+          if (!ok) break;
+          fence_after();
+          issue_dq(j - 1);
+        }
+      }
+      if (ok) ok = bar_wait(bar_ds, (uint32_t)((n_kt - 1) & 1), abort_flag, 0xC50u);
+      if (ok) { fence_after(); issue_dq(n_kt - 1); }
+      if (!ok) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) {} }
+    }
+  } else {
+    const int row = 32 * warp + lane;
+    const int qi = q0 + row;
+    const uint32_t t_lane = tmem + ((uint32_t)(32 * warp) << 16);
+    const long long ro = ((long long)b * p.H + h) * p.S;
+    const float lse = qi < p.S ? p.lse[ro + qi] : 0.f;
+    const float nd = qi < p.S ? -p.dsum[ro + qi] * p.inv_sqrt_d : 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kt; ++j) {
+      const int k0 = j * KT;
+      ok = bar_wait(bar_s, (uint32_t)(j & 1), abort_flag, 0xD10u);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      fence_after();
+      float s[KT];
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {                  // P (dP - delta) / sqrt(d), 32 columns at a time
+        float t[32], d[32];
+        ld32(t_lane + 32u * half, t);
+        ld32(t_lane + 64u + 32u * half, d);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          float pr = exp2f(fmaf(t[i], p.scale_log2, -lse));
+          if (k0 + 32 * half + i > qi) pr = 0.f;               // above the diagonal (and beyond the sequence end)
+          s[32 * half + i] = pr * fmaf(d[i], p.inv_sqrt_d, nd);
+        }
+      }
+      fence_before();
+      bar_arrive(bar_sfree);
+      if (j > 0) {                                            // the dS buffer is free once dQ of tile j - 1 has run
+        ok = bar_wait(bar_done, (uint32_t)((j - 1) & 1), abort_flag, 0xD20u);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      }
+      uint8_t* prow = smem + DQ_OFF_DS + row * 128;
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
+            make_uint4(pack2(s[8 * c], s[8 * c + 1]), pack2(s[8 * c + 2], s[8 * c + 3]), pack2(s[8 * c + 4], s[8 * c + 5]),
+                       pack2(s[8 * c + 6], s[8 * c + 7]));
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      bar_arrive(bar_ds);
+    }
+    if (ok) {
+      ok = bar_wait(bar_done, (uint32_t)((n_kt - 1) & 1), abort_flag, 0xD30u);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      fence_after();
+      uint4* dst = reinterpret_cast<uint4*>(p.dq + (seq0 + qi) * p.ldq + h * HD);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float t[32];
+        ld32(t_lane + 128u + 32u * half, t);
+        if (qi < p.S) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            dst[4 * half + c] = make_uint4(pack2(t[8 * c], t[8 * c + 1]), pack2(t[8 * c + 2], t[8 * c + 3]),
+                                           pack2(t[8 * c + 4], t[8 * c + 5]), pack2(t[8 * c + 6], t[8 * c + 7]));
+        }
+      }
+    }
+  }
+  __syncwarp();
+  fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
+  }
+}
+
+// ---- backward, dK and dV: one CTA per 128 keys of a key / value head ------------------------------------------
+// The keys are the rows (tensor-memory lanes); the CTA sweeps the (head, 64-query tile) pairs that see them:
+//   S^T = K Q_i^T, dP^T = V dO_i^T          two MMAs into one of two pairs of 64-column buffers
+//   P^T = 2^(c S^T - lse_q), dS^T = P^T (dP^T - delta_q) / sqrt(d)    one key row per thread; both written as BF16
+//                                            A operands into one of two pairs of swizzled shared-memory buffers
+//   dV += P^T dO_i, dK += dS^T Q_i           two MMAs that accumulate in 64 + 64 columns over the whole sweep
+//                                            (dO_i and Q_i read as they lie in memory: queries as contraction rows)
+// One CTA per SM; the score products of item i + 1 are issued before this item's probabilities are awaited, Q / dO
+// tiles come through three TMA stages, lse and delta of a tile's 64 queries are staged in shared memory by the
+// row threads themselves.  Queries beyond the sequence end are masked (their rows hold the next sequence's data).
+constexpr int KV_OFF_V = Q_BYTES, KV_OFF_QD = 2 * Q_BYTES, KV_STAGE = 2 * KV_BYTES, KV_STAGES = 3;
+constexpr int KV_OFF_PT = KV_OFF_QD + KV_STAGES * KV_STAGE, KV_OFF_DST = KV_OFF_PT + 2 * P_BYTES;
+constexpr int KV_OFF_ROWV = KV_OFF_DST + 2 * P_BYTES, KV_OFF_CTL = KV_OFF_ROWV + 2 * 2 * KT * 4;
+constexpr int KV_SMEM = KV_OFF_CTL + CTL + 1024;
+constexpr int KV_TMEM = 512;                      // S^T: 0 / 64, dP^T: 128 / 192, dV: 256, dK: 320
+
+__global__ void __launch_bounds__(THREADS, 1)
+attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
+                     const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const TcBwdParams p) {
+  extern __shared__ uint8_t raw[];
+  const uint32_t base = (s32(raw) + 1023u) & ~1023u;
+  uint8_t* smem = raw + (base - s32(raw));
+  const uint32_t ctl = base + KV_OFF_CTL;
+  const uint32_t bar_kv = ctl;
+  auto qfull = [&](int s) { return ctl + 8u + 8u * s; };          // 3
+  auto bar_s = [&](int s) { return ctl + 32u + 8u * s; };         // 2: score buffers of an item are complete
+  auto bar_sfree = [&](int s) { return ctl + 48u + 8u * s; };     // 2: ... have been read by all 128 rows
+  auto bar_pds = [&](int s) { return ctl + 64u + 8u * s; };       // 2: P^T / dS^T buffers written
+  auto bar_done = [&](int s) { return ctl + 80u + 8u * s; };      // 2: the accumulating MMAs of an item have run
+  auto bar_rv = [&](int s) { return ctl + 104u + 8u * s; };       // 2: lse / delta of an item staged by all 128 rows
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + KV_OFF_CTL + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + KV_OFF_CTL + 100);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const int kt = blockIdx.x, g = blockIdx.y, b = blockIdx.z;       // the first key tiles see the most queries
+  const int rep = p.H / p.Hkv;
+  const long long seq0 = (long long)b * p.S;
+  const int k0 = kt * QT;
+  const int n_qt = (p.S + KT - 1) / KT;
+  const int qt0 = k0 / KT;                                         // first query tile that sees a key of this tile
+  const int per_head = n_qt - qt0;
+  const int n_it = rep * per_head;
+
+  if (threadIdx.x == 0) {
+    bar_init(bar_kv, 1);
+    for (int s = 0; s < KV_STAGES; ++s) bar_init(qfull(s), 1);
+    for (int s = 0; s < 2; ++s) {
+      bar_init(bar_s(s), 1); bar_init(bar_done(s), 1); bar_init(bar_sfree(s), 128); bar_init(bar_pds(s), 128); bar_init(bar_rv(s), 128);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(const_cast<uint32_t*>(tmem_slot))),
+                 "r"((uint32_t)KV_TMEM) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t sKt = base, sVt = base + KV_OFF_V;
+  auto sQ = [&](int s) { return base + KV_OFF_QD + (uint32_t)s * KV_STAGE; };
+  auto sDO = [&](int s) { return sQ(s) + KV_BYTES; };
+  auto sPT = [&](int s) { return base + KV_OFF_PT + (uint32_t)s * P_BYTES; };
+  auto sDST = [&](int s) { return base + KV_OFF_DST + (uint32_t)s * P_BYTES; };
+  auto head_of = [&](int i) { return g * rep + i / per_head; };
+  auto q0_of = [&](int i) { return (qt0 + i % per_head) * KT; };
+
+  if (warp == 4) {
+    if (lane == 0) {
+      auto load_item = [&](int i) {
+        const int st = i % KV_STAGES;
+        bar_expect(qfull(st), 2 * KV_BYTES);
+        tma_2d(sQ(st), &tmQ, head_of(i) * HD, (int)(seq0 + q0_of(i)), qfull(st));
+        tma_2d(sDO(st), &tmDO, head_of(i) * HD, (int)(seq0 + q0_of(i)), qfull(st));
+      };
+      bar_expect(bar_kv, 2 * Q_BYTES);
+      tma_2d(sKt, &tmK, g * HD, (int)(seq0 + k0), bar_kv);
+      tma_2d(sVt, &tmV, g * HD, (int)(seq0 + k0), bar_kv);
+      load_item(0);
+      if (n_it > 1) load_item(1);
+      bool ok = bar_wait(bar_kv, 0u, abort_flag, 0xE01u);
+      const uint32_t id_k = idesc(0), id_n = idesc(1);
+      auto issue_s = [&](int i) {                              // S^T and dP^T of item i into buffer pair i & 1
+        const int st = i % KV_STAGES;
+        const uint64_t dk_ = desc_k_major(sKt), dq_ = desc_k_major(sQ(st)), dv_ = desc_k_major(sVt), dd = desc_k_major(sDO(st));
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) mma(tmem + 64u * (uint32_t)(i & 1), dk_ + 2u * k, dq_ + 2u * k, id_k, k != 0 ? 1u : 0u);
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) mma(tmem + 128u + 64u * (uint32_t)(i & 1), dv_ + 2u * k, dd + 2u * k, id_k, k != 0 ? 1u : 0u);
+        commit(bar_s(i & 1));
+      };
+      if (ok) ok = bar_wait(qfull(0), 0u, abort_flag, 0xE10u);
+      if (ok) { fence_after(); issue_s(0); }
+      for (int i = 0; i < n_it && ok; ++i) {
+        if (i + 1 < n_it) {
+          ok = bar_wait(qfull((i + 1) % KV_STAGES), (uint32_t)(((i + 1) / KV_STAGES) & 1), abort_flag, 0xE10u);
+          if (ok && i >= 1) ok = bar_wait(bar_sfree((i + 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), abort_flag, 0xE20u);
+          if (!ok) break;
+          fence_after();
+          issue_s(i + 1);
+        }
+        ok = bar_wait(bar_pds(i & 1), (uint32_t)((i >> 1) & 1), abort_flag, 0xE30u);
+        if (!ok) break;
+        fence_after();
+        {
+          const int st = i % KV_STAGES;
+          const uint64_t dp_ = desc_k_major(sPT(i & 1)), dd = desc_n_major(sDO(st)), ds_ = desc_k_major(sDST(i & 1)), dq_ = desc_n_major(sQ(st));
+#pragma unroll
+          for (int k = 0; k < KT / 16; ++k) mma(tmem + 256u, dp_ + 2u * k, dd + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
+#pragma unroll
+          for (int k = 0; k < KT / 16; ++k) mma(tmem + 320u, ds_ + 2u * k, dq_ + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
+        }
+        commit(bar_done(i & 1));
+        if (i + 2 < n_it) {                                    // its stage last held item i - 1
+          if (i >= 1) ok = bar_wait(bar_done((i - 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), abort_flag, 0xE40u);
+          if (!ok) break;
+          load_item(i + 2);
+        }
+      }
+      if (!ok) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) {} }
+    }
+  } else {
+    const int row = 32 * warp + lane;
+    const int kj = k0 + row;
+    const uint32_t t_lane = tmem + ((uint32_t)(32 * warp) << 16);
+    float* rowv_all = reinterpret_cast<float*>(smem + KV_OFF_ROWV);      // [2][2][KT]: lse, delta / sqrt(d) negated
+    bool ok = true;
+    for (int i = 0; i < n_it; ++i) {
+      const int q0 = q0_of(i);
+      float* rowv = rowv_all + (i & 1) * 2 * KT;
+      {                                                          // this item's 64 lse and delta values
+        const long long ro = ((long long)b * p.H + head_of(i)) * p.S;
+        const int c = row & (KT - 1);
+        const bool valid = q0 + c < p.S;
+        rowv[row] = row < KT ? (valid ? p.lse[ro + q0 + c] : 0.f) : (valid ? -p.dsum[ro + q0 + c] * p.inv_sqrt_d : 0.f);
+      }
+      bar_arrive(bar_rv(i & 1));
+      ok = bar_wait(bar_rv(i & 1), (uint32_t)((i >> 1) & 1), abort_flag, 0xF05u);
+      if (ok) ok = bar_wait(bar_s(i & 1), (uint32_t)((i >> 1) & 1), abort_flag, 0xF10u);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      fence_after();
+      const bool edge = q0 < k0 + QT || q0 + KT > p.S;         // the item crosses the diagonal or the sequence end
+      if (i >= 2) {                                              // the P^T / dS^T buffers last held item i - 2
+        ok = bar_wait(bar_done(i & 1), (uint32_t)(((i - 2) >> 1) & 1), abort_flag, 0xF20u);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      }
+      uint8_t* prow = smem + KV_OFF_PT + (i & 1) * P_BYTES + row * 128;
+      uint8_t* drow = smem + KV_OFF_DST + (i & 1) * P_BYTES + row * 128;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float t[32], d[32];
+        ld32(t_lane + 64u * (uint32_t)(i & 1) + 32u * half, t);
+        ld32(t_lane + 128u + 64u * (uint32_t)(i & 1) + 32u * half, d);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const int c = 32 * half + j;
+          float pr = exp2f(fmaf(t[j], p.scale_log2, -rowv[c]));
+          if (edge && !(kj <= q0 + c && q0 + c < p.S)) pr = 0.f;
+          t[j] = pr;
+          d[j] = pr * fmaf(d[j], p.inv_sqrt_d, rowv[KT + c]);
+        }
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          const int ch = 4 * half + c4;
+          *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) =
+              make_uint4(pack2(t[8 * c4], t[8 * c4 + 1]), pack2(t[8 * c4 + 2], t[8 * c4 + 3]), pack2(t[8 * c4 + 4], t[8 * c4 + 5]),
+                         pack2(t[8 * c4 + 6], t[8 * c4 + 7]));
+          *reinterpret_cast<uint4*>(drow + ((ch ^ (row & 7)) << 4)) =
+              make_uint4(pack2(d[8 * c4], d[8 * c4 + 1]), pack2(d[8 * c4 + 2], d[8 * c4 + 3]), pack2(d[8 * c4 + 4], d[8 * c4 + 5]),
+                         pack2(d[8 * c4 + 6], d[8 * c4 + 7]));
+        }
+      }
+      fence_before();
+      bar_arrive(bar_sfree(i & 1));
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      bar_arrive(bar_pds(i & 1));
+    }
+    if (ok) {
+      ok = bar_wait(bar_done((n_it - 1) & 1), (uint32_t)(((n_it - 1) >> 1) & 1), abort_flag, 0xF30u);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      fence_after();
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        uint4* dst = reinterpret_cast<uint4*>((which ? p.dk : p.dv) + (seq0 + kj) * p.ldk + g * HD);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          float t[32];
+          ld32(t_lane + 256u + 64u * which + 32u * half, t);
+          if (kj < p.S) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              dst[4 * half + c] = make_uint4(pack2(t[8 * c], t[8 * c + 1]), pack2(t[8 * c + 2], t[8 * c + 3]),
+                                             pack2(t[8 * c + 4], t[8 * c + 5]), pack2(t[8 * c + 6], t[8 * c + 7]));
+          }
+        }
+      }
+    }
+  }
+  __syncwarp();
+  fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)KV_TMEM) : "memory");
+  }
+}
+
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -351,6 +747,49 @@ int faar_launch_attention_fwd64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, 
   p.out = reinterpret_cast<__nv_bfloat16*>(out); p.lse = lse; p.ldo = ldo; p.S = S; p.H = H; p.Hkv = Hkv;
   p.scale_log2 = scale_log2;
   attn_fwd64_tc_kernel<<<dim3((S + QT - 1) / QT, H, B), THREADS, SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_attention_dq64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, const void* q, int64_t ldq, const void* k,
+                                  const void* v, int64_t ldk, const void* dout, int64_t ldo, const float* lse,
+                                  const float* dsum, void* dq, float scale_log2) {
+  static_assert(2 * (DQ_SMEM + 1024) <= 227 * 1024, "two CTAs per SM");
+  const long long T = (long long)B * S;
+  if (T > 0x7FFFFFFFll) return (int)cudaErrorInvalidValue;
+  CUtensorMap tmQ, tmDO, tmK, tmV;
+  int e = head_map(ctx, &tmQ, q, T, H * HD, ldq, QT);
+  if (!e) e = head_map(ctx, &tmDO, dout, T, H * HD, ldo, QT);
+  if (!e) e = head_map(ctx, &tmK, k, T, Hkv * HD, ldk, KT);
+  if (!e) e = head_map(ctx, &tmV, v, T, Hkv * HD, ldk, KT);
+  if (e) return e;
+  cudaError_t ce = cudaFuncSetAttribute(attn_dq64_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM);
+  if (ce != cudaSuccess) return (int)ce;
+  TcBwdParams p = {};
+  p.lse = lse; p.dsum = dsum; p.dq = reinterpret_cast<__nv_bfloat16*>(dq); p.ldq = ldq; p.ldk = ldk;
+  p.S = S; p.H = H; p.Hkv = Hkv; p.scale_log2 = scale_log2; p.inv_sqrt_d = scale_log2 / 1.4426950408889634f;
+  attn_dq64_tc_kernel<<<dim3((S + QT - 1) / QT, H, B), THREADS, DQ_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
+  return (int)cudaGetLastError();
+}
+
+int faar_launch_attention_dkv64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, const void* q, int64_t ldq, const void* k,
+                                   const void* v, int64_t ldk, const void* dout, int64_t ldo, const float* lse,
+                                   const float* dsum, void* dk, void* dv, float scale_log2) {
+  static_assert(KV_SMEM <= 227 * 1024, "shared memory budget");
+  const long long T = (long long)B * S;
+  if (T > 0x7FFFFFFFll) return (int)cudaErrorInvalidValue;
+  CUtensorMap tmQ, tmDO, tmK, tmV;
+  int e = head_map(ctx, &tmQ, q, T, H * HD, ldq, KT);
+  if (!e) e = head_map(ctx, &tmDO, dout, T, H * HD, ldo, KT);
+  if (!e) e = head_map(ctx, &tmK, k, T, Hkv * HD, ldk, QT);
+  if (!e) e = head_map(ctx, &tmV, v, T, Hkv * HD, ldk, QT);
+  if (e) return e;
+  cudaError_t ce = cudaFuncSetAttribute(attn_dkv64_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, KV_SMEM);
+  if (ce != cudaSuccess) return (int)ce;
+  TcBwdParams p = {};
+  p.lse = lse; p.dsum = dsum; p.dk = reinterpret_cast<__nv_bfloat16*>(dk); p.dv = reinterpret_cast<__nv_bfloat16*>(dv);
+  p.ldq = ldq; p.ldk = ldk; p.S = S; p.H = H; p.Hkv = Hkv; p.scale_log2 = scale_log2;
+  p.inv_sqrt_d = scale_log2 / 1.4426950408889634f;
+  attn_dkv64_tc_kernel<<<dim3((S + QT - 1) / QT, Hkv, B), THREADS, KV_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
   return (int)cudaGetLastError();
 }
 

@@ -89,6 +89,12 @@ int faar_launch_softquant_init(faar_ctx*, const faar_shape*, const void* W, floa
 int faar_launch_nvfp4_expand(faar_ctx*, int rows, int K, const uint8_t* packed, const uint8_t* scales, void* out, int64_t ld);
 int faar_launch_attention_fwd64_tc(faar_ctx*, int B, int S, int H, int Hkv, const void* q, int64_t ldq, const void* k,
                                    const void* v, int64_t ldk, void* out, int64_t ldo, float* lse, float scale_log2);
+int faar_launch_attention_dq64_tc(faar_ctx*, int B, int S, int H, int Hkv, const void* q, int64_t ldq, const void* k,
+                                  const void* v, int64_t ldk, const void* dout, int64_t ldo, const float* lse,
+                                  const float* dsum, void* dq, float scale_log2);
+int faar_launch_attention_dkv64_tc(faar_ctx*, int B, int S, int H, int Hkv, const void* q, int64_t ldq, const void* k,
+                                   const void* v, int64_t ldk, const void* dout, int64_t ldo, const float* lse,
+                                   const float* dsum, void* dk, void* dv, float scale_log2);
 int faar_attention_tc_status(uint32_t* code_out);
 int faar_launch_softquant_eval(faar_ctx*, const faar_shape*, const float* V, const uint8_t* code,
                                const uint8_t* scales, const float* s_global, float beta,
