@@ -327,6 +327,9 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 constexpr int DQ_OFF_DO = Q_BYTES, DQ_OFF_KV = 2 * Q_BYTES, DQ_STAGE = 2 * KV_BYTES, DQ_STAGES = 3;
 constexpr int DQ_OFF_DS = DQ_OFF_KV + DQ_STAGES * DQ_STAGE, DQ_OFF_CTL = DQ_OFF_DS + P_BYTES;
 constexpr int DQ_SMEM = DQ_OFF_CTL + CTL + 1024;
+// The backward kernels have no reduction along a row, so two threads share a row (32 of the 64 columns each:
+// warps w and w + 4 read the same tensor-memory lanes): eight row warps, the ninth issues copies and MMAs.
+constexpr int BWD_THREADS = 288, ROW_THREADS = 256;
 
 struct TcBwdParams {
   const float* lse; const float* dsum;
@@ -336,7 +339,7 @@ struct TcBwdParams {
   float scale_log2, inv_sqrt_d;
 };
 
-__global__ void __launch_bounds__(THREADS, 2)
+__global__ void __launch_bounds__(BWD_THREADS, 2)
 attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
                     const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const TcBwdParams p) {
   extern __shared__ uint8_t raw[];
@@ -361,12 +364,12 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     bar_init(bar_qd, 1);
     for (int s = 0; s < DQ_STAGES; ++s) bar_init(kvfull(s), 1);
     bar_init(bar_s, 1); bar_init(bar_done, 1);
-    bar_init(bar_sfree, 128); bar_init(bar_ds, 128);
+    bar_init(bar_sfree, ROW_THREADS); bar_init(bar_ds, ROW_THREADS);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(const_cast<uint32_t*>(tmem_slot))),
                  "r"((uint32_t)TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -379,7 +382,7 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   auto sK = [&](int s) { return base + DQ_OFF_KV + (uint32_t)s * DQ_STAGE; };
   auto sV = [&](int s) { return sK(s) + KV_BYTES; };
 
-  if (warp == 4) {
+  if (warp == 8) {
     if (lane == 0) {
       auto load_kv = [&](int j) {
         const int st = j % DQ_STAGES;
@@ -431,9 +434,9 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!ok) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) {} }
     }
   } else {
-    const int row = 32 * warp + lane;
+    const int row = 32 * (warp & 3) + lane, half = warp >> 2;    // this thread: columns 32 half .. 32 half + 31 of its row
     const int qi = q0 + row;
-    const uint32_t t_lane = tmem + ((uint32_t)(32 * warp) << 16);
+    const uint32_t t_lane = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
     const long long ro = ((long long)b * p.H + h) * p.S;
     const float lse = qi < p.S ? p.lse[ro + qi] : 0.f;
     const float nd = qi < p.S ? -p.dsum[ro + qi] * p.inv_sqrt_d : 0.f;
@@ -443,9 +446,8 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       ok = bar_wait(bar_s, (uint32_t)(j & 1), abort_flag, 0xD10u);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       fence_after();
-      float s[KT];
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {                  // P (dP - delta) / sqrt(d), 32 columns at a time
+      float s[32];
+      {                                                       // P (dP - delta) / sqrt(d)
         float t[32], d[32];
         ld32(t_lane + 32u * half, t);
         ld32(t_lane + 64u + 32u * half, d);
@@ -453,7 +455,7 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int i = 0; i < 32; ++i) {
           float pr = exp2f(fmaf(t[i], p.scale_log2, -lse));
           if (k0 + 32 * half + i > qi) pr = 0.f;               // above the diagonal (and beyond the sequence end)
-          s[32 * half + i] = pr * fmaf(d[i], p.inv_sqrt_d, nd);
+          s[i] = pr * fmaf(d[i], p.inv_sqrt_d, nd);
         }
       }
       fence_before();
@@ -464,8 +466,8 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
       uint8_t* prow = smem + DQ_OFF_DS + row * 128;
 #pragma unroll
-      for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
+      for (int c = 0; c < 4; ++c)
+        *reinterpret_cast<uint4*>(prow + (((4 * half + c) ^ (row & 7)) << 4)) =
             make_uint4(pack2(s[8 * c], s[8 * c + 1]), pack2(s[8 * c + 2], s[8 * c + 3]), pack2(s[8 * c + 4], s[8 * c + 5]),
                        pack2(s[8 * c + 6], s[8 * c + 7]));
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -478,8 +480,7 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (ok) {
       fence_after();
       uint4* dst = reinterpret_cast<uint4*>(p.dq + (seq0 + qi) * p.ldq + h * HD);
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      {
         float t[32];
         ld32(t_lane + 128u + 32u * half, t);
         if (qi < p.S) {
@@ -494,7 +495,7 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   __syncwarp();
   fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 8) {
     fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
   }
@@ -508,15 +509,15 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 //   dV += P^T dO_i, dK += dS^T Q_i           two MMAs that accumulate in 64 + 64 columns over the whole sweep
 //                                            (dO_i and Q_i read as they lie in memory: queries as contraction rows)
 // One CTA per SM; the score products of item i + 1 are issued before this item's probabilities are awaited, Q / dO
-// tiles come through three TMA stages, lse and delta of a tile's 64 queries are staged in shared memory by the
+// tiles come through four TMA stages (requested two items ahead), lse and delta of a tile's 64 queries are staged in shared memory by the
 // row threads themselves.  Queries beyond the sequence end are masked (their rows hold the next sequence's data).
-constexpr int KV_OFF_V = Q_BYTES, KV_OFF_QD = 2 * Q_BYTES, KV_STAGE = 2 * KV_BYTES, KV_STAGES = 3;
+constexpr int KV_OFF_V = Q_BYTES, KV_OFF_QD = 2 * Q_BYTES, KV_STAGE = 2 * KV_BYTES, KV_STAGES = 4;
 constexpr int KV_OFF_PT = KV_OFF_QD + KV_STAGES * KV_STAGE, KV_OFF_DST = KV_OFF_PT + 2 * P_BYTES;
 constexpr int KV_OFF_ROWV = KV_OFF_DST + 2 * P_BYTES, KV_OFF_CTL = KV_OFF_ROWV + 2 * 2 * KT * 4;
 constexpr int KV_SMEM = KV_OFF_CTL + CTL + 1024;
 constexpr int KV_TMEM = 512;                      // S^T: 0 / 64, dP^T: 128 / 192, dV: 256, dK: 320
 
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(BWD_THREADS, 1)
 attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
                      const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const TcBwdParams p) {
   extern __shared__ uint8_t raw[];
@@ -524,14 +525,14 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   uint8_t* smem = raw + (base - s32(raw));
   const uint32_t ctl = base + KV_OFF_CTL;
   const uint32_t bar_kv = ctl;
-  auto qfull = [&](int s) { return ctl + 8u + 8u * s; };          // 3
-  auto bar_s = [&](int s) { return ctl + 32u + 8u * s; };         // 2: score buffers of an item are complete
-  auto bar_sfree = [&](int s) { return ctl + 48u + 8u * s; };     // 2: ... have been read by all 128 rows
-  auto bar_pds = [&](int s) { return ctl + 64u + 8u * s; };       // 2: P^T / dS^T buffers written
-  auto bar_done = [&](int s) { return ctl + 80u + 8u * s; };      // 2: the accumulating MMAs of an item have run
-  auto bar_rv = [&](int s) { return ctl + 104u + 8u * s; };       // 2: lse / delta of an item staged by all 128 rows
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + KV_OFF_CTL + 96);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + KV_OFF_CTL + 100);
+  auto qfull = [&](int s) { return ctl + 8u + 8u * s; };          // 4
+  auto bar_s = [&](int s) { return ctl + 40u + 8u * s; };         // 2: score buffers of an item are complete
+  auto bar_sfree = [&](int s) { return ctl + 56u + 8u * s; };     // 2: ... have been read by all rows
+  auto bar_pds = [&](int s) { return ctl + 72u + 8u * s; };       // 2: P^T / dS^T buffers written
+  auto bar_done = [&](int s) { return ctl + 88u + 8u * s; };      // 2: the accumulating MMAs of an item have run
+  auto bar_rv = [&](int s) { return ctl + 112u + 8u * s; };       // 2: lse / delta of an item staged, previous use read by all
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + KV_OFF_CTL + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + KV_OFF_CTL + 132);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const int kt = blockIdx.x, g = blockIdx.y, b = blockIdx.z;       // the first key tiles see the most queries
@@ -547,13 +548,13 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     bar_init(bar_kv, 1);
     for (int s = 0; s < KV_STAGES; ++s) bar_init(qfull(s), 1);
     for (int s = 0; s < 2; ++s) {
-      bar_init(bar_s(s), 1); bar_init(bar_done(s), 1); bar_init(bar_sfree(s), 128); bar_init(bar_pds(s), 128); bar_init(bar_rv(s), 128);
+      bar_init(bar_s(s), 1); bar_init(bar_done(s), 1); bar_init(bar_sfree(s), ROW_THREADS); bar_init(bar_pds(s), ROW_THREADS); bar_init(bar_rv(s), ROW_THREADS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(const_cast<uint32_t*>(tmem_slot))),
                  "r"((uint32_t)KV_TMEM) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -570,7 +571,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   auto head_of = [&](int i) { return g * rep + i / per_head; };
   auto q0_of = [&](int i) { return (qt0 + i % per_head) * KT; };
 
-  if (warp == 4) {
+  if (warp == 8) {
     if (lane == 0) {
       auto load_item = [&](int i) {
         const int st = i % KV_STAGES;
@@ -583,6 +584,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       tma_2d(sVt, &tmV, g * HD, (int)(seq0 + k0), bar_kv);
       load_item(0);
       if (n_it > 1) load_item(1);
+      if (n_it > 2) load_item(2);
       bool ok = bar_wait(bar_kv, 0u, abort_flag, 0xE01u);
       const uint32_t id_k = idesc(0), id_n = idesc(1);
       auto issue_s = [&](int i) {                              // S^T and dP^T of item i into buffer pair i & 1
@@ -604,6 +606,11 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           fence_after();
           issue_s(i + 1);
         }
+        if (i + 3 < n_it) {                                    // its stage last held item i - 1: wait for that item's
+          if (i >= 1) ok = bar_wait(bar_done((i - 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), abort_flag, 0xE40u);   // MMAs
+          if (!ok) break;
+          load_item(i + 3);
+        }
         ok = bar_wait(bar_pds(i & 1), (uint32_t)((i >> 1) & 1), abort_flag, 0xE30u);
         if (!ok) break;
         fence_after();
@@ -616,29 +623,32 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           for (int k = 0; k < KT / 16; ++k) mma(tmem + 320u, ds_ + 2u * k, dq_ + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
         }
         commit(bar_done(i & 1));
-        if (i + 2 < n_it) {                                    // its stage last held item i - 1
-          if (i >= 1) ok = bar_wait(bar_done((i - 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), abort_flag, 0xE40u);
-          if (!ok) break;
-          load_item(i + 2);
-        }
       }
       if (!ok) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) {} }
     }
   } else {
-    const int row = 32 * warp + lane;
+    const int row = 32 * (warp & 3) + lane, half = warp >> 2;    // this thread: queries 32 half .. 32 half + 31 of an item
     const int kj = k0 + row;
-    const uint32_t t_lane = tmem + ((uint32_t)(32 * warp) << 16);
+    const uint32_t t_lane = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
     float* rowv_all = reinterpret_cast<float*>(smem + KV_OFF_ROWV);      // [2][2][KT]: lse, delta / sqrt(d) negated
     bool ok = true;
+    // this thread's share of an item's 64 lse values (rows 0..63) or 64 negated, scaled delta values (rows 64..127);
+    // the value for item i + 1 is requested at the start of item i, so its latency is off the per-item path
+    auto row_value = [&](int i) {
+      const long long ro = ((long long)b * p.H + head_of(i)) * p.S;
+      const int q = q0_of(i) + (row & (KT - 1));
+      if (q >= p.S) return 0.f;
+      return row < KT ? p.lse[ro + q] : -p.dsum[ro + q] * p.inv_sqrt_d;
+    };
+    float rv_next = half == 0 ? row_value(0) : 0.f;
     for (int i = 0; i < n_it; ++i) {
       const int q0 = q0_of(i);
       float* rowv = rowv_all + (i & 1) * 2 * KT;
-      {                                                          // this item's 64 lse and delta values
-        const long long ro = ((long long)b * p.H + head_of(i)) * p.S;
-        const int c = row & (KT - 1);
-        const bool valid = q0 + c < p.S;
-        rowv[row] = row < KT ? (valid ? p.lse[ro + q0 + c] : 0.f) : (valid ? -p.dsum[ro + q0 + c] * p.inv_sqrt_d : 0.f);
+      if (half == 0) {                                           // the first four warps stage the 128 values
+        rowv[row] = rv_next;
+        if (i + 1 < n_it) rv_next = row_value(i + 1);
       }
+      // every row thread arrives: the buffer of item i + 2 is then written only after all have read item i's
       bar_arrive(bar_rv(i & 1));
       ok = bar_wait(bar_rv(i & 1), (uint32_t)((i >> 1) & 1), abort_flag, 0xF05u);
       if (ok) ok = bar_wait(bar_s(i & 1), (uint32_t)((i >> 1) & 1), abort_flag, 0xF10u);
@@ -651,8 +661,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       }
       uint8_t* prow = smem + KV_OFF_PT + (i & 1) * P_BYTES + row * 128;
       uint8_t* drow = smem + KV_OFF_DST + (i & 1) * P_BYTES + row * 128;
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      {
         float t[32], d[32];
         ld32(t_lane + 64u * (uint32_t)(i & 1) + 32u * half, t);
         ld32(t_lane + 128u + 64u * (uint32_t)(i & 1) + 32u * half, d);
@@ -689,8 +698,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll
       for (int which = 0; which < 2; ++which) {
         uint4* dst = reinterpret_cast<uint4*>((which ? p.dk : p.dv) + (seq0 + kj) * p.ldk + g * HD);
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        {
           float t[32];
           ld32(t_lane + 256u + 64u * which + 32u * half, t);
           if (kj < p.S) {
@@ -706,7 +714,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   __syncwarp();
   fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 8) {
     fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)KV_TMEM) : "memory");
   }
@@ -767,7 +775,7 @@ int faar_launch_attention_dq64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, c
   TcBwdParams p = {};
   p.lse = lse; p.dsum = dsum; p.dq = reinterpret_cast<__nv_bfloat16*>(dq); p.ldq = ldq; p.ldk = ldk;
   p.S = S; p.H = H; p.Hkv = Hkv; p.scale_log2 = scale_log2; p.inv_sqrt_d = scale_log2 / 1.4426950408889634f;
-  attn_dq64_tc_kernel<<<dim3((S + QT - 1) / QT, H, B), THREADS, DQ_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
+  attn_dq64_tc_kernel<<<dim3((S + QT - 1) / QT, H, B), BWD_THREADS, DQ_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
   return (int)cudaGetLastError();
 }
 
@@ -789,7 +797,7 @@ int faar_launch_attention_dkv64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, 
   p.lse = lse; p.dsum = dsum; p.dk = reinterpret_cast<__nv_bfloat16*>(dk); p.dv = reinterpret_cast<__nv_bfloat16*>(dv);
   p.ldq = ldq; p.ldk = ldk; p.S = S; p.H = H; p.Hkv = Hkv; p.scale_log2 = scale_log2;
   p.inv_sqrt_d = scale_log2 / 1.4426950408889634f;
-  attn_dkv64_tc_kernel<<<dim3((S + QT - 1) / QT, Hkv, B), THREADS, KV_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
+  attn_dkv64_tc_kernel<<<dim3((S + QT - 1) / QT, Hkv, B), BWD_THREADS, KV_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
   return (int)cudaGetLastError();
 }
 
