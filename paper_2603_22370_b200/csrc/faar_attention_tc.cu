@@ -111,6 +111,13 @@ __device__ __forceinline__ void ld32(uint32_t taddr, float (&r)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
 }
+// 2^x on the special-function unit, one instruction (relative error about 2^-22; -inf gives 0; results below the
+// normal range are flushed to zero, which is what a probability that small should be)
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -256,19 +263,20 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         for (int i = 0; i < KT; ++i)
           if (!(k0 + i <= qi && k0 + i < p.S)) s[i] = -INFINITY;
       }
-      float mx = s[0];
+      float mx4[4] = {s[0], s[1], s[2], s[3]};                   // four independent chains instead of one of 64
 #pragma unroll
-      for (int i = 1; i < KT; ++i) mx = fmaxf(mx, s[i]);
+      for (int i = 4; i < KT; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], s[i]);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float m_new = fmaxf(m, mx * p.scale_log2);
       const float ref = m_new == -INFINITY ? 0.f : m_new;     // a row beyond the sequence may have seen no key
-      const float alpha = exp2f(m - ref);
-      float sum = 0.f;
+      const float alpha = ex2(m - ref);
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint8_t* prow = smem + OFF_P + (j & 1) * P_BYTES + row * 128;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         float e[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { e[i] = exp2f(fmaf(s[8 * c + i], p.scale_log2, -ref)); sum += e[i]; }
+        for (int i = 0; i < 8; ++i) { e[i] = ex2(fmaf(s[8 * c + i], p.scale_log2, -ref)); sum4[i & 3] += e[i]; }
         *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
             make_uint4(pack2(e[0], e[1]), pack2(e[2], e[3]), pack2(e[4], e[5]), pack2(e[6], e[7]));
       }
@@ -284,7 +292,7 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         fence_before();
         bar_arrive(bar_ofree);
       }
-      l = l * alpha + sum;
+      l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
 #pragma unroll
       for (int i = 0; i < HD; ++i) o_acc[i] *= alpha;
       m = m_new;
@@ -453,7 +461,7 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         ld32(t_lane + 64u + 32u * half, d);
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          float pr = exp2f(fmaf(t[i], p.scale_log2, -lse));
+          float pr = ex2(fmaf(t[i], p.scale_log2, -lse));
           if (k0 + 32 * half + i > qi) pr = 0.f;               // above the diagonal (and beyond the sequence end)
           s[i] = pr * fmaf(d[i], p.inv_sqrt_d, nd);
         }
@@ -666,12 +674,18 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         ld32(t_lane + 64u * (uint32_t)(i & 1) + 32u * half, t);
         ld32(t_lane + 128u + 64u * (uint32_t)(i & 1) + 32u * half, d);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int c = 32 * half + j;
-          float pr = exp2f(fmaf(t[j], p.scale_log2, -rowv[c]));
-          if (edge && !(kj <= q0 + c && q0 + c < p.S)) pr = 0.f;
-          t[j] = pr;
-          d[j] = pr * fmaf(d[j], p.inv_sqrt_d, rowv[KT + c]);
+        for (int j4 = 0; j4 < 32; j4 += 4) {
+          const float4 l4 = *reinterpret_cast<const float4*>(rowv + 32 * half + j4);          // the same address in every lane
+          const float4 n4 = *reinterpret_cast<const float4*>(rowv + KT + 32 * half + j4);
+          const float lq[4] = {l4.x, l4.y, l4.z, l4.w}, nq[4] = {n4.x, n4.y, n4.z, n4.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int j = j4 + e, c = 32 * half + j;
+            float pr = ex2(fmaf(t[j], p.scale_log2, -lq[e]));
+            if (edge && !(kj <= q0 + c && q0 + c < p.S)) pr = 0.f;
+            t[j] = pr;
+            d[j] = pr * fmaf(d[j], p.inv_sqrt_d, nq[e]);
+          }
         }
 #pragma unroll
         for (int c4 = 0; c4 < 4; ++c4) {
