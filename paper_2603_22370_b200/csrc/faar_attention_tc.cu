@@ -343,7 +343,7 @@ struct TcBwdParams {
   const float* lse; const float* dsum;
   __nv_bfloat16* dq; __nv_bfloat16* dk; __nv_bfloat16* dv;
   long long ldq, ldk;
-  int S, H, Hkv;
+  int B, S, H, Hkv;
   float scale_log2, inv_sqrt_d;
 };
 
@@ -543,7 +543,10 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + KV_OFF_CTL + 132);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  const int kt = blockIdx.x, g = blockIdx.y, b = blockIdx.z;       // the first key tiles see the most queries
+  // one-dimensional grid, key tile slowest: CTAs start in order of decreasing work (the first key tiles see the
+  // most queries), so the short ones fill the end of the launch
+  const int groups = p.Hkv * p.B;
+  const int kt = blockIdx.x / groups, g = (blockIdx.x % groups) % p.Hkv, b = (blockIdx.x % groups) / p.Hkv;
   const int rep = p.H / p.Hkv;
   const long long seq0 = (long long)b * p.S;
   const int k0 = kt * QT;
@@ -809,9 +812,9 @@ int faar_launch_attention_dkv64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, 
   if (ce != cudaSuccess) return (int)ce;
   TcBwdParams p = {};
   p.lse = lse; p.dsum = dsum; p.dk = reinterpret_cast<__nv_bfloat16*>(dk); p.dv = reinterpret_cast<__nv_bfloat16*>(dv);
-  p.ldq = ldq; p.ldk = ldk; p.S = S; p.H = H; p.Hkv = Hkv; p.scale_log2 = scale_log2;
+  p.ldq = ldq; p.ldk = ldk; p.B = B; p.S = S; p.H = H; p.Hkv = Hkv; p.scale_log2 = scale_log2;
   p.inv_sqrt_d = scale_log2 / 1.4426950408889634f;
-  attn_dkv64_tc_kernel<<<dim3((S + QT - 1) / QT, Hkv, B), BWD_THREADS, KV_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
+  attn_dkv64_tc_kernel<<<dim3(((S + QT - 1) / QT) * Hkv * B, 1, 1), BWD_THREADS, KV_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
   return (int)cudaGetLastError();
 }
 
