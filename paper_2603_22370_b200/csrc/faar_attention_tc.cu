@@ -34,7 +34,7 @@ __device__ uint32_t g_attn_status;                 // 0 = no wait has given up s
 struct TcParams {
   __nv_bfloat16* out; float* lse;
   long long ldo;
-  int S, H, Hkv;
+  int B, S, H, Hkv;
   float scale_log2;
 };
 
@@ -139,8 +139,10 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_CTL + 100);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;       // longest tiles first
-  const int h = blockIdx.y, b = blockIdx.z;
+  // one-dimensional grid, query tile slowest and descending: CTAs start in order of decreasing work
+  const int hb = p.H * p.B;
+  const int qt = (int)(gridDim.x / hb) - 1 - (int)(blockIdx.x / hb);
+  const int h = (blockIdx.x % hb) % p.H, b = (blockIdx.x % hb) / p.H;
   const int g = h / (p.H / p.Hkv);
   const long long seq0 = (long long)b * p.S;
   const int q0 = qt * QT;
@@ -360,8 +362,10 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + DQ_OFF_CTL + 100);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;
-  const int h = blockIdx.y, b = blockIdx.z;
+  // one-dimensional grid, query tile slowest and descending: CTAs start in order of decreasing work
+  const int hb = p.H * p.B;
+  const int qt = (int)(gridDim.x / hb) - 1 - (int)(blockIdx.x / hb);
+  const int h = (blockIdx.x % hb) % p.H, b = (blockIdx.x % hb) / p.H;
   const int g = h / (p.H / p.Hkv);
   const long long seq0 = (long long)b * p.S;
   const int q0 = qt * QT;
@@ -769,9 +773,9 @@ int faar_launch_attention_fwd64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, 
   cudaError_t ce = cudaFuncSetAttribute(attn_fwd64_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (ce != cudaSuccess) return (int)ce;
   TcParams p;
-  p.out = reinterpret_cast<__nv_bfloat16*>(out); p.lse = lse; p.ldo = ldo; p.S = S; p.H = H; p.Hkv = Hkv;
+  p.out = reinterpret_cast<__nv_bfloat16*>(out); p.lse = lse; p.ldo = ldo; p.B = B; p.S = S; p.H = H; p.Hkv = Hkv;
   p.scale_log2 = scale_log2;
-  attn_fwd64_tc_kernel<<<dim3((S + QT - 1) / QT, H, B), THREADS, SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
+  attn_fwd64_tc_kernel<<<dim3(((S + QT - 1) / QT) * H * B, 1, 1), THREADS, SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
   return (int)cudaGetLastError();
 }
 
@@ -791,8 +795,8 @@ int faar_launch_attention_dq64_tc(faar_ctx* ctx, int B, int S, int H, int Hkv, c
   if (ce != cudaSuccess) return (int)ce;
   TcBwdParams p = {};
   p.lse = lse; p.dsum = dsum; p.dq = reinterpret_cast<__nv_bfloat16*>(dq); p.ldq = ldq; p.ldk = ldk;
-  p.S = S; p.H = H; p.Hkv = Hkv; p.scale_log2 = scale_log2; p.inv_sqrt_d = scale_log2 / 1.4426950408889634f;
-  attn_dq64_tc_kernel<<<dim3((S + QT - 1) / QT, H, B), BWD_THREADS, DQ_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
+  p.B = B; p.S = S; p.H = H; p.Hkv = Hkv; p.scale_log2 = scale_log2; p.inv_sqrt_d = scale_log2 / 1.4426950408889634f;
+  attn_dq64_tc_kernel<<<dim3(((S + QT - 1) / QT) * H * B, 1, 1), BWD_THREADS, DQ_SMEM, ctx->stream>>>(tmQ, tmDO, tmK, tmV, p);
   return (int)cudaGetLastError();
 }
 
