@@ -506,8 +506,8 @@ FAAR_API int faar_add(faar_ctx* ctx, int rows, int cols, const void* a, int64_t 
  * forward call's; dsum is scratch, [batch, n_heads, seq] floats.  No matrix of seq x seq values is stored; results
  * are reproducible (no atomics).  head_dim is 64 or 128; leading dimensions multiples of 8, bases 16-byte aligned. */
 /* Which kernels head_dim 64 takes (head_dim 128 always takes the third kind):
- *   0 (default): forward on the tcgen05 tensor cores (128-query tiles, scores and the per-tile output in tensor
- *      memory, one query row per thread), backward as mode 2;
+ *   0 (default): forward, dQ and dK / dV kernels on the tcgen05 tensor cores (scores in tensor memory, one query or
+ *      key row per thread or pair of threads, gradients accumulated in tensor memory over the sweep);
  *   2: forward and backward with scores and probabilities in registers (mma.sync m16n8k16, one sweep over the
  *      keys with a running maximum);
  *   1: kernels that pass scores and probabilities through shared memory as 16 x 16 fragments (two sweeps in the

@@ -20,7 +20,7 @@ struct faar_ctx {
   int tune_bn;                            // 0 = choose the GEMM tile width automatically
   int tune_tail;                          // -1 = choose the tail split automatically, else columns to split
   int tune_wide;                          // 1 = 256 x 512 GEMM tiles wherever the shape allows; -1 (default), 0 = never
-  int tune_attention_fragments;           // head_dim 64 attention: 0 = tcgen05 forward + mma.sync backward, 2 = mma.sync both, 1 = the shared-memory fragment kernels
+  int tune_attention_fragments;           // head_dim 64 attention: 0 = tcgen05 kernels, 2 = mma.sync kernels, 1 = the shared-memory fragment kernels
   int last_gemm_bn, last_gemm_pairs, last_gemm_split;   // what the last GEMM launch used
   // CTA pairs this context's device can hold at once, per GEMM kernel instantiation (0 = not asked yet)
   int gemm_max_pairs[FAAR_GEMM_VARIANTS];

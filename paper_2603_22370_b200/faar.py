@@ -310,8 +310,8 @@ def attention_status(ctx):
 
 
 def tune_attention(ctx, mode: int):
-    """head_dim 64: 0 = tcgen05 forward + register-resident backward (default), 2 = register-resident kernels for
-    both, 1 = the shared-memory fragment kernels (as head_dim 128 always takes)."""
+    """head_dim 64: 0 = tcgen05 kernels forward and backward (default), 2 = register-resident mma.sync kernels,
+    1 = the shared-memory fragment kernels (as head_dim 128 always takes)."""
     _check(lib().faar_tune_attention(ctx._h, mode), "faar_tune_attention")
 
 

@@ -33,9 +33,9 @@ def padded(a, ld, fill=9.0):
 @pytest.mark.parametrize("B,S,H,HKV,D", [(2, 100, 4, 2, 64), (1, 64, 2, 2, 64), (3, 7, 2, 1, 64), (1, 200, 4, 1, 128),
                                          (2, 129, 8, 2, 64), (1, 321, 4, 4, 64)])
 def test_attention_forward_and_backward_match_the_oracle(ctx, B, S, H, HKV, D, fragments):
-    """fragments = 0: the default kernels (head_dim 64: forward on tcgen05, backward with scores in registers);
-    2: head_dim 64 with scores in registers forward and backward; 1: head_dim 64 through the shared-memory fragment
-    kernels that head_dim 128 always uses."""
+    """fragments = 0: the default kernels (head_dim 64: forward and backward on tcgen05); 2: head_dim 64 with scores
+    in registers (mma.sync) forward and backward; 1: head_dim 64 through the shared-memory fragment kernels that
+    head_dim 128 always uses."""
     if fragments and D != 64:
         pytest.skip("head_dim 128 has one kind of kernel")
     faar.tune_attention(ctx, fragments)
@@ -81,6 +81,7 @@ def _attention_case(ctx, B, S, H, HKV, D):
     DV = torch.full((T, ldk), 5.0, dtype=torch.bfloat16, device=DEV)
     faar.attention_bwd(ctx, B, S, H, HKV, D, Q, ldq, K, V, ldk, O, DO, ldq, lse, dsum, DQ, DK, DV)
     torch.cuda.synchronize()
+    faar.attention_status(ctx)
     dq_o, dk_o, dv_o = so.attention_bwd(do, q, k, v, P, B, S, H, HKV, D)
     for name, g_t, ref, n in (("dq", DQ, dq_o, H * D), ("dk", DK, dk_o, HKV * D), ("dv", DV, dv_o, HKV * D)):
         g = host(g_t[:, :n]).astype(np.float64)
