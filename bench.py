@@ -69,8 +69,8 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # layer, from one ncu capture each, with the SHA-256 (first 12 hex digits) of the kernel source at the time of
 # the capture.  A kernel source that has changed since makes the figure stale: `traffic` is then null.
 NCU_TRAFFIC = {
-    "gemm_bwd": {"bytes": 458.0e6, "source_sha": "7f5fb081ddf5"},
-    "gemm_fwd": {"bytes": 159.5e6, "source_sha": "7f5fb081ddf5"},
+    "gemm_bwd": {"bytes": 458.2e6, "source_sha": "4f6f41dfef24"},
+    "gemm_fwd": {"bytes": 156.3e6, "source_sha": "4f6f41dfef24"},
 }
 GEMM_SOURCE = os.path.join(ROOT, "paper_2603_22370_b200", "csrc", "faar_gemm.cu")
 

@@ -578,11 +578,14 @@ __device__ __forceinline__ float epi_bwd_rows(const KParams& p, uint32_t panel, 
 
 // ---- the kernel ------------------------------------------------------------------------------
 // Launched as clusters of two CTAs along x: CTAs 2c and 2c+1 form pair c.
-template <int MODE, int OPT, bool WIDE>
+// MN: bit 0 = the A operand, bit 1 = the B operand is stored with its M / N index contiguous (KParams.a_mn / b_mn);
+// a compile-time choice, so that the K-major kernels carry no trace of the other layout in their issue loops.
+template <int MODE, int OPT, bool WIDE, int MN>
 __global__ void __launch_bounds__(Cfg<MODE, WIDE>::THREADS, 1)
 faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmBh, const KParams p) {
   using C = Cfg<MODE, WIDE>;
+  constexpr bool A_MN = (MN & 1) != 0, B_MN = (MN & 2) != 0;
   const int BN = p.bn;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -653,13 +656,13 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             mbar_expect_tx(full_bar(stage), WIDE ? 2u * (uint32_t)(C::A_BYTES + C::B_BYTES)
                                                  : 2u * (uint32_t)(C::A_BYTES + (tc.w / 2) * BK * 2));
           const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
-          if (p.a_mn) {                                        // two boxes of 64 rows of A, each [64 k][64 m]
+          if (A_MN) {                                          // two boxes of 64 rows of A, each [64 k][64 m]
             tma_load_2d(sa, &tmA, m0, kb * BK, leader_full, keep);
             tma_load_2d(sa + MN_BOX_BYTES, &tmA, m0 + MN_BOX, kb * BK, leader_full, keep);
           } else {
             tma_load_2d(sa, &tmA, kb * BK, m0, leader_full, keep);
           }
-          if (p.b_mn) {                                        // w/2 = 128 or 64 rows of B: two boxes or one
+          if (B_MN) {                                          // w/2 = 128 or 64 rows of B: two boxes or one
             tma_load_2d(sb, &tmB, n0, kb * BK, leader_full, keep);
             if (tc.w / 2 > MN_BOX) tma_load_2d(sb + MN_BOX_BYTES, &tmB, n0 + MN_BOX, kb * BK, leader_full, keep);
           } else {
@@ -691,15 +694,15 @@ faar_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + acc * BN_MAX;
-        const uint32_t idesc = make_idesc(WIDE ? BN_MAX : tile_coord(p, tile, m_tiles).w, p.a_mn, p.b_mn);
+        const uint32_t idesc = make_idesc(WIDE ? BN_MAX : tile_coord(p, tile, m_tiles).w, A_MN ? 1 : 0, B_MN ? 1 : 0);
         for (int kb = 0; kb < k_blocks; ++kb) {
           ok = mbar_wait(full_bar(stage), phase, ac, 0x300u | stage);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-          const uint64_t da = p.a_mn ? make_smem_desc_mn(sa) : make_smem_desc(sa);
-          const uint64_t db = p.b_mn ? make_smem_desc_mn(sb) : make_smem_desc(sb);
-          const uint32_t ka = p.a_mn ? MN_KSTEP : 2u, kbs = p.b_mn ? MN_KSTEP : 2u;
+          const uint64_t da = A_MN ? make_smem_desc_mn(sa) : make_smem_desc(sa);
+          const uint64_t db = B_MN ? make_smem_desc_mn(sb) : make_smem_desc(sb);
+          constexpr uint32_t ka = A_MN ? MN_KSTEP : 2u, kbs = B_MN ? MN_KSTEP : 2u;
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 bf16 = 32 bytes inside the swizzled row: +2 in the 16-byte address field
@@ -1021,14 +1024,14 @@ bool pick_wide(const faar_ctx* ctx, int N, int bn) {
   return ctx->tune_wide == 1 && bn == BN_MAX && N > BN_MAX;
 }
 
-template <int MODE, int OPT, bool WIDE>
+template <int MODE, int OPT, bool WIDE, int MN>
 int launch_variant(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_out, int bn, int max_pairs,
                    const cudaLaunchConfig_t& base_cfg) {
   using C = Cfg<MODE, WIDE>;
   static_assert(C::STAGES >= 3, "ring too short");
   static_assert(C::SMEM_BYTES <= SMEM_LIMIT, "shared memory budget");
   static_assert(C::EPI_WARPS <= MAX_EPI_WARPS, "partials budget");
-  auto kern = faar_gemm_kernel<MODE, OPT, WIDE>;
+  auto kern = faar_gemm_kernel<MODE, OPT, WIDE, MN>;
   cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (ce != cudaSuccess) return (int)ce;
   cudaLaunchConfig_t cfg = base_cfg;
@@ -1085,7 +1088,7 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
   // per context and kernel mode, with the context's device current (every variant takes one CTA per SM)
   int& max_pairs = ctx->gemm_max_pairs[MODE == FAAR_GEMM_BWD ? 2 + OPT : MODE];
   if (max_pairs == 0) {
-    auto kern = faar_gemm_kernel<MODE, OPT, false>;
+    auto kern = faar_gemm_kernel<MODE, OPT, false, 0>;
     cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
     if (ce != cudaSuccess) return (int)ce;
     cfg.gridDim = dim3(2 * (ctx->num_sms / 2), 1, 1);
@@ -1096,9 +1099,19 @@ int launch(faar_ctx* ctx, const faar_gemm_args* a, KParams& kp, int* n_partials_
     max_pairs = n;
   }
   const int bn = pick_bn(ctx, MODE, a->M, a->N, max_pairs, a->b_mn != 0);
-  if (!a->a_mn && !a->b_mn && pick_wide(ctx, a->N, bn))
-    return launch_variant<MODE, OPT, true>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
-  return launch_variant<MODE, OPT, false>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
+  const int mn = (a->a_mn ? 1 : 0) | (a->b_mn ? 2 : 0);
+  // which operand layouts a mode is ever launched with: the plain product with A untransposed (input gradient),
+  // the dW product with B or with both untransposed
+  if constexpr (MODE == FAAR_GEMM_REF) {
+    if (mn == 1) return launch_variant<MODE, OPT, false, 1>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
+  }
+  if constexpr (MODE == FAAR_GEMM_BWD) {
+    if (mn == 2) return launch_variant<MODE, OPT, false, 2>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
+    if (mn == 3) return launch_variant<MODE, OPT, false, 3>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
+  }
+  if (mn != 0) return (int)cudaErrorInvalidValue;
+  if (pick_wide(ctx, a->N, bn)) return launch_variant<MODE, OPT, true, 0>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
+  return launch_variant<MODE, OPT, false, 0>(ctx, a, kp, n_partials_out, bn, max_pairs, cfg);
 }
 
 }  // namespace
