@@ -233,15 +233,18 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     for (int i = 0; i < HD; ++i) o_acc[i] = 0.f;
     float m = -INFINITY, l = 0.f;
     bool ok = true;
-    auto fold = [&]() {                                       // o_acc += O_j
+    // o_acc <- o_acc * a + O_j: the accumulated output moves to the maximum that P_j was formed against (factor a,
+    // computed when tile j was processed) and takes tile j's product in the same multiply-add
+    auto fold = [&](float a) {
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         float t[32];
         ld32(t_o + 32u * half, t);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) o_acc[32 * half + i] += t[i];
+        for (int i = 0; i < 32; ++i) o_acc[32 * half + i] = fmaf(o_acc[32 * half + i], a, t[i]);
       }
     };
+    float alpha_pending = 0.f;                                // factor of the tile whose P V product is still to be folded
     for (int j = 0; j < n_kt; ++j) {
       const int k0 = j * KT;
       const uint32_t t_s = t_lane + 64u * (uint32_t)(j & 1);
@@ -284,19 +287,17 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this row of P, visible to the tensor cores
       bar_arrive(bar_p);
-      // the previous tile's P V has had the whole of this tile's softmax to finish: fold it in (still relative to
-      // the maximum of tile j - 1), then move everything to the new maximum
+      // the previous tile's P V has had the whole of this tile's softmax to finish: fold it in
       if (j > 0) {
         ok = bar_wait(bar_o, (uint32_t)((j - 1) & 1), abort_flag, 0xB20u);
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         fence_after();
-        fold();
+        fold(alpha_pending);
         fence_before();
         bar_arrive(bar_ofree);
       }
+      alpha_pending = alpha;
       l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
-#pragma unroll
-      for (int i = 0; i < HD; ++i) o_acc[i] *= alpha;
       m = m_new;
     }
     if (ok) {
@@ -305,7 +306,7 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     }
     if (ok) {
       fence_after();
-      fold();
+      fold(alpha_pending);
       if (qi < p.S) {
         const float inv = l > 0.f ? 1.0f / l : 0.f;
         uint4* dst = reinterpret_cast<uint4*>(p.out + (seq0 + qi) * p.ldo + h * HD);
