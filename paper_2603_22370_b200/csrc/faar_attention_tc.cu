@@ -16,6 +16,8 @@
 // faar_attention_status), raises the CTA's abort flag and all roles leave.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "faar_internal.cuh"
 
 namespace {
@@ -460,17 +462,19 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       fence_after();
       float s[32];
-      {                                                       // P (dP - delta) / sqrt(d)
+      auto tile = [&](auto diag_tag) {                        // P (dP - delta) / sqrt(d); the mask only where needed
+        constexpr bool DIAG = decltype(diag_tag)::value;
         float t[32], d[32];
         ld32(t_lane + 32u * half, t);
         ld32(t_lane + 64u + 32u * half, d);
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           float pr = ex2(fmaf(t[i], p.scale_log2, -lse));
-          if (k0 + 32 * half + i > qi) pr = 0.f;               // above the diagonal (and beyond the sequence end)
+          if (DIAG && k0 + 32 * half + i > qi) pr = 0.f;       // above the diagonal (and beyond the sequence end)
           s[i] = pr * fmaf(d[i], p.inv_sqrt_d, nd);
         }
-      }
+      };
+      if (k0 + KT - 1 > q0) tile(std::true_type{}); else tile(std::false_type{});   // some key of the tile above some row
       fence_before();
       bar_arrive(bar_sfree);
       if (j > 0) {                                            // the dS buffer is free once dQ of tile j - 1 has run
@@ -677,7 +681,9 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       }
       uint8_t* prow = smem + KV_OFF_PT + (i & 1) * P_BYTES + row * 128;
       uint8_t* drow = smem + KV_OFF_DST + (i & 1) * P_BYTES + row * 128;
-      {
+      // the mask costs three instructions per element: only items that need it take that path
+      auto item = [&](auto edge_tag) {
+        constexpr bool EDGE = decltype(edge_tag)::value;
         float t[32], d[32];
         ld32(t_lane + 64u * (uint32_t)(i & 1) + 32u * half, t);
         ld32(t_lane + 128u + 64u * (uint32_t)(i & 1) + 32u * half, d);
@@ -690,7 +696,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           for (int e = 0; e < 4; ++e) {
             const int j = j4 + e, c = 32 * half + j;
             float pr = ex2(fmaf(t[j], p.scale_log2, -lq[e]));
-            if (edge && !(kj <= q0 + c && q0 + c < p.S)) pr = 0.f;
+            if (EDGE && !(kj <= q0 + c && q0 + c < p.S)) pr = 0.f;
             t[j] = pr;
             d[j] = pr * fmaf(d[j], p.inv_sqrt_d, nq[e]);
           }
@@ -705,7 +711,8 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
               make_uint4(pack2(d[8 * c4], d[8 * c4 + 1]), pack2(d[8 * c4 + 2], d[8 * c4 + 3]), pack2(d[8 * c4 + 4], d[8 * c4 + 5]),
                          pack2(d[8 * c4 + 6], d[8 * c4 + 7]));
         }
-      }
+      };
+      if (edge) item(std::true_type{}); else item(std::false_type{});
       fence_before();
       bar_arrive(bar_sfree(i & 1));
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
