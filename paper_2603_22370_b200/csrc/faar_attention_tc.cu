@@ -1,6 +1,7 @@
-// Causal attention forward for head_dim 64 on the tcgen05 tensor cores (sm_100a).
+// Causal attention for head_dim 64 on the tcgen05 tensor cores (sm_100a): the forward kernel first, then the two
+// backward kernels (dQ; dK and dV), which are built the same way and described where they start.
 //
-// One CTA takes 128 queries of one head and sweeps the keys in tiles of 64 (one sweep, running maximum):
+// Forward.  One CTA takes 128 queries of one head and sweeps the keys in tiles of 64 (one sweep, running maximum):
 //   S   = Q K_j^T       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 FP32 columns of tensor memory
 //   P_j = 2^(c S - m)   four warps, one query row per thread (its tensor-memory lane): no shuffles; the row
 //                       goes to shared memory as BF16 in the 128-byte-swizzled layout an A operand has
