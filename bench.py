@@ -574,6 +574,7 @@ def run_stage2(args, rt):
     faar.check_status(ctx, model.ws)
     ms_job = rt.timed(lambda: job(steps))
     faar.check_status(ctx, model.ws)
+    faar.attention_status(ctx)                      # the attention kernels' bounded waits report separately
     loss_final = model.loss.cpu().tolist()
 
     def profiled():
