@@ -94,6 +94,51 @@ def _attention_case(ctx, B, S, H, HKV, D):
     assert torch.equal(DQ2[:, :H * D], DQ[:, :H * D]) and torch.equal(DK2[:, :HKV * D], DK[:, :HKV * D])
 
 
+@pytest.mark.parametrize("fragments", [0, 2])
+def test_attention_at_the_alignment_benchmark_size_on_sampled_head_groups(ctx, fragments):
+    """4 sequences of 2048 tokens, 32 query / 8 key-value heads of 64 (the launch the full-model benchmark makes:
+    dense rows, 16 query tiles per head, CTAs ordered by work over the whole launch).  Attention separates over
+    (sequence, key/value head), so the oracle runs on three such groups, each with its 4 query heads, and every
+    output of those groups is compared."""
+    B, S, H, HKV, D = 4, 2048, 32, 8, 64
+    G = H // HKV
+    rng = np.random.default_rng(2048)
+    T = B * S
+    q = inputs.to_bf16_f32(rng.standard_normal((T, H * D)))
+    k = inputs.to_bf16_f32(rng.standard_normal((T, HKV * D)))
+    v = inputs.to_bf16_f32(rng.standard_normal((T, HKV * D)))
+    do = inputs.to_bf16_f32(rng.standard_normal((T, H * D)))
+    Q, K, V, DO = dev_bf16(q), dev_bf16(k), dev_bf16(v), dev_bf16(do)
+    O = torch.empty_like(Q)
+    lse = torch.zeros((B, H, S), dtype=torch.float32, device=DEV)
+    dsum = torch.zeros_like(lse)
+    DQ, DK, DV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    faar.tune_attention(ctx, fragments)
+    try:
+        faar.attention_fwd(ctx, B, S, H, HKV, D, Q, H * D, K, V, HKV * D, O, H * D, lse)
+        faar.attention_bwd(ctx, B, S, H, HKV, D, Q, H * D, K, V, HKV * D, O, DO, H * D, lse, dsum, DQ, DK, DV)
+        torch.cuda.synchronize()
+        faar.attention_status(ctx)
+    finally:
+        faar.tune_attention(ctx, 0)
+    got_o, got_dq = host(O).astype(np.float64), host(DQ).astype(np.float64)
+    got_dk, got_dv = host(DK).astype(np.float64), host(DV).astype(np.float64)
+    for (b, g) in [(0, 0), (3, 7), (1, 3)]:
+        rows = slice(b * S, (b + 1) * S)
+        qc, kc = slice(g * G * D, (g + 1) * G * D), slice(g * D, (g + 1) * D)
+        out_o, P = so.attention(q[rows, qc], k[rows, kc], v[rows, kc], 1, S, G, 1, D)
+        dq_o, dk_o, dv_o = so.attention_bwd(do[rows, qc], q[rows, qc], k[rows, kc], v[rows, kc], P, 1, S, G, 1, D)
+        a = got_o[rows, qc]
+        assert rel_l2(a, out_o) <= 6e-3 and max_rel_to_peak(a, out_o) <= 1e-2, (b, g)
+        for name, a, ref in (("dq", got_dq[rows, qc], dq_o), ("dk", got_dk[rows, kc], dk_o), ("dv", got_dv[rows, kc], dv_o)):
+            assert rel_l2(a, ref) <= 1e-2 and max_rel_to_peak(a, ref) <= 2e-2, (name, b, g, rel_l2(a, ref), max_rel_to_peak(a, ref))
+        # lse (log2 domain) of the group's last query head at the last position
+        h = (g + 1) * G - 1
+        sc = q[rows, qc][S - 1, (G - 1) * D:].astype(np.float64) @ k[rows, kc].astype(np.float64).T / np.sqrt(D)
+        ref = np.log2(np.sum(np.exp(sc - sc.max()))) + sc.max() * np.log2(np.e)
+        assert abs(float(lse[b, h, S - 1]) - ref) <= 1e-3 * max(1.0, abs(ref))
+
+
 def test_attention_argument_checks(ctx):
     x = torch.zeros((64, 128), dtype=torch.bfloat16, device=DEV)
     lse = torch.zeros(128, dtype=torch.float32, device=DEV)
