@@ -299,6 +299,16 @@ FAAR_API int faar_layer_dx(faar_ctx* ctx, const faar_shape* shape, float beta, c
                            const uint8_t* code, const uint8_t* scales, const float* s_global, void* WsoftT,
                            void* dX, void* workspace, size_t workspace_bytes);
 
+/* The same input gradient from soft weights that already exist: within one alignment step (Procedure steps
+ * 16-23) a layer's rounding variables change only in its own update, which follows its input gradient, so the
+ * BF16 soft weights its forward product was formed with (faar_softquant_eval's W_soft_bf16) are still the ones
+ * Eq. 2 gives, and dX = dY W_soft needs the GEMM alone.
+ *   dY    in : [T,O] bf16 (ldy, multiple of 8)      Wsoft in: [O,K] bf16 (row stride ldw, multiple of 8), read
+ *   dX    out: [T,K] bf16 (ldx, multiple of 8)                untransposed; caller-owned device memory
+ * Errors as faar_layer_dx (null pointer, shape, alignment, workspace too small). */
+FAAR_API int faar_layer_dx_operand(faar_ctx* ctx, const faar_shape* shape, const void* dY, const void* Wsoft,
+                                   void* dX, void* workspace, size_t workspace_bytes);
+
 /* ---- the MLP's gated product ---------------------------------------------------
  * Procedure step 1 runs Stage 1 "for each layer": the input of a block's down
  * projection is the frozen model's own activation silu(H W_gate^T) * (H W_up^T),

@@ -573,6 +573,26 @@ int faar_layer_dx(faar_ctx* ctx, const faar_shape* s, float beta, const void* dY
   return cuda_fail(ctx, faar_launch_gemm(ctx, &a, nullptr));
 }
 
+int faar_layer_dx_operand(faar_ctx* ctx, const faar_shape* s, const void* dY, const void* Wsoft, void* dX,
+                          void* workspace, size_t workspace_bytes) {
+  if (!ctx || !dY || !Wsoft || !dX) return FAAR_ERR_INVALID_ARG;
+  int st = check_shape(s);
+  if (st) return st;
+  if (s->ldy < s->O || s->ldx < s->K || s->ldw < s->K) return FAAR_ERR_SHAPE;
+  if (s->ldy % 8 || s->ldx % 8 || s->ldw % 8 || !aligned16(dY) || !aligned16(Wsoft) || !aligned16(dX)) return FAAR_ERR_ALIGN;
+  if ((st = check_ws(s, workspace, workspace_bytes))) return st;
+  FAAR_DEVICE_GUARD(ctx);
+  // dX^T[K,T] = W_soft^T[K,O] * dY[T,O]^T written transposed as dX[T,K], as in faar_layer_dx
+  faar_gemm_args a = {};
+  a.mode = FAAR_GEMM_REF;
+  a.M = s->K; a.N = s->T; a.Kc = s->O;
+  a.A = Wsoft; a.lda = s->ldw; a.a_mn = 1;
+  a.B = dY; a.ldb = s->ldy;
+  a.status = reinterpret_cast<uint32_t*>(workspace);
+  a.Yout = dX; a.yout_dtype = FAAR_BF16; a.ldy = s->ldx;
+  return cuda_fail(ctx, faar_launch_gemm(ctx, &a, nullptr));
+}
+
 int faar_layer_fwd(faar_ctx* ctx, const faar_shape* s, const faar_hparams* hp, const void* X, const void* Y_ref,
                    const float* V, const uint8_t* code, const uint8_t* scales, const float* s_global, void* dYt,
                    float* loss_mse, void* Y_q, void* workspace, size_t workspace_bytes) {

@@ -45,6 +45,7 @@ SIGNATURES = {
     "faar_layer_ref": (_I, [_P, _P, _P, _P, _P, _P, _Z]),
     "faar_layer_fwd": (_I, [_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
     "faar_layer_dx": (_I, [_P, _P, _F, _P, _P, _P, _P, _P, _P, _P, _P, _Z]),
+    "faar_layer_dx_operand": (_I, [_P, _P, _P, _P, _P, _P, _Z]),
     "faar_round_loss": (_I, [_P, _P, _L, _P, _P, _Z]),
     "faar_round_loss_static": (_I, [_P, _P, _L, _P]),
     "faar_round_loss_static_max_n": (_L, []),
@@ -349,6 +350,11 @@ def layer_fwd(ctx, shape, hp, X, Y_ref, V, code, scales, s_global, dYt, loss_mse
 def layer_dx(ctx, shape, beta, dY, V, code, scales, s_global, WsoftT, dX, ws):
     _check(lib().faar_layer_dx(ctx._h, C.byref(shape), C.c_float(beta), _p(dY), _p(V), _p(code), _p(scales),
                                _p(s_global), _p(WsoftT), _p(dX), _p(ws), C.c_size_t(ws.numel())), "faar_layer_dx")
+
+
+def layer_dx_operand(ctx, shape, dY, Wsoft, dX, ws):
+    _check(lib().faar_layer_dx_operand(ctx._h, C.byref(shape), _p(dY), _p(Wsoft), _p(dX), _p(ws), C.c_size_t(ws.numel())),
+           "faar_layer_dx_operand")
 
 
 def round_loss(ctx, V, N, loss_round, ws):

@@ -7,8 +7,8 @@ One step (`Stage2Model.step`):
   frozen model forward (BF16 weights)                      -> Z_fp, H_fp            Procedure 16
   quantised model forward (Eq. 2 soft weights of every V)  -> Z_q, H_q, activations Procedure 17
   faar_align_loss                                          -> L_KL, L_MSE, dZ_q, dH_q   Procedure 18-20, Eq. 6
-  backward through the quantised model; per linear: input gradient dX = dY W_soft (faar_layer_dx, at the
-  pre-update V), then dW GEMM + chain rule + Round Loss gradient + optimiser update + clip (faar_layer_bwd)
+  backward through the quantised model; per linear: input gradient dX = dY W_soft (faar_layer_dx_operand on the
+  forward pass's soft weights, i.e. at the pre-update V), then dW GEMM + chain rule + Round Loss gradient + optimiser update + clip (faar_layer_bwd)
                                                                                      Procedure 21-23
 Embedding, norms and LM head are frozen and stay in BF16 / FP32; the seven linears of every block are quantised.
 """
@@ -149,7 +149,8 @@ class Stage2Model:
         O, K = lin.O, lin.K
         shape = faar.make_shape(O, K, T, ldxt=self.ldt)
         dX = self._new(K)
-        faar.layer_dx(ctx, shape, hp.beta, dY, lin.V, lin.code, lin.scales, lin.s_global, None, dX, self.ws)
+        # lin.Wsoft still holds this step's soft weights: V changes only in the update below
+        faar.layer_dx_operand(ctx, shape, dY, lin.Wsoft, dX, self.ws)
         dV = torch.empty((O, K), dtype=torch.float32, device=self.dev) if want_dv else None
         # dY [T, O] and X [T, K] as the backward pass holds them: no transposed copies
         faar.layer_bwd_rowmajor(ctx, shape, hp, dY, X, lin.V, lin.code, lin.scales, lin.s_global, lin.m, lin.u, dV, self.ws)
@@ -157,6 +158,7 @@ class Stage2Model:
 
     def backward(self, dZ, dH, saved, hp, want_dv=False):
         """From the loss gradients at the logits and at the last hidden state back to every V (updated in place).
+        Follows the quantised forward pass of the same step: every linear's Wsoft buffer is read as that pass left it.
         Returns {(l, name): dV} if want_dv."""
         c, ctx, T = self.cfg, self.ctx, self.T
         d, qd, kvd, f = c.hidden, c.n_heads * c.head_dim, c.n_kv_heads * c.head_dim, c.ffn

@@ -910,6 +910,16 @@ def test_layer_dx(ctx, O, K, T):
     lay.check()
     dX_o = fo.layer_dx(dY, V, host(lay.code), host(lay.scales), host(lay.s_global)[0], beta, "bf16")
     assert rel_l2(host(dX), dX_o) <= 3e-3 and max_rel_to_peak(host(dX), dX_o) <= 4e-3     # BF16 output: 2^-8 rounding
+    # the same product from soft weights formed beforehand (what an alignment step's forward pass leaves): same bits
+    Wsoft = torch.empty((O, K), dtype=torch.bfloat16, device=DEV)
+    faar.softquant_eval(ctx, lay.shape, lay.V, lay.code, lay.scales, lay.s_global, beta, None, None, Wsoft)
+    dX2 = torch.full((T, K), 3.0, dtype=torch.bfloat16, device=DEV)
+    faar.layer_dx_operand(ctx, lay.shape, dYd, Wsoft, dX2, lay.ws)
+    lay.check()
+    assert torch.equal(dX2, dX)
+    with pytest.raises(faar.FaarError) as e:
+        faar.layer_dx_operand(ctx, lay.shape, dYd, None, dX2, lay.ws)
+    assert e.value.status == faar.ERR_INVALID_ARG
 
 
 @pytest.mark.parametrize("yref_dtype", [faar.BF16, faar.F32])
