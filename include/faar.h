@@ -481,6 +481,12 @@ FAAR_API int faar_swizzle_scales(faar_ctx* ctx, int rows, int cols, const uint8_
  * faar_rmsnorm_bwd: gradient towards x (g is frozen): dx = rstd * (g dy - xh * mean(g dy xh)), xh = x rstd;
  *   `add` ([rows, cols] bf16, ldadd; nullable) is added to it: the gradient that reaches x past the norm, along
  *   the residual connection.  dx may alias add.
+ * faar_add_rmsnorm: a residual connection followed by the next norm in one pass: sum = a + b (rounded to BF16
+ *   and stored, [rows, cols] bf16, lds), y = rmsnorm(sum) from the rounded values, i.e. the results of faar_add
+ *   followed by faar_rmsnorm bit for bit.  sum may alias a or b.
+ * faar_rmsnorm_bwd_sum: faar_rmsnorm_bwd with dy = dy + dy2 + dy3 formed in FP32 (the gradients of the linears
+ *   that read the norm's output meet here: q / k / v, gate / up); dy2, dy3 nullable ([rows, cols] bf16, same
+ *   leading dimension lddy; dy3 without dy2 is FAAR_ERR_INVALID_ARG).
  * faar_rope: rotary position embedding, half-split pairing: in every head, element i < head_dim/2 pairs with
  *   element i + head_dim/2 and the pair of row t turns by positions[t] * theta^(-2 i / head_dim); inverse != 0
  *   turns the other way (the backward pass).  x, y: [rows, n_heads * head_dim]; y may alias x; head_dim % 16 == 0.
@@ -492,6 +498,11 @@ FAAR_API int faar_rmsnorm(faar_ctx* ctx, int rows, int cols, const void* x, int6
                           int64_t ldy, float* rstd);
 FAAR_API int faar_rmsnorm_bwd(faar_ctx* ctx, int rows, int cols, const void* dy, int64_t lddy, const void* x, int64_t ldx,
                               const float* g, const float* rstd, const void* add, int64_t ldadd, void* dx, int64_t lddx);
+FAAR_API int faar_add_rmsnorm(faar_ctx* ctx, int rows, int cols, const void* a, int64_t lda, const void* b, int64_t ldb,
+                              void* sum, int64_t lds, const float* g, float eps, void* y, int64_t ldy, float* rstd);
+FAAR_API int faar_rmsnorm_bwd_sum(faar_ctx* ctx, int rows, int cols, const void* dy, const void* dy2, const void* dy3,
+                                  int64_t lddy, const void* x, int64_t ldx, const float* g, const float* rstd,
+                                  const void* add, int64_t ldadd, void* dx, int64_t lddx);
 FAAR_API int faar_rope(faar_ctx* ctx, int rows, int n_heads, int head_dim, const void* x, int64_t ldx, const int* positions,
                        float theta, int inverse, void* y, int64_t ldy);
 FAAR_API int faar_silu_mul_bwd(faar_ctx* ctx, int rows, int cols, const void* dout, int64_t ldd, const void* gate,

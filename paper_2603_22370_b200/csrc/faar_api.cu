@@ -851,7 +851,17 @@ int faar_rmsnorm(faar_ctx* ctx, int rows, int cols, const void* x, int64_t ldx, 
   int st = check_rows_cols(rows, cols, {ldx, ldy}, {x, g, y});
   if (st) return st;
   FAAR_DEVICE_GUARD(ctx);
-  return cuda_fail(ctx, faar_launch_rmsnorm(ctx, rows, cols, x, ldx, g, eps, y, ldy, rstd));
+  return cuda_fail(ctx, faar_launch_rmsnorm(ctx, rows, cols, x, ldx, nullptr, 0, nullptr, 0, g, eps, y, ldy, rstd));
+}
+
+int faar_add_rmsnorm(faar_ctx* ctx, int rows, int cols, const void* a, int64_t lda, const void* b, int64_t ldb, void* sum,
+                     int64_t lds, const float* g, float eps, void* y, int64_t ldy, float* rstd) {
+  if (!ctx || !a || !b || !sum || !g || !y) return FAAR_ERR_INVALID_ARG;
+  if (!(eps >= 0.f) || !isfinite(eps)) return FAAR_ERR_INVALID_ARG;
+  int st = check_rows_cols(rows, cols, {lda, ldb, lds, ldy}, {a, b, sum, g, y});
+  if (st) return st;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_rmsnorm(ctx, rows, cols, a, lda, b, ldb, sum, lds, g, eps, y, ldy, rstd));
 }
 
 int faar_rmsnorm_bwd(faar_ctx* ctx, int rows, int cols, const void* dy, int64_t lddy, const void* x, int64_t ldx,
@@ -861,7 +871,19 @@ int faar_rmsnorm_bwd(faar_ctx* ctx, int rows, int cols, const void* dy, int64_t 
   if (st) return st;
   if (add && (ldadd < cols || ldadd % 8)) return ldadd < cols ? FAAR_ERR_SHAPE : FAAR_ERR_ALIGN;
   FAAR_DEVICE_GUARD(ctx);
-  return cuda_fail(ctx, faar_launch_rmsnorm_bwd(ctx, rows, cols, dy, lddy, x, ldx, g, rstd, add, ldadd, dx, lddx));
+  return cuda_fail(ctx, faar_launch_rmsnorm_bwd(ctx, rows, cols, dy, nullptr, nullptr, lddy, x, ldx, g, rstd, add, ldadd, dx, lddx));
+}
+
+int faar_rmsnorm_bwd_sum(faar_ctx* ctx, int rows, int cols, const void* dy, const void* dy2, const void* dy3, int64_t lddy,
+                         const void* x, int64_t ldx, const float* g, const float* rstd, const void* add, int64_t ldadd,
+                         void* dx, int64_t lddx) {
+  if (!ctx || !dy || !x || !g || !rstd || !dx) return FAAR_ERR_INVALID_ARG;
+  if (dy3 && !dy2) return FAAR_ERR_INVALID_ARG;
+  int st = check_rows_cols(rows, cols, {lddy, ldx, lddx}, {dy, dy2, dy3, x, g, dx, add});
+  if (st) return st;
+  if (add && (ldadd < cols || ldadd % 8)) return ldadd < cols ? FAAR_ERR_SHAPE : FAAR_ERR_ALIGN;
+  FAAR_DEVICE_GUARD(ctx);
+  return cuda_fail(ctx, faar_launch_rmsnorm_bwd(ctx, rows, cols, dy, dy2, dy3, lddy, x, ldx, g, rstd, add, ldadd, dx, lddx));
 }
 
 int faar_rope(faar_ctx* ctx, int rows, int n_heads, int head_dim, const void* x, int64_t ldx, const int* positions,

@@ -112,10 +112,11 @@ int faar_launch_align_loss(faar_ctx*, int T, int vocab, int hidden, const void* 
                            void* dH_q, float* kl_partials, float* mse_partials, int* n_partials);
 int faar_launch_silu_mul(faar_ctx*, int rows, int cols, const void* gate, int64_t ldg, const void* up, int64_t ldu,
                          void* out, int64_t ldo);
-int faar_launch_rmsnorm(faar_ctx*, int rows, int cols, const void* x, int64_t ldx, const float* g, float eps, void* y,
-                        int64_t ldy, float* rstd);
-int faar_launch_rmsnorm_bwd(faar_ctx*, int rows, int cols, const void* dy, int64_t lddy, const void* x, int64_t ldx,
-                            const float* g, const float* rstd, const void* add, int64_t ldadd, void* dx, int64_t lddx);
+int faar_launch_rmsnorm(faar_ctx*, int rows, int cols, const void* x, int64_t ldx, const void* b, int64_t ldb,
+                        void* sum_out, int64_t lds, const float* g, float eps, void* y, int64_t ldy, float* rstd);
+int faar_launch_rmsnorm_bwd(faar_ctx*, int rows, int cols, const void* dy, const void* dy2, const void* dy3, int64_t lddy,
+                            const void* x, int64_t ldx, const float* g, const float* rstd, const void* add, int64_t ldadd,
+                            void* dx, int64_t lddx);
 int faar_launch_rope(faar_ctx*, int rows, int n_heads, int head_dim, const void* x, int64_t ldx, const int* pos, float theta,
                      int inverse, void* y, int64_t ldy);
 int faar_launch_silu_mul_bwd(faar_ctx*, int rows, int cols, const void* dout, int64_t ldd, const void* gate, int64_t ldg,

@@ -62,6 +62,8 @@ SIGNATURES = {
     "faar_silu_mul": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L]),
     "faar_rmsnorm": (_I, [_P, _I, _I, _P, _L, _P, _F, _P, _L, _P]),
     "faar_rmsnorm_bwd": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _P, _P, _L, _P, _L]),
+    "faar_add_rmsnorm": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L, _P, _F, _P, _L, _P]),
+    "faar_rmsnorm_bwd_sum": (_I, [_P, _I, _I, _P, _P, _P, _L, _P, _L, _P, _P, _P, _L, _P, _L]),
     "faar_rope": (_I, [_P, _I, _I, _I, _P, _L, _P, _F, _I, _P, _L]),
     "faar_silu_mul_bwd": (_I, [_P, _I, _I, _P, _L, _P, _L, _P, _L, _P, _L, _P, _L]),
     "faar_embedding": (_I, [_P, _I, _I, _I, _P, _L, _P, _P, _L]),
@@ -279,6 +281,17 @@ def rmsnorm(ctx, rows, cols, x, ldx, g, eps, y, ldy, rstd=None):
 def rmsnorm_bwd(ctx, rows, cols, dy, lddy, x, ldx, g, rstd, add, ldadd, dx, lddx):
     _check(lib().faar_rmsnorm_bwd(ctx._h, rows, cols, _p(dy), lddy, _p(x), ldx, _p(g), _p(rstd), _p(add), ldadd, _p(dx), lddx),
            "faar_rmsnorm_bwd")
+
+
+def add_rmsnorm(ctx, rows, cols, a, lda, b, ldb, total, lds, g, eps, y, ldy, rstd=None):
+    _check(lib().faar_add_rmsnorm(ctx._h, rows, cols, _p(a), C.c_int64(lda), _p(b), C.c_int64(ldb), _p(total), C.c_int64(lds),
+                                  _p(g), C.c_float(eps), _p(y), C.c_int64(ldy), _p(rstd)), "faar_add_rmsnorm")
+
+
+def rmsnorm_bwd_sum(ctx, rows, cols, dy, dy2, dy3, lddy, x, ldx, g, rstd, add, ldadd, dx, lddx):
+    _check(lib().faar_rmsnorm_bwd_sum(ctx._h, rows, cols, _p(dy), _p(dy2), _p(dy3), C.c_int64(lddy), _p(x), C.c_int64(ldx),
+                                      _p(g), _p(rstd), _p(add), C.c_int64(ldadd), _p(dx), C.c_int64(lddx)),
+           "faar_rmsnorm_bwd_sum")
 
 
 def rope(ctx, rows, n_heads, head_dim, x, ldx, positions, theta, inverse, y, ldy):

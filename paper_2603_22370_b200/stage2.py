@@ -112,10 +112,10 @@ class Stage2Model:
         x = self._new(d)
         faar.embedding(ctx, T, d, c.vocab, self.params["embed"], d, tokens, x, d)
         cache = []
+        hn, rstd1 = self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
+        faar.rmsnorm(ctx, T, d, x, d, self.params["attn_norm.0"], c.eps, hn, d, rstd1)
         for l in range(c.n_layers):
-            s = {"x_in": x}
-            hn, s["rstd1"] = self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
-            faar.rmsnorm(ctx, T, d, x, d, self.params[f"attn_norm.{l}"], c.eps, hn, d, s["rstd1"])
+            s = {"x_in": x, "rstd1": rstd1}
             q, k, v = (self._linear(l, n, hn, quantised, beta) for n in ("q_proj", "k_proj", "v_proj"))
             faar.rope(ctx, T, c.n_heads, c.head_dim, q, qd, self.pos, c.theta, 0, q, qd)
             faar.rope(ctx, T, c.n_kv_heads, c.head_dim, k, kvd, self.pos, c.theta, 0, k, kvd)
@@ -123,21 +123,21 @@ class Stage2Model:
             lse = torch.empty((self.batch, c.n_heads, self.seq), dtype=torch.float32, device=self.dev)
             faar.attention_fwd(ctx, self.batch, self.seq, c.n_heads, c.n_kv_heads, c.head_dim, q, qd, k, v, kvd, a, qd, lse)
             o = self._linear(l, "o_proj", a, quantised, beta)
-            x_mid = self._new(d)
-            faar.add(ctx, T, d, x, d, o, d, x_mid, d)
-            mn, s["rstd2"] = self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
-            faar.rmsnorm(ctx, T, d, x_mid, d, self.params[f"mlp_norm.{l}"], c.eps, mn, d, s["rstd2"])
+            # residual connection and the MLP's norm in one pass
+            x_mid, mn, s["rstd2"] = self._new(d), self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
+            faar.add_rmsnorm(ctx, T, d, x, d, o, d, x_mid, d, self.params[f"mlp_norm.{l}"], c.eps, mn, d, s["rstd2"])
             g, u = self._linear(l, "gate_proj", mn, quantised, beta), self._linear(l, "up_proj", mn, quantised, beta)
             act = self._new(f)
             faar.silu_mul(ctx, T, f, g, f, u, f, act, f)
             dn = self._linear(l, "down_proj", act, quantised, beta)
-            x = self._new(d)
-            faar.add(ctx, T, d, x_mid, d, dn, d, x, d)
             if keep:
                 s.update(hn=hn, q=q, k=k, v=v, a=a, lse=lse, x_mid=x_mid, mn=mn, g=g, u=u, act=act)
                 cache.append(s)
-        H, rstd_f = self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
-        faar.rmsnorm(ctx, T, d, x, d, self.params["final_norm"], c.eps, H, d, rstd_f)
+            # residual connection and the next block's attention norm (after the last block: the final norm)
+            g_next = self.params[f"attn_norm.{l + 1}"] if l + 1 < c.n_layers else self.params["final_norm"]
+            x, hn, rstd1 = self._new(d), self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
+            faar.add_rmsnorm(ctx, T, d, x_mid, d, dn, d, x, d, g_next, c.eps, hn, d, rstd1)
+        H, rstd_f = hn, rstd1
         Z = self._matmul(H, self.params["lm_head"])
         return Z, H, ((cache, x, rstd_f) if keep else None)
 
@@ -168,9 +168,8 @@ class Stage2Model:
         dHz = self._new(d)
         faar.layer_ref(ctx, faar.make_shape(d, self.lm_head_t.shape[1], T, ldw=self.lm_head_t.shape[1], ldx=dZ.shape[1]), dZ,
                        self.lm_head_t, dHz, self.ws)
-        faar.add(ctx, T, d, dHz, d, dH, d, dHz, d)
         dx = self._new(d)
-        faar.rmsnorm_bwd(ctx, T, d, dHz, d, x_last, d, self.params["final_norm"], rstd_f, None, d, dx, d)
+        faar.rmsnorm_bwd_sum(ctx, T, d, dHz, dH, None, d, x_last, d, self.params["final_norm"], rstd_f, None, d, dx, d)
         for l in reversed(range(c.n_layers)):
             s = cache[l]
             # MLP branch: x = x_mid + act W_down^T
@@ -179,8 +178,9 @@ class Stage2Model:
             faar.silu_mul_bwd(ctx, T, f, dact, f, s["g"], f, s["u"], f, dg, f, du, f)
             dmn, grads[(l, "gate_proj")] = self._linear_bwd(l, "gate_proj", dg, s["mn"], hp, want_dv)
             dmn2, grads[(l, "up_proj")] = self._linear_bwd(l, "up_proj", du, s["mn"], hp, want_dv)
-            faar.add(ctx, T, d, dmn, d, dmn2, d, dmn, d)
-            faar.rmsnorm_bwd(ctx, T, d, dmn, d, s["x_mid"], d, self.params[f"mlp_norm.{l}"], s["rstd2"], dx, d, dx, d)
+            # the two gradients that meet at the norm's output are summed inside its backward
+            faar.rmsnorm_bwd_sum(ctx, T, d, dmn, dmn2, None, d, s["x_mid"], d, self.params[f"mlp_norm.{l}"], s["rstd2"], dx, d,
+                                 dx, d)
             # attention branch: x_mid = x_in + a W_o^T
             da, grads[(l, "o_proj")] = self._linear_bwd(l, "o_proj", dx, s["a"], hp, want_dv)
             dq, dk, dv = self._new(qd), self._new(kvd), self._new(kvd)
@@ -191,9 +191,8 @@ class Stage2Model:
             dhn, grads[(l, "q_proj")] = self._linear_bwd(l, "q_proj", dq, s["hn"], hp, want_dv)
             dhk, grads[(l, "k_proj")] = self._linear_bwd(l, "k_proj", dk, s["hn"], hp, want_dv)
             dhv, grads[(l, "v_proj")] = self._linear_bwd(l, "v_proj", dv, s["hn"], hp, want_dv)
-            faar.add(ctx, T, d, dhn, d, dhk, d, dhn, d)
-            faar.add(ctx, T, d, dhn, d, dhv, d, dhn, d)
-            faar.rmsnorm_bwd(ctx, T, d, dhn, d, s["x_in"], d, self.params[f"attn_norm.{l}"], s["rstd1"], dx, d, dx, d)
+            faar.rmsnorm_bwd_sum(ctx, T, d, dhn, dhk, dhv, d, s["x_in"], d, self.params[f"attn_norm.{l}"], s["rstd1"], dx, d,
+                                 dx, d)
         return grads if want_dv else None
 
     # ---- one step of Eq. 6 -----------------------------------------------------------------------------

@@ -35,7 +35,7 @@ def close_bf16(got, ref, extra_abs=0.0):
     return np.all(np.abs(got - ref) <= (BF16_HALF_STEP + 1e-5) * np.abs(ref) + extra_abs + 1e-30)
 
 
-@pytest.mark.parametrize("rows,cols,ld", [(77, 136, 144), (5, 2048, 2048), (300, 8, 8)])
+@pytest.mark.parametrize("rows,cols,ld", [(77, 136, 144), (5, 2048, 2048), (300, 8, 8), (9, 2056, 2064), (3, 4096, 4096)])
 def test_rmsnorm_forward_and_backward(ctx, rows, cols, ld):
     rng = np.random.default_rng(rows)
     x = inputs.to_bf16_f32(rng.standard_normal((rows, cols)) * 2)
@@ -73,7 +73,66 @@ def test_rmsnorm_forward_and_backward(ctx, rows, cols, ld):
     assert torch.equal(R[:, :cols], DX[:, :cols])
 
 
-@pytest.mark.parametrize("n_heads,head_dim", [(3, 16), (8, 64), (2, 128)])
+@pytest.mark.parametrize("rows,cols,ld", [(77, 136, 144), (40, 2048, 2048), (9, 2056, 2064), (3, 4096, 4096)])
+def test_residual_add_fused_with_the_norm_and_gradient_sums_inside_its_backward(ctx, rows, cols, ld):
+    """Rows of up to 2048 elements stay in registers, longer ones are read twice: both forms, ragged widths."""
+    rng = np.random.default_rng(cols + rows)
+    a = inputs.to_bf16_f32(rng.standard_normal((rows, cols)) * 2)
+    b = inputs.to_bf16_f32(rng.standard_normal((rows, cols)))
+    g = inputs.to_bf16_f32(rng.uniform(0.5, 1.5, cols)).astype(np.float32)
+    eps = float(np.float32(1e-5))
+    A, B, G = padded(a, ld), padded(b, ld), dev_f32(g)
+    # forward: the same bits as faar_add followed by faar_rmsnorm
+    S1 = torch.full((rows, ld), 5.0, dtype=torch.bfloat16, device=DEV)
+    Y1 = torch.full((rows, ld), 5.0, dtype=torch.bfloat16, device=DEV)
+    r1 = torch.zeros(rows, dtype=torch.float32, device=DEV)
+    faar.add(ctx, rows, cols, A, ld, B, ld, S1, ld)
+    faar.rmsnorm(ctx, rows, cols, S1, ld, G, eps, Y1, ld, r1)
+    S2, Y2, r2 = torch.full_like(S1, 5.0), torch.full_like(Y1, 5.0), torch.zeros_like(r1)
+    faar.add_rmsnorm(ctx, rows, cols, A, ld, B, ld, S2, ld, G, eps, Y2, ld, r2)
+    torch.cuda.synchronize()
+    assert torch.equal(S2, S1) and torch.equal(Y2, Y1) and torch.equal(r2, r1)
+    # ... and against the oracle: the sum is one BF16 rounding of a + b, the norm is taken of the rounded sum
+    s_o = a.astype(np.float64) + b.astype(np.float64)
+    assert close_bf16(host(S2[:, :cols]).astype(np.float64), s_o, extra_abs=1e-37)
+    y_o, rstd_o = so.rmsnorm(host(S2[:, :cols]).astype(np.float64), g, eps)
+    assert np.allclose(host(r2), rstd_o, rtol=2e-6) and close_bf16(host(Y2[:, :cols]).astype(np.float64), y_o)
+    A2 = A.clone()
+    faar.add_rmsnorm(ctx, rows, cols, A2, ld, B, ld, A2, ld, G, eps, Y2, ld, None)     # sum in place, no rstd wanted
+    torch.cuda.synchronize()
+    assert torch.equal(A2[:, :cols], S1[:, :cols]) and torch.equal(Y2, Y1)
+
+    # backward with one, two and three gradients meeting at the norm's output
+    x = host(S1[:, :cols]).astype(np.float64)
+    dys = [inputs.to_bf16_f32(rng.standard_normal((rows, cols))) for _ in range(3)]
+    res = inputs.to_bf16_f32(rng.standard_normal((rows, cols)))
+    D = [padded(t, ld) for t in dys]
+    R = padded(res, ld)
+    r64 = host(r1).astype(np.float64)[:, None]
+    for n in (1, 2, 3):
+        for add in (None, R):
+            DX = torch.full((rows, ld), 5.0, dtype=torch.bfloat16, device=DEV)
+            faar.rmsnorm_bwd_sum(ctx, rows, cols, D[0], D[1] if n > 1 else None, D[2] if n > 2 else None, ld, S1, ld, G, r1,
+                                 add, ld, DX, ld)
+            torch.cuda.synchronize()
+            dy = sum(t.astype(np.float64) for t in dys[:n])
+            ref = so.rmsnorm_bwd(dy, x, g, r64[:, 0]) + (res if add is not None else 0.0)
+            w, xh = dy * g, x * r64
+            terms = r64 * (np.abs(w) + np.abs(xh) * np.abs(np.mean(w * xh, axis=1, keepdims=True))) + (np.abs(res) if add is not None else 0.0)
+            got = host(DX[:, :cols]).astype(np.float64)
+            assert np.all(np.abs(got - ref) <= BF16_HALF_STEP * np.abs(ref) + 1e-5 * terms + 1e-30), (n, add is not None)
+            assert torch.all(DX[:, cols:] == 5.0)
+            if n == 1:
+                DX1 = torch.full_like(DX, 5.0)
+                faar.rmsnorm_bwd(ctx, rows, cols, D[0], ld, S1, ld, G, r1, add, ld, DX1, ld)
+                torch.cuda.synchronize()
+                assert torch.equal(DX1, DX)
+    with pytest.raises(faar.FaarError) as e:
+        faar.rmsnorm_bwd_sum(ctx, rows, cols, D[0], None, D[2], ld, S1, ld, G, r1, None, ld, DX, ld)
+    assert e.value.status == faar.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("n_heads,head_dim", [(3, 16), (8, 64), (2, 128), (12, 64), (4, 128)])
 def test_rope_forward_inverse_and_in_place(ctx, n_heads, head_dim):
     rng = np.random.default_rng(head_dim)
     T = 50
