@@ -21,6 +21,7 @@ import torch
 from . import faar
 
 LINEARS = ("q_proj", "k_proj", "v_proj", "o_proj", "gate_proj", "up_proj", "down_proj")
+GROUPS = {"qkv": ("q_proj", "k_proj", "v_proj"), "gate_up": ("gate_proj", "up_proj")}      # linears with a common input
 
 
 @dataclass
@@ -45,7 +46,7 @@ class QuantLinear:
     """Device state of one quantised linear: frozen W, its NVFP4 bracket (scales, code, tensor scale), the
     rounding tensor V with its Adam moments, and a BF16 buffer for the soft weights of the current step."""
 
-    def __init__(self, ctx: faar.Context, W: torch.Tensor, ws: torch.Tensor, opt: int = 1):
+    def __init__(self, ctx: faar.Context, W: torch.Tensor, ws: torch.Tensor, opt: int = 1, Wsoft: torch.Tensor | None = None):
         O, K = W.shape
         dev = W.device
         self.W, self.O, self.K = W, O, K
@@ -55,7 +56,7 @@ class QuantLinear:
         self.V = torch.empty((O, K), dtype=torch.float32, device=dev)
         self.m = torch.zeros((O, K), dtype=torch.float32, device=dev) if opt == 1 else None
         self.u = torch.zeros((O, K), dtype=torch.float32, device=dev) if opt == 1 else None
-        self.Wsoft = torch.empty((O, K), dtype=torch.bfloat16, device=dev)
+        self.Wsoft = Wsoft if Wsoft is not None else torch.empty((O, K), dtype=torch.bfloat16, device=dev)
         faar.softquant_init(ctx, faar.make_shape(O, K, 8), W, 0.0, self.scales, self.s_global, self.code, self.V, ws)
 
 
@@ -70,11 +71,31 @@ class Stage2Model:
         dev = params["embed"].device
         self.dev = dev
         T, c = self.T, cfg
-        big = max(o * k for o, k in c.linear_shapes().values())
-        self.ws = torch.empty(max(faar.workspace_size(faar.make_shape(o, k, T)) for o, k in c.linear_shapes().values()),
-                              dtype=torch.uint8, device=dev)
+        shapes = c.linear_shapes()
+        # q / k / v read the same input, and so do gate / up: each group is one matrix product over the stacked
+        # weights (forward) and one input-gradient product over the stacked output gradients (backward)
+        self.group_rows = {g: [shapes[n][0] for n in names] for g, names in GROUPS.items()}
+        ws_shapes = list(shapes.values()) + [(sum(self.group_rows[g]), shapes[names[0]][1]) for g, names in GROUPS.items()]
+        self.ws = torch.empty(max(faar.workspace_size(faar.make_shape(o, k, T)) for o, k in ws_shapes), dtype=torch.uint8,
+                              device=dev)
         faar.workspace_init(ctx, self.ws)
-        self.lin = [{n: QuantLinear(ctx, weights[l][n], self.ws, opt) for n in LINEARS} for l in range(c.n_layers)]
+        self.lin, self.w_group, self.wsoft_group = [], [], []
+        for l in range(c.n_layers):
+            lins, wg, wsg = {}, {}, {}
+            for g, names in GROUPS.items():
+                wg[g] = torch.cat([weights[l][n] for n in names], dim=0).contiguous()
+                wsg[g] = torch.empty_like(wg[g])
+                r0 = 0
+                for n in names:
+                    r1 = r0 + shapes[n][0]
+                    lins[n] = QuantLinear(ctx, wg[g][r0:r1], self.ws, opt, Wsoft=wsg[g][r0:r1])
+                    r0 = r1
+            for n in LINEARS:
+                if n not in lins:
+                    lins[n] = QuantLinear(ctx, weights[l][n], self.ws, opt)
+            self.lin.append(lins)
+            self.w_group.append(wg)
+            self.wsoft_group.append(wsg)
         self.pos = torch.arange(seq, dtype=torch.int32, device=dev).repeat(batch)
         self.lm_head_t = torch.empty((c.hidden, (c.vocab + 7) // 8 * 8), dtype=torch.bfloat16, device=dev)
         faar.transpose_bf16(ctx, c.vocab, c.hidden, params["lm_head"], c.hidden, self.lm_head_t, self.lm_head_t.shape[1])
@@ -96,6 +117,17 @@ class Stage2Model:
         faar.layer_ref(self.ctx, faar.make_shape(O, K, self.T), X, W, Y, self.ws)
         return Y
 
+    def _linear_group(self, l, group, X, quantised, beta):
+        """The linears of one group on their common input: one product with the stacked weights.  Returns the
+        [T, sum of widths] result; each linear's output is a column range of it."""
+        if not quantised:
+            return self._matmul(X, self.w_group[l][group])
+        for n in GROUPS[group]:
+            lin = self.lin[l][n]
+            faar.softquant_eval(self.ctx, faar.make_shape(lin.O, lin.K, self.T), lin.V, lin.code, lin.scales, lin.s_global,
+                                beta, None, None, lin.Wsoft)
+        return self._matmul(X, self.wsoft_group[l][group])
+
     def _linear(self, l, name, X, quantised, beta):
         lin = self.lin[l][name]
         if not quantised:
@@ -116,19 +148,22 @@ class Stage2Model:
         faar.rmsnorm(ctx, T, d, x, d, self.params["attn_norm.0"], c.eps, hn, d, rstd1)
         for l in range(c.n_layers):
             s = {"x_in": x, "rstd1": rstd1}
-            q, k, v = (self._linear(l, n, hn, quantised, beta) for n in ("q_proj", "k_proj", "v_proj"))
-            faar.rope(ctx, T, c.n_heads, c.head_dim, q, qd, self.pos, c.theta, 0, q, qd)
-            faar.rope(ctx, T, c.n_kv_heads, c.head_dim, k, kvd, self.pos, c.theta, 0, k, kvd)
+            qkv = self._linear_group(l, "qkv", hn, quantised, beta)
+            ldp = qkv.shape[1]
+            q, k, v = qkv[:, :qd], qkv[:, qd:qd + kvd], qkv[:, qd + kvd:]
+            faar.rope(ctx, T, c.n_heads, c.head_dim, q, ldp, self.pos, c.theta, 0, q, ldp)
+            faar.rope(ctx, T, c.n_kv_heads, c.head_dim, k, ldp, self.pos, c.theta, 0, k, ldp)
             a = self._new(qd)
             lse = torch.empty((self.batch, c.n_heads, self.seq), dtype=torch.float32, device=self.dev)
-            faar.attention_fwd(ctx, self.batch, self.seq, c.n_heads, c.n_kv_heads, c.head_dim, q, qd, k, v, kvd, a, qd, lse)
+            faar.attention_fwd(ctx, self.batch, self.seq, c.n_heads, c.n_kv_heads, c.head_dim, q, ldp, k, v, ldp, a, qd, lse)
             o = self._linear(l, "o_proj", a, quantised, beta)
             # residual connection and the MLP's norm in one pass
             x_mid, mn, s["rstd2"] = self._new(d), self._new(d), torch.empty(T, dtype=torch.float32, device=self.dev)
             faar.add_rmsnorm(ctx, T, d, x, d, o, d, x_mid, d, self.params[f"mlp_norm.{l}"], c.eps, mn, d, s["rstd2"])
-            g, u = self._linear(l, "gate_proj", mn, quantised, beta), self._linear(l, "up_proj", mn, quantised, beta)
+            gu = self._linear_group(l, "gate_up", mn, quantised, beta)
+            g, u = gu[:, :f], gu[:, f:]
             act = self._new(f)
-            faar.silu_mul(ctx, T, f, g, f, u, f, act, f)
+            faar.silu_mul(ctx, T, f, g, 2 * f, u, 2 * f, act, f)
             dn = self._linear(l, "down_proj", act, quantised, beta)
             if keep:
                 s.update(hn=hn, q=q, k=k, v=v, a=a, lse=lse, x_mid=x_mid, mn=mn, g=g, u=u, act=act)
@@ -142,19 +177,37 @@ class Stage2Model:
         return Z, H, ((cache, x, rstd_f) if keep else None)
 
     # ---- backward ------------------------------------------------------------------------------------
+    def _update(self, l, name, dY, ldy, X, hp, want_dv):
+        """dW GEMM of one quantised linear with the chain rule into V, the Round Loss gradient, the optimiser update
+        and the clip.  dY [T, O] (row stride ldy) and X [T, K] as the backward pass holds them: no transposed
+        copies.  Returns dV or None."""
+        lin = self.lin[l][name]
+        shape = faar.make_shape(lin.O, lin.K, self.T, ldxt=self.ldt, ldy=ldy)
+        dV = torch.empty((lin.O, lin.K), dtype=torch.float32, device=self.dev) if want_dv else None
+        faar.layer_bwd_rowmajor(self.ctx, shape, hp, dY, X, lin.V, lin.code, lin.scales, lin.s_global, lin.m, lin.u, dV, self.ws)
+        return dV
+
     def _linear_bwd(self, l, name, dY, X, hp, want_dv):
-        """One quantised linear: dX = dY W_soft at the pre-update V, then the dW GEMM with the chain rule into V,
-        the Round Loss gradient, the optimiser update and the clip.  Returns (dX, dV or None)."""
-        lin, T, ctx = self.lin[l][name], self.T, self.ctx
-        O, K = lin.O, lin.K
-        shape = faar.make_shape(O, K, T, ldxt=self.ldt)
-        dX = self._new(K)
+        """One quantised linear: dX = dY W_soft at the pre-update V, then its update.  Returns (dX, dV or None)."""
+        lin = self.lin[l][name]
+        dX = self._new(lin.K)
         # lin.Wsoft still holds this step's soft weights: V changes only in the update below
-        faar.layer_dx_operand(ctx, shape, dY, lin.Wsoft, dX, self.ws)
-        dV = torch.empty((O, K), dtype=torch.float32, device=self.dev) if want_dv else None
-        # dY [T, O] and X [T, K] as the backward pass holds them: no transposed copies
-        faar.layer_bwd_rowmajor(ctx, shape, hp, dY, X, lin.V, lin.code, lin.scales, lin.s_global, lin.m, lin.u, dV, self.ws)
-        return dX, dV
+        faar.layer_dx_operand(self.ctx, faar.make_shape(lin.O, lin.K, self.T), dY, lin.Wsoft, dX, self.ws)
+        return dX, self._update(l, name, dY, lin.O, X, hp, want_dv)
+
+    def _group_bwd(self, l, group, dY, X, hp, want_dv, grads):
+        """The linears of one group: the gradient towards their common input is one product of the stacked output
+        gradients dY [T, sum of widths] with the stacked soft weights (the sum over the linears is the contraction),
+        then each linear's update from its column range of dY."""
+        K = self.lin[l][GROUPS[group][0]].K
+        dX = self._new(K)
+        faar.layer_dx_operand(self.ctx, faar.make_shape(dY.shape[1], K, self.T), dY, self.wsoft_group[l][group], dX, self.ws)
+        c0 = 0
+        for n in GROUPS[group]:
+            O = self.lin[l][n].O
+            grads[(l, n)] = self._update(l, n, dY[:, c0:c0 + O], dY.shape[1], X, hp, want_dv)
+            c0 += O
+        return dX
 
     def backward(self, dZ, dH, saved, hp, want_dv=False):
         """From the loss gradients at the logits and at the last hidden state back to every V (updated in place).
@@ -174,25 +227,21 @@ class Stage2Model:
             s = cache[l]
             # MLP branch: x = x_mid + act W_down^T
             dact, grads[(l, "down_proj")] = self._linear_bwd(l, "down_proj", dx, s["act"], hp, want_dv)
-            dg, du = self._new(f), self._new(f)
-            faar.silu_mul_bwd(ctx, T, f, dact, f, s["g"], f, s["u"], f, dg, f, du, f)
-            dmn, grads[(l, "gate_proj")] = self._linear_bwd(l, "gate_proj", dg, s["mn"], hp, want_dv)
-            dmn2, grads[(l, "up_proj")] = self._linear_bwd(l, "up_proj", du, s["mn"], hp, want_dv)
-            # the two gradients that meet at the norm's output are summed inside its backward
-            faar.rmsnorm_bwd_sum(ctx, T, d, dmn, dmn2, None, d, s["x_mid"], d, self.params[f"mlp_norm.{l}"], s["rstd2"], dx, d,
-                                 dx, d)
+            dgu = self._new(2 * f)
+            faar.silu_mul_bwd(ctx, T, f, dact, f, s["g"], 2 * f, s["u"], 2 * f, dgu[:, :f], 2 * f, dgu[:, f:], 2 * f)
+            dmn = self._group_bwd(l, "gate_up", dgu, s["mn"], hp, want_dv, grads)
+            faar.rmsnorm_bwd(ctx, T, d, dmn, d, s["x_mid"], d, self.params[f"mlp_norm.{l}"], s["rstd2"], dx, d, dx, d)
             # attention branch: x_mid = x_in + a W_o^T
             da, grads[(l, "o_proj")] = self._linear_bwd(l, "o_proj", dx, s["a"], hp, want_dv)
-            dq, dk, dv = self._new(qd), self._new(kvd), self._new(kvd)
-            faar.attention_bwd(ctx, self.batch, self.seq, c.n_heads, c.n_kv_heads, c.head_dim, s["q"], qd, s["k"], s["v"], kvd,
+            dqkv = self._new(qd + 2 * kvd)
+            ldp = qd + 2 * kvd
+            dq, dk, dv = dqkv[:, :qd], dqkv[:, qd:qd + kvd], dqkv[:, qd + kvd:]
+            faar.attention_bwd(ctx, self.batch, self.seq, c.n_heads, c.n_kv_heads, c.head_dim, s["q"], ldp, s["k"], s["v"], ldp,
                                s["a"], da, qd, s["lse"], self.dsum, dq, dk, dv)
-            faar.rope(ctx, T, c.n_heads, c.head_dim, dq, qd, self.pos, c.theta, 1, dq, qd)
-            faar.rope(ctx, T, c.n_kv_heads, c.head_dim, dk, kvd, self.pos, c.theta, 1, dk, kvd)
-            dhn, grads[(l, "q_proj")] = self._linear_bwd(l, "q_proj", dq, s["hn"], hp, want_dv)
-            dhk, grads[(l, "k_proj")] = self._linear_bwd(l, "k_proj", dk, s["hn"], hp, want_dv)
-            dhv, grads[(l, "v_proj")] = self._linear_bwd(l, "v_proj", dv, s["hn"], hp, want_dv)
-            faar.rmsnorm_bwd_sum(ctx, T, d, dhn, dhk, dhv, d, s["x_in"], d, self.params[f"attn_norm.{l}"], s["rstd1"], dx, d,
-                                 dx, d)
+            faar.rope(ctx, T, c.n_heads, c.head_dim, dq, ldp, self.pos, c.theta, 1, dq, ldp)
+            faar.rope(ctx, T, c.n_kv_heads, c.head_dim, dk, ldp, self.pos, c.theta, 1, dk, ldp)
+            dhn = self._group_bwd(l, "qkv", dqkv, s["hn"], hp, want_dv, grads)
+            faar.rmsnorm_bwd(ctx, T, d, dhn, d, s["x_in"], d, self.params[f"attn_norm.{l}"], s["rstd1"], dx, d, dx, d)
         return grads if want_dv else None
 
     # ---- one step of Eq. 6 -----------------------------------------------------------------------------
