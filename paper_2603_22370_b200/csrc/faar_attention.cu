@@ -170,24 +170,39 @@ attn_fwd_kernel(const AttnParams p) {
   }
 }
 
-// ---- backward, step 0: dsum[b, h, t] = sum_d dO[t, h, d] * O[t, h, d]  (one warp per (token, head)) -------------
+// ---- backward, step 0: dsum[b, h, t] = sum_d dO[t, h, d] * O[t, h, d] ------------------------------------------
+// D / 8 lanes share one (token, head) row, 16 bytes of O and of dO each, so a warp takes 256 / D consecutive tokens
+// of one head per pass; consecutive warps take the heads of the same tokens (whole rows of O and dO are read
+// together), and a warp's results are consecutive floats of dsum.
 template <int D>
 __global__ void __launch_bounds__(ATT_THREADS)
 attn_dsum_kernel(const AttnParams p, float* dsum) {
+  constexpr int LPR = D / 8, RPW = 32 / LPR;                 // lanes per row, rows per warp
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long total = (long long)p.B * p.S * p.H;
+  const int sub = lane / LPR, c = (lane % LPR) * 8;
+  const int nq = (p.S + RPW - 1) / RPW;
+  const long long total = (long long)p.B * p.H * nq;
   for (long long i = (long long)blockIdx.x * (ATT_THREADS / 32) + warp; i < total; i += (long long)gridDim.x * (ATT_THREADS / 32)) {
     const int h = (int)(i % p.H);
-    const long long t = i / p.H;                             // token index over all sequences
-    const __nv_bfloat16* o = p.out + t * p.ldo + h * D;
-    const __nv_bfloat16* d = p.dout + t * p.ldo + h * D;
+    const long long r = i / p.H;
+    const int tq = (int)(r % nq);
+    const long long b = r / nq;
+    const int sidx = tq * RPW + sub;
     float acc = 0.f;
-    for (int c = lane; c < D; c += 32) acc = fmaf(__bfloat162float(o[c]), __bfloat162float(d[c]), acc);
-    acc = faar_warp_sum(acc);
-    if (lane == 0) {
-      const long long b = t / p.S, sidx = t - b * p.S;
-      dsum[(b * p.H + h) * p.S + sidx] = acc;
+    if (sidx < p.S) {
+      const long long off = (b * p.S + sidx) * p.ldo + h * D + c;
+      const uint4 ov = *reinterpret_cast<const uint4*>(p.out + off);
+      const uint4 dv = *reinterpret_cast<const uint4*>(p.dout + off);
+      const uint32_t ow[4] = {ov.x, ov.y, ov.z, ov.w}, dw[4] = {dv.x, dv.y, dv.z, dv.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        acc = fmaf(__uint_as_float(ow[k] << 16), __uint_as_float(dw[k] << 16), acc);
+        acc = fmaf(__uint_as_float(ow[k] & 0xFFFF0000u), __uint_as_float(dw[k] & 0xFFFF0000u), acc);
+      }
     }
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if (lane % LPR == 0 && sidx < p.S) dsum[(b * p.H + h) * p.S + sidx] = acc;
   }
 }
 
@@ -849,7 +864,7 @@ int launch_bwd(faar_ctx* ctx, const AttnParams& p, float* dsum) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_dq64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BWD64_SMEM);
   if (e != cudaSuccess) return (int)e;
   faar_prof_scope ps(ctx, FAAR_K_ATTENTION);
-  long long rows = (long long)p.B * p.S * p.H;
+  long long rows = (long long)p.B * p.H * ((p.S + 256 / D - 1) / (256 / D));      // warp passes of the row-sum kernel
   long long blocks = (rows + 3) / 4;
   if (blocks > (long long)ctx->num_sms * 16) blocks = (long long)ctx->num_sms * 16;
   attn_dsum_kernel<D><<<(int)blocks, ATT_THREADS, 0, ctx->stream>>>(p, dsum);
