@@ -114,6 +114,24 @@ __device__ __forceinline__ void ld32(uint32_t taddr, float (&r)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
 }
+// 32 consecutive 32-bit columns of this thread's tensor-memory lane, written (BF16 pairs of an A operand)
+__device__ __forceinline__ void st32(uint32_t taddr, const uint32_t (&u)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,"
+      "%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]), "r"(u[8]), "r"(u[9]),
+        "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15]), "r"(u[16]), "r"(u[17]), "r"(u[18]), "r"(u[19]),
+        "r"(u[20]), "r"(u[21]), "r"(u[22]), "r"(u[23]), "r"(u[24]), "r"(u[25]), "r"(u[26]), "r"(u[27]), "r"(u[28]), "r"(u[29]),
+        "r"(u[30]), "r"(u[31])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+// D (+)= A B with A read from tensor memory (128 lanes = rows, two BF16 contraction elements per 32-bit column,
+// the lower index in the lower half) and B from shared memory
+__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t db, uint32_t id, uint32_t acc) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+               ::"r"(d), "r"(a_tmem), "l"(db), "r"(id), "r"(acc) : "memory");
+}
 // 2^x on the special-function unit, one instruction (relative error about 2^-22; -inf gives 0; results below the
 // normal range are flushed to zero, which is what a probability that small should be)
 __device__ __forceinline__ float ex2(float x) {
@@ -218,9 +236,10 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         if (j >= 1 && j + 1 < n_kt) load_v(j + 1);
         fence_after();
         {
-          const uint64_t da = desc_k_major(sP(st)), db = desc_n_major(sV(st));
+          const uint64_t db = desc_n_major(sV(st));
+          const uint32_t ta = tmem + 192u + 32u * (uint32_t)st;      // P_j: 16 contraction steps = 8 columns
 #pragma unroll
-          for (int k = 0; k < KT / 16; ++k) mma(tmem + 128u, da + 2u * k, db + 128u * k, id_pv, k != 0 ? 1u : 0u);
+          for (int k = 0; k < KT / 16; ++k) mma_ts(tmem + 128u, ta + 8u * k, db + 128u * k, id_pv, k != 0 ? 1u : 0u);
         }
         commit(bar_o);
       }
@@ -279,16 +298,17 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       const float ref = m_new == -INFINITY ? 0.f : m_new;     // a row beyond the sequence may have seen no key
       const float alpha = ex2(m - ref);
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      uint8_t* prow = smem + OFF_P + (j & 1) * P_BYTES + row * 128;
+      uint32_t pk[KT / 2];
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         float e[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) { e[i] = ex2(fmaf(s[8 * c + i], p.scale_log2, -ref)); sum4[i & 3] += e[i]; }
-        *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
-            make_uint4(pack2(e[0], e[1]), pack2(e[2], e[3]), pack2(e[4], e[5]), pack2(e[6], e[7]));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) pk[4 * c + i] = pack2(e[2 * i], e[2 * i + 1]);
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this row of P, visible to the tensor cores
+      st32(t_lane + 192u + 32u * (uint32_t)(j & 1), pk);             // this row of P_j, an A operand in tensor memory
+      fence_before();
       bar_arrive(bar_p);
       // the previous tile's P V has had the whole of this tile's softmax to finish: fold it in
       if (j > 0) {
