@@ -4,9 +4,10 @@
 // Forward.  One CTA takes 128 queries of one head and sweeps the keys in tiles of 64 (one sweep, running maximum):
 //   S   = Q K_j^T       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 FP32 columns of tensor memory
 //   P_j = 2^(c S - m)   four warps, one query row per thread (its tensor-memory lane): no shuffles; the row
-//                       goes to shared memory as BF16 in the 128-byte-swizzled layout an A operand has
-//   O_j = P_j V_j       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 more columns; V_j is read as it lies in
-//                       memory (keys as rows: a B operand with its N index contiguous)
+//                       goes back to tensor memory as BF16 pairs, 32 columns (tcgen05.st)
+//   O_j = P_j V_j       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 more columns; P_j is the A operand, read from
+//                       tensor memory; V_j is read from shared memory as it lies in memory (keys as rows: a B
+//                       operand with its N index contiguous)
 //   O   = O * 2^(m_old - m) + O_j   in registers of the row's thread
 // Q, K_j, V_j arrive by TMA (two stages for K and V).  A fifth warp's lane 0 issues every copy and every MMA; the
 // scores have two buffers in tensor memory, so S of tile j + 1 is formed while the warps work on tile j, and two
@@ -24,12 +25,12 @@
 namespace {
 
 constexpr int QT = 128, KT = 64, HD = 64;
-constexpr int Q_BYTES = QT * HD * 2, KV_BYTES = KT * HD * 2, P_BYTES = QT * KT * 2;
-constexpr int OFF_K = Q_BYTES, OFF_V = OFF_K + 2 * KV_BYTES, OFF_P = OFF_V + 2 * KV_BYTES, OFF_CTL = OFF_P + 2 * P_BYTES;
+constexpr int Q_BYTES = QT * HD * 2, KV_BYTES = KT * HD * 2;
+constexpr int OFF_K = Q_BYTES, OFF_V = OFF_K + 2 * KV_BYTES, OFF_CTL = OFF_V + 2 * KV_BYTES;
 constexpr int CTL = 256;
 constexpr int SMEM = OFF_CTL + CTL + 1024;
 constexpr int THREADS = 160;
-constexpr int TMEM_COLS = 256;                     // S of even / odd tiles: columns 0..63 / 64..127, O_j: 128..191
+constexpr int TMEM_COLS = 256;                     // S of even / odd tiles: columns 0..63 / 64..127, O_j: 128..191, P: 192..223 / 224..255
 constexpr unsigned long long LIMIT_NS = 2000000000ull;
 
 __device__ uint32_t g_attn_status;                 // 0 = no wait has given up since the last read-and-clear
@@ -126,6 +127,14 @@ __device__ __forceinline__ void st32(uint32_t taddr, const uint32_t (&u)[32]) {
       : "memory");
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void st16(uint32_t taddr, const uint32_t (&u)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7]), "r"(u[8]), "r"(u[9]),
+        "r"(u[10]), "r"(u[11]), "r"(u[12]), "r"(u[13]), "r"(u[14]), "r"(u[15])
+      : "memory");
+}
+__device__ __forceinline__ void wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // D (+)= A B with A read from tensor memory (128 lanes = rows, two BF16 contraction elements per 32-bit column,
 // the lower index in the lower half) and B from shared memory
 __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint64_t db, uint32_t id, uint32_t acc) {
@@ -189,7 +198,6 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t sQ = base;
-  auto sP = [&](int s) { return base + OFF_P + (uint32_t)s * P_BYTES; };
   auto sK = [&](int s) { return base + OFF_K + (uint32_t)s * KV_BYTES; };
   auto sV = [&](int s) { return base + OFF_V + (uint32_t)s * KV_BYTES; };
 
@@ -352,14 +360,15 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
 // ---- backward, dQ: one CTA per 128 queries of a head, sweeping the key tiles up to the diagonal ---------------
 //   S_j = Q K_j^T, dP_j = dO V_j^T     two MMAs into 64 + 64 columns of tensor memory
-//   dS_j = P_j (dP_j - delta) / sqrt(d), P_j = 2^(c S_j - lse)     one query row per thread, written as a BF16
-//                                                                   A operand into swizzled shared memory
+//   dS_j = P_j (dP_j - delta) / sqrt(d), P_j = 2^(c S_j - lse)     one query row per thread, written as BF16
+//                                                                   pairs into 32 columns of tensor memory, the
+//                                                                   third product's A operand
 //   dQ += dS_j K_j                       third MMA, accumulating in 64 more columns over the whole sweep (K_j read
 //                                        as it lies in memory: keys as contraction rows, d contiguous)
 // The dQ product of tile j - 1 is issued after the score products of tile j, so it runs while the rows work on
 // tile j; K / V tiles come through three TMA stages.  Only the final dQ leaves tensor memory.
 constexpr int DQ_OFF_DO = Q_BYTES, DQ_OFF_KV = 2 * Q_BYTES, DQ_STAGE = 2 * KV_BYTES, DQ_STAGES = 3;
-constexpr int DQ_OFF_DS = DQ_OFF_KV + DQ_STAGES * DQ_STAGE, DQ_OFF_CTL = DQ_OFF_DS + P_BYTES;
+constexpr int DQ_OFF_CTL = DQ_OFF_KV + DQ_STAGES * DQ_STAGE;
 constexpr int DQ_SMEM = DQ_OFF_CTL + CTL + 1024;
 // The backward kernels have no reduction along a row, so two threads share a row (32 of the 64 columns each:
 // warps w and w + 4 read the same tensor-memory lanes): eight row warps, the ninth issues copies and MMAs.
@@ -413,8 +422,8 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   fence_before();
   __syncthreads();
   fence_after();
-  const uint32_t tmem = *tmem_slot;                         // S: columns 0..63, dP: 64..127, dQ: 128..191
-  const uint32_t sQ = base, sDO = base + DQ_OFF_DO, sDS = base + DQ_OFF_DS;
+  const uint32_t tmem = *tmem_slot;                         // S: columns 0..63, dP: 64..127, dQ: 128..191, dS (BF16 pairs): 192..223
+  const uint32_t sQ = base, sDO = base + DQ_OFF_DO;
   auto sK = [&](int s) { return base + DQ_OFF_KV + (uint32_t)s * DQ_STAGE; };
   auto sV = [&](int s) { return sK(s) + KV_BYTES; };
 
@@ -434,9 +443,9 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       bool ok = bar_wait(bar_qd, 0u, abort_flag, 0xC01u);
       const uint32_t id_k = idesc(0), id_n = idesc(1);
       auto issue_dq = [&](int j) {                            // dQ += dS_j K_j
-        const uint64_t da = desc_k_major(sDS), db = desc_n_major(sK(j % DQ_STAGES));
+        const uint64_t db = desc_n_major(sK(j % DQ_STAGES));
 #pragma unroll
-        for (int k = 0; k < KT / 16; ++k) mma(tmem + 128u, da + 2u * k, db + 128u * k, id_n, (j | k) != 0 ? 1u : 0u);
+        for (int k = 0; k < KT / 16; ++k) mma_ts(tmem + 128u, tmem + 192u + 8u * k, db + 128u * k, id_n, (j | k) != 0 ? 1u : 0u);
         commit(bar_done);
       };
       for (int j = 0; j < n_kt && ok; ++j) {
@@ -502,13 +511,12 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         ok = bar_wait(bar_done, (uint32_t)((j - 1) & 1), abort_flag, 0xD20u);
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       }
-      uint8_t* prow = smem + DQ_OFF_DS + row * 128;
+      uint32_t pk[16];
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
-        *reinterpret_cast<uint4*>(prow + (((4 * half + c) ^ (row & 7)) << 4)) =
-            make_uint4(pack2(s[8 * c], s[8 * c + 1]), pack2(s[8 * c + 2], s[8 * c + 3]), pack2(s[8 * c + 4], s[8 * c + 5]),
-                       pack2(s[8 * c + 6], s[8 * c + 7]));
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      for (int w = 0; w < 16; ++w) pk[w] = pack2(s[2 * w], s[2 * w + 1]);
+      st16(t_lane + 192u + 16u * half, pk);                   // this thread's half of the row of dS_j: an A operand
+      wait_st();
+      fence_before();
       bar_arrive(bar_ds);
     }
     if (ok) {
@@ -543,17 +551,17 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 // The keys are the rows (tensor-memory lanes); the CTA sweeps the (head, 64-query tile) pairs that see them:
 //   S^T = K Q_i^T, dP^T = V dO_i^T          two MMAs into one of two pairs of 64-column buffers
 //   P^T = 2^(c S^T - lse_q), dS^T = P^T (dP^T - delta_q) / sqrt(d)    one key row per thread; both written as BF16
-//                                            A operands into one of two pairs of swizzled shared-memory buffers
+//                                            pairs into one of two pairs of 32-column buffers in tensor memory, the
+//                                            A operands of the accumulating products
 //   dV += P^T dO_i, dK += dS^T Q_i           two MMAs that accumulate in 64 + 64 columns over the whole sweep
 //                                            (dO_i and Q_i read as they lie in memory: queries as contraction rows)
 // One CTA per SM; the score products of item i + 1 are issued before this item's probabilities are awaited, Q / dO
 // tiles come through four TMA stages (requested two items ahead), lse and delta of a tile's 64 queries are staged in shared memory by the
 // row threads themselves.  Queries beyond the sequence end are masked (their rows hold the next sequence's data).
 constexpr int KV_OFF_V = Q_BYTES, KV_OFF_QD = 2 * Q_BYTES, KV_STAGE = 2 * KV_BYTES, KV_STAGES = 4;
-constexpr int KV_OFF_PT = KV_OFF_QD + KV_STAGES * KV_STAGE, KV_OFF_DST = KV_OFF_PT + 2 * P_BYTES;
-constexpr int KV_OFF_ROWV = KV_OFF_DST + 2 * P_BYTES, KV_OFF_CTL = KV_OFF_ROWV + 2 * 2 * KT * 4;
+constexpr int KV_OFF_ROWV = KV_OFF_QD + KV_STAGES * KV_STAGE, KV_OFF_CTL = KV_OFF_ROWV + 2 * 2 * KT * 4;
 constexpr int KV_SMEM = KV_OFF_CTL + CTL + 1024;
-constexpr int KV_TMEM = 512;                      // S^T: 0 / 64, dP^T: 128 / 192, dV: 256, dK: 320
+constexpr int KV_TMEM = 512;                      // S^T: 0 / 64, dP^T: 128 / 192, dV: 256, dK: 320, P^T: 384 / 416, dS^T: 448 / 480 (BF16 pairs)
 
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
@@ -607,8 +615,6 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   const uint32_t sKt = base, sVt = base + KV_OFF_V;
   auto sQ = [&](int s) { return base + KV_OFF_QD + (uint32_t)s * KV_STAGE; };
   auto sDO = [&](int s) { return sQ(s) + KV_BYTES; };
-  auto sPT = [&](int s) { return base + KV_OFF_PT + (uint32_t)s * P_BYTES; };
-  auto sDST = [&](int s) { return base + KV_OFF_DST + (uint32_t)s * P_BYTES; };
   auto head_of = [&](int i) { return g * rep + i / per_head; };
   auto q0_of = [&](int i) { return (qt0 + i % per_head) * KT; };
 
@@ -657,11 +663,12 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         fence_after();
         {
           const int st = i % KV_STAGES;
-          const uint64_t dp_ = desc_k_major(sPT(i & 1)), dd = desc_n_major(sDO(st)), ds_ = desc_k_major(sDST(i & 1)), dq_ = desc_n_major(sQ(st));
+          const uint64_t dd = desc_n_major(sDO(st)), dq_ = desc_n_major(sQ(st));
+          const uint32_t tp = tmem + 384u + 32u * (uint32_t)(i & 1), td = tmem + 448u + 32u * (uint32_t)(i & 1);
 #pragma unroll
-          for (int k = 0; k < KT / 16; ++k) mma(tmem + 256u, dp_ + 2u * k, dd + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < KT / 16; ++k) mma_ts(tmem + 256u, tp + 8u * k, dd + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < KT / 16; ++k) mma(tmem + 320u, ds_ + 2u * k, dq_ + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < KT / 16; ++k) mma_ts(tmem + 320u, td + 8u * k, dq_ + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
         }
         commit(bar_done(i & 1));
       }
@@ -700,8 +707,6 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         ok = bar_wait(bar_done(i & 1), (uint32_t)(((i - 2) >> 1) & 1), abort_flag, 0xF20u);
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       }
-      uint8_t* prow = smem + KV_OFF_PT + (i & 1) * P_BYTES + row * 128;
-      uint8_t* drow = smem + KV_OFF_DST + (i & 1) * P_BYTES + row * 128;
       // the mask costs three instructions per element: only items that need it take that path
       auto item = [&](auto edge_tag) {
         constexpr bool EDGE = decltype(edge_tag)::value;
@@ -722,21 +727,19 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             d[j] = pr * fmaf(d[j], p.inv_sqrt_d, nq[e]);
           }
         }
+        // this thread's half of the rows of P^T and dS^T: A operands in tensor memory
+        uint32_t pk[16];
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-          const int ch = 4 * half + c4;
-          *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) =
-              make_uint4(pack2(t[8 * c4], t[8 * c4 + 1]), pack2(t[8 * c4 + 2], t[8 * c4 + 3]), pack2(t[8 * c4 + 4], t[8 * c4 + 5]),
-                         pack2(t[8 * c4 + 6], t[8 * c4 + 7]));
-          *reinterpret_cast<uint4*>(drow + ((ch ^ (row & 7)) << 4)) =
-              make_uint4(pack2(d[8 * c4], d[8 * c4 + 1]), pack2(d[8 * c4 + 2], d[8 * c4 + 3]), pack2(d[8 * c4 + 4], d[8 * c4 + 5]),
-                         pack2(d[8 * c4 + 6], d[8 * c4 + 7]));
-        }
+        for (int w = 0; w < 16; ++w) pk[w] = pack2(t[2 * w], t[2 * w + 1]);
+        st16(t_lane + 384u + 32u * (uint32_t)(i & 1) + 16u * half, pk);
+#pragma unroll
+        for (int w = 0; w < 16; ++w) pk[w] = pack2(d[2 * w], d[2 * w + 1]);
+        st16(t_lane + 448u + 32u * (uint32_t)(i & 1) + 16u * half, pk);
       };
       if (edge) item(std::true_type{}); else item(std::false_type{});
+      wait_st();
       fence_before();
       bar_arrive(bar_sfree(i & 1));
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       bar_arrive(bar_pds(i & 1));
     }
     if (ok) {
