@@ -115,6 +115,19 @@ __device__ __forceinline__ void ld32(uint32_t taddr, float (&r)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
 }
+// Two such loads in flight together (one wait for both)
+__device__ __forceinline__ void ld32x2(uint32_t ta, uint32_t tb, float (&a)[32], float (&b)[32]) {
+  uint32_t u[32], v[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%64];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%65];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]), "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31]),
+        "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(ta), "r"(tb) : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) { a[i] = __uint_as_float(u[i]); b[i] = __uint_as_float(v[i]); }
+}
 // 32 consecutive 32-bit columns of this thread's tensor-memory lane, written (BF16 pairs of an A operand)
 __device__ __forceinline__ void st32(uint32_t taddr, const uint32_t (&u)[32]) {
   asm volatile(
@@ -266,12 +279,12 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     // o_acc <- o_acc * a + O_j: the accumulated output moves to the maximum that P_j was formed against (factor a,
     // computed when tile j was processed) and takes tile j's product in the same multiply-add
     auto fold = [&](float a) {
+      float t[32], t2[32];
+      ld32x2(t_o, t_o + 32u, t, t2);
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float t[32];
-        ld32(t_o + 32u * half, t);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o_acc[32 * half + i] = fmaf(o_acc[32 * half + i], a, t[i]);
+      for (int i = 0; i < 32; ++i) {
+        o_acc[i] = fmaf(o_acc[i], a, t[i]);
+        o_acc[32 + i] = fmaf(o_acc[32 + i], a, t2[i]);
       }
     };
     float alpha_pending = 0.f;                                // factor of the tile whose P V product is still to be folded
@@ -283,13 +296,10 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       fence_after();
       float s[KT];
       {
-        float t[32];
-        ld32(t_s, t);
+        float t[32], t2[32];
+        ld32x2(t_s, t_s + 32u, t, t2);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) s[i] = t[i];
-        ld32(t_s + 32u, t);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) s[32 + i] = t[i];
+        for (int i = 0; i < 32; ++i) { s[i] = t[i]; s[32 + i] = t2[i]; }
       }
       fence_before();
       bar_arrive(bar_sfree(j & 1));
@@ -495,8 +505,7 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       auto tile = [&](auto diag_tag) {                        // P (dP - delta) / sqrt(d); the mask only where needed
         constexpr bool DIAG = decltype(diag_tag)::value;
         float t[32], d[32];
-        ld32(t_lane + 32u * half, t);
-        ld32(t_lane + 64u + 32u * half, d);
+        ld32x2(t_lane + 32u * half, t_lane + 64u + 32u * half, t, d);
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           float pr = ex2(fmaf(t[i], p.scale_log2, -lse));
@@ -711,8 +720,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       auto item = [&](auto edge_tag) {
         constexpr bool EDGE = decltype(edge_tag)::value;
         float t[32], d[32];
-        ld32(t_lane + 64u * (uint32_t)(i & 1) + 32u * half, t);
-        ld32(t_lane + 128u + 64u * (uint32_t)(i & 1) + 32u * half, d);
+        ld32x2(t_lane + 64u * (uint32_t)(i & 1) + 32u * half, t_lane + 128u + 64u * (uint32_t)(i & 1) + 32u * half, t, d);
 #pragma unroll
         for (int j4 = 0; j4 < 32; j4 += 4) {
           const float4 l4 = *reinterpret_cast<const float4*>(rowv + 32 * half + j4);          // the same address in every lane
