@@ -558,21 +558,26 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
 // ---- backward, dK and dV: one CTA per 128 keys of a key / value head ------------------------------------------
 // The keys are the rows (tensor-memory lanes); the CTA sweeps the (head, 64-query tile) pairs that see them:
-//   S^T = K Q_i^T, dP^T = V dO_i^T          two MMAs into one of two pairs of 64-column buffers
+//   S^T = K Q_i^T, dP^T = V dO_i^T          two MMAs into 64 + 64 columns of tensor memory
 //   P^T = 2^(c S^T - lse_q), dS^T = P^T (dP^T - delta_q) / sqrt(d)    one key row per thread; both written as BF16
-//                                            pairs into one of two pairs of 32-column buffers in tensor memory, the
-//                                            A operands of the accumulating products
+//                                            pairs over the columns the thread has just read (its half of S^T, of
+//                                            dP^T), from where they are the A operands of the accumulating products
 //   dV += P^T dO_i, dK += dS^T Q_i           two MMAs that accumulate in 64 + 64 columns over the whole sweep
 //                                            (dO_i and Q_i read as they lie in memory: queries as contraction rows)
-// One CTA per SM; the score products of item i + 1 are issued before this item's probabilities are awaited, Q / dO
-// tiles come through four TMA stages (requested two items ahead), lse and delta of a tile's 64 queries are staged in shared memory by the
-// row threads themselves.  Queries beyond the sequence end are masked (their rows hold the next sequence's data).
+// 256 columns of tensor memory and under 100 KB of shared memory: two CTAs per SM, which overlap each other's serial
+// chain (score products -> rows -> accumulating products -> next item's score products, which overwrite P^T / dS^T
+// and so wait for the accumulating products).  Q / dO tiles come through four TMA stages (requested three items
+// ahead), lse and delta of a tile's 64 queries are staged in shared memory by the row threads themselves.  Queries
+// beyond the sequence end are masked (their rows hold the next sequence's data).
 constexpr int KV_OFF_V = Q_BYTES, KV_OFF_QD = 2 * Q_BYTES, KV_STAGE = 2 * KV_BYTES, KV_STAGES = 4;
 constexpr int KV_OFF_ROWV = KV_OFF_QD + KV_STAGES * KV_STAGE, KV_OFF_CTL = KV_OFF_ROWV + 2 * 2 * KT * 4;
 constexpr int KV_SMEM = KV_OFF_CTL + CTL + 1024;
-constexpr int KV_TMEM = 512;                      // S^T: 0 / 64, dP^T: 128 / 192, dV: 256, dK: 320, P^T: 384 / 416, dS^T: 448 / 480 (BF16 pairs)
+static_assert(2 * KV_SMEM <= 227 * 1024, "two CTAs per SM");
+// S^T: columns 0..63, dP^T: 64..127, dV: 128..191, dK: 192..255.  The thread of row half h reads columns 32 h .. 32 h + 31
+// of S^T (dP^T) and writes its 32 values of P^T (dS^T) as 16 BF16 pairs to columns 32 h .. 32 h + 15 of the same buffer.
+constexpr int KV_TMEM = 256;
 
-__global__ void __launch_bounds__(BWD_THREADS, 1)
+__global__ void __launch_bounds__(BWD_THREADS, 2)
 attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
                      const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const TcBwdParams p) {
   extern __shared__ uint8_t raw[];
@@ -581,9 +586,8 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   const uint32_t ctl = base + KV_OFF_CTL;
   const uint32_t bar_kv = ctl;
   auto qfull = [&](int s) { return ctl + 8u + 8u * s; };          // 4
-  auto bar_s = [&](int s) { return ctl + 40u + 8u * s; };         // 2: score buffers of an item are complete
-  auto bar_sfree = [&](int s) { return ctl + 56u + 8u * s; };     // 2: ... have been read by all rows
-  auto bar_pds = [&](int s) { return ctl + 72u + 8u * s; };       // 2: P^T / dS^T buffers written
+  auto bar_s = [&](int s) { return ctl + 40u + 8u * s; };         // 2 (items alternate): the score products of an item are complete
+  auto bar_pds = [&](int s) { return ctl + 72u + 8u * s; };       // 2: P^T / dS^T of an item written by all rows
   auto bar_done = [&](int s) { return ctl + 88u + 8u * s; };      // 2: the accumulating MMAs of an item have run
   auto bar_rv = [&](int s) { return ctl + 112u + 8u * s; };       // 2: lse / delta of an item staged, previous use read by all
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + KV_OFF_CTL + 128);
@@ -606,7 +610,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     bar_init(bar_kv, 1);
     for (int s = 0; s < KV_STAGES; ++s) bar_init(qfull(s), 1);
     for (int s = 0; s < 2; ++s) {
-      bar_init(bar_s(s), 1); bar_init(bar_done(s), 1); bar_init(bar_sfree(s), ROW_THREADS); bar_init(bar_pds(s), ROW_THREADS); bar_init(bar_rv(s), ROW_THREADS);
+      bar_init(bar_s(s), 1); bar_init(bar_done(s), 1); bar_init(bar_pds(s), ROW_THREADS); bar_init(bar_rv(s), ROW_THREADS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -643,25 +647,18 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       if (n_it > 2) load_item(2);
       bool ok = bar_wait(bar_kv, 0u, abort_flag, 0xE01u);
       const uint32_t id_k = idesc(0), id_n = idesc(1);
-      auto issue_s = [&](int i) {                              // S^T and dP^T of item i into buffer pair i & 1
+      auto issue_s = [&](int i) {                              // S^T and dP^T of item i
         const int st = i % KV_STAGES;
         const uint64_t dk_ = desc_k_major(sKt), dq_ = desc_k_major(sQ(st)), dv_ = desc_k_major(sVt), dd = desc_k_major(sDO(st));
 #pragma unroll
-        for (int k = 0; k < HD / 16; ++k) mma(tmem + 64u * (uint32_t)(i & 1), dk_ + 2u * k, dq_ + 2u * k, id_k, k != 0 ? 1u : 0u);
+        for (int k = 0; k < HD / 16; ++k) mma(tmem, dk_ + 2u * k, dq_ + 2u * k, id_k, k != 0 ? 1u : 0u);
 #pragma unroll
-        for (int k = 0; k < HD / 16; ++k) mma(tmem + 128u + 64u * (uint32_t)(i & 1), dv_ + 2u * k, dd + 2u * k, id_k, k != 0 ? 1u : 0u);
+        for (int k = 0; k < HD / 16; ++k) mma(tmem + 64u, dv_ + 2u * k, dd + 2u * k, id_k, k != 0 ? 1u : 0u);
         commit(bar_s(i & 1));
       };
       if (ok) ok = bar_wait(qfull(0), 0u, abort_flag, 0xE10u);
       if (ok) { fence_after(); issue_s(0); }
       for (int i = 0; i < n_it && ok; ++i) {
-        if (i + 1 < n_it) {
-          ok = bar_wait(qfull((i + 1) % KV_STAGES), (uint32_t)(((i + 1) / KV_STAGES) & 1), abort_flag, 0xE10u);
-          if (ok && i >= 1) ok = bar_wait(bar_sfree((i + 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), abort_flag, 0xE20u);
-          if (!ok) break;
-          fence_after();
-          issue_s(i + 1);
-        }
         if (i + 3 < n_it) {                                    // its stage last held item i - 1: wait for that item's
           if (i >= 1) ok = bar_wait(bar_done((i - 1) & 1), (uint32_t)(((i - 1) >> 1) & 1), abort_flag, 0xE40u);   // MMAs
           if (!ok) break;
@@ -671,15 +668,26 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         if (!ok) break;
         fence_after();
         {
+          // A operands from tensor memory: contraction steps 0, 1 (queries 0..31) in columns 0..15 of the buffer,
+          // steps 2, 3 (queries 32..63) in columns 32..47
           const int st = i % KV_STAGES;
           const uint64_t dd = desc_n_major(sDO(st)), dq_ = desc_n_major(sQ(st));
-          const uint32_t tp = tmem + 384u + 32u * (uint32_t)(i & 1), td = tmem + 448u + 32u * (uint32_t)(i & 1);
 #pragma unroll
-          for (int k = 0; k < KT / 16; ++k) mma_ts(tmem + 256u, tp + 8u * k, dd + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < KT / 16; ++k)
+            mma_ts(tmem + 128u, tmem + (uint32_t)(32 * (k >> 1) + 8 * (k & 1)), dd + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < KT / 16; ++k) mma_ts(tmem + 320u, td + 8u * k, dq_ + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < KT / 16; ++k)
+            mma_ts(tmem + 192u, tmem + 64u + (uint32_t)(32 * (k >> 1) + 8 * (k & 1)), dq_ + 128u * k, id_n, (i | k) != 0 ? 1u : 0u);
         }
         commit(bar_done(i & 1));
+        if (i + 1 < n_it) {
+          // the next item's score products overwrite P^T / dS^T: after the accumulating products have read them
+          ok = bar_wait(qfull((i + 1) % KV_STAGES), (uint32_t)(((i + 1) / KV_STAGES) & 1), abort_flag, 0xE10u);
+          if (ok) ok = bar_wait(bar_done(i & 1), (uint32_t)((i >> 1) & 1), abort_flag, 0xE20u);
+          if (!ok) break;
+          fence_after();
+          issue_s(i + 1);
+        }
       }
       if (!ok) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) {} }
     }
@@ -712,15 +720,11 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       fence_after();
       const bool edge = q0 < k0 + QT || q0 + KT > p.S;         // the item crosses the diagonal or the sequence end
-      if (i >= 2) {                                              // the P^T / dS^T buffers last held item i - 2
-        ok = bar_wait(bar_done(i & 1), (uint32_t)(((i - 2) >> 1) & 1), abort_flag, 0xF20u);
-        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-      }
       // the mask costs three instructions per element: only items that need it take that path
       auto item = [&](auto edge_tag) {
         constexpr bool EDGE = decltype(edge_tag)::value;
         float t[32], d[32];
-        ld32x2(t_lane + 64u * (uint32_t)(i & 1) + 32u * half, t_lane + 128u + 64u * (uint32_t)(i & 1) + 32u * half, t, d);
+        ld32x2(t_lane + 32u * half, t_lane + 64u + 32u * half, t, d);
 #pragma unroll
         for (int j4 = 0; j4 < 32; j4 += 4) {
           const float4 l4 = *reinterpret_cast<const float4*>(rowv + 32 * half + j4);          // the same address in every lane
@@ -739,15 +743,14 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         uint32_t pk[16];
 #pragma unroll
         for (int w = 0; w < 16; ++w) pk[w] = pack2(t[2 * w], t[2 * w + 1]);
-        st16(t_lane + 384u + 32u * (uint32_t)(i & 1) + 16u * half, pk);
+        st16(t_lane + 32u * half, pk);                           // over the first half of the columns just read
 #pragma unroll
         for (int w = 0; w < 16; ++w) pk[w] = pack2(d[2 * w], d[2 * w + 1]);
-        st16(t_lane + 448u + 32u * (uint32_t)(i & 1) + 16u * half, pk);
+        st16(t_lane + 64u + 32u * half, pk);
       };
       if (edge) item(std::true_type{}); else item(std::false_type{});
       wait_st();
       fence_before();
-      bar_arrive(bar_sfree(i & 1));
       bar_arrive(bar_pds(i & 1));
     }
     if (ok) {
@@ -761,7 +764,7 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         uint4* dst = reinterpret_cast<uint4*>((which ? p.dk : p.dv) + (seq0 + kj) * p.ldk + g * HD);
         {
           float t[32];
-          ld32(t_lane + 256u + 64u * which + 32u * half, t);
+          ld32(t_lane + 128u + 64u * which + 32u * half, t);
           if (kj < p.S) {
 #pragma unroll
             for (int c = 0; c < 4; ++c)
