@@ -1,17 +1,19 @@
 // Causal attention for head_dim 64 on the tcgen05 tensor cores (sm_100a): the forward kernel first, then the two
 // backward kernels (dQ; dK and dV), which are built the same way and described where they start.
 //
-// Forward.  One CTA takes 128 queries of one head and sweeps the keys in tiles of 64 (one sweep, running maximum):
+// Forward.  One CTA takes 128 queries of one head and sweeps the keys in tiles of 64 (one sweep):
 //   S   = Q K_j^T       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 FP32 columns of tensor memory
 //   P_j = 2^(c S - m)   four warps, one query row per thread (its tensor-memory lane): no shuffles; the row
 //                       goes back to tensor memory as BF16 pairs, 32 columns (tcgen05.st)
-//   O_j = P_j V_j       tcgen05.mma  M = 128, N = 64, K = 64   -> 64 more columns; P_j is the A operand, read from
-//                       tensor memory; V_j is read from shared memory as it lies in memory (keys as rows: a B
-//                       operand with its N index contiguous)
-//   O   = O * 2^(m_old - m) + O_j   in registers of the row's thread
+//   O  += P_j V_j       tcgen05.mma  M = 128, N = 64, K = 64   accumulating in 64 more columns over the whole sweep;
+//                       P_j is the A operand, read from tensor memory; V_j is read from shared memory as it lies
+//                       in memory (keys as rows: a B operand with its N index contiguous)
+//   m is the row's reference, not its running maximum: it moves to a tile's maximum only when that exceeds it by
+//   more than 2^8 (probabilities stay below 2^8, the final division by their sum and lse = m + log2(sum) are
+//   exact either way); only then is O rescaled, in tensor memory, between two P V products.
 // Q, K_j, V_j arrive by TMA (two stages for K and V).  A fifth warp's lane 0 issues every copy and every MMA; the
 // scores have two buffers in tensor memory, so S of tile j + 1 is formed while the warps work on tile j, and two
-// CTAs per SM overlap what remains serial (softmax -> P V -> accumulate).
+// CTAs per SM overlap what remains serial (softmax -> P V).
 // Rows of a query tile beyond the sequence end compute on whatever rows follow in memory (or zeros past the
 // tensor) and are not stored; keys beyond the end are masked.
 // Every barrier wait is bounded; a wait that gives up records a code in a status word of this module (read by
@@ -30,7 +32,8 @@ constexpr int OFF_K = Q_BYTES, OFF_V = OFF_K + 2 * KV_BYTES, OFF_CTL = OFF_V + 2
 constexpr int CTL = 256;
 constexpr int SMEM = OFF_CTL + CTL + 1024;
 constexpr int THREADS = 160;
-constexpr int TMEM_COLS = 256;                     // S of even / odd tiles: columns 0..63 / 64..127, O_j: 128..191, P: 192..223 / 224..255
+constexpr int TMEM_COLS = 256;                     // S of even / odd tiles: columns 0..63 / 64..127, O: 128..191, P: 192..223 / 224..255
+constexpr float FWD_SLACK = 8.0f;                  // log2 of how far a tile's maximum may exceed the row's reference
 constexpr unsigned long long LIMIT_NS = 2000000000ull;
 
 __device__ uint32_t g_attn_status;                 // 0 = no wait has given up since the last read-and-clear
@@ -173,7 +176,7 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   const uint32_t base = (s32(raw) + 1023u) & ~1023u;
   uint8_t* smem = raw + (base - s32(raw));
   const uint32_t ctl = base + OFF_CTL;
-  const uint32_t bar_q = ctl, bar_p = ctl + 72, bar_o = ctl + 80, bar_ofree = ctl + 88;
+  const uint32_t bar_q = ctl, bar_p = ctl + 72, bar_o = ctl + 80;
   auto kfull = [&](int s) { return ctl + 8u + 8u * s; };
   auto vfull = [&](int s) { return ctl + 24u + 8u * s; };
   auto bar_s = [&](int s) { return ctl + 40u + 8u * s; };         // scores of a tile in buffer s are complete
@@ -196,7 +199,7 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     bar_init(bar_q, 1);
     for (int s = 0; s < 2; ++s) { bar_init(kfull(s), 1); bar_init(vfull(s), 1); }
     for (int s = 0; s < 2; ++s) { bar_init(bar_s(s), 1); bar_init(bar_sfree(s), 128); }
-    bar_init(bar_o, 1); bar_init(bar_ofree, 128); bar_init(bar_p, 128);
+    bar_init(bar_o, 1); bar_init(bar_p, 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -251,8 +254,8 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         if (!ok) break;
         if (j + 2 < n_kt) load_k(j + 2);
         ok = bar_wait(vfull(st), ph, abort_flag, 0xA40u | st);
-        // O_{j-1} folded by every row: P V_{j-1} is complete, its output columns and its V stage are free
-        if (ok && j > 0) ok = bar_wait(bar_ofree, (uint32_t)((j - 1) & 1), abort_flag, 0xA50u);
+        // P V_{j-1} complete: its V stage is free
+        if (ok && j > 0) ok = bar_wait(bar_o, (uint32_t)((j - 1) & 1), abort_flag, 0xA50u);
         if (!ok) break;
         if (j >= 1 && j + 1 < n_kt) load_v(j + 1);
         fence_after();
@@ -260,34 +263,19 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           const uint64_t db = desc_n_major(sV(st));
           const uint32_t ta = tmem + 192u + 32u * (uint32_t)st;      // P_j: 16 contraction steps = 8 columns
 #pragma unroll
-          for (int k = 0; k < KT / 16; ++k) mma_ts(tmem + 128u, ta + 8u * k, db + 128u * k, id_pv, k != 0 ? 1u : 0u);
+          for (int k = 0; k < KT / 16; ++k) mma_ts(tmem + 128u, ta + 8u * k, db + 128u * k, id_pv, (j | k) != 0 ? 1u : 0u);
         }
         commit(bar_o);
       }
       if (!ok) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) {} }   // copies in flight
     }
   } else {
-    // ---------------- softmax and accumulation: thread = query row = tensor-memory lane ----------------
+    // ---------------- softmax: thread = query row = tensor-memory lane ----------------
     const int row = 32 * warp + lane;
     const int qi = q0 + row;
     const uint32_t t_lane = tmem + ((uint32_t)(32 * warp) << 16), t_o = t_lane + 128u;
-    float o_acc[HD];
-#pragma unroll
-    for (int i = 0; i < HD; ++i) o_acc[i] = 0.f;
-    float m = -INFINITY, l = 0.f;
+    float m = -INFINITY, l = 0.f;                             // the reference the row's probabilities are relative to; their sum
     bool ok = true;
-    // o_acc <- o_acc * a + O_j: the accumulated output moves to the maximum that P_j was formed against (factor a,
-    // computed when tile j was processed) and takes tile j's product in the same multiply-add
-    auto fold = [&](float a) {
-      float t[32], t2[32];
-      ld32x2(t_o, t_o + 32u, t, t2);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        o_acc[i] = fmaf(o_acc[i], a, t[i]);
-        o_acc[32 + i] = fmaf(o_acc[32 + i], a, t2[i]);
-      }
-    };
-    float alpha_pending = 0.f;                                // factor of the tile whose P V product is still to be folded
     for (int j = 0; j < n_kt; ++j) {
       const int k0 = j * KT;
       const uint32_t t_s = t_lane + 64u * (uint32_t)(j & 1);
@@ -311,10 +299,32 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       float mx4[4] = {s[0], s[1], s[2], s[3]};                   // four independent chains instead of one of 64
 #pragma unroll
       for (int i = 4; i < KT; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], s[i]);
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      const float m_new = fmaxf(m, mx * p.scale_log2);
+      const float m_tile = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+      // The output accumulates in tensor memory over the whole sweep.  The row's reference moves only when a tile's
+      // maximum exceeds it by more than 2^FWD_SLACK: until then the probabilities (at most 2^FWD_SLACK) and their sum
+      // stay relative to the old one, which the final division and lse = m + log2(l) undo exactly, and the
+      // accumulated output needs no rescaling.
+      const float m_new = m_tile > m + FWD_SLACK ? m_tile : m;
       const float ref = m_new == -INFINITY ? 0.f : m_new;     // a row beyond the sequence may have seen no key
-      const float alpha = ex2(m - ref);
+      const float alpha = ex2(m - ref);                       // 1 while the reference stays
+      const bool moved = m_new != m && j > 0;
+      bool prev_done = j == 0;                                // P V_{j-1} known to be complete
+      if (__any_sync(0xffffffffu, moved)) {                   // O = O * 2^(m_old - m_new), between P V_{j-1} and P V_j
+        ok = bar_wait(bar_o, (uint32_t)((j - 1) & 1), abort_flag, 0xB20u);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        prev_done = true;
+        fence_after();
+        const float a = moved ? alpha : 1.0f;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          float t[32];
+          uint32_t u[32];
+          ld32(t_o + 32u * half, t);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) u[i] = __float_as_uint(t[i] * a);
+          st32(t_o + 32u * half, u);
+        }
+      }
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[KT / 2];
 #pragma unroll
@@ -328,18 +338,14 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       st32(t_lane + 192u + 32u * (uint32_t)(j & 1), pk);             // this row of P_j, an A operand in tensor memory
       fence_before();
       bar_arrive(bar_p);
-      // the previous tile's P V has had the whole of this tile's softmax to finish: fold it in
-      if (j > 0) {
-        ok = bar_wait(bar_o, (uint32_t)((j - 1) & 1), abort_flag, 0xB20u);
-        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-        fence_after();
-        fold(alpha_pending);
-        fence_before();
-        bar_arrive(bar_ofree);
-      }
-      alpha_pending = alpha;
       l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
       m = m_new;
+      // every completion of bar_o is observed in order (it has had this tile's softmax to happen): P buffer j & 1 is
+      // then free for tile j + 2, and the parity of a later wait cannot be mistaken
+      if (!prev_done) {
+        ok = bar_wait(bar_o, (uint32_t)((j - 1) & 1), abort_flag, 0xB21u);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      }
     }
     if (ok) {
       ok = bar_wait(bar_o, (uint32_t)((n_kt - 1) & 1), abort_flag, 0xB30u);
@@ -347,16 +353,20 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     }
     if (ok) {
       fence_after();
-      fold(alpha_pending);
-      if (qi < p.S) {
-        const float inv = l > 0.f ? 1.0f / l : 0.f;
-        uint4* dst = reinterpret_cast<uint4*>(p.out + (seq0 + qi) * p.ldo + h * HD);
+      const float inv = l > 0.f ? 1.0f / l : 0.f;
+      uint4* dst = reinterpret_cast<uint4*>(p.out + (seq0 + qi) * p.ldo + h * HD);
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-          dst[c] = make_uint4(pack2(o_acc[8 * c] * inv, o_acc[8 * c + 1] * inv), pack2(o_acc[8 * c + 2] * inv, o_acc[8 * c + 3] * inv),
-                              pack2(o_acc[8 * c + 4] * inv, o_acc[8 * c + 5] * inv), pack2(o_acc[8 * c + 6] * inv, o_acc[8 * c + 7] * inv));
-        p.lse[((long long)b * p.H + h) * p.S + qi] = m + log2f(l);
+      for (int half = 0; half < 2; ++half) {
+        float t[32];
+        ld32(t_o + 32u * half, t);
+        if (qi < p.S) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            dst[4 * half + c] = make_uint4(pack2(t[8 * c] * inv, t[8 * c + 1] * inv), pack2(t[8 * c + 2] * inv, t[8 * c + 3] * inv),
+                                           pack2(t[8 * c + 4] * inv, t[8 * c + 5] * inv), pack2(t[8 * c + 6] * inv, t[8 * c + 7] * inv));
+        }
       }
+      if (qi < p.S) p.lse[((long long)b * p.H + h) * p.S + qi] = m + log2f(l);
     }
   }
   __syncwarp();
