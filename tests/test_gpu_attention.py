@@ -45,10 +45,17 @@ def test_attention_forward_and_backward_match_the_oracle(ctx, B, S, H, HKV, D, f
         faar.tune_attention(ctx, 0)
 
 
-def _attention_case(ctx, B, S, H, HKV, D):
+@pytest.mark.parametrize("q_scale", [3.0, 8.0])
+def test_attention_with_peaked_scores(ctx, q_scale):
+    """Scores whose row maxima keep growing along the key sweep by amounts on both sides of the forward kernel's
+    slack (it moves a row's reference only past 2^8): the result must not depend on when the reference moves."""
+    _attention_case(ctx, 2, 321, 4, 2, 64, q_scale=q_scale)
+
+
+def _attention_case(ctx, B, S, H, HKV, D, q_scale=1.0):
     rng = np.random.default_rng(S + D)
     T = B * S
-    q = inputs.to_bf16_f32(rng.standard_normal((T, H * D)))
+    q = inputs.to_bf16_f32(rng.standard_normal((T, H * D)) * q_scale)
     k = inputs.to_bf16_f32(rng.standard_normal((T, HKV * D)))
     v = inputs.to_bf16_f32(rng.standard_normal((T, HKV * D)))
     do = inputs.to_bf16_f32(rng.standard_normal((T, H * D)))
