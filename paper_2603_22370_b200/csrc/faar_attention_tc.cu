@@ -164,6 +164,12 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// max of three in one instruction
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -296,9 +302,13 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         for (int i = 0; i < KT; ++i)
           if (!(k0 + i <= qi && k0 + i < p.S)) s[i] = -INFINITY;
       }
-      float mx4[4] = {s[0], s[1], s[2], s[3]};                   // four independent chains instead of one of 64
+      float mx4[4] = {s[0], s[1], s[2], s[3]};                   // four independent chains, two scores per instruction
 #pragma unroll
-      for (int i = 4; i < KT; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], s[i]);
+      for (int i = 4; i < KT; i += 8) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (i + 2 * c + 1 < KT) mx4[c] = max3(mx4[c], s[i + 2 * c], s[i + 2 * c + 1]);
+      }
       const float m_tile = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
       // The output accumulates in tensor memory over the whole sweep.  The row's reference moves only when a tile's
       // maximum exceeds it by more than 2^FWD_SLACK: until then the probabilities (at most 2^FWD_SLACK) and their sum
@@ -325,20 +335,21 @@ attn_fwd64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           st32(t_o + 32u * half, u);
         }
       }
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      // exponent arguments and sums two at a time (packed FP32 multiply-add and add: the same roundings)
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nr2 = make_float2(-ref, -ref);
+      float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       uint32_t pk[KT / 2];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        float e[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { e[i] = ex2(fmaf(s[8 * c + i], p.scale_log2, -ref)); sum4[i & 3] += e[i]; }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) pk[4 * c + i] = pack2(e[2 * i], e[2 * i + 1]);
+      for (int w = 0; w < KT / 2; ++w) {
+        const float2 x = __ffma2_rn(make_float2(s[2 * w], s[2 * w + 1]), sc2, nr2);
+        const float2 e = make_float2(ex2(x.x), ex2(x.y));
+        sum2[w & 1] = __fadd2_rn(sum2[w & 1], e);
+        pk[w] = pack2(e.x, e.y);
       }
       st32(t_lane + 192u + 32u * (uint32_t)(j & 1), pk);             // this row of P_j, an A operand in tensor memory
       fence_before();
       bar_arrive(bar_p);
-      l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+      l = l * alpha + ((sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y));
       m = m_new;
       // every completion of bar_o is observed in order (it has had this tile's softmax to happen): P buffer j & 1 is
       // then free for tile j + 2, and the parity of a later wait cannot be mistaken
@@ -516,11 +527,18 @@ attn_dq64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         constexpr bool DIAG = decltype(diag_tag)::value;
         float t[32], d[32];
         ld32x2(t_lane + 32u * half, t_lane + 64u + 32u * half, t, d);
+        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nl2 = make_float2(-lse, -lse);
+        const float2 is2 = make_float2(p.inv_sqrt_d, p.inv_sqrt_d), nd2 = make_float2(nd, nd);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float pr = ex2(fmaf(t[i], p.scale_log2, -lse));
-          if (DIAG && k0 + 32 * half + i > qi) pr = 0.f;       // above the diagonal (and beyond the sequence end)
-          s[i] = pr * fmaf(d[i], p.inv_sqrt_d, nd);
+        for (int i = 0; i < 32; i += 2) {                        // two elements per multiply-add
+          const float2 x = __ffma2_rn(make_float2(t[i], t[i + 1]), sc2, nl2);
+          float2 pr = make_float2(ex2(x.x), ex2(x.y));
+          if (DIAG) {                                            // above the diagonal (and beyond the sequence end)
+            if (k0 + 32 * half + i > qi) pr.x = 0.f;
+            if (k0 + 32 * half + i + 1 > qi) pr.y = 0.f;
+          }
+          const float2 r = __fmul2_rn(pr, __ffma2_rn(make_float2(d[i], d[i + 1]), is2, nd2));
+          s[i] = r.x; s[i + 1] = r.y;
         }
       };
       if (k0 + KT - 1 > q0) tile(std::true_type{}); else tile(std::false_type{});   // some key of the tile above some row
@@ -741,12 +759,19 @@ attn_dkv64_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           const float4 n4 = *reinterpret_cast<const float4*>(rowv + KT + 32 * half + j4);
           const float lq[4] = {l4.x, l4.y, l4.z, l4.w}, nq[4] = {n4.x, n4.y, n4.z, n4.w};
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
+          for (int e = 0; e < 4; e += 2) {                       // two elements per multiply-add
             const int j = j4 + e, c = 32 * half + j;
-            float pr = ex2(fmaf(t[j], p.scale_log2, -lq[e]));
-            if (EDGE && !(kj <= q0 + c && q0 + c < p.S)) pr = 0.f;
-            t[j] = pr;
-            d[j] = pr * fmaf(d[j], p.inv_sqrt_d, nq[e]);
+            const float2 x = __ffma2_rn(make_float2(t[j], t[j + 1]), make_float2(p.scale_log2, p.scale_log2),
+                                        make_float2(-lq[e], -lq[e + 1]));
+            float2 pr = make_float2(ex2(x.x), ex2(x.y));
+            if (EDGE) {
+              if (!(kj <= q0 + c && q0 + c < p.S)) pr.x = 0.f;
+              if (!(kj <= q0 + c + 1 && q0 + c + 1 < p.S)) pr.y = 0.f;
+            }
+            const float2 r = __fmul2_rn(pr, __ffma2_rn(make_float2(d[j], d[j + 1]), make_float2(p.inv_sqrt_d, p.inv_sqrt_d),
+                                                       make_float2(nq[e], nq[e + 1])));
+            t[j] = pr.x; t[j + 1] = pr.y;
+            d[j] = r.x; d[j + 1] = r.y;
           }
         }
         // this thread's half of the rows of P^T and dS^T: A operands in tensor memory
